@@ -1,0 +1,153 @@
+"""fp64 CPU oracle for linear attention -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes/numpy front end of ``la_oracle.c``.  It exists so that the tests,
+the smoke check and the benchmark's CPU-baseline leg can ask "what should the
+answer be?".  The CUDA library never imports or links it, and this package
+never imports the CUDA binding.
+
+All functions take array-likes shaped ``[B, H, N, D]`` / ``[B, H, N, M]`` (or
+``[B, H, D]`` / ``[B, H, M]`` for the recurrent step), convert them to
+contiguous float64 and return float64 numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "la_oracle.c")
+_LIB = os.path.join(_HERE, "libla_oracle.so")
+
+PHI = {"elu1": 0, "identity": 1}
+
+
+def build(force: bool = False) -> str:
+    """Compile ``la_oracle.c`` into ``libla_oracle.so`` next to it (gcc -O2 -fopenmp)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+_dp = ctypes.POINTER(ctypes.c_double)
+_i64 = ctypes.c_int64
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.la_oracle_num_threads.restype = ctypes.c_int
+        _lib.la_oracle_set_threads.argtypes = [ctypes.c_int]
+        _lib.la_oracle_feature_map.argtypes = [_dp, _dp, _i64, ctypes.c_int]
+        _lib.la_oracle_attention_quadratic.argtypes = (
+            [_i64] * 5 + [ctypes.c_int, ctypes.c_int, ctypes.c_double] + [_dp] * 5)
+        _lib.la_oracle_attention_quadratic_backward.argtypes = (
+            [_i64] * 5 + [ctypes.c_int, ctypes.c_int, ctypes.c_double] + [_dp] * 7)
+        _lib.la_oracle_linear.argtypes = (
+            [_i64] * 5 + [ctypes.c_int, ctypes.c_int, ctypes.c_double] + [_dp] * 7)
+        _lib.la_oracle_linear_backward.argtypes = (
+            [_i64] * 5 + [ctypes.c_int, ctypes.c_int, ctypes.c_double] + [_dp] * 7)
+        _lib.la_oracle_recurrent_step.argtypes = (
+            [_i64] * 4 + [ctypes.c_int, ctypes.c_double] + [_dp] * 6)
+    return _lib
+
+
+def _f64(a):
+    if hasattr(a, "detach"):  # torch tensor (bf16 has no numpy dtype: widen first)
+        a = a.detach().cpu().double().numpy()
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(_dp)
+
+
+def _shapes(Q, K, V):
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    if Q.ndim != 4 or K.shape != Q.shape or V.ndim != 4 or V.shape[:3] != Q.shape[:3]:
+        raise ValueError("expected Q,K [B,H,N,D] and V [B,H,N,M]")
+    B, H, N, D = Q.shape
+    return Q, K, V, B, H, N, D, V.shape[3]
+
+
+def num_threads() -> int:
+    return _load().la_oracle_num_threads()
+
+
+def set_threads(n: int) -> None:
+    _load().la_oracle_set_threads(int(n))
+
+
+def feature_map(x, deriv: bool = False):
+    """Eq. 7: elu(x)+1 elementwise (or its slope when ``deriv``)."""
+    x = _f64(x)
+    y = np.empty_like(x)
+    _load().la_oracle_feature_map(_p(x), _p(y), x.size, int(deriv))
+    return y
+
+
+def attention_quadratic(Q, K, V, causal: bool, phi: str = "elu1", eps: float = 0.0,
+                        return_weights: bool = False):
+    """Eq. 3 / Eq. 8 with sim(q,k)=phi(q).phi(k) on the explicit N x N matrix."""
+    Q, K, V, B, H, N, D, M = _shapes(Q, K, V)
+    O = np.empty((B, H, N, M))
+    W = np.empty((B, H, N, N)) if return_weights else None
+    _load().la_oracle_attention_quadratic(B, H, N, D, M, int(causal), PHI[phi], eps,
+                                          _p(Q), _p(K), _p(V), _p(O), _p(W))
+    return (O, W) if return_weights else O
+
+
+def attention_quadratic_backward(Q, K, V, G, causal: bool, phi: str = "elu1", eps: float = 0.0):
+    """Explicit chain rule through the N x N matrix; returns (dQ, dK, dV)."""
+    Q, K, V, B, H, N, D, M = _shapes(Q, K, V)
+    G = _f64(G)
+    dQ, dK, dV = np.empty_like(Q), np.empty_like(K), np.empty_like(V)
+    _load().la_oracle_attention_quadratic_backward(
+        B, H, N, D, M, int(causal), PHI[phi], eps,
+        _p(Q), _p(K), _p(V), _p(G), _p(dQ), _p(dK), _p(dV))
+    return dQ, dK, dV
+
+
+def linear_attention(Q, K, V, causal: bool, phi: str = "elu1", eps: float = 0.0,
+                     return_state: bool = False):
+    """Eq. 5-6 (non-causal) or Eq. 9-12 / Algorithm 1 (causal); returns (O, den[, S, Z])."""
+    Q, K, V, B, H, N, D, M = _shapes(Q, K, V)
+    O = np.empty((B, H, N, M))
+    den = np.empty((B, H, N))
+    S = np.empty((B, H, D, M)) if return_state else None
+    Z = np.empty((B, H, D)) if return_state else None
+    _load().la_oracle_linear(B, H, N, D, M, int(causal), PHI[phi], eps,
+                             _p(Q), _p(K), _p(V), _p(O), _p(den), _p(S), _p(Z))
+    return (O, den, S, Z) if return_state else (O, den)
+
+
+def linear_attention_backward(Q, K, V, G, causal: bool, phi: str = "elu1", eps: float = 0.0):
+    """Eq. 13-15 on the ones-extended values, forward and reverse running sums."""
+    Q, K, V, B, H, N, D, M = _shapes(Q, K, V)
+    G = _f64(G)
+    dQ, dK, dV = np.empty_like(Q), np.empty_like(K), np.empty_like(V)
+    _load().la_oracle_linear_backward(
+        B, H, N, D, M, int(causal), PHI[phi], eps,
+        _p(Q), _p(K), _p(V), _p(G), _p(dQ), _p(dK), _p(dV))
+    return dQ, dK, dV
+
+
+def recurrent_step(q, k, v, S, Z, phi: str = "elu1", eps: float = 0.0):
+    """Eq. 18-20: update S, Z (float64 arrays, IN PLACE), then read out; returns out [B,H,M]."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    if not (isinstance(S, np.ndarray) and S.dtype == np.float64 and S.flags.c_contiguous
+            and isinstance(Z, np.ndarray) and Z.dtype == np.float64 and Z.flags.c_contiguous):
+        raise ValueError("S and Z must be contiguous float64 numpy arrays (updated in place)")
+    B, H, D = q.shape
+    M = v.shape[2]
+    if S.shape != (B, H, D, M) or Z.shape != (B, H, D):
+        raise ValueError("state shape mismatch")
+    out = np.empty((B, H, M))
+    _load().la_oracle_recurrent_step(B, H, D, M, PHI[phi], eps,
+                                     _p(q), _p(k), _p(v), _p(S), _p(Z), _p(out))
+    return out

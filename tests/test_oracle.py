@@ -1,0 +1,294 @@
+"""Pins for the fp64 oracle (no GPU).
+
+Every oracle routine is checked against something that is not the oracle:
+closed forms, a hand-worked rational example, exact-rational brute force of the
+definition, numpy/torch library one-liners, torch autograd through the
+quadratic form, central finite differences and structural invariants.
+"""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def rnd(shape, seed):
+    return np.random.default_rng(seed).standard_normal(shape)
+
+
+# ---------------------------------------------------------------- feature map
+def test_phi_closed_forms():
+    rows = []
+    with open(os.path.join(ROOT, "tests", "golden", "phi_values.txt")) as f:
+        for line in f:
+            line = line.split("#", 1)[0].split()
+            if line:
+                rows.append([float(t) for t in line])
+    rows = np.array(rows)
+    assert np.allclose(oracle.feature_map(rows[:, 0]), rows[:, 1], rtol=1e-15, atol=0)
+    assert np.allclose(oracle.feature_map(rows[:, 0], deriv=True), rows[:, 2], rtol=1e-15, atol=0)
+
+
+def test_phi_properties():
+    x = np.linspace(-30, 30, 2001)
+    y = oracle.feature_map(x)
+    assert (y > 0).all()                                   # positive similarity
+    assert (np.diff(y) > 0).all()                          # monotone
+    neg = x <= 0
+    assert np.array_equal(oracle.feature_map(x, True)[neg], y[neg])   # phi' = phi for x <= 0
+    assert (oracle.feature_map(x, True)[~neg] == 1).all()
+    # matches the library elu
+    t = torch.nn.functional.elu(torch.from_numpy(x)) + 1
+    # (elu(x) + 1 cancels for very negative x, hence the absolute tolerance)
+    assert np.allclose(y, t.numpy(), rtol=1e-15, atol=3e-16)
+
+
+# ------------------------------------------------------------ worked example
+def _ex(worked_example, *names):
+    return [worked_example[n][None, None] for n in names]
+
+
+@pytest.mark.parametrize("routine", ["quadratic", "linear"])
+def test_worked_example_forward(worked_example, routine):
+    Q, K, V = _ex(worked_example, "Q", "K", "V")
+    assert np.array_equal(oracle.feature_map(Q)[0, 0], worked_example["phiQ"])
+    assert np.array_equal(oracle.feature_map(K)[0, 0], worked_example["phiK"])
+    for causal, tag in ((True, "causal"), (False, "noncausal")):
+        if routine == "quadratic":
+            O = oracle.attention_quadratic(Q, K, V, causal)
+        else:
+            O, den = oracle.linear_attention(Q, K, V, causal)
+            assert np.allclose(den[0, 0], worked_example[tag + "_den"][0], rtol=1e-15)
+        assert np.allclose(O[0, 0], worked_example[tag + "_O"], rtol=1e-14, atol=1e-16)
+
+
+def test_worked_example_states(worked_example):
+    Q, K, V = _ex(worked_example, "Q", "K", "V")
+    S = np.zeros((1, 1, 2, 2))
+    Z = np.zeros((1, 1, 2))
+    for i in range(3):
+        out = oracle.recurrent_step(Q[:, :, i], K[:, :, i], V[:, :, i], S, Z)
+        assert np.array_equal(S[0, 0], worked_example[f"S{i + 1}"])
+        assert np.array_equal(Z[0, 0], worked_example[f"Z{i + 1}"][0])
+        assert np.allclose(out[0, 0], worked_example["causal_O"][i], rtol=1e-14, atol=1e-16)
+    _, _, S3, Z3 = oracle.linear_attention(Q, K, V, True, return_state=True)
+    assert np.array_equal(S3[0, 0], worked_example["S3"])
+    assert np.array_equal(Z3[0, 0], worked_example["Z3"][0])
+
+
+@pytest.mark.parametrize("routine", ["quadratic", "linear"])
+def test_worked_example_backward(worked_example, routine):
+    Q, K, V, G = _ex(worked_example, "Q", "K", "V", "G")
+    fn = (oracle.attention_quadratic_backward if routine == "quadratic"
+          else oracle.linear_attention_backward)
+    for causal, tag in ((True, "causal"), (False, "noncausal")):
+        dQ, dK, dV = fn(Q, K, V, G, causal)
+        assert np.allclose(dQ[0, 0], worked_example[tag + "_dQ"], rtol=1e-13, atol=1e-16)
+        assert np.allclose(dK[0, 0], worked_example[tag + "_dK"], rtol=1e-13, atol=1e-16)
+        assert np.allclose(dV[0, 0], worked_example[tag + "_dV"], rtol=1e-13, atol=1e-16)
+
+
+# -------------------------------------------- exact brute force of definition
+def _exact_attention(phiQ, phiK, V, causal):
+    """Eq. 3 / Eq. 8 in exact rationals on already-mapped integer features."""
+    N = len(phiQ)
+    out = []
+    for i in range(N):
+        js = range(i + 1) if causal else range(N)
+        w = [sum(Fraction(a) * Fraction(b) for a, b in zip(phiQ[i], phiK[j])) for j in js]
+        den = sum(w)
+        out.append([sum(wj * Fraction(V[j][e]) for wj, j in zip(w, js)) / den
+                    for e in range(len(V[0]))])
+    return out
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_exact_rational_bruteforce(causal, seed):
+    rng = np.random.default_rng(seed)
+    N, D, M = 7, 3, 4
+    Qi = rng.integers(0, 6, (N, D))          # non-negative: phi(x) = x + 1 exactly
+    Ki = rng.integers(0, 6, (N, D))
+    Vi = rng.integers(-9, 10, (N, M))
+    exact = _exact_attention((Qi + 1).tolist(), (Ki + 1).tolist(), Vi.tolist(), causal)
+    exact = np.array([[float(x) for x in r] for r in exact])
+    args = [a[None, None].astype(float) for a in (Qi, Ki, Vi)]
+    assert np.allclose(oracle.attention_quadratic(*args, causal)[0, 0], exact, rtol=1e-14, atol=1e-15)
+    assert np.allclose(oracle.linear_attention(*args, causal)[0][0, 0], exact, rtol=1e-13, atol=1e-14)
+    # identity feature map on the mapped features gives the same thing
+    argsI = [(Qi + 1)[None, None].astype(float), (Ki + 1)[None, None].astype(float), args[2]]
+    assert np.allclose(oracle.attention_quadratic(*argsI, causal, phi="identity")[0, 0], exact,
+                       rtol=1e-14, atol=1e-15)
+
+
+# ----------------------------------------------------- library one-liner form
+def _numpy_form(Q, K, V, causal, eps=0.0):
+    fq = np.where(Q > 0, Q + 1, np.exp(np.minimum(Q, 0)))
+    fk = np.where(K > 0, K + 1, np.exp(np.minimum(K, 0)))
+    A = fq @ np.swapaxes(fk, -1, -2)
+    if causal:
+        A = np.tril(A)
+    return (A @ V) / (A.sum(-1, keepdims=True) + eps), A
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("shape", [(2, 3, 17, 5, 7), (1, 2, 64, 8, 4), (1, 1, 1, 4, 4)])
+def test_quadratic_and_linear_match_matrix_form(causal, shape):
+    B, H, N, D, M = shape
+    Q, K, V = rnd((B, H, N, D), 1), rnd((B, H, N, D), 2), rnd((B, H, N, M), 3)
+    ref, A = _numpy_form(Q, K, V, causal)
+    Oq, W = oracle.attention_quadratic(Q, K, V, causal, return_weights=True)
+    Ol, den = oracle.linear_attention(Q, K, V, causal)
+    assert np.allclose(Oq, ref, rtol=1e-12, atol=1e-13)
+    assert np.allclose(Ol, ref, rtol=1e-11, atol=1e-12)
+    assert np.allclose(den, A.sum(-1), rtol=1e-12)
+    assert np.allclose(W, A / A.sum(-1, keepdims=True), rtol=1e-12, atol=0)
+    # eps enters the denominator additively
+    refe, _ = _numpy_form(Q, K, V, causal, eps=0.5)
+    assert np.allclose(oracle.attention_quadratic(Q, K, V, causal, eps=0.5), refe, rtol=1e-12, atol=1e-13)
+    assert np.allclose(oracle.linear_attention(Q, K, V, causal, eps=0.5)[0], refe, rtol=1e-11, atol=1e-12)
+
+
+# ------------------------------------------------------------------ invariants
+@pytest.mark.parametrize("causal", [True, False])
+def test_weights_positive_rows_sum_to_one_constant_v(causal):
+    B, H, N, D, M = 1, 2, 33, 6, 5
+    Q, K = rnd((B, H, N, D), 4) * 3, rnd((B, H, N, D), 5) * 3
+    V = np.broadcast_to(rnd((1, 1, 1, M), 6), (B, H, N, M)).copy()
+    O, W = oracle.attention_quadratic(Q, K, V, causal, return_weights=True)
+    allowed = np.tril(np.ones((N, N), bool)) if causal else np.ones((N, N), bool)
+    assert (W[..., allowed] > 0).all() and (W[..., ~allowed] == 0).all()
+    assert np.allclose(W.sum(-1), 1.0, rtol=1e-14)
+    assert np.allclose(O, V, rtol=1e-13)                       # constant V is reproduced
+    assert np.allclose(oracle.linear_attention(Q, K, V, causal)[0], V, rtol=1e-12)
+
+
+def test_first_causal_output_is_first_value_and_uniform_keys_give_means():
+    B, H, N, D, M = 2, 2, 19, 4, 3
+    Q, K, V = rnd((B, H, N, D), 7), rnd((B, H, N, D), 8), rnd((B, H, N, M), 9)
+    for fn in (lambda *a: oracle.attention_quadratic(*a), lambda *a: oracle.linear_attention(*a)[0]):
+        assert np.allclose(fn(Q, K, V, True)[:, :, 0], V[:, :, 0], rtol=1e-13)
+        Ku = np.broadcast_to(K[:, :, :1], K.shape).copy()     # all keys equal: uniform weights
+        run_mean = np.cumsum(V, 2) / np.arange(1, N + 1)[None, None, :, None]
+        assert np.allclose(fn(Q, Ku, V, True), run_mean, rtol=1e-12, atol=1e-13)
+        full_mean = np.broadcast_to(V.mean(2, keepdims=True), V.shape)
+        assert np.allclose(fn(Q, Ku, V, False), full_mean, rtol=1e-12, atol=1e-13)
+
+
+def test_outputs_lie_in_value_range():
+    Q, K, V = rnd((1, 1, 40, 8), 10), rnd((1, 1, 40, 8), 11), rnd((1, 1, 40, 3), 12)
+    O = oracle.linear_attention(Q, K, V, True)[0]
+    lo = np.minimum.accumulate(V, 2)
+    hi = np.maximum.accumulate(V, 2)
+    assert (O >= lo - 1e-12).all() and (O <= hi + 1e-12).all()
+
+
+# ------------------------------------------------- recurrent == parallel form
+@pytest.mark.parametrize("shape", [(2, 2, 23, 5, 3), (1, 3, 40, 8, 8)])
+def test_recurrent_unrolled_equals_causal(shape):
+    B, H, N, D, M = shape
+    Q, K, V = rnd((B, H, N, D), 13), rnd((B, H, N, D), 14), rnd((B, H, N, M), 15)
+    ref = oracle.attention_quadratic(Q, K, V, True)
+    _, _, SN, ZN = oracle.linear_attention(Q, K, V, True, return_state=True)
+    S, Z = np.zeros((B, H, D, M)), np.zeros((B, H, D))
+    for i in range(N):
+        out = oracle.recurrent_step(Q[:, :, i], K[:, :, i], V[:, :, i], S, Z)
+        assert np.allclose(out, ref[:, :, i], rtol=1e-11, atol=1e-12)
+    assert np.allclose(S, SN, rtol=1e-13, atol=1e-13) and np.allclose(Z, ZN, rtol=1e-13)
+    fk = oracle.feature_map(K)
+    assert np.allclose(S, np.einsum("bhnd,bhnm->bhdm", fk, V), rtol=1e-12, atol=1e-12)   # Eq. 10
+    assert np.allclose(Z, fk.sum(2), rtol=1e-13)                                          # Eq. 11
+
+
+# ------------------------------------------------------------------- gradients
+def _torch_quadratic(Q, K, V, causal, eps=0.0, identity=False):
+    phi = (lambda x: x) if identity else (lambda x: torch.nn.functional.elu(x) + 1)
+    A = phi(Q) @ phi(K).transpose(-1, -2)
+    if causal:
+        A = torch.tril(A)
+    return (A @ V) / (A.sum(-1, keepdim=True) + eps)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("shape", [(2, 2, 21, 5, 7), (1, 1, 48, 8, 4)])
+@pytest.mark.parametrize("eps", [0.0, 0.25])
+def test_backward_matches_autograd_through_quadratic_form(causal, shape, eps):
+    B, H, N, D, M = shape
+    Qn, Kn, Vn, Gn = rnd((B, H, N, D), 16), rnd((B, H, N, D), 17), rnd((B, H, N, M), 18), rnd((B, H, N, M), 19)
+    Q, K, V = (torch.tensor(a, requires_grad=True) for a in (Qn, Kn, Vn))
+    (_torch_quadratic(Q, K, V, causal, eps) * torch.tensor(Gn)).sum().backward()
+    for fn in (oracle.attention_quadratic_backward, oracle.linear_attention_backward):
+        dQ, dK, dV = fn(Qn, Kn, Vn, Gn, causal, eps=eps)
+        assert np.allclose(dQ, Q.grad.numpy(), rtol=1e-9, atol=1e-11)
+        assert np.allclose(dK, K.grad.numpy(), rtol=1e-9, atol=1e-11)
+        assert np.allclose(dV, V.grad.numpy(), rtol=1e-9, atol=1e-11)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_backward_identity_feature_map(causal):
+    B, H, N, D, M = 1, 2, 15, 4, 5
+    Qn, Kn = np.abs(rnd((B, H, N, D), 20)) + 0.1, np.abs(rnd((B, H, N, D), 21)) + 0.1
+    Vn, Gn = rnd((B, H, N, M), 22), rnd((B, H, N, M), 23)
+    Q, K, V = (torch.tensor(a, requires_grad=True) for a in (Qn, Kn, Vn))
+    (_torch_quadratic(Q, K, V, causal, identity=True) * torch.tensor(Gn)).sum().backward()
+    for fn in (oracle.attention_quadratic_backward, oracle.linear_attention_backward):
+        dQ, dK, dV = fn(Qn, Kn, Vn, Gn, causal, phi="identity")
+        assert np.allclose(dQ, Q.grad.numpy(), rtol=1e-9, atol=1e-11)
+        assert np.allclose(dK, K.grad.numpy(), rtol=1e-9, atol=1e-11)
+        assert np.allclose(dV, V.grad.numpy(), rtol=1e-9, atol=1e-11)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_backward_matches_finite_differences(causal):
+    B, H, N, D, M = 1, 1, 9, 3, 4
+    Q, K, V, G = rnd((B, H, N, D), 24), rnd((B, H, N, D), 25), rnd((B, H, N, M), 26), rnd((B, H, N, M), 27)
+    for a in (Q, K):                      # phi is only C^1 at 0: keep away from the kink
+        a[np.abs(a) < 1e-3] = 0.5
+    assert (Q < 0).any() and (K < 0).any() and (Q > 0).any() and (K > 0).any()
+    loss = lambda q, k, v: float((oracle.attention_quadratic(q, k, v, causal) * G).sum())
+    grads = oracle.linear_attention_backward(Q, K, V, G, causal)
+    h = 1e-6
+    for which, (arr, grad) in enumerate(zip((Q, K, V), grads)):
+        fd = np.zeros_like(arr)
+        it = np.nditer(arr, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            args_p, args_m = [Q.copy(), K.copy(), V.copy()], [Q.copy(), K.copy(), V.copy()]
+            args_p[which][idx] += h
+            args_m[which][idx] -= h
+            fd[idx] = (loss(*args_p) - loss(*args_m)) / (2 * h)
+        assert np.allclose(grad, fd, rtol=1e-6, atol=1e-8), which
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_gradient_invariants(causal):
+    B, H, N, D, M = 2, 2, 37, 6, 5
+    Q, K, V, G = rnd((B, H, N, D), 28), rnd((B, H, N, D), 29), rnd((B, H, N, M), 30), rnd((B, H, N, M), 31)
+    dQ, dK, dV = oracle.linear_attention_backward(Q, K, V, G, causal)
+    # rows of the attention matrix sum to one  =>  sum_j dV_j = sum_i G_i
+    assert np.allclose(dV.sum(2), G.sum(2), rtol=1e-11, atol=1e-12)
+    # O is homogeneous of degree 0 in phi(Q_i)  =>  <phi(Q_i), grad phi(Q_i)> = 0
+    ratio = lambda x: np.where(x > 0, x + 1.0, 1.0)           # phi / phi'
+    assert np.abs((ratio(Q) * dQ).sum(-1)).max() < 1e-12
+    # a global scale of phi(K) cancels  =>  sum_{j,d} phi(K_jd) grad phi(K_jd) = 0
+    assert np.abs((ratio(K) * dK).sum((-1, -2))).max() < 1e-11
+
+
+def test_linear_matches_quadratic_on_larger_case():
+    B, H, N, D, M = 1, 2, 300, 16, 12
+    Q, K, V, G = rnd((B, H, N, D), 32), rnd((B, H, N, D), 33), rnd((B, H, N, M), 34), rnd((B, H, N, M), 35)
+    for causal in (True, False):
+        assert np.allclose(oracle.linear_attention(Q, K, V, causal)[0],
+                           oracle.attention_quadratic(Q, K, V, causal), rtol=1e-10, atol=1e-12)
+        for a, b in zip(oracle.linear_attention_backward(Q, K, V, G, causal),
+                        oracle.attention_quadratic_backward(Q, K, V, G, causal)):
+            assert np.allclose(a, b, rtol=1e-9, atol=1e-11)
+
+
+def test_threads_reported():
+    assert oracle.num_threads() >= 1
