@@ -1,0 +1,427 @@
+#!/usr/bin/env python
+"""Benchmark of the linear-attention hot path on B200.
+
+One step = la_causal_forward + la_causal_backward over one batch of synthetic
+input (the feature map, the normalising division and the state recurrence are
+fused inside those calls).  The default workload is the N=16384 point of the
+sequence-length sweep (B=8, H=8, D=M=64, bf16); `--workload` selects any other
+named workload, and, at one GPU, the remaining rows of the hot path (non-causal
+forward+backward, the image-shaped causal case, the other sweep points and the
+3072-step recurrent decode) are timed as well and reported under "rows".
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle on a
+bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2006_16236_b200.inputs import WORKLOADS, draw_qkvg, draw_workload  # noqa: E402
+
+METRIC = "causal LA fwd+bwd tokens/s"
+DEFAULT_WORKLOAD = "causal_sweep_bf16_N16384"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from an
+# ncu capture summarised under profiles/), keyed by workload; None until captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["source"] = "measured"
+        return d
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+def elem_bytes(w):
+    return 4 if w.dtype == "f32" else 2
+
+
+def algorithmic_bytes(w, part):
+    """Compulsory HBM bytes: every input read once, every output written once."""
+    th = w.B * w.H * w.N
+    e = elem_bytes(w)
+    if w.kind == "decode":
+        return w.B * w.H * (8 * w.D * w.M + 8 * w.D + (2 * w.D + 2 * w.M) * e)
+    fwd = th * ((2 * w.D + 2 * w.M) * e + 4)                      # Q,K,V in; O, den out
+    bwd = th * ((2 * w.D + 2 * w.M) * e + (2 * w.D + w.M) * e + 4)  # Q,K,V,G (+den) in; dQ,dK,dV out
+    return {"fwd": fwd, "bwd": bwd, "both": fwd + bwd}[part]
+
+
+def algorithmic_flops(w, part):
+    th = w.B * w.H * w.N
+    if w.kind == "decode":
+        return w.B * w.H * 4 * w.D * w.M
+    if w.kind == "noncausal":
+        return {"fwd": 4, "bwd": 8, "both": 12}[part] * w.D * w.M * th
+    return {"fwd": 4, "bwd": 10, "both": 14}[part] * w.D * w.M * th
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, c[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_setup(n_gpus):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return world, rank, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(x, world, dev):
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# --------------------------------------------------------------------------- GPU arms
+class CausalStep:
+    def __init__(self, la, w, dev, seed_offset=0):
+        self.la, self.w, self.dev = la, w, dev
+        Q, K, V, G = draw_qkvg(w.B, w.H, w.N, w.D, w.M, w.seed + seed_offset, w.torch_dtype, w.scale)
+        self.host = [t.pin_memory() for t in (Q, K, V, G)]
+        self.d = [t.to(dev) for t in self.host]
+        self.O = torch.empty_like(self.d[2])
+        self.den = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device=dev)
+        self.grads = [torch.empty_like(self.d[0]), torch.empty_like(self.d[1]), torch.empty_like(self.d[2])]
+        self.host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in [self.O] + self.grads]
+        self.causal = w.kind == "causal"
+
+    def fwd(self):
+        Q, K, V, _ = self.d
+        if self.causal:
+            self.la.la_causal_forward(Q, K, V, O=self.O, den=self.den)
+        else:
+            self.la.la_linear_attention(Q, K, V, O=self.O, den=self.den)
+
+    def bwd(self):
+        Q, K, V, G = self.d
+        dQ, dK, dV = self.grads
+        if self.causal:
+            self.la.la_causal_backward(Q, K, V, G, O=self.O, den=self.den, dQ=dQ, dK=dK, dV=dV)
+        else:
+            self.la.la_linear_attention_backward(Q, K, V, G, O=self.O, den=self.den, dQ=dQ, dK=dK, dV=dV)
+
+    def step(self):
+        self.fwd()
+        self.bwd()
+
+    def e2e_step(self):
+        for h, d in zip(self.host, self.d):
+            d.copy_(h, non_blocking=True)
+        self.step()
+        for h, d in zip(self.host_out, [self.O] + self.grads):
+            h.copy_(d, non_blocking=True)
+
+    def e2e_bytes(self):
+        h2d = sum(t.numel() * t.element_size() for t in self.host)
+        d2h = sum(t.numel() * t.element_size() for t in self.host_out)
+        return h2d, d2h
+
+
+def time_steps(run, steps, warmup, world, split=None):
+    """Time `steps` calls of run() with CUDA events on the current stream; returns total ms and,
+    when split=(fwd, bwd) is given instead of run, the mean ms of each part."""
+    for _ in range(warmup):
+        run() if split is None else (split[0](), split[1]())
+    barrier(world)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(steps):
+        if split is None:
+            run()
+        else:
+            ev[i][0].record()
+            split[0]()
+            ev[i][1].record()
+            split[1]()
+            ev[i][2].record()
+    t1.record()
+    torch.cuda.synchronize()
+    total = t0.elapsed_time(t1)
+    barrier(world)
+    if split is None:
+        return total, None
+    f = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    b = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    return total, (f, b)
+
+
+def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True):
+    s = CausalStep(la, w, dev, seed_offset=rank)
+    launches0 = la.la_kernel_launches()
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    total_ms, (fwd_ms, bwd_ms) = time_steps(None, steps, warmup, world, split=(s.fwd, s.bwd))
+    clocks = sampler.stop() if sampler else None
+    launches = (la.la_kernel_launches() - launches0) * steps // (steps + warmup)
+    la.la_last_device_status()
+    total_ms = max_over_ranks(total_ms, world, dev)
+    ms = total_ms / steps
+    tokens = w.tokens * world
+    res = {
+        "value": tokens / (ms * 1e-3), "ms_per_step": ms, "fwd_ms": fwd_ms, "bwd_ms": bwd_ms,
+        "gpu_launches": int(launches), "clocks": clocks,
+        "alg_gbs": algorithmic_bytes(w, "both") / (fwd_ms + bwd_ms) * 1e-6,
+        "alg_tflops": algorithmic_flops(w, "both") / (fwd_ms + bwd_ms) * 1e-9,
+    }
+    res["hbm_frac"] = res["alg_gbs"] / pk["hbm_gbs"]
+    res["tensor_frac_alg_flops"] = res["alg_tflops"] / pk["bf16_tflops_sustained"]
+    dom = "bwd" if bwd_ms >= fwd_ms else "fwd"
+    dom_ms = max(bwd_ms, fwd_ms)
+    ach = algorithmic_bytes(w, dom) / dom_ms * 1e-6
+    res["roofline"] = {
+        "kernel": ("la_causal_" if w.kind == "causal" else "la_linear_attention_") + ("backward" if dom == "bwd" else "forward"),
+        "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
+        "peak_source": pk["source"] + " copy bandwidth",
+        "algorithmic_bytes_per_launch": algorithmic_bytes(w, dom), "ms_per_launch": dom_ms,
+        "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
+    }
+    if do_e2e:
+        e_steps = max(3, min(steps, 10))
+        e_ms, _ = time_steps(s.e2e_step, e_steps, 3, world)
+        e_ms = max_over_ranks(e_ms, world, dev) / e_steps
+        h2d, d2h = s.e2e_bytes()
+        res["e2e"] = {"value": tokens / (e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e_ms,
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e_steps}
+    del s
+    torch.cuda.empty_cache()
+    return res
+
+
+def bench_decode(la, w, dev, pk, n_steps=None):
+    """3072 sequential la_recurrent_step launches, timed as a whole."""
+    T = n_steps or w.N
+    Q, K, V, _ = draw_workload(w)
+    q_t, k_t, v_t = (t[:, :, :T].permute(2, 0, 1, 3).contiguous().to(dev) for t in (Q, K, V))
+    S = torch.zeros((w.B, w.H, w.D, w.M), device=dev)
+    Z = torch.zeros((w.B, w.H, w.D), device=dev)
+    out = torch.empty((T, w.B, w.H, w.M), dtype=w.torch_dtype, device=dev)
+    for t in range(16):
+        la.la_recurrent_step(q_t[t], k_t[t], v_t[t], S, Z, out=out[t])
+    S.zero_()
+    Z.zero_()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(T):
+        la.la_recurrent_step(q_t[t], k_t[t], v_t[t], S, Z, out=out[t])
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    la.la_last_device_status()
+    us = ms * 1e3 / T
+    gbs = algorithmic_bytes(w, "both") / us * 1e-3
+    return {"workload": w.name, "steps_per_s": 1e6 / us, "us_per_step": us, "launches": T,
+            "alg_gbs": gbs, "hbm_frac": gbs / pk["hbm_gbs"], "state_bytes": S.numel() * 4,
+            "note": "state (32 MiB) fits the 126 MB L2, so the fraction may exceed the DRAM roofline"}
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample(w, pairs):
+    """Inputs of the first `pairs` (batch, head) pairs of workload w, as [1, pairs, N, .]."""
+    Q, K, V, G = draw_qkvg(1, pairs, w.N, w.D, w.M, w.seed, w.torch_dtype, w.scale)
+    return [t.double().numpy() for t in (Q, K, V, G)]
+
+
+def oracle_step(oracle, w, data):
+    Q, K, V, G = data
+    causal = w.kind == "causal"
+    oracle.linear_attention(Q, K, V, causal)
+    oracle.linear_attention_backward(Q, K, V, G, causal)
+
+
+def cpu_baseline(w, budget_s=15.0):
+    import oracle
+    cores = oracle.num_threads()
+    data = oracle_sample(w, cores)
+    t0 = time.perf_counter()
+    oracle_step(oracle, w, data)
+    once = time.perf_counter() - t0
+    reps = max(1, min(20, int(budget_s / max(once, 1e-3))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle_step(oracle, w, data)
+    dt = (time.perf_counter() - t0) / reps
+    frac = cores / (w.B * w.H)
+    return {"value": w.tokens * frac / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": f"{cores} of {w.B * w.H} (batch, head) pairs of {w.name}, fwd+bwd, {reps} repetitions; "
+                      "rate scaled to whole-workload tokens"}
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    w = WORKLOADS[args.workload]
+    cores = oracle.num_threads()
+    data = oracle_sample(w, cores)
+    frac = cores / (w.B * w.H)
+    for _ in range(args.warmup):
+        oracle_step(oracle, w, data)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(oracle, w, data)
+    ms = (time.perf_counter() - t0) / args.steps * 1e3
+    value = w.tokens * frac / (ms * 1e-3)
+    sample = f"{cores} of {w.B * w.H} (batch, head) pairs per step; rate scaled to whole-workload tokens"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, 1),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "kind": "oracle", "cores": cores, "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def workload_config(w, world):
+    return {"workload": w.name, "mirrors": w.mirrors, "B_per_gpu": w.B, "H": w.H, "N": w.N, "D": w.D, "M": w.M,
+            "io_dtype": w.dtype, "phi": "elu+1", "eps": 0.0, "seed": w.seed,
+            "parallelism": f"{world} independent shard(s) of (batch, head) pairs, no collective",
+            "l2": "per-step working set (inputs+outputs >= 1 GiB at the default workload) exceeds the 126 MB L2; no flush needed"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[k for k, v in WORKLOADS.items() if v.kind != "decode"])
+    ap.add_argument("--main-only", action="store_true", help="skip the other hot-path rows and the CPU baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    world, rank, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    import paper_2006_16236_b200 as la
+    pk = peaks()
+    w = WORKLOADS[args.workload]
+
+    main_res = bench_attention(la, w, dev, args.steps, args.warmup, world, rank, pk)
+
+    rows = {}
+    if world == 1 and not args.main_only:
+        k, wu = max(3, min(args.steps, 10)), 3
+        for name, ww in WORKLOADS.items():
+            if name == w.name:
+                continue
+            if ww.kind == "decode":
+                rows[name] = bench_decode(la, ww, dev, pk)
+            else:
+                r = bench_attention(la, ww, dev, k, wu, 1, 0, pk, do_e2e=False)
+                rows[name] = {kk: r[kk] for kk in ("value", "ms_per_step", "fwd_ms", "bwd_ms", "alg_gbs", "hbm_frac",
+                                                   "alg_tflops", "tensor_frac_alg_flops", "gpu_launches")}
+                rows[name]["unit"] = "tokens/s"
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.main_only:
+        cpu = cpu_baseline(w)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": main_res["value"], "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": main_res["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+            "data": "synthetic", "config": workload_config(w, world), "clocks": main_res["clocks"],
+            "e2e": main_res.get("e2e"), "gpu_launches": main_res["gpu_launches"],
+            "roofline": main_res["roofline"], "cpu_baseline": cpu,
+            "breakdown": {kk: main_res[kk] for kk in ("fwd_ms", "bwd_ms", "alg_gbs", "hbm_frac", "alg_tflops",
+                                                      "tensor_frac_alg_flops")},
+            "peaks": {kk: pk.get(kk) for kk in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "source")},
+            "rows": rows,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

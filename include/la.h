@@ -1,0 +1,165 @@
+/*
+ * la.h -- C ABI of the linear-attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes the attention core of "Transformers are RNNs"
+ * (Katharopoulos et al., 2020): attention with the kernel feature map
+ * phi(x) = elu(x) + 1 in its non-causal form, its causal form with the running
+ * state S_i = sum_{j<=i} phi(K_j) V_j^T and normaliser Z_i = sum_{j<=i} phi(K_j),
+ * forward and backward, and the one-token recurrent (RNN) step.
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ *  - Every data pointer is DEVICE memory owned by the caller.  The library
+ *    allocates and frees nothing; scratch memory is passed in as `ws` and sized
+ *    with la_workspace_bytes().  `ws` contents are undefined on return.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *    Every call only enqueues work on it and returns without synchronising.
+ *  - Tensors are row-major and contiguous, one (batch, head) pair after another:
+ *        Q, K, dQ, dK : [B, H, N, D]        V, O, G, dV : [B, H, N, M]
+ *        den          : [B, H, N]  fp32     S : [B, H, D, M] fp32    Z : [B, H, D] fp32
+ *    Q, K, V, O, G and the gradients have the I/O type la_problem.dtype (fp32
+ *    or bf16, round-to-nearest-even on output); states, normalisers and all
+ *    accumulation are fp32.  Data pointers must be 16-byte aligned.
+ *  - Outputs must not alias inputs (S and Z of la_recurrent_step are in-out).
+ *  - Supported sizes: D and M multiples of 8 in [8, 128]; B, H >= 1; N >= 0
+ *    (N == 0 is a successful no-op).  bf16 problems with D = M in {32, 64} and N
+ *    a multiple of the chunk length run on the tensor-core kernels, everything
+ *    else on the general fp32-arithmetic kernels; results agree within the
+ *    rounding of the I/O type.
+ *  - Return value: LA_OK (0) or a negative la_status.  All argument checks run
+ *    on the host before anything is enqueued; a failed check enqueues nothing.
+ *    The library never aborts, throws or traps.  la_last_error() returns a
+ *    static, thread-local description of the last failure on this thread.
+ */
+#ifndef LA_H_
+#define LA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LA_OK = 0,
+    LA_ERR_INVALID_ARG = -1,    /* NULL pointer, negative size, misaligned pointer, bad enum  */
+    LA_ERR_UNSUPPORTED = -2,    /* well-formed problem outside the supported sizes/types      */
+    LA_ERR_WORKSPACE = -3,      /* ws is NULL or smaller than la_workspace_bytes()            */
+    LA_ERR_CUDA = -4,           /* a CUDA runtime call failed (see la_last_error())           */
+    LA_ERR_ARCH = -5,           /* current device is not compute capability 10.x              */
+    LA_ERR_DEVICE_TIMEOUT = -6  /* a bounded device-side wait expired (reported by
+                                   la_last_device_status())                                   */
+} la_status;
+
+typedef enum { LA_F32 = 0, LA_BF16 = 1 } la_dtype;
+
+/* LA_PHI_ELU1: the library applies phi(x) = elu(x) + 1 (Eq. 7) to Q and K and
+ * returns gradients with respect to the raw Q, K.  LA_PHI_IDENTITY: Q and K
+ * already hold phi(Q), phi(K) (the convention of Algorithm 1); gradients are
+ * with respect to those. */
+typedef enum { LA_PHI_ELU1 = 0, LA_PHI_IDENTITY = 1 } la_phi;
+
+typedef enum {
+    LA_OP_LINEAR_FORWARD = 0,
+    LA_OP_LINEAR_BACKWARD = 1,
+    LA_OP_CAUSAL_FORWARD = 2,
+    LA_OP_CAUSAL_BACKWARD = 3
+} la_op;
+
+typedef struct {
+    int64_t B, H, N, D, M;   /* batch, heads, sequence length, query/key dim, value dim */
+    int32_t dtype;           /* la_dtype of Q, K, V, O, G and the gradients             */
+    int32_t phi;             /* la_phi                                                  */
+    float   eps;             /* added to every denominator; the paper uses none (0)     */
+} la_problem;
+
+/*
+ * Feature map, Eq. 7:  y[i] = phi(x[i]) = x[i] + 1 (x[i] > 0), exp(x[i]) otherwise;
+ * with deriv != 0, y[i] = phi'(x[i]) = 1 (x[i] > 0), exp(x[i]) otherwise.
+ * x, y: n elements of `dtype` (device).  y may equal x (in place).
+ */
+int la_feature_map(const void* x, void* y, int64_t n, int32_t dtype, int32_t deriv, void* stream);
+
+/*
+ * Non-causal linear attention, Eq. 5-6:
+ *   KV = sum_j phi(K_j) V_j^T,  Zs = sum_j phi(K_j)   (formed once per head),
+ *   O_i = phi(Q_i)^T KV / (phi(Q_i)^T Zs + eps).
+ * den (optional, may be NULL): phi(Q_i)^T Zs without eps.  KV / Zs (optional): the
+ * per-head sums, [B,H,D,M] / [B,H,D] fp32.
+ */
+int la_linear_attention(const la_problem* p, const void* Q, const void* K, const void* V,
+                        void* O, float* den, float* KV, float* Zs,
+                        void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Gradient of the non-causal form for an upstream gradient G = dL/dO.  The paper
+ * leaves the division to automatic differentiation; here it is absorbed by
+ * running the cumulative-sum gradients of Eq. 13-15 (with full, unmasked sums)
+ * on the values extended by a constant 1.  O and den are accepted for symmetry
+ * with autograd-style callers and may be NULL: everything needed is recomputed.
+ */
+int la_linear_attention_backward(const la_problem* p, const void* Q, const void* K, const void* V,
+                                 const void* O, const float* den, const void* G,
+                                 void* dQ, void* dK, void* dV,
+                                 void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Causal linear attention, Eq. 9-12 (Algorithm 1, forward, plus the normaliser):
+ *   S_i = S_{i-1} + phi(K_i) V_i^T,  Z_i = Z_{i-1} + phi(K_i),  S_0 = 0, Z_0 = 0,
+ *   O_i = phi(Q_i)^T S_i / (phi(Q_i)^T Z_i + eps)       (position i sees j <= i).
+ * den (optional): phi(Q_i)^T Z_i without eps.  S_out / Z_out (optional): the final
+ * state S_N, Z_N, which continues the sequence through la_recurrent_step().
+ */
+int la_causal_forward(const la_problem* p, const void* Q, const void* K, const void* V,
+                      void* O, float* den, float* S_out, float* Z_out,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Gradient of the causal form in linear time and memory independent of N per
+ * head, Eq. 13-15 (Algorithm 1, backward): grad phi(Q_i) uses the forward running
+ * sum of phi(K_j)[V_j,1]^T, grad phi(K_i) and grad V_i the reverse running sum of
+ * phi(Q_j) Gt_j^T, where Gt_j = [G_j/den_j, -(G_j.O_j)/den_j] carries the division.
+ * No per-position state is stored.  G = dL/dO.  O and den may be NULL (recomputed).
+ */
+int la_causal_backward(const la_problem* p, const void* Q, const void* K, const void* V,
+                       const void* O, const float* den, const void* G,
+                       void* dQ, void* dK, void* dV,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * One recurrent step per (batch, head) stream, Eq. 16-20 (attention part); the
+ * state is updated BEFORE it is read:
+ *   S += phi(k) v^T,  Z += phi(k),  out = phi(q)^T S / (phi(q)^T Z + eps).
+ * q, k: [B,H,D]; v, out: [B,H,M] of p->dtype; S: [B,H,D,M], Z: [B,H,D] fp32, updated
+ * in place (zero them to start a sequence).  p->N is ignored.  Needs no workspace.
+ */
+int la_recurrent_step(const la_problem* p, const void* q, const void* k, const void* v,
+                      float* S, float* Z, void* out, void* stream);
+
+/* Bytes of workspace `op` needs for problem p (pure host function; 0 if none).
+ * Returns 0 for invalid problems as well: the entry point reports the error. */
+size_t la_workspace_bytes(const la_problem* p, int32_t op);
+
+/* Human-readable name of a status code (static string). */
+const char* la_status_string(int status);
+
+/* Description of the last failure on the calling thread ("" if none). */
+const char* la_last_error(void);
+
+/* Synchronises `stream`, then reports whether any kernel of this library gave up
+ * on a bounded wait since the last call (LA_ERR_DEVICE_TIMEOUT) and clears the
+ * flag; LA_OK otherwise.  The context stays usable either way. */
+int la_last_device_status(void* stream);
+
+/* Number of GPU kernels this library has enqueued in this process so far (all
+ * threads, all entry points); a diagnostic for benchmarks. */
+long long la_kernel_launches(void);
+
+/* Library version, "major.minor". */
+const char* la_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LA_H_ */

@@ -1,0 +1,222 @@
+"""Thin ctypes binding of the C ABI in include/la.h.
+
+Argument marshalling only: torch supplies device memory and the current
+stream; every step of the computation runs in the CUDA library.  There is no
+CPU fallback -- a missing or unloadable library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libla.so")
+
+LA_F32, LA_BF16 = 0, 1
+LA_PHI_ELU1, LA_PHI_IDENTITY = 0, 1
+LA_OP_LINEAR_FORWARD, LA_OP_LINEAR_BACKWARD, LA_OP_CAUSAL_FORWARD, LA_OP_CAUSAL_BACKWARD = 0, 1, 2, 3
+_PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
+
+EXPORTS = [
+    "la_feature_map", "la_linear_attention", "la_linear_attention_backward", "la_causal_forward",
+    "la_causal_backward", "la_recurrent_step", "la_workspace_bytes", "la_status_string",
+    "la_last_error", "la_last_device_status", "la_kernel_launches", "la_version",
+]
+
+
+class la_problem(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int64), ("H", ctypes.c_int64), ("N", ctypes.c_int64),
+                ("D", ctypes.c_int64), ("M", ctypes.c_int64), ("dtype", ctypes.c_int32),
+                ("phi", ctypes.c_int32), ("eps", ctypes.c_float)]
+
+
+class LaError(RuntimeError):
+    def __init__(self, status: int, name: str, message: str):
+        super().__init__(f"{name} ({status}): {message}")
+        self.status, self.name = status, name
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libla.so (built in-tree by ``paper_2006_16236_b200.build``); raise if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2006_16236_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
+        pp = ctypes.POINTER(la_problem)
+        L.la_feature_map.argtypes = [vp, vp, i64, i32, i32, vp]
+        L.la_linear_attention.argtypes = [pp] + [vp] * 7 + [vp, sz, vp]
+        L.la_linear_attention_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
+        L.la_causal_forward.argtypes = [pp] + [vp] * 7 + [vp, sz, vp]
+        L.la_causal_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
+        L.la_recurrent_step.argtypes = [pp] + [vp] * 6 + [vp]
+        L.la_workspace_bytes.argtypes = [pp, i32]
+        L.la_workspace_bytes.restype = sz
+        L.la_status_string.argtypes = [ctypes.c_int]
+        L.la_status_string.restype = ctypes.c_char_p
+        L.la_last_error.restype = ctypes.c_char_p
+        L.la_last_device_status.argtypes = [vp]
+        L.la_version.restype = ctypes.c_char_p
+        L.la_kernel_launches.restype = ctypes.c_longlong
+        for name in EXPORTS:
+            getattr(L, name)
+        _lib = L
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        L = lib()
+        raise LaError(rc, L.la_status_string(rc).decode(), L.la_last_error().decode())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return LA_F32
+    if t.dtype == torch.bfloat16:
+        return LA_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}: use float32 or bfloat16")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(device) -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def _dev(*ts):
+    for t in ts:
+        if t is None:
+            continue
+        if not t.is_cuda:
+            raise ValueError("tensors must live on a CUDA device")
+        if not t.is_contiguous():
+            raise ValueError("tensors must be contiguous")
+    return ts[0].device
+
+
+def make_problem(B, H, N, D, M, dtype_code, phi="elu1", eps=0.0) -> la_problem:
+    return la_problem(B, H, N, D, M, dtype_code, _PHI[phi] if isinstance(phi, str) else int(phi), float(eps))
+
+
+def _problem_of(Q, V, phi, eps) -> la_problem:
+    if Q.dim() != 4 or V.dim() != 4:
+        raise ValueError("expected Q,K [B,H,N,D] and V [B,H,N,M]")
+    B, H, N, D = Q.shape
+    return make_problem(B, H, N, D, V.shape[3], _dtype_code(Q), phi, eps)
+
+
+_ws_cache = {}
+
+
+def workspace(p: la_problem, op: int, device) -> torch.Tensor | None:
+    """A cached scratch tensor of la_workspace_bytes(p, op) bytes on `device` (None if 0)."""
+    need = lib().la_workspace_bytes(ctypes.byref(p), op)
+    if need == 0:
+        return None
+    key = (str(device), op)
+    buf = _ws_cache.get(key)
+    if buf is None or buf.numel() < need:
+        buf = torch.empty(need, dtype=torch.uint8, device=device)
+        _ws_cache[key] = buf
+    return buf
+
+
+def la_workspace_bytes(p: la_problem, op: int) -> int:
+    return lib().la_workspace_bytes(ctypes.byref(p), op)
+
+
+def la_kernel_launches() -> int:
+    return int(lib().la_kernel_launches())
+
+
+def la_version() -> str:
+    return lib().la_version().decode()
+
+
+def la_last_device_status(device=None) -> None:
+    """Synchronise the current stream; raise LaError if a kernel gave up on a bounded wait."""
+    _check(lib().la_last_device_status(_stream(device)))
+
+
+def la_feature_map(x: torch.Tensor, deriv: bool = False, out: torch.Tensor | None = None) -> torch.Tensor:
+    dev = _dev(x, out)
+    y = torch.empty_like(x) if out is None else out
+    _check(lib().la_feature_map(_ptr(x), _ptr(y), x.numel(), _dtype_code(x), int(deriv), _stream(dev)))
+    return y
+
+
+def la_linear_attention(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, KV=None, Zs=None, ws=None):
+    """Non-causal form.  Returns O; pass preallocated den / KV / Zs tensors to receive them."""
+    dev = _dev(Q, K, V, O, den, KV, Zs)
+    p = _problem_of(Q, V, phi, eps)
+    O = torch.empty_like(V) if O is None else O
+    ws = workspace(p, LA_OP_LINEAR_FORWARD, dev) if ws is None else ws
+    _check(lib().la_linear_attention(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(KV),
+                                     _ptr(Zs), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                     _stream(dev)))
+    return O
+
+
+def la_linear_attention_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None,
+                                 dQ=None, dK=None, dV=None, ws=None):
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV)
+    p = _problem_of(Q, V, phi, eps)
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(K) if dK is None else dK
+    dV = torch.empty_like(V) if dV is None else dV
+    ws = workspace(p, LA_OP_LINEAR_BACKWARD, dev) if ws is None else ws
+    _check(lib().la_linear_attention_backward(
+        ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV),
+        _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(dev)))
+    return dQ, dK, dV
+
+
+def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None, Z_out=None, ws=None):
+    """Causal form.  Returns O; pass preallocated den / S_out / Z_out tensors to receive them."""
+    dev = _dev(Q, K, V, O, den, S_out, Z_out)
+    p = _problem_of(Q, V, phi, eps)
+    O = torch.empty_like(V) if O is None else O
+    ws = workspace(p, LA_OP_CAUSAL_FORWARD, dev) if ws is None else ws
+    _check(lib().la_causal_forward(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(S_out),
+                                   _ptr(Z_out), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                   _stream(dev)))
+    return O
+
+
+def la_causal_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None, dQ=None, dK=None, dV=None, ws=None):
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV)
+    p = _problem_of(Q, V, phi, eps)
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(K) if dK is None else dK
+    dV = torch.empty_like(V) if dV is None else dV
+    ws = workspace(p, LA_OP_CAUSAL_BACKWARD, dev) if ws is None else ws
+    _check(lib().la_causal_backward(
+        ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV),
+        _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(dev)))
+    return dQ, dK, dV
+
+
+def la_recurrent_step(q, k, v, S, Z, phi="elu1", eps=0.0, out=None):
+    """One decode step: S, Z (fp32) are updated in place; returns out [B,H,M]."""
+    dev = _dev(q, k, v, S, Z, out)
+    if q.dim() != 3 or v.dim() != 3 or S.dtype != torch.float32 or Z.dtype != torch.float32:
+        raise ValueError("expected q,k [B,H,D], v [B,H,M], fp32 S [B,H,D,M] and Z [B,H,D]")
+    B, H, D = q.shape
+    M = v.shape[2]
+    if tuple(S.shape) != (B, H, D, M) or tuple(Z.shape) != (B, H, D):
+        raise ValueError("state shape mismatch")
+    p = make_problem(B, H, 1, D, M, _dtype_code(q), phi, eps)
+    out = torch.empty_like(v) if out is None else out
+    _check(lib().la_recurrent_step(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out),
+                                   _stream(dev)))
+    return out

@@ -1,0 +1,212 @@
+// C ABI of the linear-attention library: argument validation, dispatch between
+// the tensor-core and the general kernels, status reporting.  Nothing here
+// allocates device memory or synchronises (except la_last_device_status).
+#include <atomic>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "la_common.cuh"
+#include "la_tc.cuh"
+
+namespace la {
+
+static thread_local char g_error[512] = "";
+
+int fail(int status, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof(g_error), fmt, ap);
+    va_end(ap);
+    return status;
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+    return fail(LA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+static std::atomic<long long> g_launches{0};
+void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+__device__ int g_device_status_word = 0;
+
+int* device_status_ptr() {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_device_status_word) != cudaSuccess) return nullptr;
+    return (int*)p;
+}
+
+static int check_arch() {
+    static thread_local int cached_dev = -1, cached_rc = 0;
+    int dev = 0;
+    LA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev == cached_dev) return cached_rc;
+    int major = 0;
+    LA_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    cached_dev = dev;
+    cached_rc = major == 10 ? LA_OK : LA_ERR_ARCH;
+    if (cached_rc) return fail(LA_ERR_ARCH, "device %d has compute capability %d.x; this library is built for sm_100a only", dev, major);
+    return LA_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_problem(const la_problem* p, bool need_n) {
+    if (!p) return fail(LA_ERR_INVALID_ARG, "problem descriptor is NULL");
+    if (p->B < 1 || p->H < 1 || p->D < 1 || p->M < 1 || (need_n && p->N < 0))
+        return fail(LA_ERR_INVALID_ARG, "sizes must be B,H,D,M >= 1 and N >= 0 (got B=%lld H=%lld N=%lld D=%lld M=%lld)",
+                    (long long)p->B, (long long)p->H, (long long)p->N, (long long)p->D, (long long)p->M);
+    if (p->dtype != LA_F32 && p->dtype != LA_BF16) return fail(LA_ERR_INVALID_ARG, "dtype %d is not a la_dtype", p->dtype);
+    if (p->phi != LA_PHI_ELU1 && p->phi != LA_PHI_IDENTITY) return fail(LA_ERR_INVALID_ARG, "phi %d is not a la_phi", p->phi);
+    if (!(p->eps >= 0.f)) return fail(LA_ERR_INVALID_ARG, "eps must be >= 0");
+    if (p->D % 8 || p->M % 8 || p->D > 128 || p->M > 128)
+        return fail(LA_ERR_UNSUPPORTED, "D and M must be multiples of 8 in [8,128] (got D=%lld M=%lld)",
+                    (long long)p->D, (long long)p->M);
+    if (p->B * p->H > 0x7fffffffLL) return fail(LA_ERR_UNSUPPORTED, "B*H exceeds 2^31-1");
+    if (need_n && p->N > (1LL << 40) / (p->D > p->M ? p->D : p->M))
+        return fail(LA_ERR_UNSUPPORTED, "sequence too long");
+    return LA_OK;
+}
+
+#define LA_REQUIRE_PTR(ptr)                                                                \
+    do {                                                                                   \
+        if (!(ptr)) return fail(LA_ERR_INVALID_ARG, #ptr " is NULL");                      \
+        if (!aligned16(ptr)) return fail(LA_ERR_INVALID_ARG, #ptr " is not 16-byte aligned"); \
+    } while (0)
+#define LA_OPTIONAL_PTR(ptr)                                                               \
+    do {                                                                                   \
+        if ((ptr) && !aligned16(ptr)) return fail(LA_ERR_INVALID_ARG, #ptr " is not 16-byte aligned"); \
+    } while (0)
+
+static int check_ws(const la_problem* p, int op, const void* ws, size_t ws_bytes) {
+    const size_t need = la_workspace_bytes(p, op);
+    if (need == 0) return LA_OK;
+    if (!ws) return fail(LA_ERR_WORKSPACE, "workspace is NULL but %zu bytes are needed", need);
+    if (!aligned16(ws)) return fail(LA_ERR_INVALID_ARG, "workspace is not 16-byte aligned");
+    if (ws_bytes < need) return fail(LA_ERR_WORKSPACE, "workspace has %zu bytes, %zu are needed", ws_bytes, need);
+    return LA_OK;
+}
+
+}  // namespace la
+
+using namespace la;
+
+extern "C" {
+
+const char* la_version(void) { return "0.1"; }
+
+const char* la_status_string(int status) {
+    switch (status) {
+        case LA_OK: return "LA_OK";
+        case LA_ERR_INVALID_ARG: return "LA_ERR_INVALID_ARG";
+        case LA_ERR_UNSUPPORTED: return "LA_ERR_UNSUPPORTED";
+        case LA_ERR_WORKSPACE: return "LA_ERR_WORKSPACE";
+        case LA_ERR_CUDA: return "LA_ERR_CUDA";
+        case LA_ERR_ARCH: return "LA_ERR_ARCH";
+        case LA_ERR_DEVICE_TIMEOUT: return "LA_ERR_DEVICE_TIMEOUT";
+        default: return "LA_ERR_UNKNOWN";
+    }
+}
+
+const char* la_last_error(void) { return g_error; }
+
+long long la_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+size_t la_workspace_bytes(const la_problem* p, int32_t op) {
+    if (!p || p->B < 1 || p->H < 1 || p->N < 0 || p->D < 1 || p->M < 1 || p->D > 128 || p->M > 128) return 0;
+    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_CAUSAL_BACKWARD) return 0;
+    if (p->N == 0) return 0;
+    if (tc_supported(*p, op)) return tc_workspace_bytes(*p, op);
+    return general_workspace_bytes(*p, op);
+}
+
+int la_feature_map(const void* x, void* y, int64_t n, int32_t dtype, int32_t deriv, void* stream) {
+    if (n < 0) return fail(LA_ERR_INVALID_ARG, "n must be >= 0");
+    if (dtype != LA_F32 && dtype != LA_BF16) return fail(LA_ERR_INVALID_ARG, "dtype %d is not a la_dtype", dtype);
+    if (n == 0) return LA_OK;
+    LA_REQUIRE_PTR(x);
+    LA_REQUIRE_PTR(y);
+    if (int rc = check_arch()) return rc;
+    return launch_feature_map(x, y, n, dtype, deriv != 0, (cudaStream_t)stream);
+}
+
+int la_linear_attention(const la_problem* p, const void* Q, const void* K, const void* V,
+                        void* O, float* den, float* KV, float* Zs,
+                        void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_problem(p, true)) return rc;
+    if (p->N == 0) return LA_OK;
+    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(O);
+    LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(KV); LA_OPTIONAL_PTR(Zs);
+    if (int rc = check_ws(p, LA_OP_LINEAR_FORWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_arch()) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc_linear_forward(*p, Q, K, V, O, den, KV, Zs, ws, st);
+    return general_linear_forward(*p, Q, K, V, O, den, KV, Zs, ws, st);
+}
+
+int la_linear_attention_backward(const la_problem* p, const void* Q, const void* K, const void* V,
+                                 const void* O, const float* den, const void* G,
+                                 void* dQ, void* dK, void* dV,
+                                 void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_problem(p, true)) return rc;
+    if (p->N == 0) return LA_OK;
+    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(G);
+    LA_REQUIRE_PTR(dQ); LA_REQUIRE_PTR(dK); LA_REQUIRE_PTR(dV);
+    LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den);
+    if (int rc = check_ws(p, LA_OP_LINEAR_BACKWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_arch()) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc_linear_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
+    return general_linear_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
+}
+
+int la_causal_forward(const la_problem* p, const void* Q, const void* K, const void* V,
+                      void* O, float* den, float* S_out, float* Z_out,
+                      void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_problem(p, true)) return rc;
+    if (p->N == 0) return LA_OK;
+    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(O);
+    LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(S_out); LA_OPTIONAL_PTR(Z_out);
+    if (int rc = check_ws(p, LA_OP_CAUSAL_FORWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_arch()) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (tc_supported(*p, LA_OP_CAUSAL_FORWARD)) return tc_causal_forward(*p, Q, K, V, O, den, S_out, Z_out, ws, st);
+    return general_causal_forward(*p, Q, K, V, O, den, S_out, Z_out, st);
+}
+
+int la_causal_backward(const la_problem* p, const void* Q, const void* K, const void* V,
+                       const void* O, const float* den, const void* G,
+                       void* dQ, void* dK, void* dV,
+                       void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_problem(p, true)) return rc;
+    if (p->N == 0) return LA_OK;
+    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(G);
+    LA_REQUIRE_PTR(dQ); LA_REQUIRE_PTR(dK); LA_REQUIRE_PTR(dV);
+    LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den);
+    if (int rc = check_ws(p, LA_OP_CAUSAL_BACKWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_arch()) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (tc_supported(*p, LA_OP_CAUSAL_BACKWARD)) return tc_causal_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
+    return general_causal_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
+}
+
+int la_recurrent_step(const la_problem* p, const void* q, const void* k, const void* v,
+                      float* S, float* Z, void* out, void* stream) {
+    if (int rc = check_problem(p, false)) return rc;
+    LA_REQUIRE_PTR(q); LA_REQUIRE_PTR(k); LA_REQUIRE_PTR(v);
+    LA_REQUIRE_PTR(S); LA_REQUIRE_PTR(Z); LA_REQUIRE_PTR(out);
+    if (int rc = check_arch()) return rc;
+    return launch_recurrent_step(*p, q, k, v, S, Z, out, (cudaStream_t)stream);
+}
+
+int la_last_device_status(void* stream) {
+    LA_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    int word = 0;
+    LA_CUDA_TRY(cudaMemcpyFromSymbol(&word, g_device_status_word, sizeof(int)));
+    if (word == 0) return LA_OK;
+    int zero = 0;
+    LA_CUDA_TRY(cudaMemcpyToSymbol(g_device_status_word, &zero, sizeof(int)));
+    return fail(LA_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (device status 0x%x)", word);
+}
+
+}  // extern "C"

@@ -1,0 +1,78 @@
+// Shared device/host helpers of the linear-attention library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "la.h"
+
+namespace la {
+
+// ---- host-side error plumbing (defined in la_api.cu) -----------------------
+int fail(int status, const char* fmt, ...);
+int cuda_fail(cudaError_t e, const char* what);
+
+// After a <<<...>>> launch: count it and surface a launch error.
+#define LA_LAUNCHED()                          \
+    do {                                       \
+        ::la::note_launch();                   \
+        LA_CUDA_TRY(cudaGetLastError());       \
+    } while (0)
+
+#define LA_CUDA_TRY(expr)                                          \
+    do {                                                           \
+        cudaError_t e__ = (expr);                                  \
+        if (e__ != cudaSuccess) return ::la::cuda_fail(e__, #expr); \
+    } while (0)
+
+// Device status word: kernels that give up on a bounded wait OR a code into it.
+// Returns its device address for the current device (NULL on failure).
+int* device_status_ptr();
+
+// Every kernel launch of the library is counted (see la_kernel_launches()).
+void note_launch();
+
+// ---- element access in the I/O type ----------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) {
+    return __bfloat162float(x);
+}
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) {
+    return __float2bfloat16_rn(x);
+}
+
+// ---- feature map, Eq. 7 ------------------------------------------------------
+// phi(x) = x + 1 for x > 0, exp(x) otherwise; identity mode passes x through.
+__device__ __forceinline__ float phi_apply(float x, int phi) {
+    if (phi == LA_PHI_IDENTITY) return x;
+    return x > 0.f ? x + 1.f : expf(x);
+}
+// Slope of phi recovered from its value y = phi(x): x > 0 <=> y > 1, where the
+// slope is 1; otherwise the slope equals the value exp(x).
+__device__ __forceinline__ float phi_slope_from_value(float y, int phi) {
+    if (phi == LA_PHI_IDENTITY) return 1.f;
+    return y > 1.f ? 1.f : y;
+}
+
+// ---- launchers implemented in the kernel files -------------------------------
+int launch_feature_map(const void* x, void* y, int64_t n, int dtype, int deriv, cudaStream_t st);
+
+int launch_recurrent_step(const la_problem& p, const void* q, const void* k, const void* v,
+                          float* S, float* Z, void* out, cudaStream_t st);
+
+// General (any D, M multiple of 8 up to 128, any N) fp32-arithmetic kernels.
+size_t general_workspace_bytes(const la_problem& p, int op);
+int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V,
+                           void* O, float* den, float* S_out, float* Z_out, cudaStream_t st);
+int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V,
+                            const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+int general_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V,
+                           void* O, float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
+int general_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V,
+                            const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+
+}  // namespace la

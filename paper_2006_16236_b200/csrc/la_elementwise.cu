@@ -1,0 +1,191 @@
+// Feature map (Eq. 7) as a stand-alone elementwise kernel, and the one-token
+// recurrent step (Eq. 16-20, attention part).
+#include "la_common.cuh"
+
+namespace la {
+
+// ---------------------------------------------------------------------------
+// Feature map: y = phi(x) or phi'(x).  Bandwidth-bound; 16-byte accesses on the
+// aligned body, scalar accesses on the ragged tail.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float fm(float x, int deriv) {
+    if (x > 0.f) return deriv ? 1.f : x + 1.f;
+    return expf(x);
+}
+
+template <typename T>
+__global__ void feature_map_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t n, int deriv) {
+    constexpr int V = 16 / sizeof(T);
+    const int64_t nvec = n / V;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t i = t0; i < nvec; i += stride) {
+        uint4 raw = reinterpret_cast<const uint4*>(x)[i];
+        T* e = reinterpret_cast<T*>(&raw);
+#pragma unroll
+        for (int j = 0; j < V; ++j) e[j] = from_f32<T>(fm(to_f32<T>(e[j]), deriv));
+        reinterpret_cast<uint4*>(y)[i] = raw;
+    }
+    for (int64_t i = nvec * V + t0; i < n; i += stride) y[i] = from_f32<T>(fm(to_f32<T>(x[i]), deriv));
+}
+
+int launch_feature_map(const void* x, void* y, int64_t n, int dtype, int deriv, cudaStream_t st) {
+    if (n == 0) return LA_OK;
+    const int threads = 256;
+    const int64_t vec = dtype == LA_F32 ? 4 : 8;
+    int64_t blocks = (n / vec + threads - 1) / threads;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (dtype == LA_F32)
+        feature_map_kernel<float><<<(unsigned)blocks, threads, 0, st>>>((const float*)x, (float*)y, n, deriv);
+    else
+        feature_map_kernel<__nv_bfloat16><<<(unsigned)blocks, threads, 0, st>>>(
+            (const __nv_bfloat16*)x, (__nv_bfloat16*)y, n, deriv);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Recurrent step.  One CTA of 128 threads per (batch, head) state.  The D x M
+// fp32 state is streamed HBM -> registers -> HBM exactly once with 16-byte
+// accesses: a thread owns four consecutive columns of every RPP-th row, so a
+// warp covers whole 128-byte lines.  All state loads are issued before anything
+// else is waited on.  phi(q)^T S is reduced with warp shuffles and one shared
+// memory hop across the four warps; phi(q)^T Z likewise.
+// ---------------------------------------------------------------------------
+template <typename T, int D, int M>
+__global__ void __launch_bounds__(128)
+recurrent_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                      float* __restrict__ S, float* __restrict__ Z, T* __restrict__ out,
+                      float eps, int phi) {
+    constexpr int TPR = M / 4;        // threads per state row (one float4 each)
+    constexpr int RPP = 128 / TPR;    // rows covered per pass of the CTA
+    constexpr int PASSES = D / RPP;
+    static_assert(D % RPP == 0 && PASSES >= 1, "unsupported state shape");
+
+    __shared__ float sq[D], sk[D];
+    __shared__ __align__(16) float sv[M];
+    __shared__ __align__(16) float spart[4][M];
+    __shared__ float sden[4];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t bh = blockIdx.x;
+    const int c4 = tid % TPR, r0 = tid / TPR;
+
+    float4* Sp = reinterpret_cast<float4*>(S + bh * (int64_t)(D * M));
+    float4 s[PASSES];
+#pragma unroll
+    for (int p = 0; p < PASSES; ++p) s[p] = Sp[(r0 + p * RPP) * TPR + c4];
+
+    float zq = 0.f;
+    if (tid < D) {
+        float kd = phi_apply(to_f32<T>(k[bh * D + tid]), phi);
+        float qd = phi_apply(to_f32<T>(q[bh * D + tid]), phi);
+        float z = Z[bh * D + tid] + kd;
+        Z[bh * D + tid] = z;
+        sk[tid] = kd;
+        sq[tid] = qd;
+        zq = qd * z;
+    }
+    if (tid < M) sv[tid] = to_f32<T>(v[bh * M + tid]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) zq += __shfl_xor_sync(0xffffffffu, zq, off);
+    if (lane == 0) sden[warp] = zq;
+    __syncthreads();
+
+    const float4 vv = reinterpret_cast<const float4*>(sv)[c4];
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int p = 0; p < PASSES; ++p) {
+        const int d = r0 + p * RPP;
+        const float kd = sk[d], qd = sq[d];
+        s[p].x = fmaf(kd, vv.x, s[p].x);
+        s[p].y = fmaf(kd, vv.y, s[p].y);
+        s[p].z = fmaf(kd, vv.z, s[p].z);
+        s[p].w = fmaf(kd, vv.w, s[p].w);
+        Sp[d * TPR + c4] = s[p];
+        acc.x = fmaf(qd, s[p].x, acc.x);
+        acc.y = fmaf(qd, s[p].y, acc.y);
+        acc.z = fmaf(qd, s[p].z, acc.z);
+        acc.w = fmaf(qd, s[p].w, acc.w);
+    }
+#pragma unroll
+    for (int off = 16; off >= TPR; off >>= 1) {
+        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, off);
+        acc.y += __shfl_xor_sync(0xffffffffu, acc.y, off);
+        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, off);
+        acc.w += __shfl_xor_sync(0xffffffffu, acc.w, off);
+    }
+    if (lane < TPR) reinterpret_cast<float4*>(spart[warp])[lane] = acc;
+    __syncthreads();
+    if (tid < M) {
+        const float den = sden[0] + sden[1] + sden[2] + sden[3] + eps;
+        const float num = spart[0][tid] + spart[1][tid] + spart[2][tid] + spart[3][tid];
+        out[bh * M + tid] = from_f32<T>(num / den);
+    }
+}
+
+// Any D, M (multiples of 8 up to 128): thread m owns column m of the state.
+template <typename T>
+__global__ void __launch_bounds__(128)
+recurrent_step_general_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                              float* __restrict__ S, float* __restrict__ Z, T* __restrict__ out,
+                              int D, int M, float eps, int phi) {
+    __shared__ float sq[128], sk[128], sden[4];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t bh = blockIdx.x;
+    float zq = 0.f;
+    if (tid < D) {
+        float kd = phi_apply(to_f32<T>(k[bh * D + tid]), phi);
+        float qd = phi_apply(to_f32<T>(q[bh * D + tid]), phi);
+        float z = Z[bh * D + tid] + kd;
+        Z[bh * D + tid] = z;
+        sk[tid] = kd;
+        sq[tid] = qd;
+        zq = qd * z;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) zq += __shfl_xor_sync(0xffffffffu, zq, off);
+    if (lane == 0) sden[warp] = zq;
+    __syncthreads();
+    if (tid < M) {
+        const float vm = to_f32<T>(v[bh * M + tid]);
+        float* Sp = S + bh * (int64_t)D * M + tid;
+        float num = 0.f;
+        for (int d = 0; d < D; ++d) {
+            float s = fmaf(sk[d], vm, Sp[(int64_t)d * M]);
+            Sp[(int64_t)d * M] = s;
+            num = fmaf(sq[d], s, num);
+        }
+        out[bh * M + tid] = from_f32<T>(num / (sden[0] + sden[1] + sden[2] + sden[3] + eps));
+    }
+}
+
+template <typename T>
+static int recurrent_dispatch(const la_problem& p, const void* q, const void* k, const void* v,
+                              float* S, float* Z, void* out, cudaStream_t st) {
+    const unsigned grid = (unsigned)(p.B * p.H);
+    const T *qq = (const T*)q, *kk = (const T*)k, *vv = (const T*)v;
+    T* oo = (T*)out;
+#define LA_RS_CASE(DD, MM)                                                                     \
+    if (p.D == DD && p.M == MM) {                                                              \
+        recurrent_step_kernel<T, DD, MM><<<grid, 128, 0, st>>>(qq, kk, vv, S, Z, oo, p.eps, p.phi); \
+        LA_LAUNCHED();                                                       \
+        return LA_OK;                                                                          \
+    }
+    LA_RS_CASE(32, 32) LA_RS_CASE(32, 64) LA_RS_CASE(64, 32) LA_RS_CASE(64, 64)
+    LA_RS_CASE(64, 128) LA_RS_CASE(128, 64) LA_RS_CASE(128, 128)
+#undef LA_RS_CASE
+    recurrent_step_general_kernel<T><<<grid, 128, 0, st>>>(qq, kk, vv, S, Z, oo, (int)p.D, (int)p.M,
+                                                           p.eps, p.phi);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+int launch_recurrent_step(const la_problem& p, const void* q, const void* k, const void* v,
+                          float* S, float* Z, void* out, cudaStream_t st) {
+    if (p.dtype == LA_F32) return recurrent_dispatch<float>(p, q, k, v, S, Z, out, st);
+    return recurrent_dispatch<__nv_bfloat16>(p, q, k, v, S, Z, out, st);
+}
+
+}  // namespace la

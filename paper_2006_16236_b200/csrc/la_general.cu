@@ -1,0 +1,583 @@
+// General kernels: any D, M (multiples of 8 up to 128), any N, fp32 or bf16 I/O,
+// fp32 arithmetic on the CUDA cores.  They serve fp32 problems (bf16 tensor-core
+// products cannot hold the fp32 tolerance) and every shape the tensor-core
+// kernels do not cover.  All four are chunked restatements of Algorithm 1 on the
+// values extended by a ones column:
+//     Vt_j = [V_j, 1],   St = [S | Z]  (D x (M+1)),   [num_i | den_i] = phi(Q_i)^T St_i.
+// For a chunk c of T consecutive positions with L the lower-triangular mask,
+//     [num|den]_c = ((q_c k_c^T) o L) Vt_c + q_c St_{c-1},   St_c = St_{c-1} + k_c^T Vt_c,
+// which is Eq. 9-12 with the sum over j <= i split at the chunk boundary.
+#include "la_common.cuh"
+
+namespace la {
+
+namespace {
+
+constexpr int T = 32;          // positions per chunk
+constexpr int THREADS = 256;
+
+struct Dims {
+    int D, M;      // feature / value dims
+    int DS;        // row stride of q/k tiles (D + 1: conflict-free column walks)
+    int MS;        // row stride of extended value tiles and states (M + 1)
+};
+
+__device__ __forceinline__ Dims make_dims(int D, int M) { return Dims{D, M, D + 1, M + 1}; }
+
+// dst[i][d] = phi(src[i][d]) for i < cn, 0 for the padded rows (zero in feature
+// space: a padded key contributes nothing to any sum).
+template <typename IO>
+__device__ void load_mapped(float* dst, const IO* src, int cn, int D, int DS, int phi) {
+    for (int idx = threadIdx.x; idx < T * D; idx += THREADS) {
+        const int i = idx / D, d = idx - i * D;
+        dst[i * DS + d] = i < cn ? phi_apply(to_f32<IO>(src[(int64_t)i * D + d]), phi) : 0.f;
+    }
+}
+
+// dst[i][0..M) = src[i][:], dst[i][M] = 1 (the ones column); padded rows are 0.
+template <typename IO>
+__device__ void load_values_ext(float* dst, const IO* src, int cn, int M, int MS) {
+    for (int idx = threadIdx.x; idx < T * MS; idx += THREADS) {
+        const int i = idx / MS, e = idx - i * MS;
+        float x = 0.f;
+        if (i < cn) x = e < M ? to_f32<IO>(src[(int64_t)i * M + e]) : 1.f;
+        dst[i * MS + e] = x;
+    }
+}
+
+// P[i][j] = q_i . k_j for j <= i (causal) else 0.
+__device__ void masked_scores(float* P, const float* q, const float* k, int D, int DS) {
+    for (int idx = threadIdx.x; idx < T * T; idx += THREADS) {
+        const int i = idx / T, j = idx - i * T;
+        float s = 0.f;
+        if (j <= i)
+            for (int d = 0; d < D; ++d) s = fmaf(q[i * DS + d], k[j * DS + d], s);
+        P[i * (T + 1) + j] = s;
+    }
+}
+
+// nd[i][e] = sum_{j<=i} P[i][j] vt[j][e] + sum_d q[i][d] St[d][e]   (e in [0, M])
+__device__ void numerator_denominator(float* nd, const float* P, const float* vt, const float* q,
+                                      const float* St, const Dims& dm, bool causal_part) {
+    for (int idx = threadIdx.x; idx < T * dm.MS; idx += THREADS) {
+        const int i = idx / dm.MS, e = idx - i * dm.MS;
+        float s = 0.f;
+        if (causal_part)
+            for (int j = 0; j <= i; ++j) s = fmaf(P[i * (T + 1) + j], vt[j * dm.MS + e], s);
+        for (int d = 0; d < dm.D; ++d) s = fmaf(q[i * dm.DS + d], St[d * dm.MS + e], s);
+        nd[i * dm.MS + e] = s;
+    }
+}
+
+// St[d][e] += sum_i x[i][d] y[i][e]   (rank-T update of a D x (M+1) state)
+__device__ void state_update(float* St, const float* x, const float* y, const Dims& dm) {
+    for (int idx = threadIdx.x; idx < dm.D * dm.MS; idx += THREADS) {
+        const int d = idx / dm.MS, e = idx - d * dm.MS;
+        float s = St[idx];
+        for (int i = 0; i < T; ++i) s = fmaf(x[i * dm.DS + d], y[i * dm.MS + e], s);
+        St[idx] = s;
+    }
+}
+
+__device__ void zero_fill(float* p, int n) {
+    for (int idx = threadIdx.x; idx < n; idx += THREADS) p[idx] = 0.f;
+}
+
+// Turn the raw upstream gradient tile g (values in [0,M), anything in column M)
+// into Gt_i = [G_i / dn_i, -(G_i . O_i) / dn_i] with dn_i = den_i + eps and
+// O_i = num_i / dn_i taken from nd.  One warp handles rows i = warp, warp+8, ...
+__device__ void extend_upstream(float* g, const float* nd, const Dims& dm, float eps, int cn,
+                                float* dn_out, float* delta_out) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = warp; i < T; i += THREADS / 32) {
+        const float dn = nd[i * dm.MS + dm.M] + eps;
+        const float inv = i < cn ? 1.f / dn : 0.f;
+        float go = 0.f;
+        for (int e = lane; e < dm.M; e += 32) {
+            const float gi = g[i * dm.MS + e];
+            go = fmaf(gi, nd[i * dm.MS + e] * inv, go);
+            g[i * dm.MS + e] = gi * inv;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) go += __shfl_xor_sync(0xffffffffu, go, off);
+        if (lane == 0) {
+            const float delta = -go * inv;
+            g[i * dm.MS + dm.M] = delta;
+            if (dn_out && i < cn) { dn_out[i] = dn; delta_out[i] = delta; }
+        }
+    }
+}
+
+// dP[i][j] = Gt_i . Vt_j for j <= i (causal) else 0.
+__device__ void masked_dscores(float* dP, const float* gt, const float* vt, const Dims& dm) {
+    for (int idx = threadIdx.x; idx < T * T; idx += THREADS) {
+        const int i = idx / T, j = idx - i * T;
+        float s = 0.f;
+        if (j <= i)
+            for (int e = 0; e < dm.MS; ++e) s = fmaf(gt[i * dm.MS + e], vt[j * dm.MS + e], s);
+        dP[i * (T + 1) + j] = s;
+    }
+}
+
+size_t smem_floats_forward(int D, int M) {
+    return (size_t)2 * T * (D + 1) + (size_t)2 * T * (M + 1) + (size_t)D * (M + 1) + (size_t)T * (T + 1);
+}
+size_t smem_floats_backward(int D, int M) {
+    return (size_t)2 * T * (D + 1) + (size_t)3 * T * (M + 1) + (size_t)D * (M + 1) + (size_t)2 * T * (T + 1);
+}
+
+// ---------------------------------------------------------------------------
+// Causal forward: one CTA walks one (batch, head) sequence chunk by chunk.
+// ---------------------------------------------------------------------------
+template <typename IO>
+__global__ void __launch_bounds__(THREADS)
+general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K, const IO* __restrict__ V,
+                              IO* __restrict__ O, float* __restrict__ den, float* __restrict__ S_out,
+                              float* __restrict__ Z_out, int64_t N, int D, int M, float eps, int phi) {
+    extern __shared__ float smem[];
+    const Dims dm = make_dims(D, M);
+    float* sq = smem;
+    float* sk = sq + T * dm.DS;
+    float* sv = sk + T * dm.DS;
+    float* snd = sv + T * dm.MS;
+    float* sSt = snd + T * dm.MS;
+    float* sP = sSt + D * dm.MS;
+
+    const int64_t bh = blockIdx.x;
+    Q += bh * N * D; K += bh * N * D; V += bh * N * M; O += bh * N * M;
+    zero_fill(sSt, D * dm.MS);
+
+    for (int64_t n0 = 0; n0 < N; n0 += T) {
+        const int cn = (int)((N - n0) < T ? (N - n0) : T);
+        __syncthreads();
+        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
+        load_mapped<IO>(sk, K + n0 * D, cn, D, dm.DS, phi);
+        load_values_ext<IO>(sv, V + n0 * M, cn, M, dm.MS);
+        __syncthreads();
+        masked_scores(sP, sq, sk, D, dm.DS);
+        __syncthreads();
+        numerator_denominator(snd, sP, sv, sq, sSt, dm, true);
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < cn * M; idx += THREADS) {
+            const int i = idx / M, e = idx - i * M;
+            O[(n0 + i) * M + e] = from_f32<IO>(snd[i * dm.MS + e] / (snd[i * dm.MS + M] + eps));
+        }
+        if (den)
+            for (int i = threadIdx.x; i < cn; i += THREADS) den[bh * N + n0 + i] = snd[i * dm.MS + M];
+        state_update(sSt, sk, sv, dm);
+    }
+    __syncthreads();
+    if (S_out)
+        for (int idx = threadIdx.x; idx < D * M; idx += THREADS)
+            S_out[bh * D * M + idx] = sSt[(idx / M) * dm.MS + idx % M];
+    if (Z_out)
+        for (int d = threadIdx.x; d < D; d += THREADS) Z_out[bh * D + d] = sSt[d * dm.MS + M];
+}
+
+// ---------------------------------------------------------------------------
+// Causal backward: forward sweep (grad Q, Eq. 13) then reverse sweep (grad K,
+// grad V, Eq. 14-15) by the same CTA.  The per-position scalars dn_i and
+// delta_i found in the forward sweep are parked in `aux` ([B,H,N,2] fp32) for
+// the reverse sweep; no per-position state is stored.
+// ---------------------------------------------------------------------------
+template <typename IO>
+__global__ void __launch_bounds__(THREADS)
+general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K, const IO* __restrict__ V,
+                               const IO* __restrict__ G, IO* __restrict__ dQ, IO* __restrict__ dK,
+                               IO* __restrict__ dV, float* __restrict__ aux,
+                               int64_t N, int D, int M, float eps, int phi) {
+    extern __shared__ float smem[];
+    const Dims dm = make_dims(D, M);
+    float* sq = smem;
+    float* sk = sq + T * dm.DS;
+    float* sv = sk + T * dm.DS;
+    float* sg = sv + T * dm.MS;
+    float* snd = sg + T * dm.MS;
+    float* sSt = snd + T * dm.MS;
+    float* sP = sSt + D * dm.MS;
+    float* sdP = sP + T * (T + 1);
+
+    const int64_t bh = blockIdx.x;
+    Q += bh * N * D; K += bh * N * D; V += bh * N * M; G += bh * N * M;
+    dQ += bh * N * D; dK += bh * N * D; dV += bh * N * M;
+    float* dn_all = aux + bh * N * 2;
+    float* delta_all = dn_all + N;
+
+    // ---- forward sweep: St = running sum of phi(K_j) Vt_j^T -------------------
+    zero_fill(sSt, D * dm.MS);
+    for (int64_t n0 = 0; n0 < N; n0 += T) {
+        const int cn = (int)((N - n0) < T ? (N - n0) : T);
+        __syncthreads();
+        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
+        load_mapped<IO>(sk, K + n0 * D, cn, D, dm.DS, phi);
+        load_values_ext<IO>(sv, V + n0 * M, cn, M, dm.MS);
+        load_values_ext<IO>(sg, G + n0 * M, cn, M, dm.MS);
+        __syncthreads();
+        masked_scores(sP, sq, sk, D, dm.DS);
+        __syncthreads();
+        numerator_denominator(snd, sP, sv, sq, sSt, dm, true);
+        __syncthreads();
+        extend_upstream(sg, snd, dm, eps, cn, dn_all + n0, delta_all + n0);
+        __syncthreads();
+        masked_dscores(sdP, sg, sv, dm);
+        __syncthreads();
+        // grad phi(Q_i) = sum_{j<=i} dP_ij k_j + St_{c-1} Gt_i
+        for (int idx = threadIdx.x; idx < cn * D; idx += THREADS) {
+            const int i = idx / D, d = idx - i * D;
+            float s = 0.f;
+            for (int j = 0; j <= i; ++j) s = fmaf(sdP[i * (T + 1) + j], sk[j * dm.DS + d], s);
+            for (int e = 0; e < dm.MS; ++e) s = fmaf(sSt[d * dm.MS + e], sg[i * dm.MS + e], s);
+            dQ[(n0 + i) * D + d] = from_f32<IO>(s * phi_slope_from_value(sq[i * dm.DS + d], phi));
+        }
+        __syncthreads();
+        state_update(sSt, sk, sv, dm);
+    }
+
+    // ---- reverse sweep: Rt = running sum (from the end) of phi(Q_j) Gt_j^T ----
+    __syncthreads();
+    zero_fill(sSt, D * dm.MS);
+    const int64_t nchunks = (N + T - 1) / T;
+    for (int64_t c = nchunks - 1; c >= 0; --c) {
+        const int64_t n0 = c * T;
+        const int cn = (int)((N - n0) < T ? (N - n0) : T);
+        __syncthreads();
+        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
+        load_mapped<IO>(sk, K + n0 * D, cn, D, dm.DS, phi);
+        load_values_ext<IO>(sv, V + n0 * M, cn, M, dm.MS);
+        for (int idx = threadIdx.x; idx < T * dm.MS; idx += THREADS) {
+            const int i = idx / dm.MS, e = idx - i * dm.MS;
+            float x = 0.f;
+            if (i < cn)
+                x = e < M ? to_f32<IO>(G[(n0 + i) * M + e]) / dn_all[n0 + i] : delta_all[n0 + i];
+            sg[idx] = x;
+        }
+        __syncthreads();
+        masked_scores(sP, sq, sk, D, dm.DS);
+        masked_dscores(sdP, sg, sv, dm);
+        __syncthreads();
+        // grad phi(K_j) = sum_{i>=j} dP_ij q_i + Rt_{c+1} Vt_j          (Eq. 14)
+        for (int idx = threadIdx.x; idx < cn * D; idx += THREADS) {
+            const int j = idx / D, d = idx - j * D;
+            float s = 0.f;
+            for (int i = j; i < T; ++i) s = fmaf(sdP[i * (T + 1) + j], sq[i * dm.DS + d], s);
+            for (int e = 0; e < dm.MS; ++e) s = fmaf(sSt[d * dm.MS + e], sv[j * dm.MS + e], s);
+            dK[(n0 + j) * D + d] = from_f32<IO>(s * phi_slope_from_value(sk[j * dm.DS + d], phi));
+        }
+        // grad V_j = sum_{i>=j} P_ij Gt_i[0:M] + Rt_{c+1}^T k_j          (Eq. 15)
+        for (int idx = threadIdx.x; idx < cn * M; idx += THREADS) {
+            const int j = idx / M, e = idx - j * M;
+            float s = 0.f;
+            for (int i = j; i < T; ++i) s = fmaf(sP[i * (T + 1) + j], sg[i * dm.MS + e], s);
+            for (int d = 0; d < D; ++d) s = fmaf(sSt[d * dm.MS + e], sk[j * dm.DS + d], s);
+            dV[(n0 + j) * M + e] = from_f32<IO>(s);
+        }
+        __syncthreads();
+        state_update(sSt, sq, sg, dm);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Non-causal pieces (Eq. 5-6): a split-parallel sum of x_i yt_i^T and per-token
+// apply kernels that read the reduced sums.
+// ---------------------------------------------------------------------------
+struct Split { int nsplit; int64_t len; };
+
+Split choose_split(const la_problem& p) {
+    int64_t bh = p.B * p.H;
+    int64_t want = (2 * 148 + bh - 1) / bh;                // about two CTAs per SM in total
+    int64_t maxs = (p.N + 4 * T - 1) / (4 * T);            // at least four chunks per split
+    if (maxs < 1) maxs = 1;
+    if (want > maxs) want = maxs;
+    if (want < 1) want = 1;
+    if (want > 64) want = 64;
+    int64_t len = (p.N + want - 1) / want;
+    len = (len + T - 1) / T * T;
+    int64_t ns = len > 0 ? (p.N + len - 1) / len : 1;
+    if (ns < 1) ns = 1;
+    return Split{(int)ns, len};
+}
+
+// part[bh][split] = sum over the split's positions of phi(X_i) [Y_i, 1]^T.
+template <typename IO>
+__global__ void __launch_bounds__(THREADS)
+general_kv_sum_kernel(const IO* __restrict__ X, const IO* __restrict__ Y, float* __restrict__ part,
+                      int64_t N, int64_t split_len, int D, int M, int phi) {
+    extern __shared__ float smem[];
+    const Dims dm = make_dims(D, M);
+    float* sx = smem;
+    float* sy = sx + T * dm.DS;
+    float* sSt = sy + T * dm.MS;
+    const int64_t bh = blockIdx.x, sp = blockIdx.y;
+    const int64_t lo = sp * split_len, hi = (lo + split_len) < N ? (lo + split_len) : N;
+    X += bh * N * D; Y += bh * N * M;
+    zero_fill(sSt, D * dm.MS);
+    for (int64_t n0 = lo; n0 < hi; n0 += T) {
+        const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
+        __syncthreads();
+        load_mapped<IO>(sx, X + n0 * D, cn, D, dm.DS, phi);
+        load_values_ext<IO>(sy, Y + n0 * M, cn, M, dm.MS);
+        __syncthreads();
+        state_update(sSt, sx, sy, dm);
+    }
+    __syncthreads();
+    float* dst = part + (bh * gridDim.y + sp) * (int64_t)(D * dm.MS);
+    for (int idx = threadIdx.x; idx < D * dm.MS; idx += THREADS) dst[idx] = sSt[idx];
+}
+
+__device__ void load_reduced_state(float* sSt, const float* part, int nsplit, int n) {
+    for (int idx = threadIdx.x; idx < n; idx += THREADS) {
+        float s = 0.f;
+        for (int sp = 0; sp < nsplit; ++sp) s += part[(int64_t)sp * n + idx];
+        sSt[idx] = s;
+    }
+}
+
+template <typename IO>
+__global__ void __launch_bounds__(THREADS)
+general_linear_apply_kernel(const IO* __restrict__ Q, const float* __restrict__ part, IO* __restrict__ O,
+                            float* __restrict__ den, float* __restrict__ KV, float* __restrict__ Zs,
+                            int nsplit, int64_t N, int64_t split_len, int D, int M, float eps, int phi) {
+    extern __shared__ float smem[];
+    const Dims dm = make_dims(D, M);
+    float* sq = smem;
+    float* snd = sq + T * dm.DS;
+    float* sSt = snd + T * dm.MS;
+    const int64_t bh = blockIdx.x, sp = blockIdx.y;
+    const int64_t lo = sp * split_len, hi = (lo + split_len) < N ? (lo + split_len) : N;
+    Q += bh * N * D; O += bh * N * M;
+    load_reduced_state(sSt, part + bh * nsplit * (int64_t)(D * dm.MS), nsplit, D * dm.MS);
+    __syncthreads();
+    if (sp == 0) {
+        if (KV)
+            for (int idx = threadIdx.x; idx < D * M; idx += THREADS)
+                KV[bh * D * M + idx] = sSt[(idx / M) * dm.MS + idx % M];
+        if (Zs)
+            for (int d = threadIdx.x; d < D; d += THREADS) Zs[bh * D + d] = sSt[d * dm.MS + M];
+    }
+    for (int64_t n0 = lo; n0 < hi; n0 += T) {
+        const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
+        __syncthreads();
+        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
+        __syncthreads();
+        numerator_denominator(snd, nullptr, nullptr, sq, sSt, dm, false);
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < cn * M; idx += THREADS) {
+            const int i = idx / M, e = idx - i * M;
+            O[(n0 + i) * M + e] = from_f32<IO>(snd[i * dm.MS + e] / (snd[i * dm.MS + M] + eps));
+        }
+        if (den)
+            for (int i = threadIdx.x; i < cn; i += THREADS) den[bh * N + n0 + i] = snd[i * dm.MS + M];
+    }
+}
+
+// Backward, query side: with St = full sum, form Gt_i, write
+// grad phi(Q_i) = St Gt_i (Eq. 13 with the full sum) and accumulate this split's
+// part of Rt = sum_i phi(Q_i) Gt_i^T.
+template <typename IO>
+__global__ void __launch_bounds__(THREADS)
+general_linear_bwd_q_kernel(const IO* __restrict__ Q, const IO* __restrict__ G,
+                            const float* __restrict__ part_s, IO* __restrict__ dQ,
+                            float* __restrict__ part_r, int nsplit, int64_t N, int64_t split_len,
+                            int D, int M, float eps, int phi) {
+    extern __shared__ float smem[];
+    const Dims dm = make_dims(D, M);
+    float* sq = smem;
+    float* sg = sq + T * dm.DS;
+    float* snd = sg + T * dm.MS;
+    float* sSt = snd + T * dm.MS;
+    float* sRt = sSt + D * dm.MS;
+    const int64_t bh = blockIdx.x, sp = blockIdx.y;
+    const int64_t lo = sp * split_len, hi = (lo + split_len) < N ? (lo + split_len) : N;
+    Q += bh * N * D; G += bh * N * M; dQ += bh * N * D;
+    load_reduced_state(sSt, part_s + bh * nsplit * (int64_t)(D * dm.MS), nsplit, D * dm.MS);
+    zero_fill(sRt, D * dm.MS);
+    for (int64_t n0 = lo; n0 < hi; n0 += T) {
+        const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
+        __syncthreads();
+        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
+        load_values_ext<IO>(sg, G + n0 * M, cn, M, dm.MS);
+        __syncthreads();
+        numerator_denominator(snd, nullptr, nullptr, sq, sSt, dm, false);
+        __syncthreads();
+        extend_upstream(sg, snd, dm, eps, cn, nullptr, nullptr);
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < cn * D; idx += THREADS) {
+            const int i = idx / D, d = idx - i * D;
+            float s = 0.f;
+            for (int e = 0; e < dm.MS; ++e) s = fmaf(sSt[d * dm.MS + e], sg[i * dm.MS + e], s);
+            dQ[(n0 + i) * D + d] = from_f32<IO>(s * phi_slope_from_value(sq[i * dm.DS + d], phi));
+        }
+        state_update(sRt, sq, sg, dm);
+    }
+    __syncthreads();
+    float* dst = part_r + (bh * gridDim.y + sp) * (int64_t)(D * dm.MS);
+    for (int idx = threadIdx.x; idx < D * dm.MS; idx += THREADS) dst[idx] = sRt[idx];
+}
+
+// Backward, key/value side: grad phi(K_j) = Rt Vt_j (Eq. 14), grad V_j = (Rt^T phi(K_j))[0:M] (Eq. 15).
+template <typename IO>
+__global__ void __launch_bounds__(THREADS)
+general_linear_bwd_kv_kernel(const IO* __restrict__ K, const IO* __restrict__ V,
+                             const float* __restrict__ part_r, IO* __restrict__ dK, IO* __restrict__ dV,
+                             int nsplit, int64_t N, int64_t split_len, int D, int M, int phi) {
+    extern __shared__ float smem[];
+    const Dims dm = make_dims(D, M);
+    float* sk = smem;
+    float* sv = sk + T * dm.DS;
+    float* sRt = sv + T * dm.MS;
+    const int64_t bh = blockIdx.x, sp = blockIdx.y;
+    const int64_t lo = sp * split_len, hi = (lo + split_len) < N ? (lo + split_len) : N;
+    K += bh * N * D; V += bh * N * M; dK += bh * N * D; dV += bh * N * M;
+    load_reduced_state(sRt, part_r + bh * nsplit * (int64_t)(D * dm.MS), nsplit, D * dm.MS);
+    for (int64_t n0 = lo; n0 < hi; n0 += T) {
+        const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
+        __syncthreads();
+        load_mapped<IO>(sk, K + n0 * D, cn, D, dm.DS, phi);
+        load_values_ext<IO>(sv, V + n0 * M, cn, M, dm.MS);
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < cn * D; idx += THREADS) {
+            const int j = idx / D, d = idx - j * D;
+            float s = 0.f;
+            for (int e = 0; e < dm.MS; ++e) s = fmaf(sRt[d * dm.MS + e], sv[j * dm.MS + e], s);
+            dK[(n0 + j) * D + d] = from_f32<IO>(s * phi_slope_from_value(sk[j * dm.DS + d], phi));
+        }
+        for (int idx = threadIdx.x; idx < cn * M; idx += THREADS) {
+            const int j = idx / M, e = idx - j * M;
+            float s = 0.f;
+            for (int d = 0; d < D; ++d) s = fmaf(sRt[d * dm.MS + e], sk[j * dm.DS + d], s);
+            dV[(n0 + j) * M + e] = from_f32<IO>(s);
+        }
+    }
+}
+
+template <typename Kern>
+int opt_in_smem(Kern kern, size_t bytes) {
+    if (bytes > 48 * 1024)
+        LA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    return LA_OK;
+}
+
+size_t state_floats(const la_problem& p) { return (size_t)p.D * (p.M + 1); }
+
+}  // namespace
+
+size_t general_workspace_bytes(const la_problem& p, int op) {
+    const size_t bh = (size_t)(p.B * p.H);
+    switch (op) {
+        case LA_OP_CAUSAL_FORWARD: return 0;
+        case LA_OP_CAUSAL_BACKWARD: return bh * (size_t)p.N * 2 * sizeof(float);
+        case LA_OP_LINEAR_FORWARD: return bh * choose_split(p).nsplit * state_floats(p) * sizeof(float);
+        case LA_OP_LINEAR_BACKWARD: return 2 * bh * choose_split(p).nsplit * state_floats(p) * sizeof(float);
+        default: return 0;
+    }
+}
+
+template <typename IO>
+static int causal_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
+                            float* den, float* S_out, float* Z_out, cudaStream_t st) {
+    const size_t smem = smem_floats_forward((int)p.D, (int)p.M) * sizeof(float);
+    auto kern = general_causal_forward_kernel<IO>;
+    if (int rc = opt_in_smem(kern, smem)) return rc;
+    kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, (IO*)O, den,
+                                                       S_out, Z_out, p.N, (int)p.D, (int)p.M, p.eps, p.phi);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
+                           float* den, float* S_out, float* Z_out, cudaStream_t st) {
+    return p.dtype == LA_F32 ? causal_forward_t<float>(p, Q, K, V, O, den, S_out, Z_out, st)
+                             : causal_forward_t<__nv_bfloat16>(p, Q, K, V, O, den, S_out, Z_out, st);
+}
+
+template <typename IO>
+static int causal_backward_t(const la_problem& p, const void* Q, const void* K, const void* V,
+                             const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    const size_t smem = smem_floats_backward((int)p.D, (int)p.M) * sizeof(float);
+    auto kern = general_causal_backward_kernel<IO>;
+    if (int rc = opt_in_smem(kern, smem)) return rc;
+    kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, (const IO*)G,
+                                                       (IO*)dQ, (IO*)dK, (IO*)dV, (float*)ws, p.N, (int)p.D,
+                                                       (int)p.M, p.eps, p.phi);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+                            void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    return p.dtype == LA_F32 ? causal_backward_t<float>(p, Q, K, V, G, dQ, dK, dV, ws, st)
+                             : causal_backward_t<__nv_bfloat16>(p, Q, K, V, G, dQ, dK, dV, ws, st);
+}
+
+template <typename IO>
+static int linear_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
+                            float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
+    const int D = (int)p.D, M = (int)p.M;
+    const Split sp = choose_split(p);
+    const dim3 grid((unsigned)(p.B * p.H), (unsigned)sp.nsplit);
+    float* part = (float*)ws;
+    {
+        const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
+        auto kern = general_kv_sum_kernel<IO>;
+        if (int rc = opt_in_smem(kern, smem)) return rc;
+        kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part, p.N, sp.len, D, M, p.phi);
+        LA_LAUNCHED();
+    }
+    {
+        const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
+        auto kern = general_linear_apply_kernel<IO>;
+        if (int rc = opt_in_smem(kern, smem)) return rc;
+        kern<<<grid, THREADS, smem, st>>>((const IO*)Q, part, (IO*)O, den, KV, Zs, sp.nsplit, p.N, sp.len, D, M,
+                                          p.eps, p.phi);
+        LA_LAUNCHED();
+    }
+    return LA_OK;
+}
+
+int general_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
+                           float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
+    return p.dtype == LA_F32 ? linear_forward_t<float>(p, Q, K, V, O, den, KV, Zs, ws, st)
+                             : linear_forward_t<__nv_bfloat16>(p, Q, K, V, O, den, KV, Zs, ws, st);
+}
+
+template <typename IO>
+static int linear_backward_t(const la_problem& p, const void* Q, const void* K, const void* V,
+                             const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    const int D = (int)p.D, M = (int)p.M;
+    const Split sp = choose_split(p);
+    const dim3 grid((unsigned)(p.B * p.H), (unsigned)sp.nsplit);
+    float* part_s = (float*)ws;
+    float* part_r = part_s + (size_t)(p.B * p.H) * sp.nsplit * state_floats(p);
+    {
+        const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
+        auto kern = general_kv_sum_kernel<IO>;
+        if (int rc = opt_in_smem(kern, smem)) return rc;
+        kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part_s, p.N, sp.len, D, M, p.phi);
+        LA_LAUNCHED();
+    }
+    {
+        const size_t smem = ((size_t)T * (D + 1) + (size_t)2 * T * (M + 1) + 2 * state_floats(p)) * sizeof(float);
+        auto kern = general_linear_bwd_q_kernel<IO>;
+        if (int rc = opt_in_smem(kern, smem)) return rc;
+        kern<<<grid, THREADS, smem, st>>>((const IO*)Q, (const IO*)G, part_s, (IO*)dQ, part_r, sp.nsplit, p.N,
+                                          sp.len, D, M, p.eps, p.phi);
+        LA_LAUNCHED();
+    }
+    {
+        const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
+        auto kern = general_linear_bwd_kv_kernel<IO>;
+        if (int rc = opt_in_smem(kern, smem)) return rc;
+        kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part_r, (IO*)dK, (IO*)dV, sp.nsplit, p.N,
+                                          sp.len, D, M, p.phi);
+        LA_LAUNCHED();
+    }
+    return LA_OK;
+}
+
+int general_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+                            void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    return p.dtype == LA_F32 ? linear_backward_t<float>(p, Q, K, V, G, dQ, dK, dV, ws, st)
+                             : linear_backward_t<__nv_bfloat16>(p, Q, K, V, G, dQ, dK, dV, ws, st);
+}
+
+}  // namespace la

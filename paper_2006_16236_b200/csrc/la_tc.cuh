@@ -1,0 +1,20 @@
+// Tensor-core (tcgen05 / TMA) kernels for bf16 problems: interface to the API layer.
+#pragma once
+#include "la_common.cuh"
+
+namespace la {
+
+// True when problem p / operation op runs on the tensor-core kernels.
+bool tc_supported(const la_problem& p, int op);
+size_t tc_workspace_bytes(const la_problem& p, int op);
+
+int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
+                      float* den, float* S_out, float* Z_out, void* ws, cudaStream_t st);
+int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+                       void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
+                      float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
+int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+                       void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+
+}  // namespace la

@@ -1,0 +1,226 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2006_16236_b200 as la
+from paper_2006_16236_b200.inputs import WORKLOADS, draw_qkvg, draw_workload
+from parity import assert_close
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def gpu(*ts):
+    return [None if t is None else t.to(DEV) for t in ts]
+
+
+# shapes: (B, H, N, D, M); chosen to span several chunks and a ragged tail, N < chunk, D != M
+SHAPES = [(1, 2, 256, 32, 32), (2, 3, 100, 16, 48), (1, 1, 1, 8, 8), (1, 2, 31, 64, 64),
+          (2, 2, 33, 24, 40), (1, 2, 517, 128, 128), (1, 4, 384, 64, 64), (2, 2, 640, 32, 32)]
+DTYPES = [torch.float32, torch.bfloat16]
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 1000, 65536 + 3])
+def test_feature_map(dtype, n):
+    x = (torch.randn(n, generator=torch.Generator().manual_seed(n)) * 3).to(dtype)
+    for deriv in (False, True):
+        y = la.la_feature_map(x.to(DEV), deriv=deriv)
+        assert_close(y, oracle.feature_map(x, deriv), dtype, "feature map")
+    if n:
+        xi = x.to(DEV)
+        la.la_feature_map(xi, out=xi)                       # in place
+        assert_close(xi, oracle.feature_map(x), dtype, "feature map in place")
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", SHAPES)
+def test_causal_forward_backward(shape, dtype):
+    B, H, N, D, M = shape
+    Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=sum(shape), dtype=dtype)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    den = torch.empty((B, H, N), device=DEV)
+    S = torch.empty((B, H, D, M), device=DEV)
+    Z = torch.empty((B, H, D), device=DEV)
+    O = la.la_causal_forward(Qd, Kd, Vd, den=den, S_out=S, Z_out=Z)
+    Or, denr, Sr, Zr = oracle.linear_attention(Q, K, V, True, return_state=True)
+    assert_close(O, Or, dtype, "O")
+    assert_close(den, denr, dtype, "den")
+    assert_close(S, Sr, dtype, "S_N")
+    assert_close(Z, Zr, dtype, "Z_N")
+    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd)
+    rq, rk, rv = oracle.linear_attention_backward(Q, K, V, G, True)
+    assert_close(dQ, rq, dtype, "dQ")
+    assert_close(dK, rk, dtype, "dK")
+    assert_close(dV, rv, dtype, "dV")
+    la.la_last_device_status()
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", SHAPES)
+def test_noncausal_forward_backward(shape, dtype):
+    B, H, N, D, M = shape
+    Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=1 + sum(shape), dtype=dtype, scale=0.5)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    den = torch.empty((B, H, N), device=DEV)
+    KV = torch.empty((B, H, D, M), device=DEV)
+    Zs = torch.empty((B, H, D), device=DEV)
+    O = la.la_linear_attention(Qd, Kd, Vd, den=den, KV=KV, Zs=Zs)
+    Or, denr, Sr, Zr = oracle.linear_attention(Q, K, V, False, return_state=True)
+    assert_close(O, Or, dtype, "O")
+    assert_close(den, denr, dtype, "den")
+    assert_close(KV, Sr, dtype, "KV")
+    assert_close(Zs, Zr, dtype, "Zs")
+    dQ, dK, dV = la.la_linear_attention_backward(Qd, Kd, Vd, Gd)
+    rq, rk, rv = oracle.linear_attention_backward(Q, K, V, G, False)
+    assert_close(dQ, rq, dtype, "dQ")
+    assert_close(dK, rk, dtype, "dK")
+    assert_close(dV, rv, dtype, "dV")
+    la.la_last_device_status()
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_eps_and_identity_feature_map(causal, dtype):
+    B, H, N, D, M = 2, 2, 96, 32, 16
+    Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=77, dtype=torch.float32)
+    Q, K = (Q.abs() + 0.1).to(dtype), (K.abs() + 0.1).to(dtype)      # already "feature-mapped"
+    V, G = V.to(dtype), G.to(dtype)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    fwd = la.la_causal_forward if causal else la.la_linear_attention
+    bwd = la.la_causal_backward if causal else la.la_linear_attention_backward
+    O = fwd(Qd, Kd, Vd, phi="identity", eps=0.75)
+    assert_close(O, oracle.linear_attention(Q, K, V, causal, "identity", 0.75)[0], dtype, "O")
+    grads = bwd(Qd, Kd, Vd, Gd, phi="identity", eps=0.75)
+    for g, r, nm in zip(grads, oracle.linear_attention_backward(Q, K, V, G, causal, "identity", 0.75), "QKV"):
+        assert_close(g, r, dtype, "d" + nm)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", [(2, 3, 40, 64, 64), (1, 2, 24, 32, 32), (2, 2, 17, 16, 24), (1, 2, 9, 128, 64)])
+def test_recurrent_steps_equal_causal_form(shape, dtype):
+    B, H, N, D, M = shape
+    Q, K, V, _ = draw_qkvg(B, H, N, D, M, seed=5 + sum(shape), dtype=dtype, with_grad=False)
+    Qd, Kd, Vd = gpu(Q, K, V)
+    ref = oracle.attention_quadratic(Q, K, V, True)
+    S = torch.zeros((B, H, D, M), device=DEV)
+    Z = torch.zeros((B, H, D), device=DEV)
+    So, Zo = np.zeros((B, H, D, M)), np.zeros((B, H, D))
+    outs = []
+    for i in range(N):
+        out = la.la_recurrent_step(Qd[:, :, i].contiguous(), Kd[:, :, i].contiguous(), Vd[:, :, i].contiguous(), S, Z)
+        step_ref = oracle.recurrent_step(Q[:, :, i], K[:, :, i], V[:, :, i], So, Zo)
+        assert_close(out, step_ref, dtype, f"step {i}")
+        outs.append(out)
+    assert_close(torch.stack(outs, 2), ref, dtype, "steps vs quadratic form")
+    assert_close(S, So, dtype, "S")
+    assert_close(Z, Zo, dtype, "Z")
+    # the parallel form on the same sequence, and its final state, agree with the steps
+    S2 = torch.empty_like(S)
+    Z2 = torch.empty_like(Z)
+    O = la.la_causal_forward(Qd, Kd, Vd, S_out=S2, Z_out=Z2)
+    assert_close(O, torch.stack(outs, 2).double().cpu().numpy(), dtype, "parallel vs steps")
+    assert_close(S2, So, dtype, "S_N of the parallel form")
+
+
+def test_prefill_then_decode_handoff():
+    B, H, N, D, M = 2, 2, 64, 32, 32
+    Q, K, V, _ = draw_qkvg(B, H, N + 1, D, M, seed=9, dtype=torch.float32, with_grad=False)
+    Qd, Kd, Vd = gpu(Q, K, V)
+    S = torch.empty((B, H, D, M), device=DEV)
+    Z = torch.empty((B, H, D), device=DEV)
+    la.la_causal_forward(Qd[:, :, :N].contiguous(), Kd[:, :, :N].contiguous(), Vd[:, :, :N].contiguous(),
+                         S_out=S, Z_out=Z)
+    out = la.la_recurrent_step(Qd[:, :, N].contiguous(), Kd[:, :, N].contiguous(), Vd[:, :, N].contiguous(), S, Z)
+    ref = oracle.attention_quadratic(Q, K, V, True)[:, :, N]
+    assert_close(out, ref, torch.float32, "decode after prefill")
+
+
+def test_gradient_invariants_hold_on_gpu_results():
+    B, H, N, D, M = 2, 4, 512, 64, 64
+    Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=11, dtype=torch.float32)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    for bwd in (la.la_causal_backward, la.la_linear_attention_backward):
+        dQ, dK, dV = bwd(Qd, Kd, Vd, Gd)
+        assert torch.allclose(dV.sum(2), Gd.sum(2), rtol=1e-3, atol=1e-3)           # rows sum to one
+        ratio = torch.where(Qd > 0, Qd + 1, torch.ones_like(Qd))                    # phi / phi'
+        assert (ratio * dQ).sum(-1).abs().max() < 1e-3                              # degree-0 in phi(Q_i)
+
+
+# --------------------------------------------------------------------------
+# Full-size workloads, in the launch configuration the benchmark times; the
+# oracle recomputes a sample of (batch, head) pairs, which are independent.
+# --------------------------------------------------------------------------
+def _sample_heads(B, H, k=3):
+    pairs = [(0, 0), (B - 1, H - 1), (B // 2, H // 2)]
+    return list(dict.fromkeys(pairs))[:k]
+
+
+@pytest.mark.parametrize("name", ["causal_fp32_small", "causal_bf16_image", "causal_sweep_bf16_N4096",
+                                  "causal_sweep_bf16_N8192", "causal_sweep_bf16_N16384",
+                                  "causal_sweep_bf16_N32768", "causal_sweep_bf16_N65536"])
+def test_causal_workloads_full_size(name):
+    w = WORKLOADS[name]
+    dtype = w.torch_dtype
+    Q, K, V, G = draw_workload(w)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    den = torch.empty((w.B, w.H, w.N), device=DEV)
+    O = la.la_causal_forward(Qd, Kd, Vd, den=den)
+    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd, O=O, den=den)
+    la.la_last_device_status()
+    for b, h in _sample_heads(w.B, w.H):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        q, k, v, g = Q[sl], K[sl], V[sl], G[sl]
+        Or, denr = oracle.linear_attention(q, k, v, True)
+        assert_close(O[sl], Or, dtype, f"{name} O[{b},{h}]")
+        assert_close(den[sl], denr, dtype, f"{name} den[{b},{h}]")
+        for got, ref, nm in zip((dQ, dK, dV), oracle.linear_attention_backward(q, k, v, g, True), "QKV"):
+            assert_close(got[sl], ref, dtype, f"{name} d{nm}[{b},{h}]")
+    # size-independent properties on the whole result
+    assert torch.isfinite(O.float()).all() and torch.isfinite(dQ.float()).all()
+    assert torch.allclose(O[:, :, 0].float(), Vd[:, :, 0].float(), rtol=1e-2, atol=1e-2)     # O_1 = V_1
+    assert torch.allclose(dV.float().sum(2), Gd.float().sum(2), rtol=5e-2, atol=0.5 * (w.N ** 0.5) * 2e-2 + 0.5)
+
+
+def test_noncausal_workload_full_size():
+    w = WORKLOADS["noncausal_bf16_speech"]
+    dtype = w.torch_dtype
+    Q, K, V, G = draw_workload(w)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    O = la.la_linear_attention(Qd, Kd, Vd)
+    dQ, dK, dV = la.la_linear_attention_backward(Qd, Kd, Vd, Gd)
+    la.la_last_device_status()
+    for b, h in _sample_heads(w.B, w.H):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        q, k, v, g = Q[sl], K[sl], V[sl], G[sl]
+        assert_close(O[sl], oracle.linear_attention(q, k, v, False)[0], dtype, f"O[{b},{h}]")
+        for got, ref, nm in zip((dQ, dK, dV), oracle.linear_attention_backward(q, k, v, g, False), "QKV"):
+            assert_close(got[sl], ref, dtype, f"d{nm}[{b},{h}]")
+
+
+def test_decode_workload_full_size():
+    w = WORKLOADS["decode_bf16_streams"]
+    T = 3072
+    Q, K, V, _ = draw_workload(w)
+    # step-major copies, as a decoder would produce them: [T, B, H, D]
+    q_t, k_t, v_t = (t.permute(2, 0, 1, 3).contiguous().to(DEV) for t in (Q, K, V))
+    S = torch.zeros((w.B, w.H, w.D, w.M), device=DEV)
+    Z = torch.zeros((w.B, w.H, w.D), device=DEV)
+    outs = torch.empty((T, w.B, w.H, w.M), dtype=torch.bfloat16, device=DEV)
+    for t in range(T):
+        la.la_recurrent_step(q_t[t], k_t[t], v_t[t], S, Z, out=outs[t])
+    la.la_last_device_status()
+    outs = outs.permute(1, 2, 0, 3)                                   # [B, H, T, M]
+    for b, h in _sample_heads(w.B, w.H):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        Or, _, Sr, Zr = oracle.linear_attention(Q[sl], K[sl], V[sl], True, return_state=True)
+        assert_close(outs[sl], Or, torch.bfloat16, f"decode out[{b},{h}]")
+        assert_close(S[sl], Sr, torch.bfloat16, f"decode S[{b},{h}]")
+        assert_close(Z[sl], Zr, torch.bfloat16, f"decode Z[{b},{h}]")
+    # the parallel causal form of the same sequences gives the same outputs
+    bsub = slice(0, 8)
+    O = la.la_causal_forward(*(t[bsub].contiguous().to(DEV) for t in (Q, K, V)))
+    err = (O.float() - outs[bsub].float()).abs().max().item()
+    assert err < 0.05, err
