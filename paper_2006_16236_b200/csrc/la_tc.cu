@@ -1,14 +1,55 @@
-// Tensor-core kernels: dispatch (kernels are added per operation).
+// Tensor-core kernels: which problems they take, workspace sizes, tensor-map encoding.
+#include <stdlib.h>
+
 #include "la_tc.cuh"
+#include "la_tc_common.cuh"
 
 namespace la {
 
-bool tc_supported(const la_problem&, int) { return false; }
-size_t tc_workspace_bytes(const la_problem&, int) { return 0; }
+namespace tc {
 
-int tc_causal_forward(const la_problem&, const void*, const void*, const void*, void*, float*, float*,
-                      float*, void*, cudaStream_t) {
-    return fail(LA_ERR_UNSUPPORTED, "tensor-core causal forward not available");
+int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows) {
+    static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        LA_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+        if (qres != cudaDriverEntryPointSuccess || !fn)
+            return fail(LA_ERR_CUDA, "the driver does not export cuTensorMapEncodeTiled");
+        encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)kDim, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kDim * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kDim, box_rows};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                              elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(LA_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return LA_OK;
+}
+
+}  // namespace tc
+
+bool tc_supported(const la_problem& p, int op) {
+    static const bool disabled = getenv("LA_DISABLE_TC") != nullptr;
+    if (disabled) return false;
+    if (p.dtype != LA_BF16 || p.D != tc::kDim || p.M != tc::kDim) return false;
+    if (p.N < tc::kChunk || p.N % tc::kChunk) return false;
+    if (p.B * p.H * p.N >= (1LL << 31)) return false;          // TMA coordinates are 32-bit
+    return op == LA_OP_CAUSAL_FORWARD;
+}
+
+size_t tc_workspace_bytes(const la_problem& p, int op) {
+    switch (op) {
+        case LA_OP_CAUSAL_FORWARD: return tc::causal_forward_workspace(p);
+        default: return 0;
+    }
+}
+
+int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
+                      float* S_out, float* Z_out, void* ws, cudaStream_t st) {
+    return tc::causal_forward(p, Q, K, V, O, den, S_out, Z_out, ws, st);
 }
 int tc_causal_backward(const la_problem&, const void*, const void*, const void*, const void*, void*, void*,
                        void*, void*, cudaStream_t) {

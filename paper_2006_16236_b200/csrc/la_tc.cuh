@@ -17,4 +17,10 @@ int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const v
 int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
                        void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 
+namespace tc {
+size_t causal_forward_workspace(const la_problem& p);
+int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
+                   float* S_out, float* Z_out, void* ws, cudaStream_t st);
+}  // namespace tc
+
 }  // namespace la
