@@ -186,7 +186,7 @@ int la_causal_backward(const la_problem* p, const void* Q, const void* K, const 
     if (int rc = check_ws(p, LA_OP_CAUSAL_BACKWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_CAUSAL_BACKWARD)) return tc_causal_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
+    if (tc_supported(*p, LA_OP_CAUSAL_BACKWARD)) return tc_causal_backward(*p, Q, K, V, O, den, G, dQ, dK, dV, ws, st);
     return general_causal_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
 }
 

@@ -10,8 +10,8 @@ size_t tc_workspace_bytes(const la_problem& p, int op);
 
 int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
                       float* den, float* S_out, float* Z_out, void* ws, cudaStream_t st);
-int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
-                       void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* O,
+                       const float* den, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
                       float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
 int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
@@ -21,6 +21,9 @@ namespace tc {
 size_t causal_forward_workspace(const la_problem& p);
 int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
                    float* S_out, float* Z_out, void* ws, cudaStream_t st);
+size_t causal_backward_workspace(const la_problem& p);
+int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+                    void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 }  // namespace tc
 
 }  // namespace la

@@ -1,0 +1,757 @@
+// Causal linear attention backward on the tensor cores (bf16, D = M = 64).
+//
+// Eq. 13-15 / Algorithm 1 "backward" on the ones-extended values, chunked.  With
+// q = phi(Q_c), k = phi(K_c), dn_i = q_i . Z_i + eps, qh_i = q_i / dn_i,
+// dl_i = -(G_i . O_i) (so that the extended upstream gradient of the numerator is
+// [G_i, dl_i] / dn_i), L the lower-triangular mask, St = [S | Z] the forward running
+// state and Rt = [R | r] the reverse running sum of qh_j [G_j | dl_j]^T:
+//
+//   forward sweep  (kernel "dq"):   h   = ((G V^T) o L) k + G S_{c-1}^T
+//                                   gq  = (h - (q . h / dn) Z_i) / dn                 (Eq. 13)
+//                                   dl  = -(q . h) / dn,   St_c = St_{c-1} + k^T [V | 1]
+//   reverse sweep  (kernel "dkv"):  Ph  = (qh k^T) o L,   dP = (G V^T + dl 1^T) o L
+//                                   gk  = dP^T qh + V R_{c+1}^T + 1 r_{c+1}^T         (Eq. 14)
+//                                   gV  = Ph^T G + k R_{c+1}                          (Eq. 15)
+//                                   Rt_c = Rt_{c+1} + qh^T [G | dl]
+//   dQ = gq o phi'(Q),  dK = gk o phi'(K).
+// G and V enter every product exactly as given (no re-rounding); the division by dn
+// is carried by the query side, in fp32 or in the rounded qh.
+//
+// Every product runs on tcgen05 with fp32 accumulators in TMEM; the running states
+// stay in TMEM in fp32 and are re-rounded to a bf16 operand tile once per chunk.  No
+// per-position state is ever stored.  Sequences are cut into segments that run on
+// different SMs; a segment starts from the exclusive prefix (forward sweep) or suffix
+// (reverse sweep) of per-segment sums produced by a pre-pass and a scan.
+#include "la_tc.cuh"
+#include "la_tc_common.cuh"
+
+namespace la {
+namespace tc {
+
+using namespace sm100;
+
+namespace {
+
+// ===========================================================================
+// Forward sweep: dQ and delta.
+//
+// G_i . O_i is NOT taken from the stored (rounded) output.  With
+//     h_i = sum_{j<=i} (G_i . V_j) k_j        (intra-chunk MMA plus G_i S_{c-1}^T)
+// one has  G_i . O_i = (q_i . h_i) / dn_i  with  dn_i = q_i . Z_i + eps,  hence
+//     gq_i = (h_i - (q_i . h_i / dn_i) Z_i) / dn_i :
+// h_i projected so that q_i . gq_i = 0 (O is homogeneous of degree 0 in phi(Q_i)).
+// Taking the projection from the same rounded products as h keeps that cancellation
+// exact; a delta from the bf16 output loses several digits in the first rows, where
+// the two terms nearly cancel.  The per-row prefix Z_i = Z_{c-1} + sum_{j<=i in chunk} k_j
+// comes from one more MMA, T = L k with L the lower-triangular matrix of ones.  The
+// kernel needs neither the forward output nor its denominators, and hands dn_i and
+// dl_i = -(G_i . O_i) to the reverse sweep.
+// In the first chunk of a sequence a row has few keys and h_i is a difference of nearly
+// equal terms; there the scores are centred before rounding, dP_ij - m_i with
+// m_i = dP_i0, and m_i T_i is added back in fp32 (a row constant times the prefix sum).
+//
+// Warps 0-7: dP post-processing (two warps per TMEM quadrant), 8-11: state
+// conversion and dQ epilogue, 12-15: phi(K), 16: TMA, 17: MMA.
+// ===========================================================================
+constexpr int kDqStages = 3;
+constexpr int kDqThreads = 576;
+constexpr uint32_t kDqColDP = 0;       // 128
+constexpr uint32_t kDqColGt = 128;     // 2 x 64: gt of even / odd chunks
+constexpr uint32_t kDqColT = 256;      // 2 x 64: T = L k of even / odd chunks
+constexpr uint32_t kDqColS = 384;      // 64 + 16
+
+constexpr uint32_t kDqOffStage = 0;                                        // kDqStages x {K, V, G}
+constexpr uint32_t kDqOffDP = kDqOffStage + kDqStages * 3 * kTileBytes;    // 2 tiles
+constexpr uint32_t kDqOffL = kDqOffDP + 2 * kTileBytes;                    // 2 tiles: lower-triangular ones
+constexpr uint32_t kDqOffS = kDqOffL + 2 * kTileBytes;                     // bf16 S tile
+constexpr uint32_t kDqOffOnes = kDqOffS + kDim * 128;
+constexpr uint32_t kDqOffZ = kDqOffOnes + 1024;                            // fp32 [2][64]
+constexpr uint32_t kDqOffM = kDqOffZ + 512;                                // fp32 [128]: row offsets m_i of the first chunk
+constexpr uint32_t kDqOffBar = kDqOffM + 512;
+constexpr uint32_t kDqSmemBytes = kDqOffBar + 256 + 1024;
+
+struct DqBarriers {
+    uint64_t full[kDqStages], empty[kDqStages], mapped[kDqStages];
+    uint64_t dq_full[2], dq_drained[2];
+    uint64_t dp_full, dp_ready, s_full, state_ready;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct DqParams {
+    const __nv_bfloat16* Q;     // raw queries (phi and phi' in the epilogue)
+    float* dn;                  // out: dn_i = q_i . Z_i + eps per row, for the reverse sweep
+    float* dl;                  // out: dl_i = -(G_i . O_i) per row, for the reverse sweep
+    __nv_bfloat16* dQ;
+    const float* init;          // per (bh, seg) initial [S|Z] records or null
+    int* status;
+    int64_t N;
+    int chunks, chunks_per_seg, nseg;
+    float eps;
+    int phi;
+};
+
+__global__ void __launch_bounds__(kDqThreads, 1)
+causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
+                     const __grid_constant__ CUtensorMap mapG, const DqParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    DqBarriers* bars = reinterpret_cast<DqBarriers*>(smem + kDqOffBar);
+    float* sZ = reinterpret_cast<float*>(smem + kDqOffZ);
+    float* sM = reinterpret_cast<float*>(smem + kDqOffM);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int seg = blockIdx.x % prm.nseg;
+    const int64_t bh = blockIdx.x / prm.nseg;
+    const int c_begin = seg * prm.chunks_per_seg;
+    const int L = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
+    const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
+
+    if (tid == 0) {
+        for (int s = 0; s < kDqStages; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+            mbar_init(&bars->mapped[s], 128);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&bars->dq_full[b], 1);
+            mbar_init(&bars->dq_drained[b], 128);
+        }
+        mbar_init(&bars->dp_full, 1);
+        mbar_init(&bars->dp_ready, 256);
+        mbar_init(&bars->s_full, 1);
+        mbar_init(&bars->state_ready, 128);
+        bars->abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 17) {
+        __syncwarp();
+        tmem_alloc(&bars->tmem_base, 512);
+        tmem_relinquish();
+    }
+    // the score tile is zero right of the diagonal for ever: clear it once
+    for (uint32_t i = tid; i < 2 * kTileBytes / 16; i += kDqThreads) sts128(sbase + kDqOffDP + i * 16, 0u, 0u, 0u, 0u);
+    for (int i = tid; i < 256; i += kDqThreads) reinterpret_cast<uint32_t*>(smem + kDqOffOnes)[i] = 0x3F803F80u;
+    if (tid < 128) {        // L[i][j] = 1 for j <= i
+        const uint32_t r7 = tid & 7;
+        for (int cc = 0; cc < 16; ++cc) {
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int col = cc * 8 + 2 * j;
+                w[j] = (col <= tid ? 0x3F80u : 0u) | (col + 1 <= tid ? 0x3F800000u : 0u);
+            }
+            sts128(sbase + kDqOffL + (cc >> 3) * kTileBytes + tid * 128 + (((cc & 7) ^ r7) << 4), w[0], w[1], w[2], w[3]);
+        }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = bars->tmem_base;
+    volatile int* abort_flag = &bars->abort_flag;
+
+    if (warp == 16) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG);
+            for (int c = 0; c < L; ++c) {
+                const int s = c % kDqStages;
+                if (c >= kDqStages && !mbar_wait(&bars->empty[s], ((c / kDqStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
+                    *abort_flag = 1;
+                    break;
+                }
+                if (*abort_flag) break;
+                uint8_t* st = smem + kDqOffStage + s * 3 * kTileBytes;
+                const int y = (int)(row0 + (int64_t)c * kChunk);
+                mbar_arrive_expect_tx(&bars->full[s], 3 * kTileBytes);
+                tma_load_2d(st, &mapK, 0, y, &bars->full[s]);
+                tma_load_2d(st + kTileBytes, &mapV, 0, y, &bars->full[s]);
+                tma_load_2d(st + 2 * kTileBytes, &mapG, 0, y, &bars->full[s]);
+            }
+        }
+    } else if (warp == 17) {
+        // ------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_dp = umma_idesc_bf16(128, 128, 0, 0);
+            const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
+            const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
+            const uint32_t idesc_s = umma_idesc_bf16(64, 64, 1, 1);
+            const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
+            const uint32_t aS = sbase + kDqOffS, aOnes = sbase + kDqOffOnes, aL = sbase + kDqOffL,
+                           aDP = sbase + kDqOffDP;
+            bool ok = true;
+            for (int c = 0; c < L && ok; ++c) {
+                const int s = c % kDqStages, b = c & 1;
+                const uint32_t aK = sbase + kDqOffStage + s * 3 * kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
+                ok = mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok || *abort_flag) { ok = false; break; }
+                tc_fence_after_sync();
+                for (int k = 0; k < 4; ++k)      // dP = G V^T (the dP tile in TMEM is free: dp_ready(c-1) was awaited)
+                    umma_bf16(tmem + kDqColDP, desc_k(aG + k * 32), desc_k(aV + k * 32), idesc_dp, k > 0);
+                umma_commit(&bars->dp_full);
+                ok = mbar_wait(&bars->state_ready, c & 1, prm.status, kStatusPipeTimeout);
+                if (ok && c >= 2) ok = mbar_wait(&bars->dq_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int k = 0; k < 4; ++k)      // h = G S_{c-1}^T
+                    umma_bf16(tmem + kDqColGt + b * 64, desc_k(aG + k * 32), desc_k(aS + k * 32), idesc_kk, k > 0);
+                for (int k = 0; k < 8; ++k)      // T = L k  (row-wise prefix sums of k inside the chunk)
+                    umma_bf16(tmem + kDqColT + b * 64, desc_k(aL + (k >> 2) * kTileBytes + (k & 3) * 32),
+                              desc_mn(aK + k * 2048), idesc_kmn, k > 0);
+                for (int k = 0; k < 8; ++k)      // S += k^T V
+                    umma_bf16(tmem + kDqColS, desc_mn(aK + k * 2048), desc_mn(aV + k * 2048), idesc_s, 1);
+                for (int k = 0; k < 8; ++k)      // Z += k^T 1
+                    umma_bf16(tmem + kDqColS + 64, desc_mn(aK + k * 2048), desc_ones(aOnes), idesc_z, 1);
+                umma_commit(&bars->s_full);
+                ok = mbar_wait(&bars->dp_ready, c & 1, prm.status, kStatusPipeTimeout);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int k = 0; k < 8; ++k)      // h += dP k
+                    umma_bf16(tmem + kDqColGt + b * 64, desc_k(aDP + (k >> 2) * kTileBytes + (k & 3) * 32),
+                              desc_mn(aK + k * 2048), idesc_kmn, 1);
+                umma_commit(&bars->dq_full[b]);
+                umma_commit(&bars->empty[s]);
+            }
+            if (!ok) *abort_flag = 1;
+        }
+    } else if (warp >= 12) {
+        // ---------------------------------------------------- prep warps: phi(K)
+        const int t = tid - 12 * 32;
+        const uint32_t r7 = t & 7;
+        for (int c = 0; c < L; ++c) {
+            const int s = c % kDqStages;
+            if (!mbar_wait(&bars->full[s], (c / kDqStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            if (prm.phi == LA_PHI_ELU1) {
+                phi_row_inplace(sbase + kDqOffStage + s * 3 * kTileBytes + t * 128, r7);
+                fence_proxy_async_smem();
+            }
+            mbar_arrive(&bars->mapped[s]);
+        }
+    } else if (warp >= 8) {
+        // --------------------------------- state conversion and dQ epilogue warps
+        const int quad = warp - 8;
+        const int t = quad * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const float* init = prm.init ? prm.init + (bh * prm.nseg + seg) * (int64_t)kStateFloats : nullptr;
+        state_init(tmem + kDqColS, quad, lane, sbase + kDqOffS, sZ + 64, init);      // "chunk -1" -> Z buffer 1
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        named_barrier(1, 128);
+        mbar_arrive(&bars->state_ready);
+
+        for (int c = 0; c < L; ++c) {
+            const int b = c & 1;
+            const int64_t row = row0 + (int64_t)c * kChunk + t;
+            uint4 qraw[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) qraw[j] = ldg128(prm.Q + row * kDim + j * 8);
+
+            if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            tc_fence_after_sync();
+            state_to_smem(tmem + kDqColS, quad, lane, sbase + kDqOffS, sZ + (c & 1) * 64, nullptr, nullptr);
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&bars->state_ready);
+
+            if (!mbar_wait(&bars->dq_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            tc_fence_after_sync();
+            const float* zprev = sZ + ((c + 1) & 1) * 64;                // Z_{c-1}
+            const uint32_t tGt = tmem + lane_base + kDqColGt + b * 64, tT = tmem + lane_base + kDqColT + b * 64;
+            const bool elu = prm.phi == LA_PHI_ELU1;
+            const float m = (c_begin + c == 0) ? sM[t] : 0.f;          // centring offset of the first chunk
+            // pass 1: q . h and q . Z_i
+            float qg = 0.f, qz = 0.f;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t g[32], tt[32];
+                tmem_ld32(tGt + h * 32, g);
+                tmem_ld32(tT + h * 32, tt);
+                tmem_ld_wait();
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    const uint4 qv = qraw[h * 4 + cc];
+                    const uint32_t qq[4] = {qv.x, qv.y, qv.z, qv.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int d = h * 32 + cc * 8 + 2 * j;
+                        const float x0 = bf16_lo(qq[j]), x1 = bf16_hi(qq[j]);
+                        const float q0 = elu ? phi_fast(x0) : x0, q1 = elu ? phi_fast(x1) : x1;
+                        qg = fmaf(q0, fmaf(m, __uint_as_float(tt[cc * 8 + 2 * j]), __uint_as_float(g[cc * 8 + 2 * j])),
+                                  fmaf(q1, fmaf(m, __uint_as_float(tt[cc * 8 + 2 * j + 1]), __uint_as_float(g[cc * 8 + 2 * j + 1])), qg));
+                        qz = fmaf(q0, zprev[d] + __uint_as_float(tt[cc * 8 + 2 * j]),
+                                  fmaf(q1, zprev[d + 1] + __uint_as_float(tt[cc * 8 + 2 * j + 1]), qz));
+                    }
+                }
+            }
+            const float dn = qz + prm.eps;
+            const float inv = 1.f / dn;
+            const float delta = -qg * inv;          // = -(G_i . O_i)
+            prm.dn[row] = dn;
+            prm.dl[row] = delta;
+            // pass 2: gq = (h + delta Z_i) / dn, chained with phi'(Q)
+            __nv_bfloat16* dst = prm.dQ + row * kDim;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t g[32], tt[32];
+                tmem_ld32(tGt + h * 32, g);
+                tmem_ld32(tT + h * 32, tt);
+                tmem_ld_wait();
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    const uint4 qv = qraw[h * 4 + cc];
+                    const uint32_t qq[4] = {qv.x, qv.y, qv.z, qv.w};
+                    uint32_t outp[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int d = h * 32 + cc * 8 + 2 * j;
+                        const float t0 = __uint_as_float(tt[cc * 8 + 2 * j]), t1 = __uint_as_float(tt[cc * 8 + 2 * j + 1]);
+                        float g0 = inv * fmaf(delta, zprev[d] + t0, fmaf(m, t0, __uint_as_float(g[cc * 8 + 2 * j])));
+                        float g1 = inv * fmaf(delta, zprev[d + 1] + t1, fmaf(m, t1, __uint_as_float(g[cc * 8 + 2 * j + 1])));
+                        if (elu) {
+                            const float x0 = bf16_lo(qq[j]), x1 = bf16_hi(qq[j]);
+                            g0 *= x0 > 0.f ? 1.f : phi_fast(x0);
+                            g1 *= x1 > 0.f ? 1.f : phi_fast(x1);
+                        }
+                        outp[j] = pack_bf16x2(g0, g1);
+                    }
+                    stg128(dst + h * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bars->dq_drained[b]);
+            named_barrier(1, 128);          // Z double buffer: nobody reads Z_{c-1} past this point
+        }
+    } else {
+        // -------------------------------------------------- dP post-processing warps
+        const int quad = warp & 3, half = warp >> 2;
+        const int t = quad * 32 + lane;
+        const uint32_t r7 = t & 7;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        // blocks of this warp: half 0 -> {0, 2}, half 1 -> {1, 3}, restricted to blk <= quad
+        const int blk0 = half, blk1 = half + 2;
+        const bool has0 = blk0 <= quad, has1 = blk1 <= quad;
+        const uint32_t tile_row = sbase + kDqOffDP + t * 128;
+        const uint32_t src = tmem + lane_base + kDqColDP;
+        for (int c = 0; c < L; ++c) {
+            if (!mbar_wait(&bars->dp_full, c & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            tc_fence_after_sync();
+            uint32_t v0[32], v1[32];
+            float m = 0.f;
+            if (has0) tmem_ld32(src + blk0 * 32, v0);
+            if (has1) tmem_ld32(src + blk1 * 32, v1);
+            if (c_begin + c == 0) m = __uint_as_float(tmem_ld1(src));      // first chunk of the sequence: centre on dP_i0
+            tmem_ld_wait();
+            if (has0) score_block_store(v0, tile_row, r7, blk0, blk0 == quad, lane, -m);
+            if (has1) score_block_store(v1, tile_row, r7, blk1, blk1 == quad, lane, -m);
+            if (c_begin + c == 0 && half == 0) sM[t] = m;
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&bars->dp_ready);
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 17) {
+        __syncwarp();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+// ===========================================================================
+// Reverse sweep: dK, dV.  Chunks are visited from the last to the first.
+// Warps 0-7: P and dP post-processing, 8-11: state conversion and dK/dV
+// epilogue, 12-15: qh = phi(Q) / dn, phi(K), dl column, 16: TMA, 17: MMA.
+// ===========================================================================
+constexpr int kKvStages = 2;
+constexpr int kKvThreads = 576;
+constexpr uint32_t kKvColP = 0;        // 128
+constexpr uint32_t kKvColDP = 128;     // 128
+constexpr uint32_t kKvColDk = 256;     // 64
+constexpr uint32_t kKvColDv = 320;     // 64
+constexpr uint32_t kKvColR = 384;      // 64 + 16
+
+constexpr uint32_t kKvOffStage = 0;                                        // kKvStages x {Q, K, V, G}
+constexpr uint32_t kKvOffP = kKvOffStage + kKvStages * 4 * kTileBytes;     // 2 tiles
+constexpr uint32_t kKvOffDP = kKvOffP + 2 * kTileBytes;                    // 2 tiles
+constexpr uint32_t kKvOffAux = kKvOffDP + 2 * kTileBytes;                  // delta column tile
+constexpr uint32_t kKvOffR = kKvOffAux + kTileBytes;                       // bf16 R tile
+constexpr uint32_t kKvOffDelta = kKvOffR + kDim * 128;                     // fp32 [kKvStages][128]
+constexpr uint32_t kKvOffRv = kKvOffDelta + kKvStages * 512;               // fp32 r[2][64]
+constexpr uint32_t kKvOffBar = kKvOffRv + 512;
+constexpr uint32_t kKvSmemBytes = kKvOffBar + 256 + 1024;
+
+struct KvBarriers {
+    uint64_t full[kKvStages], empty[kKvStages], mapped[kKvStages];
+    uint64_t pd_full, pd_ready, r_full, state_ready, dkv_full, dkv_drained, aux_free;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct KvParams {
+    const float* dn;            // dn_i from the forward sweep
+    const float* dl;            // dl_i = -(G_i . O_i) from the forward sweep
+    __nv_bfloat16* dK;
+    __nv_bfloat16* dV;
+    const float* init;          // per (bh, seg) [R | r] records (sum over LATER segments) or null
+    int* status;
+    int64_t N;
+    int chunks, chunks_per_seg, nseg;
+    float eps;
+    int phi;
+};
+
+__global__ void __launch_bounds__(kKvThreads, 1)
+causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                      const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapG,
+                      const KvParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    KvBarriers* bars = reinterpret_cast<KvBarriers*>(smem + kKvOffBar);
+    float* sDelta = reinterpret_cast<float*>(smem + kKvOffDelta);
+    float* sRv = reinterpret_cast<float*>(smem + kKvOffRv);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int seg = blockIdx.x % prm.nseg;
+    const int64_t bh = blockIdx.x / prm.nseg;
+    const int c_begin = seg * prm.chunks_per_seg;
+    const int c_end = min(prm.chunks, c_begin + prm.chunks_per_seg);
+    const int L = c_end - c_begin;
+    // iteration i visits chunk c_end - 1 - i
+    auto chunk_row = [&](int i) { return bh * prm.N + (int64_t)(c_end - 1 - i) * kChunk; };
+
+    if (tid == 0) {
+        for (int s = 0; s < kKvStages; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1 + 128);      // MMA commit + the epilogue warps (they read phi(K) rows)
+            mbar_init(&bars->mapped[s], 128);
+        }
+        mbar_init(&bars->pd_full, 1);
+        mbar_init(&bars->pd_ready, 256);
+        mbar_init(&bars->r_full, 1);
+        mbar_init(&bars->state_ready, 128);
+        mbar_init(&bars->dkv_full, 1);
+        mbar_init(&bars->dkv_drained, 128);
+        bars->abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 17) {
+        __syncwarp();
+        tmem_alloc(&bars->tmem_base, 512);
+        tmem_relinquish();
+    }
+    for (uint32_t i = tid; i < 4 * kTileBytes / 16; i += kKvThreads) sts128(sbase + kKvOffP + i * 16, 0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = bars->tmem_base;
+    volatile int* abort_flag = &bars->abort_flag;
+
+    if (warp == 16) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG);
+            for (int i = 0; i < L; ++i) {
+                const int s = i % kKvStages;
+                if (i >= kKvStages && !mbar_wait(&bars->empty[s], ((i / kKvStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
+                    *abort_flag = 1;
+                    break;
+                }
+                if (*abort_flag) break;
+                uint8_t* st = smem + kKvOffStage + s * 4 * kTileBytes;
+                const int y = (int)chunk_row(i);
+                mbar_arrive_expect_tx(&bars->full[s], 4 * kTileBytes);
+                tma_load_2d(st, &mapQ, 0, y, &bars->full[s]);
+                tma_load_2d(st + kTileBytes, &mapK, 0, y, &bars->full[s]);
+                tma_load_2d(st + 2 * kTileBytes, &mapV, 0, y, &bars->full[s]);
+                tma_load_2d(st + 3 * kTileBytes, &mapG, 0, y, &bars->full[s]);
+            }
+        }
+    } else if (warp == 17) {
+        // ------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_pp = umma_idesc_bf16(128, 128, 0, 0);
+            const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
+            const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
+            const uint32_t idesc_mnmn = umma_idesc_bf16(128, 64, 1, 1);
+            const uint32_t idesc_s = umma_idesc_bf16(64, 64, 1, 1);
+            const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
+            const uint32_t aR = sbase + kKvOffR, aAux = sbase + kKvOffAux;
+            const uint32_t aP = sbase + kKvOffP, aDP = sbase + kKvOffDP;
+            bool ok = true;
+            for (int i = 0; i < L && ok; ++i) {
+                const int s = i % kKvStages;
+                const uint32_t aQ = sbase + kKvOffStage + s * 4 * kTileBytes, aK = aQ + kTileBytes, aV = aK + kTileBytes,
+                               aG = aV + kTileBytes;
+                ok = mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok || *abort_flag) { ok = false; break; }
+                tc_fence_after_sync();
+                for (int k = 0; k < 4; ++k)      // Ph = qh k^T
+                    umma_bf16(tmem + kKvColP, desc_k(aQ + k * 32), desc_k(aK + k * 32), idesc_pp, k > 0);
+                for (int k = 0; k < 4; ++k)      // dP = G V^T
+                    umma_bf16(tmem + kKvColDP, desc_k(aG + k * 32), desc_k(aV + k * 32), idesc_pp, k > 0);
+                umma_commit(&bars->pd_full);
+                ok = mbar_wait(&bars->state_ready, i & 1, prm.status, kStatusPipeTimeout);
+                if (ok && i >= 1) ok = mbar_wait(&bars->dkv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int k = 0; k < 4; ++k)      // gk = V R_{c+1}^T
+                    umma_bf16(tmem + kKvColDk, desc_k(aV + k * 32), desc_k(aR + k * 32), idesc_kk, k > 0);
+                for (int k = 0; k < 4; ++k)      // gV = k R_{c+1}
+                    umma_bf16(tmem + kKvColDv, desc_k(aK + k * 32), desc_mn(aR + k * 2048), idesc_kmn, k > 0);
+                for (int k = 0; k < 8; ++k)      // R += qh^T G
+                    umma_bf16(tmem + kKvColR, desc_mn(aQ + k * 2048), desc_mn(aG + k * 2048), idesc_s, 1);
+                for (int k = 0; k < 8; ++k)      // r += qh^T dl
+                    umma_bf16(tmem + kKvColR + 64, desc_mn(aQ + k * 2048), desc_mn(aAux + k * 2048), idesc_z, 1);
+                umma_commit(&bars->r_full);
+                ok = mbar_wait(&bars->pd_ready, i & 1, prm.status, kStatusPipeTimeout);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int k = 0; k < 8; ++k)      // gk += dP^T qh
+                    umma_bf16(tmem + kKvColDk, desc_mn(aDP + k * 2048), desc_mn(aQ + k * 2048), idesc_mnmn, 1);
+                for (int k = 0; k < 8; ++k)      // gV += Ph^T G
+                    umma_bf16(tmem + kKvColDv, desc_mn(aP + k * 2048), desc_mn(aG + k * 2048), idesc_mnmn, 1);
+                umma_commit(&bars->dkv_full);
+                umma_commit(&bars->empty[s]);
+            }
+            if (!ok) *abort_flag = 1;
+        }
+    } else if (warp >= 12) {
+        // ---------------------- prep warps: qh = phi(Q) / dn, phi(K), dl column
+        const int t = tid - 12 * 32;
+        const uint32_t r7 = t & 7;
+        const bool elu = prm.phi == LA_PHI_ELU1;
+        for (int i = 0; i < L; ++i) {
+            const int s = i % kKvStages;
+            const int64_t row = chunk_row(i) + t;
+            const float inv = 1.f / __ldg(prm.dn + row);
+            const float delta = __ldg(prm.dl + row);
+            if (!mbar_wait(&bars->full[s], (i / kKvStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            const uint32_t aQ = sbase + kKvOffStage + s * 4 * kTileBytes + t * 128;
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) {
+                uint32_t v[4];
+                lds128(aQ + ((cc ^ r7) << 4), v);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float x0 = bf16_lo(v[j]), x1 = bf16_hi(v[j]);
+                    v[j] = pack_bf16x2((elu ? phi_fast(x0) : x0) * inv, (elu ? phi_fast(x1) : x1) * inv);
+                }
+                sts128(aQ + ((cc ^ r7) << 4), v[0], v[1], v[2], v[3]);
+            }
+            if (elu) phi_row_inplace(aQ + kTileBytes, r7);
+            sDelta[s * 128 + t] = delta;
+            // the single dl column tile is an operand of the previous chunk's state MMAs
+            if (i >= 1 && !mbar_wait(&bars->r_full, (i - 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            const uint32_t aA = sbase + kKvOffAux + t * 128;
+            const uint32_t dd = pack_bf16x2(delta, delta);
+            sts128(aA + ((0 ^ r7) << 4), dd, dd, dd, dd);
+            sts128(aA + ((1 ^ r7) << 4), dd, dd, dd, dd);
+            fence_proxy_async_smem();
+            mbar_arrive(&bars->mapped[s]);
+        }
+    } else if (warp >= 8) {
+        // ------------------------------ state conversion and dK / dV epilogue warps
+        const int quad = warp - 8;
+        const int t = quad * 32 + lane;
+        const uint32_t r7 = t & 7;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const float* init = prm.init ? prm.init + (bh * prm.nseg + seg) * (int64_t)kStateFloats : nullptr;
+        state_init(tmem + kKvColR, quad, lane, sbase + kKvOffR, sRv + 64, init);      // "iteration -1" -> buffer 1
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        named_barrier(1, 128);
+        mbar_arrive(&bars->state_ready);
+
+        for (int i = 0; i < L; ++i) {
+            const int s = i % kKvStages;
+            const int64_t row = chunk_row(i) + t;
+            if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            uint32_t kf[8][4];                      // phi(K) row, logical chunk order
+            const uint32_t aKrow = sbase + kKvOffStage + s * 4 * kTileBytes + kTileBytes + t * 128;
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) lds128(aKrow + ((cc ^ r7) << 4), kf[cc]);
+            mbar_arrive(&bars->empty[s]);
+
+            if (!mbar_wait(&bars->r_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            tc_fence_after_sync();
+            state_to_smem(tmem + kKvColR, quad, lane, sbase + kKvOffR, sRv + (i & 1) * 64, nullptr, nullptr);
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&bars->state_ready);
+
+            if (!mbar_wait(&bars->dkv_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            tc_fence_after_sync();
+            const float* rprev = sRv + ((i + 1) & 1) * 64;               // r_{c+1}
+            __nv_bfloat16* dstK = prm.dK + row * kDim;
+            __nv_bfloat16* dstV = prm.dV + row * kDim;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_base + kKvColDk + h * 32, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t outp[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int d = h * 32 + cc * 8 + 2 * j;
+                        float g0 = __uint_as_float(v[cc * 8 + 2 * j]) + rprev[d];
+                        float g1 = __uint_as_float(v[cc * 8 + 2 * j + 1]) + rprev[d + 1];
+                        if (prm.phi == LA_PHI_ELU1) {
+                            const float k0 = bf16_lo(kf[h * 4 + cc][j]), k1 = bf16_hi(kf[h * 4 + cc][j]);
+                            g0 *= k0 > 1.f ? 1.f : k0;          // phi'(x) from phi(x): 1 where x > 0, else phi(x)
+                            g1 *= k1 > 1.f ? 1.f : k1;
+                        }
+                        outp[j] = pack_bf16x2(g0, g1);
+                    }
+                    stg128(dstK + h * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_base + kKvColDv + h * 32, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+                    stg128(dstV + h * 32 + cc * 8,
+                           pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
+                           pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
+                           pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
+                           pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bars->dkv_drained);
+            named_barrier(1, 128);          // r double buffer
+        }
+    } else {
+        // ------------------------------------------- P and dP post-processing warps
+        const int quad = warp & 3, half = warp >> 2;
+        const int t = quad * 32 + lane;
+        const uint32_t r7 = t & 7;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const int blk0 = half, blk1 = half + 2;
+        const bool has0 = blk0 <= quad, has1 = blk1 <= quad;
+        const uint32_t rowP = sbase + kKvOffP + t * 128, rowDP = sbase + kKvOffDP + t * 128;
+        for (int i = 0; i < L; ++i) {
+            const int s = i % kKvStages;
+            if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout) ||
+                !mbar_wait(&bars->pd_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            tc_fence_after_sync();
+            const float delta = sDelta[s * 128 + t];
+            uint32_t v0[32], v1[32];
+            if (has0) tmem_ld32(tmem + lane_base + kKvColP + blk0 * 32, v0);
+            if (has1) tmem_ld32(tmem + lane_base + kKvColP + blk1 * 32, v1);
+            tmem_ld_wait();
+            if (has0) score_block_store(v0, rowP, r7, blk0, blk0 == quad, lane, 0.f);
+            if (has1) score_block_store(v1, rowP, r7, blk1, blk1 == quad, lane, 0.f);
+            if (has0) tmem_ld32(tmem + lane_base + kKvColDP + blk0 * 32, v0);
+            if (has1) tmem_ld32(tmem + lane_base + kKvColDP + blk1 * 32, v1);
+            tmem_ld_wait();
+            if (has0) score_block_store(v0, rowDP, r7, blk0, blk0 == quad, lane, delta);
+            if (has1) score_block_store(v1, rowDP, r7, blk1, blk1 == quad, lane, delta);
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&bars->pd_ready);
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 17) {
+        __syncwarp();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+}  // namespace
+
+size_t causal_backward_workspace(const la_problem& p) {
+    const Segmentation sg = choose_segments(p);
+    const size_t bh = (size_t)(p.B * p.H);
+    size_t bytes = 2 * bh * sg.nseg * kStateFloats * sizeof(float);      // forward and reverse segment records
+    bytes += 2 * bh * (size_t)p.N * sizeof(float);                       // dn_i and dl_i per row
+    return bytes;
+}
+
+int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+                    void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    const Segmentation sg = choose_segments(p);
+    const int chunks = (int)(p.N / kChunk);
+    const size_t bh = (size_t)(p.B * p.H);
+    const uint64_t rows = (uint64_t)(bh * p.N);
+
+    // workspace carve-up (see causal_backward_workspace)
+    uint8_t* w = (uint8_t*)ws;
+    float* rec_s = (float*)w;            w += bh * sg.nseg * kStateFloats * sizeof(float);
+    float* rec_r = (float*)w;            w += bh * sg.nseg * kStateFloats * sizeof(float);
+    float* dn = (float*)w;               w += bh * (size_t)p.N * sizeof(float);
+    float* dl = (float*)w;
+
+    CUtensorMap mQ, mK, mV, mG;
+    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mK, K, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mV, V, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mG, G, rows, kChunk)) return rc;
+    int* status = device_status_ptr();
+    if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
+
+    static bool attr_done = false;
+    if (!attr_done) {
+        LA_CUDA_TRY(cudaFuncSetAttribute(causal_bwd_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDqSmemBytes));
+        LA_CUDA_TRY(cudaFuncSetAttribute(causal_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kKvSmemBytes));
+        attr_done = true;
+    }
+    const unsigned grid = (unsigned)(sg.nseg * bh);
+
+    // forward sweep: dQ, and dn_i, dl_i for the reverse sweep
+    if (int rc = segment_states(p, sg, mK, mV, nullptr, nullptr, rec_s, /*reverse=*/false, st)) return rc;
+    DqParams a;
+    a.Q = (const __nv_bfloat16*)Q;
+    a.dn = dn;
+    a.dl = dl;
+    a.dQ = (__nv_bfloat16*)dQ;
+    a.init = sg.nseg > 1 ? rec_s : nullptr;
+    a.status = status;
+    a.N = p.N;
+    a.chunks = chunks;
+    a.chunks_per_seg = sg.chunks_per_seg;
+    a.nseg = sg.nseg;
+    a.eps = p.eps;
+    a.phi = p.phi;
+    causal_bwd_dq_kernel<<<grid, kDqThreads, kDqSmemBytes, st>>>(mK, mV, mG, a);
+    LA_LAUNCHED();
+
+    // reverse sweep: dK, dV
+    if (int rc = segment_states(p, sg, mQ, mG, dn, dl, rec_r, /*reverse=*/true, st)) return rc;
+    KvParams b;
+    b.dn = dn;
+    b.dl = dl;
+    b.dK = (__nv_bfloat16*)dK;
+    b.dV = (__nv_bfloat16*)dV;
+    b.init = sg.nseg > 1 ? rec_r : nullptr;
+    b.status = status;
+    b.N = p.N;
+    b.chunks = chunks;
+    b.chunks_per_seg = sg.chunks_per_seg;
+    b.nseg = sg.nseg;
+    b.eps = p.eps;
+    b.phi = p.phi;
+    causal_bwd_dkv_kernel<<<grid, kKvThreads, kKvSmemBytes, st>>>(mQ, mK, mV, mG, b);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+}  // namespace tc
+}  // namespace la

@@ -64,11 +64,6 @@ struct FwdParams {
     int phi;
 };
 
-__device__ __forceinline__ uint64_t desc_k(uint32_t addr) { return umma_desc_sw128(addr, 16, 1024); }
-__device__ __forceinline__ uint64_t desc_mn(uint32_t addr, uint32_t lbo = kTileBytes) {
-    return umma_desc_sw128(addr, lbo, 1024);
-}
-
 // ---------------------------------------------------------------------------
 // Main kernel.
 // ---------------------------------------------------------------------------
@@ -371,152 +366,6 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     }
 }
 
-// ---------------------------------------------------------------------------
-// Pre-pass: per-segment sums of phi(K)^T [V | 1] (segments 0 .. nseg-2).
-// Warps 0-3: phi on K and the final read-out, warp 4: TMA, warp 5: MMA.
-// ---------------------------------------------------------------------------
-constexpr int kSumThreads = 192;
-constexpr int kSumStages = 4;
-constexpr uint32_t kSumOffOnes = kSumStages * 2 * kTileBytes;
-constexpr uint32_t kSumOffBar = kSumOffOnes + 1024;
-constexpr uint32_t kSumSmemBytes = kSumOffBar + 256 + 1024;
-
-struct SumBarriers {
-    uint64_t full[kSumStages], empty[kSumStages], mapped[kSumStages];
-    uint64_t done;
-    uint32_t tmem_base;
-    int abort_flag;
-};
-
-__global__ void __launch_bounds__(kSumThreads, 1)
-segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
-                   float* __restrict__ records, int64_t N, int chunks, int chunks_per_seg, int nseg, int phi,
-                   int* status) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const uint32_t sbase = smem_u32(smem);
-    SumBarriers* bars = reinterpret_cast<SumBarriers*>(smem + kSumOffBar);
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int seg = blockIdx.x % (nseg - 1);          // the last segment's sum is never needed
-    const int64_t bh = blockIdx.x / (nseg - 1);
-    const int c_begin = seg * chunks_per_seg;
-    const int L = min(chunks, c_begin + chunks_per_seg) - c_begin;
-    const int64_t row0 = bh * N + (int64_t)c_begin * kChunk;
-
-    if (tid == 0) {
-        for (int s = 0; s < kSumStages; ++s) {
-            mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], 1);
-            mbar_init(&bars->mapped[s], 128);
-        }
-        mbar_init(&bars->done, 1);
-        bars->abort_flag = 0;
-        fence_mbar_init();
-    }
-    if (warp == 5) {
-        __syncwarp();
-        tmem_alloc(&bars->tmem_base, 128);
-        tmem_relinquish();
-    }
-    if (tid < 128)
-        for (int i = tid; i < 256; i += 128) reinterpret_cast<uint32_t*>(smem + kSumOffOnes)[i] = 0x3F803F80u;
-    fence_proxy_async_smem();
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem = bars->tmem_base;
-    volatile int* abort_flag = &bars->abort_flag;
-
-    if (warp == 4) {
-        if (lane == 0) {
-            prefetch_tensormap(&mapX); prefetch_tensormap(&mapY);
-            for (int c = 0; c < L; ++c) {
-                const int s = c % kSumStages;
-                if (c >= kSumStages && !mbar_wait(&bars->empty[s], ((c / kSumStages) - 1) & 1, status, kStatusPipeTimeout)) {
-                    *abort_flag = 1;
-                    break;
-                }
-                if (*abort_flag) break;
-                uint8_t* st = smem + s * 2 * kTileBytes;
-                const int y = (int)(row0 + (int64_t)c * kChunk);
-                mbar_arrive_expect_tx(&bars->full[s], 2 * kTileBytes);
-                tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
-                tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
-            }
-        }
-    } else if (warp == 5) {
-        if (lane == 0) {
-            const uint32_t idesc_s = umma_idesc_bf16(64, 64, 1, 1);
-            const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
-            const uint32_t aOnes = sbase + kSumOffOnes;
-            bool ok = true;
-            for (int c = 0; c < L && ok; ++c) {
-                const int s = c % kSumStages;
-                const uint32_t aX = sbase + s * 2 * kTileBytes, aY = aX + kTileBytes;
-                ok = mbar_wait(&bars->mapped[s], (c / kSumStages) & 1, status, kStatusPipeTimeout);
-                if (!ok || *abort_flag) { ok = false; break; }
-                tc_fence_after_sync();
-                for (int k = 0; k < 8; ++k)
-                    umma_bf16(tmem, desc_mn(aX + k * 2048), desc_mn(aY + k * 2048), idesc_s, (c | k) != 0);
-                for (int k = 0; k < 8; ++k)
-                    umma_bf16(tmem + 64, desc_mn(aX + k * 2048), umma_desc_sw128(aOnes, 16, 0), idesc_z, (c | k) != 0);
-                umma_commit(&bars->empty[s]);
-            }
-            if (!ok) *abort_flag = 1;
-            umma_commit(&bars->done);
-        }
-    } else {
-        const int t = tid;
-        const uint32_t r7 = t & 7;
-        for (int c = 0; c < L; ++c) {
-            const int s = c % kSumStages;
-            if (!mbar_wait(&bars->full[s], (c / kSumStages) & 1, status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
-            if (*abort_flag) break;
-            if (phi == LA_PHI_ELU1) {
-                phi_row_inplace(sbase + s * 2 * kTileBytes + t * 128, r7);
-                fence_proxy_async_smem();
-            }
-            mbar_arrive(&bars->mapped[s]);
-        }
-        // read-out: [S | Z] record of this (bh, seg)
-        const bool ok = mbar_wait(&bars->done, 0, status, kStatusMmaTimeout) && !*abort_flag;
-        tc_fence_after_sync();
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        float* rec = records + (bh * nseg + seg) * (int64_t)kStateFloats;
-        const int d_row = warp * 16 + lane;
-        for (int h = 0; h < 2; ++h) {
-            uint32_t v[32];
-            tmem_ld32(tmem + lane_base + h * 32, v);
-            tmem_ld_wait();
-            if (ok && lane < 16)
-#pragma unroll
-                for (int j = 0; j < 32; ++j) rec[d_row * kDim + h * 32 + j] = __uint_as_float(v[j]);
-        }
-        const float z = __uint_as_float(tmem_ld1(tmem + lane_base + 64));
-        tmem_ld_wait();
-        if (ok && lane < 16) rec[kDim * kDim + d_row] = z;
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 5) {
-        __syncwarp();
-        tmem_dealloc(tmem, 128);
-    }
-}
-
-// Exclusive prefix over the segments of each (batch, head): record[seg] <- sum of records before it.
-__global__ void __launch_bounds__(256) segment_scan_kernel(float* __restrict__ records, int nseg) {
-    float* base = records + (int64_t)blockIdx.x * nseg * kStateFloats;
-    for (int i = threadIdx.x; i < kStateFloats; i += 256) {
-        float run = 0.f;
-        for (int s = 0; s < nseg; ++s) {
-            const float cur = s + 1 < nseg ? base[(int64_t)s * kStateFloats + i] : 0.f;
-            base[(int64_t)s * kStateFloats + i] = run;
-            run += cur;
-        }
-    }
-}
-
 }  // namespace
 
 Segmentation choose_segments(const la_problem& p) {
@@ -557,16 +406,11 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     static bool attr_done = false;
     if (!attr_done) {
         LA_CUDA_TRY(cudaFuncSetAttribute(causal_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-        LA_CUDA_TRY(cudaFuncSetAttribute(segment_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSumSmemBytes));
         attr_done = true;
     }
     float* records = (float*)ws;
     if (sg.nseg > 1) {
-        segment_sum_kernel<<<(unsigned)((sg.nseg - 1) * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(
-            mK, mV, records, p.N, chunks, sg.chunks_per_seg, sg.nseg, p.phi, status);
-        LA_LAUNCHED();
-        segment_scan_kernel<<<(unsigned)(p.B * p.H), 256, 0, st>>>(records, sg.nseg);
-        LA_LAUNCHED();
+        if (int rc = segment_states(p, sg, mK, mV, nullptr, nullptr, records, /*reverse=*/false, st)) return rc;
     }
     FwdParams prm;
     prm.den = den;

@@ -22,6 +22,14 @@ struct Segmentation {
     int chunks_per_seg;   // chunks in every segment but possibly the last
 };
 
+Segmentation choose_segments(const la_problem& p);
+
+// Per-segment sums of phi(X)^T [Y | a] into `records` followed by their exclusive scan
+// (prefix, or suffix when `reverse`).  dn == nullptr: a = 1; otherwise the rows of phi(X) are
+// divided by dn and a = dl.  No-op for a single segment.
+int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
+                   const float* dn, const float* dl, float* records, bool reverse, cudaStream_t st);
+
 // 2-D view of a [rows][64] bf16 tensor with a [box_rows][64] box and the 128-byte swizzle.
 int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows);
 
@@ -57,6 +65,111 @@ __device__ __forceinline__ void lds128(uint32_t addr, uint32_t (&v)[4]) {
 }
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+__device__ __forceinline__ uint64_t desc_k(uint32_t addr) { return sm100::umma_desc_sw128(addr, 16, 1024); }
+__device__ __forceinline__ uint64_t desc_mn(uint32_t addr, uint32_t lbo = kTileBytes) {
+    return sm100::umma_desc_sw128(addr, lbo, 1024);
+}
+// B operand whose every entry is 1: one 1 KB group of ones re-read for every K group (SBO = 0).
+__device__ __forceinline__ uint64_t desc_ones(uint32_t addr) { return sm100::umma_desc_sw128(addr, 16, 0); }
+
+__device__ __forceinline__ uint4 ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+__device__ __forceinline__ void stg128(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
+}
+
+// One 32-column block of a 128x128 fp32 score matrix (already loaded from TMEM into v)
+// -> + `add` -> causal mask on the diagonal block -> bf16 -> this row's 64 bytes of the
+// swizzled [128][64] tile pair.  tile_row = shared address of row t in tile 0 of the pair.
+__device__ __forceinline__ void score_block_store(const uint32_t (&v)[32], uint32_t tile_row, uint32_t r7, int blk,
+                                                  bool diagonal, int lane, float add) {
+    uint32_t packed[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float x0 = __uint_as_float(v[2 * j]) + add, x1 = __uint_as_float(v[2 * j + 1]) + add;
+        if (diagonal) {
+            if (2 * j > lane) x0 = 0.f;
+            if (2 * j + 1 > lane) x1 = 0.f;
+        }
+        packed[j] = sm100::pack_bf16x2(x0, x1);
+    }
+    const uint32_t base = tile_row + (blk >> 1) * kTileBytes;
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+        const uint32_t chunk = (blk & 1) * 4 + cc;
+        sts128(base + ((chunk ^ r7) << 4), packed[cc * 4], packed[cc * 4 + 1], packed[cc * 4 + 2], packed[cc * 4 + 3]);
+    }
+}
+
+// State accumulator (M = 64 layout: lanes 0-15 of quadrant w hold rows 16w..16w+15; 64 columns
+// of S followed by Z) -> bf16 [64][64] swizzled tile + fp32 Z; optionally the fp32 values to
+// global memory.  Executed by the four warps of one warpgroup; `quad` = warp % 4.
+__device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int lane, uint32_t s_tile, float* z_out,
+                                              float* g_S, float* g_Z) {
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const int d_row = quad * 16 + lane;
+    const bool owner = lane < 16;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint32_t v[32];
+        sm100::tmem_ld32(tmem_state + lane_base + h * 32, v);
+        sm100::tmem_ld_wait();
+        if (owner) {
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                const uint32_t chunk = h * 4 + cc;
+                sts128(s_tile + d_row * 128 + ((chunk ^ (d_row & 7)) << 4),
+                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
+                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
+                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
+                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
+            }
+            if (g_S) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) g_S[d_row * kDim + h * 32 + j] = __uint_as_float(v[j]);
+            }
+        }
+    }
+    const float z = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 64));
+    sm100::tmem_ld_wait();
+    if (owner) {
+        z_out[d_row] = z;
+        if (g_Z) g_Z[d_row] = z;
+    }
+}
+
+// Load an initial [S | Z] record (or zeros) into the TMEM state accumulator, its bf16 tile and z_out.
+__device__ __forceinline__ void state_init(uint32_t tmem_state, int quad, int lane, uint32_t s_tile, float* z_out,
+                                           const float* rec) {
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const int d_row = quad * 16 + lane;
+    const bool owner = lane < 16;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint32_t v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = (rec && owner) ? __float_as_uint(rec[d_row * kDim + h * 32 + j]) : 0u;
+        sm100::tmem_st32(tmem_state + lane_base + h * 32, v);
+        if (owner) {
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                const uint32_t chunk = h * 4 + cc;
+                sts128(s_tile + d_row * 128 + ((chunk ^ (d_row & 7)) << 4),
+                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
+                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
+                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
+                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
+            }
+        }
+    }
+    const float z = (rec && owner) ? rec[kDim * kDim + d_row] : 0.f;
+    uint32_t zz[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) zz[j] = __float_as_uint(z);
+    sm100::tmem_st16(tmem_state + lane_base + 64, zz);
+    sm100::tmem_st_wait();
+    if (owner) z_out[d_row] = z;
 }
 
 }  // namespace tc

@@ -1,0 +1,236 @@
+// Segment pre-pass of the tensor-core causal kernels: per-segment sums of
+//     phi(X_i) [Y_i | a_i]^T        (64 x 65 per segment, fp32)
+// and their exclusive scan over the segments of a sequence.
+//   forward state  St: X = K, Y = V,            a_i = 1        (Eq. 10-11), exclusive prefix
+//   reverse state  Rt: X = Q (rows / dn_i), Y = G, a_i = dl_i  (the cumulative sum of Eq. 14-15),
+//                                                               exclusive suffix
+// so that every segment can start from the state the sequential recurrence would have
+// reached.  Warps 0-3: phi on X, scaling of Y and the final read-out; warp 4: TMA;
+// warp 5: MMA (M = 64 accumulators in TMEM).
+#include "la_tc.cuh"
+#include "la_tc_common.cuh"
+
+namespace la {
+namespace tc {
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kSumThreads = 192;
+constexpr int kSumStages = 3;
+constexpr uint32_t kSumStageBytes = 3 * kTileBytes;                  // X, Y, aux column tile
+constexpr uint32_t kSumOffOnes = kSumStages * kSumStageBytes;
+constexpr uint32_t kSumOffBar = kSumOffOnes + 1024;
+constexpr uint32_t kSumSmemBytes = kSumOffBar + 256 + 1024;
+
+struct SumBarriers {
+    uint64_t full[kSumStages], empty[kSumStages], mapped[kSumStages];
+    uint64_t done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct SumParams {
+    float* records;        // [BH][nseg][kStateFloats]
+    const float* dn;       // null: phi(X) is used as is and a_i = 1; else phi(X_i) is divided by dn_i
+    const float* dl;       // with dn: a_i = dl_i
+    int* status;
+    int64_t N;
+    int chunks, chunks_per_seg, nseg;
+    int first_seg;         // segments first_seg .. first_seg + segs_per_seq - 1 are summed
+    int segs_per_seq;
+    float eps;
+    int phi;
+};
+
+__global__ void __launch_bounds__(kSumThreads, 1)
+segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
+                   const SumParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    SumBarriers* bars = reinterpret_cast<SumBarriers*>(smem + kSumOffBar);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int seg = prm.first_seg + blockIdx.x % prm.segs_per_seq;
+    const int64_t bh = blockIdx.x / prm.segs_per_seq;
+    const int c_begin = seg * prm.chunks_per_seg;
+    const int L = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
+    const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
+    const bool scaled = prm.dn != nullptr;
+
+    if (tid == 0) {
+        for (int s = 0; s < kSumStages; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+            mbar_init(&bars->mapped[s], 128);
+        }
+        mbar_init(&bars->done, 1);
+        bars->abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 5) {
+        __syncwarp();
+        tmem_alloc(&bars->tmem_base, 128);
+        tmem_relinquish();
+    }
+    if (tid < 128)
+        for (int i = tid; i < 256; i += 128) reinterpret_cast<uint32_t*>(smem + kSumOffOnes)[i] = 0x3F803F80u;
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = bars->tmem_base;
+    volatile int* abort_flag = &bars->abort_flag;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            prefetch_tensormap(&mapX); prefetch_tensormap(&mapY);
+            for (int c = 0; c < L; ++c) {
+                const int s = c % kSumStages;
+                if (c >= kSumStages && !mbar_wait(&bars->empty[s], ((c / kSumStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
+                    *abort_flag = 1;
+                    break;
+                }
+                if (*abort_flag) break;
+                uint8_t* st = smem + s * kSumStageBytes;
+                const int y = (int)(row0 + (int64_t)c * kChunk);
+                mbar_arrive_expect_tx(&bars->full[s], 2 * kTileBytes);
+                tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
+                tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            const uint32_t idesc_s = umma_idesc_bf16(64, 64, 1, 1);
+            const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
+            const uint32_t aOnes = sbase + kSumOffOnes;
+            bool ok = true;
+            for (int c = 0; c < L && ok; ++c) {
+                const int s = c % kSumStages;
+                const uint32_t aX = sbase + s * kSumStageBytes, aY = aX + kTileBytes, aA = aY + kTileBytes;
+                ok = mbar_wait(&bars->mapped[s], (c / kSumStages) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok || *abort_flag) { ok = false; break; }
+                tc_fence_after_sync();
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16(tmem, desc_mn(aX + k * 2048), desc_mn(aY + k * 2048), idesc_s, (c | k) != 0);
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16(tmem + 64, desc_mn(aX + k * 2048), scaled ? desc_mn(aA + k * 2048) : desc_ones(aOnes),
+                              idesc_z, (c | k) != 0);
+                umma_commit(&bars->empty[s]);
+            }
+            if (!ok) *abort_flag = 1;
+            umma_commit(&bars->done);
+        }
+    } else {
+        const int t = tid;
+        const uint32_t r7 = t & 7;
+        for (int c = 0; c < L; ++c) {
+            const int s = c % kSumStages;
+            const int64_t row = row0 + (int64_t)c * kChunk + t;
+            float inv = 1.f, delta = 0.f;
+            if (scaled) {
+                inv = 1.f / __ldg(prm.dn + row);
+                delta = __ldg(prm.dl + row);
+            }
+            if (!mbar_wait(&bars->full[s], (c / kSumStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            const uint32_t aX = sbase + s * kSumStageBytes + t * 128;
+            if (!scaled) {
+                if (prm.phi == LA_PHI_ELU1) phi_row_inplace(aX, r7);
+            } else {
+                const bool elu = prm.phi == LA_PHI_ELU1;
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc) {
+                    uint32_t v[4];
+                    lds128(aX + ((cc ^ r7) << 4), v);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float x0 = bf16_lo(v[j]), x1 = bf16_hi(v[j]);
+                        v[j] = pack_bf16x2((elu ? phi_fast(x0) : x0) * inv, (elu ? phi_fast(x1) : x1) * inv);
+                    }
+                    sts128(aX + ((cc ^ r7) << 4), v[0], v[1], v[2], v[3]);
+                }
+                const uint32_t aA = aX + 2 * kTileBytes;
+                const uint32_t dd = pack_bf16x2(delta, delta);      // columns 0..15 of the aux tile
+                sts128(aA + ((0 ^ r7) << 4), dd, dd, dd, dd);
+                sts128(aA + ((1 ^ r7) << 4), dd, dd, dd, dd);
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&bars->mapped[s]);
+        }
+        // read-out: the [S | Z]-shaped record of this (bh, seg)
+        const bool ok = mbar_wait(&bars->done, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
+        tc_fence_after_sync();
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        float* rec = prm.records + (bh * prm.nseg + seg) * (int64_t)kStateFloats;
+        const int d_row = warp * 16 + lane;
+        for (int h = 0; h < 2; ++h) {
+            uint32_t v[32];
+            tmem_ld32(tmem + lane_base + h * 32, v);
+            tmem_ld_wait();
+            if (ok && lane < 16)
+#pragma unroll
+                for (int j = 0; j < 32; ++j) rec[d_row * kDim + h * 32 + j] = __uint_as_float(v[j]);
+        }
+        const float z = __uint_as_float(tmem_ld1(tmem + lane_base + 64));
+        tmem_ld_wait();
+        if (ok && lane < 16) rec[kDim * kDim + d_row] = z;
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        __syncwarp();
+        tmem_dealloc(tmem, 128);
+    }
+}
+
+// Exclusive scan over the segments of each (batch, head): forward -> record[s] = sum of the
+// records before s; reverse -> record[s] = sum of the records after s.  The record at the
+// open end (last for forward, first for reverse) was never computed and is not read.
+__global__ void __launch_bounds__(256) segment_scan_kernel(float* __restrict__ records, int nseg, int reverse) {
+    float* base = records + (int64_t)blockIdx.x * nseg * kStateFloats;
+    for (int i = threadIdx.x; i < kStateFloats; i += 256) {
+        float run = 0.f;
+        for (int n = 0; n < nseg; ++n) {
+            const int s = reverse ? nseg - 1 - n : n;
+            const float cur = n + 1 < nseg ? base[(int64_t)s * kStateFloats + i] : 0.f;
+            base[(int64_t)s * kStateFloats + i] = run;
+            run += cur;
+        }
+    }
+}
+
+}  // namespace
+
+int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
+                   const float* dn, const float* dl, float* records, bool reverse, cudaStream_t st) {
+    if (sg.nseg <= 1) return LA_OK;
+    static bool attr_done = false;
+    if (!attr_done) {
+        LA_CUDA_TRY(cudaFuncSetAttribute(segment_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSumSmemBytes));
+        attr_done = true;
+    }
+    SumParams prm;
+    prm.records = records;
+    prm.dn = dn;
+    prm.dl = dl;
+    prm.status = device_status_ptr();
+    if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
+    prm.N = p.N;
+    prm.chunks = (int)(p.N / kChunk);
+    prm.chunks_per_seg = sg.chunks_per_seg;
+    prm.nseg = sg.nseg;
+    prm.first_seg = reverse ? 1 : 0;          // the open-end segment's own sum is never needed
+    prm.segs_per_seq = sg.nseg - 1;
+    prm.eps = p.eps;
+    prm.phi = p.phi;
+    segment_sum_kernel<<<(unsigned)((sg.nseg - 1) * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
+    LA_LAUNCHED();
+    segment_scan_kernel<<<(unsigned)(p.B * p.H), 256, 0, st>>>(records, sg.nseg, reverse ? 1 : 0);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+}  // namespace tc
+}  // namespace la

@@ -52,9 +52,9 @@ def test_causal_forward_backward(shape, dtype):
     assert_close(Z, Zr, dtype, "Z_N")
     dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd)
     rq, rk, rv = oracle.linear_attention_backward(Q, K, V, G, True)
-    assert_close(dQ, rq, dtype, "dQ")
-    assert_close(dK, rk, dtype, "dK")
-    assert_close(dV, rv, dtype, "dV")
+    assert_close(dQ, rq, dtype, "dQ", grad=True)
+    assert_close(dK, rk, dtype, "dK", grad=True)
+    assert_close(dV, rv, dtype, "dV", grad=True)
     la.la_last_device_status()
 
 
@@ -75,9 +75,9 @@ def test_noncausal_forward_backward(shape, dtype):
     assert_close(Zs, Zr, dtype, "Zs")
     dQ, dK, dV = la.la_linear_attention_backward(Qd, Kd, Vd, Gd)
     rq, rk, rv = oracle.linear_attention_backward(Q, K, V, G, False)
-    assert_close(dQ, rq, dtype, "dQ")
-    assert_close(dK, rk, dtype, "dK")
-    assert_close(dV, rv, dtype, "dV")
+    assert_close(dQ, rq, dtype, "dQ", grad=True)
+    assert_close(dK, rk, dtype, "dK", grad=True)
+    assert_close(dV, rv, dtype, "dV", grad=True)
     la.la_last_device_status()
 
 
@@ -95,7 +95,7 @@ def test_eps_and_identity_feature_map(causal, dtype):
     assert_close(O, oracle.linear_attention(Q, K, V, causal, "identity", 0.75)[0], dtype, "O")
     grads = bwd(Qd, Kd, Vd, Gd, phi="identity", eps=0.75)
     for g, r, nm in zip(grads, oracle.linear_attention_backward(Q, K, V, G, causal, "identity", 0.75), "QKV"):
-        assert_close(g, r, dtype, "d" + nm)
+        assert_close(g, r, dtype, "d" + nm, grad=True)
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
@@ -177,7 +177,7 @@ def test_causal_workloads_full_size(name):
         assert_close(O[sl], Or, dtype, f"{name} O[{b},{h}]")
         assert_close(den[sl], denr, dtype, f"{name} den[{b},{h}]")
         for got, ref, nm in zip((dQ, dK, dV), oracle.linear_attention_backward(q, k, v, g, True), "QKV"):
-            assert_close(got[sl], ref, dtype, f"{name} d{nm}[{b},{h}]")
+            assert_close(got[sl], ref, dtype, f"{name} d{nm}[{b},{h}]", grad=True)
     # size-independent properties on the whole result
     assert torch.isfinite(O.float()).all() and torch.isfinite(dQ.float()).all()
     assert torch.allclose(O[:, :, 0].float(), Vd[:, :, 0].float(), rtol=1e-2, atol=1e-2)     # O_1 = V_1
@@ -197,7 +197,7 @@ def test_noncausal_workload_full_size():
         q, k, v, g = Q[sl], K[sl], V[sl], G[sl]
         assert_close(O[sl], oracle.linear_attention(q, k, v, False)[0], dtype, f"O[{b},{h}]")
         for got, ref, nm in zip((dQ, dK, dV), oracle.linear_attention_backward(q, k, v, g, False), "QKV"):
-            assert_close(got[sl], ref, dtype, f"d{nm}[{b},{h}]")
+            assert_close(got[sl], ref, dtype, f"d{nm}[{b},{h}]", grad=True)
 
 
 def test_decode_workload_full_size():
