@@ -30,6 +30,9 @@ namespace tc {
 
 using namespace sm100;
 
+LA_TRACE_DECL(g_trace_dq)
+LA_TRACE_DECL(g_trace_dkv)
+
 namespace {
 
 // ===========================================================================
@@ -188,6 +191,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 ok = mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout);
                 if (!ok || *abort_flag) { ok = false; break; }
                 tc_fence_after_sync();
+                LA_TRACE(g_trace_dq, c, 0);
                 for (int k = 0; k < 4; ++k)      // dP = G V^T (the dP tile in TMEM is free: dp_ready(c-1) was awaited)
                     umma_bf16(tmem + kDqColDP, desc_k(aG + k * 32), desc_k(aV + k * 32), idesc_dp, k > 0);
                 umma_commit(&bars->dp_full);
@@ -195,6 +199,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 if (ok && c >= 2) ok = mbar_wait(&bars->dq_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
                 if (!ok) break;
                 tc_fence_after_sync();
+                LA_TRACE(g_trace_dq, c, 1);
                 for (int k = 0; k < 4; ++k)      // h = G S_{c-1}^T
                     umma_bf16(tmem + kDqColGt + b * 64, desc_k(aG + k * 32), desc_k(aS + k * 32), idesc_kk, k > 0);
                 for (int k = 0; k < 8; ++k)      // T = L k  (row-wise prefix sums of k inside the chunk)
@@ -205,14 +210,17 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 for (int k = 0; k < 8; ++k)      // Z += k^T 1
                     umma_bf16(tmem + kDqColS + 64, desc_mn(aK + k * 2048), desc_ones(aOnes), idesc_z, 1);
                 umma_commit(&bars->s_full);
+                LA_TRACE(g_trace_dq, c, 2);
                 ok = mbar_wait(&bars->dp_ready, c & 1, prm.status, kStatusPipeTimeout);
                 if (!ok) break;
                 tc_fence_after_sync();
+                LA_TRACE(g_trace_dq, c, 3);
                 for (int k = 0; k < 8; ++k)      // h += dP k
                     umma_bf16(tmem + kDqColGt + b * 64, desc_k(aDP + (k >> 2) * kTileBytes + (k & 3) * 32),
                               desc_mn(aK + k * 2048), idesc_kmn, 1);
                 umma_commit(&bars->dq_full[b]);
                 umma_commit(&bars->empty[s]);
+                LA_TRACE(g_trace_dq, c, 4);
             }
             if (!ok) *abort_flag = 1;
         }
@@ -224,11 +232,13 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             const int s = c % kDqStages;
             if (!mbar_wait(&bars->full[s], (c / kDqStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
+            if (t == 0) LA_TRACE(g_trace_dq, c, 5);
             if (prm.phi == LA_PHI_ELU1) {
                 phi_row_inplace(sbase + kDqOffStage + s * 3 * kTileBytes + t * 128, r7);
                 fence_proxy_async_smem();
             }
             mbar_arrive(&bars->mapped[s]);
+            if (t == 0) LA_TRACE(g_trace_dq, c, 6);
         }
     } else if (warp >= 8) {
         // --------------------------------- state conversion and dQ epilogue warps
@@ -252,13 +262,16 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             tc_fence_after_sync();
+            if (t == 0) LA_TRACE(g_trace_dq, c, 7);
             state_to_smem(tmem + kDqColS, quad, lane, sbase + kDqOffS, sZ + (c & 1) * 64, nullptr, nullptr);
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->state_ready);
+            if (t == 0) LA_TRACE(g_trace_dq, c, 8);
 
             if (!mbar_wait(&bars->dq_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
+            if (t == 0) LA_TRACE(g_trace_dq, c, 9);
             const float* zprev = sZ + ((c + 1) & 1) * 64;                // Z_{c-1}
             const uint32_t tGt = tmem + lane_base + kDqColGt + b * 64, tT = tmem + lane_base + kDqColT + b * 64;
             const bool elu = prm.phi == LA_PHI_ELU1;
@@ -323,6 +336,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             }
             tc_fence_before_sync();
             mbar_arrive(&bars->dq_drained[b]);
+            if (t == 0) LA_TRACE(g_trace_dq, c, 10);
             named_barrier(1, 128);          // Z double buffer: nobody reads Z_{c-1} past this point
         }
     } else {
@@ -340,6 +354,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             if (!mbar_wait(&bars->dp_full, c & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             tc_fence_after_sync();
+            if (warp == 3 && lane == 0) LA_TRACE(g_trace_dq, c, 11);
             uint32_t v0[32], v1[32];
             float m = 0.f;
             if (has0) tmem_ld32(src + blk0 * 32, v0);
@@ -352,6 +367,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->dp_ready);
+            if (warp == 3 && lane == 0) LA_TRACE(g_trace_dq, c, 12);
         }
     }
 
@@ -493,6 +509,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 ok = mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout);
                 if (!ok || *abort_flag) { ok = false; break; }
                 tc_fence_after_sync();
+                LA_TRACE(g_trace_dkv, i, 0);
                 for (int k = 0; k < 4; ++k)      // Ph = qh k^T
                     umma_bf16(tmem + kKvColP, desc_k(aQ + k * 32), desc_k(aK + k * 32), idesc_pp, k > 0);
                 for (int k = 0; k < 4; ++k)      // dP = G V^T
@@ -502,6 +519,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 if (ok && i >= 1) ok = mbar_wait(&bars->dkv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
                 if (!ok) break;
                 tc_fence_after_sync();
+                LA_TRACE(g_trace_dkv, i, 1);
                 for (int k = 0; k < 4; ++k)      // gk = V R_{c+1}^T
                     umma_bf16(tmem + kKvColDk, desc_k(aV + k * 32), desc_k(aR + k * 32), idesc_kk, k > 0);
                 for (int k = 0; k < 4; ++k)      // gV = k R_{c+1}
@@ -511,15 +529,18 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 for (int k = 0; k < 8; ++k)      // r += qh^T dl
                     umma_bf16(tmem + kKvColR + 64, desc_mn(aQ + k * 2048), desc_mn(aAux + k * 2048), idesc_z, 1);
                 umma_commit(&bars->r_full);
+                LA_TRACE(g_trace_dkv, i, 2);
                 ok = mbar_wait(&bars->pd_ready, i & 1, prm.status, kStatusPipeTimeout);
                 if (!ok) break;
                 tc_fence_after_sync();
+                LA_TRACE(g_trace_dkv, i, 3);
                 for (int k = 0; k < 8; ++k)      // gk += dP^T qh
                     umma_bf16(tmem + kKvColDk, desc_mn(aDP + k * 2048), desc_mn(aQ + k * 2048), idesc_mnmn, 1);
                 for (int k = 0; k < 8; ++k)      // gV += Ph^T G
                     umma_bf16(tmem + kKvColDv, desc_mn(aP + k * 2048), desc_mn(aG + k * 2048), idesc_mnmn, 1);
                 umma_commit(&bars->dkv_full);
                 umma_commit(&bars->empty[s]);
+                LA_TRACE(g_trace_dkv, i, 4);
             }
             if (!ok) *abort_flag = 1;
         }
@@ -535,6 +556,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             const float delta = __ldg(prm.dl + row);
             if (!mbar_wait(&bars->full[s], (i / kKvStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
+            if (t == 0) LA_TRACE(g_trace_dkv, i, 5);
             const uint32_t aQ = sbase + kKvOffStage + s * 4 * kTileBytes + t * 128;
 #pragma unroll
             for (int cc = 0; cc < 8; ++cc) {
@@ -557,6 +579,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             sts128(aA + ((1 ^ r7) << 4), dd, dd, dd, dd);
             fence_proxy_async_smem();
             mbar_arrive(&bars->mapped[s]);
+            if (t == 0) LA_TRACE(g_trace_dkv, i, 6);
         }
     } else if (warp >= 8) {
         // ------------------------------ state conversion and dK / dV epilogue warps
@@ -584,13 +607,16 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
 
             if (!mbar_wait(&bars->r_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
+            if (t == 0) LA_TRACE(g_trace_dkv, i, 7);
             state_to_smem(tmem + kKvColR, quad, lane, sbase + kKvOffR, sRv + (i & 1) * 64, nullptr, nullptr);
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->state_ready);
+            if (t == 0) LA_TRACE(g_trace_dkv, i, 8);
 
             if (!mbar_wait(&bars->dkv_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
+            if (t == 0) LA_TRACE(g_trace_dkv, i, 9);
             const float* rprev = sRv + ((i + 1) & 1) * 64;               // r_{c+1}
             __nv_bfloat16* dstK = prm.dK + row * kDim;
             __nv_bfloat16* dstV = prm.dV + row * kDim;
@@ -632,6 +658,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             }
             tc_fence_before_sync();
             mbar_arrive(&bars->dkv_drained);
+            if (t == 0) LA_TRACE(g_trace_dkv, i, 10);
             named_barrier(1, 128);          // r double buffer
         }
     } else {
@@ -649,6 +676,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 !mbar_wait(&bars->pd_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             tc_fence_after_sync();
+            if (warp == 3 && lane == 0) LA_TRACE(g_trace_dkv, i, 11);
             const float delta = sDelta[s * 128 + t];
             uint32_t v0[32], v1[32];
             if (has0) tmem_ld32(tmem + lane_base + kKvColP + blk0 * 32, v0);
@@ -664,6 +692,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->pd_ready);
+            if (warp == 3 && lane == 0) LA_TRACE(g_trace_dkv, i, 12);
         }
     }
 
@@ -755,3 +784,12 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
 
 }  // namespace tc
 }  // namespace la
+
+#ifdef LA_TC_TRACE
+extern "C" int la_debug_read_trace_dq(long long* out, int n) {
+    return (int)cudaMemcpyFromSymbol(out, la::tc::g_trace_dq, n * sizeof(long long));
+}
+extern "C" int la_debug_read_trace_dkv(long long* out, int n) {
+    return (int)cudaMemcpyFromSymbol(out, la::tc::g_trace_dkv, n * sizeof(long long));
+}
+#endif

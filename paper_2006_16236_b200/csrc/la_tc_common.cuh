@@ -11,6 +11,16 @@
 namespace la {
 namespace tc {
 
+// Optional pipeline trace (compile with -DLA_TC_TRACE): CTA 0 stamps clock64() per chunk and
+// event into a per-file buffer that la_debug_read_trace_*() copies out.  Compiled out otherwise.
+#ifdef LA_TC_TRACE
+#define LA_TRACE_DECL(name) __device__ long long name[512 * 32];
+#define LA_TRACE(buf, c, slot) do { if (blockIdx.x == 0 && (c) < 512) buf[(c) * 32 + (slot)] = clock64(); } while (0)
+#else
+#define LA_TRACE_DECL(name)
+#define LA_TRACE(buf, c, slot) do { } while (0)
+#endif
+
 constexpr int kChunk = 128;                  // positions per chunk = MMA M
 constexpr int kDim = 64;                     // D = M = 64: one 128-byte swizzle row
 constexpr int kTileBytes = kChunk * kDim * 2;  // one [128][64] bf16 tile
