@@ -137,6 +137,35 @@ int la_causal_backward(const la_problem* p, const void* Q, const void* K, const 
 int la_recurrent_step(const la_problem* p, const void* q, const void* k, const void* v,
                       float* S, float* Z, void* out, void* stream);
 
+/*
+ * Non-causal forward for callers that cannot allocate device memory (the paper has no
+ * counterpart: this is a deployment convenience, not part of the method).
+ *
+ * Same computation, arguments and results as la_linear_attention(), minus `ws`: the
+ * scratch for the per-split partial sums is a fixed array of LA_NOALLOC_SCRATCH_BYTES
+ * inside the library's device image.  It is meant for callers that receive only input
+ * and output buffers and may not call cudaMalloc or ask their framework for memory at
+ * that point: plugin-style integrations, code that runs after a framework has frozen its
+ * memory plan, latency-critical loops where an allocation (which can synchronise the
+ * device) is not tolerable.  The price: every GPU on which the library is loaded holds
+ * those LA_NOALLOC_SCRATCH_BYTES until the process exits, used or not.
+ *
+ *  - The call allocates and frees nothing, on the host or the device, and calls no
+ *    allocating library routine.  It always runs the general fp32-arithmetic kernels.
+ *  - Problems whose scratch need (B*H*splits*D*(M+1)*4 bytes, at most a few splits per
+ *    head) exceeds the array are rejected with LA_ERR_WORKSPACE and a message naming
+ *    both sizes; nothing is enqueued.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current) and caches it; make that first call before starting any stream capture.
+ *  - All calls on a device share the one array, which keeps the previous call's contents.
+ *    Nothing in it needs clearing between calls (each call overwrites what it reads), but
+ *    two calls whose kernels overlap on the GPU (different streams) race on it: run them
+ *    on one stream or order them with events.
+ */
+#define LA_NOALLOC_SCRATCH_BYTES (8u << 20)
+int la_linear_attention_noalloc(const la_problem* p, const void* Q, const void* K, const void* V,
+                                void* O, float* den, float* KV, float* Zs, void* stream);
+
 /* Bytes of workspace `op` needs for problem p (pure host function; 0 if none).
  * Returns 0 for invalid problems as well: the entry point reports the error. */
 size_t la_workspace_bytes(const la_problem* p, int32_t op);

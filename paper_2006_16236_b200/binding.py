@@ -20,7 +20,8 @@ LA_OP_LINEAR_FORWARD, LA_OP_LINEAR_BACKWARD, LA_OP_CAUSAL_FORWARD, LA_OP_CAUSAL_
 _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
-    "la_feature_map", "la_linear_attention", "la_linear_attention_backward", "la_causal_forward",
+    "la_feature_map", "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
+    "la_causal_forward",
     "la_causal_backward", "la_recurrent_step", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_version",
 ]
@@ -53,6 +54,7 @@ def lib() -> ctypes.CDLL:
         pp = ctypes.POINTER(la_problem)
         L.la_feature_map.argtypes = [vp, vp, i64, i32, i32, vp]
         L.la_linear_attention.argtypes = [pp] + [vp] * 7 + [vp, sz, vp]
+        L.la_linear_attention_noalloc.argtypes = [pp] + [vp] * 7 + [vp]
         L.la_linear_attention_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
         L.la_causal_forward.argtypes = [pp] + [vp] * 7 + [vp, sz, vp]
         L.la_causal_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
@@ -164,6 +166,20 @@ def la_linear_attention(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, KV=None,
     _check(lib().la_linear_attention(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(KV),
                                      _ptr(Zs), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                                      _stream(dev)))
+    return O
+
+
+def la_linear_attention_noalloc(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, KV=None, Zs=None):
+    """Non-causal forward through the entry point that uses the library's built-in scratch array.
+
+    For callers that may not allocate device memory around the call; here only the output
+    tensor is created when `O` is not passed in.  Raises LaError (LA_ERR_WORKSPACE) when the
+    problem needs more scratch than the array holds."""
+    dev = _dev(Q, K, V, O, den, KV, Zs)
+    p = _problem_of(Q, V, phi, eps)
+    O = torch.empty_like(V) if O is None else O
+    _check(lib().la_linear_attention_noalloc(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den),
+                                             _ptr(KV), _ptr(Zs), _stream(dev)))
     return O
 
 
