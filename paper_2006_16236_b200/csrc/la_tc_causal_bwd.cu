@@ -53,24 +53,26 @@ namespace {
 // equal terms; there the scores are centred before rounding, dP_ij - m_i with
 // m_i = dP_i0, and m_i T_i is added back in fp32 (a row constant times the prefix sum).
 //
-// Warps 0-7: dP post-processing (two warps per TMEM quadrant), 8-11: state
-// conversion and dQ epilogue, 12-15: phi(K), 16: TMA, 17: MMA.
+// Warps 0-7 ("score/epilogue" warps, two per TMEM quadrant: the pair shares the 128 rows
+// of the quadrant, one warp per 32-column half): mask + round dP of chunk c+1, then the dQ
+// epilogue of chunk c.  Warps 8-11: phi(K), phi(Q) in place and the state conversion.
+// Warp 12: TMA.  Warp 13: MMA issue.
 // ===========================================================================
-constexpr int kDqStages = 3;
-constexpr int kDqThreads = 576;
+constexpr int kDqStages = 2;
+constexpr int kDqThreads = 448;
 constexpr uint32_t kDqColDP = 0;       // 128
-constexpr uint32_t kDqColGt = 128;     // 2 x 64: gt of even / odd chunks
+constexpr uint32_t kDqColGt = 128;     // 2 x 64: h of even / odd chunks
 constexpr uint32_t kDqColT = 256;      // 2 x 64: T = L k of even / odd chunks
 constexpr uint32_t kDqColS = 384;      // 64 + 16
 
-constexpr uint32_t kDqOffStage = 0;                                        // kDqStages x {K, V, G}
-constexpr uint32_t kDqOffDP = kDqOffStage + kDqStages * 3 * kTileBytes;    // 2 tiles
+constexpr uint32_t kDqOffStage = 0;                                        // kDqStages x {K, V, G, Q}
+constexpr uint32_t kDqOffDP = kDqOffStage + kDqStages * 4 * kTileBytes;    // 2 tiles
 constexpr uint32_t kDqOffL = kDqOffDP + 2 * kTileBytes;                    // 2 tiles: lower-triangular ones
 constexpr uint32_t kDqOffS = kDqOffL + 2 * kTileBytes;                     // bf16 S tile
 constexpr uint32_t kDqOffOnes = kDqOffS + kDim * 128;
-constexpr uint32_t kDqOffZ = kDqOffOnes + 1024;                            // fp32 [2][64]
-constexpr uint32_t kDqOffM = kDqOffZ + 512;                                // fp32 [128]: row offsets m_i of the first chunk
-constexpr uint32_t kDqOffBar = kDqOffM + 512;
+constexpr uint32_t kDqOffZ = kDqOffOnes + 1024;                            // fp32 [3][64]
+constexpr uint32_t kDqOffX = kDqOffZ + 768;                                // fp32 [2 halves][128][2]: row-pair exchange
+constexpr uint32_t kDqOffBar = kDqOffX + 2048;
 constexpr uint32_t kDqSmemBytes = kDqOffBar + 256 + 1024;
 
 struct DqBarriers {
@@ -82,7 +84,6 @@ struct DqBarriers {
 };
 
 struct DqParams {
-    const __nv_bfloat16* Q;     // raw queries (phi and phi' in the epilogue)
     float* dn;                  // out: dn_i = q_i . Z_i + eps per row, for the reverse sweep
     float* dl;                  // out: dl_i = -(G_i . O_i) per row, for the reverse sweep
     __nv_bfloat16* dQ;
@@ -96,13 +97,14 @@ struct DqParams {
 
 __global__ void __launch_bounds__(kDqThreads, 1)
 causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
-                     const __grid_constant__ CUtensorMap mapG, const DqParams prm) {
+                     const __grid_constant__ CUtensorMap mapG, const __grid_constant__ CUtensorMap mapQ,
+                     const DqParams prm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
     DqBarriers* bars = reinterpret_cast<DqBarriers*>(smem + kDqOffBar);
     float* sZ = reinterpret_cast<float*>(smem + kDqOffZ);
-    float* sM = reinterpret_cast<float*>(smem + kDqOffM);
+    float* sX = reinterpret_cast<float*>(smem + kDqOffX);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int seg = blockIdx.x % prm.nseg;
@@ -114,12 +116,12 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     if (tid == 0) {
         for (int s = 0; s < kDqStages; ++s) {
             mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], 1);
+            mbar_init(&bars->empty[s], 1 + 256);      // MMA commit + the epilogue warps (they read phi(Q) rows)
             mbar_init(&bars->mapped[s], 128);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&bars->dq_full[b], 1);
-            mbar_init(&bars->dq_drained[b], 128);
+            mbar_init(&bars->dq_drained[b], 256);
         }
         mbar_init(&bars->dp_full, 1);
         mbar_init(&bars->dp_ready, 256);
@@ -128,13 +130,13 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         bars->abort_flag = 0;
         fence_mbar_init();
     }
-    if (warp == 17) {
+    if (warp == 13) {
         __syncwarp();
         tmem_alloc(&bars->tmem_base, 512);
         tmem_relinquish();
     }
     // the score tile is zero right of the diagonal for ever: clear it once
-    for (uint32_t i = tid; i < 2 * kTileBytes / 16; i += kDqThreads) sts128(sbase + kDqOffDP + i * 16, 0u, 0u, 0u, 0u);
+    for (uint32_t i = tid; i < 2 * kTileBytes / 16; i += kDqThreads) sts128(smem + kDqOffDP + i * 16, 0u, 0u, 0u, 0u);
     for (int i = tid; i < 256; i += kDqThreads) reinterpret_cast<uint32_t*>(smem + kDqOffOnes)[i] = 0x3F803F80u;
     if (tid < 128) {        // L[i][j] = 1 for j <= i
         const uint32_t r7 = tid & 7;
@@ -145,7 +147,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 const int col = cc * 8 + 2 * j;
                 w[j] = (col <= tid ? 0x3F80u : 0u) | (col + 1 <= tid ? 0x3F800000u : 0u);
             }
-            sts128(sbase + kDqOffL + (cc >> 3) * kTileBytes + tid * 128 + (((cc & 7) ^ r7) << 4), w[0], w[1], w[2], w[3]);
+            sts128(smem + kDqOffL + (cc >> 3) * kTileBytes + tid * 128 + (((cc & 7) ^ r7) << 4), w[0], w[1], w[2], w[3]);
         }
     }
     fence_proxy_async_smem();
@@ -155,10 +157,10 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
-    if (warp == 16) {
+    if (warp == 12) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG);
+            prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG); prefetch_tensormap(&mapQ);
             for (int c = 0; c < L; ++c) {
                 const int s = c % kDqStages;
                 if (c >= kDqStages && !mbar_wait(&bars->empty[s], ((c / kDqStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
@@ -166,15 +168,16 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                     break;
                 }
                 if (*abort_flag) break;
-                uint8_t* st = smem + kDqOffStage + s * 3 * kTileBytes;
+                uint8_t* st = smem + kDqOffStage + s * 4 * kTileBytes;
                 const int y = (int)(row0 + (int64_t)c * kChunk);
-                mbar_arrive_expect_tx(&bars->full[s], 3 * kTileBytes);
-                tma_load_2d(st, &mapK, 0, y, &bars->full[s]);
+                mbar_arrive_expect_tx(&bars->full[s], 4 * kTileBytes);
                 tma_load_2d(st + kTileBytes, &mapV, 0, y, &bars->full[s]);
                 tma_load_2d(st + 2 * kTileBytes, &mapG, 0, y, &bars->full[s]);
+                tma_load_2d(st, &mapK, 0, y, &bars->full[s]);
+                tma_load_2d(st + 3 * kTileBytes, &mapQ, 0, y, &bars->full[s]);
             }
         }
-    } else if (warp == 17) {
+    } else if (warp == 13) {
         // ------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             const uint32_t idesc_dp = umma_idesc_bf16(128, 128, 0, 0);
@@ -187,29 +190,31 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             bool ok = true;
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kDqStages, b = c & 1;
-                const uint32_t aK = sbase + kDqOffStage + s * 3 * kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
-                ok = mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout);
+                const uint32_t aK = sbase + kDqOffStage + s * 4 * kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
+                // dP = G V^T needs only the raw tiles (the dP tile in TMEM is free: dp_ready(c-1) was awaited)
+                ok = mbar_wait(&bars->full[s], (c / kDqStages) & 1, prm.status, kStatusTmaTimeout);
                 if (!ok || *abort_flag) { ok = false; break; }
                 tc_fence_after_sync();
                 LA_TRACE(g_trace_dq, c, 0);
-                for (int k = 0; k < 4; ++k)      // dP = G V^T (the dP tile in TMEM is free: dp_ready(c-1) was awaited)
+                for (int k = 0; k < 4; ++k)
                     umma_bf16(tmem + kDqColDP, desc_k(aG + k * 32), desc_k(aV + k * 32), idesc_dp, k > 0);
                 umma_commit(&bars->dp_full);
-                ok = mbar_wait(&bars->state_ready, c & 1, prm.status, kStatusPipeTimeout);
+                ok = mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout) &&
+                     mbar_wait(&bars->state_ready, c & 1, prm.status, kStatusPipeTimeout);
                 if (ok && c >= 2) ok = mbar_wait(&bars->dq_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
                 if (!ok) break;
                 tc_fence_after_sync();
                 LA_TRACE(g_trace_dq, c, 1);
                 for (int k = 0; k < 4; ++k)      // h = G S_{c-1}^T
                     umma_bf16(tmem + kDqColGt + b * 64, desc_k(aG + k * 32), desc_k(aS + k * 32), idesc_kk, k > 0);
-                for (int k = 0; k < 8; ++k)      // T = L k  (row-wise prefix sums of k inside the chunk)
-                    umma_bf16(tmem + kDqColT + b * 64, desc_k(aL + (k >> 2) * kTileBytes + (k & 3) * 32),
-                              desc_mn(aK + k * 2048), idesc_kmn, k > 0);
                 for (int k = 0; k < 8; ++k)      // S += k^T V
                     umma_bf16(tmem + kDqColS, desc_mn(aK + k * 2048), desc_mn(aV + k * 2048), idesc_s, 1);
                 for (int k = 0; k < 8; ++k)      // Z += k^T 1
                     umma_bf16(tmem + kDqColS + 64, desc_mn(aK + k * 2048), desc_ones(aOnes), idesc_z, 1);
                 umma_commit(&bars->s_full);
+                for (int k = 0; k < 8; ++k)      // T = L k  (row-wise prefix sums of k inside the chunk)
+                    umma_bf16(tmem + kDqColT + b * 64, desc_k(aL + (k >> 2) * kTileBytes + (k & 3) * 32),
+                              desc_mn(aK + k * 2048), idesc_kmn, k > 0);
                 LA_TRACE(g_trace_dq, c, 2);
                 ok = mbar_wait(&bars->dp_ready, c & 1, prm.status, kStatusPipeTimeout);
                 if (!ok) break;
@@ -224,137 +229,61 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             }
             if (!ok) *abort_flag = 1;
         }
-    } else if (warp >= 12) {
-        // ---------------------------------------------------- prep warps: phi(K)
-        const int t = tid - 12 * 32;
+    } else if (warp >= 8) {
+        // ---------------- operand warps: phi(K), phi(Q) in place, then the state conversion
+        const int quad = warp - 8;
+        const int t = tid - 8 * 32;
         const uint32_t r7 = t & 7;
-        for (int c = 0; c < L; ++c) {
+        const float* init = prm.init ? prm.init + (bh * prm.nseg + seg) * (int64_t)kStateFloats : nullptr;
+        state_init(tmem + kDqColS, quad, lane, smem + kDqOffS, sZ + 2 * 64, init);      // "chunk -1" -> Z buffer 2
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        mbar_arrive(&bars->state_ready);
+        auto map_chunk = [&](int c) -> bool {
             const int s = c % kDqStages;
-            if (!mbar_wait(&bars->full[s], (c / kDqStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
-            if (*abort_flag) break;
+            if (!mbar_wait(&bars->full[s], (c / kDqStages) & 1, prm.status, kStatusTmaTimeout)) return false;
             if (t == 0) LA_TRACE(g_trace_dq, c, 5);
             if (prm.phi == LA_PHI_ELU1) {
-                phi_row_inplace(sbase + kDqOffStage + s * 3 * kTileBytes + t * 128, r7);
+                uint8_t* rowK = smem + kDqOffStage + s * 4 * kTileBytes + t * 128;
+                phi_row_inplace(rowK, r7);
+                phi_row_inplace(rowK + 3 * kTileBytes, r7);
                 fence_proxy_async_smem();
             }
             mbar_arrive(&bars->mapped[s]);
             if (t == 0) LA_TRACE(g_trace_dq, c, 6);
-        }
-    } else if (warp >= 8) {
-        // --------------------------------- state conversion and dQ epilogue warps
-        const int quad = warp - 8;
-        const int t = quad * 32 + lane;
-        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        const float* init = prm.init ? prm.init + (bh * prm.nseg + seg) * (int64_t)kStateFloats : nullptr;
-        state_init(tmem + kDqColS, quad, lane, sbase + kDqOffS, sZ + 64, init);      // "chunk -1" -> Z buffer 1
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
-        named_barrier(1, 128);
-        mbar_arrive(&bars->state_ready);
-
-        for (int c = 0; c < L; ++c) {
-            const int b = c & 1;
-            const int64_t row = row0 + (int64_t)c * kChunk + t;
-            uint4 qraw[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) qraw[j] = ldg128(prm.Q + row * kDim + j * 8);
-
-            if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
-            if (*abort_flag) break;
+            return true;
+        };
+        bool ok = map_chunk(0);
+        for (int c = 0; c < L && ok; ++c) {
+            if (c + 1 < L) ok = map_chunk(c + 1);
+            if (!ok || *abort_flag) { ok = false; break; }
+            if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
             tc_fence_after_sync();
             if (t == 0) LA_TRACE(g_trace_dq, c, 7);
-            state_to_smem(tmem + kDqColS, quad, lane, sbase + kDqOffS, sZ + (c & 1) * 64, nullptr, nullptr);
+            // Z_c goes to buffer c % 3: the epilogue of chunk c still reads Z_{c-1}, and Z_{c-2}'s
+            // readers are done (the MMA warp waited for that epilogue before issuing chunk c)
+            state_to_smem(tmem + kDqColS, quad, lane, smem + kDqOffS, sZ + (c % 3) * 64, nullptr, nullptr);
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->state_ready);
             if (t == 0) LA_TRACE(g_trace_dq, c, 8);
-
-            if (!mbar_wait(&bars->dq_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
-            tc_fence_after_sync();
-            if (t == 0) LA_TRACE(g_trace_dq, c, 9);
-            const float* zprev = sZ + ((c + 1) & 1) * 64;                // Z_{c-1}
-            const uint32_t tGt = tmem + lane_base + kDqColGt + b * 64, tT = tmem + lane_base + kDqColT + b * 64;
-            const bool elu = prm.phi == LA_PHI_ELU1;
-            const float m = (c_begin + c == 0) ? sM[t] : 0.f;          // centring offset of the first chunk
-            // pass 1: q . h and q . Z_i
-            float qg = 0.f, qz = 0.f;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t g[32], tt[32];
-                tmem_ld32(tGt + h * 32, g);
-                tmem_ld32(tT + h * 32, tt);
-                tmem_ld_wait();
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    const uint4 qv = qraw[h * 4 + cc];
-                    const uint32_t qq[4] = {qv.x, qv.y, qv.z, qv.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int d = h * 32 + cc * 8 + 2 * j;
-                        const float x0 = bf16_lo(qq[j]), x1 = bf16_hi(qq[j]);
-                        const float q0 = elu ? phi_fast(x0) : x0, q1 = elu ? phi_fast(x1) : x1;
-                        qg = fmaf(q0, fmaf(m, __uint_as_float(tt[cc * 8 + 2 * j]), __uint_as_float(g[cc * 8 + 2 * j])),
-                                  fmaf(q1, fmaf(m, __uint_as_float(tt[cc * 8 + 2 * j + 1]), __uint_as_float(g[cc * 8 + 2 * j + 1])), qg));
-                        qz = fmaf(q0, zprev[d] + __uint_as_float(tt[cc * 8 + 2 * j]),
-                                  fmaf(q1, zprev[d + 1] + __uint_as_float(tt[cc * 8 + 2 * j + 1]), qz));
-                    }
-                }
-            }
-            const float dn = qz + prm.eps;
-            const float inv = 1.f / dn;
-            const float delta = -qg * inv;          // = -(G_i . O_i)
-            prm.dn[row] = dn;
-            prm.dl[row] = delta;
-            // pass 2: gq = (h + delta Z_i) / dn, chained with phi'(Q)
-            __nv_bfloat16* dst = prm.dQ + row * kDim;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t g[32], tt[32];
-                tmem_ld32(tGt + h * 32, g);
-                tmem_ld32(tT + h * 32, tt);
-                tmem_ld_wait();
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    const uint4 qv = qraw[h * 4 + cc];
-                    const uint32_t qq[4] = {qv.x, qv.y, qv.z, qv.w};
-                    uint32_t outp[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int d = h * 32 + cc * 8 + 2 * j;
-                        const float t0 = __uint_as_float(tt[cc * 8 + 2 * j]), t1 = __uint_as_float(tt[cc * 8 + 2 * j + 1]);
-                        float g0 = inv * fmaf(delta, zprev[d] + t0, fmaf(m, t0, __uint_as_float(g[cc * 8 + 2 * j])));
-                        float g1 = inv * fmaf(delta, zprev[d + 1] + t1, fmaf(m, t1, __uint_as_float(g[cc * 8 + 2 * j + 1])));
-                        if (elu) {
-                            const float x0 = bf16_lo(qq[j]), x1 = bf16_hi(qq[j]);
-                            g0 *= x0 > 0.f ? 1.f : phi_fast(x0);
-                            g1 *= x1 > 0.f ? 1.f : phi_fast(x1);
-                        }
-                        outp[j] = pack_bf16x2(g0, g1);
-                    }
-                    stg128(dst + h * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
-                }
-            }
-            tc_fence_before_sync();
-            mbar_arrive(&bars->dq_drained[b]);
-            if (t == 0) LA_TRACE(g_trace_dq, c, 10);
-            named_barrier(1, 128);          // Z double buffer: nobody reads Z_{c-1} past this point
         }
+        if (!ok) *abort_flag = 1;
     } else {
-        // -------------------------------------------------- dP post-processing warps
+        // ------------------------------------------------ score / epilogue warps
         const int quad = warp & 3, half = warp >> 2;
-        const int t = quad * 32 + lane;
+        const int t = quad * 32 + lane;                     // chunk row = TMEM lane
         const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        // blocks of this warp: half 0 -> {0, 2}, half 1 -> {1, 3}, restricted to blk <= quad
+        // score blocks of this warp: half 0 -> {0, 2}, half 1 -> {1, 3}, restricted to blk <= quad
         const int blk0 = half, blk1 = half + 2;
         const bool has0 = blk0 <= quad, has1 = blk1 <= quad;
-        const uint32_t tile_row = sbase + kDqOffDP + t * 128;
+        uint8_t* tile_row = smem + kDqOffDP + t * 128;
         const uint32_t src = tmem + lane_base + kDqColDP;
-        for (int c = 0; c < L; ++c) {
-            if (!mbar_wait(&bars->dp_full, c & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
-            if (*abort_flag) break;
-            tc_fence_after_sync();
-            if (warp == 3 && lane == 0) LA_TRACE(g_trace_dq, c, 11);
+        const bool elu = prm.phi == LA_PHI_ELU1;
+        float m_prev = 0.f;                                 // centring offset of the chunk whose epilogue is pending
+
+        auto process_scores = [&](int c) -> float {         // chunk c: TMEM dP -> masked bf16 tile
             uint32_t v0[32], v1[32];
             float m = 0.f;
             if (has0) tmem_ld32(src + blk0 * 32, v0);
@@ -363,17 +292,106 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             tmem_ld_wait();
             if (has0) score_block_store(v0, tile_row, r7, blk0, blk0 == quad, lane, -m);
             if (has1) score_block_store(v1, tile_row, r7, blk1, blk1 == quad, lane, -m);
-            if (c_begin + c == 0 && half == 0) sM[t] = m;
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->dp_ready);
-            if (warp == 3 && lane == 0) LA_TRACE(g_trace_dq, c, 12);
+            return m;
+        };
+
+        bool ok = mbar_wait(&bars->dp_full, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
+        if (ok) {
+            tc_fence_after_sync();
+            m_prev = process_scores(0);
         }
+        for (int c = 0; c < L && ok; ++c) {
+            const int s = c % kDqStages, b = c & 1;
+            float m_next = 0.f;
+            if (c + 1 < L) {            // scores of the next chunk first: its MMAs then overlap this chunk's epilogue
+                if (!mbar_wait(&bars->dp_full, (c + 1) & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
+                tc_fence_after_sync();
+                if (warp == 3 && lane == 0) LA_TRACE(g_trace_dq, c + 1, 11);
+                m_next = process_scores(c + 1);
+                if (warp == 3 && lane == 0) LA_TRACE(g_trace_dq, c + 1, 12);
+            }
+            // ---- epilogue of chunk c: this thread owns columns [32 half, 32 half + 32) of row t
+            if (!mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout)) { ok = false; break; }
+            uint32_t qv[4][4];                               // phi(Q) row, logical chunks 4 half .. 4 half + 3
+            {
+                const uint8_t* rowQ = smem + kDqOffStage + s * 4 * kTileBytes + 3 * kTileBytes + t * 128;
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) lds128(rowQ + (((half * 4 + cc) ^ r7) << 4), qv[cc]);
+            }
+            if (!mbar_wait(&bars->dq_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
+            if (*abort_flag) { ok = false; break; }
+            tc_fence_after_sync();
+            if (tid == 0) LA_TRACE(g_trace_dq, c, 9);
+            const float* zprev = sZ + ((c + 2) % 3) * 64 + half * 32;           // Z_{c-1}
+            uint32_t g[32], tt[32];
+            tmem_ld32(tmem + lane_base + kDqColGt + b * 64 + half * 32, g);
+            tmem_ld32(tmem + lane_base + kDqColT + b * 64 + half * 32, tt);
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            mbar_arrive(&bars->dq_drained[b]);              // both accumulators are in registers now
+            mbar_arrive(&bars->empty[s]);                   // and so is this thread's part of phi(Q)
+            const float m = m_prev;
+            float qg4[4] = {0.f, 0.f, 0.f, 0.f}, qz4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int e = cc * 8 + 2 * j;
+                    const float q0 = bf16_lo(qv[cc][j]), q1 = bf16_hi(qv[cc][j]);
+                    const float t0 = __uint_as_float(tt[e]), t1 = __uint_as_float(tt[e + 1]);
+                    const float h0 = fmaf(m, t0, __uint_as_float(g[e])), h1 = fmaf(m, t1, __uint_as_float(g[e + 1]));
+                    const float z0 = zprev[e] + t0, z1 = zprev[e + 1] + t1;
+                    g[e] = __float_as_uint(h0); g[e + 1] = __float_as_uint(h1);
+                    tt[e] = __float_as_uint(z0); tt[e + 1] = __float_as_uint(z1);
+                    qg4[j] = fmaf(q0, h0, fmaf(q1, h1, qg4[j]));
+                    qz4[j] = fmaf(q0, z0, fmaf(q1, z1, qz4[j]));
+                }
+            // combine the two halves of the row
+            float* xch = sX + (half * 128 + t) * 2;
+            xch[0] = (qg4[0] + qg4[1]) + (qg4[2] + qg4[3]);
+            xch[1] = (qz4[0] + qz4[1]) + (qz4[2] + qz4[3]);
+            named_barrier(2 + quad, 64);
+            const float* other = sX + ((half ^ 1) * 128 + t) * 2;
+            const float qg = xch[0] + other[0], qz = xch[1] + other[1];
+            named_barrier(2 + quad, 64);                    // the exchange slots may be rewritten after this
+            const float dn = qz + prm.eps;
+            const float inv = 1.f / dn;
+            const float delta = -qg * inv;                  // = -(G_i . O_i)
+            const int64_t row = row0 + (int64_t)c * kChunk + t;
+            if (half == 0) {
+                prm.dn[row] = dn;
+                prm.dl[row] = delta;
+            }
+            __nv_bfloat16* dst = prm.dQ + row * kDim + half * 32;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t outp[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int e = cc * 8 + 2 * j;
+                    float g0 = inv * fmaf(delta, __uint_as_float(tt[e]), __uint_as_float(g[e]));
+                    float g1 = inv * fmaf(delta, __uint_as_float(tt[e + 1]), __uint_as_float(g[e + 1]));
+                    if (elu) {          // phi'(x) from phi(x): 1 where x > 0 (phi > 1), else phi(x)
+                        const float q0 = bf16_lo(qv[cc][j]), q1 = bf16_hi(qv[cc][j]);
+                        g0 *= q0 > 1.f ? 1.f : q0;
+                        g1 *= q1 > 1.f ? 1.f : q1;
+                    }
+                    outp[j] = pack_bf16x2(g0, g1);
+                }
+                stg128(dst + cc * 8, outp[0], outp[1], outp[2], outp[3]);
+            }
+            if (tid == 0) LA_TRACE(g_trace_dq, c, 10);
+            m_prev = m_next;
+        }
+        if (!ok) *abort_flag = 1;
     }
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 17) {
+    if (warp == 13) {
         __syncwarp();
         tmem_dealloc(tmem, 512);
     }
@@ -462,7 +480,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         tmem_alloc(&bars->tmem_base, 512);
         tmem_relinquish();
     }
-    for (uint32_t i = tid; i < 4 * kTileBytes / 16; i += kKvThreads) sts128(sbase + kKvOffP + i * 16, 0u, 0u, 0u, 0u);
+    for (uint32_t i = tid; i < 4 * kTileBytes / 16; i += kKvThreads) sts128(smem + kKvOffP + i * 16, 0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
@@ -557,23 +575,16 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             if (!mbar_wait(&bars->full[s], (i / kKvStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             if (t == 0) LA_TRACE(g_trace_dkv, i, 5);
-            const uint32_t aQ = sbase + kKvOffStage + s * 4 * kTileBytes + t * 128;
-#pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {
-                uint32_t v[4];
-                lds128(aQ + ((cc ^ r7) << 4), v);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float x0 = bf16_lo(v[j]), x1 = bf16_hi(v[j]);
-                    v[j] = pack_bf16x2((elu ? phi_fast(x0) : x0) * inv, (elu ? phi_fast(x1) : x1) * inv);
-                }
-                sts128(aQ + ((cc ^ r7) << 4), v[0], v[1], v[2], v[3]);
-            }
-            if (elu) phi_row_inplace(aQ + kTileBytes, r7);
+            uint8_t* rowQ = smem + kKvOffStage + s * 4 * kTileBytes + t * 128;
+            if (elu) map_row_inplace<true>(rowQ, r7, inv); else map_row_inplace<false>(rowQ, r7, inv);
+            if (t == 0) LA_TRACE(g_trace_dkv, i, 13);
+            if (elu) phi_row_inplace(rowQ + kTileBytes, r7);
+            if (t == 0) LA_TRACE(g_trace_dkv, i, 14);
             sDelta[s * 128 + t] = delta;
             // the single dl column tile is an operand of the previous chunk's state MMAs
             if (i >= 1 && !mbar_wait(&bars->r_full, (i - 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
-            const uint32_t aA = sbase + kKvOffAux + t * 128;
+            if (t == 0) LA_TRACE(g_trace_dkv, i, 15);
+            uint8_t* aA = smem + kKvOffAux + t * 128;
             const uint32_t dd = pack_bf16x2(delta, delta);
             sts128(aA + ((0 ^ r7) << 4), dd, dd, dd, dd);
             sts128(aA + ((1 ^ r7) << 4), dd, dd, dd, dd);
@@ -588,7 +599,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const float* init = prm.init ? prm.init + (bh * prm.nseg + seg) * (int64_t)kStateFloats : nullptr;
-        state_init(tmem + kKvColR, quad, lane, sbase + kKvOffR, sRv + 64, init);      // "iteration -1" -> buffer 1
+        state_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, init);      // "iteration -1" -> buffer 1
         fence_proxy_async_smem();
         tc_fence_before_sync();
         named_barrier(1, 128);
@@ -600,15 +611,13 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             uint32_t kf[8][4];                      // phi(K) row, logical chunk order
-            const uint32_t aKrow = sbase + kKvOffStage + s * 4 * kTileBytes + kTileBytes + t * 128;
-#pragma unroll
-            for (int cc = 0; cc < 8; ++cc) lds128(aKrow + ((cc ^ r7) << 4), kf[cc]);
+            load_row(smem + kKvOffStage + s * 4 * kTileBytes + kTileBytes + t * 128, r7, kf);
             mbar_arrive(&bars->empty[s]);
 
             if (!mbar_wait(&bars->r_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
             if (t == 0) LA_TRACE(g_trace_dkv, i, 7);
-            state_to_smem(tmem + kKvColR, quad, lane, sbase + kKvOffR, sRv + (i & 1) * 64, nullptr, nullptr);
+            state_to_smem(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + (i & 1) * 64, nullptr, nullptr);
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->state_ready);
@@ -669,7 +678,8 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const int blk0 = half, blk1 = half + 2;
         const bool has0 = blk0 <= quad, has1 = blk1 <= quad;
-        const uint32_t rowP = sbase + kKvOffP + t * 128, rowDP = sbase + kKvOffDP + t * 128;
+        uint8_t* rowP = smem + kKvOffP + t * 128;
+        uint8_t* rowDP = smem + kKvOffDP + t * 128;
         for (int i = 0; i < L; ++i) {
             const int s = i % kKvStages;
             if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout) ||
@@ -747,7 +757,6 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     // forward sweep: dQ, and dn_i, dl_i for the reverse sweep
     if (int rc = segment_states(p, sg, mK, mV, nullptr, nullptr, rec_s, /*reverse=*/false, st)) return rc;
     DqParams a;
-    a.Q = (const __nv_bfloat16*)Q;
     a.dn = dn;
     a.dl = dl;
     a.dQ = (__nv_bfloat16*)dQ;
@@ -759,7 +768,7 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.nseg = sg.nseg;
     a.eps = p.eps;
     a.phi = p.phi;
-    causal_bwd_dq_kernel<<<grid, kDqThreads, kDqSmemBytes, st>>>(mK, mV, mG, a);
+    causal_bwd_dq_kernel<<<grid, kDqThreads, kDqSmemBytes, st>>>(mK, mV, mG, mQ, a);
     LA_LAUNCHED();
 
     // reverse sweep: dK, dV

@@ -180,9 +180,9 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             if (!mbar_wait(&bars->full[s], (c / kStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             if (prm.phi == LA_PHI_ELU1) {
-                const uint32_t aQ = sbase + kOffStage + s * 3 * kTileBytes + t * 128;
-                phi_row_inplace(aQ, r7);
-                phi_row_inplace(aQ + kTileBytes, r7);
+                uint8_t* rowQ = smem + kOffStage + s * 3 * kTileBytes + t * 128;
+                phi_row_inplace(rowQ, r7);
+                phi_row_inplace(rowQ + kTileBytes, r7);
                 fence_proxy_async_smem();
             }
             mbar_arrive(&bars->mapped[s]);
@@ -199,32 +199,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         for (int i = tid; i < 256; i += 128) reinterpret_cast<uint32_t*>(smem + kOffOnes)[i] = 0x3F803F80u;
         {
             const float* init = prm.init ? prm.init + (bh * prm.nseg + seg) * (int64_t)kStateFloats : nullptr;
-            uint32_t v[32];
-            float z = 0.f;
-            for (int h = 0; h < 2; ++h) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    v[j] = (init && owns_state_row) ? __float_as_uint(init[d_row * kDim + h * 32 + j]) : 0u;
-                tmem_st32(tmem + lane_base + kColS + h * 32, v);
-                if (owns_state_row) {
-#pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        const int chunk = h * 4 + cc;
-                        sts128(sbase + kOffS + d_row * 128 + ((chunk ^ (d_row & 7)) << 4),
-                               pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
-                               pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
-                               pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
-                               pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
-                    }
-                }
-            }
-            if (init && owns_state_row) z = init[kDim * kDim + d_row];
-            uint32_t zz[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) zz[j] = __float_as_uint(z);
-            tmem_st16(tmem + lane_base + kColS + 64, zz);
-            tmem_st_wait();
-            if (owns_state_row) sZ[d_row] = z;
+            state_init(tmem + kColS, warp, lane, smem + kOffS, sZ, init);
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
@@ -233,7 +208,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 
         for (int c = 0; c < L; ++c) {
             const int s = c % kStages, b = c & 1;
-            const uint32_t aQrow = sbase + kOffStage + s * 3 * kTileBytes + t * 128;
+            const uint8_t* rowQ = smem + kOffStage + s * 3 * kTileBytes + t * 128;
             if (!mbar_wait(&bars->mapped[s], (c / kStages) & 1, prm.status, kStatusPipeTimeout) ||
                 !mbar_wait(&bars->p_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
@@ -241,13 +216,16 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 
             // q . Z_{c-1} on the rounded features the MMA consumed
             float qz = 0.f;
+            {
+                uint32_t qv[8][4];
+                load_row(rowQ, r7, qv);
+                float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {
-                uint32_t v[4];
-                lds128(aQrow + ((cc ^ r7) << 4), v);
-                const float* zp = sZ + cc * 8;
+                for (int cc = 0; cc < 8; ++cc)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) qz = fmaf(bf16_lo(v[j]), zp[2 * j], fmaf(bf16_hi(v[j]), zp[2 * j + 1], qz));
+                    for (int j = 0; j < 4; ++j)
+                        part[j] = fmaf(bf16_lo(qv[cc][j]), sZ[cc * 8 + 2 * j], fmaf(bf16_hi(qv[cc][j]), sZ[cc * 8 + 2 * j + 1], part[j]));
+                qz = (part[0] + part[1]) + (part[2] + part[3]);
             }
 
             // P: TMEM -> mask -> bf16 -> swizzled smem (K-major A operand of P V), row sums
@@ -274,7 +252,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 #pragma unroll
                     for (int j = 0; j < 16; ++j) packed[j] = 0u;
                 }
-                const uint32_t tile = sbase + kOffP + (blk >> 1) * kTileBytes + t * 128;
+                uint8_t* tile = smem + kOffP + (blk >> 1) * kTileBytes + t * 128;
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     const int chunk = (blk & 1) * 4 + cc;
@@ -305,7 +283,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     const int chunk = h * 4 + cc;
-                    sts128(sbase + kOffO + t * 128 + ((chunk ^ r7) << 4),
+                    sts128(smem + kOffO + t * 128 + ((chunk ^ r7) << 4),
                            pack_bf16x2(__uint_as_float(v[cc * 8 + 0]) * inv, __uint_as_float(v[cc * 8 + 1]) * inv),
                            pack_bf16x2(__uint_as_float(v[cc * 8 + 2]) * inv, __uint_as_float(v[cc * 8 + 3]) * inv),
                            pack_bf16x2(__uint_as_float(v[cc * 8 + 4]) * inv, __uint_as_float(v[cc * 8 + 5]) * inv),
@@ -314,37 +292,11 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             }
 
             // state S_c, Z_c: TMEM (fp32) -> bf16 B operand for the next chunk, fp32 Z for q.Z
-            const bool last = (c == L - 1);
-            const bool emit_final = last && (seg == prm.nseg - 1) && prm.S_out;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t v[32];
-                tmem_ld32(tmem + lane_base + kColS + h * 32, v);
-                tmem_ld_wait();
-                if (owns_state_row) {
-#pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        const int chunk = h * 4 + cc;
-                        sts128(sbase + kOffS + d_row * 128 + ((chunk ^ (d_row & 7)) << 4),
-                               pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
-                               pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
-                               pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
-                               pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
-                    }
-                    if (emit_final) {
-                        float* dst = prm.S_out + bh * (int64_t)(kDim * kDim) + d_row * kDim + h * 32;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) dst[j] = __uint_as_float(v[j]);
-                    }
-                }
-            }
             {
-                const float z = __uint_as_float(tmem_ld1(tmem + lane_base + kColS + 64));
-                tmem_ld_wait();
-                if (owns_state_row) {
-                    sZ[d_row] = z;
-                    if (last && (seg == prm.nseg - 1) && prm.Z_out) prm.Z_out[bh * kDim + d_row] = z;
-                }
+                const bool fin = (c == L - 1) && (seg == prm.nseg - 1);
+                state_to_smem(tmem + kColS, warp, lane, smem + kOffS, sZ,
+                              fin && prm.S_out ? prm.S_out + bh * (int64_t)(kDim * kDim) : nullptr,
+                              fin && prm.Z_out ? prm.Z_out + bh * kDim : nullptr);
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();

@@ -54,28 +54,45 @@ __device__ __forceinline__ float phi_fast(float x) {
     return x > 0.f ? x + 1.f : e;
 }
 
-__device__ __forceinline__ void phi_row_inplace(uint32_t row_base, uint32_t r7) {
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        // elementwise, so the logical order is irrelevant; visiting chunk c ^ r7 keeps the
-        // eight rows of a quarter-warp on eight different bank groups
-        const uint32_t addr = row_base + ((c ^ r7) << 4);
-        uint32_t v0, v1, v2, v3;
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(addr));
-        v0 = sm100::pack_bf16x2(phi_fast(sm100::bf16_lo(v0)), phi_fast(sm100::bf16_hi(v0)));
-        v1 = sm100::pack_bf16x2(phi_fast(sm100::bf16_lo(v1)), phi_fast(sm100::bf16_hi(v1)));
-        v2 = sm100::pack_bf16x2(phi_fast(sm100::bf16_lo(v2)), phi_fast(sm100::bf16_hi(v2)));
-        v3 = sm100::pack_bf16x2(phi_fast(sm100::bf16_lo(v3)), phi_fast(sm100::bf16_hi(v3)));
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v0), "r"(v1), "r"(v2), "r"(v3) : "memory");
-    }
+// Shared-memory accesses of the CUDA-core roles are plain C++ vector accesses on pointers
+// derived from the dynamic shared-memory base, so that the compiler can batch and schedule
+// them (the waits and fences around them are asm statements with memory clobbers).
+__device__ __forceinline__ void lds128(const uint8_t* p, uint32_t (&v)[4]) {
+    const uint4 x = *reinterpret_cast<const uint4*>(p);
+    v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+}
+__device__ __forceinline__ void sts128(uint8_t* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
 }
 
-__device__ __forceinline__ void lds128(uint32_t addr, uint32_t (&v)[4]) {
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(addr));
+// One 128-byte row (64 bf16) of a swizzled tile into registers / back, in LOGICAL chunk order
+// (chunk c of row r lives at physical chunk c ^ (r & 7); visiting it that way also keeps the
+// eight rows of a quarter-warp on eight different bank groups).
+__device__ __forceinline__ void load_row(const uint8_t* row, uint32_t r7, uint32_t (&v)[8][4]) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) lds128(row + ((c ^ r7) << 4), v[c]);
 }
-__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+__device__ __forceinline__ void store_row(uint8_t* row, uint32_t r7, const uint32_t (&v)[8][4]) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) sts128(row + ((c ^ r7) << 4), v[c][0], v[c][1], v[c][2], v[c][3]);
 }
+
+// Feature map on one row in place (optionally scaled): all loads first, then the arithmetic,
+// then all stores.
+template <bool kElu>
+__device__ __forceinline__ void map_row_inplace(uint8_t* row, uint32_t r7, float scale) {
+    uint32_t v[8][4];
+    load_row(row, r7, v);
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float x0 = sm100::bf16_lo(v[c][j]), x1 = sm100::bf16_hi(v[c][j]);
+            v[c][j] = sm100::pack_bf16x2((kElu ? phi_fast(x0) : x0) * scale, (kElu ? phi_fast(x1) : x1) * scale);
+        }
+    store_row(row, r7, v);
+}
+__device__ __forceinline__ void phi_row_inplace(uint8_t* row, uint32_t r7) { map_row_inplace<true>(row, r7, 1.f); }
 
 __device__ __forceinline__ uint64_t desc_k(uint32_t addr) { return sm100::umma_desc_sw128(addr, 16, 1024); }
 __device__ __forceinline__ uint64_t desc_mn(uint32_t addr, uint32_t lbo = kTileBytes) {
@@ -92,7 +109,7 @@ __device__ __forceinline__ void stg128(void* p, uint32_t a, uint32_t b, uint32_t
 // One 32-column block of a 128x128 fp32 score matrix (already loaded from TMEM into v)
 // -> + `add` -> causal mask on the diagonal block -> bf16 -> this row's 64 bytes of the
 // swizzled [128][64] tile pair.  tile_row = shared address of row t in tile 0 of the pair.
-__device__ __forceinline__ void score_block_store(const uint32_t (&v)[32], uint32_t tile_row, uint32_t r7, int blk,
+__device__ __forceinline__ void score_block_store(const uint32_t (&v)[32], uint8_t* tile_row, uint32_t r7, int blk,
                                                   bool diagonal, int lane, float add) {
     uint32_t packed[16];
 #pragma unroll
@@ -104,7 +121,7 @@ __device__ __forceinline__ void score_block_store(const uint32_t (&v)[32], uint3
         }
         packed[j] = sm100::pack_bf16x2(x0, x1);
     }
-    const uint32_t base = tile_row + (blk >> 1) * kTileBytes;
+    uint8_t* base = tile_row + (blk >> 1) * kTileBytes;
 #pragma unroll
     for (int cc = 0; cc < 4; ++cc) {
         const uint32_t chunk = (blk & 1) * 4 + cc;
@@ -115,7 +132,7 @@ __device__ __forceinline__ void score_block_store(const uint32_t (&v)[32], uint3
 // State accumulator (M = 64 layout: lanes 0-15 of quadrant w hold rows 16w..16w+15; 64 columns
 // of S followed by Z) -> bf16 [64][64] swizzled tile + fp32 Z; optionally the fp32 values to
 // global memory.  Executed by the four warps of one warpgroup; `quad` = warp % 4.
-__device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int lane, uint32_t s_tile, float* z_out,
+__device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, float* z_out,
                                               float* g_S, float* g_Z) {
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
@@ -150,7 +167,7 @@ __device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int
 }
 
 // Load an initial [S | Z] record (or zeros) into the TMEM state accumulator, its bf16 tile and z_out.
-__device__ __forceinline__ void state_init(uint32_t tmem_state, int quad, int lane, uint32_t s_tile, float* z_out,
+__device__ __forceinline__ void state_init(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, float* z_out,
                                            const float* rec) {
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;

@@ -135,26 +135,13 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             }
             if (!mbar_wait(&bars->full[s], (c / kSumStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
-            const uint32_t aX = sbase + s * kSumStageBytes + t * 128;
-            if (!scaled) {
-                if (prm.phi == LA_PHI_ELU1) phi_row_inplace(aX, r7);
-            } else {
-                const bool elu = prm.phi == LA_PHI_ELU1;
-#pragma unroll
-                for (int cc = 0; cc < 8; ++cc) {
-                    uint32_t v[4];
-                    lds128(aX + ((cc ^ r7) << 4), v);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float x0 = bf16_lo(v[j]), x1 = bf16_hi(v[j]);
-                        v[j] = pack_bf16x2((elu ? phi_fast(x0) : x0) * inv, (elu ? phi_fast(x1) : x1) * inv);
-                    }
-                    sts128(aX + ((cc ^ r7) << 4), v[0], v[1], v[2], v[3]);
-                }
-                const uint32_t aA = aX + 2 * kTileBytes;
+            uint8_t* rowX = smem + s * kSumStageBytes + t * 128;
+            if (prm.phi == LA_PHI_ELU1) map_row_inplace<true>(rowX, r7, inv); else if (scaled) map_row_inplace<false>(rowX, r7, inv);
+            if (scaled) {
+                uint8_t* rowA = rowX + 2 * kTileBytes;
                 const uint32_t dd = pack_bf16x2(delta, delta);      // columns 0..15 of the aux tile
-                sts128(aA + ((0 ^ r7) << 4), dd, dd, dd, dd);
-                sts128(aA + ((1 ^ r7) << 4), dd, dd, dd, dd);
+                sts128(rowA + ((0 ^ r7) << 4), dd, dd, dd, dd);
+                sts128(rowA + ((1 ^ r7) << 4), dd, dd, dd, dd);
             }
             fence_proxy_async_smem();
             mbar_arrive(&bars->mapped[s]);
