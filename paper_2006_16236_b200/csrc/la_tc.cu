@@ -37,11 +37,13 @@ bool tc_supported(const la_problem& p, int op) {
     if (p.dtype != LA_BF16 || p.D != tc::kDim || p.M != tc::kDim) return false;
     if (p.N < tc::kChunk || p.N % tc::kChunk) return false;
     if (p.B * p.H * p.N >= (1LL << 31)) return false;          // TMA coordinates are 32-bit
-    return op == LA_OP_CAUSAL_FORWARD || op == LA_OP_CAUSAL_BACKWARD;
+    return op >= LA_OP_LINEAR_FORWARD && op <= LA_OP_CAUSAL_BACKWARD;
 }
 
 size_t tc_workspace_bytes(const la_problem& p, int op) {
     switch (op) {
+        case LA_OP_LINEAR_FORWARD: return tc::linear_forward_workspace(p);
+        case LA_OP_LINEAR_BACKWARD: return tc::linear_backward_workspace(p);
         case LA_OP_CAUSAL_FORWARD: return tc::causal_forward_workspace(p);
         case LA_OP_CAUSAL_BACKWARD: return tc::causal_backward_workspace(p);
         default: return 0;
@@ -57,13 +59,13 @@ int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const 
     (void)O; (void)den;      // everything needed is recomputed consistently
     return tc::causal_backward(p, Q, K, V, G, dQ, dK, dV, ws, st);
 }
-int tc_linear_forward(const la_problem&, const void*, const void*, const void*, void*, float*, float*,
-                      float*, void*, cudaStream_t) {
-    return fail(LA_ERR_UNSUPPORTED, "tensor-core linear forward not available");
+int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
+                      float* KV, float* Zs, void* ws, cudaStream_t st) {
+    return tc::linear_forward(p, Q, K, V, O, den, KV, Zs, ws, st);
 }
-int tc_linear_backward(const la_problem&, const void*, const void*, const void*, const void*, void*, void*,
-                       void*, void*, cudaStream_t) {
-    return fail(LA_ERR_UNSUPPORTED, "tensor-core linear backward not available");
+int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G, void* dQ,
+                       void* dK, void* dV, void* ws, cudaStream_t st) {
+    return tc::linear_backward(p, Q, K, V, G, dQ, dK, dV, ws, st);
 }
 
 }  // namespace la

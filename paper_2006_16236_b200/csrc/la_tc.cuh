@@ -24,6 +24,12 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
 size_t causal_backward_workspace(const la_problem& p);
 int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
                     void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+size_t linear_forward_workspace(const la_problem& p);
+size_t linear_backward_workspace(const la_problem& p);
+int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
+                   float* KV, float* Zs, void* ws, cudaStream_t st);
+int linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+                    void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 }  // namespace tc
 
 }  // namespace la

@@ -40,6 +40,9 @@ Segmentation choose_segments(const la_problem& p);
 int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
                    const float* dn, const float* dl, float* records, bool reverse, cudaStream_t st);
 
+int segment_totals(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
+                   const float* dn, const float* dl, float* records, cudaStream_t st);
+
 // 2-D view of a [rows][64] bf16 tensor with a [box_rows][64] box and the 128-byte swizzle.
 int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows);
 

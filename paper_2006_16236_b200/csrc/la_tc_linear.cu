@@ -1,0 +1,701 @@
+// Non-causal linear attention on the tensor cores (bf16, D = M = 64), Eq. 5-6 and the
+// gradient of Eq. 13-15 with full (unmasked) sums.
+//
+// The per-head sums are formed once (pre-pass: every sequence is cut into splits, each
+// split's sums go to a record; consumers add the records) and reused for every position
+// by three "apply" passes that share one kernel:
+//   forward        O_i  = q_i S / (q_i . Z + eps)                        X = Q
+//   backward, Q    h_i  = G_i S^T,  dn_i = q_i . Z + eps,  dl_i = -(q_i . h_i) / dn_i,
+//                  gq_i = (h_i + dl_i Z) / dn_i,  dQ = gq o phi'(Q)      X = Q, Y = G
+//   backward, K/V  gk_j = V_j R^T + r,  dK = gk o phi'(K),  dV_j = k_j R  X = K, Y = V
+// with St = [S | Z] = sum_j k_j [V_j | 1]^T and Rt = [R | r] = sum_i (q_i / dn_i) [G_i | dl_i]^T.
+// As in the causal kernels, -(G_i . O_i) is taken from the same rounded products as h_i
+// (projection form), never from a stored output.
+//
+// Centred operands.  phi = elu + 1 is positive, so phi(X) ~ 1 + (something small) whenever
+// the inputs are small, and every sum above is dominated by a rank-one part that carries
+// none of the Q / K gradient.  Rounding phi(X) or the sums to bf16 as they stand would
+// spend the 8 mantissa bits on that part.  The tensor cores therefore only see centred
+// operands, and every rank-one part is carried in fp32:
+//   x' = elu(X) = phi(X) - 1                     (tile operand; full bf16 relative precision)
+//   S  = 1 (ysum + mu)^T + S'',  S'' = sum_j k'_j V_j^T - 1 mu^T  (mu = column means), Z = N 1 + Z'
+//   R  = 1 (gsum + rho)^T + R'', R'' = sum_i qh'_i G_i^T - 1 rho^T,  r = rho0 1 + r'
+// with ysum = sum_j V_j, gsum = sum_i G_i / dn_i, rho0 = sum_i dl_i / dn_i, qh' = q' / dn.
+// The column sums of S'' and R'' vanish, so (1 + x')^T S'' = x'^T S''.
+//
+// CTA = 10 warps: warps 0-3 epilogue (thread t owns chunk row t = TMEM lane t), warps 4-7
+// apply elu to the X tile in place, warp 8 TMA, warp 9 MMA issue.
+#include "la_tc.cuh"
+#include "la_tc_common.cuh"
+
+namespace la {
+namespace tc {
+
+using namespace sm100;
+
+namespace {
+
+// Record of one split: [A' (64x64) | a' (64) | ysum (64) | w0 (1) | pad]:
+//   forward sums : A' = sum k'_j V_j^T, a' = sum k'_j, ysum = sum V_j,        w0 unused
+//   reverse sums : A' = sum qh'_i G_i^T, a' = sum qh'_i dl_i, ysum = sum G_i / dn_i, w0 = sum dl_i / dn_i
+constexpr int kRecFloats = kDim * kDim + kDim + kDim + 8;
+
+__device__ __forceinline__ float elu_fast(float x) {      // elu(x) = phi(x) - 1
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * 1.4426950408889634f));
+    return x > 0.f ? x : e - 1.f;
+}
+
+// elu (optionally scaled) on one row of a swizzled tile, in place; returns nothing.
+template <bool kElu>
+__device__ __forceinline__ void elu_row_inplace(uint8_t* row, uint32_t r7, float scale) {
+    uint32_t v[8][4];
+    load_row(row, r7, v);
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float x0 = bf16_lo(v[c][j]), x1 = bf16_hi(v[c][j]);
+            v[c][j] = pack_bf16x2((kElu ? elu_fast(x0) : x0 - 1.f) * scale, (kElu ? elu_fast(x1) : x1 - 1.f) * scale);
+        }
+    store_row(row, r7, v);
+}
+
+// ===========================================================================
+// Pre-pass: per-split sums.  Warps 0-3: elu on X (scaled by w_i), weight and aux tiles,
+// final read-out; warp 4: TMA; warp 5: MMA.
+// ===========================================================================
+constexpr int kLsThreads = 192;
+constexpr int kLsStages = 2;
+constexpr uint32_t kLsStageBytes = 4 * kTileBytes;                  // X, Y, W (rows of w_i), aux (dl_i in 16 columns)
+constexpr uint32_t kLsOffOnes = kLsStages * kLsStageBytes;
+constexpr uint32_t kLsOffBar = kLsOffOnes + 1024;
+constexpr uint32_t kLsSmemBytes = kLsOffBar + 256 + 1024;
+
+struct LsBarriers {
+    uint64_t full[kLsStages], empty[kLsStages], mapped[kLsStages];
+    uint64_t done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct LsParams {
+    float* records;        // [BH][nseg][kRecFloats]
+    const float* dn;       // null: forward sums (w_i = 1, aux = 1); else w_i = 1 / dn_i, aux = dl_i
+    const float* dl;
+    int* status;
+    int64_t N;
+    int chunks, chunks_per_seg, nseg;
+    int phi;
+};
+
+__global__ void __launch_bounds__(kLsThreads, 1)
+linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
+                  const LsParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    LsBarriers* bars = reinterpret_cast<LsBarriers*>(smem + kLsOffBar);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int seg = blockIdx.x % prm.nseg;
+    const int64_t bh = blockIdx.x / prm.nseg;
+    const int c_begin = seg * prm.chunks_per_seg;
+    const int L = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
+    const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
+    const bool reverse = prm.dn != nullptr;
+
+    if (tid == 0) {
+        for (int s = 0; s < kLsStages; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+            mbar_init(&bars->mapped[s], 128);
+        }
+        mbar_init(&bars->done, 1);
+        bars->abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 5) {
+        __syncwarp();
+        tmem_alloc(&bars->tmem_base, 256);
+        tmem_relinquish();
+    }
+    if (tid < 128)
+        for (int i = tid; i < 256; i += 128) reinterpret_cast<uint32_t*>(smem + kLsOffOnes)[i] = 0x3F803F80u;
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = bars->tmem_base;
+    volatile int* abort_flag = &bars->abort_flag;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            prefetch_tensormap(&mapX); prefetch_tensormap(&mapY);
+            for (int c = 0; c < L; ++c) {
+                const int s = c % kLsStages;
+                if (c >= kLsStages && !mbar_wait(&bars->empty[s], ((c / kLsStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
+                    *abort_flag = 1;
+                    break;
+                }
+                if (*abort_flag) break;
+                uint8_t* st = smem + s * kLsStageBytes;
+                const int y = (int)(row0 + (int64_t)c * kChunk);
+                mbar_arrive_expect_tx(&bars->full[s], 2 * kTileBytes);
+                tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
+                tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            const uint32_t idesc_s = umma_idesc_bf16(64, 64, 1, 1);
+            const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
+            const uint32_t aOnes = sbase + kLsOffOnes;
+            bool ok = true;
+            for (int c = 0; c < L && ok; ++c) {
+                const int s = c % kLsStages;
+                const uint32_t aX = sbase + s * kLsStageBytes, aY = aX + kTileBytes, aW = aY + kTileBytes, aA = aW + kTileBytes;
+                ok = mbar_wait(&bars->mapped[s], (c / kLsStages) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok || *abort_flag) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t acc = (c != 0);
+                for (int k = 0; k < 8; ++k) {
+                    const uint32_t a = acc | (k != 0);
+                    const uint64_t dX = desc_mn(aX + k * 2048), dY = desc_mn(aY + k * 2048);
+                    const uint64_t dW = reverse ? desc_mn(aW + k * 2048) : desc_ones(aOnes);
+                    const uint64_t dA = reverse ? desc_mn(aA + k * 2048) : desc_ones(aOnes);
+                    umma_bf16(tmem, dX, dY, idesc_s, a);                 // A' += x'^T Y
+                    umma_bf16(tmem + 64, dX, dA, idesc_z, a);            // a' += x'^T aux
+                    umma_bf16(tmem + 128, dW, dY, idesc_s, a);           // ysum += w^T Y (all 64 rows alike)
+                    if (reverse) umma_bf16(tmem + 192, dW, dA, idesc_z, a);   // w0 += w^T aux
+                }
+                umma_commit(&bars->empty[s]);
+            }
+            if (!ok) *abort_flag = 1;
+            umma_commit(&bars->done);
+        }
+    } else {
+        const int t = tid;
+        const uint32_t r7 = t & 7;
+        const bool elu = prm.phi == LA_PHI_ELU1;
+        for (int c = 0; c < L; ++c) {
+            const int s = c % kLsStages;
+            const int64_t row = row0 + (int64_t)c * kChunk + t;
+            float w = 1.f, delta = 0.f;
+            if (reverse) {
+                w = 1.f / __ldg(prm.dn + row);
+                delta = __ldg(prm.dl + row);
+            }
+            if (!mbar_wait(&bars->full[s], (c / kLsStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            uint8_t* rowX = smem + s * kLsStageBytes + t * 128;
+            if (elu) elu_row_inplace<true>(rowX, r7, w); else elu_row_inplace<false>(rowX, r7, w);
+            if (reverse) {
+                uint8_t* rowW = rowX + 2 * kTileBytes;
+                uint8_t* rowA = rowX + 3 * kTileBytes;
+                const uint32_t ww = pack_bf16x2(w, w), dd = pack_bf16x2(delta, delta);
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc) sts128(rowW + (cc << 4), ww, ww, ww, ww);
+                sts128(rowA + ((0 ^ r7) << 4), dd, dd, dd, dd);
+                sts128(rowA + ((1 ^ r7) << 4), dd, dd, dd, dd);
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&bars->mapped[s]);
+        }
+        // read-out of this split's record
+        const bool ok = mbar_wait(&bars->done, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
+        tc_fence_after_sync();
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        float* rec = prm.records + (bh * prm.nseg + seg) * (int64_t)kRecFloats;
+        const int d_row = warp * 16 + lane;
+        for (int h = 0; h < 2; ++h) {
+            uint32_t v[32];
+            tmem_ld32(tmem + lane_base + h * 32, v);
+            tmem_ld_wait();
+            if (ok && lane < 16)
+#pragma unroll
+                for (int j = 0; j < 32; ++j) rec[d_row * kDim + h * 32 + j] = __uint_as_float(v[j]);
+        }
+        const float z = __uint_as_float(tmem_ld1(tmem + lane_base + 64));
+        tmem_ld_wait();
+        if (ok && lane < 16) rec[kDim * kDim + d_row] = z;
+        if (warp == 0) {            // row 0 of the w-weighted sums
+            for (int h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                tmem_ld32(tmem + 128 + h * 32, v);
+                tmem_ld_wait();
+                if (ok && lane == 0)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) rec[kDim * kDim + kDim + h * 32 + j] = __uint_as_float(v[j]);
+            }
+            const float w0 = __uint_as_float(tmem_ld1(tmem + 192));
+            tmem_ld_wait();
+            if (ok && lane == 0) rec[kDim * kDim + 2 * kDim] = reverse ? w0 : 0.f;
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        __syncwarp();
+        tmem_dealloc(tmem, 256);
+    }
+}
+
+// ===========================================================================
+// Apply passes.
+// ===========================================================================
+enum ApplyMode { kApplyForward = 0, kApplyBackwardQ = 1, kApplyBackwardKV = 2 };
+
+constexpr int kApStages = 3;
+constexpr int kApThreads = 320;
+constexpr uint32_t kApOffStage = 0;                                   // kApStages x {X, Y}
+constexpr uint32_t kApOffState = kApOffStage + kApStages * 2 * kTileBytes;   // bf16 centred state tile [64][64]
+constexpr uint32_t kApOffVec = kApOffState + kDim * 128;              // fp32 [3][64]: a' (Z' or r'), nu, scratch
+constexpr uint32_t kApOffBar = kApOffVec + 1024;
+constexpr uint32_t kApSmemBytes = kApOffBar + 256 + 1024;
+
+struct ApBarriers {
+    uint64_t full[kApStages], empty[kApStages], mapped[kApStages];
+    uint64_t acc_full[2], acc_free[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct ApParams {
+    const float* records;       // [BH][nseg][kRecFloats]: summed by every CTA
+    __nv_bfloat16* out0;        // forward: O;  backward Q: dQ;  backward K/V: dK
+    __nv_bfloat16* out1;        // backward K/V: dV
+    float* den;                 // forward: q.Z (optional);  backward Q: dn_i (out)
+    float* dl;                  // backward Q: dl_i (out)
+    float* state_out;           // forward: KV [BH][64][64] (optional)
+    float* vec_out;             // forward: Zs [BH][64] (optional)
+    int* status;
+    int64_t N;
+    int chunks, chunks_per_seg, nseg;
+    float eps;
+    int phi;
+};
+
+template <int kMode>
+__global__ void __launch_bounds__(kApThreads, 1)
+linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
+                    const ApParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    ApBarriers* bars = reinterpret_cast<ApBarriers*>(smem + kApOffBar);
+    float* sA = reinterpret_cast<float*>(smem + kApOffVec);      // a': Z' (forward, backward Q) or r' (backward K/V)
+    float* sNu = sA + 64;                                        // rank-one part along 1: ysum + mu  /  gsum + rho
+    float* sScal = sA + 128;                                     // [0] = sum_d a'_d, [1] = w0
+    constexpr bool kHasY = kMode != kApplyForward;
+    constexpr uint32_t kTiles = kHasY ? 2 : 1;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int seg = blockIdx.x % prm.nseg;
+    const int64_t bh = blockIdx.x / prm.nseg;
+    const int c_begin = seg * prm.chunks_per_seg;
+    const int L = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
+    const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
+
+    if (tid == 0) {
+        for (int s = 0; s < kApStages; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1 + 128);      // MMA commit + epilogue threads (they read the X and Y rows)
+            mbar_init(&bars->mapped[s], 128);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&bars->acc_full[b], 1);
+            mbar_init(&bars->acc_free[b], 128);
+        }
+        bars->abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 9) {
+        __syncwarp();
+        tmem_alloc(&bars->tmem_base, 256);
+        tmem_relinquish();
+    }
+    // state of this head: add the split records (fp32), remove the column means, round the
+    // centred remainder to a bf16 operand tile.  The stage area is free until the pipeline starts.
+    {
+        const float* rec = prm.records + bh * prm.nseg * (int64_t)kRecFloats;
+        float* sF = reinterpret_cast<float*>(smem + kApOffStage);                 // fp32 [64][64] scratch
+        for (int idx = tid; idx < kDim * kDim / 4; idx += kApThreads) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int n = 0; n < prm.nseg; ++n) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(rec + (int64_t)n * kRecFloats) + idx);
+                acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
+            }
+            reinterpret_cast<float4*>(sF)[idx] = acc;
+        }
+        if (tid < 2 * kDim + 1) {       // a' (64), ysum (64), w0 (1)
+            float z = 0.f;
+            for (int n = 0; n < prm.nseg; ++n) z += __ldg(rec + (int64_t)n * kRecFloats + kDim * kDim + tid);
+            if (tid < kDim) sA[tid] = z;
+            else if (tid < 2 * kDim) sNu[tid - kDim] = z;
+            else sScal[1] = z;
+        }
+        __syncthreads();
+        if (tid < kDim) {               // column tid: mean over d; nu = ysum + mu
+            float m = 0.f;
+            for (int d = 0; d < kDim; ++d) m += sF[d * kDim + tid];
+            m *= 1.f / kDim;
+            const float ysum = sNu[tid];
+            sNu[tid] = ysum + m;
+            sF[kDim * kDim + tid] = m;                                            // mu, just past the matrix
+            if (kMode == kApplyForward && seg == 0) {
+                // true sums for the caller: S = 1 ysum^T + A', Z = N 1 + a'
+                if (prm.vec_out) prm.vec_out[bh * kDim + tid] = (float)prm.N + sA[tid];
+                if (prm.state_out)
+                    for (int d = 0; d < kDim; ++d)
+                        prm.state_out[bh * (int64_t)(kDim * kDim) + d * kDim + tid] = sF[d * kDim + tid] + ysum;
+            }
+        }
+        if (tid == 64) {
+            float z = 0.f;
+            for (int d = 0; d < kDim; ++d) z += sA[d];
+            sScal[0] = z;
+        }
+        __syncthreads();
+        for (int idx = tid; idx < kDim * kDim / 8; idx += kApThreads) {       // 8 consecutive columns of one row
+            const int d = idx >> 3, c8 = idx & 7;
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = sF[d * kDim + c8 * 8 + j] - sF[kDim * kDim + c8 * 8 + j];
+            sts128(smem + kApOffState + d * 128 + ((c8 ^ (d & 7)) << 4), pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]),
+                   pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+        }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = bars->tmem_base;
+    volatile int* abort_flag = &bars->abort_flag;
+
+    if (warp == 8) {
+        if (lane == 0) {
+            prefetch_tensormap(&mapX);
+            if (kHasY) prefetch_tensormap(&mapY);
+            for (int c = 0; c < L; ++c) {
+                const int s = c % kApStages;
+                if (c >= kApStages && !mbar_wait(&bars->empty[s], ((c / kApStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
+                    *abort_flag = 1;
+                    break;
+                }
+                if (*abort_flag) break;
+                uint8_t* st = smem + kApOffStage + s * 2 * kTileBytes;
+                const int y = (int)(row0 + (int64_t)c * kChunk);
+                mbar_arrive_expect_tx(&bars->full[s], kTiles * kTileBytes);
+                tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
+                if (kHasY) tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
+            }
+        }
+    } else if (warp == 9) {
+        if (lane == 0) {
+            const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
+            const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
+            const uint32_t aSt = sbase + kApOffState;
+            bool ok = true;
+            for (int c = 0; c < L && ok; ++c) {
+                const int s = c % kApStages, b = c & 1;
+                const uint32_t aX = sbase + kApOffStage + s * 2 * kTileBytes, aY = aX + kTileBytes;
+                ok = mbar_wait(&bars->mapped[s], (c / kApStages) & 1, prm.status, kStatusPipeTimeout);
+                if (ok && c >= 2) ok = mbar_wait(&bars->acc_free[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok || *abort_flag) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d0 = tmem + b * 128, d1 = d0 + 64;
+                if (kMode == kApplyForward) {
+                    for (int k = 0; k < 4; ++k)      // q' S''
+                        umma_bf16(d0, desc_k(aX + k * 32), desc_mn(aSt + k * 2048), idesc_kmn, k > 0);
+                } else if (kMode == kApplyBackwardQ) {
+                    for (int k = 0; k < 4; ++k)      // h'' = G S''^T
+                        umma_bf16(d0, desc_k(aY + k * 32), desc_k(aSt + k * 32), idesc_kk, k > 0);
+                } else {
+                    for (int k = 0; k < 4; ++k)      // V R''^T
+                        umma_bf16(d0, desc_k(aY + k * 32), desc_k(aSt + k * 32), idesc_kk, k > 0);
+                    for (int k = 0; k < 4; ++k)      // k' R''
+                        umma_bf16(d1, desc_k(aX + k * 32), desc_mn(aSt + k * 2048), idesc_kmn, k > 0);
+                }
+                umma_commit(&bars->acc_full[b]);
+                umma_commit(&bars->empty[s]);
+            }
+            if (!ok) *abort_flag = 1;
+        }
+    } else if (warp >= 4) {
+        const int t = tid - 128;
+        const uint32_t r7 = t & 7;
+        const bool elu = prm.phi == LA_PHI_ELU1;
+        for (int c = 0; c < L; ++c) {
+            const int s = c % kApStages;
+            if (!mbar_wait(&bars->full[s], (c / kApStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            uint8_t* rowX = smem + kApOffStage + s * 2 * kTileBytes + t * 128;
+            if (elu) elu_row_inplace<true>(rowX, r7, 1.f); else elu_row_inplace<false>(rowX, r7, 1.f);
+            fence_proxy_async_smem();
+            mbar_arrive(&bars->mapped[s]);
+        }
+    } else {
+        const int t = tid;
+        const uint32_t r7 = t & 7;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const bool elu = prm.phi == LA_PHI_ELU1;
+        const float fD = (float)kDim, fN = (float)prm.N;
+        for (int c = 0; c < L; ++c) {
+            const int s = c % kApStages, b = c & 1;
+            const int64_t row = row0 + (int64_t)c * kChunk + t;
+            if (!mbar_wait(&bars->mapped[s], (c / kApStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
+            if (*abort_flag) break;
+            uint32_t xv[8][4];                       // x' = elu(X) row
+            load_row(smem + kApOffStage + s * 2 * kTileBytes + t * 128, r7, xv);
+            float ynu = 0.f;                         // Y_i . nu (backward)
+            if (kHasY) {
+                uint32_t yv[8][4];
+                load_row(smem + kApOffStage + s * 2 * kTileBytes + kTileBytes + t * 128, r7, yv);
+                float p4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        p4[j] = fmaf(bf16_lo(yv[cc][j]), sNu[cc * 8 + 2 * j], fmaf(bf16_hi(yv[cc][j]), sNu[cc * 8 + 2 * j + 1], p4[j]));
+                ynu = (p4[0] + p4[1]) + (p4[2] + p4[3]);
+            }
+            mbar_arrive(&bars->empty[s]);
+            // sx = sum_d x'_d  and  xa = x' . a'
+            float sx4[4] = {0.f, 0.f, 0.f, 0.f}, xa4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float x0 = bf16_lo(xv[cc][j]), x1 = bf16_hi(xv[cc][j]);
+                    sx4[j] += x0 + x1;
+                    xa4[j] = fmaf(x0, sA[cc * 8 + 2 * j], fmaf(x1, sA[cc * 8 + 2 * j + 1], xa4[j]));
+                }
+            const float sx = (sx4[0] + sx4[1]) + (sx4[2] + sx4[3]);
+            const float xa = (xa4[0] + xa4[1]) + (xa4[2] + xa4[3]);
+            const float x1sum = fD + sx;             // (1 + x') . 1
+            if (!mbar_wait(&bars->acc_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            tc_fence_after_sync();
+            uint32_t a0[32], a1[32];
+            tmem_ld32(tmem + lane_base + b * 128, a0);
+            tmem_ld32(tmem + lane_base + b * 128 + 32, a1);
+            tmem_ld_wait();
+            __nv_bfloat16* dst = prm.out0 + row * kDim;
+            if (kMode == kApplyForward) {
+                // den = (1 + q') . (N 1 + Z');  num = (1 + q').1 nu + q' S''
+                const float den = fN * x1sum + sScal[0] + xa;
+                const float inv = 1.f / (den + prm.eps);
+                const float w = x1sum * inv;
+                if (prm.den) prm.den[row] = den;
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        const uint32_t* acc = hh ? a1 : a0;
+                        const float* nu = sNu + hh * 32 + cc * 8;
+                        stg128(dst + hh * 32 + cc * 8,
+                               pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 0]), inv, w * nu[0]), fmaf(__uint_as_float(acc[cc * 8 + 1]), inv, w * nu[1])),
+                               pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 2]), inv, w * nu[2]), fmaf(__uint_as_float(acc[cc * 8 + 3]), inv, w * nu[3])),
+                               pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 4]), inv, w * nu[4]), fmaf(__uint_as_float(acc[cc * 8 + 5]), inv, w * nu[5])),
+                               pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 6]), inv, w * nu[6]), fmaf(__uint_as_float(acc[cc * 8 + 7]), inv, w * nu[7])));
+                    }
+            } else {
+                // backward Q:  h = (G.nu) 1 + h'',  Z = N 1 + Z',  gq = (h - (q.h / dn) Z) / dn
+                // backward KV: gk = (V.nu_R + w0) 1 + V R''^T + r'
+                float c1 = 0.f, cz = 0.f, scale = 1.f;          // out_d = scale * (acc_d + c1 + cz * a'_d)
+                if (kMode == kApplyBackwardQ) {
+                    float sh4[4] = {0.f, 0.f, 0.f, 0.f}, qh4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float h0 = __uint_as_float(a0[cc * 8 + 2 * j]), h1 = __uint_as_float(a0[cc * 8 + 2 * j + 1]);
+                            const float h2 = __uint_as_float(a1[cc * 8 + 2 * j]), h3 = __uint_as_float(a1[cc * 8 + 2 * j + 1]);
+                            sh4[j] += (h0 + h1) + (h2 + h3);
+                            qh4[j] = fmaf(bf16_lo(xv[cc][j]), h0, fmaf(bf16_hi(xv[cc][j]), h1, qh4[j]));
+                            qh4[j] = fmaf(bf16_lo(xv[cc + 4][j]), h2, fmaf(bf16_hi(xv[cc + 4][j]), h3, qh4[j]));
+                        }
+                    const float sh = (sh4[0] + sh4[1]) + (sh4[2] + sh4[3]);       // 1 . h''
+                    const float qh = (qh4[0] + qh4[1]) + (qh4[2] + qh4[3]);       // q' . h''
+                    const float den = fN * x1sum + sScal[0] + xa;
+                    const float dn = den + prm.eps;
+                    scale = 1.f / dn;
+                    const float q_h = ynu * x1sum + sh + qh;                      // q . h
+                    const float dl = -q_h * scale;                                // dl_i = -(G_i . O_i)
+                    c1 = fmaf(dl, fN, ynu);                                       // (G.nu) + dl N
+                    cz = dl;
+                    prm.den[row] = dn;
+                    prm.dl[row] = dl;
+                } else {
+                    c1 = ynu + sScal[1];
+                    cz = 1.f;
+                }
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t outp[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int e = cc * 8 + 2 * j, d = hh * 32 + e;
+                            const uint32_t* acc = hh ? a1 : a0;
+                            float g0 = scale * (fmaf(cz, sA[d], __uint_as_float(acc[e])) + c1);
+                            float g1 = scale * (fmaf(cz, sA[d + 1], __uint_as_float(acc[e + 1])) + c1);
+                            if (elu) {          // phi'(x) from x' = elu(x): 1 where x' > 0, else 1 + x'
+                                const float x0 = bf16_lo(xv[hh * 4 + cc][j]), x1 = bf16_hi(xv[hh * 4 + cc][j]);
+                                g0 *= x0 > 0.f ? 1.f : 1.f + x0;
+                                g1 *= x1 > 0.f ? 1.f : 1.f + x1;
+                            }
+                            outp[j] = pack_bf16x2(g0, g1);
+                        }
+                        stg128(dst + hh * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
+                    }
+                if (kMode == kApplyBackwardKV) {
+                    tmem_ld32(tmem + lane_base + b * 128 + 64, a0);
+                    tmem_ld32(tmem + lane_base + b * 128 + 96, a1);
+                    tmem_ld_wait();
+                    __nv_bfloat16* dstV = prm.out1 + row * kDim;
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) {       // gV = (1 + k').1 nu_R + k' R''
+                            const uint32_t* acc = hh ? a1 : a0;
+                            const float* nu = sNu + hh * 32 + cc * 8;
+                            stg128(dstV + hh * 32 + cc * 8,
+                                   pack_bf16x2(fmaf(x1sum, nu[0], __uint_as_float(acc[cc * 8 + 0])), fmaf(x1sum, nu[1], __uint_as_float(acc[cc * 8 + 1]))),
+                                   pack_bf16x2(fmaf(x1sum, nu[2], __uint_as_float(acc[cc * 8 + 2])), fmaf(x1sum, nu[3], __uint_as_float(acc[cc * 8 + 3]))),
+                                   pack_bf16x2(fmaf(x1sum, nu[4], __uint_as_float(acc[cc * 8 + 4])), fmaf(x1sum, nu[5], __uint_as_float(acc[cc * 8 + 5]))),
+                                   pack_bf16x2(fmaf(x1sum, nu[6], __uint_as_float(acc[cc * 8 + 6])), fmaf(x1sum, nu[7], __uint_as_float(acc[cc * 8 + 7]))));
+                        }
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bars->acc_free[b]);
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 9) {
+        __syncwarp();
+        tmem_dealloc(tmem, 256);
+    }
+}
+
+// Splits per sequence: about two CTAs per SM over all heads, at least two chunks each.
+Segmentation choose_splits(const la_problem& p) {
+    const int chunks = (int)(p.N / kChunk);
+    const int64_t bh = p.B * p.H;
+    int nseg = (int)((2 * 148 + bh - 1) / bh);
+    if (nseg > chunks / 2) nseg = chunks / 2;
+    if (nseg < 1) nseg = 1;
+    const int cps = (chunks + nseg - 1) / nseg;
+    nseg = (chunks + cps - 1) / cps;
+    return Segmentation{nseg, cps};
+}
+
+int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
+                const float* dn, const float* dl, float* records, cudaStream_t st) {
+    static bool attr_done = false;
+    if (!attr_done) {
+        LA_CUDA_TRY(cudaFuncSetAttribute(linear_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLsSmemBytes));
+        attr_done = true;
+    }
+    LsParams prm;
+    prm.records = records;
+    prm.dn = dn;
+    prm.dl = dl;
+    prm.status = device_status_ptr();
+    if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
+    prm.N = p.N;
+    prm.chunks = (int)(p.N / kChunk);
+    prm.chunks_per_seg = sg.chunks_per_seg;
+    prm.nseg = sg.nseg;
+    prm.phi = p.phi;
+    linear_sum_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kLsThreads, kLsSmemBytes, st>>>(mX, mY, prm);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+template <int kMode>
+int launch_apply(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
+                 ApParams prm, cudaStream_t st) {
+    static bool attr_done = false;
+    if (!attr_done) {
+        LA_CUDA_TRY(cudaFuncSetAttribute(linear_apply_kernel<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kApSmemBytes));
+        attr_done = true;
+    }
+    prm.status = device_status_ptr();
+    if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
+    prm.N = p.N;
+    prm.chunks = (int)(p.N / kChunk);
+    prm.chunks_per_seg = sg.chunks_per_seg;
+    prm.nseg = sg.nseg;
+    prm.eps = p.eps;
+    prm.phi = p.phi;
+    linear_apply_kernel<kMode><<<(unsigned)(sg.nseg * p.B * p.H), kApThreads, kApSmemBytes, st>>>(mX, mY, prm);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+}  // namespace
+
+size_t linear_forward_workspace(const la_problem& p) {
+    return (size_t)(p.B * p.H) * choose_splits(p).nseg * kRecFloats * sizeof(float);
+}
+
+size_t linear_backward_workspace(const la_problem& p) {
+    return 2 * linear_forward_workspace(p) + 2 * (size_t)(p.B * p.H) * (size_t)p.N * sizeof(float);
+}
+
+int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
+                   float* KV, float* Zs, void* ws, cudaStream_t st) {
+    const Segmentation sg = choose_splits(p);
+    const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
+    CUtensorMap mQ, mK, mV;
+    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mK, K, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mV, V, rows, kChunk)) return rc;
+    float* rec = (float*)ws;
+    if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, rec, st)) return rc;
+    ApParams a = {};
+    a.records = rec;
+    a.out0 = (__nv_bfloat16*)O;
+    a.den = den;
+    a.state_out = KV;
+    a.vec_out = Zs;
+    return launch_apply<kApplyForward>(p, sg, mQ, mQ, a, st);
+}
+
+int linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+                    void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    const Segmentation sg = choose_splits(p);
+    const size_t bh = (size_t)(p.B * p.H);
+    const uint64_t rows = (uint64_t)(bh * p.N);
+    CUtensorMap mQ, mK, mV, mG;
+    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mK, K, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mV, V, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mG, G, rows, kChunk)) return rc;
+    uint8_t* w = (uint8_t*)ws;
+    float* rec_s = (float*)w;   w += bh * sg.nseg * kRecFloats * sizeof(float);
+    float* rec_r = (float*)w;   w += bh * sg.nseg * kRecFloats * sizeof(float);
+    float* dn = (float*)w;      w += bh * (size_t)p.N * sizeof(float);
+    float* dl = (float*)w;
+
+    if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, rec_s, st)) return rc;
+    ApParams a = {};
+    a.records = rec_s;
+    a.out0 = (__nv_bfloat16*)dQ;
+    a.den = dn;
+    a.dl = dl;
+    if (int rc = launch_apply<kApplyBackwardQ>(p, sg, mQ, mG, a, st)) return rc;
+    if (int rc = launch_sums(p, sg, mQ, mG, dn, dl, rec_r, st)) return rc;
+    ApParams b = {};
+    b.records = rec_r;
+    b.out0 = (__nv_bfloat16*)dK;
+    b.out1 = (__nv_bfloat16*)dV;
+    return launch_apply<kApplyBackwardKV>(p, sg, mK, mV, b, st);
+}
+
+}  // namespace tc
+}  // namespace la

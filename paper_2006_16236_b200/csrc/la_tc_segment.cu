@@ -219,5 +219,33 @@ int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMa
     return LA_OK;
 }
 
+// Per-segment sums of ALL segments, no scan: the consumer adds the nseg records of a sequence
+// (the non-causal form needs the full sums of Eq. 5 only).
+int segment_totals(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
+                   const float* dn, const float* dl, float* records, cudaStream_t st) {
+    static bool attr_done = false;
+    if (!attr_done) {
+        LA_CUDA_TRY(cudaFuncSetAttribute(segment_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSumSmemBytes));
+        attr_done = true;
+    }
+    SumParams prm;
+    prm.records = records;
+    prm.dn = dn;
+    prm.dl = dl;
+    prm.status = device_status_ptr();
+    if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
+    prm.N = p.N;
+    prm.chunks = (int)(p.N / kChunk);
+    prm.chunks_per_seg = sg.chunks_per_seg;
+    prm.nseg = sg.nseg;
+    prm.first_seg = 0;
+    prm.segs_per_seq = sg.nseg;
+    prm.eps = p.eps;
+    prm.phi = p.phi;
+    segment_sum_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
 }  // namespace tc
 }  // namespace la
