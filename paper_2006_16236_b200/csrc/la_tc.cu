@@ -8,7 +8,7 @@ namespace la {
 
 namespace tc {
 
-int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows) {
+int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols) {
     static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     if (!encode) {
         void* fn = nullptr;
@@ -18,8 +18,8 @@ int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t 
             return fail(LA_ERR_CUDA, "the driver does not export cuTensorMapEncodeTiled");
         encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
     }
-    const cuuint64_t dims[2] = {(cuuint64_t)kDim, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)kDim * 2};
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kDim, box_rows};
     const cuuint32_t elem_strides[2] = {1, 1};
     const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
@@ -34,7 +34,7 @@ int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t 
 bool tc_supported(const la_problem& p, int op) {
     static const bool disabled = getenv("LA_DISABLE_TC") != nullptr;
     if (disabled) return false;
-    if (p.dtype != LA_BF16 || p.D != tc::kDim || p.M != tc::kDim) return false;
+    if (p.dtype != LA_BF16 || p.D != p.M || (p.D != 32 && p.D != 64)) return false;
     if (p.N < tc::kChunk || p.N % tc::kChunk) return false;
     if (p.B * p.H * p.N >= (1LL << 31)) return false;          // TMA coordinates are 32-bit
     return op >= LA_OP_LINEAR_FORWARD && op <= LA_OP_CAUSAL_BACKWARD;

@@ -93,6 +93,7 @@ struct DqParams {
     int chunks, chunks_per_seg, nseg;
     float eps;
     int phi;
+    int dim;                    // D = M: 64, or 32 (tiles zero-padded to 64 columns)
 };
 
 __global__ void __launch_bounds__(kDqThreads, 1)
@@ -245,8 +246,8 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             if (t == 0) LA_TRACE(g_trace_dq, c, 5);
             if (prm.phi == LA_PHI_ELU1) {
                 uint8_t* rowK = smem + kDqOffStage + s * 4 * kTileBytes + t * 128;
-                phi_row_inplace(rowK, r7);
-                phi_row_inplace(rowK + 3 * kTileBytes, r7);
+                phi_row_inplace(rowK, r7, prm.dim >> 3);
+                phi_row_inplace(rowK + 3 * kTileBytes, r7, prm.dim >> 3);
                 fence_proxy_async_smem();
             }
             mbar_arrive(&bars->mapped[s]);
@@ -365,9 +366,10 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 prm.dn[row] = dn;
                 prm.dl[row] = delta;
             }
-            __nv_bfloat16* dst = prm.dQ + row * kDim + half * 32;
+            __nv_bfloat16* dst = prm.dQ + row * prm.dim + half * 32;
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
+                if (half * 32 >= prm.dim) break;          // columns beyond a 32-wide problem are padding
                 uint32_t outp[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -438,6 +440,7 @@ struct KvParams {
     int chunks, chunks_per_seg, nseg;
     float eps;
     int phi;
+    int dim;
 };
 
 __global__ void __launch_bounds__(kKvThreads, 1)
@@ -576,9 +579,9 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             if (*abort_flag) break;
             if (t == 0) LA_TRACE(g_trace_dkv, i, 5);
             uint8_t* rowQ = smem + kKvOffStage + s * 4 * kTileBytes + t * 128;
-            if (elu) map_row_inplace<true>(rowQ, r7, inv); else map_row_inplace<false>(rowQ, r7, inv);
+            if (elu) map_row_inplace<true>(rowQ, r7, inv, prm.dim >> 3); else map_row_inplace<false>(rowQ, r7, inv, prm.dim >> 3);
             if (t == 0) LA_TRACE(g_trace_dkv, i, 13);
-            if (elu) phi_row_inplace(rowQ + kTileBytes, r7);
+            if (elu) phi_row_inplace(rowQ + kTileBytes, r7, prm.dim >> 3);
             if (t == 0) LA_TRACE(g_trace_dkv, i, 14);
             sDelta[s * 128 + t] = delta;
             // the single dl column tile is an operand of the previous chunk's state MMAs
@@ -627,10 +630,11 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             tc_fence_after_sync();
             if (t == 0) LA_TRACE(g_trace_dkv, i, 9);
             const float* rprev = sRv + ((i + 1) & 1) * 64;               // r_{c+1}
-            __nv_bfloat16* dstK = prm.dK + row * kDim;
-            __nv_bfloat16* dstV = prm.dV + row * kDim;
+            __nv_bfloat16* dstK = prm.dK + row * prm.dim;
+            __nv_bfloat16* dstV = prm.dV + row * prm.dim;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
+                if (h * 32 >= prm.dim) break;             // columns beyond a 32-wide problem are padding
                 uint32_t v[32];
                 tmem_ld32(tmem + lane_base + kKvColDk + h * 32, v);
                 tmem_ld_wait();
@@ -654,6 +658,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
+                if (h * 32 >= prm.dim) break;
                 uint32_t v[32];
                 tmem_ld32(tmem + lane_base + kKvColDv + h * 32, v);
                 tmem_ld_wait();
@@ -739,10 +744,10 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     float* dl = (float*)w;
 
     CUtensorMap mQ, mK, mV, mG;
-    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mK, K, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mV, V, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mG, G, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mG, G, rows, kChunk, (int)p.D)) return rc;
     int* status = device_status_ptr();
     if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
 
@@ -768,6 +773,7 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.nseg = sg.nseg;
     a.eps = p.eps;
     a.phi = p.phi;
+    a.dim = (int)p.D;
     causal_bwd_dq_kernel<<<grid, kDqThreads, kDqSmemBytes, st>>>(mK, mV, mG, mQ, a);
     LA_LAUNCHED();
 
@@ -786,6 +792,7 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     b.nseg = sg.nseg;
     b.eps = p.eps;
     b.phi = p.phi;
+    b.dim = (int)p.D;
     causal_bwd_dkv_kernel<<<grid, kKvThreads, kKvSmemBytes, st>>>(mQ, mK, mV, mG, b);
     LA_LAUNCHED();
     return LA_OK;

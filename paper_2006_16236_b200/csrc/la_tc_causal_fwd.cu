@@ -62,6 +62,7 @@ struct FwdParams {
     int nseg;
     float eps;
     int phi;
+    int dim;               // D = M: 64, or 32 (tiles zero-padded to 64 columns)
 };
 
 // ---------------------------------------------------------------------------
@@ -181,8 +182,8 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             if (*abort_flag) break;
             if (prm.phi == LA_PHI_ELU1) {
                 uint8_t* rowQ = smem + kOffStage + s * 3 * kTileBytes + t * 128;
-                phi_row_inplace(rowQ, r7);
-                phi_row_inplace(rowQ + kTileBytes, r7);
+                phi_row_inplace(rowQ, r7, prm.dim >> 3);
+                phi_row_inplace(rowQ + kTileBytes, r7, prm.dim >> 3);
                 fence_proxy_async_smem();
             }
             mbar_arrive(&bars->mapped[s]);
@@ -295,8 +296,8 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             {
                 const bool fin = (c == L - 1) && (seg == prm.nseg - 1);
                 state_to_smem(tmem + kColS, warp, lane, smem + kOffS, sZ,
-                              fin && prm.S_out ? prm.S_out + bh * (int64_t)(kDim * kDim) : nullptr,
-                              fin && prm.Z_out ? prm.Z_out + bh * kDim : nullptr);
+                              fin && prm.S_out ? prm.S_out + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
+                              fin && prm.Z_out ? prm.Z_out + bh * prm.dim : nullptr, prm.dim);
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();
@@ -348,10 +349,10 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     const int chunks = (int)(p.N / kChunk);
     const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
     CUtensorMap mQ, mK, mV, mO;
-    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mK, K, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mV, V, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mO, O, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mO, O, rows, kChunk, (int)p.D)) return rc;
     int* status = device_status_ptr();
     if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
 
@@ -376,6 +377,7 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     prm.nseg = sg.nseg;
     prm.eps = p.eps;
     prm.phi = p.phi;
+    prm.dim = (int)p.D;
     causal_fwd_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kThreads, kSmemBytes, st>>>(mQ, mK, mV, mO, prm);
     LA_LAUNCHED();
     return LA_OK;

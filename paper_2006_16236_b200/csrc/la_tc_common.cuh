@@ -43,8 +43,11 @@ int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMa
 int segment_totals(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
                    const float* dn, const float* dl, float* records, cudaStream_t st);
 
-// 2-D view of a [rows][64] bf16 tensor with a [box_rows][64] box and the 128-byte swizzle.
-int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows);
+// 2-D view of a [rows][cols] bf16 tensor (cols = 32 or 64) with a [box_rows][64] box and the
+// 128-byte swizzle.  With cols = 32 the upper half of every 128-byte tile row is out of bounds:
+// loads fill it with zeros (zero features and zero values contribute nothing to any product),
+// stores clip it.  The kernels then run as for 64 and only touch `cols` columns in global memory.
+int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols = kDim);
 
 // ---------------------------------------------------------------------------
 // Feature map on one 128-byte row of a swizzled tile, in place: thread-per-row.
@@ -75,15 +78,17 @@ __device__ __forceinline__ void load_row(const uint8_t* row, uint32_t r7, uint32
 #pragma unroll
     for (int c = 0; c < 8; ++c) lds128(row + ((c ^ r7) << 4), v[c]);
 }
-__device__ __forceinline__ void store_row(uint8_t* row, uint32_t r7, const uint32_t (&v)[8][4]) {
+// first `nch` logical chunks only (nch = 4 when the row holds 32 real columns)
+__device__ __forceinline__ void store_row(uint8_t* row, uint32_t r7, const uint32_t (&v)[8][4], int nch = 8) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) sts128(row + ((c ^ r7) << 4), v[c][0], v[c][1], v[c][2], v[c][3]);
+    for (int c = 0; c < 8; ++c)
+        if (c < nch) sts128(row + ((c ^ r7) << 4), v[c][0], v[c][1], v[c][2], v[c][3]);
 }
 
 // Feature map on one row in place (optionally scaled): all loads first, then the arithmetic,
 // then all stores.
 template <bool kElu>
-__device__ __forceinline__ void map_row_inplace(uint8_t* row, uint32_t r7, float scale) {
+__device__ __forceinline__ void map_row_inplace(uint8_t* row, uint32_t r7, float scale, int nch = 8) {
     uint32_t v[8][4];
     load_row(row, r7, v);
 #pragma unroll
@@ -93,9 +98,11 @@ __device__ __forceinline__ void map_row_inplace(uint8_t* row, uint32_t r7, float
             const float x0 = sm100::bf16_lo(v[c][j]), x1 = sm100::bf16_hi(v[c][j]);
             v[c][j] = sm100::pack_bf16x2((kElu ? phi_fast(x0) : x0) * scale, (kElu ? phi_fast(x1) : x1) * scale);
         }
-    store_row(row, r7, v);
+    store_row(row, r7, v, nch);          // the zero padding of a 32-column row stays zero
 }
-__device__ __forceinline__ void phi_row_inplace(uint8_t* row, uint32_t r7) { map_row_inplace<true>(row, r7, 1.f); }
+__device__ __forceinline__ void phi_row_inplace(uint8_t* row, uint32_t r7, int nch = 8) {
+    map_row_inplace<true>(row, r7, 1.f, nch);
+}
 
 __device__ __forceinline__ uint64_t desc_k(uint32_t addr) { return sm100::umma_desc_sw128(addr, 16, 1024); }
 __device__ __forceinline__ uint64_t desc_mn(uint32_t addr, uint32_t lbo = kTileBytes) {
@@ -136,7 +143,7 @@ __device__ __forceinline__ void score_block_store(const uint32_t (&v)[32], uint8
 // of S followed by Z) -> bf16 [64][64] swizzled tile + fp32 Z; optionally the fp32 values to
 // global memory.  Executed by the four warps of one warpgroup; `quad` = warp % 4.
 __device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, float* z_out,
-                                              float* g_S, float* g_Z) {
+                                              float* g_S, float* g_Z, int dim = kDim) {
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
@@ -155,9 +162,9 @@ __device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int
                        sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
                        sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
             }
-            if (g_S) {
+            if (g_S && d_row < dim && h * 32 < dim) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) g_S[d_row * kDim + h * 32 + j] = __uint_as_float(v[j]);
+                for (int j = 0; j < 32; ++j) g_S[d_row * dim + h * 32 + j] = __uint_as_float(v[j]);
             }
         }
     }
@@ -165,7 +172,7 @@ __device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int
     sm100::tmem_ld_wait();
     if (owner) {
         z_out[d_row] = z;
-        if (g_Z) g_Z[d_row] = z;
+        if (g_Z && d_row < dim) g_Z[d_row] = z;
     }
 }
 

@@ -48,7 +48,7 @@ __device__ __forceinline__ float elu_fast(float x) {      // elu(x) = phi(x) - 1
 
 // elu (optionally scaled) on one row of a swizzled tile, in place; returns nothing.
 template <bool kElu>
-__device__ __forceinline__ void elu_row_inplace(uint8_t* row, uint32_t r7, float scale) {
+__device__ __forceinline__ void elu_row_inplace(uint8_t* row, uint32_t r7, float scale, int nch) {
     uint32_t v[8][4];
     load_row(row, r7, v);
 #pragma unroll
@@ -58,7 +58,7 @@ __device__ __forceinline__ void elu_row_inplace(uint8_t* row, uint32_t r7, float
             const float x0 = bf16_lo(v[c][j]), x1 = bf16_hi(v[c][j]);
             v[c][j] = pack_bf16x2((kElu ? elu_fast(x0) : x0 - 1.f) * scale, (kElu ? elu_fast(x1) : x1 - 1.f) * scale);
         }
-    store_row(row, r7, v);
+    store_row(row, r7, v, nch);          // the zero padding of a 32-column row stays zero
 }
 
 // ===========================================================================
@@ -87,6 +87,7 @@ struct LsParams {
     int64_t N;
     int chunks, chunks_per_seg, nseg;
     int phi;
+    int dim;
 };
 
 __global__ void __launch_bounds__(kLsThreads, 1)
@@ -188,7 +189,7 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             if (!mbar_wait(&bars->full[s], (c / kLsStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             uint8_t* rowX = smem + s * kLsStageBytes + t * 128;
-            if (elu) elu_row_inplace<true>(rowX, r7, w); else elu_row_inplace<false>(rowX, r7, w);
+            if (elu) elu_row_inplace<true>(rowX, r7, w, prm.dim >> 3); else elu_row_inplace<false>(rowX, r7, w, prm.dim >> 3);
             if (reverse) {
                 uint8_t* rowW = rowX + 2 * kTileBytes;
                 uint8_t* rowA = rowX + 3 * kTileBytes;
@@ -273,6 +274,7 @@ struct ApParams {
     int chunks, chunks_per_seg, nseg;
     float eps;
     int phi;
+    int dim;                    // D = M: 64, or 32 (tiles zero-padded to 64 columns)
 };
 
 template <int kMode>
@@ -335,19 +337,20 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             else sScal[1] = z;
         }
         __syncthreads();
-        if (tid < kDim) {               // column tid: mean over d; nu = ysum + mu
+        const int dim = prm.dim;
+        if (tid < kDim) {               // column tid: mean over the dim real rows; nu = ysum + mu
             float m = 0.f;
-            for (int d = 0; d < kDim; ++d) m += sF[d * kDim + tid];
-            m *= 1.f / kDim;
+            for (int d = 0; d < dim; ++d) m += sF[d * kDim + tid];
+            m *= 1.f / dim;
             const float ysum = sNu[tid];
             sNu[tid] = ysum + m;
             sF[kDim * kDim + tid] = m;                                            // mu, just past the matrix
-            if (kMode == kApplyForward && seg == 0) {
+            if (kMode == kApplyForward && seg == 0 && tid < dim) {
                 // true sums for the caller: S = 1 ysum^T + A', Z = N 1 + a'
-                if (prm.vec_out) prm.vec_out[bh * kDim + tid] = (float)prm.N + sA[tid];
+                if (prm.vec_out) prm.vec_out[bh * dim + tid] = (float)prm.N + sA[tid];
                 if (prm.state_out)
-                    for (int d = 0; d < kDim; ++d)
-                        prm.state_out[bh * (int64_t)(kDim * kDim) + d * kDim + tid] = sF[d * kDim + tid] + ysum;
+                    for (int d = 0; d < dim; ++d)
+                        prm.state_out[bh * (int64_t)(dim * dim) + d * dim + tid] = sF[d * kDim + tid] + ysum;
             }
         }
         if (tid == 64) {
@@ -360,7 +363,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             const int d = idx >> 3, c8 = idx & 7;
             float v[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = sF[d * kDim + c8 * 8 + j] - sF[kDim * kDim + c8 * 8 + j];
+            for (int j = 0; j < 8; ++j) v[j] = d < dim ? sF[d * kDim + c8 * 8 + j] - sF[kDim * kDim + c8 * 8 + j] : 0.f;
             sts128(smem + kApOffState + d * 128 + ((c8 ^ (d & 7)) << 4), pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]),
                    pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
         }
@@ -430,7 +433,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             if (!mbar_wait(&bars->full[s], (c / kApStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             uint8_t* rowX = smem + kApOffStage + s * 2 * kTileBytes + t * 128;
-            if (elu) elu_row_inplace<true>(rowX, r7, 1.f); else elu_row_inplace<false>(rowX, r7, 1.f);
+            if (elu) elu_row_inplace<true>(rowX, r7, 1.f, prm.dim >> 3); else elu_row_inplace<false>(rowX, r7, 1.f, prm.dim >> 3);
             fence_proxy_async_smem();
             mbar_arrive(&bars->mapped[s]);
         }
@@ -439,7 +442,8 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         const bool elu = prm.phi == LA_PHI_ELU1;
-        const float fD = (float)kDim, fN = (float)prm.N;
+        const float fD = (float)prm.dim, fN = (float)prm.N;
+        const int nhalf = prm.dim >> 5;             // 32-column halves that hold real columns
         for (int c = 0; c < L; ++c) {
             const int s = c % kApStages, b = c & 1;
             const int64_t row = row0 + (int64_t)c * kChunk + t;
@@ -479,7 +483,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             tmem_ld32(tmem + lane_base + b * 128, a0);
             tmem_ld32(tmem + lane_base + b * 128 + 32, a1);
             tmem_ld_wait();
-            __nv_bfloat16* dst = prm.out0 + row * kDim;
+            __nv_bfloat16* dst = prm.out0 + row * prm.dim;
             if (kMode == kApplyForward) {
                 // den = (1 + q') . (N 1 + Z');  num = (1 + q').1 nu + q' S''
                 const float den = fN * x1sum + sScal[0] + xa;
@@ -490,6 +494,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
+                        if (hh >= nhalf) break;
                         const uint32_t* acc = hh ? a1 : a0;
                         const float* nu = sNu + hh * 32 + cc * 8;
                         stg128(dst + hh * 32 + cc * 8,
@@ -533,6 +538,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
+                        if (hh >= nhalf) break;
                         uint32_t outp[4];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -553,11 +559,12 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     tmem_ld32(tmem + lane_base + b * 128 + 64, a0);
                     tmem_ld32(tmem + lane_base + b * 128 + 96, a1);
                     tmem_ld_wait();
-                    __nv_bfloat16* dstV = prm.out1 + row * kDim;
+                    __nv_bfloat16* dstV = prm.out1 + row * prm.dim;
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
                         for (int cc = 0; cc < 4; ++cc) {       // gV = (1 + k').1 nu_R + k' R''
+                            if (hh >= nhalf) break;
                             const uint32_t* acc = hh ? a1 : a0;
                             const float* nu = sNu + hh * 32 + cc * 8;
                             stg128(dstV + hh * 32 + cc * 8,
@@ -611,6 +618,7 @@ int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& 
     prm.chunks_per_seg = sg.chunks_per_seg;
     prm.nseg = sg.nseg;
     prm.phi = p.phi;
+    prm.dim = (int)p.D;
     linear_sum_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kLsThreads, kLsSmemBytes, st>>>(mX, mY, prm);
     LA_LAUNCHED();
     return LA_OK;
@@ -632,6 +640,7 @@ int launch_apply(const la_problem& p, const Segmentation& sg, const CUtensorMap&
     prm.nseg = sg.nseg;
     prm.eps = p.eps;
     prm.phi = p.phi;
+    prm.dim = (int)p.D;
     linear_apply_kernel<kMode><<<(unsigned)(sg.nseg * p.B * p.H), kApThreads, kApSmemBytes, st>>>(mX, mY, prm);
     LA_LAUNCHED();
     return LA_OK;
@@ -652,9 +661,9 @@ int linear_forward(const la_problem& p, const void* Q, const void* K, const void
     const Segmentation sg = choose_splits(p);
     const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
     CUtensorMap mQ, mK, mV;
-    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mK, K, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mV, V, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
     float* rec = (float*)ws;
     if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, rec, st)) return rc;
     ApParams a = {};
@@ -672,10 +681,10 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
     const size_t bh = (size_t)(p.B * p.H);
     const uint64_t rows = (uint64_t)(bh * p.N);
     CUtensorMap mQ, mK, mV, mG;
-    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mK, K, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mV, V, rows, kChunk)) return rc;
-    if (int rc = encode_tile_map(&mG, G, rows, kChunk)) return rc;
+    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mG, G, rows, kChunk, (int)p.D)) return rc;
     uint8_t* w = (uint8_t*)ws;
     float* rec_s = (float*)w;   w += bh * sg.nseg * kRecFloats * sizeof(float);
     float* rec_r = (float*)w;   w += bh * sg.nseg * kRecFloats * sizeof(float);

@@ -42,6 +42,7 @@ struct SumParams {
     int segs_per_seq;
     float eps;
     int phi;
+    int dim;
 };
 
 __global__ void __launch_bounds__(kSumThreads, 1)
@@ -136,7 +137,8 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             if (!mbar_wait(&bars->full[s], (c / kSumStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             uint8_t* rowX = smem + s * kSumStageBytes + t * 128;
-            if (prm.phi == LA_PHI_ELU1) map_row_inplace<true>(rowX, r7, inv); else if (scaled) map_row_inplace<false>(rowX, r7, inv);
+            if (prm.phi == LA_PHI_ELU1) map_row_inplace<true>(rowX, r7, inv, prm.dim >> 3);
+            else if (scaled) map_row_inplace<false>(rowX, r7, inv, prm.dim >> 3);
             if (scaled) {
                 uint8_t* rowA = rowX + 2 * kTileBytes;
                 const uint32_t dd = pack_bf16x2(delta, delta);      // columns 0..15 of the aux tile
@@ -212,6 +214,7 @@ int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMa
     prm.segs_per_seq = sg.nseg - 1;
     prm.eps = p.eps;
     prm.phi = p.phi;
+    prm.dim = (int)p.D;
     segment_sum_kernel<<<(unsigned)((sg.nseg - 1) * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
     LA_LAUNCHED();
     segment_scan_kernel<<<(unsigned)(p.B * p.H), 256, 0, st>>>(records, sg.nseg, reverse ? 1 : 0);
@@ -242,6 +245,7 @@ int segment_totals(const la_problem& p, const Segmentation& sg, const CUtensorMa
     prm.segs_per_seq = sg.nseg;
     prm.eps = p.eps;
     prm.phi = p.phi;
+    prm.dim = (int)p.D;
     segment_sum_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
     LA_LAUNCHED();
     return LA_OK;
