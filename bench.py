@@ -37,7 +37,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from an
 # ncu capture summarised under profiles/), keyed by workload; None until captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/ncu_full_causal_kernels_N16384.md
+    ("causal_sweep_bf16_N16384", "causal_fwd_kernel"): 519_617_792,
+    ("causal_sweep_bf16_N16384", "causal_bwd_dq_kernel"): 660_542_208,
+    ("causal_sweep_bf16_N16384", "causal_bwd_dkv_kernel"): 781_910_528,
+}
 
 
 def peaks():
@@ -75,8 +80,10 @@ def algorithmic_flops(w, part):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """Samples nvidia-smi clocks and throttle reasons in the background; stop() keeps the samples that
+    fall inside the given wall-clock windows (the timed region, extended by identical steps when it is
+    shorter than a few sampling periods)."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -85,11 +92,12 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+                                       "-lms", "20", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             pass
 
-    def stop(self):
+    def stop(self, windows):
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
             return out
@@ -107,10 +115,14 @@ class ClockSampler:
             if len(c) < 9:
                 continue
             try:
-                sm.append(float(c[1]))
-                mx.append(float(c[2]))
+                ts = datetime.datetime.strptime(c[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                clock, cmax = float(c[1]), float(c[2])
             except ValueError:
                 continue
+            if not any(lo <= ts <= hi for lo, hi in windows):
+                continue
+            sm.append(clock)
+            mx.append(cmax)
             for nm, val in zip(names, c[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(nm)
@@ -224,13 +236,38 @@ def time_steps(run, steps, warmup, world, split=None):
     return total, (f, b)
 
 
+# Compulsory HBM bytes of one launch of each main kernel, per token-head (D = M = dim, e = element bytes):
+# the tensors that kernel has to read or write once (tile inputs, outputs, per-position scalars).
+KERNEL_ALG_BYTES = {
+    "causal_fwd_kernel": lambda d, e: 4 * d * e + 4,            # Q, K, V in; O, den out
+    "causal_bwd_dq_kernel": lambda d, e: 5 * d * e + 8,         # Q, K, V, G in; dQ, dn, dl out
+    "causal_bwd_dkv_kernel": lambda d, e: 6 * d * e + 8,        # Q, K, V, G, dn, dl in; dK, dV out
+    "linear_apply_kernel": None,                                # three variants share the name: not ranked
+}
+
+
 def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True):
     s = CausalStep(la, w, dev, seed_offset=rank)
-    launches0 = la.la_kernel_launches()
     sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
-    total_ms, (fwd_ms, bwd_ms) = time_steps(None, steps, warmup, world, split=(s.fwd, s.bwd))
-    clocks = sampler.stop() if sampler else None
-    launches = (la.la_kernel_launches() - launches0) * steps // (steps + warmup)
+    for _ in range(warmup):
+        s.step()
+    torch.cuda.synchronize()
+    launches0 = la.la_kernel_launches()
+    la.la_profile_enable(True)
+    t_lo = time.time()
+    total_ms, (fwd_ms, bwd_ms) = time_steps(None, steps, 0, world, split=(s.fwd, s.bwd))
+    t_hi = time.time()
+    launches = la.la_kernel_launches() - launches0
+    kernels = la.la_profile_read()
+    la.la_profile_enable(False)
+    windows = [(t_lo, t_hi)]
+    if sampler:                 # the timed region may be shorter than a few sampling periods: keep the
+        t2 = time.time()        # same load running for half a second so that the clocks are seen under it
+        while time.time() - t2 < 0.5:
+            s.step()
+        torch.cuda.synchronize()
+        windows.append((t2, time.time()))
+    clocks = sampler.stop(windows) if sampler else None
     la.la_last_device_status()
     total_ms = max_over_ranks(total_ms, world, dev)
     ms = total_ms / steps
@@ -240,17 +277,25 @@ def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True):
         "gpu_launches": int(launches), "clocks": clocks,
         "alg_gbs": algorithmic_bytes(w, "both") / (fwd_ms + bwd_ms) * 1e-6,
         "alg_tflops": algorithmic_flops(w, "both") / (fwd_ms + bwd_ms) * 1e-9,
+        "kernels_ms": {k: {"ms_per_launch": v[0], "launches": v[1]} for k, v in kernels.items()},
     }
     res["hbm_frac"] = res["alg_gbs"] / pk["hbm_gbs"]
     res["tensor_frac_alg_flops"] = res["alg_tflops"] / pk["bf16_tflops_sustained"]
-    dom = "bwd" if bwd_ms >= fwd_ms else "fwd"
-    dom_ms = max(bwd_ms, fwd_ms)
-    ach = algorithmic_bytes(w, dom) / dom_ms * 1e-6
+    # dominant kernel: the one with the largest total time among those with a defined byte count
+    th = w.B * w.H * w.N
+    ranked = [(v[0] * v[1], k, v[0]) for k, v in kernels.items() if KERNEL_ALG_BYTES.get(k)]
+    if ranked:
+        _, dom, dom_ms = max(ranked)
+        dom_bytes = KERNEL_ALG_BYTES[dom](w.D, elem_bytes(w)) * th
+    else:                       # general kernels: one kernel per call
+        dom = ("la_causal_" if w.kind == "causal" else "la_linear_attention_") + ("backward" if bwd_ms >= fwd_ms else "forward")
+        dom_ms = max(bwd_ms, fwd_ms)
+        dom_bytes = algorithmic_bytes(w, "bwd" if bwd_ms >= fwd_ms else "fwd")
+    ach = dom_bytes / dom_ms * 1e-6
     res["roofline"] = {
-        "kernel": ("la_causal_" if w.kind == "causal" else "la_linear_attention_") + ("backward" if dom == "bwd" else "forward"),
-        "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
-        "peak_source": pk["source"] + " copy bandwidth",
-        "algorithmic_bytes_per_launch": algorithmic_bytes(w, dom), "ms_per_launch": dom_ms,
+        "kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
+        "peak_source": pk["source"] + " copy bandwidth (burst figure: the kernel is timed alone by its own event pair)",
+        "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms,
         "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
     }
     if do_e2e:
@@ -265,10 +310,13 @@ def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True):
     return res
 
 
-def bench_decode(la, w, dev, pk, n_steps=None):
+def bench_decode(la, w, dev, pk, n_steps=None, batch=None):
     """3072 sequential la_recurrent_step launches, timed as a whole: once issued one by one
     from the host, once replayed from a CUDA graph that holds the same 3072 launches."""
     T = n_steps or w.N
+    if batch:                   # same recipe, other batch size (a state that cannot stay in L2)
+        import dataclasses
+        w = dataclasses.replace(w, B=batch, N=T, name=f"{w.name}_B{batch}")
     Q, K, V, _ = draw_workload(w)
     q_t, k_t, v_t = (t[:, :, :T].permute(2, 0, 1, 3).contiguous().to(dev) for t in (Q, K, V))
     S = torch.zeros((w.B, w.H, w.D, w.M), device=dev)
@@ -313,7 +361,8 @@ def bench_decode(la, w, dev, pk, n_steps=None):
     res = {"workload": w.name, "steps_per_s": 1e6 / us, "us_per_step": us, "launches": T,
            "us_per_step_host_issued": us_eager, "us_per_step_cuda_graph": us_graph,
            "alg_gbs": gbs, "hbm_frac": gbs / pk["hbm_gbs"], "state_bytes": S.numel() * 4,
-           "note": "state (32 MiB) fits the 126 MB L2, so the fraction may exceed the DRAM roofline"}
+           "note": ("state fits the 126 MB L2, so the fraction may exceed the DRAM roofline"
+                    if S.numel() * 4 < 100e6 else "state exceeds L2: every step streams it from and to HBM")}
     if us_graph is None:
         res["graph_error"] = graph_error
     return res
@@ -420,10 +469,11 @@ def main():
                 continue
             if ww.kind == "decode":
                 rows[name] = bench_decode(la, ww, dev, pk)
+                rows[name + "_B2048"] = bench_decode(la, ww, dev, pk, n_steps=256, batch=2048)
             else:
                 r = bench_attention(la, ww, dev, k, wu, 1, 0, pk, do_e2e=False)
                 rows[name] = {kk: r[kk] for kk in ("value", "ms_per_step", "fwd_ms", "bwd_ms", "alg_gbs", "hbm_frac",
-                                                   "alg_tflops", "tensor_frac_alg_flops", "gpu_launches")}
+                                                   "alg_tflops", "tensor_frac_alg_flops", "gpu_launches", "kernels_ms")}
                 rows[name]["unit"] = "tokens/s"
 
     cpu = None
@@ -439,7 +489,7 @@ def main():
             "e2e": main_res.get("e2e"), "gpu_launches": main_res["gpu_launches"],
             "roofline": main_res["roofline"], "cpu_baseline": cpu,
             "breakdown": {kk: main_res[kk] for kk in ("fwd_ms", "bwd_ms", "alg_gbs", "hbm_frac", "alg_tflops",
-                                                      "tensor_frac_alg_flops")},
+                                                      "tensor_frac_alg_flops", "kernels_ms")},
             "peaks": {kk: pk.get(kk) for kk in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "source")},
             "rows": rows,
         }

@@ -185,6 +185,21 @@ int la_last_device_status(void* stream);
  * threads, all entry points); a diagnostic for benchmarks. */
 long long la_kernel_launches(void);
 
+/*
+ * Optional per-kernel timing (a measurement aid, no counterpart in the paper).  While
+ * switched on, every launch of the library's main kernels is bracketed by a pair of CUDA
+ * events recorded on the launch stream (up to 512 launches per kernel are kept).
+ * la_profile_enable(1) creates the events on first use and clears the counts;
+ * la_profile_enable(0) stops recording.  la_profile_read() waits for the recorded events and
+ * returns the mean duration in milliseconds and the number of launches of one kernel:
+ * 0 causal_fwd_kernel, 1 causal_bwd_dq_kernel, 2 causal_bwd_dkv_kernel, 3 segment_sum_kernel,
+ * 4 segment_scan_kernel, 5 linear_sum_kernel, 6 linear_apply_kernel, 7 recurrent_step_kernel.
+ * Not thread-safe; meant for a benchmark's single launching thread.
+ */
+int la_profile_enable(int on);
+int la_profile_read(int kernel, double* mean_ms, int* launches);
+const char* la_profile_kernel_name(int kernel);
+
 /* Library version, "major.minor". */
 const char* la_version(void);
 

@@ -23,7 +23,8 @@ EXPORTS = [
     "la_feature_map", "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
     "la_causal_forward",
     "la_causal_backward", "la_recurrent_step", "la_workspace_bytes", "la_status_string",
-    "la_last_error", "la_last_device_status", "la_kernel_launches", "la_version",
+    "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
+    "la_profile_kernel_name", "la_version",
 ]
 
 
@@ -67,6 +68,10 @@ def lib() -> ctypes.CDLL:
         L.la_last_device_status.argtypes = [vp]
         L.la_version.restype = ctypes.c_char_p
         L.la_kernel_launches.restype = ctypes.c_longlong
+        L.la_profile_enable.argtypes = [ctypes.c_int]
+        L.la_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int)]
+        L.la_profile_kernel_name.argtypes = [ctypes.c_int]
+        L.la_profile_kernel_name.restype = ctypes.c_char_p
         for name in EXPORTS:
             getattr(L, name)
         _lib = L
@@ -139,6 +144,21 @@ def la_workspace_bytes(p: la_problem, op: int) -> int:
 
 def la_kernel_launches() -> int:
     return int(lib().la_kernel_launches())
+
+
+def la_profile_enable(on: bool) -> None:
+    _check(lib().la_profile_enable(int(on)))
+
+
+def la_profile_read() -> dict:
+    """{kernel name: (mean ms per launch, launches)} for every kernel recorded since la_profile_enable(True)."""
+    out = {}
+    for k in range(8):
+        ms, n = ctypes.c_double(), ctypes.c_int()
+        _check(lib().la_profile_read(k, ctypes.byref(ms), ctypes.byref(n)))
+        if n.value:
+            out[lib().la_profile_kernel_name(k).decode()] = (ms.value, n.value)
+    return out
 
 
 def la_version() -> str:

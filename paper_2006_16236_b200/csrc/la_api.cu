@@ -28,6 +28,23 @@ int cuda_fail(cudaError_t e, const char* what) {
 static std::atomic<long long> g_launches{0};
 void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
+// ---- optional per-kernel event timing --------------------------------------
+static constexpr int kProfSamples = 512;
+static bool g_prof_on = false;
+static cudaEvent_t g_prof_ev[kProfCount][2][kProfSamples];
+static bool g_prof_created = false;
+static int g_prof_n[kProfCount];
+
+void prof_begin(int kernel, cudaStream_t st) {
+    if (!g_prof_on || g_prof_n[kernel] >= kProfSamples) return;
+    cudaEventRecord(g_prof_ev[kernel][0][g_prof_n[kernel]], st);
+}
+void prof_end(int kernel, cudaStream_t st) {
+    if (!g_prof_on || g_prof_n[kernel] >= kProfSamples) return;
+    cudaEventRecord(g_prof_ev[kernel][1][g_prof_n[kernel]], st);
+    ++g_prof_n[kernel];
+}
+
 __device__ int g_device_status_word = 0;
 
 int* device_status_ptr() {
@@ -111,6 +128,40 @@ const char* la_status_string(int status) {
 const char* la_last_error(void) { return g_error; }
 
 long long la_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int la_profile_enable(int on) {
+    if (on && !g_prof_created) {
+        for (int k = 0; k < kProfCount; ++k)
+            for (int e = 0; e < 2; ++e)
+                for (int i = 0; i < kProfSamples; ++i) LA_CUDA_TRY(cudaEventCreate(&g_prof_ev[k][e][i]));
+        g_prof_created = true;
+    }
+    for (int k = 0; k < kProfCount; ++k) g_prof_n[k] = 0;
+    g_prof_on = on != 0;
+    return LA_OK;
+}
+
+int la_profile_read(int kernel, double* mean_ms, int* launches) {
+    if (kernel < 0 || kernel >= kProfCount || !mean_ms || !launches) return fail(LA_ERR_INVALID_ARG, "bad profile query");
+    double total = 0.0;
+    const int n = g_prof_n[kernel];
+    for (int i = 0; i < n; ++i) {
+        LA_CUDA_TRY(cudaEventSynchronize(g_prof_ev[kernel][1][i]));
+        float ms = 0.f;
+        LA_CUDA_TRY(cudaEventElapsedTime(&ms, g_prof_ev[kernel][0][i], g_prof_ev[kernel][1][i]));
+        total += ms;
+    }
+    *launches = n;
+    *mean_ms = n ? total / n : 0.0;
+    return LA_OK;
+}
+
+const char* la_profile_kernel_name(int kernel) {
+    static const char* names[kProfCount] = {"causal_fwd_kernel", "causal_bwd_dq_kernel", "causal_bwd_dkv_kernel",
+                                            "segment_sum_kernel", "segment_scan_kernel", "linear_sum_kernel",
+                                            "linear_apply_kernel", "recurrent_step_kernel"};
+    return kernel >= 0 && kernel < kProfCount ? names[kernel] : "";
+}
 
 size_t la_workspace_bytes(const la_problem* p, int32_t op) {
     if (!p || p->B < 1 || p->H < 1 || p->N < 0 || p->D < 1 || p->M < 1 || p->D > 128 || p->M > 128) return 0;

@@ -33,6 +33,15 @@ int* device_status_ptr();
 // Every kernel launch of the library is counted (see la_kernel_launches()).
 void note_launch();
 
+// Optional per-kernel timing with CUDA events on the launch stream (see la_profile_enable()).
+// Indices are part of the C ABI (la_profile_read); no-ops unless profiling is switched on.
+enum ProfKernel {
+    kProfCausalFwd = 0, kProfCausalBwdDq = 1, kProfCausalBwdDkv = 2, kProfSegmentSum = 3, kProfSegmentScan = 4,
+    kProfLinearSum = 5, kProfLinearApply = 6, kProfRecurrent = 7, kProfCount = 8
+};
+void prof_begin(int kernel, cudaStream_t st);
+void prof_end(int kernel, cudaStream_t st);
+
 // ---- element access in the I/O type ----------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T x);
 template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }

@@ -184,8 +184,11 @@ static int recurrent_dispatch(const la_problem& p, const void* q, const void* k,
 
 int launch_recurrent_step(const la_problem& p, const void* q, const void* k, const void* v,
                           float* S, float* Z, void* out, cudaStream_t st) {
-    if (p.dtype == LA_F32) return recurrent_dispatch<float>(p, q, k, v, S, Z, out, st);
-    return recurrent_dispatch<__nv_bfloat16>(p, q, k, v, S, Z, out, st);
+    prof_begin(kProfRecurrent, st);
+    const int rc = p.dtype == LA_F32 ? recurrent_dispatch<float>(p, q, k, v, S, Z, out, st)
+                                     : recurrent_dispatch<__nv_bfloat16>(p, q, k, v, S, Z, out, st);
+    prof_end(kProfRecurrent, st);
+    return rc;
 }
 
 }  // namespace la

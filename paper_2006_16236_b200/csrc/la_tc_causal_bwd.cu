@@ -774,8 +774,10 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.eps = p.eps;
     a.phi = p.phi;
     a.dim = (int)p.D;
+    prof_begin(kProfCausalBwdDq, st);
     causal_bwd_dq_kernel<<<grid, kDqThreads, kDqSmemBytes, st>>>(mK, mV, mG, mQ, a);
     LA_LAUNCHED();
+    prof_end(kProfCausalBwdDq, st);
 
     // reverse sweep: dK, dV
     if (int rc = segment_states(p, sg, mQ, mG, dn, dl, rec_r, /*reverse=*/true, st)) return rc;
@@ -793,8 +795,10 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     b.eps = p.eps;
     b.phi = p.phi;
     b.dim = (int)p.D;
+    prof_begin(kProfCausalBwdDkv, st);
     causal_bwd_dkv_kernel<<<grid, kKvThreads, kKvSmemBytes, st>>>(mQ, mK, mV, mG, b);
     LA_LAUNCHED();
+    prof_end(kProfCausalBwdDkv, st);
     return LA_OK;
 }
 

@@ -378,8 +378,10 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     prm.eps = p.eps;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
+    prof_begin(kProfCausalFwd, st);
     causal_fwd_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kThreads, kSmemBytes, st>>>(mQ, mK, mV, mO, prm);
     LA_LAUNCHED();
+    prof_end(kProfCausalFwd, st);
     return LA_OK;
 }
 

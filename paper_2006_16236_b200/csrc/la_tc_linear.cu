@@ -619,8 +619,10 @@ int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& 
     prm.nseg = sg.nseg;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
+    prof_begin(kProfLinearSum, st);
     linear_sum_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kLsThreads, kLsSmemBytes, st>>>(mX, mY, prm);
     LA_LAUNCHED();
+    prof_end(kProfLinearSum, st);
     return LA_OK;
 }
 
@@ -641,8 +643,10 @@ int launch_apply(const la_problem& p, const Segmentation& sg, const CUtensorMap&
     prm.eps = p.eps;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
+    prof_begin(kProfLinearApply, st);
     linear_apply_kernel<kMode><<<(unsigned)(sg.nseg * p.B * p.H), kApThreads, kApSmemBytes, st>>>(mX, mY, prm);
     LA_LAUNCHED();
+    prof_end(kProfLinearApply, st);
     return LA_OK;
 }
 

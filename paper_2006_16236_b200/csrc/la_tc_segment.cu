@@ -215,10 +215,14 @@ int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMa
     prm.eps = p.eps;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
+    prof_begin(kProfSegmentSum, st);
     segment_sum_kernel<<<(unsigned)((sg.nseg - 1) * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
     LA_LAUNCHED();
+    prof_end(kProfSegmentSum, st);
+    prof_begin(kProfSegmentScan, st);
     segment_scan_kernel<<<(unsigned)(p.B * p.H), 256, 0, st>>>(records, sg.nseg, reverse ? 1 : 0);
     LA_LAUNCHED();
+    prof_end(kProfSegmentScan, st);
     return LA_OK;
 }
 
@@ -246,8 +250,10 @@ int segment_totals(const la_problem& p, const Segmentation& sg, const CUtensorMa
     prm.eps = p.eps;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
+    prof_begin(kProfSegmentSum, st);
     segment_sum_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
     LA_LAUNCHED();
+    prof_end(kProfSegmentSum, st);
     return LA_OK;
 }
 
