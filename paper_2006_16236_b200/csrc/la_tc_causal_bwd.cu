@@ -87,7 +87,8 @@ struct DqParams {
     float* dn;                  // out: dn_i = q_i . Z_i + eps per row, for the reverse sweep
     float* dl;                  // out: dl_i = -(G_i . O_i) per row, for the reverse sweep
     __nv_bfloat16* dQ;
-    const float* init;          // per (bh, seg) initial [S|Z] records or null
+    const float* init;          // per (bh, part) [S|Z] records of the pre-pass, or null (single segment)
+    int sub;                    // parts per segment
     int* status;
     int64_t N;
     int chunks, chunks_per_seg, nseg;
@@ -235,8 +236,8 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         const int quad = warp - 8;
         const int t = tid - 8 * 32;
         const uint32_t r7 = t & 7;
-        const float* init = prm.init ? prm.init + (bh * prm.nseg + seg) * (int64_t)kStateFloats : nullptr;
-        state_init(tmem + kDqColS, quad, lane, smem + kDqOffS, sZ + 2 * 64, init);      // "chunk -1" -> Z buffer 2
+        const float* rec = prm.init ? prm.init + bh * (int64_t)(prm.nseg * prm.sub) * kStateFloats : nullptr;
+        state_init(tmem + kDqColS, quad, lane, smem + kDqOffS, sZ + 2 * 64, rec, 0, rec ? seg * prm.sub : 0);   // "chunk -1" -> Z buffer 2
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(&bars->state_ready);
@@ -285,14 +286,23 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         float m_prev = 0.f;                                 // centring offset of the chunk whose epilogue is pending
 
         auto process_scores = [&](int c) -> float {         // chunk c: TMEM dP -> masked bf16 tile
-            uint32_t v0[32], v1[32];
             float m = 0.f;
-            if (has0) tmem_ld32(src + blk0 * 32, v0);
-            if (has1) tmem_ld32(src + blk1 * 32, v1);
-            if (c_begin + c == 0) m = __uint_as_float(tmem_ld1(src));      // first chunk of the sequence: centre on dP_i0
-            tmem_ld_wait();
-            if (has0) score_block_store(v0, tile_row, r7, blk0, blk0 == quad, lane, -m);
-            if (has1) score_block_store(v1, tile_row, r7, blk1, blk1 == quad, lane, -m);
+            if (c_begin + c == 0) {                          // first chunk of the sequence: centre on dP_i0
+                m = __uint_as_float(tmem_ld1(src));
+                tmem_ld_wait();
+            }
+            if (has0) {
+                uint32_t v[32];
+                tmem_ld32(src + blk0 * 32, v);
+                tmem_ld_wait();
+                score_block_store(v, tile_row, r7, blk0, blk0 == quad, lane, -m);
+            }
+            if (has1) {
+                uint32_t v[32];
+                tmem_ld32(src + blk1 * 32, v);
+                tmem_ld_wait();
+                score_block_store(v, tile_row, r7, blk1, blk1 == quad, lane, -m);
+            }
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->dp_ready);
@@ -434,7 +444,8 @@ struct KvParams {
     const float* dl;            // dl_i = -(G_i . O_i) from the forward sweep
     __nv_bfloat16* dK;
     __nv_bfloat16* dV;
-    const float* init;          // per (bh, seg) [R | r] records (sum over LATER segments) or null
+    const float* init;          // per (bh, part) [R | r] records of the pre-pass, or null (single segment)
+    int sub;
     int* status;
     int64_t N;
     int chunks, chunks_per_seg, nseg;
@@ -601,8 +612,9 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const int t = quad * 32 + lane;
         const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        const float* init = prm.init ? prm.init + (bh * prm.nseg + seg) * (int64_t)kStateFloats : nullptr;
-        state_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, init);      // "iteration -1" -> buffer 1
+        const float* rec = prm.init ? prm.init + bh * (int64_t)(prm.nseg * prm.sub) * kStateFloats : nullptr;
+        state_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, rec, rec ? (seg + 1) * prm.sub : 0,
+                   rec ? prm.nseg * prm.sub : 0);                                     // "iteration -1" -> buffer 1
         fence_proxy_async_smem();
         tc_fence_before_sync();
         named_barrier(1, 128);
@@ -724,7 +736,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
 size_t causal_backward_workspace(const la_problem& p) {
     const Segmentation sg = choose_segments(p);
     const size_t bh = (size_t)(p.B * p.H);
-    size_t bytes = 2 * bh * sg.nseg * kStateFloats * sizeof(float);      // forward and reverse segment records
+    size_t bytes = 2 * bh * sg.parts() * kStateFloats * sizeof(float);    // forward and reverse pre-pass records
     bytes += 2 * bh * (size_t)p.N * sizeof(float);                       // dn_i and dl_i per row
     return bytes;
 }
@@ -738,8 +750,8 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
 
     // workspace carve-up (see causal_backward_workspace)
     uint8_t* w = (uint8_t*)ws;
-    float* rec_s = (float*)w;            w += bh * sg.nseg * kStateFloats * sizeof(float);
-    float* rec_r = (float*)w;            w += bh * sg.nseg * kStateFloats * sizeof(float);
+    float* rec_s = (float*)w;            w += bh * sg.parts() * kStateFloats * sizeof(float);
+    float* rec_r = (float*)w;            w += bh * sg.parts() * kStateFloats * sizeof(float);
     float* dn = (float*)w;               w += bh * (size_t)p.N * sizeof(float);
     float* dl = (float*)w;
 
@@ -771,6 +783,7 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.chunks = chunks;
     a.chunks_per_seg = sg.chunks_per_seg;
     a.nseg = sg.nseg;
+    a.sub = sg.sub;
     a.eps = p.eps;
     a.phi = p.phi;
     a.dim = (int)p.D;
@@ -792,6 +805,7 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     b.chunks = chunks;
     b.chunks_per_seg = sg.chunks_per_seg;
     b.nseg = sg.nseg;
+    b.sub = sg.sub;
     b.eps = p.eps;
     b.phi = p.phi;
     b.dim = (int)p.D;

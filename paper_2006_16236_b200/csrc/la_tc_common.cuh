@@ -28,20 +28,18 @@ constexpr int kStateFloats = kDim * (kDim + 1);  // [S (64x64) | Z (64)] per rec
 
 // How a (batch, head) sequence is cut into segments that run concurrently.
 struct Segmentation {
-    int nseg;             // segments per sequence
+    int nseg;             // segments per sequence (one CTA of the main kernels each)
     int chunks_per_seg;   // chunks in every segment but possibly the last
+    int sub;              // parts per segment in the pre-pass (chunks_per_seg is a multiple of chunks_per_part)
+    int chunks_per_part;
+    int parts() const { return nseg * sub; }      // records per (batch, head)
 };
 
 Segmentation choose_segments(const la_problem& p);
 
 // Per-segment sums of phi(X)^T [Y | a] into `records` followed by their exclusive scan
-// (prefix, or suffix when `reverse`).  dn == nullptr: a = 1; otherwise the rows of phi(X) are
-// divided by dn and a = dl.  No-op for a single segment.
 int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
                    const float* dn, const float* dl, float* records, bool reverse, cudaStream_t st);
-
-int segment_totals(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
-                   const float* dn, const float* dl, float* records, cudaStream_t st);
 
 // 2-D view of a [rows][cols] bf16 tensor (cols = 32 or 64) with a [box_rows][64] box and the
 // 128-byte swizzle.  With cols = 32 the upper half of every 128-byte tile row is out of bounds:
@@ -176,31 +174,44 @@ __device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int
     }
 }
 
-// Load an initial [S | Z] record (or zeros) into the TMEM state accumulator, its bf16 tile and z_out.
+// Initial state of a segment: the sum of the records of parts [part_lo, part_hi) of this
+// (batch, head) (none: zeros) goes into the TMEM state accumulator, its bf16 tile and z_out.
 __device__ __forceinline__ void state_init(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, float* z_out,
-                                           const float* rec) {
+                                           const float* rec, int part_lo, int part_hi) {
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
+        float acc[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+        if (owner)
+            for (int p = part_lo; p < part_hi; ++p) {
+                const float4* src = reinterpret_cast<const float4*>(rec + (int64_t)p * kStateFloats + d_row * kDim + h * 32);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float4 a = __ldg(src + j);
+                    acc[4 * j] += a.x; acc[4 * j + 1] += a.y; acc[4 * j + 2] += a.z; acc[4 * j + 3] += a.w;
+                }
+            }
         uint32_t v[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = (rec && owner) ? __float_as_uint(rec[d_row * kDim + h * 32 + j]) : 0u;
+        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j]);
         sm100::tmem_st32(tmem_state + lane_base + h * 32, v);
         if (owner) {
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
                 const uint32_t chunk = h * 4 + cc;
                 sts128(s_tile + d_row * 128 + ((chunk ^ (d_row & 7)) << 4),
-                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
-                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
-                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
-                       sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
+                       sm100::pack_bf16x2(acc[cc * 8 + 0], acc[cc * 8 + 1]), sm100::pack_bf16x2(acc[cc * 8 + 2], acc[cc * 8 + 3]),
+                       sm100::pack_bf16x2(acc[cc * 8 + 4], acc[cc * 8 + 5]), sm100::pack_bf16x2(acc[cc * 8 + 6], acc[cc * 8 + 7]));
             }
         }
     }
-    const float z = (rec && owner) ? rec[kDim * kDim + d_row] : 0.f;
+    float z = 0.f;
+    if (owner)
+        for (int p = part_lo; p < part_hi; ++p) z += __ldg(rec + (int64_t)p * kStateFloats + kDim * kDim + d_row);
     uint32_t zz[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) zz[j] = __float_as_uint(z);

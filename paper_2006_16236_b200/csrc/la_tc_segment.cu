@@ -1,11 +1,10 @@
 // Segment pre-pass of the tensor-core causal kernels: per-segment sums of
 //     phi(X_i) [Y_i | a_i]^T        (64 x 65 per segment, fp32)
-// and their exclusive scan over the segments of a sequence.
-//   forward state  St: X = K, Y = V,            a_i = 1        (Eq. 10-11), exclusive prefix
-//   reverse state  Rt: X = Q (rows / dn_i), Y = G, a_i = dl_i  (the cumulative sum of Eq. 14-15),
-//                                                               exclusive suffix
-// so that every segment can start from the state the sequential recurrence would have
-// reached.  Warps 0-3: phi on X, scaling of Y and the final read-out; warp 4: TMA;
+// over parts of a sequence (a segment of the main kernels is one or several parts).
+//   forward state  St: X = K, Y = V,            a_i = 1        (Eq. 10-11)
+//   reverse state  Rt: X = Q (rows / dn_i), Y = G, a_i = dl_i  (the cumulative sum of Eq. 14-15)
+// A segment of the main kernels starts from the sum of the records before it (forward sweep)
+// or after it (reverse sweep): the state the sequential recurrence would have reached.  Warps 0-3: phi on X, scaling of Y and the final read-out; warp 4: TMA;
 // warp 5: MMA (M = 64 accumulators in TMEM).
 #include "la_tc.cuh"
 #include "la_tc_common.cuh"
@@ -18,7 +17,7 @@ using namespace sm100;
 namespace {
 
 constexpr int kSumThreads = 192;
-constexpr int kSumStages = 3;
+constexpr int kSumStages = 2;
 constexpr uint32_t kSumStageBytes = 3 * kTileBytes;                  // X, Y, aux column tile
 constexpr uint32_t kSumOffOnes = kSumStages * kSumStageBytes;
 constexpr uint32_t kSumOffBar = kSumOffOnes + 1024;
@@ -32,20 +31,20 @@ struct SumBarriers {
 };
 
 struct SumParams {
-    float* records;        // [BH][nseg][kStateFloats]
+    float* records;        // [BH][parts][kStateFloats]
     const float* dn;       // null: phi(X) is used as is and a_i = 1; else phi(X_i) is divided by dn_i
     const float* dl;       // with dn: a_i = dl_i
     int* status;
     int64_t N;
-    int chunks, chunks_per_seg, nseg;
-    int first_seg;         // segments first_seg .. first_seg + segs_per_seq - 1 are summed
-    int segs_per_seq;
+    int chunks, chunks_per_part, parts;
+    int first_part;        // parts first_part .. first_part + parts_per_seq - 1 are summed
+    int parts_per_seq;
     float eps;
     int phi;
     int dim;
 };
 
-__global__ void __launch_bounds__(kSumThreads, 1)
+__global__ void __launch_bounds__(kSumThreads, 2)
 segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                    const SumParams prm) {
     extern __shared__ uint8_t smem_raw[];
@@ -53,10 +52,10 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     const uint32_t sbase = smem_u32(smem);
     SumBarriers* bars = reinterpret_cast<SumBarriers*>(smem + kSumOffBar);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int seg = prm.first_seg + blockIdx.x % prm.segs_per_seq;
-    const int64_t bh = blockIdx.x / prm.segs_per_seq;
-    const int c_begin = seg * prm.chunks_per_seg;
-    const int L = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
+    const int seg = prm.first_part + blockIdx.x % prm.parts_per_seq;       // index of this part
+    const int64_t bh = blockIdx.x / prm.parts_per_seq;
+    const int c_begin = seg * prm.chunks_per_part;
+    const int L = min(prm.chunks, c_begin + prm.chunks_per_part) - c_begin;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
     const bool scaled = prm.dn != nullptr;
 
@@ -152,7 +151,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
         const bool ok = mbar_wait(&bars->done, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
         tc_fence_after_sync();
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        float* rec = prm.records + (bh * prm.nseg + seg) * (int64_t)kStateFloats;
+        float* rec = prm.records + (bh * prm.parts + seg) * (int64_t)kStateFloats;
         const int d_row = warp * 16 + lane;
         for (int h = 0; h < 2; ++h) {
             uint32_t v[32];
@@ -174,22 +173,6 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     }
 }
 
-// Exclusive scan over the segments of each (batch, head): forward -> record[s] = sum of the
-// records before s; reverse -> record[s] = sum of the records after s.  The record at the
-// open end (last for forward, first for reverse) was never computed and is not read.
-__global__ void __launch_bounds__(256) segment_scan_kernel(float* __restrict__ records, int nseg, int reverse) {
-    float* base = records + (int64_t)blockIdx.x * nseg * kStateFloats;
-    for (int i = threadIdx.x; i < kStateFloats; i += 256) {
-        float run = 0.f;
-        for (int n = 0; n < nseg; ++n) {
-            const int s = reverse ? nseg - 1 - n : n;
-            const float cur = n + 1 < nseg ? base[(int64_t)s * kStateFloats + i] : 0.f;
-            base[(int64_t)s * kStateFloats + i] = run;
-            run += cur;
-        }
-    }
-}
-
 }  // namespace
 
 int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
@@ -208,50 +191,15 @@ int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMa
     if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
     prm.N = p.N;
     prm.chunks = (int)(p.N / kChunk);
-    prm.chunks_per_seg = sg.chunks_per_seg;
-    prm.nseg = sg.nseg;
-    prm.first_seg = reverse ? 1 : 0;          // the open-end segment's own sum is never needed
-    prm.segs_per_seq = sg.nseg - 1;
+    prm.chunks_per_part = sg.chunks_per_part;
+    prm.parts = sg.parts();
+    prm.first_part = reverse ? sg.sub : 0;    // the open-end segment's own sums are never needed
+    prm.parts_per_seq = (sg.nseg - 1) * sg.sub;
     prm.eps = p.eps;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
     prof_begin(kProfSegmentSum, st);
-    segment_sum_kernel<<<(unsigned)((sg.nseg - 1) * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
-    LA_LAUNCHED();
-    prof_end(kProfSegmentSum, st);
-    prof_begin(kProfSegmentScan, st);
-    segment_scan_kernel<<<(unsigned)(p.B * p.H), 256, 0, st>>>(records, sg.nseg, reverse ? 1 : 0);
-    LA_LAUNCHED();
-    prof_end(kProfSegmentScan, st);
-    return LA_OK;
-}
-
-// Per-segment sums of ALL segments, no scan: the consumer adds the nseg records of a sequence
-// (the non-causal form needs the full sums of Eq. 5 only).
-int segment_totals(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
-                   const float* dn, const float* dl, float* records, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        LA_CUDA_TRY(cudaFuncSetAttribute(segment_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSumSmemBytes));
-        attr_done = true;
-    }
-    SumParams prm;
-    prm.records = records;
-    prm.dn = dn;
-    prm.dl = dl;
-    prm.status = device_status_ptr();
-    if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
-    prm.N = p.N;
-    prm.chunks = (int)(p.N / kChunk);
-    prm.chunks_per_seg = sg.chunks_per_seg;
-    prm.nseg = sg.nseg;
-    prm.first_seg = 0;
-    prm.segs_per_seq = sg.nseg;
-    prm.eps = p.eps;
-    prm.phi = p.phi;
-    prm.dim = (int)p.D;
-    prof_begin(kProfSegmentSum, st);
-    segment_sum_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
+    segment_sum_kernel<<<(unsigned)(prm.parts_per_seq * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
     LA_LAUNCHED();
     prof_end(kProfSegmentSum, st);
     return LA_OK;
