@@ -342,8 +342,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             tmem_ld32(tmem + lane_base + kDqColT + b * 64 + half * 32, tt);
             tmem_ld_wait();
             tc_fence_before_sync();
-            mbar_arrive(&bars->dq_drained[b]);              // both accumulators are in registers now
-            mbar_arrive(&bars->empty[s]);                   // and so is this thread's part of phi(Q)
+            mbar_arrive(&bars->empty[s]);                   // this thread's part of phi(Q) is in registers
             const float m = m_prev;
             float qg4[4] = {0.f, 0.f, 0.f, 0.f}, qz4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -360,6 +359,9 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                     qg4[j] = fmaf(q0, h0, fmaf(q1, h1, qg4[j]));
                     qz4[j] = fmaf(q0, z0, fmaf(q1, z1, qz4[j]));
                 }
+            // both accumulators are in registers and Z_{c-1} has been consumed: the MMA warp may reuse
+            // this accumulator pair, and the state warps the Z buffer (only after this arrival)
+            mbar_arrive(&bars->dq_drained[b]);
             // combine the two halves of the row
             float* xch = sX + (half * 128 + t) * 2;
             xch[0] = (qg4[0] + qg4[1]) + (qg4[2] + qg4[3]);

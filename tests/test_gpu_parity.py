@@ -184,6 +184,25 @@ def test_causal_workloads_full_size(name):
     assert torch.allclose(dV.float().sum(2), Gd.float().sum(2), rtol=5e-2, atol=0.5 * (w.N ** 0.5) * 2e-2 + 0.5)
 
 
+@pytest.mark.parametrize("name", ["causal_sweep_bf16_N8192", "causal_sweep_bf16_N32768", "noncausal_bf16_speech"])
+def test_results_are_repeatable_bit_for_bit(name):
+    """No atomics and a fixed summation order: repeated calls give identical bits.  A difference
+    between repeats means one warp role read a buffer while another was still writing it."""
+    w = WORKLOADS[name]
+    Q, K, V, G = gpu(*draw_workload(w))
+    fwd = la.la_causal_forward if w.kind == "causal" else la.la_linear_attention
+    bwd = la.la_causal_backward if w.kind == "causal" else la.la_linear_attention_backward
+    first = None
+    for _ in range(6):
+        cur = [fwd(Q, K, V)] + list(bwd(Q, K, V, G))
+        la.la_last_device_status()
+        if first is None:
+            first = [t.clone() for t in cur]
+        else:
+            for a, b, nm in zip(first, cur, ("O", "dQ", "dK", "dV")):
+                assert torch.equal(a, b), f"{name}: {nm} differs between repeats"
+
+
 def test_noncausal_workload_full_size():
     w = WORKLOADS["noncausal_bf16_speech"]
     dtype = w.torch_dtype
