@@ -29,6 +29,7 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
+from paper_2006_16236_b200 import shard  # noqa: E402
 from paper_2006_16236_b200.inputs import WORKLOADS, draw_qkvg, draw_workload  # noqa: E402
 
 METRIC = "causal LA fwd+bwd tokens/s"
@@ -134,38 +135,22 @@ class ClockSampler:
 
 
 def dist_setup(n_gpus):
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        import torch.distributed as dist
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    return world, rank, local
+    return shard.init_process_group("nccl")
 
 
 def barrier(world):
-    if world > 1:
-        import torch.distributed as dist
-        dist.barrier()
-    torch.cuda.synchronize()
+    shard.barrier(world)
 
 
 def max_over_ranks(x, world, dev):
-    if world == 1:
-        return x
-    import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device=dev)
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
+    return shard.max_over_ranks(x, world, dev)
 
 
 # --------------------------------------------------------------------------- GPU arms
 class CausalStep:
-    def __init__(self, la, w, dev, seed_offset=0):
+    def __init__(self, la, w, dev):
         self.la, self.w, self.dev = la, w, dev
-        Q, K, V, G = draw_qkvg(w.B, w.H, w.N, w.D, w.M, w.seed + seed_offset, w.torch_dtype, w.scale)
+        Q, K, V, G = draw_qkvg(w.B, w.H, w.N, w.D, w.M, w.seed, w.torch_dtype, w.scale)
         self.host = [t.pin_memory() for t in (Q, K, V, G)]
         self.d = [t.to(dev) for t in self.host]
         self.O = torch.empty_like(self.d[2])
@@ -247,7 +232,7 @@ KERNEL_ALG_BYTES = {
 
 
 def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True):
-    s = CausalStep(la, w, dev, seed_offset=rank)
+    s = CausalStep(la, shard.rank_workload(w, world, rank), dev)
     sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
     for _ in range(warmup):
         s.step()
