@@ -65,9 +65,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: returns false (after OR-ing `code` into *status) if the phase never
 // completes.  Callers then drain and leave; nothing spins for ever.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int code) {
+#pragma unroll 1
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (it > 64) __nanosleep(64);
+        if (it > 1024) __nanosleep(32);
     }
     if (status) atomicOr(status, code);
     return false;

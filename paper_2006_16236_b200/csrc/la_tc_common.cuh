@@ -14,11 +14,13 @@ namespace tc {
 // Optional pipeline trace (compile with -DLA_TC_TRACE): CTA 0 stamps clock64() per chunk and
 // event into a per-file buffer that la_debug_read_trace_*() copies out.  Compiled out otherwise.
 #ifdef LA_TC_TRACE
-#define LA_TRACE_DECL(name) __device__ long long name[512 * 32];
+#define LA_TRACE_DECL(name) __device__ long long name[1536 * 32];
 #define LA_TRACE(buf, c, slot) do { if (blockIdx.x == 0 && (c) < 512) buf[(c) * 32 + (slot)] = clock64(); } while (0)
+#define LA_TRACE_CTA(buf, slot) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); buf[(512 + (blockIdx.x & 1023)) * 32 + (slot)] = (long long)t_; } } while (0)
 #else
 #define LA_TRACE_DECL(name)
 #define LA_TRACE(buf, c, slot) do { } while (0)
+#define LA_TRACE_CTA(buf, slot) do { } while (0)
 #endif
 
 constexpr int kChunk = 128;                  // positions per chunk = MMA M
@@ -83,20 +85,26 @@ __device__ __forceinline__ void store_row(uint8_t* row, uint32_t r7, const uint3
         if (c < nch) sts128(row + ((c ^ r7) << 4), v[c][0], v[c][1], v[c][2], v[c][3]);
 }
 
-// Feature map on one row in place (optionally scaled): all loads first, then the arithmetic,
-// then all stores.
+// Feature map on one row in place (optionally scaled), two 16-byte chunks per iteration of a
+// rolled loop: the loop body stays small enough to live in the instruction cache next to the
+// other roles' loops (a fully unrolled row is 8 KB of code per call site).
 template <bool kElu>
 __device__ __forceinline__ void map_row_inplace(uint8_t* row, uint32_t r7, float scale, int nch = 8) {
-    uint32_t v[8][4];
-    load_row(row, r7, v);
+#pragma unroll 1
+    for (int c = 0; c < nch; c += 2) {
+        uint32_t v[2][4];
+        lds128(row + ((c ^ r7) << 4), v[0]);
+        lds128(row + (((c + 1) ^ r7) << 4), v[1]);
 #pragma unroll
-    for (int c = 0; c < 8; ++c)
+        for (int i = 0; i < 2; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float x0 = sm100::bf16_lo(v[c][j]), x1 = sm100::bf16_hi(v[c][j]);
-            v[c][j] = sm100::pack_bf16x2((kElu ? phi_fast(x0) : x0) * scale, (kElu ? phi_fast(x1) : x1) * scale);
-        }
-    store_row(row, r7, v, nch);          // the zero padding of a 32-column row stays zero
+            for (int j = 0; j < 4; ++j) {
+                const float x0 = sm100::bf16_lo(v[i][j]), x1 = sm100::bf16_hi(v[i][j]);
+                v[i][j] = sm100::pack_bf16x2((kElu ? phi_fast(x0) : x0) * scale, (kElu ? phi_fast(x1) : x1) * scale);
+            }
+        sts128(row + ((c ^ r7) << 4), v[0][0], v[0][1], v[0][2], v[0][3]);
+        sts128(row + (((c + 1) ^ r7) << 4), v[1][0], v[1][1], v[1][2], v[1][3]);
+    }
 }
 __device__ __forceinline__ void phi_row_inplace(uint8_t* row, uint32_t r7, int nch = 8) {
     map_row_inplace<true>(row, r7, 1.f, nch);
@@ -218,6 +226,128 @@ __device__ __forceinline__ void state_init(uint32_t tmem_state, int quad, int la
     sm100::tmem_st16(tmem_state + lane_base + 64, zz);
     sm100::tmem_st_wait();
     if (owner) z_out[d_row] = z;
+}
+
+// ---------------------------------------------------------------------------
+// Variants that keep Z as a bf16 MMA operand next to S: the 8 KB tile `z_tile` ([64][64]
+// swizzled, row d = Z_d in its first 16 columns) is the second 64-column block of an MN-major
+// B operand [S | Z] of width 80, so that q [S | Z] yields the numerator and q . Z in one MMA.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void z_row_store(uint8_t* z_tile, int d_row, float z) {
+    const uint32_t zz = sm100::pack_bf16x2(z, z);
+    uint8_t* row = z_tile + d_row * 128;
+    const uint32_t r7 = d_row & 7;
+    sts128(row + ((0 ^ r7) << 4), zz, zz, zz, zz);
+    sts128(row + ((1 ^ r7) << 4), zz, zz, zz, zz);
+}
+
+__device__ __forceinline__ void state_row_store(uint8_t* s_tile, int d_row, int h, const uint32_t (&v)[32]) {
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+        const uint32_t chunk = h * 4 + cc;
+        sts128(s_tile + d_row * 128 + ((chunk ^ (d_row & 7)) << 4),
+               sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
+               sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
+               sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
+               sm100::pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
+    }
+}
+
+// State accumulator -> registers (then `drained` is signalled: the accumulator may be updated
+// again) -> bf16 tiles; optionally the fp32 values to global memory.
+__device__ __forceinline__ void state_to_tiles(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, uint8_t* z_tile,
+                                               uint64_t* drained, float* g_S, float* g_Z, int dim) {
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const int d_row = quad * 16 + lane;
+    const bool owner = lane < 16;
+    uint32_t v[32];
+    sm100::tmem_ld32(tmem_state + lane_base, v);
+    sm100::tmem_ld_wait();
+    if (owner) {
+        state_row_store(s_tile, d_row, 0, v);
+        if (g_S && d_row < dim) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) g_S[d_row * dim + j] = __uint_as_float(v[j]);
+        }
+    }
+    sm100::tmem_ld32(tmem_state + lane_base + 32, v);
+    const float z = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 64));
+    sm100::tmem_ld_wait();
+    sm100::tc_fence_before_sync();
+    if (drained) sm100::mbar_arrive(drained);
+    if (owner) {
+        state_row_store(s_tile, d_row, 1, v);
+        z_row_store(z_tile, d_row, z);
+        if (g_S && d_row < dim && dim > 32) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) g_S[d_row * dim + 32 + j] = __uint_as_float(v[j]);
+        }
+        if (g_Z && d_row < dim) g_Z[d_row] = z;
+    }
+}
+
+// Initial state of a segment (sum of the records of parts [part_lo, part_hi), or zeros) into
+// the TMEM accumulator (S in 64 columns, Z replicated in 16) and the bf16 tiles.
+__device__ __forceinline__ void state_init_tiles(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, uint8_t* z_tile,
+                                                 const float* rec, int part_lo, int part_hi) {
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const int d_row = quad * 16 + lane;
+    const bool owner = lane < 16;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        float acc[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+        if (owner)
+            for (int p = part_lo; p < part_hi; ++p) {
+                const float4* src = reinterpret_cast<const float4*>(rec + (int64_t)p * kStateFloats + d_row * kDim + h * 32);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float4 a = __ldg(src + j);
+                    acc[4 * j] += a.x; acc[4 * j + 1] += a.y; acc[4 * j + 2] += a.z; acc[4 * j + 3] += a.w;
+                }
+            }
+        uint32_t v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j]);
+        sm100::tmem_st32(tmem_state + lane_base + h * 32, v);
+        if (owner) state_row_store(s_tile, d_row, h, v);
+    }
+    float z = 0.f;
+    if (owner)
+        for (int p = part_lo; p < part_hi; ++p) z += __ldg(rec + (int64_t)p * kStateFloats + kDim * kDim + d_row);
+    uint32_t zz[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) zz[j] = __float_as_uint(z);
+    sm100::tmem_st16(tmem_state + lane_base + 64, zz);
+    sm100::tmem_st_wait();
+    if (owner) z_row_store(z_tile, d_row, z);
+}
+
+// One 32-column block of fp32 scores -> 16 packed bf16 pairs (pair j = columns 2j, 2j+1), with
+// the causal mask on the diagonal block; a block above the diagonal (`present` false) is zeros.
+__device__ __forceinline__ void score_block_pack(const uint32_t (&v)[32], bool present, bool diagonal, int lane,
+                                                 uint32_t (&packed)[16]) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float x0 = __uint_as_float(v[2 * j]), x1 = __uint_as_float(v[2 * j + 1]);
+        if (diagonal) {
+            if (2 * j > lane) x0 = 0.f;
+            if (2 * j + 1 > lane) x1 = 0.f;
+        }
+        packed[j] = present ? sm100::pack_bf16x2(x0, x1) : 0u;
+    }
+}
+
+// tcgen05.mma with the A operand read from TMEM (bf16 pairs: column j of lane i = A[i][2j], A[i][2j+1]).
+__device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 
 }  // namespace tc
