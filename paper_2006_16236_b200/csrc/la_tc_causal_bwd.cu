@@ -163,6 +163,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG); prefetch_tensormap(&mapQ);
+            #pragma unroll 1
             for (int c = 0; c < L; ++c) {
                 const int s = c % kDqStages;
                 if (c >= kDqStages && !mbar_wait(&bars->empty[s], ((c / kDqStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
@@ -190,6 +191,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             const uint32_t aS = sbase + kDqOffS, aOnes = sbase + kDqOffOnes, aL = sbase + kDqOffL,
                            aDP = sbase + kDqOffDP;
             bool ok = true;
+            #pragma unroll 1
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kDqStages, b = c & 1;
                 const uint32_t aK = sbase + kDqOffStage + s * 4 * kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
@@ -256,6 +258,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             return true;
         };
         bool ok = map_chunk(0);
+        #pragma unroll 1
         for (int c = 0; c < L && ok; ++c) {
             if (c + 1 < L) ok = map_chunk(c + 1);
             if (!ok || *abort_flag) { ok = false; break; }
@@ -314,6 +317,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             tc_fence_after_sync();
             m_prev = process_scores(0);
         }
+        #pragma unroll 1
         for (int c = 0; c < L && ok; ++c) {
             const int s = c % kDqStages, b = c & 1;
             float m_next = 0.f;
@@ -508,6 +512,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG);
+            #pragma unroll 1
             for (int i = 0; i < L; ++i) {
                 const int s = i % kKvStages;
                 if (i >= kKvStages && !mbar_wait(&bars->empty[s], ((i / kKvStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
@@ -536,6 +541,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             const uint32_t aR = sbase + kKvOffR, aAux = sbase + kKvOffAux;
             const uint32_t aP = sbase + kKvOffP, aDP = sbase + kKvOffDP;
             bool ok = true;
+            #pragma unroll 1
             for (int i = 0; i < L && ok; ++i) {
                 const int s = i % kKvStages;
                 const uint32_t aQ = sbase + kKvOffStage + s * 4 * kTileBytes, aK = aQ + kTileBytes, aV = aK + kTileBytes,
@@ -583,6 +589,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const int t = tid - 12 * 32;
         const uint32_t r7 = t & 7;
         const bool elu = prm.phi == LA_PHI_ELU1;
+        #pragma unroll 1
         for (int i = 0; i < L; ++i) {
             const int s = i % kKvStages;
             const int64_t row = chunk_row(i) + t;
@@ -622,6 +629,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         named_barrier(1, 128);
         mbar_arrive(&bars->state_ready);
 
+        #pragma unroll 1
         for (int i = 0; i < L; ++i) {
             const int s = i % kKvStages;
             const int64_t row = chunk_row(i) + t;
@@ -699,6 +707,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const bool has0 = blk0 <= quad, has1 = blk1 <= quad;
         uint8_t* rowP = smem + kKvOffP + t * 128;
         uint8_t* rowDP = smem + kKvOffDP + t * 128;
+        #pragma unroll 1
         for (int i = 0; i < L; ++i) {
             const int s = i % kKvStages;
             if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout) ||

@@ -17,11 +17,11 @@
 // The only chain between chunks is the state (S update -> bf16 copy -> q S of the next chunk),
 // which runs one chunk ahead of its use.
 //
-// CTA = 18 warps.  Warps 0-7 ("score/epilogue" warps, two per TMEM quadrant: the pair
+// CTA = 19 warps.  Warps 0-7 ("score/epilogue" warps, two per TMEM quadrant: the pair
 // shares the 32 rows of the quadrant; one takes score columns 0-63 and output columns 0-31,
 // the other 64-127 and 32-63): mask and round P of chunk c, then the output epilogue of chunk
 // c-1.  Warps 8-11: phi(K) in place (two chunks ahead) and the state conversion.  Warps 12-15:
-// phi(Q) in place.  Warp 16: TMA.  Warp 17: MMA issue and TMEM allocation.
+// phi(Q) in place.  Warp 16: TMA.  Warps 17, 18: MMA issue (17 also allocates TMEM).
 #include "la_tc.cuh"
 #include "la_tc_common.cuh"
 
@@ -35,7 +35,7 @@ LA_TRACE_DECL(g_trace_fwd)
 namespace {
 
 constexpr int kStages = 4;
-constexpr int kThreads = 576;
+constexpr int kThreads = 608;
 constexpr uint32_t kTmemCols = 512;
 // TMEM columns
 constexpr uint32_t kColP = 0;        // 2 x 128: scores of even / odd chunks (fp32, then bf16 pairs in place)
@@ -55,7 +55,7 @@ static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
 struct Barriers {
     uint64_t full[kStages], empty[kStages], mapped[kStages];
-    uint64_t p_full[2], p_ready[2], o_full[2], o_drained[2], state_ready[2];
+    uint64_t p_full[2], p_ready[2], o_full[2], o_drained[2], state_ready[2], qs_full[2];
     uint64_t s_full, s_drained;
     uint32_t tmem_base;
     int abort_flag;
@@ -117,6 +117,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             mbar_init(&bars->o_full[b], 1);
             mbar_init(&bars->o_drained[b], 256);
             mbar_init(&bars->state_ready[b], 128);
+            mbar_init(&bars->qs_full[b], 1);
         }
         mbar_init(&bars->s_full, 1);
         mbar_init(&bars->s_drained, 128);
@@ -156,8 +157,13 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 tma_load_2d(st + 2 * kTileBytes, &mapV, 0, y, &bars->full[s]);
             }
         }
-    } else if (warp == 17) {
-        // ------------------------------------------------------------- MMA issuer
+    } else if (warp >= 17) {
+        // ------------------------------------------------------------- MMA issuers
+        // Two threads share the issue work (a tcgen05.mma occupies its issuing thread for about
+        // as long as it occupies the tensor pipe, and the waits of one stream would otherwise hold
+        // up the other): warp 17 issues the score products P and P [V | 1], warp 18 the state
+        // update and q [S | Z].  MMAs of one thread execute in order; the two accumulations into
+        // the same numerator are ordered through qs_full.
         if (lane == 0) {
             const uint32_t idesc_p = umma_idesc_bf16(128, 128, 0, 0);
             const uint32_t idesc_num = umma_idesc_bf16(128, 80, 0, 1);
@@ -173,66 +179,71 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             auto lo_mn = [&](uint32_t a, uint32_t lbo) { return (uint32_t)desc_mn(a, lbo); };
             auto stage_addr = [&](int c) { return sbase + kOffStage + (uint32_t)(c % kStages) * kStageBytes; };
             constexpr uint32_t kStepV1 = 128u - (128u << 16);
-            bool ok = mbar_wait(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !*abort_flag;
-            if (ok) {
-                tc_fence_after_sync();
-                const uint32_t dQ = lo_k(stage_addr(0)), dK = lo_k(stage_addr(0) + kTileBytes);
+            bool ok = true;
+            if (warp == 17) {
+                #pragma unroll 1
+                for (int c = -1; c < L && ok; ++c) {        // step c: P of chunk c + 1, then P [V | 1] of chunk c
+                    const int b = c & 1;
+                    if (c + 1 < L) {
+                        // the buffer's previous readers are done: p_ready(c-1) was awaited before
+                        // P [V | 1] of chunk c-1 was issued, and this thread's MMAs run in order
+                        ok = mbar_wait(&bars->mapped[(c + 1) % kStages], ((c + 1) / kStages) & 1, prm.status, kStatusPipeTimeout);
+                        if (!ok || *abort_flag) { ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t nQ = lo_k(stage_addr(c + 1)), nK = lo_k(stage_addr(c + 1) + kTileBytes);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColP, mk(dQ + 2 * k), mk(dK + 2 * k), idesc_p, k > 0);
-                umma_commit(&bars->p_full[0]);
-            }
-            #pragma unroll 1
-            for (int c = 0; c < L && ok; ++c) {
-                const int s = c % kStages, b = c & 1;
-                const uint32_t aQ = stage_addr(c), aK = aQ + kTileBytes, aV = aK + kTileBytes;
-                const uint32_t dQ = lo_k(aQ), dKmn = lo_mn(aK, kTileBytes), dV1 = lo_mn(aV, aOnes - aV);
-                LA_TRACE(g_trace_fwd, c, 0);
-                // (a) St_c = St_{c-1} + k^T [V | 1]: the accumulator must have been read out (or initialised)
-                ok = c == 0 ? mbar_wait(&bars->state_ready[1], 0, prm.status, kStatusPipeTimeout)
-                            : mbar_wait(&bars->s_drained, (c - 1) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok || *abort_flag) { ok = false; break; }
-                tc_fence_after_sync();
-#pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    umma_bf16(tmem + kColS, mk(dKmn + 128 * k), mk(dV1 + kStepV1 * k), idesc_s, 1);
-                umma_commit(&bars->s_full);
-                LA_TRACE(g_trace_fwd, c, 1);
-                // (b) scores of the next chunk into the other buffer (its previous readers are done:
-                //     p_ready(c-1) was awaited before P V of chunk c-1 was issued, and MMAs run in order)
-                if (c + 1 < L) {
-                    ok = mbar_wait(&bars->mapped[(c + 1) % kStages], ((c + 1) / kStages) & 1, prm.status, kStatusPipeTimeout);
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16(tmem + kColP + (b ^ 1) * 128, mk(nQ + 2 * k), mk(nK + 2 * k), idesc_p, k > 0);
+                        umma_commit(&bars->p_full[b ^ 1]);
+                    }
+                    if (c < 0) continue;
+                    LA_TRACE(g_trace_fwd, c, 2);
+                    // += P [V | 1] with the rounded, masked P read from TMEM, on top of q [S | Z]
+                    ok = mbar_wait(&bars->p_ready[b], (c >> 1) & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait(&bars->qs_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t nQ = lo_k(stage_addr(c + 1)), nK = lo_k(stage_addr(c + 1) + kTileBytes);
+                    LA_TRACE(g_trace_fwd, c, 3);
+                    const uint32_t aV = stage_addr(c) + 2 * kTileBytes;
+                    const uint32_t dV1 = lo_mn(aV, aOnes - aV);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16(tmem + kColP + (b ^ 1) * 128, mk(nQ + 2 * k), mk(nK + 2 * k), idesc_p, k > 0);
-                    umma_commit(&bars->p_full[b ^ 1]);
+                    for (int k = 0; k < 8; ++k)
+                        umma_bf16_ta(tmem + kColNum + b * kNumStride, tmem + kColP + b * 128 + (k >> 2) * 64 + (k & 3) * 8,
+                                     mk(dV1 + kStepV1 * k), idesc_num, 1);
+                    umma_commit(&bars->o_full[b]);
+                    // qs_full(c) was awaited: every MMA of either thread that reads this stage is covered
+                    umma_commit(&bars->empty[c % kStages]);
+                    LA_TRACE(g_trace_fwd, c, 4);
                 }
-                LA_TRACE(g_trace_fwd, c, 2);
-                // (c) [num | den] = q [S | Z]_{c-1}: tile (c-1) & 1 holds the state before this chunk
-                ok = mbar_wait(&bars->state_ready[b ^ 1], (c >> 1) & 1, prm.status, kStatusPipeTimeout);
-                if (ok && c >= 2) ok = mbar_wait(&bars->o_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok) break;
-                tc_fence_after_sync();
-                {
+            } else {
+                #pragma unroll 1
+                for (int c = 0; c < L && ok; ++c) {
+                    const int s = c % kStages, b = c & 1;
+                    const uint32_t aQ = stage_addr(c), aK = aQ + kTileBytes, aV = aK + kTileBytes;
+                    const uint32_t dQ = lo_k(aQ), dKmn = lo_mn(aK, kTileBytes), dV1 = lo_mn(aV, aOnes - aV);
+                    LA_TRACE(g_trace_fwd, c, 0);
+                    // St_c = St_{c-1} + k^T [V | 1]: the accumulator must have been read out (or initialised)
+                    ok = mbar_wait(&bars->mapped[s], (c / kStages) & 1, prm.status, kStatusPipeTimeout) &&
+                         (c == 0 ? mbar_wait(&bars->state_ready[1], 0, prm.status, kStatusPipeTimeout)
+                                 : mbar_wait(&bars->s_drained, (c - 1) & 1, prm.status, kStatusPipeTimeout));
+                    if (!ok || *abort_flag) { ok = false; break; }
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        umma_bf16(tmem + kColS, mk(dKmn + 128 * k), mk(dV1 + kStepV1 * k), idesc_s, 1);
+                    umma_commit(&bars->s_full);
+                    LA_TRACE(g_trace_fwd, c, 1);
+                    // [num | den] = q [S | Z]_{c-1}: tile (c-1) & 1 holds the state before this chunk
+                    ok = mbar_wait(&bars->state_ready[b ^ 1], (c >> 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (ok && c >= 2) ok = mbar_wait(&bars->o_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (!ok) break;
+                    tc_fence_after_sync();
                     const uint32_t dS = lo_mn(sbase + kOffS + (b ^ 1) * kStateTileBytes, kDim * 128);
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
                         umma_bf16(tmem + kColNum + b * kNumStride, mk(dQ + 2 * k), mk(dS + 128 * k), idesc_num, k > 0);
+                    umma_commit(&bars->qs_full[b]);
                 }
-                // (d) += P [V | 1] with the rounded, masked P read from TMEM
-                ok = mbar_wait(&bars->p_ready[b], (c >> 1) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok) break;
-                tc_fence_after_sync();
-                LA_TRACE(g_trace_fwd, c, 3);
-#pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    umma_bf16_ta(tmem + kColNum + b * kNumStride, tmem + kColP + b * 128 + (k >> 2) * 64 + (k & 3) * 8,
-                                 mk(dV1 + kStepV1 * k), idesc_num, 1);
-                umma_commit(&bars->o_full[b]);
-                umma_commit(&bars->empty[s]);
-                LA_TRACE(g_trace_fwd, c, 4);
             }
             if (!ok) *abort_flag = 1;
         }

@@ -132,6 +132,7 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     if (warp == 4) {
         if (lane == 0) {
             prefetch_tensormap(&mapX); prefetch_tensormap(&mapY);
+            #pragma unroll 1
             for (int c = 0; c < L; ++c) {
                 const int s = c % kLsStages;
                 if (c >= kLsStages && !mbar_wait(&bars->empty[s], ((c / kLsStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
@@ -152,6 +153,7 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
             const uint32_t aOnes = sbase + kLsOffOnes;
             bool ok = true;
+            #pragma unroll 1
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kLsStages;
                 const uint32_t aX = sbase + s * kLsStageBytes, aY = aX + kTileBytes, aW = aY + kTileBytes, aA = aW + kTileBytes;
@@ -178,6 +180,7 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         const int t = tid;
         const uint32_t r7 = t & 7;
         const bool elu = prm.phi == LA_PHI_ELU1;
+        #pragma unroll 1
         for (int c = 0; c < L; ++c) {
             const int s = c % kLsStages;
             const int64_t row = row0 + (int64_t)c * kChunk + t;
@@ -379,6 +382,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         if (lane == 0) {
             prefetch_tensormap(&mapX);
             if (kHasY) prefetch_tensormap(&mapY);
+            #pragma unroll 1
             for (int c = 0; c < L; ++c) {
                 const int s = c % kApStages;
                 if (c >= kApStages && !mbar_wait(&bars->empty[s], ((c / kApStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
@@ -399,6 +403,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
             const uint32_t aSt = sbase + kApOffState;
             bool ok = true;
+            #pragma unroll 1
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kApStages, b = c & 1;
                 const uint32_t aX = sbase + kApOffStage + s * 2 * kTileBytes, aY = aX + kTileBytes;
@@ -428,6 +433,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         const int t = tid - 128;
         const uint32_t r7 = t & 7;
         const bool elu = prm.phi == LA_PHI_ELU1;
+        #pragma unroll 1
         for (int c = 0; c < L; ++c) {
             const int s = c % kApStages;
             if (!mbar_wait(&bars->full[s], (c / kApStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
@@ -444,6 +450,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         const bool elu = prm.phi == LA_PHI_ELU1;
         const float fD = (float)prm.dim, fN = (float)prm.N;
         const int nhalf = prm.dim >> 5;             // 32-column halves that hold real columns
+        #pragma unroll 1
         for (int c = 0; c < L; ++c) {
             const int s = c % kApStages, b = c & 1;
             const int64_t row = row0 + (int64_t)c * kChunk + t;

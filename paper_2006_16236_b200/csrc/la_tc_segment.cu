@@ -86,6 +86,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     if (warp == 4) {
         if (lane == 0) {
             prefetch_tensormap(&mapX); prefetch_tensormap(&mapY);
+            #pragma unroll 1
             for (int c = 0; c < L; ++c) {
                 const int s = c % kSumStages;
                 if (c >= kSumStages && !mbar_wait(&bars->empty[s], ((c / kSumStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
@@ -106,6 +107,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
             const uint32_t aOnes = sbase + kSumOffOnes;
             bool ok = true;
+            #pragma unroll 1
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kSumStages;
                 const uint32_t aX = sbase + s * kSumStageBytes, aY = aX + kTileBytes, aA = aY + kTileBytes;
@@ -125,6 +127,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     } else {
         const int t = tid;
         const uint32_t r7 = t & 7;
+        #pragma unroll 1
         for (int c = 0; c < L; ++c) {
             const int s = c % kSumStages;
             const int64_t row = row0 + (int64_t)c * kChunk + t;
@@ -136,7 +139,10 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             if (!mbar_wait(&bars->full[s], (c / kSumStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             uint8_t* rowX = smem + s * kSumStageBytes + t * 128;
-            if (prm.phi == LA_PHI_ELU1) map_row_inplace<true>(rowX, r7, inv, prm.dim >> 3);
+            if (prm.phi == LA_PHI_ELU1) {
+                if (scaled) map_row_inplace<true>(rowX, r7, inv, prm.dim >> 3);
+                else phi_row_inplace(rowX, r7, prm.dim >> 3);
+            }
             else if (scaled) map_row_inplace<false>(rowX, r7, inv, prm.dim >> 3);
             if (scaled) {
                 uint8_t* rowA = rowX + 2 * kTileBytes;
