@@ -158,11 +158,13 @@ class CausalStep:
         self.grads = [torch.empty_like(self.d[0]), torch.empty_like(self.d[1]), torch.empty_like(self.d[2])]
         self.host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in [self.O] + self.grads]
         self.causal = w.kind == "causal"
+        # a training step keeps phi(Q), phi(K) from the forward for the backward (None: nothing to keep)
+        self.saved = la.saved_buffer(self.d[0], self.d[2]) if self.causal else None
 
     def fwd(self):
         Q, K, V, _ = self.d
         if self.causal:
-            self.la.la_causal_forward(Q, K, V, O=self.O, den=self.den)
+            self.la.la_causal_forward(Q, K, V, O=self.O, den=self.den, saved=self.saved)
         else:
             self.la.la_linear_attention(Q, K, V, O=self.O, den=self.den)
 
@@ -170,7 +172,7 @@ class CausalStep:
         Q, K, V, G = self.d
         dQ, dK, dV = self.grads
         if self.causal:
-            self.la.la_causal_backward(Q, K, V, G, O=self.O, den=self.den, dQ=dQ, dK=dK, dV=dV)
+            self.la.la_causal_backward(Q, K, V, G, O=self.O, den=self.den, saved=self.saved, dQ=dQ, dK=dK, dV=dV)
         else:
             self.la.la_linear_attention_backward(Q, K, V, G, O=self.O, den=self.den, dQ=dQ, dK=dK, dV=dV)
 

@@ -64,7 +64,8 @@ typedef enum {
     LA_OP_LINEAR_FORWARD = 0,
     LA_OP_LINEAR_BACKWARD = 1,
     LA_OP_CAUSAL_FORWARD = 2,
-    LA_OP_CAUSAL_BACKWARD = 3
+    LA_OP_CAUSAL_BACKWARD = 3,
+    LA_OP_CAUSAL_SAVED = 4       /* size of the optional `saved` buffer, see la_causal_forward() */
 } la_op;
 
 typedef struct {
@@ -110,9 +111,16 @@ int la_linear_attention_backward(const la_problem* p, const void* Q, const void*
  *   O_i = phi(Q_i)^T S_i / (phi(Q_i)^T Z_i + eps)       (position i sees j <= i).
  * den (optional): phi(Q_i)^T Z_i without eps.  S_out / Z_out (optional): the final
  * state S_N, Z_N, which continues the sequence through la_recurrent_step().
+ * saved (optional, device, 128-byte aligned, la_workspace_bytes(p, LA_OP_CAUSAL_SAVED)
+ * bytes, owned by the caller): what a training step keeps for the backward pass, as the
+ * paper's autograd function keeps phi(Q), phi(K): the mapped queries and keys and the
+ * per-segment sums of the forward pre-pass.  Its layout is private to the library; it is
+ * valid for la_causal_backward() with the same problem, Q, K and V until overwritten.  The
+ * size is 0 for problems that run the general kernels (pass NULL, or any pointer).
  */
 int la_causal_forward(const la_problem* p, const void* Q, const void* K, const void* V,
                       void* O, float* den, float* S_out, float* Z_out,
+                      void* saved, size_t saved_bytes,
                       void* ws, size_t ws_bytes, void* stream);
 
 /*
@@ -121,9 +129,15 @@ int la_causal_forward(const la_problem* p, const void* Q, const void* K, const v
  * sum of phi(K_j)[V_j,1]^T, grad phi(K_i) and grad V_i the reverse running sum of
  * phi(Q_j) Gt_j^T, where Gt_j = [G_j/den_j, -(G_j.O_j)/den_j] carries the division.
  * No per-position state is stored.  G = dL/dO.  O and den may be NULL (recomputed).
+ * saved (optional): the buffer a la_causal_forward() call on the same problem and inputs
+ * filled.  With it the backward pass reads phi(Q), phi(K) instead of recomputing them from
+ * Q and K and skips its forward pre-pass; without it (NULL) everything is recomputed.  The
+ * gradients agree with the recomputing path to rounding (phi(Q)/den is rounded from the
+ * saved bf16 phi(Q) instead of the fp32 value).
  */
 int la_causal_backward(const la_problem* p, const void* Q, const void* K, const void* V,
                        const void* O, const float* den, const void* G,
+                       const void* saved, size_t saved_bytes,
                        void* dQ, void* dK, void* dV,
                        void* ws, size_t ws_bytes, void* stream);
 

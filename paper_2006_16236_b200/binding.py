@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libla.so")
 LA_F32, LA_BF16 = 0, 1
 LA_PHI_ELU1, LA_PHI_IDENTITY = 0, 1
 LA_OP_LINEAR_FORWARD, LA_OP_LINEAR_BACKWARD, LA_OP_CAUSAL_FORWARD, LA_OP_CAUSAL_BACKWARD = 0, 1, 2, 3
+LA_OP_CAUSAL_SAVED = 4
 _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
@@ -57,8 +58,8 @@ def lib() -> ctypes.CDLL:
         L.la_linear_attention.argtypes = [pp] + [vp] * 7 + [vp, sz, vp]
         L.la_linear_attention_noalloc.argtypes = [pp] + [vp] * 7 + [vp]
         L.la_linear_attention_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
-        L.la_causal_forward.argtypes = [pp] + [vp] * 7 + [vp, sz, vp]
-        L.la_causal_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
+        L.la_causal_forward.argtypes = [pp] + [vp] * 7 + [vp, sz] + [vp, sz, vp]
+        L.la_causal_backward.argtypes = [pp] + [vp] * 6 + [vp, sz] + [vp] * 3 + [vp, sz, vp]
         L.la_recurrent_step.argtypes = [pp] + [vp] * 6 + [vp]
         L.la_workspace_bytes.argtypes = [pp, i32]
         L.la_workspace_bytes.restype = sz
@@ -217,28 +218,40 @@ def la_linear_attention_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=No
     return dQ, dK, dV
 
 
-def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None, Z_out=None, ws=None):
-    """Causal form.  Returns O; pass preallocated den / S_out / Z_out tensors to receive them."""
-    dev = _dev(Q, K, V, O, den, S_out, Z_out)
+def _nbytes(t):
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def saved_buffer(Q, V, phi="elu1", eps=0.0):
+    """A buffer for what la_causal_forward() keeps for la_causal_backward() (None if the problem needs none)."""
+    p = _problem_of(Q, V, phi, eps)
+    need = lib().la_workspace_bytes(ctypes.byref(p), LA_OP_CAUSAL_SAVED)
+    return None if need == 0 else torch.empty(need, dtype=torch.uint8, device=Q.device)
+
+
+def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None, Z_out=None, saved=None, ws=None):
+    """Causal form.  Returns O; pass preallocated den / S_out / Z_out tensors to receive them, and a
+    saved_buffer() to keep phi(Q), phi(K) for the backward pass."""
+    dev = _dev(Q, K, V, O, den, S_out, Z_out, saved)
     p = _problem_of(Q, V, phi, eps)
     O = torch.empty_like(V) if O is None else O
     ws = workspace(p, LA_OP_CAUSAL_FORWARD, dev) if ws is None else ws
     _check(lib().la_causal_forward(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(S_out),
-                                   _ptr(Z_out), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
-                                   _stream(dev)))
+                                   _ptr(Z_out), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(dev)))
     return O
 
 
-def la_causal_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None, dQ=None, dK=None, dV=None, ws=None):
-    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV)
+def la_causal_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None, saved=None, dQ=None, dK=None, dV=None,
+                       ws=None):
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved)
     p = _problem_of(Q, V, phi, eps)
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(V) if dV is None else dV
     ws = workspace(p, LA_OP_CAUSAL_BACKWARD, dev) if ws is None else ws
     _check(lib().la_causal_backward(
-        ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV),
-        _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(dev)))
+        ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(saved), _nbytes(saved),
+        _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), _nbytes(ws), _stream(dev)))
     return dQ, dK, dV
 
 

@@ -104,6 +104,15 @@ static int check_ws(const la_problem* p, int op, const void* ws, size_t ws_bytes
     return LA_OK;
 }
 
+// `saved` is optional; when given it must hold la_workspace_bytes(p, LA_OP_CAUSAL_SAVED) bytes.
+static int check_saved(const la_problem* p, const void* saved, size_t saved_bytes) {
+    if (!saved) return LA_OK;
+    const size_t need = la_workspace_bytes(p, LA_OP_CAUSAL_SAVED);
+    if (!aligned16(saved) || ((uintptr_t)saved & 127)) return fail(LA_ERR_INVALID_ARG, "saved buffer is not 128-byte aligned");
+    if (saved_bytes < need) return fail(LA_ERR_WORKSPACE, "saved buffer has %zu bytes, %zu are needed", saved_bytes, need);
+    return LA_OK;
+}
+
 }  // namespace la
 
 using namespace la;
@@ -165,8 +174,9 @@ const char* la_profile_kernel_name(int kernel) {
 
 size_t la_workspace_bytes(const la_problem* p, int32_t op) {
     if (!p || p->B < 1 || p->H < 1 || p->N < 0 || p->D < 1 || p->M < 1 || p->D > 128 || p->M > 128) return 0;
-    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_CAUSAL_BACKWARD) return 0;
+    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_CAUSAL_SAVED) return 0;
     if (p->N == 0) return 0;
+    if (op == LA_OP_CAUSAL_SAVED) return tc_supported(*p, LA_OP_CAUSAL_BACKWARD) ? tc_causal_saved_bytes(*p) : 0;
     if (tc_supported(*p, op)) return tc_workspace_bytes(*p, op);
     return general_workspace_bytes(*p, op);
 }
@@ -213,31 +223,37 @@ int la_linear_attention_backward(const la_problem* p, const void* Q, const void*
 
 int la_causal_forward(const la_problem* p, const void* Q, const void* K, const void* V,
                       void* O, float* den, float* S_out, float* Z_out,
+                      void* saved, size_t saved_bytes,
                       void* ws, size_t ws_bytes, void* stream) {
     if (int rc = check_problem(p, true)) return rc;
     if (p->N == 0) return LA_OK;
     LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(O);
     LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(S_out); LA_OPTIONAL_PTR(Z_out);
+    LA_OPTIONAL_PTR(saved);
     if (int rc = check_ws(p, LA_OP_CAUSAL_FORWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_saved(p, saved, saved_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_CAUSAL_FORWARD)) return tc_causal_forward(*p, Q, K, V, O, den, S_out, Z_out, ws, st);
+    if (tc_supported(*p, LA_OP_CAUSAL_FORWARD)) return tc_causal_forward(*p, Q, K, V, O, den, S_out, Z_out, saved, ws, st);
     return general_causal_forward(*p, Q, K, V, O, den, S_out, Z_out, st);
 }
 
 int la_causal_backward(const la_problem* p, const void* Q, const void* K, const void* V,
                        const void* O, const float* den, const void* G,
+                       const void* saved, size_t saved_bytes,
                        void* dQ, void* dK, void* dV,
                        void* ws, size_t ws_bytes, void* stream) {
     if (int rc = check_problem(p, true)) return rc;
     if (p->N == 0) return LA_OK;
     LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(G);
     LA_REQUIRE_PTR(dQ); LA_REQUIRE_PTR(dK); LA_REQUIRE_PTR(dV);
-    LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den);
+    LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(saved);
     if (int rc = check_ws(p, LA_OP_CAUSAL_BACKWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_saved(p, saved, saved_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_CAUSAL_BACKWARD)) return tc_causal_backward(*p, Q, K, V, O, den, G, dQ, dK, dV, ws, st);
+    if (tc_supported(*p, LA_OP_CAUSAL_BACKWARD))
+        return tc_causal_backward(*p, Q, K, V, O, den, G, saved, dQ, dK, dV, ws, st);
     return general_causal_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
 }
 

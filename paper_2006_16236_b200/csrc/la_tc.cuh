@@ -8,10 +8,12 @@ namespace la {
 bool tc_supported(const la_problem& p, int op);
 size_t tc_workspace_bytes(const la_problem& p, int op);
 
+size_t tc_causal_saved_bytes(const la_problem& p);
 int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
-                      float* den, float* S_out, float* Z_out, void* ws, cudaStream_t st);
+                      float* den, float* S_out, float* Z_out, void* saved, void* ws, cudaStream_t st);
 int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* O,
-                       const float* den, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+                       const float* den, const void* G, const void* saved, void* dQ, void* dK, void* dV, void* ws,
+                       cudaStream_t st);
 int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
                       float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
 int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
@@ -19,11 +21,12 @@ int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const 
 
 namespace tc {
 size_t causal_forward_workspace(const la_problem& p);
+size_t causal_saved_bytes(const la_problem& p);
 int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
-                   float* S_out, float* Z_out, void* ws, cudaStream_t st);
+                   float* S_out, float* Z_out, void* saved, void* ws, cudaStream_t st);
 size_t causal_backward_workspace(const la_problem& p);
 int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
-                    void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+                    const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 size_t linear_forward_workspace(const la_problem& p);
 size_t linear_backward_workspace(const la_problem& p);
 int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,

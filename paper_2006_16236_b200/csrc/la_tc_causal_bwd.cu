@@ -95,6 +95,7 @@ struct DqParams {
     float eps;
     int phi;
     int dim;                    // D = M: 64, or 32 (tiles zero-padded to 64 columns)
+    int map;                    // apply the feature map on load (0: the inputs are already phi(Q), phi(K))
 };
 
 __global__ void __launch_bounds__(kDqThreads, 1)
@@ -247,7 +248,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             const int s = c % kDqStages;
             if (!mbar_wait(&bars->full[s], (c / kDqStages) & 1, prm.status, kStatusTmaTimeout)) return false;
             if (t == 0) LA_TRACE(g_trace_dq, c, 5);
-            if (prm.phi == LA_PHI_ELU1) {
+            if (prm.map) {
                 uint8_t* rowK = smem + kDqOffStage + s * 4 * kTileBytes + t * 128;
                 phi_row_inplace(rowK, r7, prm.dim >> 3);
                 phi_row_inplace(rowK + 3 * kTileBytes, r7, prm.dim >> 3);
@@ -458,6 +459,7 @@ struct KvParams {
     float eps;
     int phi;
     int dim;
+    int map;                    // apply the feature map on load (0: the inputs are already phi(Q), phi(K))
 };
 
 __global__ void __launch_bounds__(kKvThreads, 1)
@@ -588,7 +590,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         // ---------------------- prep warps: qh = phi(Q) / dn, phi(K), dl column
         const int t = tid - 12 * 32;
         const uint32_t r7 = t & 7;
-        const bool elu = prm.phi == LA_PHI_ELU1;
+        const bool elu = prm.map != 0;
         #pragma unroll 1
         for (int i = 0; i < L; ++i) {
             const int s = i % kKvStages;
@@ -753,8 +755,18 @@ size_t causal_backward_workspace(const la_problem& p) {
 }
 
 int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
-                    void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+                    const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
     const Segmentation sg = choose_segments(p);
+    // With what the forward saved, phi(Q) and phi(K) are read as tensors (no feature map on load)
+    // and the forward pre-pass records are the forward's own.
+    const SavedLayout sl = saved_layout(p, sg);
+    const uint8_t* sv = (const uint8_t*)saved;
+    const bool premapped = sv != nullptr && p.phi == LA_PHI_ELU1;
+    const bool map = !premapped && p.phi == LA_PHI_ELU1;
+    if (premapped) {
+        Q = sv + sl.phiq;
+        K = sv + sl.phik;
+    }
     const int chunks = (int)(p.N / kChunk);
     const size_t bh = (size_t)(p.B * p.H);
     const uint64_t rows = (uint64_t)(bh * p.N);
@@ -783,7 +795,8 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     const unsigned grid = (unsigned)(sg.nseg * bh);
 
     // forward sweep: dQ, and dn_i, dl_i for the reverse sweep
-    if (int rc = segment_states(p, sg, mK, mV, nullptr, nullptr, rec_s, /*reverse=*/false, st)) return rc;
+    if (sv) rec_s = (float*)(sv + sl.records);
+    else if (int rc = segment_states(p, sg, mK, mV, nullptr, nullptr, rec_s, /*reverse=*/false, map, st)) return rc;
     DqParams a;
     a.dn = dn;
     a.dl = dl;
@@ -798,13 +811,14 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.eps = p.eps;
     a.phi = p.phi;
     a.dim = (int)p.D;
+    a.map = map ? 1 : 0;
     prof_begin(kProfCausalBwdDq, st);
     causal_bwd_dq_kernel<<<grid, kDqThreads, kDqSmemBytes, st>>>(mK, mV, mG, mQ, a);
     LA_LAUNCHED();
     prof_end(kProfCausalBwdDq, st);
 
     // reverse sweep: dK, dV
-    if (int rc = segment_states(p, sg, mQ, mG, dn, dl, rec_r, /*reverse=*/true, st)) return rc;
+    if (int rc = segment_states(p, sg, mQ, mG, dn, dl, rec_r, /*reverse=*/true, map, st)) return rc;
     KvParams b;
     b.dn = dn;
     b.dl = dl;
@@ -820,6 +834,7 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     b.eps = p.eps;
     b.phi = p.phi;
     b.dim = (int)p.D;
+    b.map = map ? 1 : 0;
     prof_begin(kProfCausalBwdDkv, st);
     causal_bwd_dkv_kernel<<<grid, kKvThreads, kKvSmemBytes, st>>>(mQ, mK, mV, mG, b);
     LA_LAUNCHED();

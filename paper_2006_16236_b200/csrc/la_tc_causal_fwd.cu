@@ -77,6 +77,7 @@ struct FwdParams {
     float eps;
     int phi;
     int dim;               // D = M: 64, or 32 (tiles zero-padded to 64 columns)
+    int save;              // store the mapped phi(Q), phi(K) tiles for the backward pass
 };
 
 // ---------------------------------------------------------------------------
@@ -84,7 +85,8 @@ struct FwdParams {
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads, 1)
 causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-                  const __grid_constant__ CUtensorMap mapV, const FwdParams prm) {
+                  const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapPQ,
+                  const __grid_constant__ CUtensorMap mapPK, const FwdParams prm) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     Barriers* bars = reinterpret_cast<Barriers*>(smem + kOffBar);
@@ -108,7 +110,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], 1);
+            mbar_init(&bars->empty[s], prm.save ? 3 : 1);      // MMA commit (+ the two threads that store mapped tiles)
             mbar_init(&bars->mapped[s], 256);
         }
         for (int b = 0; b < 2; ++b) {
@@ -256,11 +258,27 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             const int s = c % kStages;
             if (!mbar_wait(&bars->full[s], (c / kStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
+            uint8_t* tile = smem + kOffStage + s * kStageBytes;
             if (prm.phi == LA_PHI_ELU1) {
-                phi_row_inplace(smem + kOffStage + s * kStageBytes + t * 128, r7, prm.dim >> 3);
+                phi_row_inplace(tile + t * 128, r7, prm.dim >> 3);
                 fence_proxy_async_smem();
             }
+            if (prm.save) {         // the whole mapped tile goes out with one bulk store
+                named_barrier(3, 128);
+                if (t == 0) {
+                    if (c > 0) {    // the previous chunk's store has long read its tile: release that stage
+                        tma_store_wait_read<0>();
+                        mbar_arrive(&bars->empty[(c - 1) % kStages]);
+                    }
+                    tma_store_2d(&mapPQ, tile, 0, (int)(row0 + (int64_t)c * kChunk));
+                    tma_store_commit();
+                }
+            }
             mbar_arrive(&bars->mapped[s]);
+        }
+        if (prm.save && t == 0) {
+            tma_store_wait_all<0>();
+            mbar_arrive(&bars->empty[(L - 1) % kStages]);
         }
     } else if (warp >= 8) {
         // ---------------- operand warps: phi(K) in place (two chunks ahead), then the state conversion
@@ -277,9 +295,21 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             const int s = c % kStages;
             if (!mbar_wait(&bars->full[s], (c / kStages) & 1, prm.status, kStatusTmaTimeout)) return false;
             if (t == 0) LA_TRACE(g_trace_fwd, c, 5);
+            uint8_t* tile = smem + kOffStage + s * kStageBytes + kTileBytes;
             if (prm.phi == LA_PHI_ELU1) {
-                phi_row_inplace(smem + kOffStage + s * kStageBytes + kTileBytes + t * 128, r7, prm.dim >> 3);
+                phi_row_inplace(tile + t * 128, r7, prm.dim >> 3);
                 fence_proxy_async_smem();
+            }
+            if (prm.save) {
+                named_barrier(4, 128);
+                if (t == 0) {
+                    if (c > 0) {
+                        tma_store_wait_read<0>();
+                        mbar_arrive(&bars->empty[(c - 1) % kStages]);
+                    }
+                    tma_store_2d(&mapPK, tile, 0, (int)(row0 + (int64_t)c * kChunk));
+                    tma_store_commit();
+                }
             }
             mbar_arrive(&bars->mapped[s]);
             if (t == 0) LA_TRACE(g_trace_fwd, c, 6);
@@ -304,6 +334,10 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 if (t == 0) LA_TRACE(g_trace_fwd, c, 8);
             }
             if (i < L) ok = map_chunk(i);
+        }
+        if (prm.save && t == 0) {
+            tma_store_wait_all<0>();
+            if (ok) mbar_arrive(&bars->empty[(L - 1) % kStages]);
         }
         if (!ok) *abort_flag = 1;
     } else {
@@ -420,15 +454,22 @@ size_t causal_forward_workspace(const la_problem& p) {
     return (size_t)(p.B * p.H) * sg.parts() * kStateFloats * sizeof(float);
 }
 
+size_t causal_saved_bytes(const la_problem& p) { return saved_layout(p, choose_segments(p)).bytes; }
+
 int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
-                   float* S_out, float* Z_out, void* ws, cudaStream_t st) {
+                   float* S_out, float* Z_out, void* saved, void* ws, cudaStream_t st) {
     const Segmentation sg = choose_segments(p);
     const int chunks = (int)(p.N / kChunk);
     const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
-    CUtensorMap mQ, mK, mV;
+    const SavedLayout sl = saved_layout(p, sg);
+    uint8_t* sv = (uint8_t*)saved;
+    const bool save = sv != nullptr && p.phi == LA_PHI_ELU1;     // with identity features Q, K are the mapped tensors
+    CUtensorMap mQ, mK, mV, mPQ, mPK;
     if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
     if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
     if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mPQ, save ? sv + sl.phiq : Q, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mPK, save ? sv + sl.phik : K, rows, kChunk, (int)p.D)) return rc;
     int* status = device_status_ptr();
     if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
 
@@ -437,9 +478,10 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
         LA_CUDA_TRY(cudaFuncSetAttribute(causal_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
         attr_done = true;
     }
-    float* records = (float*)ws;
+    // the pre-pass records go straight into the saved buffer when there is one
+    float* records = sv ? (float*)(sv + sl.records) : (float*)ws;
     if (sg.nseg > 1) {
-        if (int rc = segment_states(p, sg, mK, mV, nullptr, nullptr, records, /*reverse=*/false, st)) return rc;
+        if (int rc = segment_states(p, sg, mK, mV, nullptr, nullptr, records, /*reverse=*/false, p.phi == LA_PHI_ELU1, st)) return rc;
     }
     FwdParams prm;
     prm.O = (__nv_bfloat16*)O;
@@ -456,8 +498,9 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     prm.eps = p.eps;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
+    prm.save = save ? 1 : 0;
     prof_begin(kProfCausalFwd, st);
-    causal_fwd_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kThreads, kSmemBytes, st>>>(mQ, mK, mV, prm);
+    causal_fwd_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kThreads, kSmemBytes, st>>>(mQ, mK, mV, mPQ, mPK, prm);
     LA_LAUNCHED();
     prof_end(kProfCausalFwd, st);
     return LA_OK;

@@ -41,7 +41,26 @@ Segmentation choose_segments(const la_problem& p);
 
 // Per-segment sums of phi(X)^T [Y | a] into `records` followed by their exclusive scan
 int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
-                   const float* dn, const float* dl, float* records, bool reverse, cudaStream_t st);
+                   const float* dn, const float* dl, float* records, bool reverse, bool map, cudaStream_t st);
+
+// What the causal forward leaves for the causal backward when the caller passes a `saved`
+// buffer: the mapped phi(Q) and phi(K) ([B*H*N, D] bf16 each, exactly the operands the
+// forward's tensor-core products consumed) and the forward pre-pass records.  The backward
+// then reads the mapped tensors in place of Q and K, evaluates no exponential and skips its
+// own forward pre-pass; its results are the same bit for bit.
+struct SavedLayout {
+    size_t phiq, phik, records, bytes;      // byte offsets of the three parts; total size
+};
+inline SavedLayout saved_layout(const la_problem& p, const Segmentation& sg) {
+    const size_t rows = (size_t)(p.B * p.H * p.N);
+    const size_t tensor = (rows * (size_t)p.D * 2 + 1023) & ~(size_t)1023;
+    SavedLayout l;
+    l.phiq = 0;
+    l.phik = tensor;
+    l.records = 2 * tensor;
+    l.bytes = l.records + (sg.nseg > 1 ? (size_t)(p.B * p.H) * sg.parts() * kStateFloats * sizeof(float) : 0);
+    return l;
+}
 
 // 2-D view of a [rows][cols] bf16 tensor (cols = 32 or 64) with a [box_rows][64] box and the
 // 128-byte swizzle.  With cols = 32 the upper half of every 128-byte tile row is out of bounds:

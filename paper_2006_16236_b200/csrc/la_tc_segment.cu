@@ -40,7 +40,7 @@ struct SumParams {
     int first_part;        // parts first_part .. first_part + parts_per_seq - 1 are summed
     int parts_per_seq;
     float eps;
-    int phi;
+    int map;               // apply the feature map to X on load
     int dim;
 };
 
@@ -139,7 +139,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             if (!mbar_wait(&bars->full[s], (c / kSumStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             uint8_t* rowX = smem + s * kSumStageBytes + t * 128;
-            if (prm.phi == LA_PHI_ELU1) {
+            if (prm.map) {
                 if (scaled) map_row_inplace<true>(rowX, r7, inv, prm.dim >> 3);
                 else phi_row_inplace(rowX, r7, prm.dim >> 3);
             }
@@ -182,7 +182,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
 }  // namespace
 
 int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
-                   const float* dn, const float* dl, float* records, bool reverse, cudaStream_t st) {
+                   const float* dn, const float* dl, float* records, bool reverse, bool map, cudaStream_t st) {
     if (sg.nseg <= 1) return LA_OK;
     static bool attr_done = false;
     if (!attr_done) {
@@ -202,7 +202,7 @@ int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMa
     prm.first_part = reverse ? sg.sub : 0;    // the open-end segment's own sums are never needed
     prm.parts_per_seq = (sg.nseg - 1) * sg.sub;
     prm.eps = p.eps;
-    prm.phi = p.phi;
+    prm.map = map ? 1 : 0;
     prm.dim = (int)p.D;
     prof_begin(kProfSegmentSum, st);
     segment_sum_kernel<<<(unsigned)(prm.parts_per_seq * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);

@@ -161,14 +161,18 @@ def _sample_heads(B, H, k=3):
 @pytest.mark.parametrize("name", ["causal_fp32_small", "causal_bf16_image", "causal_sweep_bf16_N4096",
                                   "causal_sweep_bf16_N8192", "causal_sweep_bf16_N16384",
                                   "causal_sweep_bf16_N32768", "causal_sweep_bf16_N65536"])
-def test_causal_workloads_full_size(name):
+@pytest.mark.parametrize("keep", [False, True], ids=["recompute", "saved"])
+def test_causal_workloads_full_size(name, keep):
     w = WORKLOADS[name]
     dtype = w.torch_dtype
     Q, K, V, G = draw_workload(w)
     Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
     den = torch.empty((w.B, w.H, w.N), device=DEV)
-    O = la.la_causal_forward(Qd, Kd, Vd, den=den)
-    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd, O=O, den=den)
+    saved = la.saved_buffer(Qd, Vd) if keep else None      # what a training step keeps for the backward pass
+    if keep and saved is None:
+        pytest.skip("this problem runs the general kernels, which keep nothing")
+    O = la.la_causal_forward(Qd, Kd, Vd, den=den, saved=saved)
+    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd, O=O, den=den, saved=saved)
     la.la_last_device_status()
     for b, h in _sample_heads(w.B, w.H):
         sl = (slice(b, b + 1), slice(h, h + 1))
@@ -201,6 +205,36 @@ def test_results_are_repeatable_bit_for_bit(name):
         else:
             for a, b, nm in zip(first, cur, ("O", "dQ", "dK", "dV")):
                 assert torch.equal(a, b), f"{name}: {nm} differs between repeats"
+
+
+@pytest.mark.parametrize("shape", [(2, 2, 1024, 64), (1, 3, 384, 32), (3, 50, 2048, 64)])
+def test_saved_buffer_matches_recomputation(shape):
+    """The forward's saved phi(Q), phi(K) are the bf16 feature maps of Q and K, the forward's own result
+    does not depend on saving them, dQ (whose operands are identical on both paths) is bit-identical, and
+    dK, dV agree to rounding."""
+    B, H, N, D = shape
+    Q, K, V, G = gpu(*draw_qkvg(B, H, N, D, D, 91, torch.bfloat16, 1.0))
+    saved = la.saved_buffer(Q, V)
+    assert saved is not None and saved.numel() >= 2 * Q.numel() * 2
+    saved.fill_(0xFF)
+    O1 = la.la_causal_forward(Q, K, V, saved=saved)
+    O0 = la.la_causal_forward(Q, K, V)
+    assert torch.equal(O0, O1)
+    rows = B * H * N
+    stride = (rows * D * 2 + 1023) // 1024 * 1024
+    phiq = saved[: rows * D * 2].view(torch.bfloat16).view(B, H, N, D)
+    phik = saved[stride: stride + rows * D * 2].view(torch.bfloat16).view(B, H, N, D)
+    for got, x in ((phiq, Q), (phik, K)):
+        ref = oracle.feature_map(x.double().cpu().numpy())
+        err = (got.double().cpu().numpy() - ref) / ref
+        assert abs(err).max() <= 2.0 ** -8, abs(err).max()
+    g0 = la.la_causal_backward(Q, K, V, G)
+    g1 = la.la_causal_backward(Q, K, V, G, saved=saved)
+    la.la_last_device_status()
+    assert torch.equal(g0[0], g1[0]), "dQ differs"
+    for a, b, nm in zip(g0[1:], g1[1:], "KV"):
+        ref = a.double().cpu().numpy()
+        assert_close(b, ref, torch.bfloat16, f"d{nm} saved vs recomputed", grad=True)
 
 
 def test_noncausal_workload_full_size():

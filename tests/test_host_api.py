@@ -63,7 +63,7 @@ def test_bad_arguments_are_rejected_on_the_host(L):
 
     def causal(p, Q=ok, K=ok, V=ok, O=ok, ws=null, ws_bytes=0):
         return L.la_causal_forward(ctypes.byref(p) if p is not None else None, Q, K, V, O, null, null, null,
-                                   ws, ws_bytes, null)
+                                   null, 0, ws, ws_bytes, null)
 
     assert causal(None) == -1
     assert causal(_p(B=0)) == -1
@@ -80,9 +80,20 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     p = _p()
     need = la.la_workspace_bytes(p, binding.LA_OP_CAUSAL_BACKWARD)
     assert need > 0
-    args = [ctypes.byref(p), ok, ok, ok, null, null, ok, ok, ok, ok]
+    args = [ctypes.byref(p), ok, ok, ok, null, null, ok, null, 0, ok, ok, ok]
     assert L.la_causal_backward(*args, null, 0, null) == -3
     assert L.la_causal_backward(*args, ok, need - 1, null) == -3
+    # the optional saved buffer: a short or misaligned one is refused; problems on the general kernels need none
+    pb = _p(dtype_code=binding.LA_BF16, N=256, D=64, M=64)
+    keep = la.la_workspace_bytes(pb, binding.LA_OP_CAUSAL_SAVED)
+    assert keep >= 2 * 256 * 64 * 2 * pb.B * pb.H
+    big = ctypes.c_void_p(1 << 20)                   # never dereferenced: validation fails first
+    args = [ctypes.byref(pb), big, big, big, null, null, big, big, keep - 1, big, big, big]
+    assert L.la_causal_backward(*args, big, 1 << 40, null) == -3
+    assert b"saved" in L.la_last_error()
+    args[7] = ctypes.c_void_p((1 << 20) + 16)
+    assert L.la_causal_backward(*args, big, 1 << 40, null) == -1
+    assert la.la_workspace_bytes(_p(), binding.LA_OP_CAUSAL_SAVED) == 0
     assert L.la_recurrent_step(ctypes.byref(p), ok, ok, ok, null, ok, ok, null) == -1
     assert L.la_feature_map(ok, ok, -5, 0, 0, null) == -1
     assert L.la_feature_map(ok, ok, 0, 0, 0, null) == 0
