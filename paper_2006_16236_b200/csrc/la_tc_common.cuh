@@ -272,34 +272,32 @@ __device__ __forceinline__ void state_row_store(uint8_t* s_tile, int d_row, int 
     }
 }
 
-// State accumulator -> registers (then `drained` is signalled: the accumulator may be updated
-// again) -> bf16 tiles; optionally the fp32 values to global memory.
+// State accumulator -> registers, `drained` is signalled at once (the accumulator may be updated
+// again: the update of the next chunk waits for exactly this), then the bf16 tiles are written;
+// optionally the fp32 values go to global memory.
 __device__ __forceinline__ void state_to_tiles(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, uint8_t* z_tile,
                                                uint64_t* drained, float* g_S, float* g_Z, int dim) {
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
-    uint32_t v[32];
-    sm100::tmem_ld32(tmem_state + lane_base, v);
-    sm100::tmem_ld_wait();
-    if (owner) {
-        state_row_store(s_tile, d_row, 0, v);
-        if (g_S && d_row < dim) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) g_S[d_row * dim + j] = __uint_as_float(v[j]);
-        }
-    }
-    sm100::tmem_ld32(tmem_state + lane_base + 32, v);
+    uint32_t v0[32], v1[32];
+    sm100::tmem_ld32(tmem_state + lane_base, v0);
+    sm100::tmem_ld32(tmem_state + lane_base + 32, v1);
     const float z = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 64));
     sm100::tmem_ld_wait();
     sm100::tc_fence_before_sync();
     if (drained) sm100::mbar_arrive(drained);
     if (owner) {
-        state_row_store(s_tile, d_row, 1, v);
+        state_row_store(s_tile, d_row, 0, v0);
+        state_row_store(s_tile, d_row, 1, v1);
         z_row_store(z_tile, d_row, z);
-        if (g_S && d_row < dim && dim > 32) {
+        if (g_S && d_row < dim) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) g_S[d_row * dim + 32 + j] = __uint_as_float(v[j]);
+            for (int j = 0; j < 32; ++j) g_S[d_row * dim + j] = __uint_as_float(v0[j]);
+            if (dim > 32) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) g_S[d_row * dim + 32 + j] = __uint_as_float(v1[j]);
+            }
         }
         if (g_Z && d_row < dim) g_Z[d_row] = z;
     }
