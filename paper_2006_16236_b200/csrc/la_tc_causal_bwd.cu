@@ -680,7 +680,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     stg128(dstK + h * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
                 }
             }
-#pragma unroll
+#pragma unroll 1
             for (int h = 0; h < 2; ++h) {
                 if (h * 32 >= prm.dim) break;
                 uint32_t v[32];
@@ -718,17 +718,19 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             tc_fence_after_sync();
             if (warp == 3 && lane == 0) LA_TRACE(g_trace_dkv, i, 11);
             const float delta = sDelta[s * 128 + t];
-            uint32_t v0[32], v1[32];
-            if (has0) tmem_ld32(tmem + lane_base + kKvColP + blk0 * 32, v0);
-            if (has1) tmem_ld32(tmem + lane_base + kKvColP + blk1 * 32, v1);
-            tmem_ld_wait();
-            if (has0) score_block_store(v0, rowP, r7, blk0, blk0 == quad, lane, 0.f);
-            if (has1) score_block_store(v1, rowP, r7, blk1, blk1 == quad, lane, 0.f);
-            if (has0) tmem_ld32(tmem + lane_base + kKvColDP + blk0 * 32, v0);
-            if (has1) tmem_ld32(tmem + lane_base + kKvColDP + blk1 * 32, v1);
-            tmem_ld_wait();
-            if (has0) score_block_store(v0, rowDP, r7, blk0, blk0 == quad, lane, delta);
-            if (has1) score_block_store(v1, rowDP, r7, blk1, blk1 == quad, lane, delta);
+            // the two score tiles (Ph, then dP + dl) go through the same rolled code
+#pragma unroll 1
+            for (int m = 0; m < 2; ++m) {
+                const uint32_t src = tmem + lane_base + (m ? kKvColDP : kKvColP);
+                uint8_t* dst = m ? rowDP : rowP;
+                const float add = m ? delta : 0.f;
+                uint32_t v0[32], v1[32];
+                if (has0) tmem_ld32(src + blk0 * 32, v0);
+                if (has1) tmem_ld32(src + blk1 * 32, v1);
+                tmem_ld_wait();
+                if (has0) score_block_store(v0, dst, r7, blk0, blk0 == quad, lane, add);
+                if (has1) score_block_store(v1, dst, r7, blk1, blk1 == quad, lane, add);
+            }
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->pd_ready);
