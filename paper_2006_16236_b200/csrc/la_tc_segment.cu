@@ -14,14 +14,20 @@ namespace tc {
 
 using namespace sm100;
 
+LA_TRACE_DECL(g_trace_seg)
+
 namespace {
 
 constexpr int kSumThreads = 192;
-constexpr int kSumStages = 2;
-constexpr uint32_t kSumStageBytes = 3 * kTileBytes;                  // X, Y, aux column tile
-constexpr uint32_t kSumOffOnes = kSumStages * kSumStageBytes;
-constexpr uint32_t kSumOffBar = kSumOffOnes + 1024;
-constexpr uint32_t kSumSmemBytes = kSumOffBar + 256 + 1024;
+// Three stages of {X, Y} and one shared column tile (the ones, or the dl column of the chunk in
+// flight): the loads have to run about two chunks ahead to cover the TMA latency, and two CTAs
+// share an SM (2 x (112.25 KB + 1 KB reserved) fits the 228 KB of an SM).
+constexpr int kSumStages = 3;
+constexpr uint32_t kSumStageBytes = 2 * kTileBytes;                  // X, Y
+constexpr uint32_t kSumOffAux = kSumStages * kSumStageBytes;         // [128][64] column tile: B operand block [64, 80)
+constexpr uint32_t kSumOffBar = kSumOffAux + kTileBytes;
+constexpr uint32_t kSumSmemBytes = kSumOffBar + 256;
+static_assert(2 * (kSumSmemBytes + 1024) <= 233472, "two CTAs per SM");
 
 struct SumBarriers {
     uint64_t full[kSumStages], empty[kSumStages], mapped[kSumStages];
@@ -47,11 +53,11 @@ struct SumParams {
 __global__ void __launch_bounds__(kSumThreads, 2)
 segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                    const SumParams prm) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     SumBarriers* bars = reinterpret_cast<SumBarriers*>(smem + kSumOffBar);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    LA_TRACE_CTA(g_trace_seg, 0);
     const int seg = prm.first_part + blockIdx.x % prm.parts_per_seq;       // index of this part
     const int64_t bh = blockIdx.x / prm.parts_per_seq;
     const int c_begin = seg * prm.chunks_per_part;
@@ -59,6 +65,10 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
     const bool scaled = prm.dn != nullptr;
 
+    if (sbase & 1023u) {            // the swizzled tiles need a 1 KB aligned base: report, touch nothing
+        if (tid == 0) atomicOr(prm.status, kStatusPipeTimeout);
+        return;
+    }
     if (tid == 0) {
         for (int s = 0; s < kSumStages; ++s) {
             mbar_init(&bars->full[s], 1);
@@ -74,8 +84,9 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
         tmem_alloc(&bars->tmem_base, 128);
         tmem_relinquish();
     }
-    if (tid < 128)
-        for (int i = tid; i < 256; i += 128) reinterpret_cast<uint32_t*>(smem + kSumOffOnes)[i] = 0x3F803F80u;
+    // the column tile: ones (a_i = 1) unless the mapping threads write dl there chunk by chunk
+    for (int i = tid; i < kTileBytes / 4; i += kSumThreads)
+        reinterpret_cast<uint32_t*>(smem + kSumOffAux)[i] = scaled ? 0u : 0x3F803F80u;
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
@@ -96,6 +107,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
                 if (*abort_flag) break;
                 uint8_t* st = smem + s * kSumStageBytes;
                 const int y = (int)(row0 + (int64_t)c * kChunk);
+                LA_TRACE(g_trace_seg, c, 2);
                 mbar_arrive_expect_tx(&bars->full[s], 2 * kTileBytes);
                 tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
                 tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
@@ -103,23 +115,24 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
         }
     } else if (warp == 5) {
         if (lane == 0) {
-            const uint32_t idesc_s = umma_idesc_bf16(64, 64, 1, 1);
-            const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
-            const uint32_t aOnes = sbase + kSumOffOnes;
+            // one M = 64, N = 80 product per K group: B = [Y | a], the second 64-column block being the
+            // column tile (same K group)
+            const uint32_t idesc = umma_idesc_bf16(64, 80, 1, 1);
+            const uint32_t aAux = sbase + kSumOffAux;
             bool ok = true;
             #pragma unroll 1
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kSumStages;
-                const uint32_t aX = sbase + s * kSumStageBytes, aY = aX + kTileBytes, aA = aY + kTileBytes;
+                const uint32_t aX = sbase + s * kSumStageBytes, aY = aX + kTileBytes;
                 ok = mbar_wait(&bars->mapped[s], (c / kSumStages) & 1, prm.status, kStatusPipeTimeout);
                 if (!ok || *abort_flag) { ok = false; break; }
                 tc_fence_after_sync();
+                LA_TRACE(g_trace_seg, c, 0);
+#pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    umma_bf16(tmem, desc_mn(aX + k * 2048), desc_mn(aY + k * 2048), idesc_s, (c | k) != 0);
-                for (int k = 0; k < 8; ++k)
-                    umma_bf16(tmem + 64, desc_mn(aX + k * 2048), scaled ? desc_mn(aA + k * 2048) : desc_ones(aOnes),
-                              idesc_z, (c | k) != 0);
+                    umma_bf16(tmem, desc_mn(aX + k * 2048), desc_mn(aY + k * 2048, aAux - aY), idesc, (c | k) != 0);
                 umma_commit(&bars->empty[s]);
+                LA_TRACE(g_trace_seg, c, 1);
             }
             if (!ok) *abort_flag = 1;
             umma_commit(&bars->done);
@@ -138,6 +151,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             }
             if (!mbar_wait(&bars->full[s], (c / kSumStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
+            if (t == 0) LA_TRACE(g_trace_seg, c, 5);
             uint8_t* rowX = smem + s * kSumStageBytes + t * 128;
             if (prm.map) {
                 if (scaled) map_row_inplace<true>(rowX, r7, inv, prm.dim >> 3);
@@ -145,14 +159,19 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             }
             else if (scaled) map_row_inplace<false>(rowX, r7, inv, prm.dim >> 3);
             if (scaled) {
-                uint8_t* rowA = rowX + 2 * kTileBytes;
-                const uint32_t dd = pack_bf16x2(delta, delta);      // columns 0..15 of the aux tile
+                // the single column tile is still an operand of the previous chunk's products
+                if (c >= 1 && !mbar_wait(&bars->empty[(c - 1) % kSumStages], ((c - 1) / kSumStages) & 1, prm.status,
+                                         kStatusMmaTimeout)) { *abort_flag = 1; break; }
+                uint8_t* rowA = smem + kSumOffAux + t * 128;
+                const uint32_t dd = pack_bf16x2(delta, delta);      // columns 0..15 of the column tile
                 sts128(rowA + ((0 ^ r7) << 4), dd, dd, dd, dd);
                 sts128(rowA + ((1 ^ r7) << 4), dd, dd, dd, dd);
             }
             fence_proxy_async_smem();
             mbar_arrive(&bars->mapped[s]);
+            if (t == 0) LA_TRACE(g_trace_seg, c, 6);
         }
+        if (t == 0) LA_TRACE(g_trace_seg, 100, 7);
         // read-out: the [S | Z]-shaped record of this (bh, seg)
         const bool ok = mbar_wait(&bars->done, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
         tc_fence_after_sync();
@@ -173,6 +192,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     }
     tc_fence_before_sync();
     __syncthreads();
+    LA_TRACE_CTA(g_trace_seg, 1);
     if (warp == 5) {
         __syncwarp();
         tmem_dealloc(tmem, 128);
@@ -213,3 +233,9 @@ int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMa
 
 }  // namespace tc
 }  // namespace la
+
+#ifdef LA_TC_TRACE
+extern "C" int la_debug_read_trace_seg(long long* out, int n) {
+    return (int)cudaMemcpyFromSymbol(out, la::tc::g_trace_seg, n * sizeof(long long));
+}
+#endif
