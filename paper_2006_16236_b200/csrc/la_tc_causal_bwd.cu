@@ -433,15 +433,16 @@ constexpr uint32_t kKvOffStage = 0;                                        // kK
 constexpr uint32_t kKvOffP = kKvOffStage + kKvStages * 4 * kTileBytes;     // 2 tiles
 constexpr uint32_t kKvOffDP = kKvOffP + 2 * kTileBytes;                    // 2 tiles
 constexpr uint32_t kKvOffAux = kKvOffDP + 2 * kTileBytes;                  // delta column tile
-constexpr uint32_t kKvOffR = kKvOffAux + kTileBytes;                       // bf16 R tile
-constexpr uint32_t kKvOffDelta = kKvOffR + kDim * 128;                     // fp32 [kKvStages][128]
+constexpr uint32_t kKvOffR = kKvOffAux + kTileBytes;                       // 2 bf16 R tiles (iteration i reads tile i & 1)
+constexpr uint32_t kKvOffDelta = kKvOffR + 2 * kDim * 128;                     // fp32 [kKvStages][128]
 constexpr uint32_t kKvOffRv = kKvOffDelta + kKvStages * 512;               // fp32 r[2][64]
 constexpr uint32_t kKvOffBar = kKvOffRv + 512;
 constexpr uint32_t kKvSmemBytes = kKvOffBar + 256 + 1024;
+static_assert(kKvSmemBytes <= 232448, "shared memory budget of one CTA");
 
 struct KvBarriers {
     uint64_t full[kKvStages], empty[kKvStages], mapped[kKvStages];
-    uint64_t pd_full, pd_ready, r_full, state_ready, dkv_full, dkv_drained, aux_free;
+    uint64_t p_full, dp_full, p_ready, dp_ready, r_full, state_ready, dkv_full, dk_drained, dv_drained, aux_free;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -488,12 +489,15 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             mbar_init(&bars->empty[s], 1 + 128);      // MMA commit + the epilogue warps (they read phi(K) rows)
             mbar_init(&bars->mapped[s], 128);
         }
-        mbar_init(&bars->pd_full, 1);
-        mbar_init(&bars->pd_ready, 256);
+        mbar_init(&bars->p_full, 1);
+        mbar_init(&bars->dp_full, 1);
+        mbar_init(&bars->p_ready, 256);
+        mbar_init(&bars->dp_ready, 256);
         mbar_init(&bars->r_full, 1);
         mbar_init(&bars->state_ready, 128);
         mbar_init(&bars->dkv_full, 1);
-        mbar_init(&bars->dkv_drained, 128);
+        mbar_init(&bars->dk_drained, 128);
+        mbar_init(&bars->dv_drained, 128);
         bars->abort_flag = 0;
         fence_mbar_init();
     }
@@ -538,50 +542,79 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
             const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
             const uint32_t idesc_mnmn = umma_idesc_bf16(128, 64, 1, 1);
-            const uint32_t idesc_s = umma_idesc_bf16(64, 64, 1, 1);
-            const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
-            const uint32_t aR = sbase + kKvOffR, aAux = sbase + kKvOffAux;
+            const uint32_t idesc_r = umma_idesc_bf16(64, 80, 1, 1);
+            const uint32_t aAux = sbase + kKvOffAux;
             const uint32_t aP = sbase + kKvOffP, aDP = sbase + kKvOffDP;
-            bool ok = true;
+            auto stage_q = [&](int i) { return sbase + kKvOffStage + (uint32_t)(i % kKvStages) * 4 * kTileBytes; };
+            // The two score tiles run as two interleaved pipelines, so that the score warps always have
+            // a tile to work on: Ph of chunk i+1 is issued as soon as the rounded Ph of chunk i has been
+            // consumed (gV += Ph^T G), while the score warps are busy with dP of chunk i, and likewise dP.
+            // A commit covers every earlier MMA of this thread, so p_full(i+1) / dp_full(i+1) also tell
+            // the score warps that the products reading the shared-memory copies of chunk i are done.
+            bool ok = mbar_wait(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !*abort_flag;
+            if (ok) {
+                tc_fence_after_sync();
+                const uint32_t aQ = stage_q(0), aK = aQ + kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
+                for (int k = 0; k < 4; ++k)      // Ph = qh k^T
+                    umma_bf16(tmem + kKvColP, desc_k(aQ + k * 32), desc_k(aK + k * 32), idesc_pp, k > 0);
+                umma_commit(&bars->p_full);
+                for (int k = 0; k < 4; ++k)      // dP = G V^T
+                    umma_bf16(tmem + kKvColDP, desc_k(aG + k * 32), desc_k(aV + k * 32), idesc_pp, k > 0);
+                umma_commit(&bars->dp_full);
+            }
             #pragma unroll 1
             for (int i = 0; i < L && ok; ++i) {
                 const int s = i % kKvStages;
-                const uint32_t aQ = sbase + kKvOffStage + s * 4 * kTileBytes, aK = aQ + kTileBytes, aV = aK + kTileBytes,
-                               aG = aV + kTileBytes;
-                ok = mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout);
+                const uint32_t aQ = stage_q(i), aK = aQ + kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
+                const uint32_t nQ = stage_q(i + 1), nK = nQ + kTileBytes, nV = nK + kTileBytes, nG = nV + kTileBytes;
+                LA_TRACE(g_trace_dkv, i, 0);
+                const uint32_t aR = sbase + kKvOffR + (i & 1) * kDim * 128;      // R_{c+1}: the state before this chunk
+                // gV = k R_{c+1}, once the epilogue of the previous chunk has taken its gV out of TMEM, and the
+                // state update right away: the operand warps wait for it before they reuse the dl column tile
+                ok = mbar_wait(&bars->state_ready, i & 1, prm.status, kStatusPipeTimeout);
+                if (ok && i >= 1) ok = mbar_wait(&bars->dv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
                 if (!ok || *abort_flag) { ok = false; break; }
                 tc_fence_after_sync();
-                LA_TRACE(g_trace_dkv, i, 0);
-                for (int k = 0; k < 4; ++k)      // Ph = qh k^T
-                    umma_bf16(tmem + kKvColP, desc_k(aQ + k * 32), desc_k(aK + k * 32), idesc_pp, k > 0);
-                for (int k = 0; k < 4; ++k)      // dP = G V^T
-                    umma_bf16(tmem + kKvColDP, desc_k(aG + k * 32), desc_k(aV + k * 32), idesc_pp, k > 0);
-                umma_commit(&bars->pd_full);
-                ok = mbar_wait(&bars->state_ready, i & 1, prm.status, kStatusPipeTimeout);
-                if (ok && i >= 1) ok = mbar_wait(&bars->dkv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok) break;
-                tc_fence_after_sync();
                 LA_TRACE(g_trace_dkv, i, 1);
-                for (int k = 0; k < 4; ++k)      // gk = V R_{c+1}^T
-                    umma_bf16(tmem + kKvColDk, desc_k(aV + k * 32), desc_k(aR + k * 32), idesc_kk, k > 0);
-                for (int k = 0; k < 4; ++k)      // gV = k R_{c+1}
+                for (int k = 0; k < 4; ++k)
                     umma_bf16(tmem + kKvColDv, desc_k(aK + k * 32), desc_mn(aR + k * 2048), idesc_kmn, k > 0);
-                for (int k = 0; k < 8; ++k)      // R += qh^T G
-                    umma_bf16(tmem + kKvColR, desc_mn(aQ + k * 2048), desc_mn(aG + k * 2048), idesc_s, 1);
-                for (int k = 0; k < 8; ++k)      // r += qh^T dl
-                    umma_bf16(tmem + kKvColR + 64, desc_mn(aQ + k * 2048), desc_mn(aAux + k * 2048), idesc_z, 1);
+                for (int k = 0; k < 8; ++k)      // [R | r] += qh^T [G | dl]: the dl column tile is the second 64-column block
+                    umma_bf16(tmem + kKvColR, desc_mn(aQ + k * 2048), desc_mn(aG + k * 2048, aAux - aG), idesc_r, 1);
                 umma_commit(&bars->r_full);
                 LA_TRACE(g_trace_dkv, i, 2);
-                ok = mbar_wait(&bars->pd_ready, i & 1, prm.status, kStatusPipeTimeout);
+                ok = mbar_wait(&bars->p_ready, i & 1, prm.status, kStatusPipeTimeout);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int k = 0; k < 8; ++k)      // gV += Ph^T G
+                    umma_bf16(tmem + kKvColDv, desc_mn(aP + k * 2048), desc_mn(aG + k * 2048), idesc_mnmn, 1);
+                if (i + 1 < L) {
+                    ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    for (int k = 0; k < 4; ++k)
+                        umma_bf16(tmem + kKvColP, desc_k(nQ + k * 32), desc_k(nK + k * 32), idesc_pp, k > 0);
+                    umma_commit(&bars->p_full);
+                }
+                // gk = V R_{c+1}^T, once the previous gk has been taken out (the other R tile is being rewritten
+                // meanwhile: this one stays valid until the next r_full)
+                if (i >= 1) ok = mbar_wait(&bars->dk_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int k = 0; k < 4; ++k)
+                    umma_bf16(tmem + kKvColDk, desc_k(aV + k * 32), desc_k(aR + k * 32), idesc_kk, k > 0);
+                ok = mbar_wait(&bars->dp_ready, i & 1, prm.status, kStatusPipeTimeout);
                 if (!ok) break;
                 tc_fence_after_sync();
                 LA_TRACE(g_trace_dkv, i, 3);
                 for (int k = 0; k < 8; ++k)      // gk += dP^T qh
                     umma_bf16(tmem + kKvColDk, desc_mn(aDP + k * 2048), desc_mn(aQ + k * 2048), idesc_mnmn, 1);
-                for (int k = 0; k < 8; ++k)      // gV += Ph^T G
-                    umma_bf16(tmem + kKvColDv, desc_mn(aP + k * 2048), desc_mn(aG + k * 2048), idesc_mnmn, 1);
                 umma_commit(&bars->dkv_full);
                 umma_commit(&bars->empty[s]);
+                if (i + 1 < L) {
+                    for (int k = 0; k < 4; ++k)
+                        umma_bf16(tmem + kKvColDP, desc_k(nG + k * 32), desc_k(nV + k * 32), idesc_pp, k > 0);
+                    umma_commit(&bars->dp_full);
+                }
                 LA_TRACE(g_trace_dkv, i, 4);
             }
             if (!ok) *abort_flag = 1;
@@ -644,7 +677,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             if (!mbar_wait(&bars->r_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
             if (t == 0) LA_TRACE(g_trace_dkv, i, 7);
-            state_to_smem(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + (i & 1) * 64, nullptr, nullptr);
+            state_to_smem(tmem + kKvColR, quad, lane, smem + kKvOffR + ((i + 1) & 1) * kDim * 128, sRv + (i & 1) * 64, nullptr, nullptr);
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->state_ready);
@@ -656,46 +689,55 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             const float* rprev = sRv + ((i + 1) & 1) * 64;               // r_{c+1}
             __nv_bfloat16* dstK = prm.dK + row * prm.dim;
             __nv_bfloat16* dstV = prm.dV + row * prm.dim;
+            // gV first (plain rounding), so that the next chunk's k R can start early; then gk
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                if (h * 32 >= prm.dim) break;             // columns beyond a 32-wide problem are padding
-                uint32_t v[32];
-                tmem_ld32(tmem + lane_base + kKvColDk + h * 32, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    uint32_t outp[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int d = h * 32 + cc * 8 + 2 * j;
-                        float g0 = __uint_as_float(v[cc * 8 + 2 * j]) + rprev[d];
-                        float g1 = __uint_as_float(v[cc * 8 + 2 * j + 1]) + rprev[d + 1];
-                        if (prm.phi == LA_PHI_ELU1) {
-                            const float k0 = bf16_lo(kf[h * 4 + cc][j]), k1 = bf16_hi(kf[h * 4 + cc][j]);
-                            g0 *= k0 > 1.f ? 1.f : k0;          // phi'(x) from phi(x): 1 where x > 0, else phi(x)
-                            g1 *= k1 > 1.f ? 1.f : k1;
-                        }
-                        outp[j] = pack_bf16x2(g0, g1);
-                    }
-                    stg128(dstK + h * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
-                }
-            }
-#pragma unroll 1
-            for (int h = 0; h < 2; ++h) {
-                if (h * 32 >= prm.dim) break;
                 uint32_t v[32];
                 tmem_ld32(tmem + lane_base + kKvColDv + h * 32, v);
                 tmem_ld_wait();
+                if (h == 1) {
+                    tc_fence_before_sync();
+                    mbar_arrive(&bars->dv_drained);
+                }
+                if (h * 32 < prm.dim) {                   // columns beyond a 32-wide problem are padding
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
-                    stg128(dstV + h * 32 + cc * 8,
-                           pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
-                           pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
-                           pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
-                           pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
+                    for (int cc = 0; cc < 4; ++cc)
+                        stg128(dstV + h * 32 + cc * 8,
+                               pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
+                               pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
+                               pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
+                               pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
+                }
             }
-            tc_fence_before_sync();
-            mbar_arrive(&bars->dkv_drained);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_base + kKvColDk + h * 32, v);
+                tmem_ld_wait();
+                if (h == 1) {
+                    tc_fence_before_sync();
+                    mbar_arrive(&bars->dk_drained);
+                }
+                if (h * 32 < prm.dim) {
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint32_t outp[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int d = h * 32 + cc * 8 + 2 * j;
+                            float g0 = __uint_as_float(v[cc * 8 + 2 * j]) + rprev[d];
+                            float g1 = __uint_as_float(v[cc * 8 + 2 * j + 1]) + rprev[d + 1];
+                            if (prm.phi == LA_PHI_ELU1) {
+                                const float k0 = bf16_lo(kf[h * 4 + cc][j]), k1 = bf16_hi(kf[h * 4 + cc][j]);
+                                g0 *= k0 > 1.f ? 1.f : k0;          // phi'(x) from phi(x): 1 where x > 0, else phi(x)
+                                g1 *= k1 > 1.f ? 1.f : k1;
+                            }
+                            outp[j] = pack_bf16x2(g0, g1);
+                        }
+                        stg128(dstK + h * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
+                    }
+                }
+            }
             if (t == 0) LA_TRACE(g_trace_dkv, i, 10);
             named_barrier(1, 128);          // r double buffer
         }
@@ -712,15 +754,17 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         #pragma unroll 1
         for (int i = 0; i < L; ++i) {
             const int s = i % kKvStages;
-            if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout) ||
-                !mbar_wait(&bars->pd_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
-            tc_fence_after_sync();
-            if (warp == 3 && lane == 0) LA_TRACE(g_trace_dkv, i, 11);
             const float delta = sDelta[s * 128 + t];
-            // the two score tiles (Ph, then dP + dl) go through the same rolled code
+            bool ok = true;
+            // the two score tiles (Ph, then dP + dl) go through the same rolled code, each with its own hand-off
 #pragma unroll 1
-            for (int m = 0; m < 2; ++m) {
+            for (int m = 0; m < 2 && ok; ++m) {
+                ok = mbar_wait(m ? &bars->dp_full : &bars->p_full, i & 1, prm.status, kStatusMmaTimeout);
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (warp == 3 && lane == 0 && m == 0) LA_TRACE(g_trace_dkv, i, 11);
                 const uint32_t src = tmem + lane_base + (m ? kKvColDP : kKvColP);
                 uint8_t* dst = m ? rowDP : rowP;
                 const float add = m ? delta : 0.f;
@@ -730,10 +774,11 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 tmem_ld_wait();
                 if (has0) score_block_store(v0, dst, r7, blk0, blk0 == quad, lane, add);
                 if (has1) score_block_store(v1, dst, r7, blk1, blk1 == quad, lane, add);
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                mbar_arrive(m ? &bars->dp_ready : &bars->p_ready);
             }
-            fence_proxy_async_smem();
-            tc_fence_before_sync();
-            mbar_arrive(&bars->pd_ready);
+            if (!ok) { *abort_flag = 1; break; }
             if (warp == 3 && lane == 0) LA_TRACE(g_trace_dkv, i, 12);
         }
     }
