@@ -421,28 +421,54 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
 // Warps 0-7: P and dP post-processing, 8-11: state conversion and dK/dV
 // epilogue, 12-15: qh = phi(Q) / dn, phi(K), dl column, 16: TMA, 17: MMA.
 // ===========================================================================
-constexpr int kKvStages = 2;
-constexpr int kKvThreads = 576;
-constexpr uint32_t kKvColP = 0;        // 128
-constexpr uint32_t kKvColDP = 128;     // 128
+// One transposed score tile (rows = keys, columns = queries; fp32 in TMEM at `pb`, this thread's
+// lane): wait for it, mask (keep query >= key), round to bf16 pairs in place, signal `ready`.
+// Deliberately not inlined: the two tiles of a chunk share one copy of this code, whose shape
+// then does not depend on what the compiler makes of the surrounding role loops.
+__device__ __noinline__ bool kv_round_tile(uint32_t pb, uint64_t* full, uint64_t* ready, uint32_t parity, int quad,
+                                           int half, int lane, int* status) {
+    if (!mbar_wait(full, parity, status, kStatusMmaTimeout)) return false;
+    tc_fence_after_sync();
+    const int blkA = 2 * half, blkB = 2 * half + 1;     // blocks left of the diagonal block `quad` are zeros
+    const bool hasA = blkA >= quad, hasB = blkB >= quad;
+    uint32_t v[32], pk[16];
+    if (hasA) tmem_ld32(pb + blkA * 32, v);
+    tmem_ld_wait();
+    score_block_pack_t(v, hasA, blkA == quad, lane, pk);
+    if (hasB) tmem_ld32(pb + blkB * 32, v);
+    // bf16 block j of this warp goes to columns 64 half + 16 j .. + 15: inside the fp32 columns
+    // of block 2 half, which this thread has read, so nothing another thread still needs is lost
+    tmem_st16(pb + half * 64, pk);
+    tmem_ld_wait();
+    score_block_pack_t(v, hasB, blkB == quad, lane, pk);
+    tmem_st16(pb + half * 64 + 16, pk);
+    tmem_st_wait();
+    tc_fence_before_sync();
+    mbar_arrive(ready);
+    return true;
+}
+
+constexpr int kKvStages = 3;
+constexpr int kKvThreads = 608;
+constexpr uint32_t kKvColP = 0;        // 128: Ph^T (fp32, then bf16 pairs in place)
+constexpr uint32_t kKvColDP = 128;     // 128: dP^T
 constexpr uint32_t kKvColDk = 256;     // 64
 constexpr uint32_t kKvColDv = 320;     // 64
 constexpr uint32_t kKvColR = 384;      // 64 + 16
 
-constexpr uint32_t kKvOffStage = 0;                                        // kKvStages x {Q, K, V, G}
-constexpr uint32_t kKvOffP = kKvOffStage + kKvStages * 4 * kTileBytes;     // 2 tiles
-constexpr uint32_t kKvOffDP = kKvOffP + 2 * kTileBytes;                    // 2 tiles
-constexpr uint32_t kKvOffAux = kKvOffDP + 2 * kTileBytes;                  // delta column tile
+constexpr uint32_t kKvStageBytes = 4 * kTileBytes;                         // {Q, K, V, G}
+constexpr uint32_t kKvOffStage = 0;
+constexpr uint32_t kKvOffAux = kKvOffStage + kKvStages * kKvStageBytes;    // dl column tile: (hi, lo) in columns 0, 1
 constexpr uint32_t kKvOffR = kKvOffAux + kTileBytes;                       // 2 bf16 R tiles (iteration i reads tile i & 1)
-constexpr uint32_t kKvOffDelta = kKvOffR + 2 * kDim * 128;                     // fp32 [kKvStages][128]
-constexpr uint32_t kKvOffRv = kKvOffDelta + kKvStages * 512;               // fp32 r[2][64]
+constexpr uint32_t kKvOffOnes = kKvOffR + 2 * kDim * 128;                  // 1 KB group: ones in columns 0, 1 (A operand)
+constexpr uint32_t kKvOffRv = kKvOffOnes + 1024;                           // fp32 r[2][64]
 constexpr uint32_t kKvOffBar = kKvOffRv + 512;
-constexpr uint32_t kKvSmemBytes = kKvOffBar + 256 + 1024;
+constexpr uint32_t kKvSmemBytes = kKvOffBar + 256;
 static_assert(kKvSmemBytes <= 232448, "shared memory budget of one CTA");
 
 struct KvBarriers {
     uint64_t full[kKvStages], empty[kKvStages], mapped[kKvStages];
-    uint64_t p_full, dp_full, p_ready, dp_ready, r_full, state_ready, dkv_full, dk_drained, dv_drained, aux_free;
+    uint64_t p_full, dp_full, p_ready, dp_ready, r_full, state_ready, dkv_full, dk_drained, dv_drained, kr_full, vr_full;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -467,11 +493,9 @@ __global__ void __launch_bounds__(kKvThreads, 1)
 causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                       const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapG,
                       const KvParams prm) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     KvBarriers* bars = reinterpret_cast<KvBarriers*>(smem + kKvOffBar);
-    float* sDelta = reinterpret_cast<float*>(smem + kKvOffDelta);
     float* sRv = reinterpret_cast<float*>(smem + kKvOffRv);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -483,6 +507,11 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
     // iteration i visits chunk c_end - 1 - i
     auto chunk_row = [&](int i) { return bh * prm.N + (int64_t)(c_end - 1 - i) * kChunk; };
 
+    LA_TRACE_CTA(g_trace_dkv, 0);
+    if (sbase & 1023u) {            // the swizzled tiles need a 1 KB aligned base: report, touch nothing
+        if (tid == 0) atomicOr(prm.status, kStatusPipeTimeout);
+        return;
+    }
     if (tid == 0) {
         for (int s = 0; s < kKvStages; ++s) {
             mbar_init(&bars->full[s], 1);
@@ -498,6 +527,8 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         mbar_init(&bars->dkv_full, 1);
         mbar_init(&bars->dk_drained, 128);
         mbar_init(&bars->dv_drained, 128);
+        mbar_init(&bars->kr_full, 1);
+        mbar_init(&bars->vr_full, 1);
         bars->abort_flag = 0;
         fence_mbar_init();
     }
@@ -506,7 +537,14 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         tmem_alloc(&bars->tmem_base, 512);
         tmem_relinquish();
     }
-    for (uint32_t i = tid; i < 4 * kTileBytes / 16; i += kKvThreads) sts128(smem + kKvOffP + i * 16, 0u, 0u, 0u, 0u);
+    // the dl column tile keeps zeros outside its first two columns; the ones group (8 rows, re-read for
+    // every row group through a zero stride) has ones in columns 0 and 1: together they add dl_i to dP_ij
+    for (uint32_t i = tid; i < kTileBytes / 16; i += kKvThreads) sts128(smem + kKvOffAux + i * 16, 0u, 0u, 0u, 0u);
+    if (tid < 64) {
+        const uint32_t row = tid >> 3, chunk = tid & 7;
+        const uint32_t w0 = chunk == 0 ? 0x3F803F80u : 0u;
+        sts128(smem + kKvOffOnes + row * 128 + ((chunk ^ row) << 4), w0, 0u, 0u, 0u);
+    }
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
@@ -526,96 +564,133 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     break;
                 }
                 if (*abort_flag) break;
-                uint8_t* st = smem + kKvOffStage + s * 4 * kTileBytes;
+                uint8_t* st = smem + kKvOffStage + s * kKvStageBytes;
                 const int y = (int)chunk_row(i);
-                mbar_arrive_expect_tx(&bars->full[s], 4 * kTileBytes);
+                mbar_arrive_expect_tx(&bars->full[s], kKvStageBytes);
                 tma_load_2d(st, &mapQ, 0, y, &bars->full[s]);
                 tma_load_2d(st + kTileBytes, &mapK, 0, y, &bars->full[s]);
                 tma_load_2d(st + 2 * kTileBytes, &mapV, 0, y, &bars->full[s]);
                 tma_load_2d(st + 3 * kTileBytes, &mapG, 0, y, &bars->full[s]);
             }
         }
-    } else if (warp == 17) {
-        // ------------------------------------------------------------- MMA issuer
+    } else if (warp >= 17) {
+        // ------------------------------------------------------------- MMA issuers
+        // Two threads share the issue work (an issuing thread needs about 100 cycles per tcgen05.mma here,
+        // more than the tensor pipe does).  Warp 17: the score tiles and the products that consume them
+        // (transposed tiles, rows = keys: Ph^T = k qh^T, dP^T = [V | 1] [G | dl]^T whose fifth K step is
+        // (ones in two columns) x (dl_i split into a bf16 high and low part); gV += Ph^T G, gk += dP^T qh with
+        // the rounded tiles read from TMEM).  Warp 18: everything that involves the running state
+        // ([R | r] += qh^T [G | dl]; gV = k R, gk = V R^T, which start the two accumulators).  MMAs of one
+        // thread execute in order; kr_full / vr_full order the two threads' writes to one accumulator.
         if (lane == 0) {
             const uint32_t idesc_pp = umma_idesc_bf16(128, 128, 0, 0);
             const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
-            const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
-            const uint32_t idesc_mnmn = umma_idesc_bf16(128, 64, 1, 1);
+            const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);     // also: A from TMEM, B MN-major
             const uint32_t idesc_r = umma_idesc_bf16(64, 80, 1, 1);
-            const uint32_t aAux = sbase + kKvOffAux;
-            const uint32_t aP = sbase + kKvOffP, aDP = sbase + kKvOffDP;
-            auto stage_q = [&](int i) { return sbase + kKvOffStage + (uint32_t)(i % kKvStages) * 4 * kTileBytes; };
-            // The two score tiles run as two interleaved pipelines, so that the score warps always have
-            // a tile to work on: Ph of chunk i+1 is issued as soon as the rounded Ph of chunk i has been
-            // consumed (gV += Ph^T G), while the score warps are busy with dP of chunk i, and likewise dP.
-            // A commit covers every earlier MMA of this thread, so p_full(i+1) / dp_full(i+1) also tell
-            // the score warps that the products reading the shared-memory copies of chunk i are done.
-            bool ok = mbar_wait(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !*abort_flag;
-            if (ok) {
-                tc_fence_after_sync();
-                const uint32_t aQ = stage_q(0), aK = aQ + kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
-                for (int k = 0; k < 4; ++k)      // Ph = qh k^T
-                    umma_bf16(tmem + kKvColP, desc_k(aQ + k * 32), desc_k(aK + k * 32), idesc_pp, k > 0);
-                umma_commit(&bars->p_full);
-                for (int k = 0; k < 4; ++k)      // dP = G V^T
-                    umma_bf16(tmem + kKvColDP, desc_k(aG + k * 32), desc_k(aV + k * 32), idesc_pp, k > 0);
-                umma_commit(&bars->dp_full);
-            }
-            #pragma unroll 1
-            for (int i = 0; i < L && ok; ++i) {
-                const int s = i % kKvStages;
-                const uint32_t aQ = stage_q(i), aK = aQ + kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
-                const uint32_t nQ = stage_q(i + 1), nK = nQ + kTileBytes, nV = nK + kTileBytes, nG = nV + kTileBytes;
-                LA_TRACE(g_trace_dkv, i, 0);
-                const uint32_t aR = sbase + kKvOffR + (i & 1) * kDim * 128;      // R_{c+1}: the state before this chunk
-                // gV = k R_{c+1}, once the epilogue of the previous chunk has taken its gV out of TMEM, and the
-                // state update right away: the operand warps wait for it before they reuse the dl column tile
-                ok = mbar_wait(&bars->state_ready, i & 1, prm.status, kStatusPipeTimeout);
-                if (ok && i >= 1) ok = mbar_wait(&bars->dv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok || *abort_flag) { ok = false; break; }
-                tc_fence_after_sync();
-                LA_TRACE(g_trace_dkv, i, 1);
-                for (int k = 0; k < 4; ++k)
-                    umma_bf16(tmem + kKvColDv, desc_k(aK + k * 32), desc_mn(aR + k * 2048), idesc_kmn, k > 0);
-                for (int k = 0; k < 8; ++k)      // [R | r] += qh^T [G | dl]: the dl column tile is the second 64-column block
-                    umma_bf16(tmem + kKvColR, desc_mn(aQ + k * 2048), desc_mn(aG + k * 2048, aAux - aG), idesc_r, 1);
-                umma_commit(&bars->r_full);
-                LA_TRACE(g_trace_dkv, i, 2);
-                ok = mbar_wait(&bars->p_ready, i & 1, prm.status, kStatusPipeTimeout);
-                if (!ok) break;
-                tc_fence_after_sync();
-                for (int k = 0; k < 8; ++k)      // gV += Ph^T G
-                    umma_bf16(tmem + kKvColDv, desc_mn(aP + k * 2048), desc_mn(aG + k * 2048), idesc_mnmn, 1);
-                if (i + 1 < L) {
-                    ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
+            const uint32_t aAux = sbase + kKvOffAux, aOnes = sbase + kKvOffOnes;
+            const uint32_t hi = (uint32_t)(desc_k(0) >> 32);
+            auto mk = [&](uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
+            auto lo_k = [&](uint32_t a) { return (uint32_t)desc_k(a); };
+            auto lo_mn = [&](uint32_t a, uint32_t lbo) { return (uint32_t)desc_mn(a, lbo); };
+            auto stage_q = [&](int i) { return sbase + kKvOffStage + (uint32_t)(i % kKvStages) * kKvStageBytes; };
+            bool ok = true;
+            if (warp == 17) {
+                auto issue_pt = [&](int i) {
+                    const uint32_t dQ = lo_k(stage_q(i)), dK = lo_k(stage_q(i) + kTileBytes);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kKvColP, mk(dK + 2 * k), mk(dQ + 2 * k), idesc_pp, k > 0);
+                    umma_commit(&bars->p_full);
+                };
+                auto issue_dpt = [&](int i) {
+                    const uint32_t dV = lo_k(stage_q(i) + 2 * kTileBytes), dG = lo_k(stage_q(i) + 3 * kTileBytes);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kKvColDP, mk(dV + 2 * k), mk(dG + 2 * k), idesc_pp, k > 0);
+                    umma_bf16(tmem + kKvColDP, desc_ones(aOnes), desc_k(aAux), idesc_pp, 1);
+                    umma_commit(&bars->dp_full);
+                };
+                // The two score tiles run as two interleaved pipelines, so that the score warps always have a
+                // tile to work on: Ph^T of chunk i+1 is issued as soon as the rounded Ph^T of chunk i has been
+                // consumed, while the score warps are busy with dP^T of chunk i, and likewise dP^T.  The next
+                // tile overwrites the rounded copy only after the product that reads it (in-order execution).
+                ok = mbar_wait(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !*abort_flag;
+                if (ok) {
+                    tc_fence_after_sync();
+                    issue_pt(0);
+                    issue_dpt(0);
+                }
+                #pragma unroll 1
+                for (int i = 0; i < L && ok; ++i) {
+                    const uint32_t aQ = stage_q(i), aG = aQ + 3 * kTileBytes;
+                    const uint32_t dGmn = lo_mn(aG, kTileBytes), dQmn = lo_mn(aQ, kTileBytes);
+                    LA_TRACE(g_trace_dkv, i, 0);
+                    ok = mbar_wait(&bars->p_ready, i & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait(&bars->kr_full, i & 1, prm.status, kStatusMmaTimeout);
+                    if (!ok || *abort_flag) { ok = false; break; }
+                    tc_fence_after_sync();
+                    LA_TRACE(g_trace_dkv, i, 1);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)      // gV += Ph^T G
+                        umma_bf16_ta(tmem + kKvColDv, tmem + kKvColP + (k >> 2) * 64 + (k & 3) * 8, mk(dGmn + 128 * k), idesc_kmn, 1);
+                    if (i + 1 < L) {
+                        ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_pt(i + 1);
+                    }
+                    LA_TRACE(g_trace_dkv, i, 2);
+                    ok = mbar_wait(&bars->dp_ready, i & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait(&bars->vr_full, i & 1, prm.status, kStatusMmaTimeout);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16(tmem + kKvColP, desc_k(nQ + k * 32), desc_k(nK + k * 32), idesc_pp, k > 0);
-                    umma_commit(&bars->p_full);
+                    LA_TRACE(g_trace_dkv, i, 3);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)      // gk += dP^T qh
+                        umma_bf16_ta(tmem + kKvColDk, tmem + kKvColDP + (k >> 2) * 64 + (k & 3) * 8, mk(dQmn + 128 * k), idesc_kmn, 1);
+                    umma_commit(&bars->dkv_full);
+                    // vr_full(i) was awaited and covers the other thread's three products on this stage
+                    umma_commit(&bars->empty[i % kKvStages]);
+                    if (i + 1 < L) issue_dpt(i + 1);
+                    LA_TRACE(g_trace_dkv, i, 4);
                 }
-                // gk = V R_{c+1}^T, once the previous gk has been taken out (the other R tile is being rewritten
-                // meanwhile: this one stays valid until the next r_full)
-                if (i >= 1) ok = mbar_wait(&bars->dk_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok) break;
-                tc_fence_after_sync();
-                for (int k = 0; k < 4; ++k)
-                    umma_bf16(tmem + kKvColDk, desc_k(aV + k * 32), desc_k(aR + k * 32), idesc_kk, k > 0);
-                ok = mbar_wait(&bars->dp_ready, i & 1, prm.status, kStatusPipeTimeout);
-                if (!ok) break;
-                tc_fence_after_sync();
-                LA_TRACE(g_trace_dkv, i, 3);
-                for (int k = 0; k < 8; ++k)      // gk += dP^T qh
-                    umma_bf16(tmem + kKvColDk, desc_mn(aDP + k * 2048), desc_mn(aQ + k * 2048), idesc_mnmn, 1);
-                umma_commit(&bars->dkv_full);
-                umma_commit(&bars->empty[s]);
-                if (i + 1 < L) {
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16(tmem + kKvColDP, desc_k(nG + k * 32), desc_k(nV + k * 32), idesc_pp, k > 0);
-                    umma_commit(&bars->dp_full);
+            } else {
+                #pragma unroll 1
+                for (int i = 0; i < L && ok; ++i) {
+                    const uint32_t aQ = stage_q(i), aK = aQ + kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
+                    const uint32_t aR = sbase + kKvOffR + (i & 1) * kDim * 128;      // R_{c+1}: the state before this chunk
+                    const uint32_t dQmn = lo_mn(aQ, kTileBytes), dG1 = lo_mn(aG, aAux - aG);
+                    // [R | r] += qh^T [G | dl], the dl column tile being the second 64-column block of B.  The
+                    // previous state must have been converted (state_ready), and dP^T of this chunk, which reads
+                    // the same column tile, must be done (dp_full): the operand warps take r_full as the signal
+                    // that the tile may be rewritten.
+                    ok = mbar_wait(&bars->mapped[i % kKvStages], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait(&bars->state_ready, i & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait(&bars->dp_full, i & 1, prm.status, kStatusMmaTimeout);
+                    if (!ok || *abort_flag) { ok = false; break; }
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) umma_bf16(tmem + kKvColR, mk(dQmn + 128 * k), mk(dG1 + 128 * k), idesc_r, 1);
+                    umma_commit(&bars->r_full);
+                    // gV = k R_{c+1} and gk = V R_{c+1}^T start the accumulators, each once the epilogue of the
+                    // previous chunk has taken its values out of TMEM
+                    if (i >= 1) ok = mbar_wait(&bars->dv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    {
+                        const uint32_t dK = lo_k(aK), dRmn = lo_mn(aR, kTileBytes);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kKvColDv, mk(dK + 2 * k), mk(dRmn + 128 * k), idesc_kmn, k > 0);
+                    }
+                    umma_commit(&bars->kr_full);
+                    if (i >= 1) ok = mbar_wait(&bars->dk_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    {
+                        const uint32_t dV = lo_k(aV), dR = lo_k(aR);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kKvColDk, mk(dV + 2 * k), mk(dR + 2 * k), idesc_kk, k > 0);
+                    }
+                    umma_commit(&bars->vr_full);
                 }
-                LA_TRACE(g_trace_dkv, i, 4);
             }
             if (!ok) *abort_flag = 1;
         }
@@ -633,19 +708,17 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             if (!mbar_wait(&bars->full[s], (i / kKvStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             if (t == 0) LA_TRACE(g_trace_dkv, i, 5);
-            uint8_t* rowQ = smem + kKvOffStage + s * 4 * kTileBytes + t * 128;
+            uint8_t* rowQ = smem + kKvOffStage + s * kKvStageBytes + t * 128;
             if (elu) map_row_inplace<true>(rowQ, r7, inv, prm.dim >> 3); else map_row_inplace<false>(rowQ, r7, inv, prm.dim >> 3);
             if (t == 0) LA_TRACE(g_trace_dkv, i, 13);
             if (elu) phi_row_inplace(rowQ + kTileBytes, r7, prm.dim >> 3);
             if (t == 0) LA_TRACE(g_trace_dkv, i, 14);
-            sDelta[s * 128 + t] = delta;
-            // the single dl column tile is an operand of the previous chunk's state MMAs
+            // the single dl column tile is an operand of the previous chunk's dP^T and state MMAs
             if (i >= 1 && !mbar_wait(&bars->r_full, (i - 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             if (t == 0) LA_TRACE(g_trace_dkv, i, 15);
-            uint8_t* aA = smem + kKvOffAux + t * 128;
-            const uint32_t dd = pack_bf16x2(delta, delta);
-            sts128(aA + ((0 ^ r7) << 4), dd, dd, dd, dd);
-            sts128(aA + ((1 ^ r7) << 4), dd, dd, dd, dd);
+            // dl_i as a bf16 high and low part in columns 0 and 1 (the rest of the row stays zero)
+            const float dl_hi = bf16_lo(pack_bf16x2(delta, 0.f));
+            sts128(smem + kKvOffAux + t * 128 + ((0 ^ r7) << 4), pack_bf16x2(dl_hi, delta - dl_hi), 0u, 0u, 0u);
             fence_proxy_async_smem();
             mbar_arrive(&bars->mapped[s]);
             if (t == 0) LA_TRACE(g_trace_dkv, i, 6);
@@ -657,7 +730,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const float* rec = prm.init ? prm.init + bh * (int64_t)(prm.nseg * prm.sub) * kStateFloats : nullptr;
-        state_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, rec, rec ? (seg + 1) * prm.sub : 0,
+        rstate_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, rec, rec ? (seg + 1) * prm.sub : 0,
                    rec ? prm.nseg * prm.sub : 0);                                     // "iteration -1" -> buffer 1
         fence_proxy_async_smem();
         tc_fence_before_sync();
@@ -670,14 +743,12 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             const int64_t row = chunk_row(i) + t;
             if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
-            uint32_t kf[8][4];                      // phi(K) row, logical chunk order
-            load_row(smem + kKvOffStage + s * 4 * kTileBytes + kTileBytes + t * 128, r7, kf);
-            mbar_arrive(&bars->empty[s]);
+            const uint8_t* rowK = smem + kKvOffStage + s * kKvStageBytes + kTileBytes + t * 128;     // phi(K) row, for phi'
 
             if (!mbar_wait(&bars->r_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
             if (t == 0) LA_TRACE(g_trace_dkv, i, 7);
-            state_to_smem(tmem + kKvColR, quad, lane, smem + kKvOffR + ((i + 1) & 1) * kDim * 128, sRv + (i & 1) * 64, nullptr, nullptr);
+            rstate_to_smem(tmem + kKvColR, quad, lane, smem + kKvOffR + ((i + 1) & 1) * kDim * 128, sRv + (i & 1) * 64);
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars->state_ready);
@@ -721,14 +792,15 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 if (h * 32 < prm.dim) {
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
-                        uint32_t outp[4];
+                        uint32_t outp[4], kf[4];
+                        lds128(rowK + (((h * 4 + cc) ^ r7) << 4), kf);
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const int d = h * 32 + cc * 8 + 2 * j;
                             float g0 = __uint_as_float(v[cc * 8 + 2 * j]) + rprev[d];
                             float g1 = __uint_as_float(v[cc * 8 + 2 * j + 1]) + rprev[d + 1];
                             if (prm.phi == LA_PHI_ELU1) {
-                                const float k0 = bf16_lo(kf[h * 4 + cc][j]), k1 = bf16_hi(kf[h * 4 + cc][j]);
+                                const float k0 = bf16_lo(kf[j]), k1 = bf16_hi(kf[j]);
                                 g0 *= k0 > 1.f ? 1.f : k0;          // phi'(x) from phi(x): 1 where x > 0, else phi(x)
                                 g1 *= k1 > 1.f ? 1.f : k1;
                             }
@@ -738,53 +810,30 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     }
                 }
             }
+            mbar_arrive(&bars->empty[s]);           // this thread's phi(K) row has been read
             if (t == 0) LA_TRACE(g_trace_dkv, i, 10);
             named_barrier(1, 128);          // r double buffer
         }
     } else {
-        // ------------------------------------------- P and dP post-processing warps
+        // ------------------------------------------- score warps: Ph^T and dP^T, masked and rounded in place
         const int quad = warp & 3, half = warp >> 2;
-        const int t = quad * 32 + lane;
-        const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        const int blk0 = half, blk1 = half + 2;
-        const bool has0 = blk0 <= quad, has1 = blk1 <= quad;
-        uint8_t* rowP = smem + kKvOffP + t * 128;
-        uint8_t* rowDP = smem + kKvOffDP + t * 128;
         #pragma unroll 1
         for (int i = 0; i < L; ++i) {
-            const int s = i % kKvStages;
-            if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
-            if (*abort_flag) break;
-            const float delta = sDelta[s * 128 + t];
-            bool ok = true;
-            // the two score tiles (Ph, then dP + dl) go through the same rolled code, each with its own hand-off
-#pragma unroll 1
-            for (int m = 0; m < 2 && ok; ++m) {
-                ok = mbar_wait(m ? &bars->dp_full : &bars->p_full, i & 1, prm.status, kStatusMmaTimeout);
-                if (!ok) break;
-                tc_fence_after_sync();
-                if (warp == 3 && lane == 0 && m == 0) LA_TRACE(g_trace_dkv, i, 11);
-                const uint32_t src = tmem + lane_base + (m ? kKvColDP : kKvColP);
-                uint8_t* dst = m ? rowDP : rowP;
-                const float add = m ? delta : 0.f;
-                uint32_t v0[32], v1[32];
-                if (has0) tmem_ld32(src + blk0 * 32, v0);
-                if (has1) tmem_ld32(src + blk1 * 32, v1);
-                tmem_ld_wait();
-                if (has0) score_block_store(v0, dst, r7, blk0, blk0 == quad, lane, add);
-                if (has1) score_block_store(v1, dst, r7, blk1, blk1 == quad, lane, add);
-                fence_proxy_async_smem();
-                tc_fence_before_sync();
-                mbar_arrive(m ? &bars->dp_ready : &bars->p_ready);
+            if (warp == 3 && lane == 0) LA_TRACE(g_trace_dkv, i, 11);
+            if (*abort_flag ||
+                !kv_round_tile(tmem + lane_base + kKvColP, &bars->p_full, &bars->p_ready, i & 1, quad, half, lane, prm.status) ||
+                !kv_round_tile(tmem + lane_base + kKvColDP, &bars->dp_full, &bars->dp_ready, i & 1, quad, half, lane, prm.status)) {
+                *abort_flag = 1;
+                break;
             }
-            if (!ok) { *abort_flag = 1; break; }
             if (warp == 3 && lane == 0) LA_TRACE(g_trace_dkv, i, 12);
         }
     }
 
     tc_fence_before_sync();
     __syncthreads();
+    LA_TRACE_CTA(g_trace_dkv, 1);
     if (warp == 17) {
         __syncwarp();
         tmem_dealloc(tmem, 512);

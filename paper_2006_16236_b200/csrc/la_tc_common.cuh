@@ -356,6 +356,86 @@ __device__ __forceinline__ void score_block_pack(const uint32_t (&v)[32], bool p
     }
 }
 
+// The same for a transposed score tile (rows = keys j, columns = queries i): the causal mask
+// keeps i >= j, so a block left of the diagonal (`present` false) is zeros and the diagonal
+// block keeps local columns >= lane.
+__device__ __forceinline__ void score_block_pack_t(const uint32_t (&v)[32], bool present, bool diagonal, int lane,
+                                                   uint32_t (&packed)[16]) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float x0 = __uint_as_float(v[2 * j]), x1 = __uint_as_float(v[2 * j + 1]);
+        if (diagonal) {
+            if (2 * j < lane) x0 = 0.f;
+            if (2 * j + 1 < lane) x1 = 0.f;
+        }
+        packed[j] = present ? sm100::pack_bf16x2(x0, x1) : 0u;
+    }
+}
+
+// Reverse-sweep state [R | r]: r is carried as two columns (the dl column tile holds a bf16
+// high and low part of dl_i in its columns 0 and 1), so r = column 64 + column 65.
+// Accumulator (M = 64 layout) -> bf16 R tile + fp32 r.
+__device__ __forceinline__ void rstate_to_smem(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, float* r_out) {
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const int d_row = quad * 16 + lane;
+    const bool owner = lane < 16;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint32_t v[32];
+        sm100::tmem_ld32(tmem_state + lane_base + h * 32, v);
+        sm100::tmem_ld_wait();
+        if (owner) state_row_store(s_tile, d_row, h, v);
+    }
+    const float r0 = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 64));
+    const float r1 = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 65));
+    sm100::tmem_ld_wait();
+    if (owner) r_out[d_row] = r0 + r1;
+}
+// Initial [R | r] of a segment: the sum of the records of parts [part_lo, part_hi), or zeros.
+// Sixteen columns at a time (rolled): this runs once per CTA and must not raise the register
+// pressure of the role that calls it.
+__device__ __forceinline__ void rstate_init(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, float* r_out,
+                                            const float* rec, int part_lo, int part_hi) {
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const int d_row = quad * 16 + lane;
+    const bool owner = lane < 16;
+#pragma unroll 1
+    for (int g = 0; g < 4; ++g) {
+        float acc[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+        if (owner)
+            for (int p = part_lo; p < part_hi; ++p) {
+                const float4* src = reinterpret_cast<const float4*>(rec + (int64_t)p * kStateFloats + d_row * kDim + g * 16);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float4 a = __ldg(src + j);
+                    acc[4 * j] += a.x; acc[4 * j + 1] += a.y; acc[4 * j + 2] += a.z; acc[4 * j + 3] += a.w;
+                }
+            }
+        uint32_t v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(acc[j]);
+        sm100::tmem_st16(tmem_state + lane_base + g * 16, v);
+        if (owner) {
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc)
+                sts128(s_tile + d_row * 128 + (((2 * g + cc) ^ (d_row & 7)) << 4),
+                       sm100::pack_bf16x2(acc[cc * 8 + 0], acc[cc * 8 + 1]), sm100::pack_bf16x2(acc[cc * 8 + 2], acc[cc * 8 + 3]),
+                       sm100::pack_bf16x2(acc[cc * 8 + 4], acc[cc * 8 + 5]), sm100::pack_bf16x2(acc[cc * 8 + 6], acc[cc * 8 + 7]));
+        }
+    }
+    float r = 0.f;
+    if (owner)
+        for (int p = part_lo; p < part_hi; ++p) r += __ldg(rec + (int64_t)p * kStateFloats + kDim * kDim + d_row);
+    uint32_t rr[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) rr[j] = j == 0 ? __float_as_uint(r) : 0u;      // all of r in column 64
+    sm100::tmem_st16(tmem_state + lane_base + 64, rr);
+    sm100::tmem_st_wait();
+    if (owner) r_out[d_row] = r;
+}
+
 // tcgen05.mma with the A operand read from TMEM (bf16 pairs: column j of lane i = A[i][2j], A[i][2j+1]).
 __device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                              uint32_t accumulate) {
