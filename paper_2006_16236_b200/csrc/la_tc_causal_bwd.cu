@@ -421,33 +421,6 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
 // Warps 0-7: P and dP post-processing, 8-11: state conversion and dK/dV
 // epilogue, 12-15: qh = phi(Q) / dn, phi(K), dl column, 16: TMA, 17: MMA.
 // ===========================================================================
-// One transposed score tile (rows = keys, columns = queries; fp32 in TMEM at `pb`, this thread's
-// lane): wait for it, mask (keep query >= key), round to bf16 pairs in place, signal `ready`.
-// Deliberately not inlined: the two tiles of a chunk share one copy of this code, whose shape
-// then does not depend on what the compiler makes of the surrounding role loops.
-__device__ __noinline__ bool kv_round_tile(uint32_t pb, uint64_t* full, uint64_t* ready, uint32_t parity, int quad,
-                                           int half, int lane, int* status) {
-    if (!mbar_wait(full, parity, status, kStatusMmaTimeout)) return false;
-    tc_fence_after_sync();
-    const int blkA = 2 * half, blkB = 2 * half + 1;     // blocks left of the diagonal block `quad` are zeros
-    const bool hasA = blkA >= quad, hasB = blkB >= quad;
-    uint32_t v[32], pk[16];
-    if (hasA) tmem_ld32(pb + blkA * 32, v);
-    tmem_ld_wait();
-    score_block_pack_t(v, hasA, blkA == quad, lane, pk);
-    if (hasB) tmem_ld32(pb + blkB * 32, v);
-    // bf16 block j of this warp goes to columns 64 half + 16 j .. + 15: inside the fp32 columns
-    // of block 2 half, which this thread has read, so nothing another thread still needs is lost
-    tmem_st16(pb + half * 64, pk);
-    tmem_ld_wait();
-    score_block_pack_t(v, hasB, blkB == quad, lane, pk);
-    tmem_st16(pb + half * 64 + 16, pk);
-    tmem_st_wait();
-    tc_fence_before_sync();
-    mbar_arrive(ready);
-    return true;
-}
-
 constexpr int kKvStages = 3;
 constexpr int kKvThreads = 608;
 constexpr uint32_t kKvColP = 0;        // 128: Ph^T (fp32, then bf16 pairs in place)
@@ -822,8 +795,8 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         for (int i = 0; i < L; ++i) {
             if (warp == 3 && lane == 0) LA_TRACE(g_trace_dkv, i, 11);
             if (*abort_flag ||
-                !kv_round_tile(tmem + lane_base + kKvColP, &bars->p_full, &bars->p_ready, i & 1, quad, half, lane, prm.status) ||
-                !kv_round_tile(tmem + lane_base + kKvColDP, &bars->dp_full, &bars->dp_ready, i & 1, quad, half, lane, prm.status)) {
+                !round_score_tile<true>(tmem + lane_base + kKvColP, &bars->p_full, &bars->p_ready, i & 1, quad, half, lane, prm.status) ||
+                !round_score_tile<true>(tmem + lane_base + kKvColDP, &bars->dp_full, &bars->dp_ready, i & 1, quad, half, lane, prm.status)) {
                 *abort_flag = 1;
                 break;
             }

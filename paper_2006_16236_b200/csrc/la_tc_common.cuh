@@ -436,6 +436,37 @@ __device__ __forceinline__ void rstate_init(uint32_t tmem_state, int quad, int l
     if (owner) r_out[d_row] = r;
 }
 
+// One 128 x 128 score tile (fp32 in TMEM at `pb`, this thread's lane): wait for it, apply the
+// causal mask, round to bf16 pairs in place, signal `ready`.  kTransposed: rows are keys and
+// columns queries (keep query >= key), else rows are queries (keep key <= query).  The warp
+// (quad, half) owns the 32-column blocks 2 half and 2 half + 1 of the quadrant's 32 rows; the bf16
+// block j of a warp goes to columns 64 half + 16 j .. + 15, inside fp32 columns this thread has
+// already read, so nothing another thread still needs is overwritten.
+// Deliberately not inlined: every caller shares one copy, whose shape does not depend on what the
+// compiler makes of the surrounding role loops (inlined, the same source ran up to 1.5x slower
+// depending on unrelated statements nearby).
+template <bool kTransposed>
+__device__ __noinline__ bool round_score_tile(uint32_t pb, uint64_t* full, uint64_t* ready, uint32_t parity, int quad,
+                                              int half, int lane, int* status) {
+    if (!sm100::mbar_wait(full, parity, status, sm100::kStatusMmaTimeout)) return false;
+    sm100::tc_fence_after_sync();
+    const int blkA = 2 * half, blkB = 2 * half + 1;
+    const bool hasA = kTransposed ? blkA >= quad : blkA <= quad, hasB = kTransposed ? blkB >= quad : blkB <= quad;
+    uint32_t v[32], pk[16];
+    if (hasA) sm100::tmem_ld32(pb + blkA * 32, v);
+    sm100::tmem_ld_wait();
+    if (kTransposed) score_block_pack_t(v, hasA, blkA == quad, lane, pk); else score_block_pack(v, hasA, blkA == quad, lane, pk);
+    if (hasB) sm100::tmem_ld32(pb + blkB * 32, v);
+    sm100::tmem_st16(pb + half * 64, pk);
+    sm100::tmem_ld_wait();
+    if (kTransposed) score_block_pack_t(v, hasB, blkB == quad, lane, pk); else score_block_pack(v, hasB, blkB == quad, lane, pk);
+    sm100::tmem_st16(pb + half * 64 + 16, pk);
+    sm100::tmem_st_wait();
+    sm100::tc_fence_before_sync();
+    sm100::mbar_arrive(ready);
+    return true;
+}
+
 // tcgen05.mma with the A operand read from TMEM (bf16 pairs: column j of lane i = A[i][2j], A[i][2j+1]).
 __device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                              uint32_t accumulate) {
