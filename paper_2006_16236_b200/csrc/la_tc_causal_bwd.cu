@@ -59,7 +59,7 @@ namespace {
 // Warp 12: TMA.  Warp 13: MMA issue.
 // ===========================================================================
 constexpr int kDqStages = 2;
-constexpr int kDqThreads = 448;
+constexpr int kDqThreads = 480;
 constexpr uint32_t kDqColDP = 0;       // 128
 constexpr uint32_t kDqColGt = 128;     // 2 x 64: h of even / odd chunks
 constexpr uint32_t kDqColT = 256;      // 2 x 64: T = L k of even / odd chunks
@@ -70,14 +70,14 @@ constexpr uint32_t kDqOffDP = kDqOffStage + kDqStages * 4 * kTileBytes;    // 2 
 constexpr uint32_t kDqOffL = kDqOffDP + 2 * kTileBytes;                    // 2 tiles: lower-triangular ones
 constexpr uint32_t kDqOffS = kDqOffL + 2 * kTileBytes;                     // bf16 S tile
 constexpr uint32_t kDqOffOnes = kDqOffS + kDim * 128;
-constexpr uint32_t kDqOffZ = kDqOffOnes + 1024;                            // fp32 [3][64]
+constexpr uint32_t kDqOffZ = kDqOffOnes + 2048;                            // fp32 [3][64]
 constexpr uint32_t kDqOffX = kDqOffZ + 768;                                // fp32 [2 halves][128][2]: row-pair exchange
 constexpr uint32_t kDqOffBar = kDqOffX + 2048;
 constexpr uint32_t kDqSmemBytes = kDqOffBar + 256 + 1024;
 
 struct DqBarriers {
     uint64_t full[kDqStages], empty[kDqStages], mapped[kDqStages];
-    uint64_t dq_full[2], dq_drained[2];
+    uint64_t dq_full[2], dq_drained[2], gst_full[2];
     uint64_t dp_full, dp_ready, s_full, state_ready;
     uint32_t tmem_base;
     int abort_flag;
@@ -125,6 +125,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         for (int b = 0; b < 2; ++b) {
             mbar_init(&bars->dq_full[b], 1);
             mbar_init(&bars->dq_drained[b], 256);
+            mbar_init(&bars->gst_full[b], 1);
         }
         mbar_init(&bars->dp_full, 1);
         mbar_init(&bars->dp_ready, 256);
@@ -140,7 +141,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     }
     // the score tile is zero right of the diagonal for ever: clear it once
     for (uint32_t i = tid; i < 2 * kTileBytes / 16; i += kDqThreads) sts128(smem + kDqOffDP + i * 16, 0u, 0u, 0u, 0u);
-    for (int i = tid; i < 256; i += kDqThreads) reinterpret_cast<uint32_t*>(smem + kDqOffOnes)[i] = 0x3F803F80u;
+    for (int i = tid; i < 512; i += kDqThreads) reinterpret_cast<uint32_t*>(smem + kDqOffOnes)[i] = 0x3F803F80u;
     if (tid < 128) {        // L[i][j] = 1 for j <= i
         const uint32_t r7 = tid & 7;
         for (int cc = 0; cc < 16; ++cc) {
@@ -181,56 +182,92 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 tma_load_2d(st + 3 * kTileBytes, &mapQ, 0, y, &bars->full[s]);
             }
         }
-    } else if (warp == 13) {
-        // ------------------------------------------------------------- MMA issuer
+    } else if (warp >= 13) {
+        // ------------------------------------------------------------- MMA issuers
+        // Two threads share the issue work (an issuing thread needs about 100 cycles per tcgen05.mma here,
+        // more than the tensor pipe does).  Warp 13: the score tile dP = G V^T and the product that consumes
+        // its rounded copy, h += dP k.  Warp 14: everything that involves the running state (h = G S^T,
+        // St += k^T [V | 1]) and T = L k.  MMAs of one thread execute in order; gst_full orders the two
+        // threads' writes to the h accumulator and tells warp 13 that warp 14 is done with a stage.
         if (lane == 0) {
             const uint32_t idesc_dp = umma_idesc_bf16(128, 128, 0, 0);
             const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
             const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
-            const uint32_t idesc_s = umma_idesc_bf16(64, 64, 1, 1);
-            const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
+            const uint32_t idesc_s = umma_idesc_bf16(64, 80, 1, 1);
             const uint32_t aS = sbase + kDqOffS, aOnes = sbase + kDqOffOnes, aL = sbase + kDqOffL,
                            aDP = sbase + kDqOffDP;
+            const uint32_t hi = (uint32_t)(desc_k(0) >> 32);
+            auto mk = [&](uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
+            auto lo_k = [&](uint32_t a) { return (uint32_t)desc_k(a); };
+            auto lo_mn = [&](uint32_t a, uint32_t lbo) { return (uint32_t)desc_mn(a, lbo); };
+            auto stage_k = [&](int c) { return sbase + kDqOffStage + (uint32_t)(c % kDqStages) * 4 * kTileBytes; };
             bool ok = true;
-            #pragma unroll 1
-            for (int c = 0; c < L && ok; ++c) {
-                const int s = c % kDqStages, b = c & 1;
-                const uint32_t aK = sbase + kDqOffStage + s * 4 * kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
-                // dP = G V^T needs only the raw tiles (the dP tile in TMEM is free: dp_ready(c-1) was awaited)
-                ok = mbar_wait(&bars->full[s], (c / kDqStages) & 1, prm.status, kStatusTmaTimeout);
-                if (!ok || *abort_flag) { ok = false; break; }
-                tc_fence_after_sync();
-                LA_TRACE(g_trace_dq, c, 0);
-                for (int k = 0; k < 4; ++k)
-                    umma_bf16(tmem + kDqColDP, desc_k(aG + k * 32), desc_k(aV + k * 32), idesc_dp, k > 0);
-                umma_commit(&bars->dp_full);
-                ok = mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout) &&
-                     mbar_wait(&bars->state_ready, c & 1, prm.status, kStatusPipeTimeout);
-                if (ok && c >= 2) ok = mbar_wait(&bars->dq_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok) break;
-                tc_fence_after_sync();
-                LA_TRACE(g_trace_dq, c, 1);
-                for (int k = 0; k < 4; ++k)      // h = G S_{c-1}^T
-                    umma_bf16(tmem + kDqColGt + b * 64, desc_k(aG + k * 32), desc_k(aS + k * 32), idesc_kk, k > 0);
-                for (int k = 0; k < 8; ++k)      // S += k^T V
-                    umma_bf16(tmem + kDqColS, desc_mn(aK + k * 2048), desc_mn(aV + k * 2048), idesc_s, 1);
-                for (int k = 0; k < 8; ++k)      // Z += k^T 1
-                    umma_bf16(tmem + kDqColS + 64, desc_mn(aK + k * 2048), desc_ones(aOnes), idesc_z, 1);
-                umma_commit(&bars->s_full);
-                for (int k = 0; k < 8; ++k)      // T = L k  (row-wise prefix sums of k inside the chunk)
-                    umma_bf16(tmem + kDqColT + b * 64, desc_k(aL + (k >> 2) * kTileBytes + (k & 3) * 32),
-                              desc_mn(aK + k * 2048), idesc_kmn, k > 0);
-                LA_TRACE(g_trace_dq, c, 2);
-                ok = mbar_wait(&bars->dp_ready, c & 1, prm.status, kStatusPipeTimeout);
-                if (!ok) break;
-                tc_fence_after_sync();
-                LA_TRACE(g_trace_dq, c, 3);
-                for (int k = 0; k < 8; ++k)      // h += dP k
-                    umma_bf16(tmem + kDqColGt + b * 64, desc_k(aDP + (k >> 2) * kTileBytes + (k & 3) * 32),
-                              desc_mn(aK + k * 2048), idesc_kmn, 1);
-                umma_commit(&bars->dq_full[b]);
-                umma_commit(&bars->empty[s]);
-                LA_TRACE(g_trace_dq, c, 4);
+            if (warp == 13) {
+                auto issue_dp = [&](int c) {    // dP = G V^T needs only the raw tiles
+                    const uint32_t dV = lo_k(stage_k(c) + kTileBytes), dG = lo_k(stage_k(c) + 2 * kTileBytes);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kDqColDP, mk(dG + 2 * k), mk(dV + 2 * k), idesc_dp, k > 0);
+                    umma_commit(&bars->dp_full);
+                };
+                ok = mbar_wait(&bars->full[0], 0, prm.status, kStatusTmaTimeout) && !*abort_flag;
+                if (ok) {
+                    tc_fence_after_sync();
+                    issue_dp(0);
+                }
+                #pragma unroll 1
+                for (int c = 0; c < L && ok; ++c) {
+                    const int b = c & 1;
+                    LA_TRACE(g_trace_dq, c, 0);
+                    ok = mbar_wait(&bars->dp_ready, c & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait(&bars->gst_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout);
+                    if (!ok || *abort_flag) { ok = false; break; }
+                    tc_fence_after_sync();
+                    LA_TRACE(g_trace_dq, c, 3);
+                    const uint32_t dDP = lo_k(aDP), dKmn = lo_mn(stage_k(c), kTileBytes);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)      // h += dP k
+                        umma_bf16(tmem + kDqColGt + b * 64, mk(dDP + (k >> 2) * (kTileBytes >> 4) + (k & 3) * 2), mk(dKmn + 128 * k),
+                                  idesc_kmn, 1);
+                    umma_commit(&bars->dq_full[b]);
+                    // gst_full(c) was awaited: it covers the other thread's products on this stage
+                    umma_commit(&bars->empty[c % kDqStages]);
+                    LA_TRACE(g_trace_dq, c, 4);
+                    // the score tile in TMEM is free (dp_ready(c)); the shared-memory copy is rewritten only after
+                    // dp_full(c+1), which this commit orders behind h += dP k
+                    if (c + 1 < L) {
+                        ok = mbar_wait(&bars->full[(c + 1) % kDqStages], ((c + 1) / kDqStages) & 1, prm.status, kStatusTmaTimeout);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_dp(c + 1);
+                    }
+                }
+            } else {
+                #pragma unroll 1
+                for (int c = 0; c < L && ok; ++c) {
+                    const int s = c % kDqStages, b = c & 1;
+                    const uint32_t aK = stage_k(c), aV = aK + kTileBytes, aG = aV + kTileBytes;
+                    const uint32_t dKmn = lo_mn(aK, kTileBytes), dV1 = lo_mn(aV, aOnes - aV), dG = lo_k(aG), dS = lo_k(aS), dL = lo_k(aL);
+                    constexpr uint32_t kStepV1 = 128u - (128u << 16);
+                    ok = mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait(&bars->state_ready, c & 1, prm.status, kStatusPipeTimeout);
+                    if (ok && c >= 2) ok = mbar_wait(&bars->dq_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (!ok || *abort_flag) { ok = false; break; }
+                    tc_fence_after_sync();
+                    LA_TRACE(g_trace_dq, c, 1);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)      // h = G S_{c-1}^T (before the state tile is rewritten)
+                        umma_bf16(tmem + kDqColGt + b * 64, mk(dG + 2 * k), mk(dS + 2 * k), idesc_kk, k > 0);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)      // [S | Z] += k^T [V | 1]: the ones region is the second 64-column block
+                        umma_bf16(tmem + kDqColS, mk(dKmn + 128 * k), mk(dV1 + kStepV1 * k), idesc_s, 1);
+                    umma_commit(&bars->s_full);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)      // T = L k  (row-wise prefix sums of k inside the chunk)
+                        umma_bf16(tmem + kDqColT + b * 64, mk(dL + (k >> 2) * (kTileBytes >> 4) + (k & 3) * 2), mk(dKmn + 128 * k),
+                                  idesc_kmn, k > 0);
+                    umma_commit(&bars->gst_full[b]);
+                    LA_TRACE(g_trace_dq, c, 2);
+                }
             }
             if (!ok) *abort_flag = 1;
         }
@@ -261,8 +298,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         bool ok = map_chunk(0);
         #pragma unroll 1
         for (int c = 0; c < L && ok; ++c) {
-            if (c + 1 < L) ok = map_chunk(c + 1);
-            if (!ok || *abort_flag) { ok = false; break; }
+            if (*abort_flag) { ok = false; break; }
             if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
             tc_fence_after_sync();
             if (t == 0) LA_TRACE(g_trace_dq, c, 7);
@@ -273,6 +309,9 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             tc_fence_before_sync();
             mbar_arrive(&bars->state_ready);
             if (t == 0) LA_TRACE(g_trace_dq, c, 8);
+            // the state conversion first (the state chain waits for it), then the next chunk's operands
+            // (which may still be in flight)
+            if (c + 1 < L) ok = map_chunk(c + 1);
         }
         if (!ok) *abort_flag = 1;
     } else {
@@ -313,14 +352,28 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             return m;
         };
 
+        // This thread's part of the phi(Q) row of a chunk (logical 16-byte chunks 4 half .. 4 half + 3) is taken
+        // into registers at the end of the previous chunk's epilogue, ahead of its own, so that the stage goes
+        // back to the TMA producer early.
+        uint32_t qv[4][4];
+        auto load_q = [&](int c) -> bool {
+            const int s = c % kDqStages;
+            if (!mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout)) return false;
+            const uint8_t* rowQ = smem + kDqOffStage + s * 4 * kTileBytes + 3 * kTileBytes + t * 128;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) lds128(rowQ + (((half * 4 + cc) ^ r7) << 4), qv[cc]);
+            mbar_arrive(&bars->empty[s]);
+            return true;
+        };
         bool ok = mbar_wait(&bars->dp_full, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
         if (ok) {
             tc_fence_after_sync();
             m_prev = process_scores(0);
+            ok = load_q(0);
         }
         #pragma unroll 1
         for (int c = 0; c < L && ok; ++c) {
-            const int s = c % kDqStages, b = c & 1;
+            const int b = c & 1;
             float m_next = 0.f;
             if (c + 1 < L) {            // scores of the next chunk first: its MMAs then overlap this chunk's epilogue
                 if (!mbar_wait(&bars->dp_full, (c + 1) & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
@@ -330,13 +383,6 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 if (warp == 3 && lane == 0) LA_TRACE(g_trace_dq, c + 1, 12);
             }
             // ---- epilogue of chunk c: this thread owns columns [32 half, 32 half + 32) of row t
-            if (!mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout)) { ok = false; break; }
-            uint32_t qv[4][4];                               // phi(Q) row, logical chunks 4 half .. 4 half + 3
-            {
-                const uint8_t* rowQ = smem + kDqOffStage + s * 4 * kTileBytes + 3 * kTileBytes + t * 128;
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) lds128(rowQ + (((half * 4 + cc) ^ r7) << 4), qv[cc]);
-            }
             if (!mbar_wait(&bars->dq_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
             if (*abort_flag) { ok = false; break; }
             tc_fence_after_sync();
@@ -347,7 +393,6 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             tmem_ld32(tmem + lane_base + kDqColT + b * 64 + half * 32, tt);
             tmem_ld_wait();
             tc_fence_before_sync();
-            mbar_arrive(&bars->empty[s]);                   // this thread's part of phi(Q) is in registers
             const float m = m_prev;
             float qg4[4] = {0.f, 0.f, 0.f, 0.f}, qz4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -404,6 +449,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             }
             if (tid == 0) LA_TRACE(g_trace_dq, c, 10);
             m_prev = m_next;
+            if (c + 1 < L) ok = load_q(c + 1);
         }
         if (!ok) *abort_flag = 1;
     }
