@@ -487,7 +487,7 @@ static_assert(kKvSmemBytes <= 232448, "shared memory budget of one CTA");
 
 struct KvBarriers {
     uint64_t full[kKvStages], empty[kKvStages], mapped[kKvStages];
-    uint64_t p_full, dp_full, p_ready, dp_ready, r_full, state_ready, dkv_full, dk_drained, dv_drained, kr_full, vr_full;
+    uint64_t p_full, dp_full, p_ready, dp_ready, r_full, state_ready, dkv_full, dv_full, dk_drained, dv_drained, kr_full, vr_full;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -544,6 +544,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         mbar_init(&bars->r_full, 1);
         mbar_init(&bars->state_ready, 128);
         mbar_init(&bars->dkv_full, 1);
+        mbar_init(&bars->dv_full, 1);
         mbar_init(&bars->dk_drained, 128);
         mbar_init(&bars->dv_drained, 128);
         mbar_init(&bars->kr_full, 1);
@@ -650,6 +651,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
 #pragma unroll
                     for (int k = 0; k < 8; ++k)      // gV += Ph^T G
                         umma_bf16_ta(tmem + kKvColDv, tmem + kKvColP + (k >> 2) * 64 + (k & 3) * 8, mk(dGmn + 128 * k), idesc_kmn, 1);
+                    umma_commit(&bars->dv_full);    // gV of this chunk is complete: its epilogue overlaps gk
                     if (i + 1 < L) {
                         ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
                         if (!ok) break;
@@ -773,7 +775,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             mbar_arrive(&bars->state_ready);
             if (t == 0) LA_TRACE(g_trace_dkv, i, 8);
 
-            if (!mbar_wait(&bars->dkv_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            if (!mbar_wait(&bars->dv_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
             if (t == 0) LA_TRACE(g_trace_dkv, i, 9);
             const float* rprev = sRv + ((i + 1) & 1) * 64;               // r_{c+1}
@@ -799,6 +801,8 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                                pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
                 }
             }
+            if (!mbar_wait(&bars->dkv_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+            tc_fence_after_sync();
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 uint32_t v[32];
