@@ -679,22 +679,12 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     const uint32_t aQ = stage_q(i), aK = aQ + kTileBytes, aV = aK + kTileBytes, aG = aV + kTileBytes;
                     const uint32_t aR = sbase + kKvOffR + (i & 1) * kDim * 128;      // R_{c+1}: the state before this chunk
                     const uint32_t dQmn = lo_mn(aQ, kTileBytes), dG1 = lo_mn(aG, aAux - aG);
-                    // [R | r] += qh^T [G | dl], the dl column tile being the second 64-column block of B.  The
-                    // previous state must have been converted (state_ready), and dP^T of this chunk, which reads
-                    // the same column tile, must be done (dp_full): the operand warps take r_full as the signal
-                    // that the tile may be rewritten.
+                    // gV = k R_{c+1} starts its accumulator as soon as the epilogue of the previous chunk has taken the
+                    // old values out of TMEM (the score thread waits for it before gV += Ph^T G)
                     ok = mbar_wait(&bars->mapped[i % kKvStages], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout) &&
-                         mbar_wait(&bars->state_ready, i & 1, prm.status, kStatusPipeTimeout) &&
-                         mbar_wait(&bars->dp_full, i & 1, prm.status, kStatusMmaTimeout);
+                         mbar_wait(&bars->state_ready, i & 1, prm.status, kStatusPipeTimeout);
+                    if (ok && i >= 1) ok = mbar_wait(&bars->dv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
                     if (!ok || *abort_flag) { ok = false; break; }
-                    tc_fence_after_sync();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) umma_bf16(tmem + kKvColR, mk(dQmn + 128 * k), mk(dG1 + 128 * k), idesc_r, 1);
-                    umma_commit(&bars->r_full);
-                    // gV = k R_{c+1} and gk = V R_{c+1}^T start the accumulators, each once the epilogue of the
-                    // previous chunk has taken its values out of TMEM
-                    if (i >= 1) ok = mbar_wait(&bars->dv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
-                    if (!ok) break;
                     tc_fence_after_sync();
                     {
                         const uint32_t dK = lo_k(aK), dRmn = lo_mn(aR, kTileBytes);
@@ -702,6 +692,17 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                         for (int k = 0; k < 4; ++k) umma_bf16(tmem + kKvColDv, mk(dK + 2 * k), mk(dRmn + 128 * k), idesc_kmn, k > 0);
                     }
                     umma_commit(&bars->kr_full);
+                    // [R | r] += qh^T [G | dl], the dl column tile being the second 64-column block of B.  The
+                    // previous state has been converted (state_ready), and dP^T of this chunk, which reads the same
+                    // column tile, must be done (dp_full): the operand warps take r_full as the signal that the tile
+                    // may be rewritten.
+                    ok = mbar_wait(&bars->dp_full, i & 1, prm.status, kStatusMmaTimeout);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) umma_bf16(tmem + kKvColR, mk(dQmn + 128 * k), mk(dG1 + 128 * k), idesc_r, 1);
+                    umma_commit(&bars->r_full);
+                    // gk = V R_{c+1}^T likewise, once the previous gk has been taken out
                     if (i >= 1) ok = mbar_wait(&bars->dk_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
                     if (!ok) break;
                     tc_fence_after_sync();
