@@ -752,6 +752,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const float* rec = prm.init ? prm.init + bh * (int64_t)(prm.nseg * prm.sub) * kStateFloats : nullptr;
+        const float slope_floor = prm.phi == LA_PHI_ELU1 ? 0.f : 1.f;
         rstate_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, rec, rec ? (seg + 1) * prm.sub : 0,
                    rec ? prm.nseg * prm.sub : 0);                                     // "iteration -1" -> buffer 1
         fence_proxy_async_smem();
@@ -804,7 +805,10 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             }
             if (!mbar_wait(&bars->dkv_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
-#pragma unroll
+            // gk + r_{c+1}, times phi'(K) = min(phi(K), 1) for elu + 1 (phi > 1 exactly where the slope is 1;
+            // elsewhere the slope equals phi), times 1 for the identity map.  Rolled over the two halves:
+            // the role loops of this kernel together have to fit the instruction cache.
+            #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
                 uint32_t v[32];
                 tmem_ld32(tmem + lane_base + kKvColDk + h * 32, v);
@@ -818,17 +822,16 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     for (int cc = 0; cc < 4; ++cc) {
                         uint32_t outp[4], kf[4];
                         lds128(rowK + (((h * 4 + cc) ^ r7) << 4), kf);
+                        const float4 ra = *reinterpret_cast<const float4*>(rprev + h * 32 + cc * 8);
+                        const float4 rb = *reinterpret_cast<const float4*>(rprev + h * 32 + cc * 8 + 4);
+                        const float rr[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const int d = h * 32 + cc * 8 + 2 * j;
-                            float g0 = __uint_as_float(v[cc * 8 + 2 * j]) + rprev[d];
-                            float g1 = __uint_as_float(v[cc * 8 + 2 * j + 1]) + rprev[d + 1];
-                            if (prm.phi == LA_PHI_ELU1) {
-                                const float k0 = bf16_lo(kf[j]), k1 = bf16_hi(kf[j]);
-                                g0 *= k0 > 1.f ? 1.f : k0;          // phi'(x) from phi(x): 1 where x > 0, else phi(x)
-                                g1 *= k1 > 1.f ? 1.f : k1;
-                            }
-                            outp[j] = pack_bf16x2(g0, g1);
+                            const float g0 = __uint_as_float(v[cc * 8 + 2 * j]) + rr[2 * j];
+                            const float g1 = __uint_as_float(v[cc * 8 + 2 * j + 1]) + rr[2 * j + 1];
+                            const float s0 = fmaxf(fminf(bf16_lo(kf[j]), 1.f), slope_floor);
+                            const float s1 = fmaxf(fminf(bf16_hi(kf[j]), 1.f), slope_floor);
+                            outp[j] = pack_bf16x2(g0 * s0, g1 * s1);
                         }
                         stg128(dstK + h * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
                     }

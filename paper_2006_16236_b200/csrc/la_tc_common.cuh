@@ -372,6 +372,28 @@ __device__ __forceinline__ void score_block_pack_t(const uint32_t (&v)[32], bool
     }
 }
 
+// The same with one warp-uniform branch per block instead of per-element selects: a block off the
+// diagonal costs sixteen conversions, an absent block none.  (The score warps of the quadrant with
+// four present blocks set the pace of a chunk, and most of their blocks are off the diagonal.)
+template <bool kTransposed>
+__device__ __forceinline__ void score_block_round(const uint32_t (&v)[32], bool present, bool diagonal, int lane,
+                                                  uint32_t (&packed)[16]) {
+    if (!present) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) packed[j] = 0u;
+    } else if (!diagonal) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) packed[j] = sm100::pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+    } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const bool drop0 = kTransposed ? 2 * j < lane : 2 * j > lane;
+            const bool drop1 = kTransposed ? 2 * j + 1 < lane : 2 * j + 1 > lane;
+            packed[j] = sm100::pack_bf16x2(drop0 ? 0.f : __uint_as_float(v[2 * j]), drop1 ? 0.f : __uint_as_float(v[2 * j + 1]));
+        }
+    }
+}
+
 // Reverse-sweep state [R | r]: r is carried as two columns (the dl column tile holds a bf16
 // high and low part of dl_i in its columns 0 and 1), so r = column 64 + column 65.
 // Accumulator (M = 64 layout) -> bf16 R tile + fp32 r.
@@ -455,11 +477,11 @@ __device__ __noinline__ bool round_score_tile(uint32_t pb, uint64_t* full, uint6
     uint32_t v[32], pk[16];
     if (hasA) sm100::tmem_ld32(pb + blkA * 32, v);
     sm100::tmem_ld_wait();
-    if (kTransposed) score_block_pack_t(v, hasA, blkA == quad, lane, pk); else score_block_pack(v, hasA, blkA == quad, lane, pk);
+    score_block_round<kTransposed>(v, hasA, blkA == quad, lane, pk);
     if (hasB) sm100::tmem_ld32(pb + blkB * 32, v);
     sm100::tmem_st16(pb + half * 64, pk);
     sm100::tmem_ld_wait();
-    if (kTransposed) score_block_pack_t(v, hasB, blkB == quad, lane, pk); else score_block_pack(v, hasB, blkB == quad, lane, pk);
+    score_block_round<kTransposed>(v, hasB, blkB == quad, lane, pk);
     sm100::tmem_st16(pb + half * 64 + 16, pk);
     sm100::tmem_st_wait();
     sm100::tc_fence_before_sync();
