@@ -608,8 +608,6 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);     // also: A from TMEM, B MN-major
             const uint32_t idesc_r = umma_idesc_bf16(64, 80, 1, 1);
             const uint32_t aAux = sbase + kKvOffAux, aOnes = sbase + kKvOffOnes;
-            const uint32_t hi = (uint32_t)(desc_k(0) >> 32);
-            auto mk = [&](uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
             auto lo_k = [&](uint32_t a) { return (uint32_t)desc_k(a); };
             auto lo_mn = [&](uint32_t a, uint32_t lbo) { return (uint32_t)desc_mn(a, lbo); };
             auto stage_q = [&](int i) { return sbase + kKvOffStage + (uint32_t)(i % kKvStages) * kKvStageBytes; };
@@ -617,14 +615,12 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             if (warp == 17) {
                 auto issue_pt = [&](int i) {
                     const uint32_t dQ = lo_k(stage_q(i)), dK = lo_k(stage_q(i) + kTileBytes);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kKvColP, mk(dK + 2 * k), mk(dQ + 2 * k), idesc_pp, k > 0);
+                    umma_group4(tmem + kKvColP, dK, 2, dQ, 2, idesc_pp, 0);
                     umma_commit(&bars->p_full);
                 };
                 auto issue_dpt = [&](int i) {
                     const uint32_t dV = lo_k(stage_q(i) + 2 * kTileBytes), dG = lo_k(stage_q(i) + 3 * kTileBytes);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kKvColDP, mk(dV + 2 * k), mk(dG + 2 * k), idesc_pp, k > 0);
+                    umma_group4(tmem + kKvColDP, dV, 2, dG, 2, idesc_pp, 0);
                     umma_bf16(tmem + kKvColDP, desc_ones(aOnes), desc_k(aAux), idesc_pp, 1);
                     umma_commit(&bars->dp_full);
                 };
@@ -648,9 +644,8 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     if (!ok || *abort_flag) { ok = false; break; }
                     tc_fence_after_sync();
                     LA_TRACE(g_trace_dkv, i, 1);
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)      // gV += Ph^T G
-                        umma_bf16_ta(tmem + kKvColDv, tmem + kKvColP + (k >> 2) * 64 + (k & 3) * 8, mk(dGmn + 128 * k), idesc_kmn, 1);
+                    umma_group4_ta(tmem + kKvColDv, tmem + kKvColP, dGmn, 128, idesc_kmn, 1);            // gV += Ph^T G
+                    umma_group4_ta(tmem + kKvColDv, tmem + kKvColP + 64, dGmn + 512, 128, idesc_kmn, 1);
                     umma_commit(&bars->dv_full);    // gV of this chunk is complete: its epilogue overlaps gk
                     if (i + 1 < L) {
                         ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
@@ -664,9 +659,8 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     if (!ok) break;
                     tc_fence_after_sync();
                     LA_TRACE(g_trace_dkv, i, 3);
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)      // gk += dP^T qh
-                        umma_bf16_ta(tmem + kKvColDk, tmem + kKvColDP + (k >> 2) * 64 + (k & 3) * 8, mk(dQmn + 128 * k), idesc_kmn, 1);
+                    umma_group4_ta(tmem + kKvColDk, tmem + kKvColDP, dQmn, 128, idesc_kmn, 1);           // gk += dP^T qh
+                    umma_group4_ta(tmem + kKvColDk, tmem + kKvColDP + 64, dQmn + 512, 128, idesc_kmn, 1);
                     umma_commit(&bars->dkv_full);
                     // vr_full(i) was awaited and covers the other thread's three products on this stage
                     umma_commit(&bars->empty[i % kKvStages]);
@@ -686,11 +680,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     if (ok && i >= 1) ok = mbar_wait(&bars->dv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
                     if (!ok || *abort_flag) { ok = false; break; }
                     tc_fence_after_sync();
-                    {
-                        const uint32_t dK = lo_k(aK), dRmn = lo_mn(aR, kTileBytes);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kKvColDv, mk(dK + 2 * k), mk(dRmn + 128 * k), idesc_kmn, k > 0);
-                    }
+                    umma_group4(tmem + kKvColDv, lo_k(aK), 2, lo_mn(aR, kTileBytes), 128, idesc_kmn, 0);
                     umma_commit(&bars->kr_full);
                     // [R | r] += qh^T [G | dl], the dl column tile being the second 64-column block of B.  The
                     // previous state has been converted (state_ready), and dP^T of this chunk, which reads the same
@@ -699,18 +689,14 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     ok = mbar_wait(&bars->dp_full, i & 1, prm.status, kStatusMmaTimeout);
                     if (!ok) break;
                     tc_fence_after_sync();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) umma_bf16(tmem + kKvColR, mk(dQmn + 128 * k), mk(dG1 + 128 * k), idesc_r, 1);
+                    umma_group4(tmem + kKvColR, dQmn, 128, dG1, 128, idesc_r, 1);
+                    umma_group4(tmem + kKvColR, dQmn + 512, 128, dG1 + 512, 128, idesc_r, 1);
                     umma_commit(&bars->r_full);
                     // gk = V R_{c+1}^T likewise, once the previous gk has been taken out
                     if (i >= 1) ok = mbar_wait(&bars->dk_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    {
-                        const uint32_t dV = lo_k(aV), dR = lo_k(aR);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kKvColDk, mk(dV + 2 * k), mk(dR + 2 * k), idesc_kk, k > 0);
-                    }
+                    umma_group4(tmem + kKvColDk, lo_k(aV), 2, lo_k(aR), 2, idesc_kk, 0);
                     umma_commit(&bars->vr_full);
                 }
             }
@@ -784,7 +770,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             __nv_bfloat16* dstK = prm.dK + row * prm.dim;
             __nv_bfloat16* dstV = prm.dV + row * prm.dim;
             // gV first (plain rounding), so that the next chunk's k R can start early; then gk
-#pragma unroll
+            #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
                 uint32_t v[32];
                 tmem_ld32(tmem + lane_base + kKvColDv + h * 32, v);

@@ -401,7 +401,7 @@ __device__ __forceinline__ void rstate_to_smem(uint32_t tmem_state, int quad, in
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
-#pragma unroll
+#pragma unroll 1
     for (int h = 0; h < 2; ++h) {
         uint32_t v[32];
         sm100::tmem_ld32(tmem_state + lane_base + h * 32, v);
@@ -472,17 +472,20 @@ __device__ __noinline__ bool round_score_tile(uint32_t pb, uint64_t* full, uint6
                                               int half, int lane, int* status) {
     if (!sm100::mbar_wait(full, parity, status, sm100::kStatusMmaTimeout)) return false;
     sm100::tc_fence_after_sync();
-    const int blkA = 2 * half, blkB = 2 * half + 1;
-    const bool hasA = kTransposed ? blkA >= quad : blkA <= quad, hasB = kTransposed ? blkB >= quad : blkB <= quad;
-    uint32_t v[32], pk[16];
-    if (hasA) sm100::tmem_ld32(pb + blkA * 32, v);
-    sm100::tmem_ld_wait();
-    score_block_round<kTransposed>(v, hasA, blkA == quad, lane, pk);
-    if (hasB) sm100::tmem_ld32(pb + blkB * 32, v);
-    sm100::tmem_st16(pb + half * 64, pk);
-    sm100::tmem_ld_wait();
-    score_block_round<kTransposed>(v, hasB, blkB == quad, lane, pk);
-    sm100::tmem_st16(pb + half * 64 + 16, pk);
+    // rolled over the warp's two blocks: this routine is on the critical path of a chunk and has to stay
+    // resident in the instruction cache next to every other role's loop
+#pragma unroll 1
+    for (int b = 0; b < 2; ++b) {
+        const int blk = 2 * half + b;
+        const bool has = kTransposed ? blk >= quad : blk <= quad;
+        uint32_t v[32], pk[16];
+        if (has) {
+            sm100::tmem_ld32(pb + blk * 32, v);
+            sm100::tmem_ld_wait();
+        }
+        score_block_round<kTransposed>(v, has, blk == quad, lane, pk);
+        sm100::tmem_st16(pb + half * 64 + b * 16, pk);
+    }
     sm100::tmem_st_wait();
     sm100::tc_fence_before_sync();
     sm100::mbar_arrive(ready);
@@ -498,6 +501,28 @@ __device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, u
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+
+// Four tcgen05.mma over consecutive K groups of one product, out of line: the low descriptor words
+// advance by a_step / b_step per K group (2 for a K-major operand inside a 128-byte swizzle row, 128
+// for an MN-major operand whose K groups are 2 KB apart); the first one accumulates only if
+// `acc_first`.  An issuing thread spends about a dozen instructions per MMA on moving operands to
+// uniform registers; sharing one copy between all products of a kernel keeps the issuing loops, which
+// run next to every other role's loop, small enough for the instruction cache.
+static __device__ __noinline__ void umma_group4(uint32_t d_tmem, uint32_t a_lo, uint32_t a_step, uint32_t b_lo, uint32_t b_step,
+                                         uint32_t idesc, uint32_t acc_first) {
+    const uint64_t hi = desc_k(0) & 0xFFFFFFFF00000000ull;
+#pragma unroll
+    for (uint32_t k = 0; k < 4; ++k)
+        sm100::umma_bf16(d_tmem, hi | (a_lo + k * a_step), hi | (b_lo + k * b_step), idesc, k > 0 ? 1u : acc_first);
+}
+// The same with the A operand in TMEM (eight columns of bf16 pairs per K group).
+static __device__ __noinline__ void umma_group4_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_step, uint32_t idesc,
+                                            uint32_t acc_first) {
+    const uint64_t hi = desc_k(0) & 0xFFFFFFFF00000000ull;
+#pragma unroll
+    for (uint32_t k = 0; k < 4; ++k)
+        umma_bf16_ta(d_tmem, a_tmem + k * 8, hi | (b_lo + k * b_step), idesc, k > 0 ? 1u : acc_first);
 }
 
 }  // namespace tc
