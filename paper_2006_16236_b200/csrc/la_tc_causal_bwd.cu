@@ -465,10 +465,10 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
 // ===========================================================================
 // Reverse sweep: dK, dV.  Chunks are visited from the last to the first.
 // Warps 0-7: P and dP post-processing, 8-11: state conversion and dK/dV
-// epilogue, 12-15: qh = phi(Q) / dn, phi(K), dl column, 16: TMA, 17: MMA.
+// epilogue, 12-15: qh = phi(Q) / dn, phi(K), dl column, 16: TMA, 17-19: MMA.
 // ===========================================================================
 constexpr int kKvStages = 3;
-constexpr int kKvThreads = 608;
+constexpr int kKvThreads = 640;
 constexpr uint32_t kKvColP = 0;        // 128: Ph^T (fp32, then bf16 pairs in place)
 constexpr uint32_t kKvColDP = 128;     // 128: dP^T
 constexpr uint32_t kKvColDk = 256;     // 64
@@ -534,7 +534,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
     if (tid == 0) {
         for (int s = 0; s < kKvStages; ++s) {
             mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], 1 + 128);      // MMA commit + the epilogue warps (they read phi(K) rows)
+            mbar_init(&bars->empty[s], 2 + 128);      // two MMA commits + the epilogue warps (they read phi(K) rows)
             mbar_init(&bars->mapped[s], 128);
         }
         mbar_init(&bars->p_full, 1);
@@ -595,13 +595,13 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         }
     } else if (warp >= 17) {
         // ------------------------------------------------------------- MMA issuers
-        // Two threads share the issue work (an issuing thread needs about 100 cycles per tcgen05.mma here,
-        // more than the tensor pipe does).  Warp 17: the score tiles and the products that consume them
-        // (transposed tiles, rows = keys: Ph^T = k qh^T, dP^T = [V | 1] [G | dl]^T whose fifth K step is
-        // (ones in two columns) x (dl_i split into a bf16 high and low part); gV += Ph^T G, gk += dP^T qh with
-        // the rounded tiles read from TMEM).  Warp 18: everything that involves the running state
-        // ([R | r] += qh^T [G | dl]; gV = k R, gk = V R^T, which start the two accumulators).  MMAs of one
-        // thread execute in order; kr_full / vr_full order the two threads' writes to one accumulator.
+        // Three threads share the issue work (an issuing thread needs 100 to 140 cycles per tcgen05.mma here,
+        // about twice what the tensor pipe does).  Warps 17 and 19: one score tile each and the product that
+        // consumes it (transposed tiles, rows = keys: Ph^T = k qh^T, then gV += Ph^T G; dP^T = [V | 1] [G | dl]^T,
+        // whose fifth K step is (ones in two columns) x (dl_i split into a bf16 high and low part), then
+        // gk += dP^T qh; the rounded tiles are read from TMEM).  Warp 18: everything that involves the running
+        // state ([R | r] += qh^T [G | dl]; gV = k R, gk = V R^T, which start the two accumulators).  MMAs of
+        // one thread execute in order; kr_full / vr_full order two threads' writes to one accumulator.
         if (lane == 0) {
             const uint32_t idesc_pp = umma_idesc_bf16(128, 128, 0, 0);
             const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
@@ -618,26 +618,18 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     umma_group4(tmem + kKvColP, dK, 2, dQ, 2, idesc_pp, 0);
                     umma_commit(&bars->p_full);
                 };
-                auto issue_dpt = [&](int i) {
-                    const uint32_t dV = lo_k(stage_q(i) + 2 * kTileBytes), dG = lo_k(stage_q(i) + 3 * kTileBytes);
-                    umma_group4(tmem + kKvColDP, dV, 2, dG, 2, idesc_pp, 0);
-                    umma_bf16(tmem + kKvColDP, desc_ones(aOnes), desc_k(aAux), idesc_pp, 1);
-                    umma_commit(&bars->dp_full);
-                };
-                // The two score tiles run as two interleaved pipelines, so that the score warps always have a
-                // tile to work on: Ph^T of chunk i+1 is issued as soon as the rounded Ph^T of chunk i has been
-                // consumed, while the score warps are busy with dP^T of chunk i, and likewise dP^T.  The next
-                // tile overwrites the rounded copy only after the product that reads it (in-order execution).
+                // The two score tiles are two independent pipelines, each with its own issuing thread, so that
+                // the score warps always have a tile to work on: Ph^T of chunk i+1 is issued as soon as the
+                // rounded Ph^T of chunk i has been consumed, and likewise dP^T.  The next tile overwrites the
+                // rounded copy only after the product that reads it (in-order execution within a thread).
                 ok = mbar_wait(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !*abort_flag;
                 if (ok) {
                     tc_fence_after_sync();
                     issue_pt(0);
-                    issue_dpt(0);
                 }
                 #pragma unroll 1
                 for (int i = 0; i < L && ok; ++i) {
-                    const uint32_t aQ = stage_q(i), aG = aQ + 3 * kTileBytes;
-                    const uint32_t dGmn = lo_mn(aG, kTileBytes), dQmn = lo_mn(aQ, kTileBytes);
+                    const uint32_t dGmn = lo_mn(stage_q(i) + 3 * kTileBytes, kTileBytes);
                     LA_TRACE(g_trace_dkv, i, 0);
                     ok = mbar_wait(&bars->p_ready, i & 1, prm.status, kStatusPipeTimeout) &&
                          mbar_wait(&bars->kr_full, i & 1, prm.status, kStatusMmaTimeout);
@@ -647,6 +639,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     umma_group4_ta(tmem + kKvColDv, tmem + kKvColP, dGmn, 128, idesc_kmn, 1);            // gV += Ph^T G
                     umma_group4_ta(tmem + kKvColDv, tmem + kKvColP + 64, dGmn + 512, 128, idesc_kmn, 1);
                     umma_commit(&bars->dv_full);    // gV of this chunk is complete: its epilogue overlaps gk
+                    umma_commit(&bars->empty[i % kKvStages]);      // this thread's reads of the stage
                     if (i + 1 < L) {
                         ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
                         if (!ok) break;
@@ -654,17 +647,39 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                         issue_pt(i + 1);
                     }
                     LA_TRACE(g_trace_dkv, i, 2);
+                }
+            } else if (warp == 19) {
+                auto issue_dpt = [&](int i) {
+                    const uint32_t dV = lo_k(stage_q(i) + 2 * kTileBytes), dG = lo_k(stage_q(i) + 3 * kTileBytes);
+                    umma_group4(tmem + kKvColDP, dV, 2, dG, 2, idesc_pp, 0);
+                    umma_bf16(tmem + kKvColDP, desc_ones(aOnes), desc_k(aAux), idesc_pp, 1);
+                    umma_commit(&bars->dp_full);
+                };
+                ok = mbar_wait(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !*abort_flag;
+                if (ok) {
+                    tc_fence_after_sync();
+                    issue_dpt(0);
+                }
+                #pragma unroll 1
+                for (int i = 0; i < L && ok; ++i) {
+                    const uint32_t dQmn = lo_mn(stage_q(i), kTileBytes);
                     ok = mbar_wait(&bars->dp_ready, i & 1, prm.status, kStatusPipeTimeout) &&
                          mbar_wait(&bars->vr_full, i & 1, prm.status, kStatusMmaTimeout);
-                    if (!ok) break;
+                    if (!ok || *abort_flag) { ok = false; break; }
                     tc_fence_after_sync();
                     LA_TRACE(g_trace_dkv, i, 3);
                     umma_group4_ta(tmem + kKvColDk, tmem + kKvColDP, dQmn, 128, idesc_kmn, 1);           // gk += dP^T qh
                     umma_group4_ta(tmem + kKvColDk, tmem + kKvColDP + 64, dQmn + 512, 128, idesc_kmn, 1);
                     umma_commit(&bars->dkv_full);
-                    // vr_full(i) was awaited and covers the other thread's three products on this stage
+                    // vr_full(i) was awaited and covers the state thread's three products on this stage
                     umma_commit(&bars->empty[i % kKvStages]);
-                    if (i + 1 < L) issue_dpt(i + 1);
+                    if (i + 1 < L) {
+                        // mapped(i+1) also says that the dl column tile holds chunk i+1
+                        ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_dpt(i + 1);
+                    }
                     LA_TRACE(g_trace_dkv, i, 4);
                 }
             } else {
