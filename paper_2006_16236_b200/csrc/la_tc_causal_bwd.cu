@@ -495,8 +495,6 @@ struct KvBarriers {
 struct KvParams {
     const float* dn;            // dn_i from the forward sweep
     const float* dl;            // dl_i = -(G_i . O_i) from the forward sweep
-    __nv_bfloat16* dK;
-    __nv_bfloat16* dV;
     const float* init;          // per (bh, part) [R | r] records of the pre-pass, or null (single segment)
     int sub;
     int* status;
@@ -511,6 +509,7 @@ struct KvParams {
 __global__ void __launch_bounds__(kKvThreads, 1)
 causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                       const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapG,
+                      const __grid_constant__ CUtensorMap mapDK, const __grid_constant__ CUtensorMap mapDV,
                       const KvParams prm) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -534,7 +533,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
     if (tid == 0) {
         for (int s = 0; s < kKvStages; ++s) {
             mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], 2 + 128);      // two MMA commits + the epilogue warps (they read phi(K) rows)
+            mbar_init(&bars->empty[s], 2 + 1);        // two MMA commits + the epilogue (its stores leave from the stage)
             mbar_init(&bars->mapped[s], 128);
         }
         mbar_init(&bars->p_full, 1);
@@ -576,6 +575,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG);
+            prefetch_tensormap(&mapDK); prefetch_tensormap(&mapDV);
             #pragma unroll 1
             for (int i = 0; i < L; ++i) {
                 const int s = i % kKvStages;
@@ -764,7 +764,6 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         #pragma unroll 1
         for (int i = 0; i < L; ++i) {
             const int s = i % kKvStages;
-            const int64_t row = chunk_row(i) + t;
             if (!mbar_wait(&bars->mapped[s], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             const uint8_t* rowK = smem + kKvOffStage + s * kKvStageBytes + kTileBytes + t * 128;     // phi(K) row, for phi'
@@ -782,8 +781,11 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             tc_fence_after_sync();
             if (t == 0) LA_TRACE(g_trace_dkv, i, 9);
             const float* rprev = sRv + ((i + 1) & 1) * 64;               // r_{c+1}
-            __nv_bfloat16* dstK = prm.dK + row * prm.dim;
-            __nv_bfloat16* dstV = prm.dV + row * prm.dim;
+            // The results leave through the stage: dV rows overwrite this chunk's G tile and dK rows its phi(K)
+            // tile (every product that reads them is complete by then, and a thread reads its phi(K) row before
+            // it writes there), and one thread stores each tile with TMA: full 128-byte rows per request instead
+            // of 32 rows per store instruction.
+            uint8_t* rowG = smem + kKvOffStage + s * kKvStageBytes + 3 * kTileBytes + t * 128;
             // gV first (plain rounding), so that the next chunk's k R can start early; then gk
             #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
@@ -797,12 +799,18 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 if (h * 32 < prm.dim) {                   // columns beyond a 32-wide problem are padding
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc)
-                        stg128(dstV + h * 32 + cc * 8,
+                        sts128(rowG + (((h * 4 + cc) ^ r7) << 4),
                                pack_bf16x2(__uint_as_float(v[cc * 8 + 0]), __uint_as_float(v[cc * 8 + 1])),
                                pack_bf16x2(__uint_as_float(v[cc * 8 + 2]), __uint_as_float(v[cc * 8 + 3])),
                                pack_bf16x2(__uint_as_float(v[cc * 8 + 4]), __uint_as_float(v[cc * 8 + 5])),
                                pack_bf16x2(__uint_as_float(v[cc * 8 + 6]), __uint_as_float(v[cc * 8 + 7])));
                 }
+            }
+            fence_proxy_async_smem();
+            named_barrier(1, 128);
+            if (t == 0) {
+                tma_store_2d(&mapDV, smem + kKvOffStage + s * kKvStageBytes + 3 * kTileBytes, 0, (int)chunk_row(i));
+                tma_store_commit();
             }
             if (!mbar_wait(&bars->dkv_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
@@ -834,14 +842,21 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                             const float s1 = fmaxf(fminf(bf16_hi(kf[j]), 1.f), slope_floor);
                             outp[j] = pack_bf16x2(g0 * s0, g1 * s1);
                         }
-                        stg128(dstK + h * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
+                        sts128(const_cast<uint8_t*>(rowK) + (((h * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
                     }
                 }
             }
-            mbar_arrive(&bars->empty[s]);           // this thread's phi(K) row has been read
+            fence_proxy_async_smem();
+            named_barrier(1, 128);          // all dK rows are in the tile; also orders the r double buffer
+            if (t == 0) {
+                tma_store_2d(&mapDK, smem + kKvOffStage + s * kKvStageBytes + kTileBytes, 0, (int)chunk_row(i));
+                tma_store_commit();
+                tma_store_wait_read<0>();           // both tiles have been read: the stage may be refilled
+                mbar_arrive(&bars->empty[s]);
+            }
             if (t == 0) LA_TRACE(g_trace_dkv, i, 10);
-            named_barrier(1, 128);          // r double buffer
         }
+        if (t == 0) tma_store_wait_all<0>();
     } else {
         // ------------------------------------------- score warps: Ph^T and dP^T, masked and rounded in place
         const int quad = warp & 3, half = warp >> 2;
@@ -946,8 +961,6 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     KvParams b;
     b.dn = dn;
     b.dl = dl;
-    b.dK = (__nv_bfloat16*)dK;
-    b.dV = (__nv_bfloat16*)dV;
     b.init = sg.nseg > 1 ? rec_r : nullptr;
     b.status = status;
     b.N = p.N;
@@ -960,7 +973,10 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     b.dim = (int)p.D;
     b.map = map ? 1 : 0;
     prof_begin(kProfCausalBwdDkv, st);
-    causal_bwd_dkv_kernel<<<grid, kKvThreads, kKvSmemBytes, st>>>(mQ, mK, mV, mG, b);
+    CUtensorMap mDK, mDV;
+    if (int rc = encode_tile_map(&mDK, dK, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mDV, dV, rows, kChunk, (int)p.D)) return rc;
+    causal_bwd_dkv_kernel<<<grid, kKvThreads, kKvSmemBytes, st>>>(mQ, mK, mV, mG, mDK, mDV, b);
     LA_LAUNCHED();
     prof_end(kProfCausalBwdDkv, st);
     return LA_OK;
