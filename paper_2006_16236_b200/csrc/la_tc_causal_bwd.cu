@@ -73,7 +73,9 @@ constexpr uint32_t kDqOffOnes = kDqOffS + kDim * 128;
 constexpr uint32_t kDqOffZ = kDqOffOnes + 2048;                            // fp32 [3][64]
 constexpr uint32_t kDqOffX = kDqOffZ + 768;                                // fp32 [2 halves][128][2]: row-pair exchange
 constexpr uint32_t kDqOffBar = kDqOffX + 2048;
-constexpr uint32_t kDqSmemBytes = kDqOffBar + 256 + 1024;
+constexpr uint32_t kDqOffOut = (kDqOffBar + 256 + 1023) & ~1023u;          // dQ tile on its way out
+constexpr uint32_t kDqSmemBytes = kDqOffOut + kTileBytes + 1024;           // + slack for the 1 KB alignment of the base
+static_assert(kDqSmemBytes <= 232448, "shared memory budget of one CTA");
 
 struct DqBarriers {
     uint64_t full[kDqStages], empty[kDqStages], mapped[kDqStages];
@@ -86,7 +88,6 @@ struct DqBarriers {
 struct DqParams {
     float* dn;                  // out: dn_i = q_i . Z_i + eps per row, for the reverse sweep
     float* dl;                  // out: dl_i = -(G_i . O_i) per row, for the reverse sweep
-    __nv_bfloat16* dQ;
     const float* init;          // per (bh, part) [S|Z] records of the pre-pass, or null (single segment)
     int sub;                    // parts per segment
     int* status;
@@ -101,7 +102,7 @@ struct DqParams {
 __global__ void __launch_bounds__(kDqThreads, 1)
 causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                      const __grid_constant__ CUtensorMap mapG, const __grid_constant__ CUtensorMap mapQ,
-                     const DqParams prm) {
+                     const __grid_constant__ CUtensorMap mapDQ, const DqParams prm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
@@ -165,6 +166,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG); prefetch_tensormap(&mapQ);
+            prefetch_tensormap(&mapDQ);
             #pragma unroll 1
             for (int c = 0; c < L; ++c) {
                 const int s = c % kDqStages;
@@ -413,6 +415,8 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             // this accumulator pair, and the state warps the Z buffer (only after this arrival)
             mbar_arrive(&bars->dq_drained[b]);
             // combine the two halves of the row
+            // the quadrant's previous dQ slab must have left the staging tile before it is rewritten below
+            if (half == 0 && lane == 0) tma_store_wait_read<0>();
             float* xch = sX + (half * 128 + t) * 2;
             xch[0] = (qg4[0] + qg4[1]) + (qg4[2] + qg4[3]);
             xch[1] = (qz4[0] + qz4[1]) + (qz4[2] + qz4[3]);
@@ -428,10 +432,12 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 prm.dn[row] = dn;
                 prm.dl[row] = delta;
             }
-            __nv_bfloat16* dst = prm.dQ + row * prm.dim + half * 32;
+            // dQ leaves through a staging tile: each quadrant (two warps, 32 rows) fills its 4 KB slab and one
+            // of its threads stores it with TMA: full 128-byte rows per request instead of 32 rows per store
+            // instruction.  Columns beyond a 32-wide problem are padding: the store clips them.
+            uint8_t* out_row = smem + kDqOffOut + t * 128;
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
-                if (half * 32 >= prm.dim) break;          // columns beyond a 32-wide problem are padding
                 uint32_t outp[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -445,12 +451,19 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                     }
                     outp[j] = pack_bf16x2(g0, g1);
                 }
-                stg128(dst + cc * 8, outp[0], outp[1], outp[2], outp[3]);
+                sts128(out_row + (((half * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
+            }
+            fence_proxy_async_smem();
+            named_barrier(2 + quad, 64);
+            if (half == 0 && lane == 0) {
+                tma_store_2d(&mapDQ, smem + kDqOffOut + quad * 32 * 128, 0, (int)(row0 + (int64_t)c * kChunk + quad * 32));
+                tma_store_commit();
             }
             if (tid == 0) LA_TRACE(g_trace_dq, c, 10);
             m_prev = m_next;
             if (c + 1 < L) ok = load_q(c + 1);
         }
+        if (half == 0 && lane == 0) tma_store_wait_all<0>();
         if (!ok) *abort_flag = 1;
     }
 
@@ -939,7 +952,6 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     DqParams a;
     a.dn = dn;
     a.dl = dl;
-    a.dQ = (__nv_bfloat16*)dQ;
     a.init = sg.nseg > 1 ? rec_s : nullptr;
     a.status = status;
     a.N = p.N;
@@ -952,7 +964,9 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.dim = (int)p.D;
     a.map = map ? 1 : 0;
     prof_begin(kProfCausalBwdDq, st);
-    causal_bwd_dq_kernel<<<grid, kDqThreads, kDqSmemBytes, st>>>(mK, mV, mG, mQ, a);
+    CUtensorMap mDQ;
+    if (int rc = encode_tile_map(&mDQ, dQ, rows, 32, (int)p.D)) return rc;      // one quadrant's rows per store
+    causal_bwd_dq_kernel<<<grid, kDqThreads, kDqSmemBytes, st>>>(mK, mV, mG, mQ, mDQ, a);
     LA_LAUNCHED();
     prof_end(kProfCausalBwdDq, st);
 
