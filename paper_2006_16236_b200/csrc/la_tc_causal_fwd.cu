@@ -118,11 +118,11 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             mbar_init(&bars->p_ready[b], 256);
             mbar_init(&bars->o_full[b], 1);
             mbar_init(&bars->o_drained[b], 256);
-            mbar_init(&bars->state_ready[b], 128);
+            mbar_init(&bars->state_ready[b], 256);
             mbar_init(&bars->qs_full[b], 1);
         }
         mbar_init(&bars->s_full, 1);
-        mbar_init(&bars->s_drained, 128);
+        mbar_init(&bars->s_drained, 256);
         bars->abort_flag = 0;
         fence_mbar_init();
     }
@@ -250,14 +250,14 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             if (!ok) *abort_flag = 1;
         }
     } else if (warp >= 12) {
-        // ------------------------------------------------ operand warps: phi(Q) in place
+        // ------- operand warps: phi(Q) in place, and the upper half (columns 32..63) of the state conversion
+        const int quad = warp - 12;
         const int t = tid - 12 * 32;
         const uint32_t r7 = t & 7;
-        #pragma unroll 1
-        for (int c = 0; c < L; ++c) {
+        mbar_arrive(&bars->state_ready[1]);         // the initial state is written by the other group alone
+        auto map_chunk = [&](int c) -> bool {
             const int s = c % kStages;
-            if (!mbar_wait(&bars->full[s], (c / kStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
-            if (*abort_flag) break;
+            if (!mbar_wait(&bars->full[s], (c / kStages) & 1, prm.status, kStatusTmaTimeout)) return false;
             uint8_t* tile = smem + kOffStage + s * kStageBytes;
             if (prm.phi == LA_PHI_ELU1) {
                 phi_row_inplace(tile + t * 128, r7, prm.dim >> 3);
@@ -275,13 +275,33 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 }
             }
             mbar_arrive(&bars->mapped[s]);
+            return true;
+        };
+        bool ok = true;
+        #pragma unroll 1
+        for (int i = 0; i < L + 2 && ok; ++i) {         // step i: state conversion of chunk i - 2, then phi(Q) of chunk i
+            const int c = i - 2;
+            if (c >= 0) {
+                if (*abort_flag) { ok = false; break; }
+                if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
+                tc_fence_after_sync();
+                const bool fin = (c == L - 1) && (seg == prm.nseg - 1);
+                uint8_t* tile = smem + kOffS + (c & 1) * kStateTileBytes;
+                state_half_to_tiles(tmem + kColS, quad, lane, 1, tile, nullptr, &bars->s_drained,
+                                    fin && prm.S_out ? prm.S_out + bh * (int64_t)(prm.dim * prm.dim) : nullptr, nullptr, prm.dim);
+                fence_proxy_async_smem();
+                mbar_arrive(&bars->state_ready[c & 1]);
+            }
+            if (i < L) ok = map_chunk(i);
         }
         if (prm.save && t == 0) {
             tma_store_wait_all<0>();
-            mbar_arrive(&bars->empty[(L - 1) % kStages]);
+            if (ok) mbar_arrive(&bars->empty[(L - 1) % kStages]);
         }
+        if (!ok) *abort_flag = 1;
     } else if (warp >= 8) {
-        // ---------------- operand warps: phi(K) in place (two chunks ahead), then the state conversion
+        // ---- operand warps: phi(K) in place (two chunks ahead), then the lower half (columns 0..31 and Z)
+        // ---- of the state conversion
         const int quad = warp - 8;
         const int t = tid - 8 * 32;
         const uint32_t r7 = t & 7;
@@ -326,9 +346,9 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 if (t == 0) LA_TRACE(g_trace_fwd, c, 7);
                 const bool fin = (c == L - 1) && (seg == prm.nseg - 1);
                 uint8_t* tile = smem + kOffS + (c & 1) * kStateTileBytes;
-                state_to_tiles(tmem + kColS, quad, lane, tile, tile + kDim * 128, &bars->s_drained,
-                               fin && prm.S_out ? prm.S_out + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
-                               fin && prm.Z_out ? prm.Z_out + bh * prm.dim : nullptr, prm.dim);
+                state_half_to_tiles(tmem + kColS, quad, lane, 0, tile, tile + kDim * 128, &bars->s_drained,
+                                    fin && prm.S_out ? prm.S_out + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
+                                    fin && prm.Z_out ? prm.Z_out + bh * prm.dim : nullptr, prm.dim);
                 fence_proxy_async_smem();
                 mbar_arrive(&bars->state_ready[c & 1]);
                 if (t == 0) LA_TRACE(g_trace_fwd, c, 8);

@@ -107,7 +107,7 @@ __device__ __forceinline__ void store_row(uint8_t* row, uint32_t r7, const uint3
 // Feature map on one row in place (optionally scaled), two 16-byte chunks per iteration of a
 // rolled loop: the loop body stays small enough to live in the instruction cache next to the
 // other roles' loops (a fully unrolled row is 8 KB of code per call site).
-template <bool kElu>
+template <bool kElu, bool kScale = true>
 __device__ __forceinline__ void map_row_inplace(uint8_t* row, uint32_t r7, float scale, int nch = 8) {
 #pragma unroll 1
     for (int c = 0; c < nch; c += 2) {
@@ -119,14 +119,15 @@ __device__ __forceinline__ void map_row_inplace(uint8_t* row, uint32_t r7, float
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const float x0 = sm100::bf16_lo(v[i][j]), x1 = sm100::bf16_hi(v[i][j]);
-                v[i][j] = sm100::pack_bf16x2((kElu ? phi_fast(x0) : x0) * scale, (kElu ? phi_fast(x1) : x1) * scale);
+                const float y0 = kElu ? phi_fast(x0) : x0, y1 = kElu ? phi_fast(x1) : x1;
+                v[i][j] = kScale ? sm100::pack_bf16x2(y0 * scale, y1 * scale) : sm100::pack_bf16x2(y0, y1);
             }
         sts128(row + ((c ^ r7) << 4), v[0][0], v[0][1], v[0][2], v[0][3]);
         sts128(row + (((c + 1) ^ r7) << 4), v[1][0], v[1][1], v[1][2], v[1][3]);
     }
 }
 __device__ __forceinline__ void phi_row_inplace(uint8_t* row, uint32_t r7, int nch = 8) {
-    map_row_inplace<true>(row, r7, 1.f, nch);
+    map_row_inplace<true, false>(row, r7, 1.f, nch);
 }
 
 __device__ __forceinline__ uint64_t desc_k(uint32_t addr) { return sm100::umma_desc_sw128(addr, 16, 1024); }
@@ -272,34 +273,30 @@ __device__ __forceinline__ void state_row_store(uint8_t* s_tile, int d_row, int 
     }
 }
 
-// State accumulator -> registers, `drained` is signalled at once (the accumulator may be updated
-// again: the update of the next chunk waits for exactly this), then the bf16 tiles are written;
-// optionally the fp32 values go to global memory.
-__device__ __forceinline__ void state_to_tiles(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, uint8_t* z_tile,
-                                               uint64_t* drained, float* g_S, float* g_Z, int dim) {
+// One half (columns 32 h .. 32 h + 31; h = 0 also carries Z) of the state accumulator -> registers,
+// `drained` is signalled at once (the accumulator may be updated again: the update of the next chunk
+// waits for exactly this), then the bf16 tiles are written; optionally the fp32 values go to global
+// memory.  Two groups of four warps convert one half each.
+__device__ __forceinline__ void state_half_to_tiles(uint32_t tmem_state, int quad, int lane, int h, uint8_t* s_tile,
+                                                    uint8_t* z_tile, uint64_t* drained, float* g_S, float* g_Z, int dim) {
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
-    uint32_t v0[32], v1[32];
-    sm100::tmem_ld32(tmem_state + lane_base, v0);
-    sm100::tmem_ld32(tmem_state + lane_base + 32, v1);
-    const float z = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 64));
+    uint32_t v[32];
+    sm100::tmem_ld32(tmem_state + lane_base + h * 32, v);
+    float z = 0.f;
+    if (h == 0) z = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 64));
     sm100::tmem_ld_wait();
     sm100::tc_fence_before_sync();
     if (drained) sm100::mbar_arrive(drained);
     if (owner) {
-        state_row_store(s_tile, d_row, 0, v0);
-        state_row_store(s_tile, d_row, 1, v1);
-        z_row_store(z_tile, d_row, z);
-        if (g_S && d_row < dim) {
+        state_row_store(s_tile, d_row, h, v);
+        if (h == 0) z_row_store(z_tile, d_row, z);
+        if (g_S && d_row < dim && h * 32 < dim) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) g_S[d_row * dim + j] = __uint_as_float(v0[j]);
-            if (dim > 32) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) g_S[d_row * dim + 32 + j] = __uint_as_float(v1[j]);
-            }
+            for (int j = 0; j < 32; ++j) g_S[d_row * dim + h * 32 + j] = __uint_as_float(v[j]);
         }
-        if (g_Z && d_row < dim) g_Z[d_row] = z;
+        if (h == 0 && g_Z && d_row < dim) g_Z[d_row] = z;
     }
 }
 
