@@ -88,11 +88,10 @@ struct DqBarriers {
 struct DqParams {
     float* dn;                  // out: dn_i = q_i . Z_i + eps per row, for the reverse sweep
     float* dl;                  // out: dl_i = -(G_i . O_i) per row, for the reverse sweep
-    const float* init;          // per (bh, part) [S|Z] records of the pre-pass, or null (single segment)
-    int sub;                    // parts per segment
+    const float* init;          // per (bh, part) [S|Z] records of the pre-pass, or null (single piece)
+    CausalPlan plan;            // pieces of a sequence and their pre-pass parts
     int* status;
     int64_t N;
-    int chunks, chunks_per_seg, nseg;
     float eps;
     int phi;
     int dim;                    // D = M: 64, or 32 (tiles zero-padded to 64 columns)
@@ -111,10 +110,11 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     float* sX = reinterpret_cast<float*>(smem + kDqOffX);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int seg = blockIdx.x % prm.nseg;
-    const int64_t bh = blockIdx.x / prm.nseg;
-    const int c_begin = seg * prm.chunks_per_seg;
-    const int L = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
+    const CausalPlan& plan = prm.plan;
+    const int64_t bh = blockIdx.x % plan.bh;                        // long pieces first: see CausalPlan
+    const int piece = plan.piece_of_slot(blockIdx.x / plan.bh);
+    const int c_begin = plan.piece_begin(piece);
+    const int L = plan.piece_begin(piece + 1) - c_begin;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
 
     if (tid == 0) {
@@ -278,8 +278,8 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         const int quad = warp - 8;
         const int t = tid - 8 * 32;
         const uint32_t r7 = t & 7;
-        const float* rec = prm.init ? prm.init + bh * (int64_t)(prm.nseg * prm.sub) * kStateFloats : nullptr;
-        state_init(tmem + kDqColS, quad, lane, smem + kDqOffS, sZ + 2 * 64, rec, 0, rec ? seg * prm.sub : 0);   // "chunk -1" -> Z buffer 2
+        const float* rec = prm.init ? prm.init + bh * (int64_t)plan.nparts() * kStateFloats : nullptr;
+        state_init(tmem + kDqColS, quad, lane, smem + kDqOffS, sZ + 2 * 64, rec, 0, rec ? plan.piece_first_part(piece) : 0);   // "chunk -1" -> Z buffer 2
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(&bars->state_ready);
@@ -508,11 +508,10 @@ struct KvBarriers {
 struct KvParams {
     const float* dn;            // dn_i from the forward sweep
     const float* dl;            // dl_i = -(G_i . O_i) from the forward sweep
-    const float* init;          // per (bh, part) [R | r] records of the pre-pass, or null (single segment)
-    int sub;
+    const float* init;          // per (bh, part) [R | r] records of the pre-pass, or null (single piece)
+    CausalPlan plan;            // pieces of a sequence and their pre-pass parts
     int* status;
     int64_t N;
-    int chunks, chunks_per_seg, nseg;
     float eps;
     int phi;
     int dim;
@@ -530,10 +529,11 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
     float* sRv = reinterpret_cast<float*>(smem + kKvOffRv);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int seg = blockIdx.x % prm.nseg;
-    const int64_t bh = blockIdx.x / prm.nseg;
-    const int c_begin = seg * prm.chunks_per_seg;
-    const int c_end = min(prm.chunks, c_begin + prm.chunks_per_seg);
+    const CausalPlan& plan = prm.plan;
+    const int64_t bh = blockIdx.x % plan.bh;                        // long pieces first: see CausalPlan
+    const int piece = plan.piece_of_slot(blockIdx.x / plan.bh);
+    const int c_begin = plan.piece_begin(piece);
+    const int c_end = plan.piece_begin(piece + 1);
     const int L = c_end - c_begin;
     // iteration i visits chunk c_end - 1 - i
     auto chunk_row = [&](int i) { return bh * prm.N + (int64_t)(c_end - 1 - i) * kChunk; };
@@ -765,10 +765,10 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const int t = quad * 32 + lane;
         const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        const float* rec = prm.init ? prm.init + bh * (int64_t)(prm.nseg * prm.sub) * kStateFloats : nullptr;
+        const float* rec = prm.init ? prm.init + bh * (int64_t)plan.nparts() * kStateFloats : nullptr;
         const float slope_floor = prm.phi == LA_PHI_ELU1 ? 0.f : 1.f;
-        rstate_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, rec, rec ? (seg + 1) * prm.sub : 0,
-                   rec ? prm.nseg * prm.sub : 0);                                     // "iteration -1" -> buffer 1
+        rstate_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, rec, rec ? plan.piece_first_part(piece + 1) : 0,
+                   rec ? plan.nparts() : 0);                                     // "iteration -1" -> buffer 1
         fence_proxy_async_smem();
         tc_fence_before_sync();
         named_barrier(1, 128);
@@ -899,19 +899,19 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
 }  // namespace
 
 size_t causal_backward_workspace(const la_problem& p) {
-    const Segmentation sg = choose_segments(p);
+    const CausalPlan pl = choose_plan(p);
     const size_t bh = (size_t)(p.B * p.H);
-    size_t bytes = 2 * bh * sg.parts() * kStateFloats * sizeof(float);    // forward and reverse pre-pass records
+    size_t bytes = 2 * bh * pl.nparts() * kStateFloats * sizeof(float);    // forward and reverse pre-pass records
     bytes += 2 * bh * (size_t)p.N * sizeof(float);                       // dn_i and dl_i per row
     return bytes;
 }
 
 int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
                     const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
-    const Segmentation sg = choose_segments(p);
+    const CausalPlan pl = choose_plan(p);
     // With what the forward saved, phi(Q) and phi(K) are read as tensors (no feature map on load)
     // and the forward pre-pass records are the forward's own.
-    const SavedLayout sl = saved_layout(p, sg);
+    const SavedLayout sl = saved_layout(p, pl);
     const uint8_t* sv = (const uint8_t*)saved;
     const bool premapped = sv != nullptr && p.phi == LA_PHI_ELU1;
     const bool map = !premapped && p.phi == LA_PHI_ELU1;
@@ -919,14 +919,13 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
         Q = sv + sl.phiq;
         K = sv + sl.phik;
     }
-    const int chunks = (int)(p.N / kChunk);
     const size_t bh = (size_t)(p.B * p.H);
     const uint64_t rows = (uint64_t)(bh * p.N);
 
     // workspace carve-up (see causal_backward_workspace)
     uint8_t* w = (uint8_t*)ws;
-    float* rec_s = (float*)w;            w += bh * sg.parts() * kStateFloats * sizeof(float);
-    float* rec_r = (float*)w;            w += bh * sg.parts() * kStateFloats * sizeof(float);
+    float* rec_s = (float*)w;            w += bh * pl.nparts() * kStateFloats * sizeof(float);
+    float* rec_r = (float*)w;            w += bh * pl.nparts() * kStateFloats * sizeof(float);
     float* dn = (float*)w;               w += bh * (size_t)p.N * sizeof(float);
     float* dl = (float*)w;
 
@@ -944,21 +943,18 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
         LA_CUDA_TRY(cudaFuncSetAttribute(causal_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kKvSmemBytes));
         attr_done = true;
     }
-    const unsigned grid = (unsigned)(sg.nseg * bh);
+    const unsigned grid = (unsigned)(pl.npieces() * bh);
 
     // forward sweep: dQ, and dn_i, dl_i for the reverse sweep
     if (sv) rec_s = (float*)(sv + sl.records);
-    else if (int rc = segment_states(p, sg, mK, mV, nullptr, nullptr, rec_s, /*reverse=*/false, map, st)) return rc;
+    else if (int rc = segment_states(p, pl, mK, mV, nullptr, nullptr, rec_s, /*reverse=*/false, map, st)) return rc;
     DqParams a;
     a.dn = dn;
     a.dl = dl;
-    a.init = sg.nseg > 1 ? rec_s : nullptr;
+    a.init = pl.npieces() > 1 ? rec_s : nullptr;
+    a.plan = pl;
     a.status = status;
     a.N = p.N;
-    a.chunks = chunks;
-    a.chunks_per_seg = sg.chunks_per_seg;
-    a.nseg = sg.nseg;
-    a.sub = sg.sub;
     a.eps = p.eps;
     a.phi = p.phi;
     a.dim = (int)p.D;
@@ -971,17 +967,14 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     prof_end(kProfCausalBwdDq, st);
 
     // reverse sweep: dK, dV
-    if (int rc = segment_states(p, sg, mQ, mG, dn, dl, rec_r, /*reverse=*/true, map, st)) return rc;
+    if (int rc = segment_states(p, pl, mQ, mG, dn, dl, rec_r, /*reverse=*/true, map, st)) return rc;
     KvParams b;
     b.dn = dn;
     b.dl = dl;
-    b.init = sg.nseg > 1 ? rec_r : nullptr;
+    b.init = pl.npieces() > 1 ? rec_r : nullptr;
+    b.plan = pl;
     b.status = status;
     b.N = p.N;
-    b.chunks = chunks;
-    b.chunks_per_seg = sg.chunks_per_seg;
-    b.nseg = sg.nseg;
-    b.sub = sg.sub;
     b.eps = p.eps;
     b.phi = p.phi;
     b.dim = (int)p.D;

@@ -65,15 +65,12 @@ static_assert(sizeof(Barriers) <= 256, "barrier block");
 struct FwdParams {
     __nv_bfloat16* O;
     float* den;            // [BH, N] or null
-    const float* init;     // per (bh, part) [S|Z] records of the pre-pass, or null (single segment)
-    int sub;               // parts per segment
+    const float* init;     // per (bh, part) [S|Z] records of the pre-pass, or null (single piece)
+    CausalPlan plan;       // pieces of a sequence and their pre-pass parts
     float* S_out;          // [BH, D, M] or null
     float* Z_out;          // [BH, D] or null
     int* status;
     int64_t N;
-    int chunks;            // chunks per sequence
-    int chunks_per_seg;
-    int nseg;
     float eps;
     int phi;
     int dim;               // D = M: 64, or 32 (tiles zero-padded to 64 columns)
@@ -92,11 +89,12 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     Barriers* bars = reinterpret_cast<Barriers*>(smem + kOffBar);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int seg = blockIdx.x % prm.nseg;
-    const int64_t bh = blockIdx.x / prm.nseg;
-    const int c_begin = seg * prm.chunks_per_seg;
-    const int c_end = min(prm.chunks, c_begin + prm.chunks_per_seg);
-    const int L = c_end - c_begin;
+    const CausalPlan& plan = prm.plan;
+    const int64_t bh = blockIdx.x % plan.bh;                        // long pieces first: see CausalPlan
+    const int piece = plan.piece_of_slot(blockIdx.x / plan.bh);
+    const bool last_piece = piece == plan.npieces() - 1;
+    const int c_begin = plan.piece_begin(piece);
+    const int L = plan.piece_begin(piece + 1) - c_begin;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;      // first global row of this segment
 
     LA_TRACE_CTA(g_trace_fwd, 0);
@@ -285,7 +283,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 if (*abort_flag) { ok = false; break; }
                 if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
                 tc_fence_after_sync();
-                const bool fin = (c == L - 1) && (seg == prm.nseg - 1);
+                const bool fin = (c == L - 1) && last_piece;
                 uint8_t* tile = smem + kOffS + (c & 1) * kStateTileBytes;
                 state_half_to_tiles(tmem + kColS, quad, lane, 1, tile, nullptr, &bars->s_drained,
                                     fin && prm.S_out ? prm.S_out + bh * (int64_t)(prm.dim * prm.dim) : nullptr, nullptr, prm.dim);
@@ -305,9 +303,9 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         const int quad = warp - 8;
         const int t = tid - 8 * 32;
         const uint32_t r7 = t & 7;
-        const float* rec = prm.init ? prm.init + bh * (int64_t)(prm.nseg * prm.sub) * kStateFloats : nullptr;
+        const float* rec = prm.init ? prm.init + bh * (int64_t)plan.nparts() * kStateFloats : nullptr;
         uint8_t* tile1 = smem + kOffS + kStateTileBytes;            // the state before chunk 0 lives in tile 1
-        state_init_tiles(tmem + kColS, quad, lane, tile1, tile1 + kDim * 128, rec, 0, rec ? seg * prm.sub : 0);
+        state_init_tiles(tmem + kColS, quad, lane, tile1, tile1 + kDim * 128, rec, 0, rec ? plan.piece_first_part(piece) : 0);
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(&bars->state_ready[1]);
@@ -344,7 +342,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
                 tc_fence_after_sync();
                 if (t == 0) LA_TRACE(g_trace_fwd, c, 7);
-                const bool fin = (c == L - 1) && (seg == prm.nseg - 1);
+                const bool fin = (c == L - 1) && last_piece;
                 uint8_t* tile = smem + kOffS + (c & 1) * kStateTileBytes;
                 state_half_to_tiles(tmem + kColS, quad, lane, 0, tile, tile + kDim * 128, &bars->s_drained,
                                     fin && prm.S_out ? prm.S_out + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
@@ -445,43 +443,61 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 
 }  // namespace
 
-Segmentation choose_segments(const la_problem& p) {
-    const int chunks = (int)(p.N / kChunk);
-    const int64_t bh = p.B * p.H;
-    int nseg = 1;
-    if (const char* e = getenv("LA_TC_NSEG")) {
-        nseg = atoi(e);
-    } else if (bh < 120) {
-        nseg = (int)((120 + bh - 1) / bh);
+CausalPlan choose_plan(const la_problem& p) {
+    constexpr int kSms = 148;
+    CausalPlan pl;
+    pl.chunks = (int)(p.N / kChunk);
+    pl.bh = (int)(p.B * p.H);
+    pl.nlong = 1;
+    pl.m = 0;
+    pl.spos = 0;
+    pl.sub = 1;
+    const char* forced = getenv("LA_TC_NSEG");         // equal pieces, for A/B checks
+    int nlong = forced ? atoi(forced) : (pl.bh < 120 ? kSms / pl.bh : 1);
+    if (nlong > pl.chunks / 2) nlong = pl.chunks / 2;   // a piece is at least two chunks
+    if (nlong < 1) nlong = 1;
+    pl.nlong = nlong;
+    // With B*H*nlong CTAs on 148 SMs, `rest` SMs would idle.  They take one short piece per sequence, several
+    // in a row each (`rounds` at most): the short length m balances a long piece against `rounds` short ones,
+    // each CTA costing about five chunk times to start up and drain (measured: records summed, pipeline filled,
+    // last stores out).  The short piece sits in the middle of the sequence, so that the pre-passes (which skip
+    // the last piece forward, the first one backward) skip a long one.
+    const int rest = kSms - pl.bh * nlong;
+    if (!forced && nlong >= 2 && rest >= 8) {
+        const int rounds = (pl.bh + rest - 1) / rest;
+        const double startup = 5.0;
+        int m = (int)(((double)pl.chunks / nlong - (rounds - 1) * startup) / (rounds + 1.0 / nlong));
+        if (const char* e = getenv("LA_TC_SHORT")) m = atoi(e);        // A/B checks
+        if (m >= 4 && (pl.chunks - m) / nlong >= 2) {
+            pl.m = m;
+            pl.spos = nlong / 2;
+        }
     }
-    if (nseg > chunks / 2) nseg = chunks / 2;
-    if (nseg < 1) nseg = 1;
-    const int cps = (chunks + nseg - 1) / nseg;
-    nseg = (chunks + cps - 1) / cps;
-    // pre-pass parts: about two CTAs per SM in total, each part a whole number of chunks that divides a segment
-    int sub = 1;
-    if (nseg > 1) {
-        const int64_t want = (2 * 148 + bh * (nseg - 1) - 1) / (bh * (nseg - 1));
-        for (int d = 1; d <= cps; ++d)
-            if (cps % d == 0 && d <= want && cps / d >= 2) sub = d;
+    // pre-pass parts: about two CTAs per SM over the parts one pre-pass computes (all but one long piece)
+    if (pl.npieces() > 1) {
+        const int covered = nlong > 1 ? nlong - 1 : 1;
+        int sub = (2 * kSms / pl.bh - pl.has_short()) / covered;
+        const int shortest = (pl.chunks - pl.m) / nlong;
+        if (sub > shortest / 2) sub = shortest / 2;
+        if (sub < 1) sub = 1;
+        pl.sub = sub;
     }
-    return Segmentation{nseg, cps, sub, cps / sub};
+    return pl;
 }
 
 size_t causal_forward_workspace(const la_problem& p) {
-    const Segmentation sg = choose_segments(p);
-    if (sg.nseg <= 1) return 0;
-    return (size_t)(p.B * p.H) * sg.parts() * kStateFloats * sizeof(float);
+    const CausalPlan pl = choose_plan(p);
+    if (pl.npieces() <= 1) return 0;
+    return (size_t)(p.B * p.H) * pl.nparts() * kStateFloats * sizeof(float);
 }
 
-size_t causal_saved_bytes(const la_problem& p) { return saved_layout(p, choose_segments(p)).bytes; }
+size_t causal_saved_bytes(const la_problem& p) { return saved_layout(p, choose_plan(p)).bytes; }
 
 int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
                    float* S_out, float* Z_out, void* saved, void* ws, cudaStream_t st) {
-    const Segmentation sg = choose_segments(p);
-    const int chunks = (int)(p.N / kChunk);
+    const CausalPlan pl = choose_plan(p);
     const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
-    const SavedLayout sl = saved_layout(p, sg);
+    const SavedLayout sl = saved_layout(p, pl);
     uint8_t* sv = (uint8_t*)saved;
     const bool save = sv != nullptr && p.phi == LA_PHI_ELU1;     // with identity features Q, K are the mapped tensors
     CUtensorMap mQ, mK, mV, mPQ, mPK;
@@ -500,27 +516,24 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     }
     // the pre-pass records go straight into the saved buffer when there is one
     float* records = sv ? (float*)(sv + sl.records) : (float*)ws;
-    if (sg.nseg > 1) {
-        if (int rc = segment_states(p, sg, mK, mV, nullptr, nullptr, records, /*reverse=*/false, p.phi == LA_PHI_ELU1, st)) return rc;
+    if (pl.npieces() > 1) {
+        if (int rc = segment_states(p, pl, mK, mV, nullptr, nullptr, records, /*reverse=*/false, p.phi == LA_PHI_ELU1, st)) return rc;
     }
     FwdParams prm;
     prm.O = (__nv_bfloat16*)O;
     prm.den = den;
-    prm.init = sg.nseg > 1 ? records : nullptr;
+    prm.init = pl.npieces() > 1 ? records : nullptr;
+    prm.plan = pl;
     prm.S_out = S_out;
     prm.Z_out = Z_out;
     prm.status = status;
     prm.N = p.N;
-    prm.chunks = chunks;
-    prm.chunks_per_seg = sg.chunks_per_seg;
-    prm.nseg = sg.nseg;
-    prm.sub = sg.sub;
     prm.eps = p.eps;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
     prm.save = save ? 1 : 0;
     prof_begin(kProfCausalFwd, st);
-    causal_fwd_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kThreads, kSmemBytes, st>>>(mQ, mK, mV, mPQ, mPK, prm);
+    causal_fwd_kernel<<<(unsigned)(pl.npieces() * pl.bh), kThreads, kSmemBytes, st>>>(mQ, mK, mV, mPQ, mPK, prm);
     LA_LAUNCHED();
     prof_end(kProfCausalFwd, st);
     return LA_OK;

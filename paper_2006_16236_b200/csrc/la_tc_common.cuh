@@ -28,19 +28,71 @@ constexpr int kDim = 64;                     // D = M = 64: one 128-byte swizzle
 constexpr int kTileBytes = kChunk * kDim * 2;  // one [128][64] bf16 tile
 constexpr int kStateFloats = kDim * (kDim + 1);  // [S (64x64) | Z (64)] per record
 
-// How a (batch, head) sequence is cut into segments that run concurrently.
+// How a (batch, head) sequence of the non-causal kernels is cut into segments that run concurrently.
 struct Segmentation {
     int nseg;             // segments per sequence (one CTA of the main kernels each)
     int chunks_per_seg;   // chunks in every segment but possibly the last
-    int sub;              // parts per segment in the pre-pass (chunks_per_seg is a multiple of chunks_per_part)
-    int chunks_per_part;
-    int parts() const { return nseg * sub; }      // records per (batch, head)
 };
 
-Segmentation choose_segments(const la_problem& p);
+// How the causal kernels cut a sequence into pieces (one CTA of a main kernel each) and the pieces
+// into pre-pass parts (one CTA of the pre-pass and one [S | Z]-shaped record each).
+//   `nlong` long pieces of near-equal length and, if m > 0, one short piece of m chunks at position
+//   `spos` of the sequence.  The CTAs of the long pieces have the lowest block indices and start first;
+//   when B*H*nlong is less than the SM count, the SMs left over take the short pieces, several each, one
+//   after the other, so that every SM is busy for about the same time although B*H does not divide 148.
+//   Every long piece has `sub` parts of near-equal length, the short piece is one part.  A piece starts
+//   from the sum of the records of the parts before it (forward sweep) or after it (reverse sweep).
+// All fields are small integers: the struct is passed to the kernels by value.
+struct CausalPlan {
+    int chunks, bh;       // chunks per sequence; sequences (batch x head pairs)
+    int nlong, m, spos, sub;
 
-// Per-segment sums of phi(X)^T [Y | a] into `records` followed by their exclusive scan
-int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
+    __host__ __device__ int has_short() const { return m > 0 ? 1 : 0; }
+    __host__ __device__ int npieces() const { return nlong + has_short(); }
+    __host__ __device__ int nparts() const { return nlong * sub + has_short(); }
+    // first chunk of the j-th long piece, counted without the short piece
+    __host__ __device__ int long_start(int j) const {
+        const int lt = chunks - m;
+        return j * (lt / nlong) + (j < lt % nlong ? j : lt % nlong);
+    }
+    // piece k of the sequence: first chunk, and first part; k = npieces() gives the end
+    __host__ __device__ int piece_begin(int k) const {
+        if (!has_short() || k <= spos) return long_start(k);
+        return long_start(k - 1) + m;
+    }
+    __host__ __device__ int piece_first_part(int k) const {
+        if (!has_short() || k <= spos) return k * sub;
+        return (k - 1) * sub + 1;
+    }
+    // launch slot (blockIdx.x / bh) -> piece: long pieces first, the short one last
+    __host__ __device__ int piece_of_slot(int slot) const {
+        if (!has_short()) return slot;
+        if (slot == nlong) return spos;
+        return slot < spos ? slot : slot + 1;
+    }
+    // part q of the sequence: first chunk; q = nparts() gives the end
+    __host__ __device__ int part_begin(int q) const {
+        int k, i;                               // piece and index of the part inside it
+        if (has_short() && q >= spos * sub + 1) {
+            k = (q - 1) / sub + 1;
+            i = (q - 1) % sub;
+        } else if (has_short() && q == spos * sub) {
+            return piece_begin(spos);
+        } else {
+            k = q / sub;
+            i = q % sub;
+        }
+        if (k >= npieces()) return chunks;
+        const int b = piece_begin(k), len = piece_begin(k + 1) - b;
+        return b + i * (len / sub) + (i < len % sub ? i : len % sub);
+    }
+};
+
+CausalPlan choose_plan(const la_problem& p);
+
+// Per-part sums of phi(X)^T [Y | a] into `records` (forward: the parts before the last piece; reverse:
+// the parts after the first piece)
+int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap& mapX, const CUtensorMap& mapY,
                    const float* dn, const float* dl, float* records, bool reverse, bool map, cudaStream_t st);
 
 // What the causal forward leaves for the causal backward when the caller passes a `saved`
@@ -51,14 +103,14 @@ int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMa
 struct SavedLayout {
     size_t phiq, phik, records, bytes;      // byte offsets of the three parts; total size
 };
-inline SavedLayout saved_layout(const la_problem& p, const Segmentation& sg) {
+inline SavedLayout saved_layout(const la_problem& p, const CausalPlan& pl) {
     const size_t rows = (size_t)(p.B * p.H * p.N);
     const size_t tensor = (rows * (size_t)p.D * 2 + 1023) & ~(size_t)1023;
     SavedLayout l;
     l.phiq = 0;
     l.phik = tensor;
     l.records = 2 * tensor;
-    l.bytes = l.records + (sg.nseg > 1 ? (size_t)(p.B * p.H) * sg.parts() * kStateFloats * sizeof(float) : 0);
+    l.bytes = l.records + (pl.npieces() > 1 ? (size_t)(p.B * p.H) * pl.nparts() * kStateFloats * sizeof(float) : 0);
     return l;
 }
 

@@ -42,8 +42,8 @@ struct SumParams {
     const float* dl;       // with dn: a_i = dl_i
     int* status;
     int64_t N;
-    int chunks, chunks_per_part, parts;
-    int first_part;        // parts first_part .. first_part + parts_per_seq - 1 are summed
+    CausalPlan plan;
+    int first_part;        // parts first_part .. first_part + parts_per_seq - 1 of every sequence are summed
     int parts_per_seq;
     float eps;
     int map;               // apply the feature map to X on load
@@ -60,8 +60,8 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     LA_TRACE_CTA(g_trace_seg, 0);
     const int seg = prm.first_part + blockIdx.x % prm.parts_per_seq;       // index of this part
     const int64_t bh = blockIdx.x / prm.parts_per_seq;
-    const int c_begin = seg * prm.chunks_per_part;
-    const int L = min(prm.chunks, c_begin + prm.chunks_per_part) - c_begin;
+    const int c_begin = prm.plan.part_begin(seg);
+    const int L = prm.plan.part_begin(seg + 1) - c_begin;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
     const bool scaled = prm.dn != nullptr;
 
@@ -176,7 +176,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
         const bool ok = mbar_wait(&bars->done, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
         tc_fence_after_sync();
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        float* rec = prm.records + (bh * prm.parts + seg) * (int64_t)kStateFloats;
+        float* rec = prm.records + (bh * prm.plan.nparts() + seg) * (int64_t)kStateFloats;
         const int d_row = warp * 16 + lane;
         for (int h = 0; h < 2; ++h) {
             uint32_t v[32];
@@ -201,9 +201,9 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
 
 }  // namespace
 
-int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMap& mapX, const CUtensorMap& mapY,
+int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap& mapX, const CUtensorMap& mapY,
                    const float* dn, const float* dl, float* records, bool reverse, bool map, cudaStream_t st) {
-    if (sg.nseg <= 1) return LA_OK;
+    if (pl.npieces() <= 1) return LA_OK;
     static bool attr_done = false;
     if (!attr_done) {
         LA_CUDA_TRY(cudaFuncSetAttribute(segment_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSumSmemBytes));
@@ -216,11 +216,10 @@ int segment_states(const la_problem& p, const Segmentation& sg, const CUtensorMa
     prm.status = device_status_ptr();
     if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
     prm.N = p.N;
-    prm.chunks = (int)(p.N / kChunk);
-    prm.chunks_per_part = sg.chunks_per_part;
-    prm.parts = sg.parts();
-    prm.first_part = reverse ? sg.sub : 0;    // the open-end segment's own sums are never needed
-    prm.parts_per_seq = (sg.nseg - 1) * sg.sub;
+    prm.plan = pl;
+    // the sums of the piece at the open end of a sweep are never needed
+    prm.first_part = reverse ? pl.piece_first_part(1) : 0;
+    prm.parts_per_seq = reverse ? pl.nparts() - prm.first_part : pl.piece_first_part(pl.npieces() - 1);
     prm.eps = p.eps;
     prm.map = map ? 1 : 0;
     prm.dim = (int)p.D;
