@@ -459,13 +459,13 @@ CausalPlan choose_plan(const la_problem& p) {
     pl.nlong = nlong;
     // With B*H*nlong CTAs on 148 SMs, `rest` SMs would idle.  They take one short piece per sequence, several
     // in a row each (`rounds` at most): the short length m balances a long piece against `rounds` short ones,
-    // each CTA costing about five chunk times to start up and drain (measured: records summed, pipeline filled,
-    // last stores out).  The short piece sits in the middle of the sequence, so that the pre-passes (which skip
+    // each CTA costing about three chunk times to start up and drain (measured: records summed, pipeline
+    // filled, last stores out).  The short piece sits in the middle of the sequence, so that the pre-passes (which skip
     // the last piece forward, the first one backward) skip a long one.
     const int rest = kSms - pl.bh * nlong;
     if (!forced && nlong >= 2 && rest >= 8) {
         const int rounds = (pl.bh + rest - 1) / rest;
-        const double startup = 5.0;
+        const double startup = 3.0;
         int m = (int)(((double)pl.chunks / nlong - (rounds - 1) * startup) / (rounds + 1.0 / nlong));
         if (const char* e = getenv("LA_TC_SHORT")) m = atoi(e);        // A/B checks
         if (m >= 4 && (pl.chunks - m) / nlong >= 2) {

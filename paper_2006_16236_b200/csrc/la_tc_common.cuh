@@ -254,6 +254,45 @@ __device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int
     }
 }
 
+// Sum over the records of parts [part_lo, part_hi) of sixteen consecutive floats (at `offset` inside a
+// record), in part order, with the loads of four records in flight: a piece late in a sequence starts
+// from several records, and one round trip to L2 per record and column group would cost microseconds
+// on the critical start-up of its CTA.
+__device__ __forceinline__ void sum_records16(const float* rec, int part_lo, int part_hi, int offset, float (&acc)[16]) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+#pragma unroll 1
+    for (int p = part_lo; p < part_hi; p += 4) {
+        float4 a[4][4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const bool on = p + u < part_hi;
+            const float4* src = reinterpret_cast<const float4*>(rec + (int64_t)(on ? p + u : p) * kStateFloats + offset);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) a[u][j] = on ? __ldg(src + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc[4 * j] += a[u][j].x; acc[4 * j + 1] += a[u][j].y; acc[4 * j + 2] += a[u][j].z; acc[4 * j + 3] += a[u][j].w;
+            }
+    }
+}
+// The same for one float per record.
+__device__ __forceinline__ float sum_records1(const float* rec, int part_lo, int part_hi, int offset) {
+    float z = 0.f;
+#pragma unroll 1
+    for (int p = part_lo; p < part_hi; p += 4) {
+        float a[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a[u] = p + u < part_hi ? __ldg(rec + (int64_t)(p + u) * kStateFloats + offset) : 0.f;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) z += a[u];
+    }
+    return z;
+}
+
 // Initial state of a segment: the sum of the records of parts [part_lo, part_hi) of this
 // (batch, head) (none: zeros) goes into the TMEM state accumulator, its bf16 tile and z_out.
 __device__ __forceinline__ void state_init(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, float* z_out,
@@ -261,37 +300,23 @@ __device__ __forceinline__ void state_init(uint32_t tmem_state, int quad, int la
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
+#pragma unroll 1
+    for (int g = 0; g < 4; ++g) {
+        float acc[16];
+        sum_records16(rec, owner ? part_lo : 0, owner ? part_hi : 0, d_row * kDim + g * 16, acc);
+        uint32_t v[16];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        float acc[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-        if (owner)
-            for (int p = part_lo; p < part_hi; ++p) {
-                const float4* src = reinterpret_cast<const float4*>(rec + (int64_t)p * kStateFloats + d_row * kDim + h * 32);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float4 a = __ldg(src + j);
-                    acc[4 * j] += a.x; acc[4 * j + 1] += a.y; acc[4 * j + 2] += a.z; acc[4 * j + 3] += a.w;
-                }
-            }
-        uint32_t v[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j]);
-        sm100::tmem_st32(tmem_state + lane_base + h * 32, v);
+        for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(acc[j]);
+        sm100::tmem_st16(tmem_state + lane_base + g * 16, v);
         if (owner) {
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-                const uint32_t chunk = h * 4 + cc;
-                sts128(s_tile + d_row * 128 + ((chunk ^ (d_row & 7)) << 4),
+            for (int cc = 0; cc < 2; ++cc)
+                sts128(s_tile + d_row * 128 + (((2 * g + cc) ^ (d_row & 7)) << 4),
                        sm100::pack_bf16x2(acc[cc * 8 + 0], acc[cc * 8 + 1]), sm100::pack_bf16x2(acc[cc * 8 + 2], acc[cc * 8 + 3]),
                        sm100::pack_bf16x2(acc[cc * 8 + 4], acc[cc * 8 + 5]), sm100::pack_bf16x2(acc[cc * 8 + 6], acc[cc * 8 + 7]));
-            }
         }
     }
-    float z = 0.f;
-    if (owner)
-        for (int p = part_lo; p < part_hi; ++p) z += __ldg(rec + (int64_t)p * kStateFloats + kDim * kDim + d_row);
+    const float z = owner ? sum_records1(rec, part_lo, part_hi, kDim * kDim + d_row) : 0.f;
     uint32_t zz[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) zz[j] = __float_as_uint(z);
@@ -359,29 +384,23 @@ __device__ __forceinline__ void state_init_tiles(uint32_t tmem_state, int quad, 
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
+#pragma unroll 1
+    for (int g = 0; g < 4; ++g) {
+        float acc[16];
+        sum_records16(rec, owner ? part_lo : 0, owner ? part_hi : 0, d_row * kDim + g * 16, acc);
+        uint32_t v[16];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        float acc[32];
+        for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(acc[j]);
+        sm100::tmem_st16(tmem_state + lane_base + g * 16, v);
+        if (owner) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-        if (owner)
-            for (int p = part_lo; p < part_hi; ++p) {
-                const float4* src = reinterpret_cast<const float4*>(rec + (int64_t)p * kStateFloats + d_row * kDim + h * 32);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float4 a = __ldg(src + j);
-                    acc[4 * j] += a.x; acc[4 * j + 1] += a.y; acc[4 * j + 2] += a.z; acc[4 * j + 3] += a.w;
-                }
-            }
-        uint32_t v[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j]);
-        sm100::tmem_st32(tmem_state + lane_base + h * 32, v);
-        if (owner) state_row_store(s_tile, d_row, h, v);
+            for (int cc = 0; cc < 2; ++cc)
+                sts128(s_tile + d_row * 128 + (((2 * g + cc) ^ (d_row & 7)) << 4),
+                       sm100::pack_bf16x2(acc[cc * 8 + 0], acc[cc * 8 + 1]), sm100::pack_bf16x2(acc[cc * 8 + 2], acc[cc * 8 + 3]),
+                       sm100::pack_bf16x2(acc[cc * 8 + 4], acc[cc * 8 + 5]), sm100::pack_bf16x2(acc[cc * 8 + 6], acc[cc * 8 + 7]));
+        }
     }
-    float z = 0.f;
-    if (owner)
-        for (int p = part_lo; p < part_hi; ++p) z += __ldg(rec + (int64_t)p * kStateFloats + kDim * kDim + d_row);
+    const float z = owner ? sum_records1(rec, part_lo, part_hi, kDim * kDim + d_row) : 0.f;
     uint32_t zz[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) zz[j] = __float_as_uint(z);
@@ -473,17 +492,7 @@ __device__ __forceinline__ void rstate_init(uint32_t tmem_state, int quad, int l
 #pragma unroll 1
     for (int g = 0; g < 4; ++g) {
         float acc[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) acc[j] = 0.f;
-        if (owner)
-            for (int p = part_lo; p < part_hi; ++p) {
-                const float4* src = reinterpret_cast<const float4*>(rec + (int64_t)p * kStateFloats + d_row * kDim + g * 16);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float4 a = __ldg(src + j);
-                    acc[4 * j] += a.x; acc[4 * j + 1] += a.y; acc[4 * j + 2] += a.z; acc[4 * j + 3] += a.w;
-                }
-            }
+        sum_records16(rec, owner ? part_lo : 0, owner ? part_hi : 0, d_row * kDim + g * 16, acc);
         uint32_t v[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(acc[j]);
@@ -496,9 +505,7 @@ __device__ __forceinline__ void rstate_init(uint32_t tmem_state, int quad, int l
                        sm100::pack_bf16x2(acc[cc * 8 + 4], acc[cc * 8 + 5]), sm100::pack_bf16x2(acc[cc * 8 + 6], acc[cc * 8 + 7]));
         }
     }
-    float r = 0.f;
-    if (owner)
-        for (int p = part_lo; p < part_hi; ++p) r += __ldg(rec + (int64_t)p * kStateFloats + kDim * kDim + d_row);
+    const float r = owner ? sum_records1(rec, part_lo, part_hi, kDim * kDim + d_row) : 0.f;
     uint32_t rr[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) rr[j] = j == 0 ? __float_as_uint(r) : 0u;      // all of r in column 64
