@@ -66,7 +66,7 @@ __device__ __forceinline__ void elu_row_inplace(uint8_t* row, uint32_t r7, float
 // final read-out; warp 4: TMA; warp 5: MMA.
 // ===========================================================================
 constexpr int kLsThreads = 192;
-constexpr int kLsStages = 2;
+constexpr int kLsStages = 3;
 constexpr uint32_t kLsStageBytes = 4 * kTileBytes;                  // X, Y, W (rows of w_i), aux (dl_i in 16 columns)
 constexpr uint32_t kLsOffOnes = kLsStages * kLsStageBytes;
 constexpr uint32_t kLsOffBar = kLsOffOnes + 1024;
