@@ -195,6 +195,22 @@ const char* la_last_error(void);
  * flag; LA_OK otherwise.  The context stays usable either way. */
 int la_last_device_status(void* stream);
 
+/*
+ * How the tensor-core causal kernels cut the sequences of problem p (a diagnostic, no counterpart
+ * in the paper; host only, nothing is enqueued).  A sequence of N / 128 chunks is cut into pieces,
+ * one CTA of a main kernel each, launched in the order the function reports, so that B*H*pieces
+ * CTAs keep all SMs busy; every piece is cut into pre-pass parts whose sums give a piece its
+ * starting state.  Writes up to `capacity` 32-bit integers to `out` (host memory) and returns how
+ * many the full description has, or 0 when p does not run the tensor-core kernels, or a negative
+ * status:  out = { pieces, parts,
+ *                  piece_begin[0..pieces]  (chunk index; piece_begin[pieces] = N / 128),
+ *                  piece_first_part[0..pieces],
+ *                  part_begin[0..parts],
+ *                  launch_order[0..pieces-1]  (CTA b handles piece launch_order[b / (B*H)] of
+ *                                              sequence b % (B*H)) }.
+ */
+int la_causal_plan(const la_problem* p, int32_t* out, int capacity);
+
 /* Number of GPU kernels this library has enqueued in this process so far (all
  * threads, all entry points); a diagnostic for benchmarks. */
 long long la_kernel_launches(void);

@@ -25,7 +25,7 @@ EXPORTS = [
     "la_causal_forward",
     "la_causal_backward", "la_recurrent_step", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
-    "la_profile_kernel_name", "la_version",
+    "la_profile_kernel_name", "la_version", "la_causal_plan",
 ]
 
 
@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
         L.la_last_device_status.argtypes = [vp]
         L.la_version.restype = ctypes.c_char_p
         L.la_kernel_launches.restype = ctypes.c_longlong
+        L.la_causal_plan.argtypes = [pp, ctypes.POINTER(ctypes.c_int32), ctypes.c_int]
         L.la_profile_enable.argtypes = [ctypes.c_int]
         L.la_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int)]
         L.la_profile_kernel_name.argtypes = [ctypes.c_int]
@@ -145,6 +146,29 @@ def la_workspace_bytes(p: la_problem, op: int) -> int:
 
 def la_kernel_launches() -> int:
     return int(lib().la_kernel_launches())
+
+
+def la_causal_plan(p: la_problem):
+    """How the tensor-core causal kernels cut the sequences of p: a dict of plain lists, or None when p runs
+    the general kernels.  Host only."""
+    n = lib().la_causal_plan(ctypes.byref(p), None, 0)
+    if n < 0:
+        _check(n)
+    if n == 0:
+        return None
+    buf = (ctypes.c_int32 * n)()
+    got = lib().la_causal_plan(ctypes.byref(p), buf, n)
+    if got != n:
+        raise RuntimeError("la_causal_plan changed its size between two calls")
+    v = list(buf)
+    pieces, parts = v[0], v[1]
+    o = 2
+    out = {"pieces": pieces, "parts": parts}
+    out["piece_begin"] = v[o:o + pieces + 1]; o += pieces + 1
+    out["piece_first_part"] = v[o:o + pieces + 1]; o += pieces + 1
+    out["part_begin"] = v[o:o + parts + 1]; o += parts + 1
+    out["launch_order"] = v[o:o + pieces]
+    return out
 
 
 def la_profile_enable(on: bool) -> None:

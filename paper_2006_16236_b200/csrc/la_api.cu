@@ -181,6 +181,13 @@ size_t la_workspace_bytes(const la_problem* p, int32_t op) {
     return general_workspace_bytes(*p, op);
 }
 
+int la_causal_plan(const la_problem* p, int32_t* out, int capacity) {
+    if (int rc = check_problem(p, true)) return rc;
+    if (capacity < 0 || (capacity > 0 && !out)) return fail(LA_ERR_INVALID_ARG, "out is NULL or capacity is negative");
+    if (p->N == 0 || !tc_supported(*p, LA_OP_CAUSAL_FORWARD)) return 0;
+    return tc_causal_plan(*p, out, capacity);
+}
+
 int la_feature_map(const void* x, void* y, int64_t n, int32_t dtype, int32_t deriv, void* stream) {
     if (n < 0) return fail(LA_ERR_INVALID_ARG, "n must be >= 0");
     if (dtype != LA_F32 && dtype != LA_BF16) return fail(LA_ERR_INVALID_ARG, "dtype %d is not a la_dtype", dtype);

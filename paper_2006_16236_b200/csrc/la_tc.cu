@@ -51,6 +51,22 @@ size_t tc_workspace_bytes(const la_problem& p, int op) {
 }
 
 size_t tc_causal_saved_bytes(const la_problem& p) { return tc::causal_saved_bytes(p); }
+int tc_causal_plan(const la_problem& p, int32_t* out, int capacity) {
+    const tc::CausalPlan pl = tc::choose_plan(p);
+    const int np = pl.npieces(), nq = pl.nparts();
+    int n = 0;
+    auto put = [&](int v) {
+        if (out && n < capacity) out[n] = v;
+        ++n;
+    };
+    put(np);
+    put(nq);
+    for (int k = 0; k <= np; ++k) put(pl.piece_begin(k));
+    for (int k = 0; k <= np; ++k) put(pl.piece_first_part(k));
+    for (int q = 0; q <= nq; ++q) put(pl.part_begin(q));
+    for (int s = 0; s < np; ++s) put(pl.piece_of_slot(s));
+    return n;
+}
 int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
                       float* S_out, float* Z_out, void* saved, void* ws, cudaStream_t st) {
     return tc::causal_forward(p, Q, K, V, O, den, S_out, Z_out, saved, ws, st);

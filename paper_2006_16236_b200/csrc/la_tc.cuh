@@ -9,6 +9,8 @@ bool tc_supported(const la_problem& p, int op);
 size_t tc_workspace_bytes(const la_problem& p, int op);
 
 size_t tc_causal_saved_bytes(const la_problem& p);
+// pieces, parts, piece_begin[], piece_first_part[], part_begin[], launch_order[] (see la_causal_plan)
+int tc_causal_plan(const la_problem& p, int32_t* out, int capacity);
 int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
                       float* den, float* S_out, float* Z_out, void* saved, void* ws, cudaStream_t st);
 int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* O,

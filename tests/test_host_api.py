@@ -55,6 +55,45 @@ def _p(**kw):
     return la.make_problem(**base)
 
 
+@pytest.mark.parametrize("bh", [1, 2, 3, 5, 8, 16, 32, 48, 50, 64, 70, 74, 75, 100, 119, 120, 128, 148, 256])
+@pytest.mark.parametrize("chunks", [1, 2, 3, 4, 8, 17, 64, 100, 128, 256, 1024])
+def test_causal_plan_tiles_every_sequence(L, bh, chunks):
+    """Pieces and pre-pass parts of the tensor-core causal kernels: both tile [0, N / 128) in order, a
+    piece starts on a part boundary, every piece is launched exactly once, and the parts a pre-pass
+    computes (all before the last piece, all after the first) are the ones a piece's start needs."""
+    p = la.make_problem(bh, 1, chunks * 128, 64, 64, la.LA_BF16)
+    plan = la.la_causal_plan(p)
+    assert plan is not None
+    n, q = plan["pieces"], plan["parts"]
+    pb, fp, qb = plan["piece_begin"], plan["piece_first_part"], plan["part_begin"]
+    assert n >= 1 and q >= n
+    assert pb[0] == 0 and pb[n] == chunks and qb[0] == 0 and qb[q] == chunks
+    assert all(pb[k] < pb[k + 1] for k in range(n)) and all(qb[j] < qb[j + 1] for j in range(q))
+    assert fp[0] == 0 and fp[n] == q and all(fp[k] < fp[k + 1] for k in range(n))
+    assert all(qb[fp[k]] == pb[k] for k in range(n + 1))
+    if n > 1:
+        assert min(pb[k + 1] - pb[k] for k in range(n)) >= 2          # a piece is at least two chunks
+    assert sorted(plan["launch_order"]) == list(range(n))
+    # long pieces are launched before a shorter one, so that the left-over SMs take the short pieces last
+    lens = [pb[k + 1] - pb[k] for k in plan["launch_order"]]
+    assert all(lens[i] + 1 >= lens[i + 1] for i in range(n - 1))
+    # work per SM: no more CTAs of the long kind than SMs
+    nlong = sum(1 for x in lens if x + 1 >= lens[0])
+    assert bh * nlong <= 148 or n == 1 or nlong == 1 or os.environ.get("LA_TC_NSEG")
+
+
+def test_causal_plan_of_the_bench_workload(L):
+    # B*H = 64, 128 chunks: two long pieces around one short middle piece, 192 CTAs for 148 SMs
+    plan = la.la_causal_plan(la.make_problem(8, 8, 16384, 64, 64, la.LA_BF16))
+    assert plan["pieces"] == 3 and plan["launch_order"] == [0, 2, 1]
+    pb = plan["piece_begin"]
+    short = pb[2] - pb[1]
+    assert 8 <= short <= 16 and abs((pb[1] - pb[0]) - (pb[3] - pb[2])) <= 1
+    # problems that run the general kernels have no plan
+    assert la.la_causal_plan(la.make_problem(1, 2, 256, 32, 32, la.LA_F32)) is None
+    assert la.la_causal_plan(la.make_problem(1, 2, 200, 64, 64, la.LA_BF16)) is None
+
+
 def test_bad_arguments_are_rejected_on_the_host(L):
     buf = ctypes.create_string_buffer(64)
     ok = ctypes.c_void_p((ctypes.addressof(buf) + 15) & ~15)
