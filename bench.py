@@ -239,12 +239,16 @@ def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True):
     for _ in range(warmup):
         s.step()
     torch.cuda.synchronize()
+    # Timed region: K plain steps.  The per-kernel durations (roofline, breakdown) come from a second pass
+    # of K steps right after it with the library's event pairs around every kernel and an event between
+    # forward and backward: those records cost about 7 % of a step, so they stay out of the timed region.
     launches0 = la.la_kernel_launches()
-    la.la_profile_enable(True)
     t_lo = time.time()
-    total_ms, (fwd_ms, bwd_ms) = time_steps(None, steps, 0, world, split=(s.fwd, s.bwd))
-    t_hi = time.time()
+    total_ms, _ = time_steps(s.step, steps, 0, world)
     launches = la.la_kernel_launches() - launches0
+    la.la_profile_enable(True)
+    _, (fwd_ms, bwd_ms) = time_steps(None, steps, 0, world, split=(s.fwd, s.bwd))
+    t_hi = time.time()
     kernels = la.la_profile_read()
     la.la_profile_enable(False)
     windows = [(t_lo, t_hi)]
@@ -262,17 +266,21 @@ def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True):
     res = {
         "value": tokens / (ms * 1e-3), "ms_per_step": ms, "fwd_ms": fwd_ms, "bwd_ms": bwd_ms,
         "gpu_launches": int(launches), "clocks": clocks,
-        "alg_gbs": algorithmic_bytes(w, "both") / (fwd_ms + bwd_ms) * 1e-6,
-        "alg_tflops": algorithmic_flops(w, "both") / (fwd_ms + bwd_ms) * 1e-9,
+        "alg_gbs": algorithmic_bytes(w, "both") / ms * 1e-6,
+        "alg_tflops": algorithmic_flops(w, "both") / ms * 1e-9,
         "kernels_ms": {k: {"ms_per_launch": v[0], "launches": v[1]} for k, v in kernels.items()},
     }
     res["hbm_frac"] = res["alg_gbs"] / pk["hbm_gbs"]
     res["tensor_frac_alg_flops"] = res["alg_tflops"] / pk["bf16_tflops_sustained"]
     # dominant kernel: the one with the largest total time among those with a defined byte count
     th = w.B * w.H * w.N
+    # (kernels within 2 % of the largest total time count as tied: run-to-run noise would otherwise pick
+    # between them; the tie goes to the one that moves the most algorithmic bytes)
     ranked = [(v[0] * v[1], k, v[0]) for k, v in kernels.items() if KERNEL_ALG_BYTES.get(k)]
     if ranked:
-        _, dom, dom_ms = max(ranked)
+        top = max(r[0] for r in ranked)
+        tied = [r for r in ranked if r[0] >= 0.98 * top]
+        _, dom, dom_ms = max(tied, key=lambda r: KERNEL_ALG_BYTES[r[1]](w.D, elem_bytes(w)))
         dom_bytes = KERNEL_ALG_BYTES[dom](w.D, elem_bytes(w)) * th
     else:                       # general kernels: one kernel per call
         dom = ("la_causal_" if w.kind == "causal" else "la_linear_attention_") + ("backward" if bwd_ms >= fwd_ms else "forward")
@@ -419,7 +427,9 @@ def workload_config(w, world):
     return {"workload": w.name, "mirrors": w.mirrors, "B_per_gpu": w.B, "H": w.H, "N": w.N, "D": w.D, "M": w.M,
             "io_dtype": w.dtype, "phi": "elu+1", "eps": 0.0, "seed": w.seed,
             "parallelism": f"{world} independent shard(s) of (batch, head) pairs, no collective",
-            "l2": "per-step working set (inputs+outputs >= 1 GiB at the default workload) exceeds the 126 MB L2; no flush needed"}
+            "l2": "per-step working set (inputs+outputs >= 1 GiB at the default workload) exceeds the 126 MB L2; no flush needed",
+            "timing": "value: K plain steps between two CUDA events; roofline and breakdown: a second pass of K steps "
+                      "with an event pair around every kernel (the records cost about 7 % of a step)"}
 
 
 def main():
