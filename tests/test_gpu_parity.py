@@ -81,6 +81,41 @@ def test_noncausal_forward_backward(shape, dtype):
     la.la_last_device_status()
 
 
+@pytest.mark.parametrize("plan", [{"LA_TC_NSEG": "1"}, {"LA_TC_NSEG": "3"}, {"LA_TC_NSEG": "5"}, {"LA_TC_SHORT": "0"},
+                                  {"LA_TC_SHORT": "4"}, {"LA_TC_SHORT": "7"}],
+                         ids=lambda d: ",".join(f"{k[6:].lower()}={v}" for k, v in d.items()))
+@pytest.mark.parametrize("keep", [False, True], ids=["recompute", "saved"])
+def test_causal_results_do_not_depend_on_the_piece_plan(monkeypatch, plan, keep):
+    """The cut of a sequence into pieces and pre-pass parts (ragged lengths, a short middle piece, one piece)
+    is an implementation choice: every plan has to give the oracle's result.  B*H = 64, 18 chunks."""
+    for k, v in plan.items():
+        monkeypatch.setenv(k, v)
+    B, H, N, D = 4, 16, 18 * 128, 64
+    p = la.make_problem(B, H, N, D, D, la.LA_BF16)
+    pl = la.la_causal_plan(p)
+    if "LA_TC_NSEG" in plan:
+        assert pl["pieces"] == int(plan["LA_TC_NSEG"])
+    else:
+        short = int(plan["LA_TC_SHORT"])
+        assert pl["pieces"] == (3 if short >= 4 else 2)
+        if short >= 4:
+            assert pl["piece_begin"][2] - pl["piece_begin"][1] == short
+    Q, K, V, G = draw_qkvg(B, H, N, D, D, seed=77, dtype=torch.bfloat16)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    saved = la.saved_buffer(Qd, Vd) if keep else None
+    O = la.la_causal_forward(Qd, Kd, Vd, saved=saved)
+    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd, saved=saved)
+    la.la_last_device_status()
+    for b, h in ((0, 0), (1, 7), (3, 15)):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        q, k, v, g = Q[sl], K[sl], V[sl], G[sl]
+        assert_close(O[sl], oracle.linear_attention(q, k, v, True)[0], torch.bfloat16, f"O[{b},{h}]")
+        rq, rk, rv = oracle.linear_attention_backward(q, k, v, g, True)
+        assert_close(dQ[sl], rq, torch.bfloat16, f"dQ[{b},{h}]", grad=True)
+        assert_close(dK[sl], rk, torch.bfloat16, f"dK[{b},{h}]", grad=True)
+        assert_close(dV[sl], rv, torch.bfloat16, f"dV[{b},{h}]", grad=True)
+
+
 @pytest.mark.parametrize("causal", [True, False])
 @pytest.mark.parametrize("dtype", DTYPES)
 def test_eps_and_identity_feature_map(causal, dtype):
