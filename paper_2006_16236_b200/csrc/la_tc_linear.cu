@@ -122,6 +122,12 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     }
     if (tid < 128)
         for (int i = tid; i < 256; i += 128) reinterpret_cast<uint32_t*>(smem + kLsOffOnes)[i] = 0x3F803F80u;
+    // The aux tile of a stage is the second 64-column block of the B operand [Y | aux] (N = 80: its first 16
+    // columns are read).  Without per-position weights it is constant ones: written once here.
+    if (!reverse)
+        for (int s = 0; s < kLsStages; ++s)
+            for (int i = tid; i < kTileBytes / 4; i += kLsThreads)
+                reinterpret_cast<uint32_t*>(smem + s * kLsStageBytes + 3 * kTileBytes)[i] = 0x3F803F80u;
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
@@ -149,8 +155,9 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         }
     } else if (warp == 5) {
         if (lane == 0) {
-            const uint32_t idesc_s = umma_idesc_bf16(64, 64, 1, 1);
-            const uint32_t idesc_z = umma_idesc_bf16(64, 16, 1, 1);
+            // one M = 64, N = 80 product per K group and accumulator: B = [Y | aux], the aux tile (two tiles
+            // further on in the stage) being the second 64-column block through the leading-offset field
+            const uint32_t idesc = umma_idesc_bf16(64, 80, 1, 1);
             const uint32_t aOnes = sbase + kLsOffOnes;
             bool ok = true;
             #pragma unroll 1
@@ -161,15 +168,13 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 if (!ok || *abort_flag) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t acc = (c != 0);
+#pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const uint32_t a = acc | (k != 0);
-                    const uint64_t dX = desc_mn(aX + k * 2048), dY = desc_mn(aY + k * 2048);
+                    const uint64_t dX = desc_mn(aX + k * 2048), dYA = desc_mn(aY + k * 2048, aA - aY);
                     const uint64_t dW = reverse ? desc_mn(aW + k * 2048) : desc_ones(aOnes);
-                    const uint64_t dA = reverse ? desc_mn(aA + k * 2048) : desc_ones(aOnes);
-                    umma_bf16(tmem, dX, dY, idesc_s, a);                 // A' += x'^T Y
-                    umma_bf16(tmem + 64, dX, dA, idesc_z, a);            // a' += x'^T aux
-                    umma_bf16(tmem + 128, dW, dY, idesc_s, a);           // ysum += w^T Y (all 64 rows alike)
-                    if (reverse) umma_bf16(tmem + 192, dW, dA, idesc_z, a);   // w0 += w^T aux
+                    umma_bf16(tmem, dX, dYA, idesc, a);                  // [A' | a'] += x'^T [Y | aux]
+                    umma_bf16(tmem + 128, dW, dYA, idesc, a);            // [ysum | w0] += w^T [Y | aux] (all 64 rows alike)
                 }
                 umma_commit(&bars->empty[s]);
             }
