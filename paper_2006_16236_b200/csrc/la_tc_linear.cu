@@ -260,7 +260,8 @@ constexpr uint32_t kApOffStage = 0;                                   // kApStag
 constexpr uint32_t kApOffState = kApOffStage + kApStages * 2 * kTileBytes;   // bf16 centred state tile [64][64]
 constexpr uint32_t kApOffVec = kApOffState + kDim * 128;              // fp32 [3][64]: a' (Z' or r'), nu, scratch
 constexpr uint32_t kApOffBar = kApOffVec + 1024;
-constexpr uint32_t kApSmemBytes = kApOffBar + 256 + 1024;
+constexpr uint32_t kApOffOut = (kApOffBar + 256 + 1023) & ~1023u;      // two result tiles on their way out
+constexpr uint32_t kApSmemBytes = kApOffOut + 2 * kTileBytes + 1024;   // + slack for the 1 KB alignment of the base
 
 struct ApBarriers {
     uint64_t full[kApStages], empty[kApStages], mapped[kApStages];
@@ -288,6 +289,7 @@ struct ApParams {
 template <int kMode>
 __global__ void __launch_bounds__(kApThreads, 1)
 linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
+                    const __grid_constant__ CUtensorMap mapOut0, const __grid_constant__ CUtensorMap mapOut1,
                     const ApParams prm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -495,7 +497,12 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             tmem_ld32(tmem + lane_base + b * 128, a0);
             tmem_ld32(tmem + lane_base + b * 128 + 32, a1);
             tmem_ld_wait();
-            __nv_bfloat16* dst = prm.out0 + row * prm.dim;
+            // Results leave through a staging tile: each warp fills the 4 KB slab of its 32 rows and one of its
+            // lanes stores it with TMA (full 128-byte rows per request; columns beyond a 32-wide problem are
+            // clipped by the store).  The previous chunk's store must have read the slab before it is rewritten.
+            uint8_t* out_row = smem + kApOffOut + t * 128;
+            if (lane == 0) tma_store_wait_read<0>();
+            __syncwarp();
             if (kMode == kApplyForward) {
                 // den = (1 + q') . (N 1 + Z');  num = (1 + q').1 nu + q' S''
                 const float den = fN * x1sum + sScal[0] + xa;
@@ -509,7 +516,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                         if (hh >= nhalf) break;
                         const uint32_t* acc = hh ? a1 : a0;
                         const float* nu = sNu + hh * 32 + cc * 8;
-                        stg128(dst + hh * 32 + cc * 8,
+                        sts128(out_row + (((hh * 4 + cc) ^ r7) << 4),
                                pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 0]), inv, w * nu[0]), fmaf(__uint_as_float(acc[cc * 8 + 1]), inv, w * nu[1])),
                                pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 2]), inv, w * nu[2]), fmaf(__uint_as_float(acc[cc * 8 + 3]), inv, w * nu[3])),
                                pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 4]), inv, w * nu[4]), fmaf(__uint_as_float(acc[cc * 8 + 5]), inv, w * nu[5])),
@@ -565,13 +572,12 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                             }
                             outp[j] = pack_bf16x2(g0, g1);
                         }
-                        stg128(dst + hh * 32 + cc * 8, outp[0], outp[1], outp[2], outp[3]);
+                        sts128(out_row + (((hh * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
                     }
                 if (kMode == kApplyBackwardKV) {
                     tmem_ld32(tmem + lane_base + b * 128 + 64, a0);
                     tmem_ld32(tmem + lane_base + b * 128 + 96, a1);
                     tmem_ld_wait();
-                    __nv_bfloat16* dstV = prm.out1 + row * prm.dim;
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
@@ -579,7 +585,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                             if (hh >= nhalf) break;
                             const uint32_t* acc = hh ? a1 : a0;
                             const float* nu = sNu + hh * 32 + cc * 8;
-                            stg128(dstV + hh * 32 + cc * 8,
+                            sts128(out_row + kTileBytes + (((hh * 4 + cc) ^ r7) << 4),
                                    pack_bf16x2(fmaf(x1sum, nu[0], __uint_as_float(acc[cc * 8 + 0])), fmaf(x1sum, nu[1], __uint_as_float(acc[cc * 8 + 1]))),
                                    pack_bf16x2(fmaf(x1sum, nu[2], __uint_as_float(acc[cc * 8 + 2])), fmaf(x1sum, nu[3], __uint_as_float(acc[cc * 8 + 3]))),
                                    pack_bf16x2(fmaf(x1sum, nu[4], __uint_as_float(acc[cc * 8 + 4])), fmaf(x1sum, nu[5], __uint_as_float(acc[cc * 8 + 5]))),
@@ -589,7 +595,16 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             }
             tc_fence_before_sync();
             mbar_arrive(&bars->acc_free[b]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                const int y = (int)(row0 + (int64_t)c * kChunk + warp * 32);
+                tma_store_2d(&mapOut0, smem + kApOffOut + warp * 32 * 128, 0, y);
+                if (kMode == kApplyBackwardKV) tma_store_2d(&mapOut1, smem + kApOffOut + kTileBytes + warp * 32 * 128, 0, y);
+                tma_store_commit();
+            }
         }
+        if (lane == 0) tma_store_wait_all<0>();
     }
 
     tc_fence_before_sync();
@@ -658,8 +673,12 @@ int launch_apply(const la_problem& p, const Segmentation& sg, const CUtensorMap&
     prm.eps = p.eps;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
+    const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
+    CUtensorMap mO0, mO1;                   // one warp's 32 rows per store
+    if (int rc = encode_tile_map(&mO0, prm.out0, rows, 32, (int)p.D)) return rc;
+    if (int rc = encode_tile_map(&mO1, prm.out1 ? prm.out1 : prm.out0, rows, 32, (int)p.D)) return rc;
     prof_begin(kProfLinearApply, st);
-    linear_apply_kernel<kMode><<<(unsigned)(sg.nseg * p.B * p.H), kApThreads, kApSmemBytes, st>>>(mX, mY, prm);
+    linear_apply_kernel<kMode><<<(unsigned)(sg.nseg * p.B * p.H), kApThreads, kApSmemBytes, st>>>(mX, mY, mO0, mO1, prm);
     LA_LAUNCHED();
     prof_end(kProfLinearApply, st);
     return LA_OK;
