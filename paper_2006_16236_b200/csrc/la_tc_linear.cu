@@ -255,13 +255,14 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 enum ApplyMode { kApplyForward = 0, kApplyBackwardQ = 1, kApplyBackwardKV = 2 };
 
 constexpr int kApStages = 3;
-constexpr int kApThreads = 320;
+constexpr int kApThreads = 448;
 constexpr uint32_t kApOffStage = 0;                                   // kApStages x {X, Y}
 constexpr uint32_t kApOffState = kApOffStage + kApStages * 2 * kTileBytes;   // bf16 centred state tile [64][64]
 constexpr uint32_t kApOffVec = kApOffState + kDim * 128;              // fp32 [3][64]: a' (Z' or r'), nu, scratch
 constexpr uint32_t kApOffBar = kApOffVec + 1024;
 constexpr uint32_t kApOffOut = (kApOffBar + 256 + 1023) & ~1023u;      // two result tiles on their way out
-constexpr uint32_t kApSmemBytes = kApOffOut + 2 * kTileBytes + 1024;   // + slack for the 1 KB alignment of the base
+constexpr uint32_t kApOffX = kApOffOut + 2 * kTileBytes;               // fp32 [2 halves][128 rows][8]: partial sums exchanged
+constexpr uint32_t kApSmemBytes = kApOffX + 2 * 128 * 8 * 4 + 1024;    // + slack for the 1 KB alignment of the base
 
 struct ApBarriers {
     uint64_t full[kApStages], empty[kApStages], mapped[kApStages];
@@ -311,12 +312,12 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     if (tid == 0) {
         for (int s = 0; s < kApStages; ++s) {
             mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], 1 + 128);      // MMA commit + epilogue threads (they read the X and Y rows)
+            mbar_init(&bars->empty[s], 1 + 256);      // MMA commit + epilogue threads (they read the X and Y rows)
             mbar_init(&bars->mapped[s], 128);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&bars->acc_full[b], 1);
-            mbar_init(&bars->acc_free[b], 128);
+            mbar_init(&bars->acc_free[b], 256);
         }
         bars->abort_flag = 0;
         fence_mbar_init();
@@ -436,7 +437,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             }
             if (!ok) *abort_flag = 1;
         }
-    } else if (warp >= 4) {
+    } else if (warp >= 4 && warp < 8) {
         const int t = tid - 128;
         const uint32_t r7 = t & 7;
         const bool elu = prm.phi == LA_PHI_ELU1;
@@ -451,95 +452,109 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             mbar_arrive(&bars->mapped[s]);
         }
     } else {
-        const int t = tid;
+        // Epilogue: two warps per TMEM quadrant (warps 0-3: columns 0..31 of a row, warps 10-13: columns 32..63;
+        // one thread per row and half).  The sums that run over a whole row (x'.1, x'.a', Y.nu, 1.h'', q'.h'') are
+        // formed per half and exchanged through shared memory inside the pair.
+        const int hf = warp >= 10 ? 1 : 0;
+        const int quad = warp & 3;
+        const int t = quad * 32 + lane;
         const uint32_t r7 = t & 7;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const bool elu = prm.phi == LA_PHI_ELU1;
         const float fD = (float)prm.dim, fN = (float)prm.N;
-        const int nhalf = prm.dim >> 5;             // 32-column halves that hold real columns
+        // (columns beyond a 32-wide problem are zero padding: they add nothing to the sums, and the store clips them)
+        float* sX = reinterpret_cast<float*>(smem + kApOffX);
+        float* mine = sX + (hf * 128 + t) * 8;
+        const float* other = sX + ((hf ^ 1) * 128 + t) * 8;
+        const float* aH = sA + hf * 32;
+        const float* nuH = sNu + hf * 32;
         #pragma unroll 1
         for (int c = 0; c < L; ++c) {
             const int s = c % kApStages, b = c & 1;
             const int64_t row = row0 + (int64_t)c * kChunk + t;
             if (!mbar_wait(&bars->mapped[s], (c / kApStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
-            uint32_t xv[8][4];                       // x' = elu(X) row
-            load_row(smem + kApOffStage + s * 2 * kTileBytes + t * 128, r7, xv);
-            float ynu = 0.f;                         // Y_i . nu (backward)
+            uint32_t xv[4][4];                       // this half of the x' = elu(X) row
+            const uint8_t* rowX = smem + kApOffStage + s * 2 * kTileBytes + t * 128;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) lds128(rowX + (((hf * 4 + cc) ^ r7) << 4), xv[cc]);
+            float ynu_h = 0.f;                       // this half of Y_i . nu (backward)
             if (kHasY) {
-                uint32_t yv[8][4];
-                load_row(smem + kApOffStage + s * 2 * kTileBytes + kTileBytes + t * 128, r7, yv);
+                uint32_t yv[4][4];
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) lds128(rowX + kTileBytes + (((hf * 4 + cc) ^ r7) << 4), yv[cc]);
                 float p4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int cc = 0; cc < 8; ++cc)
+                for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        p4[j] = fmaf(bf16_lo(yv[cc][j]), sNu[cc * 8 + 2 * j], fmaf(bf16_hi(yv[cc][j]), sNu[cc * 8 + 2 * j + 1], p4[j]));
-                ynu = (p4[0] + p4[1]) + (p4[2] + p4[3]);
+                        p4[j] = fmaf(bf16_lo(yv[cc][j]), nuH[cc * 8 + 2 * j], fmaf(bf16_hi(yv[cc][j]), nuH[cc * 8 + 2 * j + 1], p4[j]));
+                ynu_h = (p4[0] + p4[1]) + (p4[2] + p4[3]);
             }
             mbar_arrive(&bars->empty[s]);
-            // sx = sum_d x'_d  and  xa = x' . a'
             float sx4[4] = {0.f, 0.f, 0.f, 0.f}, xa4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int cc = 0; cc < 8; ++cc)
+            for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float x0 = bf16_lo(xv[cc][j]), x1 = bf16_hi(xv[cc][j]);
                     sx4[j] += x0 + x1;
-                    xa4[j] = fmaf(x0, sA[cc * 8 + 2 * j], fmaf(x1, sA[cc * 8 + 2 * j + 1], xa4[j]));
+                    xa4[j] = fmaf(x0, aH[cc * 8 + 2 * j], fmaf(x1, aH[cc * 8 + 2 * j + 1], xa4[j]));
                 }
-            const float sx = (sx4[0] + sx4[1]) + (sx4[2] + sx4[3]);
-            const float xa = (xa4[0] + xa4[1]) + (xa4[2] + xa4[3]);
-            const float x1sum = fD + sx;             // (1 + x') . 1
             if (!mbar_wait(&bars->acc_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
-            uint32_t a0[32], a1[32];
-            tmem_ld32(tmem + lane_base + b * 128, a0);
-            tmem_ld32(tmem + lane_base + b * 128 + 32, a1);
+            uint32_t acc[32];
+            tmem_ld32(tmem + lane_base + b * 128 + hf * 32, acc);
             tmem_ld_wait();
-            // Results leave through a staging tile: each warp fills the 4 KB slab of its 32 rows and one of its
-            // lanes stores it with TMA (full 128-byte rows per request; columns beyond a 32-wide problem are
-            // clipped by the store).  The previous chunk's store must have read the slab before it is rewritten.
+            float sh_h = 0.f, qh_h = 0.f;
+            if (kMode == kApplyBackwardQ) {
+                float sh4[4] = {0.f, 0.f, 0.f, 0.f}, qh4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float h0 = __uint_as_float(acc[cc * 8 + 2 * j]), h1 = __uint_as_float(acc[cc * 8 + 2 * j + 1]);
+                        sh4[j] += h0 + h1;
+                        qh4[j] = fmaf(bf16_lo(xv[cc][j]), h0, fmaf(bf16_hi(xv[cc][j]), h1, qh4[j]));
+                    }
+                sh_h = (sh4[0] + sh4[1]) + (sh4[2] + sh4[3]);
+                qh_h = (qh4[0] + qh4[1]) + (qh4[2] + qh4[3]);
+            }
+            // the pair's previous slab must have left the staging tile before either warp rewrites it below
+            if (hf == 0 && lane == 0) tma_store_wait_read<0>();
+            mine[0] = (sx4[0] + sx4[1]) + (sx4[2] + sx4[3]);
+            mine[1] = (xa4[0] + xa4[1]) + (xa4[2] + xa4[3]);
+            mine[2] = ynu_h;
+            mine[3] = sh_h;
+            mine[4] = qh_h;
+            named_barrier(2 + quad, 64);
+            // both threads of a row add the halves in the same order (half 0 first): identical totals
+            const float* lo = hf ? other : mine;
+            const float* hi = hf ? mine : other;
+            const float sx = lo[0] + hi[0], xa = lo[1] + hi[1], ynu = lo[2] + hi[2], sh = lo[3] + hi[3], qh = lo[4] + hi[4];
+            named_barrier(2 + quad, 64);            // the exchange slots may be rewritten after this
+            const float x1sum = fD + sx;             // (1 + x') . 1
             uint8_t* out_row = smem + kApOffOut + t * 128;
-            if (lane == 0) tma_store_wait_read<0>();
-            __syncwarp();
             if (kMode == kApplyForward) {
                 // den = (1 + q') . (N 1 + Z');  num = (1 + q').1 nu + q' S''
                 const float den = fN * x1sum + sScal[0] + xa;
                 const float inv = 1.f / (den + prm.eps);
                 const float w = x1sum * inv;
-                if (prm.den) prm.den[row] = den;
+                if (hf == 0 && prm.den) prm.den[row] = den;
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        if (hh >= nhalf) break;
-                        const uint32_t* acc = hh ? a1 : a0;
-                        const float* nu = sNu + hh * 32 + cc * 8;
-                        sts128(out_row + (((hh * 4 + cc) ^ r7) << 4),
-                               pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 0]), inv, w * nu[0]), fmaf(__uint_as_float(acc[cc * 8 + 1]), inv, w * nu[1])),
-                               pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 2]), inv, w * nu[2]), fmaf(__uint_as_float(acc[cc * 8 + 3]), inv, w * nu[3])),
-                               pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 4]), inv, w * nu[4]), fmaf(__uint_as_float(acc[cc * 8 + 5]), inv, w * nu[5])),
-                               pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 6]), inv, w * nu[6]), fmaf(__uint_as_float(acc[cc * 8 + 7]), inv, w * nu[7])));
-                    }
+                for (int cc = 0; cc < 4; ++cc) {
+                    const float* nu = nuH + cc * 8;
+                    sts128(out_row + (((hf * 4 + cc) ^ r7) << 4),
+                           pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 0]), inv, w * nu[0]), fmaf(__uint_as_float(acc[cc * 8 + 1]), inv, w * nu[1])),
+                           pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 2]), inv, w * nu[2]), fmaf(__uint_as_float(acc[cc * 8 + 3]), inv, w * nu[3])),
+                           pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 4]), inv, w * nu[4]), fmaf(__uint_as_float(acc[cc * 8 + 5]), inv, w * nu[5])),
+                           pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 6]), inv, w * nu[6]), fmaf(__uint_as_float(acc[cc * 8 + 7]), inv, w * nu[7])));
+                }
             } else {
                 // backward Q:  h = (G.nu) 1 + h'',  Z = N 1 + Z',  gq = (h - (q.h / dn) Z) / dn
                 // backward KV: gk = (V.nu_R + w0) 1 + V R''^T + r'
                 float c1 = 0.f, cz = 0.f, scale = 1.f;          // out_d = scale * (acc_d + c1 + cz * a'_d)
                 if (kMode == kApplyBackwardQ) {
-                    float sh4[4] = {0.f, 0.f, 0.f, 0.f}, qh4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                    for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float h0 = __uint_as_float(a0[cc * 8 + 2 * j]), h1 = __uint_as_float(a0[cc * 8 + 2 * j + 1]);
-                            const float h2 = __uint_as_float(a1[cc * 8 + 2 * j]), h3 = __uint_as_float(a1[cc * 8 + 2 * j + 1]);
-                            sh4[j] += (h0 + h1) + (h2 + h3);
-                            qh4[j] = fmaf(bf16_lo(xv[cc][j]), h0, fmaf(bf16_hi(xv[cc][j]), h1, qh4[j]));
-                            qh4[j] = fmaf(bf16_lo(xv[cc + 4][j]), h2, fmaf(bf16_hi(xv[cc + 4][j]), h3, qh4[j]));
-                        }
-                    const float sh = (sh4[0] + sh4[1]) + (sh4[2] + sh4[3]);       // 1 . h''
-                    const float qh = (qh4[0] + qh4[1]) + (qh4[2] + qh4[3]);       // q' . h''
                     const float den = fN * x1sum + sScal[0] + xa;
                     const float dn = den + prm.eps;
                     scale = 1.f / dn;
@@ -547,64 +562,57 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     const float dl = -q_h * scale;                                // dl_i = -(G_i . O_i)
                     c1 = fmaf(dl, fN, ynu);                                       // (G.nu) + dl N
                     cz = dl;
-                    prm.den[row] = dn;
-                    prm.dl[row] = dl;
+                    if (hf == 0) {
+                        prm.den[row] = dn;
+                        prm.dl[row] = dl;
+                    }
                 } else {
                     c1 = ynu + sScal[1];
                     cz = 1.f;
                 }
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh)
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint32_t outp[4];
 #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        if (hh >= nhalf) break;
-                        uint32_t outp[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int e = cc * 8 + 2 * j, d = hh * 32 + e;
-                            const uint32_t* acc = hh ? a1 : a0;
-                            float g0 = scale * (fmaf(cz, sA[d], __uint_as_float(acc[e])) + c1);
-                            float g1 = scale * (fmaf(cz, sA[d + 1], __uint_as_float(acc[e + 1])) + c1);
-                            if (elu) {          // phi'(x) from x' = elu(x): 1 where x' > 0, else 1 + x'
-                                const float x0 = bf16_lo(xv[hh * 4 + cc][j]), x1 = bf16_hi(xv[hh * 4 + cc][j]);
-                                g0 *= x0 > 0.f ? 1.f : 1.f + x0;
-                                g1 *= x1 > 0.f ? 1.f : 1.f + x1;
-                            }
-                            outp[j] = pack_bf16x2(g0, g1);
+                    for (int j = 0; j < 4; ++j) {
+                        const int e = cc * 8 + 2 * j;
+                        float g0 = scale * (fmaf(cz, aH[e], __uint_as_float(acc[e])) + c1);
+                        float g1 = scale * (fmaf(cz, aH[e + 1], __uint_as_float(acc[e + 1])) + c1);
+                        if (elu) {          // phi'(x) from x' = elu(x): 1 where x' > 0, else 1 + x'
+                            const float x0 = bf16_lo(xv[cc][j]), x1 = bf16_hi(xv[cc][j]);
+                            g0 *= x0 > 0.f ? 1.f : 1.f + x0;
+                            g1 *= x1 > 0.f ? 1.f : 1.f + x1;
                         }
-                        sts128(out_row + (((hh * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
+                        outp[j] = pack_bf16x2(g0, g1);
                     }
+                    sts128(out_row + (((hf * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
+                }
                 if (kMode == kApplyBackwardKV) {
-                    tmem_ld32(tmem + lane_base + b * 128 + 64, a0);
-                    tmem_ld32(tmem + lane_base + b * 128 + 96, a1);
+                    tmem_ld32(tmem + lane_base + b * 128 + 64 + hf * 32, acc);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-                        for (int cc = 0; cc < 4; ++cc) {       // gV = (1 + k').1 nu_R + k' R''
-                            if (hh >= nhalf) break;
-                            const uint32_t* acc = hh ? a1 : a0;
-                            const float* nu = sNu + hh * 32 + cc * 8;
-                            sts128(out_row + kTileBytes + (((hh * 4 + cc) ^ r7) << 4),
-                                   pack_bf16x2(fmaf(x1sum, nu[0], __uint_as_float(acc[cc * 8 + 0])), fmaf(x1sum, nu[1], __uint_as_float(acc[cc * 8 + 1]))),
-                                   pack_bf16x2(fmaf(x1sum, nu[2], __uint_as_float(acc[cc * 8 + 2])), fmaf(x1sum, nu[3], __uint_as_float(acc[cc * 8 + 3]))),
-                                   pack_bf16x2(fmaf(x1sum, nu[4], __uint_as_float(acc[cc * 8 + 4])), fmaf(x1sum, nu[5], __uint_as_float(acc[cc * 8 + 5]))),
-                                   pack_bf16x2(fmaf(x1sum, nu[6], __uint_as_float(acc[cc * 8 + 6])), fmaf(x1sum, nu[7], __uint_as_float(acc[cc * 8 + 7]))));
-                        }
+                    for (int cc = 0; cc < 4; ++cc) {       // gV = (1 + k').1 nu_R + k' R''
+                        const float* nu = nuH + cc * 8;
+                        sts128(out_row + kTileBytes + (((hf * 4 + cc) ^ r7) << 4),
+                               pack_bf16x2(fmaf(x1sum, nu[0], __uint_as_float(acc[cc * 8 + 0])), fmaf(x1sum, nu[1], __uint_as_float(acc[cc * 8 + 1]))),
+                               pack_bf16x2(fmaf(x1sum, nu[2], __uint_as_float(acc[cc * 8 + 2])), fmaf(x1sum, nu[3], __uint_as_float(acc[cc * 8 + 3]))),
+                               pack_bf16x2(fmaf(x1sum, nu[4], __uint_as_float(acc[cc * 8 + 4])), fmaf(x1sum, nu[5], __uint_as_float(acc[cc * 8 + 5]))),
+                               pack_bf16x2(fmaf(x1sum, nu[6], __uint_as_float(acc[cc * 8 + 6])), fmaf(x1sum, nu[7], __uint_as_float(acc[cc * 8 + 7]))));
+                    }
                 }
             }
             tc_fence_before_sync();
             mbar_arrive(&bars->acc_free[b]);
             fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                const int y = (int)(row0 + (int64_t)c * kChunk + warp * 32);
-                tma_store_2d(&mapOut0, smem + kApOffOut + warp * 32 * 128, 0, y);
-                if (kMode == kApplyBackwardKV) tma_store_2d(&mapOut1, smem + kApOffOut + kTileBytes + warp * 32 * 128, 0, y);
+            named_barrier(2 + quad, 64);            // both halves of the 32 rows are in the slab
+            if (hf == 0 && lane == 0) {
+                const int y = (int)(row0 + (int64_t)c * kChunk + quad * 32);
+                tma_store_2d(&mapOut0, smem + kApOffOut + quad * 32 * 128, 0, y);
+                if (kMode == kApplyBackwardKV) tma_store_2d(&mapOut1, smem + kApOffOut + kTileBytes + quad * 32 * 128, 0, y);
                 tma_store_commit();
             }
         }
-        if (lane == 0) tma_store_wait_all<0>();
+        if (hf == 0 && lane == 0) tma_store_wait_all<0>();
     }
 
     tc_fence_before_sync();
