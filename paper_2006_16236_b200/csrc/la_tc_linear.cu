@@ -254,7 +254,7 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 // ===========================================================================
 enum ApplyMode { kApplyForward = 0, kApplyBackwardQ = 1, kApplyBackwardKV = 2 };
 
-constexpr int kApStages = 3;
+constexpr int kApStages = 4;
 constexpr int kApThreads = 448;
 constexpr uint32_t kApOffStage = 0;                                   // kApStages x {X, Y}
 constexpr uint32_t kApOffState = kApOffStage + kApStages * 2 * kTileBytes;   // bf16 centred state tile [64][64]
