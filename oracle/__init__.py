@@ -52,6 +52,8 @@ def _load():
             [_i64] * 5 + [ctypes.c_int, ctypes.c_int, ctypes.c_double] + [_dp] * 7)
         _lib.la_oracle_linear_backward.argtypes = (
             [_i64] * 5 + [ctypes.c_int, ctypes.c_int, ctypes.c_double] + [_dp] * 7)
+        _lib.la_oracle_causal_from_state.argtypes = (
+            [_i64] * 5 + [ctypes.c_int, ctypes.c_double] + [_dp] * 9)
         _lib.la_oracle_recurrent_step.argtypes = (
             [_i64] * 4 + [ctypes.c_int, ctypes.c_double] + [_dp] * 6)
     return _lib
@@ -124,6 +126,22 @@ def linear_attention(Q, K, V, causal: bool, phi: str = "elu1", eps: float = 0.0,
     _load().la_oracle_linear(B, H, N, D, M, int(causal), PHI[phi], eps,
                              _p(Q), _p(K), _p(V), _p(O), _p(den), _p(S), _p(Z))
     return (O, den, S, Z) if return_state else (O, den)
+
+
+def causal_from_state(Q, K, V, S0, Z0, phi: str = "elu1", eps: float = 0.0):
+    """Eq. 16-20 (attention part) run over N tokens from the state S0 [B,H,D,M], Z0 [B,H,D];
+    returns (O, den, S_N, Z_N)."""
+    Q, K, V, B, H, N, D, M = _shapes(Q, K, V)
+    S0, Z0 = _f64(S0), _f64(Z0)
+    if S0.shape != (B, H, D, M) or Z0.shape != (B, H, D):
+        raise ValueError("state shape mismatch")
+    O = np.empty((B, H, N, M))
+    den = np.empty((B, H, N))
+    S = np.empty((B, H, D, M))
+    Z = np.empty((B, H, D))
+    _load().la_oracle_causal_from_state(B, H, N, D, M, PHI[phi], eps, _p(Q), _p(K), _p(V), _p(S0), _p(Z0),
+                                        _p(O), _p(den), _p(S), _p(Z))
+    return O, den, S, Z
 
 
 def linear_attention_backward(Q, K, V, G, causal: bool, phi: str = "elu1", eps: float = 0.0):

@@ -23,7 +23,8 @@
  *       with the gradients of Eq. 13-15 (Algorithm 1, backward) applied to the
  *       value matrix extended by a column of ones, which carries the
  *       normaliser Z (Eq. 11) and its gradient; the recurrent step is
- *       Eq. 16-20 restricted to the attention part.
+ *       Eq. 16-20 restricted to the attention part, and the causal form
+ *       continued from a given state is that recurrence started from it.
  * The tests pin (1) to closed forms, a hand-worked rational example, library
  * one-liners and finite differences, and (2) to (1).  No function here is
  * "parity unpinned".
@@ -247,6 +248,51 @@ void la_oracle_linear(int64_t B, int64_t H, int64_t N, int64_t D, int64_t M,
         if (S_out) memcpy(S_out + bh * D * M, S, (size_t)(D * M) * sizeof(double));
         if (Z_out) memcpy(Z_out + bh * D, Z, (size_t)D * sizeof(double));
         free(Z); free(S); free(k); free(q);
+    }
+}
+
+/*
+ * Causal form continued from a given state: the recurrence of Eq. 16-20 (attention part) started
+ * from s_0 = S0, z_0 = Z0 instead of zero, which is what the state carried over from the tokens
+ * before this call amounts to (a long sequence processed in several calls):
+ *     for i = 1..N:  s_i = s_{i-1} + phi(K_i) V_i^T ;  z_i = z_{i-1} + phi(K_i) ;
+ *                    O_i = phi(Q_i)^T s_i / (phi(Q_i)^T z_i + eps).
+ * S0 / Z0: [B, H, D, M] / [B, H, D].  den, S_out, Z_out as in la_oracle_linear.
+ */
+void la_oracle_causal_from_state(int64_t B, int64_t H, int64_t N, int64_t D, int64_t M,
+                                 int phi, double eps,
+                                 const double *Q, const double *K, const double *V,
+                                 const double *S0, const double *Z0,
+                                 double *O, double *den, double *S_out, double *Z_out)
+{
+    int64_t BH = B * H;
+#pragma omp parallel for schedule(dynamic)
+    for (int64_t bh = 0; bh < BH; ++bh) {
+        const double *Vh = V + bh * N * M;
+        double *Oh = O + bh * N * M;
+        double *q = mapped(Q + bh * N * D, N * D, phi);
+        double *k = mapped(K + bh * N * D, N * D, phi);
+        double *s = (double *)malloc((size_t)(D * M > 0 ? D * M : 1) * sizeof(double));
+        double *z = (double *)malloc((size_t)(D > 0 ? D : 1) * sizeof(double));
+        memcpy(s, S0 + bh * D * M, (size_t)(D * M) * sizeof(double));
+        memcpy(z, Z0 + bh * D, (size_t)D * sizeof(double));
+        for (int64_t i = 0; i < N; ++i) {
+            for (int64_t d = 0; d < D; ++d) {
+                for (int64_t e = 0; e < M; ++e) s[d * M + e] += k[i * D + d] * Vh[i * M + e];
+                z[d] += k[i * D + d];
+            }
+            double dn = 0.0;
+            for (int64_t d = 0; d < D; ++d) dn += q[i * D + d] * z[d];
+            for (int64_t e = 0; e < M; ++e) {
+                double num = 0.0;
+                for (int64_t d = 0; d < D; ++d) num += q[i * D + d] * s[d * M + e];
+                Oh[i * M + e] = num / (dn + eps);
+            }
+            if (den) den[bh * N + i] = dn;
+        }
+        if (S_out) memcpy(S_out + bh * D * M, s, (size_t)(D * M) * sizeof(double));
+        if (Z_out) memcpy(Z_out + bh * D, z, (size_t)D * sizeof(double));
+        free(z); free(s); free(k); free(q);
     }
 }
 

@@ -205,6 +205,48 @@ def test_recurrent_unrolled_equals_causal(shape):
     assert np.allclose(Z, fk.sum(2), rtol=1e-13)                                          # Eq. 11
 
 
+# ------------------------------------------------ continuation from a state
+def test_causal_from_state_hand_example():
+    # D = M = 1, identity features, q = k = 1, s_0 = 3, z_0 = 2, v = 1, 2, 3 (Eq. 18-20 by hand):
+    # O_i = (3 + v_1 + .. + v_i) / (2 + i) = 4/3, 6/4, 9/5; final state s = 9, z = 5
+    one = np.ones((1, 1, 3, 1))
+    V = np.array([1.0, 2.0, 3.0]).reshape(1, 1, 3, 1)
+    O, den, S, Z = oracle.causal_from_state(one, one, V, np.full((1, 1, 1, 1), 3.0), np.full((1, 1, 1), 2.0), phi="identity")
+    assert np.allclose(O.ravel(), [4 / 3, 6 / 4, 9 / 5], rtol=1e-15)
+    assert np.allclose(den.ravel(), [3.0, 4.0, 5.0]) and S.item() == 9.0 and Z.item() == 5.0
+
+
+@pytest.mark.parametrize("shape", [(2, 2, 23, 5, 3), (1, 3, 40, 8, 8)])
+def test_causal_from_state_equals_unrolled_recurrent_steps(shape):
+    # Eq. 18-20 step by step from an arbitrary (positive-normaliser) state
+    B, H, N, D, M = shape
+    Q, K, V = rnd((B, H, N, D), 33), rnd((B, H, N, D), 34), rnd((B, H, N, M), 35)
+    S0, Z0 = rnd((B, H, D, M), 36), np.abs(rnd((B, H, D), 37)) + 0.5
+    O, den, SN, ZN = oracle.causal_from_state(Q, K, V, S0, Z0)
+    S, Z = S0.copy(), Z0.copy()
+    for i in range(N):
+        out = oracle.recurrent_step(Q[:, :, i], K[:, :, i], V[:, :, i], S, Z)
+        assert np.allclose(out, O[:, :, i], rtol=1e-11, atol=1e-12)
+    assert np.allclose(S, SN, rtol=1e-13, atol=1e-13) and np.allclose(Z, ZN, rtol=1e-13)
+
+
+@pytest.mark.parametrize("cut", [1, 17, 39])
+def test_a_sequence_cut_in_two_calls_reproduces_the_definition(cut):
+    # the definition (explicit N x N masked attention) on the whole sequence against: first part from zero,
+    # second part continued from the first part's final state; zero state reduces to the causal form
+    B, H, N, D, M = 2, 2, 40, 6, 5
+    Q, K, V = rnd((B, H, N, D), 43), rnd((B, H, N, D), 44), rnd((B, H, N, M), 45)
+    ref = oracle.attention_quadratic(Q, K, V, True)
+    O1, _, S1, Z1 = oracle.linear_attention(Q[:, :, :cut], K[:, :, :cut], V[:, :, :cut], True, return_state=True)
+    O2, den2, S2, Z2 = oracle.causal_from_state(Q[:, :, cut:], K[:, :, cut:], V[:, :, cut:], S1, Z1)
+    assert np.allclose(np.concatenate([O1, O2], axis=2), ref, rtol=1e-11, atol=1e-12)
+    _, denf, SN, ZN = oracle.linear_attention(Q, K, V, True, return_state=True)
+    assert np.allclose(den2, denf[:, :, cut:], rtol=1e-12) and np.allclose(S2, SN, rtol=1e-12, atol=1e-13)
+    assert np.allclose(Z2, ZN, rtol=1e-13)
+    Oz, denz, Sz, Zz = oracle.causal_from_state(Q, K, V, np.zeros((B, H, D, M)), np.zeros((B, H, D)))
+    assert np.allclose(Oz, ref, rtol=1e-11, atol=1e-12)
+
+
 # ------------------------------------------------------------------- gradients
 def _torch_quadratic(Q, K, V, causal, eps=0.0, identity=False):
     phi = (lambda x: x) if identity else (lambda x: torch.nn.functional.elu(x) + 1)
