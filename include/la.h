@@ -124,6 +124,25 @@ int la_causal_forward(const la_problem* p, const void* Q, const void* K, const v
                       void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The causal form continued from a state: the recurrence of Eq. 16-20 run over the N positions of
+ * this call from S_0 = S_in, Z_0 = Z_in instead of zero,
+ *   O_i = phi(Q_i)^T (S_in + sum_{j<=i} phi(K_j) V_j^T) / (phi(Q_i)^T (Z_in + sum_{j<=i} phi(K_j)) + eps),
+ * so that a long sequence can be processed in several calls (chunked prefill) and S_out / Z_out of
+ * one call are S_in / Z_in of the next, or the state la_recurrent_step() continues from.
+ * S_in [B,H,D,M] and Z_in [B,H,D]: device, fp32, 16-byte aligned, both given or both NULL (NULL:
+ * the call is la_causal_forward()); they are only read and must not overlap S_out / Z_out
+ * (LA_ERR_INVALID_ARG: the pieces of a sequence run concurrently and all start from S_in).  den
+ * includes the Z_in term.  With N = 0 the state is copied to S_out / Z_out.  There is no backward
+ * pass from a non-zero state in this library, so `saved` must be NULL when S_in is given
+ * (LA_ERR_UNSUPPORTED).  Everything else as for la_causal_forward().
+ */
+int la_causal_forward_from(const la_problem* p, const void* Q, const void* K, const void* V,
+                           const float* S_in, const float* Z_in,
+                           void* O, float* den, float* S_out, float* Z_out,
+                           void* saved, size_t saved_bytes,
+                           void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Gradient of the causal form in linear time and memory independent of N per
  * head, Eq. 13-15 (Algorithm 1, backward): grad phi(Q_i) uses the forward running
  * sum of phi(K_j)[V_j,1]^T, grad phi(K_i) and grad V_i the reverse running sum of

@@ -22,7 +22,7 @@ _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
     "la_feature_map", "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
-    "la_causal_forward",
+    "la_causal_forward", "la_causal_forward_from",
     "la_causal_backward", "la_recurrent_step", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
     "la_profile_kernel_name", "la_version", "la_causal_plan",
@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.la_linear_attention_noalloc.argtypes = [pp] + [vp] * 7 + [vp]
         L.la_linear_attention_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
         L.la_causal_forward.argtypes = [pp] + [vp] * 7 + [vp, sz] + [vp, sz, vp]
+        L.la_causal_forward_from.argtypes = [pp] + [vp] * 9 + [vp, sz] + [vp, sz, vp]
         L.la_causal_backward.argtypes = [pp] + [vp] * 6 + [vp, sz] + [vp] * 3 + [vp, sz, vp]
         L.la_recurrent_step.argtypes = [pp] + [vp] * 6 + [vp]
         L.la_workspace_bytes.argtypes = [pp, i32]
@@ -253,15 +254,25 @@ def saved_buffer(Q, V, phi="elu1", eps=0.0):
     return None if need == 0 else torch.empty(need, dtype=torch.uint8, device=Q.device)
 
 
-def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None, Z_out=None, saved=None, ws=None):
+def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None, Z_out=None, saved=None, ws=None,
+                      S_in=None, Z_in=None):
     """Causal form.  Returns O; pass preallocated den / S_out / Z_out tensors to receive them, and a
-    saved_buffer() to keep phi(Q), phi(K) for the backward pass."""
-    dev = _dev(Q, K, V, O, den, S_out, Z_out, saved)
+    saved_buffer() to keep phi(Q), phi(K) for the backward pass.  S_in / Z_in (fp32 [B,H,D,M] / [B,H,D]):
+    the state the sequence continues from (la_causal_forward_from)."""
+    dev = _dev(Q, K, V, O, den, S_out, Z_out, saved, S_in, Z_in)
     p = _problem_of(Q, V, phi, eps)
     O = torch.empty_like(V) if O is None else O
     ws = workspace(p, LA_OP_CAUSAL_FORWARD, dev) if ws is None else ws
-    _check(lib().la_causal_forward(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(S_out),
-                                   _ptr(Z_out), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(dev)))
+    if S_in is None and Z_in is None:
+        _check(lib().la_causal_forward(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(S_out),
+                                       _ptr(Z_out), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(dev)))
+    else:
+        for t, shape in ((S_in, (p.B, p.H, p.D, p.M)), (Z_in, (p.B, p.H, p.D))):
+            if t is not None and (t.dtype != torch.float32 or tuple(t.shape) != shape or not t.is_contiguous()):
+                raise ValueError("S_in / Z_in must be contiguous fp32 tensors of shape [B,H,D,M] / [B,H,D]")
+        _check(lib().la_causal_forward_from(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(S_in), _ptr(Z_in), _ptr(O),
+                                            _ptr(den), _ptr(S_out), _ptr(Z_out), _ptr(saved), _nbytes(saved), _ptr(ws),
+                                            _nbytes(ws), _stream(dev)))
     return O
 
 

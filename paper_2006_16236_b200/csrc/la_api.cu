@@ -228,21 +228,46 @@ int la_linear_attention_backward(const la_problem* p, const void* Q, const void*
     return general_linear_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
 }
 
-int la_causal_forward(const la_problem* p, const void* Q, const void* K, const void* V,
-                      void* O, float* den, float* S_out, float* Z_out,
-                      void* saved, size_t saved_bytes,
-                      void* ws, size_t ws_bytes, void* stream) {
+static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return a && b && x < y + nb && y < x + na;
+}
+
+int la_causal_forward_from(const la_problem* p, const void* Q, const void* K, const void* V,
+                           const float* S_in, const float* Z_in,
+                           void* O, float* den, float* S_out, float* Z_out,
+                           void* saved, size_t saved_bytes,
+                           void* ws, size_t ws_bytes, void* stream) {
     if (int rc = check_problem(p, true)) return rc;
-    if (p->N == 0) return LA_OK;
-    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(O);
+    if ((S_in == nullptr) != (Z_in == nullptr)) return fail(LA_ERR_INVALID_ARG, "S_in and Z_in must both be given or both be NULL");
+    LA_OPTIONAL_PTR(S_in); LA_OPTIONAL_PTR(Z_in);
     LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(S_out); LA_OPTIONAL_PTR(Z_out);
+    const size_t s_bytes = (size_t)(p->B * p->H * p->D * p->M) * sizeof(float), z_bytes = (size_t)(p->B * p->H * p->D) * sizeof(float);
+    if (overlaps(S_in, s_bytes, S_out, s_bytes) || overlaps(S_in, s_bytes, Z_out, z_bytes) ||
+        overlaps(Z_in, z_bytes, S_out, s_bytes) || overlaps(Z_in, z_bytes, Z_out, z_bytes))
+        return fail(LA_ERR_INVALID_ARG, "S_in / Z_in overlap S_out / Z_out");
+    if (S_in && saved) return fail(LA_ERR_UNSUPPORTED, "no backward pass from a non-zero state: saved must be NULL with S_in");
+    cudaStream_t st = (cudaStream_t)stream;
+    if (p->N == 0) {
+        if (S_in && S_out) LA_CUDA_TRY(cudaMemcpyAsync(S_out, S_in, s_bytes, cudaMemcpyDeviceToDevice, st));
+        if (Z_in && Z_out) LA_CUDA_TRY(cudaMemcpyAsync(Z_out, Z_in, z_bytes, cudaMemcpyDeviceToDevice, st));
+        return LA_OK;
+    }
+    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(O);
     LA_OPTIONAL_PTR(saved);
     if (int rc = check_ws(p, LA_OP_CAUSAL_FORWARD, ws, ws_bytes)) return rc;
     if (int rc = check_saved(p, saved, saved_bytes)) return rc;
     if (int rc = check_arch()) return rc;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_CAUSAL_FORWARD)) return tc_causal_forward(*p, Q, K, V, O, den, S_out, Z_out, saved, ws, st);
-    return general_causal_forward(*p, Q, K, V, O, den, S_out, Z_out, st);
+    if (tc_supported(*p, LA_OP_CAUSAL_FORWARD))
+        return tc_causal_forward(*p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
+    return general_causal_forward(*p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, st);
+}
+
+int la_causal_forward(const la_problem* p, const void* Q, const void* K, const void* V,
+                      void* O, float* den, float* S_out, float* Z_out,
+                      void* saved, size_t saved_bytes,
+                      void* ws, size_t ws_bytes, void* stream) {
+    return la_causal_forward_from(p, Q, K, V, nullptr, nullptr, O, den, S_out, Z_out, saved, saved_bytes, ws, ws_bytes, stream);
 }
 
 int la_causal_backward(const la_problem* p, const void* Q, const void* K, const void* V,

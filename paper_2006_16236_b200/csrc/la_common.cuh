@@ -76,6 +76,7 @@ int launch_recurrent_step(const la_problem& p, const void* q, const void* k, con
 // General (any D, M multiple of 8 up to 128, any N) fp32-arithmetic kernels.
 size_t general_workspace_bytes(const la_problem& p, int op);
 int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V,
+                           const float* S_in, const float* Z_in,
                            void* O, float* den, float* S_out, float* Z_out, cudaStream_t st);
 int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V,
                             const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);

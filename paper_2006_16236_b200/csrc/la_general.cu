@@ -132,6 +132,7 @@ size_t smem_floats_backward(int D, int M) {
 template <typename IO>
 __global__ void __launch_bounds__(THREADS)
 general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K, const IO* __restrict__ V,
+                              const float* __restrict__ S_in, const float* __restrict__ Z_in,
                               IO* __restrict__ O, float* __restrict__ den, float* __restrict__ S_out,
                               float* __restrict__ Z_out, int64_t N, int D, int M, float eps, int phi) {
     extern __shared__ float smem[];
@@ -146,6 +147,12 @@ general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K
     const int64_t bh = blockIdx.x;
     Q += bh * N * D; K += bh * N * D; V += bh * N * M; O += bh * N * M;
     zero_fill(sSt, D * dm.MS);
+    if (S_in) {                 // continue from a given state (Eq. 16-20 started from S_in, Z_in)
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < D * M; idx += THREADS)
+            sSt[(idx / M) * dm.MS + idx % M] = S_in[bh * D * M + idx];
+        for (int d = threadIdx.x; d < D; d += THREADS) sSt[d * dm.MS + M] = Z_in[bh * D + d];
+    }
 
     for (int64_t n0 = 0; n0 < N; n0 += T) {
         const int cn = (int)((N - n0) < T ? (N - n0) : T);
@@ -473,21 +480,21 @@ size_t general_workspace_bytes(const la_problem& p, int op) {
 }
 
 template <typename IO>
-static int causal_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
-                            float* den, float* S_out, float* Z_out, cudaStream_t st) {
+static int causal_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+                            const float* Z_in, void* O, float* den, float* S_out, float* Z_out, cudaStream_t st) {
     const size_t smem = smem_floats_forward((int)p.D, (int)p.M) * sizeof(float);
     auto kern = general_causal_forward_kernel<IO>;
     if (int rc = opt_in_smem(kern, smem)) return rc;
-    kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, (IO*)O, den,
+    kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, S_in, Z_in, (IO*)O, den,
                                                        S_out, Z_out, p.N, (int)p.D, (int)p.M, p.eps, p.phi);
     LA_LAUNCHED();
     return LA_OK;
 }
 
-int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
-                           float* den, float* S_out, float* Z_out, cudaStream_t st) {
-    return p.dtype == LA_F32 ? causal_forward_t<float>(p, Q, K, V, O, den, S_out, Z_out, st)
-                             : causal_forward_t<__nv_bfloat16>(p, Q, K, V, O, den, S_out, Z_out, st);
+int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+                           const float* Z_in, void* O, float* den, float* S_out, float* Z_out, cudaStream_t st) {
+    return p.dtype == LA_F32 ? causal_forward_t<float>(p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, st)
+                             : causal_forward_t<__nv_bfloat16>(p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, st);
 }
 
 template <typename IO>

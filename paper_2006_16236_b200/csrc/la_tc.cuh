@@ -11,8 +11,9 @@ size_t tc_workspace_bytes(const la_problem& p, int op);
 size_t tc_causal_saved_bytes(const la_problem& p);
 // pieces, parts, piece_begin[], piece_first_part[], part_begin[], launch_order[] (see la_causal_plan)
 int tc_causal_plan(const la_problem& p, int32_t* out, int capacity);
-int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
-                      float* den, float* S_out, float* Z_out, void* saved, void* ws, cudaStream_t st);
+int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+                      const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
+                      cudaStream_t st);
 int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* O,
                        const float* den, const void* G, const void* saved, void* dQ, void* dK, void* dV, void* ws,
                        cudaStream_t st);
@@ -24,8 +25,9 @@ int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const 
 namespace tc {
 size_t causal_forward_workspace(const la_problem& p);
 size_t causal_saved_bytes(const la_problem& p);
-int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
-                   float* S_out, float* Z_out, void* saved, void* ws, cudaStream_t st);
+int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+                   const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
+                   cudaStream_t st);
 size_t causal_backward_workspace(const la_problem& p);
 int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
                     const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);

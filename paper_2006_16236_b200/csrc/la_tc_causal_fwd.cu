@@ -66,6 +66,8 @@ struct FwdParams {
     __nv_bfloat16* O;
     float* den;            // [BH, N] or null
     const float* init;     // per (bh, part) [S|Z] records of the pre-pass, or null (single piece)
+    const float* S_in;     // [BH, D, M] state the sequence continues from, or null (zero)
+    const float* Z_in;     // [BH, D]
     CausalPlan plan;       // pieces of a sequence and their pre-pass parts
     float* S_out;          // [BH, D, M] or null
     float* Z_out;          // [BH, D] or null
@@ -305,7 +307,9 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         const uint32_t r7 = t & 7;
         const float* rec = prm.init ? prm.init + bh * (int64_t)plan.nparts() * kStateFloats : nullptr;
         uint8_t* tile1 = smem + kOffS + kStateTileBytes;            // the state before chunk 0 lives in tile 1
-        state_init_tiles(tmem + kColS, quad, lane, tile1, tile1 + kDim * 128, rec, 0, rec ? plan.piece_first_part(piece) : 0);
+        state_init_tiles(tmem + kColS, quad, lane, tile1, tile1 + kDim * 128, rec, 0, rec ? plan.piece_first_part(piece) : 0,
+                         prm.S_in ? prm.S_in + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
+                         prm.Z_in ? prm.Z_in + bh * prm.dim : nullptr, prm.dim);
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(&bars->state_ready[1]);
@@ -493,8 +497,9 @@ size_t causal_forward_workspace(const la_problem& p) {
 
 size_t causal_saved_bytes(const la_problem& p) { return saved_layout(p, choose_plan(p)).bytes; }
 
-int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
-                   float* S_out, float* Z_out, void* saved, void* ws, cudaStream_t st) {
+int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+                   const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
+                   cudaStream_t st) {
     const CausalPlan pl = choose_plan(p);
     const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
     const SavedLayout sl = saved_layout(p, pl);
@@ -524,6 +529,8 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     prm.den = den;
     prm.init = pl.npieces() > 1 ? records : nullptr;
     prm.plan = pl;
+    prm.S_in = S_in;
+    prm.Z_in = Z_in;
     prm.S_out = S_out;
     prm.Z_out = Z_out;
     prm.status = status;

@@ -258,9 +258,13 @@ __device__ __forceinline__ void state_to_smem(uint32_t tmem_state, int quad, int
 // record), in part order, with the loads of four records in flight: a piece late in a sequence starts
 // from several records, and one round trip to L2 per record and column group would cost microseconds
 // on the critical start-up of its CTA.
-__device__ __forceinline__ void sum_records16(const float* rec, int part_lo, int part_hi, int offset, float (&acc)[16]) {
+__device__ __forceinline__ void sum_records16(const float* rec, int part_lo, int part_hi, int offset, float (&acc)[16],
+                                              const float* base = nullptr) {
 #pragma unroll
-    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+    for (int j = 0; j < 4; ++j) {      // `base` (16 floats, 16-byte aligned, or null): the value the sum starts from
+        const float4 b = base ? __ldg(reinterpret_cast<const float4*>(base) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc[4 * j] = b.x; acc[4 * j + 1] = b.y; acc[4 * j + 2] = b.z; acc[4 * j + 3] = b.w;
+    }
 #pragma unroll 1
     for (int p = part_lo; p < part_hi; p += 4) {
         float4 a[4][4];
@@ -379,15 +383,19 @@ __device__ __forceinline__ void state_half_to_tiles(uint32_t tmem_state, int qua
 
 // Initial state of a segment (sum of the records of parts [part_lo, part_hi), or zeros) into
 // the TMEM accumulator (S in 64 columns, Z replicated in 16) and the bf16 tiles.
+// s_in / z_in (or null): the [dim][dim] / [dim] fp32 state of this (batch, head) the sequence continues from.
 __device__ __forceinline__ void state_init_tiles(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, uint8_t* z_tile,
-                                                 const float* rec, int part_lo, int part_hi) {
+                                                 const float* rec, int part_lo, int part_hi,
+                                                 const float* s_in = nullptr, const float* z_in = nullptr, int dim = kDim) {
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
+    const bool in_row = owner && s_in && d_row < dim;
 #pragma unroll 1
     for (int g = 0; g < 4; ++g) {
         float acc[16];
-        sum_records16(rec, owner ? part_lo : 0, owner ? part_hi : 0, d_row * kDim + g * 16, acc);
+        sum_records16(rec, owner ? part_lo : 0, owner ? part_hi : 0, d_row * kDim + g * 16, acc,
+                      in_row && g * 16 < dim ? s_in + d_row * dim + g * 16 : nullptr);
         uint32_t v[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(acc[j]);
@@ -400,7 +408,7 @@ __device__ __forceinline__ void state_init_tiles(uint32_t tmem_state, int quad, 
                        sm100::pack_bf16x2(acc[cc * 8 + 4], acc[cc * 8 + 5]), sm100::pack_bf16x2(acc[cc * 8 + 6], acc[cc * 8 + 7]));
         }
     }
-    const float z = owner ? sum_records1(rec, part_lo, part_hi, kDim * kDim + d_row) : 0.f;
+    const float z = (owner ? sum_records1(rec, part_lo, part_hi, kDim * kDim + d_row) : 0.f) + (in_row ? __ldg(z_in + d_row) : 0.f);
     uint32_t zz[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) zz[j] = __float_as_uint(z);

@@ -173,6 +173,58 @@ def test_prefill_then_decode_handoff():
     assert_close(out, ref, torch.float32, "decode after prefill")
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", [(2, 3, 100, 16, 48), (1, 2, 31, 64, 64), (2, 2, 640, 32, 32), (1, 4, 384, 64, 64),
+                                   (4, 16, 18 * 128, 64, 64)])
+def test_causal_forward_from_a_state(shape, dtype):
+    """The recurrence of Eq. 16-20 started from a given S_0, Z_0 (general kernels and, for bf16 D = M in
+    {32, 64} with N a multiple of 128, the tensor-core kernel with several pieces per sequence)."""
+    B, H, N, D, M = shape
+    Q, K, V, _ = draw_qkvg(B, H, N, D, M, seed=sum(shape) + 1, dtype=dtype, with_grad=False)
+    g = torch.Generator().manual_seed(5)
+    S0 = torch.randn((B, H, D, M), generator=g) * 3.0
+    Z0 = torch.rand((B, H, D), generator=g) * 4.0 + 1.0
+    Qd, Kd, Vd, S0d, Z0d = gpu(Q, K, V, S0, Z0)
+    den = torch.empty((B, H, N), device=DEV)
+    S = torch.empty((B, H, D, M), device=DEV)
+    Z = torch.empty((B, H, D), device=DEV)
+    O = la.la_causal_forward(Qd, Kd, Vd, den=den, S_out=S, Z_out=Z, S_in=S0d, Z_in=Z0d)
+    la.la_last_device_status()
+    sel = [(0, 0), (B - 1, H - 1)] if B * H > 8 else [(b, h) for b in range(B) for h in range(H)]
+    for b, h in sel:
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        Or, denr, Sr, Zr = oracle.causal_from_state(Q[sl], K[sl], V[sl], S0[sl].double().numpy(), Z0[sl].double().numpy())
+        assert_close(O[sl], Or, dtype, f"O[{b},{h}]")
+        assert_close(den[sl], denr, dtype, f"den[{b},{h}]")
+        assert_close(S[sl], Sr, dtype, f"S_N[{b},{h}]")
+        assert_close(Z[sl], Zr, dtype, f"Z_N[{b},{h}]")
+    assert torch.equal(S0d.cpu(), S0) and torch.equal(Z0d.cpu(), Z0)        # the given state is only read
+
+
+@pytest.mark.parametrize("dtype,D,chunks", [(torch.float32, 32, (100, 60, 96)), (torch.bfloat16, 64, (1024, 512, 2560))])
+def test_chunked_prefill_then_decode(dtype, D, chunks):
+    """A sequence processed in three calls, each continuing from the state the previous one returned, then one
+    recurrent step: every output equals the definition on the whole sequence."""
+    B, H = 2, 2
+    N = sum(chunks)
+    Q, K, V, _ = draw_qkvg(B, H, N + 1, D, D, seed=19, dtype=dtype, with_grad=False)
+    Qd, Kd, Vd = gpu(Q, K, V)
+    S = [torch.zeros((B, H, D, D), device=DEV), torch.empty((B, H, D, D), device=DEV)]
+    Z = [torch.zeros((B, H, D), device=DEV), torch.empty((B, H, D), device=DEV)]
+    outs, lo = [], 0
+    for i, n in enumerate(chunks):
+        sl = slice(lo, lo + n)
+        outs.append(la.la_causal_forward(Qd[:, :, sl].contiguous(), Kd[:, :, sl].contiguous(), Vd[:, :, sl].contiguous(),
+                                         S_in=S[i & 1], Z_in=Z[i & 1], S_out=S[(i + 1) & 1], Z_out=Z[(i + 1) & 1]))
+        lo += n
+    k = len(chunks) & 1
+    last = la.la_recurrent_step(Qd[:, :, N].contiguous(), Kd[:, :, N].contiguous(), Vd[:, :, N].contiguous(), S[k], Z[k])
+    la.la_last_device_status()
+    ref = oracle.linear_attention(Q, K, V, True)[0]
+    assert_close(torch.cat(outs, dim=2), ref[:, :, :N], dtype, "chunked prefill")
+    assert_close(last, ref[:, :, N], dtype, "decode after chunked prefill")
+
+
 def test_gradient_invariants_hold_on_gpu_results():
     B, H, N, D, M = 2, 4, 512, 64, 64
     Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=11, dtype=torch.float32)

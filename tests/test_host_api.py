@@ -134,6 +134,18 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert L.la_causal_backward(*args, big, 1 << 40, null) == -1
     assert la.la_workspace_bytes(_p(), binding.LA_OP_CAUSAL_SAVED) == 0
     assert L.la_recurrent_step(ctypes.byref(p), ok, ok, ok, null, ok, ok, null) == -1
+    # continuation from a state: S_in and Z_in come together, must not overlap the outputs, exclude `saved`
+    def cont(p, S_in, Z_in, S_out=null, Z_out=null, saved=null, saved_bytes=0):
+        return L.la_causal_forward_from(ctypes.byref(p), ok, ok, ok, S_in, Z_in, ok, null, S_out, Z_out,
+                                        saved, saved_bytes, null, 0, null)
+    far = ctypes.c_void_p(1 << 30)
+    assert cont(_p(), far, null) == -1
+    assert cont(_p(), null, far) == -1
+    assert cont(_p(), far, ctypes.c_void_p((1 << 30) + (1 << 20)), S_out=far) == -1
+    assert b"overlap" in L.la_last_error()
+    assert cont(_p(), odd, far) == -1
+    assert cont(pb, far, ctypes.c_void_p((1 << 30) + (1 << 24)), saved=big, saved_bytes=keep) == -2
+    assert cont(_p(N=0), null, null) == 0
     assert L.la_feature_map(ok, ok, -5, 0, 0, null) == -1
     assert L.la_feature_map(ok, ok, 0, 0, 0, null) == 0
     assert L.la_feature_map(ok, ok, 4, 9, 0, null) == -1
