@@ -54,6 +54,8 @@ def _load():
             [_i64] * 5 + [ctypes.c_int, ctypes.c_int, ctypes.c_double] + [_dp] * 7)
         _lib.la_oracle_causal_from_state.argtypes = (
             [_i64] * 5 + [ctypes.c_int, ctypes.c_double] + [_dp] * 9)
+        _lib.la_oracle_causal_backward_from_state.argtypes = (
+            [_i64] * 5 + [ctypes.c_int, ctypes.c_double] + [_dp] * 13)
         _lib.la_oracle_recurrent_step.argtypes = (
             [_i64] * 4 + [ctypes.c_int, ctypes.c_double] + [_dp] * 6)
     return _lib
@@ -142,6 +144,22 @@ def causal_from_state(Q, K, V, S0, Z0, phi: str = "elu1", eps: float = 0.0):
     _load().la_oracle_causal_from_state(B, H, N, D, M, PHI[phi], eps, _p(Q), _p(K), _p(V), _p(S0), _p(Z0),
                                         _p(O), _p(den), _p(S), _p(Z))
     return O, den, S, Z
+
+
+def causal_backward_from_state(Q, K, V, S0, Z0, G, dSN=None, dZN=None, phi: str = "elu1", eps: float = 0.0):
+    """Gradient of sum(G * O) + <dSN, S_N> + <dZN, Z_N> for causal_from_state; returns (dQ, dK, dV, dS0, dZ0)."""
+    Q, K, V, B, H, N, D, M = _shapes(Q, K, V)
+    S0, Z0, G = _f64(S0), _f64(Z0), _f64(G)
+    dSN = None if dSN is None else _f64(dSN)
+    dZN = None if dZN is None else _f64(dZN)
+    if S0.shape != (B, H, D, M) or Z0.shape != (B, H, D):
+        raise ValueError("state shape mismatch")
+    dQ, dK, dV = np.empty_like(Q), np.empty_like(K), np.empty_like(V)
+    dS0, dZ0 = np.empty((B, H, D, M)), np.empty((B, H, D))
+    _load().la_oracle_causal_backward_from_state(
+        B, H, N, D, M, PHI[phi], eps, _p(Q), _p(K), _p(V), _p(S0), _p(Z0), _p(G), _p(dSN), _p(dZN),
+        _p(dQ), _p(dK), _p(dV), _p(dS0), _p(dZ0))
+    return dQ, dK, dV, dS0, dZ0
 
 
 def linear_attention_backward(Q, K, V, G, causal: bool, phi: str = "elu1", eps: float = 0.0):

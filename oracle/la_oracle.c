@@ -399,6 +399,95 @@ void la_oracle_linear_backward(int64_t B, int64_t H, int64_t N, int64_t D, int64
 }
 
 /*
+ * Gradient of the causal form continued from a state (la_oracle_causal_from_state), for
+ *     L = sum_{i,e} G_ie O_ie + <dS_N, S_N> + <dZ_N, Z_N>,
+ * i.e. an upstream gradient on the outputs and (optionally, NULL = zero) on the final state, as
+ * needed when a sequence is processed, and differentiated, in several calls.  With the values
+ * extended by a constant 1 (see la_oracle_linear_backward) the state is st_i = [s_i | z_i],
+ * st_0 = [S0 | Z0], and Algorithm 1 "backward" applies with two changes only: the forward
+ * running sum starts from st_0, and the reverse running sum starts from the upstream gradient
+ * of the final state instead of zero:
+ *     St = [S0|Z0]; for i = 1..N: St += phi(K_i) [V_i,1]^T ; grad phi(Q_i) = St Gt_i       (Eq. 13)
+ *     Rt = [dS_N|dZ_N]; for i = N..1: Rt += phi(Q_i) Gt_i^T ;
+ *                       grad V_i = (Rt^T phi(K_i))[0:M] ; grad phi(K_i) = Rt [V_i,1]      (Eq. 14-15)
+ * and the state the call started from receives what is left in the reverse sum:
+ *     [dS0 | dZ0] = Rt after the sweep      (st_0 enters every st_i with coefficient one).
+ */
+void la_oracle_causal_backward_from_state(int64_t B, int64_t H, int64_t N, int64_t D, int64_t M,
+                                          int phi, double eps,
+                                          const double *Q, const double *K, const double *V,
+                                          const double *S0, const double *Z0,
+                                          const double *G, const double *dSN, const double *dZN,
+                                          double *dQ, double *dK, double *dV, double *dS0, double *dZ0)
+{
+    int64_t BH = B * H;
+    int64_t M1 = M + 1;
+#pragma omp parallel for schedule(dynamic)
+    for (int64_t bh = 0; bh < BH; ++bh) {
+        const double *Qh = Q + bh * N * D, *Kh = K + bh * N * D;
+        const double *Vh = V + bh * N * M, *Gh = G + bh * N * M;
+        double *dQh = dQ + bh * N * D, *dKh = dK + bh * N * D, *dVh = dV + bh * N * M;
+        double *q = mapped(Qh, N * D, phi);
+        double *k = mapped(Kh, N * D, phi);
+        double *St = (double *)calloc((size_t)(D * M1), sizeof(double));
+        double *Rt = (double *)calloc((size_t)(D * M1), sizeof(double));
+        double *Gt = (double *)malloc((size_t)(N > 0 ? N * M1 : 1) * sizeof(double));
+        for (int64_t d = 0; d < D; ++d) {
+            for (int64_t e = 0; e < M; ++e) {
+                St[d * M1 + e] = S0[bh * D * M + d * M + e];
+                if (dSN) Rt[d * M1 + e] = dSN[bh * D * M + d * M + e];
+            }
+            St[d * M1 + M] = Z0[bh * D + d];
+            if (dZN) Rt[d * M1 + M] = dZN[bh * D + d];
+        }
+        for (int64_t i = 0; i < N; ++i) {
+            for (int64_t d = 0; d < D; ++d) {
+                for (int64_t e = 0; e < M; ++e) St[d * M1 + e] += k[i * D + d] * Vh[i * M + e];
+                St[d * M1 + M] += k[i * D + d];
+            }
+            double dn = eps;
+            for (int64_t d = 0; d < D; ++d) dn += q[i * D + d] * St[d * M1 + M];
+            double go = 0.0;
+            for (int64_t e = 0; e < M; ++e) {
+                double num = 0.0;
+                for (int64_t d = 0; d < D; ++d) num += q[i * D + d] * St[d * M1 + e];
+                go += Gh[i * M + e] * (num / dn);
+                Gt[i * M1 + e] = Gh[i * M + e] / dn;
+            }
+            Gt[i * M1 + M] = -go / dn;
+            for (int64_t d = 0; d < D; ++d) {
+                double s = 0.0;
+                for (int64_t e = 0; e < M1; ++e) s += St[d * M1 + e] * Gt[i * M1 + e];
+                dQh[i * D + d] = s;
+            }
+        }
+        for (int64_t i = N - 1; i >= 0; --i) {
+            for (int64_t d = 0; d < D; ++d)
+                for (int64_t e = 0; e < M1; ++e) Rt[d * M1 + e] += q[i * D + d] * Gt[i * M1 + e];
+            for (int64_t e = 0; e < M; ++e) {
+                double s = 0.0;
+                for (int64_t d = 0; d < D; ++d) s += Rt[d * M1 + e] * k[i * D + d];
+                dVh[i * M + e] = s;
+            }
+            for (int64_t d = 0; d < D; ++d) {
+                double s = Rt[d * M1 + M];
+                for (int64_t e = 0; e < M; ++e) s += Rt[d * M1 + e] * Vh[i * M + e];
+                dKh[i * D + d] = s;
+            }
+        }
+        for (int64_t i = 0; i < N * D; ++i) {
+            dQh[i] *= phi_slope(Qh[i], phi);
+            dKh[i] *= phi_slope(Kh[i], phi);
+        }
+        for (int64_t d = 0; d < D; ++d) {
+            for (int64_t e = 0; e < M; ++e) dS0[bh * D * M + d * M + e] = Rt[d * M1 + e];
+            dZ0[bh * D + d] = Rt[d * M1 + M];
+        }
+        free(Gt); free(Rt); free(St); free(k); free(q);
+    }
+}
+
+/*
  * One recurrent step, Eq. 18-20 (attention part): the state is updated first
  * and read afterwards.   S += phi(k) v^T ; Z += phi(k) ;
  *                        out = phi(q)^T S / (phi(q)^T Z + eps).

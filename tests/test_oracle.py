@@ -247,6 +247,50 @@ def test_a_sequence_cut_in_two_calls_reproduces_the_definition(cut):
     assert np.allclose(Oz, ref, rtol=1e-11, atol=1e-12)
 
 
+def test_backward_from_state_matches_finite_differences():
+    # every argument, including the state the call starts from, with an upstream gradient on the final state
+    B, H, N, D, M = 1, 2, 6, 3, 2
+    Q, K, V, G = rnd((B, H, N, D), 51), rnd((B, H, N, D), 52), rnd((B, H, N, M), 53), rnd((B, H, N, M), 54)
+    S0, Z0 = rnd((B, H, D, M), 55), np.abs(rnd((B, H, D), 56)) + 1.0
+    dSN, dZN = rnd((B, H, D, M), 57), rnd((B, H, D), 58)
+
+    def loss(Q, K, V, S0, Z0):
+        O, _, SN, ZN = oracle.causal_from_state(Q, K, V, S0, Z0)
+        return (G * O).sum() + (dSN * SN).sum() + (dZN * ZN).sum()
+
+    grads = oracle.causal_backward_from_state(Q, K, V, S0, Z0, G, dSN, dZN)
+    args = [Q, K, V, S0, Z0]
+    h = 1e-6
+    for a, g in zip(range(5), grads):
+        x = args[a]
+        for idx in np.ndindex(x.shape):
+            up, dn = [t.copy() for t in args], [t.copy() for t in args]
+            up[a][idx] += h
+            dn[a][idx] -= h
+            fd = (loss(*up) - loss(*dn)) / (2 * h)
+            assert abs(fd - g[idx]) <= 1e-6 * max(1.0, abs(fd)), (a, idx, fd, g[idx])
+
+
+@pytest.mark.parametrize("cut", [1, 9, 22])
+def test_backward_chained_over_two_calls_equals_backward_of_the_whole(cut):
+    # the gradient of the whole sequence (a routine pinned to autograd through the N x N definition above)
+    # against two calls: the second part from the first part's final state, its state gradient fed to the first
+    B, H, N, D, M = 2, 2, 23, 5, 4
+    Q, K, V, G = rnd((B, H, N, D), 61), rnd((B, H, N, D), 62), rnd((B, H, N, M), 63), rnd((B, H, N, M), 64)
+    rq, rk, rv = oracle.linear_attention_backward(Q, K, V, G, True)
+    a, b = slice(0, cut), slice(cut, N)
+    _, _, S1, Z1 = oracle.linear_attention(Q[:, :, a], K[:, :, a], V[:, :, a], True, return_state=True)
+    q2, k2, v2, dS1, dZ1 = oracle.causal_backward_from_state(Q[:, :, b], K[:, :, b], V[:, :, b], S1, Z1, G[:, :, b])
+    zS, zZ = np.zeros((B, H, D, M)), np.zeros((B, H, D))
+    q1, k1, v1, dS0, dZ0 = oracle.causal_backward_from_state(Q[:, :, a], K[:, :, a], V[:, :, a], zS, zZ, G[:, :, a], dS1, dZ1)
+    for got, ref in ((np.concatenate([q1, q2], 2), rq), (np.concatenate([k1, k2], 2), rk), (np.concatenate([v1, v2], 2), rv)):
+        assert np.allclose(got, ref, rtol=1e-10, atol=1e-12)
+    # from a zero state and without a state gradient the routine is the causal backward itself
+    q0, k0, v0, _, _ = oracle.causal_backward_from_state(Q, K, V, zS, zZ, G)
+    assert np.allclose(q0, rq, rtol=1e-12, atol=1e-13) and np.allclose(k0, rk, rtol=1e-12, atol=1e-13)
+    assert np.allclose(v0, rv, rtol=1e-12, atol=1e-13)
+
+
 # ------------------------------------------------------------------- gradients
 def _torch_quadratic(Q, K, V, causal, eps=0.0, identity=False):
     phi = (lambda x: x) if identity else (lambda x: torch.nn.functional.elu(x) + 1)
