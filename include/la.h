@@ -132,9 +132,9 @@ int la_causal_forward(const la_problem* p, const void* Q, const void* K, const v
  * S_in [B,H,D,M] and Z_in [B,H,D]: device, fp32, 16-byte aligned, both given or both NULL (NULL:
  * the call is la_causal_forward()); they are only read and must not overlap S_out / Z_out
  * (LA_ERR_INVALID_ARG: the pieces of a sequence run concurrently and all start from S_in).  den
- * includes the Z_in term.  With N = 0 the state is copied to S_out / Z_out.  There is no backward
- * pass from a non-zero state in this library, so `saved` must be NULL when S_in is given
- * (LA_ERR_UNSUPPORTED).  Everything else as for la_causal_forward().
+ * includes the Z_in term.  With N = 0 the state is copied to S_out / Z_out.  `saved` as for
+ * la_causal_forward(): it is valid for la_causal_backward_from() with the same S_in, Z_in (the
+ * state itself is not kept in it).  Everything else as for la_causal_forward().
  */
 int la_causal_forward_from(const la_problem* p, const void* Q, const void* K, const void* V,
                            const float* S_in, const float* Z_in,
@@ -229,6 +229,29 @@ int la_last_device_status(void* stream);
  *                                              sequence b % (B*H)) }.
  */
 int la_causal_plan(const la_problem* p, int32_t* out, int capacity);
+
+/*
+ * Gradient of the causal form continued from a state, for
+ *   L = sum G . O + <dS_out, S_N> + <dZ_out, Z_N>
+ * (an upstream gradient on the outputs and, optionally, on the final state: what a sequence
+ * processed and differentiated in several calls needs).  Algorithm 1 (backward) with two changes:
+ * the forward running sum starts from [S_in | Z_in] and the reverse running sum from
+ * [dS_out | dZ_out]; what is left in the reverse sum after the sweep is the gradient of the state
+ * the call started from, written to dS_in [B,H,D,M] and dZ_in [B,H,D] (fp32; either may be NULL:
+ * not wanted).  S_in / Z_in: both or neither (NULL: zero state).  dS_out / dZ_out: each may be NULL
+ * (zero).  All state pointers are device, fp32, 16-byte aligned; dS_in / dZ_in must not overlap
+ * dS_out / dZ_out (LA_ERR_INVALID_ARG: the pieces of a sequence run concurrently and all start from
+ * the upstream gradient).  With N = 0 the upstream state gradient is copied to dS_in / dZ_in (zeros
+ * when it is NULL).  Everything else as for la_causal_backward(), which is this call with every
+ * state pointer NULL.
+ */
+int la_causal_backward_from(const la_problem* p, const void* Q, const void* K, const void* V,
+                            const float* S_in, const float* Z_in,
+                            const void* O, const float* den, const void* G,
+                            const float* dS_out, const float* dZ_out,
+                            const void* saved, size_t saved_bytes,
+                            void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
+                            void* ws, size_t ws_bytes, void* stream);
 
 /* Number of GPU kernels this library has enqueued in this process so far (all
  * threads, all entry points); a diagnostic for benchmarks. */

@@ -22,7 +22,7 @@ _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
     "la_feature_map", "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
-    "la_causal_forward", "la_causal_forward_from",
+    "la_causal_forward", "la_causal_forward_from", "la_causal_backward_from",
     "la_causal_backward", "la_recurrent_step", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
     "la_profile_kernel_name", "la_version", "la_causal_plan",
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.la_linear_attention_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
         L.la_causal_forward.argtypes = [pp] + [vp] * 7 + [vp, sz] + [vp, sz, vp]
         L.la_causal_forward_from.argtypes = [pp] + [vp] * 9 + [vp, sz] + [vp, sz, vp]
+        L.la_causal_backward_from.argtypes = [pp] + [vp] * 10 + [vp, sz] + [vp] * 5 + [vp, sz, vp]
         L.la_causal_backward.argtypes = [pp] + [vp] * 6 + [vp, sz] + [vp] * 3 + [vp, sz, vp]
         L.la_recurrent_step.argtypes = [pp] + [vp] * 6 + [vp]
         L.la_workspace_bytes.argtypes = [pp, i32]
@@ -277,16 +278,29 @@ def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None
 
 
 def la_causal_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None, saved=None, dQ=None, dK=None, dV=None,
-                       ws=None):
-    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved)
+                       ws=None, S_in=None, Z_in=None, dS_out=None, dZ_out=None, dS_in=None, dZ_in=None):
+    """Gradients of the causal form; returns (dQ, dK, dV).  With any of the state arguments (fp32 [B,H,D,M] /
+    [B,H,D]: the state the forward started from, the upstream gradient of its final state, and tensors that
+    receive the gradient of the initial state) the call is la_causal_backward_from."""
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved, S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in)
     p = _problem_of(Q, V, phi, eps)
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(V) if dV is None else dV
     ws = workspace(p, LA_OP_CAUSAL_BACKWARD, dev) if ws is None else ws
-    _check(lib().la_causal_backward(
-        ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(saved), _nbytes(saved),
-        _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), _nbytes(ws), _stream(dev)))
+    state = (S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in)
+    if all(t is None for t in state):
+        _check(lib().la_causal_backward(
+            ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(saved), _nbytes(saved),
+            _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), _nbytes(ws), _stream(dev)))
+    else:
+        for t, shape in zip(state, ((p.B, p.H, p.D, p.M), (p.B, p.H, p.D)) * 3):
+            if t is not None and (t.dtype != torch.float32 or tuple(t.shape) != shape or not t.is_contiguous()):
+                raise ValueError("state arguments must be contiguous fp32 tensors of shape [B,H,D,M] / [B,H,D]")
+        _check(lib().la_causal_backward_from(
+            ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(S_in), _ptr(Z_in), _ptr(O), _ptr(den), _ptr(G),
+            _ptr(dS_out), _ptr(dZ_out), _ptr(saved), _nbytes(saved), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dS_in), _ptr(dZ_in),
+            _ptr(ws), _nbytes(ws), _stream(dev)))
     return dQ, dK, dV
 
 

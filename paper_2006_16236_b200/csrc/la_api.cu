@@ -246,7 +246,6 @@ int la_causal_forward_from(const la_problem* p, const void* Q, const void* K, co
     if (overlaps(S_in, s_bytes, S_out, s_bytes) || overlaps(S_in, s_bytes, Z_out, z_bytes) ||
         overlaps(Z_in, z_bytes, S_out, s_bytes) || overlaps(Z_in, z_bytes, Z_out, z_bytes))
         return fail(LA_ERR_INVALID_ARG, "S_in / Z_in overlap S_out / Z_out");
-    if (S_in && saved) return fail(LA_ERR_UNSUPPORTED, "no backward pass from a non-zero state: saved must be NULL with S_in");
     cudaStream_t st = (cudaStream_t)stream;
     if (p->N == 0) {
         if (S_in && S_out) LA_CUDA_TRY(cudaMemcpyAsync(S_out, S_in, s_bytes, cudaMemcpyDeviceToDevice, st));
@@ -270,23 +269,53 @@ int la_causal_forward(const la_problem* p, const void* Q, const void* K, const v
     return la_causal_forward_from(p, Q, K, V, nullptr, nullptr, O, den, S_out, Z_out, saved, saved_bytes, ws, ws_bytes, stream);
 }
 
-int la_causal_backward(const la_problem* p, const void* Q, const void* K, const void* V,
-                       const void* O, const float* den, const void* G,
-                       const void* saved, size_t saved_bytes,
-                       void* dQ, void* dK, void* dV,
-                       void* ws, size_t ws_bytes, void* stream) {
+int la_causal_backward_from(const la_problem* p, const void* Q, const void* K, const void* V,
+                            const float* S_in, const float* Z_in,
+                            const void* O, const float* den, const void* G,
+                            const float* dS_out, const float* dZ_out,
+                            const void* saved, size_t saved_bytes,
+                            void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
+                            void* ws, size_t ws_bytes, void* stream) {
     if (int rc = check_problem(p, true)) return rc;
-    if (p->N == 0) return LA_OK;
+    if ((S_in == nullptr) != (Z_in == nullptr)) return fail(LA_ERR_INVALID_ARG, "S_in and Z_in must both be given or both be NULL");
+    LA_OPTIONAL_PTR(S_in); LA_OPTIONAL_PTR(Z_in); LA_OPTIONAL_PTR(dS_out); LA_OPTIONAL_PTR(dZ_out);
+    LA_OPTIONAL_PTR(dS_in); LA_OPTIONAL_PTR(dZ_in);
+    const size_t s_bytes = (size_t)(p->B * p->H * p->D * p->M) * sizeof(float), z_bytes = (size_t)(p->B * p->H * p->D) * sizeof(float);
+    if (overlaps(dS_out, s_bytes, dS_in, s_bytes) || overlaps(dS_out, s_bytes, dZ_in, z_bytes) ||
+        overlaps(dZ_out, z_bytes, dS_in, s_bytes) || overlaps(dZ_out, z_bytes, dZ_in, z_bytes))
+        return fail(LA_ERR_INVALID_ARG, "dS_in / dZ_in overlap dS_out / dZ_out");
+    cudaStream_t st = (cudaStream_t)stream;
+    if (p->N == 0) {            // nothing between the two states: the gradient passes through
+        if (dS_in) {
+            if (dS_out) LA_CUDA_TRY(cudaMemcpyAsync(dS_in, dS_out, s_bytes, cudaMemcpyDeviceToDevice, st));
+            else LA_CUDA_TRY(cudaMemsetAsync(dS_in, 0, s_bytes, st));
+        }
+        if (dZ_in) {
+            if (dZ_out) LA_CUDA_TRY(cudaMemcpyAsync(dZ_in, dZ_out, z_bytes, cudaMemcpyDeviceToDevice, st));
+            else LA_CUDA_TRY(cudaMemsetAsync(dZ_in, 0, z_bytes, st));
+        }
+        return LA_OK;
+    }
     LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(G);
     LA_REQUIRE_PTR(dQ); LA_REQUIRE_PTR(dK); LA_REQUIRE_PTR(dV);
     LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(saved);
     if (int rc = check_ws(p, LA_OP_CAUSAL_BACKWARD, ws, ws_bytes)) return rc;
     if (int rc = check_saved(p, saved, saved_bytes)) return rc;
     if (int rc = check_arch()) return rc;
-    cudaStream_t st = (cudaStream_t)stream;
+    StateArgs sa;
+    sa.S_in = S_in; sa.Z_in = Z_in; sa.dS_out = dS_out; sa.dZ_out = dZ_out; sa.dS_in = dS_in; sa.dZ_in = dZ_in;
     if (tc_supported(*p, LA_OP_CAUSAL_BACKWARD))
-        return tc_causal_backward(*p, Q, K, V, O, den, G, saved, dQ, dK, dV, ws, st);
-    return general_causal_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
+        return tc_causal_backward(*p, Q, K, V, O, den, G, sa, saved, dQ, dK, dV, ws, st);
+    return general_causal_backward(*p, Q, K, V, G, sa, dQ, dK, dV, ws, st);
+}
+
+int la_causal_backward(const la_problem* p, const void* Q, const void* K, const void* V,
+                       const void* O, const float* den, const void* G,
+                       const void* saved, size_t saved_bytes,
+                       void* dQ, void* dK, void* dV,
+                       void* ws, size_t ws_bytes, void* stream) {
+    return la_causal_backward_from(p, Q, K, V, nullptr, nullptr, O, den, G, nullptr, nullptr, saved, saved_bytes,
+                                   dQ, dK, dV, nullptr, nullptr, ws, ws_bytes, stream);
 }
 
 int la_recurrent_step(const la_problem* p, const void* q, const void* k, const void* v,

@@ -73,13 +73,26 @@ int launch_feature_map(const void* x, void* y, int64_t n, int dtype, int deriv, 
 int launch_recurrent_step(const la_problem& p, const void* q, const void* k, const void* v,
                           float* S, float* Z, void* out, cudaStream_t st);
 
+// State arguments of the causal backward pass (device, fp32, any of them may be null): the state the
+// forward started from, the upstream gradient of the final state, and where the gradient of the
+// initial state goes.  S: [B,H,D,M], Z: [B,H,D].
+struct StateArgs {
+    const float* S_in = nullptr;
+    const float* Z_in = nullptr;
+    const float* dS_out = nullptr;
+    const float* dZ_out = nullptr;
+    float* dS_in = nullptr;
+    float* dZ_in = nullptr;
+};
+
 // General (any D, M multiple of 8 up to 128, any N) fp32-arithmetic kernels.
 size_t general_workspace_bytes(const la_problem& p, int op);
 int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V,
                            const float* S_in, const float* Z_in,
                            void* O, float* den, float* S_out, float* Z_out, cudaStream_t st);
 int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V,
-                            const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+                            const void* G, const StateArgs& sa, void* dQ, void* dK, void* dV, void* ws,
+                            cudaStream_t st);
 int general_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V,
                            void* O, float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
 int general_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V,

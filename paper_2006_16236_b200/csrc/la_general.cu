@@ -190,8 +190,8 @@ general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K
 template <typename IO>
 __global__ void __launch_bounds__(THREADS)
 general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K, const IO* __restrict__ V,
-                               const IO* __restrict__ G, IO* __restrict__ dQ, IO* __restrict__ dK,
-                               IO* __restrict__ dV, float* __restrict__ aux,
+                               const IO* __restrict__ G, const StateArgs sa, IO* __restrict__ dQ,
+                               IO* __restrict__ dK, IO* __restrict__ dV, float* __restrict__ aux,
                                int64_t N, int D, int M, float eps, int phi) {
     extern __shared__ float smem[];
     const Dims dm = make_dims(D, M);
@@ -210,8 +210,14 @@ general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ 
     float* dn_all = aux + bh * N * 2;
     float* delta_all = dn_all + N;
 
-    // ---- forward sweep: St = running sum of phi(K_j) Vt_j^T -------------------
+    // ---- forward sweep: St = running sum of phi(K_j) Vt_j^T (from the given state, if any) ----
     zero_fill(sSt, D * dm.MS);
+    if (sa.S_in) {
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < D * M; idx += THREADS)
+            sSt[(idx / M) * dm.MS + idx % M] = sa.S_in[bh * D * M + idx];
+        for (int d = threadIdx.x; d < D; d += THREADS) sSt[d * dm.MS + M] = sa.Z_in[bh * D + d];
+    }
     for (int64_t n0 = 0; n0 < N; n0 += T) {
         const int cn = (int)((N - n0) < T ? (N - n0) : T);
         __syncthreads();
@@ -240,9 +246,18 @@ general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ 
         state_update(sSt, sk, sv, dm);
     }
 
-    // ---- reverse sweep: Rt = running sum (from the end) of phi(Q_j) Gt_j^T ----
+    // ---- reverse sweep: Rt = running sum (from the end) of phi(Q_j) Gt_j^T, started from the upstream
+    // ---- gradient of the final state, if any ----
     __syncthreads();
     zero_fill(sSt, D * dm.MS);
+    if (sa.dS_out || sa.dZ_out) {
+        __syncthreads();
+        if (sa.dS_out)
+            for (int idx = threadIdx.x; idx < D * M; idx += THREADS)
+                sSt[(idx / M) * dm.MS + idx % M] = sa.dS_out[bh * D * M + idx];
+        if (sa.dZ_out)
+            for (int d = threadIdx.x; d < D; d += THREADS) sSt[d * dm.MS + M] = sa.dZ_out[bh * D + d];
+    }
     const int64_t nchunks = (N + T - 1) / T;
     for (int64_t c = nchunks - 1; c >= 0; --c) {
         const int64_t n0 = c * T;
@@ -281,6 +296,13 @@ general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ 
         __syncthreads();
         state_update(sSt, sq, sg, dm);
     }
+    // what is left in the reverse sum is the gradient of the state the sequence started from
+    __syncthreads();
+    if (sa.dS_in)
+        for (int idx = threadIdx.x; idx < D * M; idx += THREADS)
+            sa.dS_in[bh * D * M + idx] = sSt[(idx / M) * dm.MS + idx % M];
+    if (sa.dZ_in)
+        for (int d = threadIdx.x; d < D; d += THREADS) sa.dZ_in[bh * D + d] = sSt[d * dm.MS + M];
 }
 
 // ---------------------------------------------------------------------------
@@ -499,11 +521,12 @@ int general_causal_forward(const la_problem& p, const void* Q, const void* K, co
 
 template <typename IO>
 static int causal_backward_t(const la_problem& p, const void* Q, const void* K, const void* V,
-                             const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+                             const void* G, const StateArgs& sa, void* dQ, void* dK, void* dV, void* ws,
+                             cudaStream_t st) {
     const size_t smem = smem_floats_backward((int)p.D, (int)p.M) * sizeof(float);
     auto kern = general_causal_backward_kernel<IO>;
     if (int rc = opt_in_smem(kern, smem)) return rc;
-    kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, (const IO*)G,
+    kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, (const IO*)G, sa,
                                                        (IO*)dQ, (IO*)dK, (IO*)dV, (float*)ws, p.N, (int)p.D,
                                                        (int)p.M, p.eps, p.phi);
     LA_LAUNCHED();
@@ -511,9 +534,9 @@ static int causal_backward_t(const la_problem& p, const void* Q, const void* K, 
 }
 
 int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
-                            void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
-    return p.dtype == LA_F32 ? causal_backward_t<float>(p, Q, K, V, G, dQ, dK, dV, ws, st)
-                             : causal_backward_t<__nv_bfloat16>(p, Q, K, V, G, dQ, dK, dV, ws, st);
+                            const StateArgs& sa, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    return p.dtype == LA_F32 ? causal_backward_t<float>(p, Q, K, V, G, sa, dQ, dK, dV, ws, st)
+                             : causal_backward_t<__nv_bfloat16>(p, Q, K, V, G, sa, dQ, dK, dV, ws, st);
 }
 
 template <typename IO>

@@ -73,10 +73,10 @@ int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const v
     return tc::causal_forward(p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
 }
 int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* O,
-                       const float* den, const void* G, const void* saved, void* dQ, void* dK, void* dV, void* ws,
-                       cudaStream_t st) {
+                       const float* den, const void* G, const StateArgs& sa, const void* saved, void* dQ, void* dK,
+                       void* dV, void* ws, cudaStream_t st) {
     (void)O; (void)den;      // everything needed is recomputed consistently
-    return tc::causal_backward(p, Q, K, V, G, saved, dQ, dK, dV, ws, st);
+    return tc::causal_backward(p, Q, K, V, G, sa, saved, dQ, dK, dV, ws, st);
 }
 int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
                       float* KV, float* Zs, void* ws, cudaStream_t st) {

@@ -15,8 +15,8 @@ int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const v
                       const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
                       cudaStream_t st);
 int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* O,
-                       const float* den, const void* G, const void* saved, void* dQ, void* dK, void* dV, void* ws,
-                       cudaStream_t st);
+                       const float* den, const void* G, const StateArgs& sa, const void* saved, void* dQ, void* dK,
+                       void* dV, void* ws, cudaStream_t st);
 int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
                       float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
 int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
@@ -30,7 +30,7 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
                    cudaStream_t st);
 size_t causal_backward_workspace(const la_problem& p);
 int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
-                    const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+                    const StateArgs& sa, const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 size_t linear_forward_workspace(const la_problem& p);
 size_t linear_backward_workspace(const la_problem& p);
 int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,

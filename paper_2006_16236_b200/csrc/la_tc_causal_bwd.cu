@@ -89,6 +89,8 @@ struct DqParams {
     float* dn;                  // out: dn_i = q_i . Z_i + eps per row, for the reverse sweep
     float* dl;                  // out: dl_i = -(G_i . O_i) per row, for the reverse sweep
     const float* init;          // per (bh, part) [S|Z] records of the pre-pass, or null (single piece)
+    const float* S_in;          // [BH, D, M] / [BH, D] state the sequence started from, or null (zero)
+    const float* Z_in;
     CausalPlan plan;            // pieces of a sequence and their pre-pass parts
     int* status;
     int64_t N;
@@ -279,7 +281,9 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         const int t = tid - 8 * 32;
         const uint32_t r7 = t & 7;
         const float* rec = prm.init ? prm.init + bh * (int64_t)plan.nparts() * kStateFloats : nullptr;
-        state_init(tmem + kDqColS, quad, lane, smem + kDqOffS, sZ + 2 * 64, rec, 0, rec ? plan.piece_first_part(piece) : 0);   // "chunk -1" -> Z buffer 2
+        state_init(tmem + kDqColS, quad, lane, smem + kDqOffS, sZ + 2 * 64, rec, 0, rec ? plan.piece_first_part(piece) : 0,
+                   prm.S_in ? prm.S_in + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
+                   prm.Z_in ? prm.Z_in + bh * prm.dim : nullptr, prm.dim);   // "chunk -1" -> Z buffer 2
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(&bars->state_ready);
@@ -509,6 +513,10 @@ struct KvParams {
     const float* dn;            // dn_i from the forward sweep
     const float* dl;            // dl_i = -(G_i . O_i) from the forward sweep
     const float* init;          // per (bh, part) [R | r] records of the pre-pass, or null (single piece)
+    const float* dS_out;        // [BH, D, M] / [BH, D] upstream gradient of the final state, or null (zero)
+    const float* dZ_out;
+    float* dS_in;               // [BH, D, M] / [BH, D] gradient of the state the sequence started from, or null
+    float* dZ_in;
     CausalPlan plan;            // pieces of a sequence and their pre-pass parts
     int* status;
     int64_t N;
@@ -768,7 +776,11 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const float* rec = prm.init ? prm.init + bh * (int64_t)plan.nparts() * kStateFloats : nullptr;
         const float slope_floor = prm.phi == LA_PHI_ELU1 ? 0.f : 1.f;
         rstate_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, rec, rec ? plan.piece_first_part(piece + 1) : 0,
-                   rec ? plan.nparts() : 0);                                     // "iteration -1" -> buffer 1
+                   rec ? plan.nparts() : 0);
+        if (prm.dS_out || prm.dZ_out)       // upstream gradient of the final state: every piece's reverse sum starts from it
+            state_add_given<false>(tmem + kKvColR, quad, lane, smem + kKvOffR, nullptr, sRv + 64,
+                                   prm.dS_out ? prm.dS_out + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
+                                   prm.dZ_out ? prm.dZ_out + bh * prm.dim : nullptr, prm.dim);                                     // "iteration -1" -> buffer 1
         fence_proxy_async_smem();
         tc_fence_before_sync();
         named_barrier(1, 128);
@@ -869,6 +881,11 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             }
             if (t == 0) LA_TRACE(g_trace_dkv, i, 10);
         }
+        // after the first chunk of the sequence the reverse sum is the gradient of the state the sequence started
+        // from (the last conversion above waited for its final update)
+        if (piece == 0 && (prm.dS_in || prm.dZ_in))
+            rstate_write(tmem + kKvColR, quad, lane, prm.dS_in ? prm.dS_in + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
+                         prm.dZ_in ? prm.dZ_in + bh * prm.dim : nullptr, prm.dim);
         if (t == 0) tma_store_wait_all<0>();
     } else {
         // ------------------------------------------- score warps: Ph^T and dP^T, masked and rounded in place
@@ -907,7 +924,7 @@ size_t causal_backward_workspace(const la_problem& p) {
 }
 
 int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
-                    const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+                    const StateArgs& sa, const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
     const CausalPlan pl = choose_plan(p);
     // With what the forward saved, phi(Q) and phi(K) are read as tensors (no feature map on load)
     // and the forward pre-pass records are the forward's own.
@@ -952,6 +969,8 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.dn = dn;
     a.dl = dl;
     a.init = pl.npieces() > 1 ? rec_s : nullptr;
+    a.S_in = sa.S_in;
+    a.Z_in = sa.Z_in;
     a.plan = pl;
     a.status = status;
     a.N = p.N;
@@ -972,6 +991,10 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     b.dn = dn;
     b.dl = dl;
     b.init = pl.npieces() > 1 ? rec_r : nullptr;
+    b.dS_out = sa.dS_out;
+    b.dZ_out = sa.dZ_out;
+    b.dS_in = sa.dS_in;
+    b.dZ_in = sa.dZ_in;
     b.plan = pl;
     b.status = status;
     b.N = p.N;

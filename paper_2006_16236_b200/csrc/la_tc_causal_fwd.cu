@@ -307,9 +307,10 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         const uint32_t r7 = t & 7;
         const float* rec = prm.init ? prm.init + bh * (int64_t)plan.nparts() * kStateFloats : nullptr;
         uint8_t* tile1 = smem + kOffS + kStateTileBytes;            // the state before chunk 0 lives in tile 1
-        state_init_tiles(tmem + kColS, quad, lane, tile1, tile1 + kDim * 128, rec, 0, rec ? plan.piece_first_part(piece) : 0,
-                         prm.S_in ? prm.S_in + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
-                         prm.Z_in ? prm.Z_in + bh * prm.dim : nullptr, prm.dim);
+        state_init_tiles(tmem + kColS, quad, lane, tile1, tile1 + kDim * 128, rec, 0, rec ? plan.piece_first_part(piece) : 0);
+        if (prm.S_in)           // the sequence continues from a given state: every piece starts from it
+            state_add_given<true>(tmem + kColS, quad, lane, tile1, tile1 + kDim * 128, nullptr,
+                                  prm.S_in + bh * (int64_t)(prm.dim * prm.dim), prm.Z_in + bh * prm.dim, prm.dim);
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(&bars->state_ready[1]);

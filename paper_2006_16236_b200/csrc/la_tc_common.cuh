@@ -299,15 +299,19 @@ __device__ __forceinline__ float sum_records1(const float* rec, int part_lo, int
 
 // Initial state of a segment: the sum of the records of parts [part_lo, part_hi) of this
 // (batch, head) (none: zeros) goes into the TMEM state accumulator, its bf16 tile and z_out.
+// s_in / z_in (or null): the [dim][dim] / [dim] fp32 state of this (batch, head) the sequence continues from.
 __device__ __forceinline__ void state_init(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, float* z_out,
-                                           const float* rec, int part_lo, int part_hi) {
+                                           const float* rec, int part_lo, int part_hi,
+                                           const float* s_in = nullptr, const float* z_in = nullptr, int dim = kDim) {
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
+    const bool in_row = owner && s_in && d_row < dim;
 #pragma unroll 1
     for (int g = 0; g < 4; ++g) {
         float acc[16];
-        sum_records16(rec, owner ? part_lo : 0, owner ? part_hi : 0, d_row * kDim + g * 16, acc);
+        sum_records16(rec, owner ? part_lo : 0, owner ? part_hi : 0, d_row * kDim + g * 16, acc,
+                      in_row && g * 16 < dim ? s_in + d_row * dim + g * 16 : nullptr);
         uint32_t v[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(acc[j]);
@@ -320,7 +324,7 @@ __device__ __forceinline__ void state_init(uint32_t tmem_state, int quad, int la
                        sm100::pack_bf16x2(acc[cc * 8 + 4], acc[cc * 8 + 5]), sm100::pack_bf16x2(acc[cc * 8 + 6], acc[cc * 8 + 7]));
         }
     }
-    const float z = owner ? sum_records1(rec, part_lo, part_hi, kDim * kDim + d_row) : 0.f;
+    const float z = (owner ? sum_records1(rec, part_lo, part_hi, kDim * kDim + d_row) : 0.f) + (in_row ? __ldg(z_in + d_row) : 0.f);
     uint32_t zz[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) zz[j] = __float_as_uint(z);
@@ -383,19 +387,15 @@ __device__ __forceinline__ void state_half_to_tiles(uint32_t tmem_state, int qua
 
 // Initial state of a segment (sum of the records of parts [part_lo, part_hi), or zeros) into
 // the TMEM accumulator (S in 64 columns, Z replicated in 16) and the bf16 tiles.
-// s_in / z_in (or null): the [dim][dim] / [dim] fp32 state of this (batch, head) the sequence continues from.
 __device__ __forceinline__ void state_init_tiles(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, uint8_t* z_tile,
-                                                 const float* rec, int part_lo, int part_hi,
-                                                 const float* s_in = nullptr, const float* z_in = nullptr, int dim = kDim) {
+                                                 const float* rec, int part_lo, int part_hi) {
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const int d_row = quad * 16 + lane;
     const bool owner = lane < 16;
-    const bool in_row = owner && s_in && d_row < dim;
 #pragma unroll 1
     for (int g = 0; g < 4; ++g) {
         float acc[16];
-        sum_records16(rec, owner ? part_lo : 0, owner ? part_hi : 0, d_row * kDim + g * 16, acc,
-                      in_row && g * 16 < dim ? s_in + d_row * dim + g * 16 : nullptr);
+        sum_records16(rec, owner ? part_lo : 0, owner ? part_hi : 0, d_row * kDim + g * 16, acc);
         uint32_t v[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(acc[j]);
@@ -408,13 +408,88 @@ __device__ __forceinline__ void state_init_tiles(uint32_t tmem_state, int quad, 
                        sm100::pack_bf16x2(acc[cc * 8 + 4], acc[cc * 8 + 5]), sm100::pack_bf16x2(acc[cc * 8 + 6], acc[cc * 8 + 7]));
         }
     }
-    const float z = (owner ? sum_records1(rec, part_lo, part_hi, kDim * kDim + d_row) : 0.f) + (in_row ? __ldg(z_in + d_row) : 0.f);
+    const float z = owner ? sum_records1(rec, part_lo, part_hi, kDim * kDim + d_row) : 0.f;
     uint32_t zz[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) zz[j] = __float_as_uint(z);
     sm100::tmem_st16(tmem_state + lane_base + 64, zz);
     sm100::tmem_st_wait();
     if (owner) z_row_store(z_tile, d_row, z);
+}
+
+// A state given by the caller ([dim][dim] and [dim] fp32 of this (batch, head): the state a sequence continues
+// from, or the upstream gradient of its final state) added to a freshly initialised accumulator and its
+// bf16 tile.  Out of line and only called when such a state is given: the kernels' own code keeps its shape.
+// kForward: the 65th column is replicated over 16 columns and mirrored in `z_tile`; else it lives in column 64
+// alone and is mirrored in `r_out`.
+template <bool kForward>
+__device__ __noinline__ void state_add_given(uint32_t tmem_state, int quad, int lane, uint8_t* s_tile, uint8_t* z_tile,
+                                             float* r_out, const float* s_in, const float* z_in, int dim) {
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const int d_row = quad * 16 + lane;
+    const bool owner = lane < 16;
+    const bool in_row = owner && d_row < dim;
+    sm100::tc_fence_after_sync();
+#pragma unroll 1
+    for (int g = 0; g < 4; ++g) {
+        uint32_t v[16];
+        sm100::tmem_ld16(tmem_state + lane_base + g * 16, v);
+        sm100::tmem_ld_wait();
+        float acc[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) acc[j] = __uint_as_float(v[j]);
+        if (in_row && s_in && g * 16 < dim) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float4 b = __ldg(reinterpret_cast<const float4*>(s_in + d_row * dim + g * 16) + j);
+                acc[4 * j] += b.x; acc[4 * j + 1] += b.y; acc[4 * j + 2] += b.z; acc[4 * j + 3] += b.w;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(acc[j]);
+        sm100::tmem_st16(tmem_state + lane_base + g * 16, v);
+        if (owner) {
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc)
+                sts128(s_tile + d_row * 128 + (((2 * g + cc) ^ (d_row & 7)) << 4),
+                       sm100::pack_bf16x2(acc[cc * 8 + 0], acc[cc * 8 + 1]), sm100::pack_bf16x2(acc[cc * 8 + 2], acc[cc * 8 + 3]),
+                       sm100::pack_bf16x2(acc[cc * 8 + 4], acc[cc * 8 + 5]), sm100::pack_bf16x2(acc[cc * 8 + 6], acc[cc * 8 + 7]));
+        }
+    }
+    float z = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 64));
+    sm100::tmem_ld_wait();
+    if (in_row && z_in) z += __ldg(z_in + d_row);
+    uint32_t zz[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) zz[j] = (kForward || j == 0) ? __float_as_uint(z) : 0u;
+    sm100::tmem_st16(tmem_state + lane_base + 64, zz);
+    sm100::tmem_st_wait();
+    if (owner) {
+        if (kForward) z_row_store(z_tile, d_row, z); else r_out[d_row] = z;
+    }
+}
+
+// The reverse-sweep state [R | r] of the accumulator to global memory ([dim][dim] and [dim] fp32): after the
+// first chunk of a sequence it is the gradient of the state the sequence started from.  Out of line, called once.
+static __device__ __noinline__ void rstate_write(uint32_t tmem_state, int quad, int lane, float* g_R, float* g_r, int dim) {
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const int d_row = quad * 16 + lane;
+    const bool in_row = lane < 16 && d_row < dim;
+    sm100::tc_fence_after_sync();
+#pragma unroll 1
+    for (int g = 0; g < 4; ++g) {
+        uint32_t v[16];
+        sm100::tmem_ld16(tmem_state + lane_base + g * 16, v);
+        sm100::tmem_ld_wait();
+        if (g_R && in_row && g * 16 < dim) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) g_R[d_row * dim + g * 16 + j] = __uint_as_float(v[j]);
+        }
+    }
+    const float r0 = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 64));
+    const float r1 = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 65));
+    sm100::tmem_ld_wait();
+    if (g_r && in_row) g_r[d_row] = r0 + r1;
 }
 
 // One 32-column block of fp32 scores -> 16 packed bf16 pairs (pair j = columns 2j, 2j+1), with

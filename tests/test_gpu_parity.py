@@ -225,6 +225,63 @@ def test_chunked_prefill_then_decode(dtype, D, chunks):
     assert_close(last, ref[:, :, N], dtype, "decode after chunked prefill")
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("keep", [False, True], ids=["recompute", "saved"])
+@pytest.mark.parametrize("shape", [(2, 3, 100, 16, 48), (1, 2, 31, 64, 64), (2, 2, 640, 32, 32), (4, 16, 18 * 128, 64, 64)])
+def test_causal_backward_from_a_state(shape, keep, dtype):
+    """Algorithm 1 (backward) with the forward sum started from [S_0 | Z_0] and the reverse sum from an upstream
+    gradient of the final state; the gradient of the initial state is what the reverse sum ends with."""
+    B, H, N, D, M = shape
+    Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=sum(shape) + 2, dtype=dtype)
+    g = torch.Generator().manual_seed(6)
+    S0 = torch.randn((B, H, D, M), generator=g) * 3.0
+    Z0 = torch.rand((B, H, D), generator=g) * 4.0 + 1.0
+    dSN = torch.randn((B, H, D, M), generator=g) * 0.05
+    dZN = torch.randn((B, H, D), generator=g) * 0.05
+    Qd, Kd, Vd, Gd, S0d, Z0d, dSNd, dZNd = gpu(Q, K, V, G, S0, Z0, dSN, dZN)
+    dS0 = torch.empty((B, H, D, M), device=DEV)
+    dZ0 = torch.empty((B, H, D), device=DEV)
+    saved = la.saved_buffer(Qd, Vd) if keep else None
+    if keep and saved is None:
+        pytest.skip("no saved buffer for problems on the general kernels")
+    if keep:
+        la.la_causal_forward(Qd, Kd, Vd, S_in=S0d, Z_in=Z0d, saved=saved)
+    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd, saved=saved, S_in=S0d, Z_in=Z0d, dS_out=dSNd, dZ_out=dZNd,
+                                       dS_in=dS0, dZ_in=dZ0)
+    la.la_last_device_status()
+    sel = [(0, 0), (B - 1, H - 1)] if B * H > 8 else [(b, h) for b in range(B) for h in range(H)]
+    for b, h in sel:
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        rq, rk, rv, rS, rZ = oracle.causal_backward_from_state(
+            Q[sl], K[sl], V[sl], S0[sl].double().numpy(), Z0[sl].double().numpy(), G[sl],
+            dSN[sl].double().numpy(), dZN[sl].double().numpy())
+        assert_close(dQ[sl], rq, dtype, f"dQ[{b},{h}]", grad=True)
+        assert_close(dK[sl], rk, dtype, f"dK[{b},{h}]", grad=True)
+        assert_close(dV[sl], rv, dtype, f"dV[{b},{h}]", grad=True)
+        assert_close(dS0[sl], rS, dtype, f"dS_0[{b},{h}]", grad=True)
+        assert_close(dZ0[sl], rZ, dtype, f"dZ_0[{b},{h}]", grad=True)
+
+
+def test_backward_chained_over_two_calls():
+    """A sequence processed and differentiated in two calls (the state and its gradient handed across) against
+    the oracle's gradient of the whole sequence."""
+    B, H, N, D, cut = 2, 4, 3072, 64, 1280
+    Q, K, V, G = draw_qkvg(B, H, N, D, D, seed=23, dtype=torch.bfloat16)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    a, b = slice(0, cut), slice(cut, N)
+    part = lambda t, s: t[:, :, s].contiguous()
+    S1 = torch.empty((B, H, D, D), device=DEV)
+    Z1 = torch.empty((B, H, D), device=DEV)
+    dS1, dZ1 = torch.empty_like(S1), torch.empty_like(Z1)
+    la.la_causal_forward(part(Qd, a), part(Kd, a), part(Vd, a), S_out=S1, Z_out=Z1)
+    q2, k2, v2 = la.la_causal_backward(part(Qd, b), part(Kd, b), part(Vd, b), part(Gd, b), S_in=S1, Z_in=Z1, dS_in=dS1, dZ_in=dZ1)
+    q1, k1, v1 = la.la_causal_backward(part(Qd, a), part(Kd, a), part(Vd, a), part(Gd, a), dS_out=dS1, dZ_out=dZ1)
+    la.la_last_device_status()
+    rq, rk, rv = oracle.linear_attention_backward(Q, K, V, G, True)
+    for got, ref, nm in ((torch.cat([q1, q2], 2), rq, "dQ"), (torch.cat([k1, k2], 2), rk, "dK"), (torch.cat([v1, v2], 2), rv, "dV")):
+        assert_close(got, ref, torch.bfloat16, nm, grad=True)
+
+
 def test_gradient_invariants_hold_on_gpu_results():
     B, H, N, D, M = 2, 4, 512, 64, 64
     Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=11, dtype=torch.float32)

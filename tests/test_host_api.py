@@ -144,8 +144,17 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert cont(_p(), far, ctypes.c_void_p((1 << 30) + (1 << 20)), S_out=far) == -1
     assert b"overlap" in L.la_last_error()
     assert cont(_p(), odd, far) == -1
-    assert cont(pb, far, ctypes.c_void_p((1 << 30) + (1 << 24)), saved=big, saved_bytes=keep) == -2
     assert cont(_p(N=0), null, null) == 0
+
+    def back(p, S_in=null, Z_in=null, dS_out=null, dZ_out=null, dS_in=null, dZ_in=null):
+        return L.la_causal_backward_from(ctypes.byref(p), ok, ok, ok, S_in, Z_in, null, null, ok, dS_out, dZ_out,
+                                         null, 0, ok, ok, ok, dS_in, dZ_in, null, 0, null)
+    assert back(_p(), S_in=far) == -1                                   # Z_in missing
+    assert back(_p(), dS_out=far, dS_in=far) == -1                      # gradient in and out overlap
+    assert b"overlap" in L.la_last_error()
+    assert back(_p(), dZ_in=odd) == -1
+    assert back(_p()) == -3                                             # plain backward: needs its workspace
+    assert back(_p(N=0)) == 0
     assert L.la_feature_map(ok, ok, -5, 0, 0, null) == -1
     assert L.la_feature_map(ok, ok, 0, 0, 0, null) == 0
     assert L.la_feature_map(ok, ok, 4, 9, 0, null) == -1
