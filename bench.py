@@ -148,7 +148,7 @@ def max_over_ranks(x, world, dev):
 
 # --------------------------------------------------------------------------- GPU arms
 class CausalStep:
-    def __init__(self, la, w, dev):
+    def __init__(self, la, w, dev, from_state=False):
         self.la, self.w, self.dev = la, w, dev
         Q, K, V, G = draw_qkvg(w.B, w.H, w.N, w.D, w.M, w.seed, w.torch_dtype, w.scale)
         self.host = [t.pin_memory() for t in (Q, K, V, G)]
@@ -160,10 +160,24 @@ class CausalStep:
         self.causal = w.kind == "causal"
         # a training step keeps phi(Q), phi(K) from the forward for the backward (None: nothing to keep)
         self.saved = la.saved_buffer(self.d[0], self.d[2]) if self.causal else None
+        # a step in the middle of a longer sequence: the forward continues from a given state and returns the
+        # final one, the backward takes the final state's upstream gradient and returns the initial state's
+        self.state = None
+        if from_state:
+            g = torch.Generator().manual_seed(w.seed + 1)
+            sS, sZ = (w.B, w.H, w.D, w.M), (w.B, w.H, w.D)
+            mk = lambda shape, scale, shift=0.0: (torch.rand(shape, generator=g) * scale + shift).to(dev)
+            self.state = {"S_in": mk(sS, 2.0, -1.0), "Z_in": mk(sZ, 4.0, 1.0), "dS_out": mk(sS, 0.02, -0.01),
+                          "dZ_out": mk(sZ, 0.02, -0.01), "S_out": torch.empty(sS, device=dev), "Z_out": torch.empty(sZ, device=dev),
+                          "dS_in": torch.empty(sS, device=dev), "dZ_in": torch.empty(sZ, device=dev)}
 
     def fwd(self):
         Q, K, V, _ = self.d
-        if self.causal:
+        if self.causal and self.state:
+            st = self.state
+            self.la.la_causal_forward(Q, K, V, O=self.O, den=self.den, saved=self.saved, S_in=st["S_in"], Z_in=st["Z_in"],
+                                      S_out=st["S_out"], Z_out=st["Z_out"])
+        elif self.causal:
             self.la.la_causal_forward(Q, K, V, O=self.O, den=self.den, saved=self.saved)
         else:
             self.la.la_linear_attention(Q, K, V, O=self.O, den=self.den)
@@ -171,7 +185,12 @@ class CausalStep:
     def bwd(self):
         Q, K, V, G = self.d
         dQ, dK, dV = self.grads
-        if self.causal:
+        if self.causal and self.state:
+            st = self.state
+            self.la.la_causal_backward(Q, K, V, G, O=self.O, den=self.den, saved=self.saved, dQ=dQ, dK=dK, dV=dV,
+                                       S_in=st["S_in"], Z_in=st["Z_in"], dS_out=st["dS_out"], dZ_out=st["dZ_out"],
+                                       dS_in=st["dS_in"], dZ_in=st["dZ_in"])
+        elif self.causal:
             self.la.la_causal_backward(Q, K, V, G, O=self.O, den=self.den, saved=self.saved, dQ=dQ, dK=dK, dV=dV)
         else:
             self.la.la_linear_attention_backward(Q, K, V, G, O=self.O, den=self.den, dQ=dQ, dK=dK, dV=dV)
@@ -270,8 +289,8 @@ KERNEL_ALG_BYTES = {
 }
 
 
-def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True):
-    s = CausalStep(la, shard.rank_workload(w, world, rank), dev)
+def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True, from_state=False):
+    s = CausalStep(la, shard.rank_workload(w, world, rank), dev, from_state=from_state)
     sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
     for _ in range(warmup):
         s.step()
@@ -512,6 +531,11 @@ def main():
                 rows[name] = {kk: r[kk] for kk in ("value", "ms_per_step", "fwd_ms", "bwd_ms", "alg_gbs", "hbm_frac",
                                                    "alg_tflops", "tensor_frac_alg_flops", "gpu_launches", "kernels_ms")}
                 rows[name]["unit"] = "tokens/s"
+        # the headline workload as a step in the middle of a longer sequence (state in and out, both passes)
+        r = bench_attention(la, w, dev, k, wu, 1, 0, pk, do_e2e=False, from_state=True)
+        rows[w.name + "_from_state"] = {kk: r[kk] for kk in ("value", "ms_per_step", "fwd_ms", "bwd_ms", "alg_gbs", "hbm_frac",
+                                                              "gpu_launches", "kernels_ms")}
+        rows[w.name + "_from_state"]["unit"] = "tokens/s"
 
     cpu = None
     if rank == 0 and world == 1 and not args.main_only:
