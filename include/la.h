@@ -171,6 +171,19 @@ int la_recurrent_step(const la_problem* p, const void* q, const void* k, const v
                       float* S, float* Z, void* out, void* stream);
 
 /*
+ * p->N recurrent steps per (batch, head) stream in one launch, for steps whose inputs are all known
+ * beforehand (a prompt continued token by token, scoring a given continuation, several drafted
+ * tokens at once): Eq. 18-20 for t = 1..N,
+ *   S += phi(k_t) v_t^T,  Z += phi(k_t),  out_t = phi(q_t)^T S / (phi(q_t)^T Z + eps),
+ * with the state read from and written to memory once instead of once per step.  q, k: [B,H,N,D];
+ * v, out: [B,H,N,M] of p->dtype; S, Z as for la_recurrent_step(), updated in place.  The results
+ * are bit-identical to N calls of la_recurrent_step() on the same inputs.  N = 0: no-op.
+ * Needs no workspace.
+ */
+int la_recurrent_steps(const la_problem* p, const void* q, const void* k, const void* v,
+                       float* S, float* Z, void* out, void* stream);
+
+/*
  * Non-causal forward for callers that cannot allocate device memory (the paper has no
  * counterpart: this is a deployment convenience, not part of the method).
  *

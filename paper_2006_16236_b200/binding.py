@@ -23,7 +23,7 @@ _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 EXPORTS = [
     "la_feature_map", "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
     "la_causal_forward", "la_causal_forward_from", "la_causal_backward_from",
-    "la_causal_backward", "la_recurrent_step", "la_workspace_bytes", "la_status_string",
+    "la_causal_backward", "la_recurrent_step", "la_recurrent_steps", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
     "la_profile_kernel_name", "la_version", "la_causal_plan",
 ]
@@ -63,6 +63,7 @@ def lib() -> ctypes.CDLL:
         L.la_causal_backward_from.argtypes = [pp] + [vp] * 10 + [vp, sz] + [vp] * 5 + [vp, sz, vp]
         L.la_causal_backward.argtypes = [pp] + [vp] * 6 + [vp, sz] + [vp] * 3 + [vp, sz, vp]
         L.la_recurrent_step.argtypes = [pp] + [vp] * 6 + [vp]
+        L.la_recurrent_steps.argtypes = [pp] + [vp] * 6 + [vp]
         L.la_workspace_bytes.argtypes = [pp, i32]
         L.la_workspace_bytes.restype = sz
         L.la_status_string.argtypes = [ctypes.c_int]
@@ -317,4 +318,19 @@ def la_recurrent_step(q, k, v, S, Z, phi="elu1", eps=0.0, out=None):
     out = torch.empty_like(v) if out is None else out
     _check(lib().la_recurrent_step(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out),
                                    _stream(dev)))
+    return out
+
+
+def la_recurrent_steps(q, k, v, S, Z, phi="elu1", eps=0.0, out=None):
+    """N decode steps in one launch (all inputs known beforehand): q, k [B,H,N,D], v [B,H,N,M]; S, Z (fp32)
+    are updated in place; returns out [B,H,N,M]."""
+    dev = _dev(q, k, v, S, Z, out)
+    if q.dim() != 4 or v.dim() != 4 or S.dtype != torch.float32 or Z.dtype != torch.float32:
+        raise ValueError("expected q,k [B,H,N,D], v [B,H,N,M], fp32 S [B,H,D,M] and Z [B,H,D]")
+    p = _problem_of(q, v, phi, eps)
+    if tuple(S.shape) != (p.B, p.H, p.D, p.M) or tuple(Z.shape) != (p.B, p.H, p.D):
+        raise ValueError("state shape mismatch")
+    out = torch.empty_like(v) if out is None else out
+    _check(lib().la_recurrent_steps(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out),
+                                    _stream(dev)))
     return out

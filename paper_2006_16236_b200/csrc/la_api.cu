@@ -327,6 +327,16 @@ int la_recurrent_step(const la_problem* p, const void* q, const void* k, const v
     return launch_recurrent_step(*p, q, k, v, S, Z, out, (cudaStream_t)stream);
 }
 
+int la_recurrent_steps(const la_problem* p, const void* q, const void* k, const void* v,
+                       float* S, float* Z, void* out, void* stream) {
+    if (int rc = check_problem(p, true)) return rc;
+    if (p->N == 0) return LA_OK;
+    LA_REQUIRE_PTR(q); LA_REQUIRE_PTR(k); LA_REQUIRE_PTR(v);
+    LA_REQUIRE_PTR(S); LA_REQUIRE_PTR(Z); LA_REQUIRE_PTR(out);
+    if (int rc = check_arch()) return rc;
+    return launch_recurrent_steps(*p, q, k, v, S, Z, out, (cudaStream_t)stream);
+}
+
 int la_last_device_status(void* stream) {
     LA_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     int word = 0;

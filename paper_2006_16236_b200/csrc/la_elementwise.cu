@@ -161,6 +161,169 @@ recurrent_step_general_kernel(const T* __restrict__ q, const T* __restrict__ k, 
     }
 }
 
+// ---------------------------------------------------------------------------
+// Several recurrent steps in one launch (Eq. 18-20 for t = 1..N with the inputs of all steps
+// given): the state is read from HBM once, kept in registers across the steps (Z by the first D
+// threads) and written back once; per step only q_t, k_t, v_t come in and out_t goes out.  The
+// arithmetic of a step is that of recurrent_step_kernel, in the same order: the results are
+// bit-identical to N single-step launches.  Shared buffers alternate between steps, so two
+// barriers per step suffice.
+// q, k: [B,H,N,D]; v, out: [B,H,N,M].
+// ---------------------------------------------------------------------------
+template <typename T, int D, int M>
+__global__ void __launch_bounds__(128)
+recurrent_steps_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                       float* __restrict__ S, float* __restrict__ Z, T* __restrict__ out,
+                       int64_t N, float eps, int phi) {
+    constexpr int TPR = M / 4;
+    constexpr int RPP = 128 / TPR;
+    constexpr int PASSES = D / RPP;
+    static_assert(D % RPP == 0 && PASSES >= 1, "unsupported state shape");
+
+    __shared__ float sq[2][D], sk[2][D];
+    __shared__ __align__(16) float sv[2][M];
+    __shared__ __align__(16) float spart[2][4][M];
+    __shared__ float sden[2][4];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t bh = blockIdx.x;
+    const int c4 = tid % TPR, r0 = tid / TPR;
+
+    float4* Sp = reinterpret_cast<float4*>(S + bh * (int64_t)(D * M));
+    float4 s[PASSES];
+#pragma unroll
+    for (int p = 0; p < PASSES; ++p) s[p] = Sp[(r0 + p * RPP) * TPR + c4];
+    float z = tid < D ? Z[bh * D + tid] : 0.f;
+
+    const T* qb = q + bh * N * D;
+    const T* kb = k + bh * N * D;
+    const T* vb = v + bh * N * M;
+    T* ob = out + bh * N * M;
+    #pragma unroll 1
+    for (int64_t t = 0; t < N; ++t) {
+        const int b = (int)(t & 1);
+        float zq = 0.f;
+        if (tid < D) {
+            const float kd = phi_apply(to_f32<T>(kb[t * D + tid]), phi);
+            const float qd = phi_apply(to_f32<T>(qb[t * D + tid]), phi);
+            z += kd;
+            sk[b][tid] = kd;
+            sq[b][tid] = qd;
+            zq = qd * z;
+        }
+        if (tid < M) sv[b][tid] = to_f32<T>(vb[t * M + tid]);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) zq += __shfl_xor_sync(0xffffffffu, zq, off);
+        if (lane == 0) sden[b][warp] = zq;
+        __syncthreads();
+
+        const float4 vv = reinterpret_cast<const float4*>(sv[b])[c4];
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int p = 0; p < PASSES; ++p) {
+            const int d = r0 + p * RPP;
+            const float kd = sk[b][d], qd = sq[b][d];
+            s[p].x = fmaf(kd, vv.x, s[p].x);
+            s[p].y = fmaf(kd, vv.y, s[p].y);
+            s[p].z = fmaf(kd, vv.z, s[p].z);
+            s[p].w = fmaf(kd, vv.w, s[p].w);
+            acc.x = fmaf(qd, s[p].x, acc.x);
+            acc.y = fmaf(qd, s[p].y, acc.y);
+            acc.z = fmaf(qd, s[p].z, acc.z);
+            acc.w = fmaf(qd, s[p].w, acc.w);
+        }
+#pragma unroll
+        for (int off = 16; off >= TPR; off >>= 1) {
+            acc.x += __shfl_xor_sync(0xffffffffu, acc.x, off);
+            acc.y += __shfl_xor_sync(0xffffffffu, acc.y, off);
+            acc.z += __shfl_xor_sync(0xffffffffu, acc.z, off);
+            acc.w += __shfl_xor_sync(0xffffffffu, acc.w, off);
+        }
+        if (lane < TPR) reinterpret_cast<float4*>(spart[b][warp])[lane] = acc;
+        __syncthreads();
+        if (tid < M) {
+            const float den = sden[b][0] + sden[b][1] + sden[b][2] + sden[b][3] + eps;
+            const float num = spart[b][0][tid] + spart[b][1][tid] + spart[b][2][tid] + spart[b][3][tid];
+            ob[t * M + tid] = from_f32<T>(num / den);
+        }
+    }
+#pragma unroll
+    for (int p = 0; p < PASSES; ++p) Sp[(r0 + p * RPP) * TPR + c4] = s[p];
+    if (tid < D) Z[bh * D + tid] = z;
+}
+
+// Any D, M (multiples of 8 up to 128): the single-step arithmetic of recurrent_step_general_kernel looped
+// over the steps; the state stays in global memory (cached) between them.
+template <typename T>
+__global__ void __launch_bounds__(128)
+recurrent_steps_general_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                               float* __restrict__ S, float* __restrict__ Z, T* __restrict__ out,
+                               int64_t N, int D, int M, float eps, int phi) {
+    __shared__ float sq[2][128], sk[2][128], sden[2][4];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t bh = blockIdx.x;
+    float z = tid < D ? Z[bh * D + tid] : 0.f;
+    #pragma unroll 1
+    for (int64_t t = 0; t < N; ++t) {
+        const int b = (int)(t & 1);
+        float zq = 0.f;
+        if (tid < D) {
+            const float kd = phi_apply(to_f32<T>(k[(bh * N + t) * D + tid]), phi);
+            const float qd = phi_apply(to_f32<T>(q[(bh * N + t) * D + tid]), phi);
+            z += kd;
+            sk[b][tid] = kd;
+            sq[b][tid] = qd;
+            zq = qd * z;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) zq += __shfl_xor_sync(0xffffffffu, zq, off);
+        if (lane == 0) sden[b][warp] = zq;
+        __syncthreads();
+        if (tid < M) {
+            const float vm = to_f32<T>(v[(bh * N + t) * M + tid]);
+            float* Sp = S + bh * (int64_t)D * M + tid;
+            float num = 0.f;
+            for (int d = 0; d < D; ++d) {
+                float sv = fmaf(sk[b][d], vm, Sp[(int64_t)d * M]);
+                Sp[(int64_t)d * M] = sv;
+                num = fmaf(sq[b][d], sv, num);
+            }
+            out[(bh * N + t) * M + tid] = from_f32<T>(num / (sden[b][0] + sden[b][1] + sden[b][2] + sden[b][3] + eps));
+        }
+    }
+    if (tid < D) Z[bh * D + tid] = z;
+}
+
+template <typename T>
+static int recurrent_steps_dispatch(const la_problem& p, const void* q, const void* k, const void* v,
+                                    float* S, float* Z, void* out, cudaStream_t st) {
+    const unsigned grid = (unsigned)(p.B * p.H);
+    const T *qq = (const T*)q, *kk = (const T*)k, *vv = (const T*)v;
+    T* oo = (T*)out;
+#define LA_RS_CASE(DD, MM)                                                                     \
+    if (p.D == DD && p.M == MM) {                                                              \
+        recurrent_steps_kernel<T, DD, MM><<<grid, 128, 0, st>>>(qq, kk, vv, S, Z, oo, p.N, p.eps, p.phi); \
+        LA_LAUNCHED();                                                       \
+        return LA_OK;                                                                          \
+    }
+    LA_RS_CASE(32, 32) LA_RS_CASE(32, 64) LA_RS_CASE(64, 32) LA_RS_CASE(64, 64)
+    LA_RS_CASE(64, 128) LA_RS_CASE(128, 64) LA_RS_CASE(128, 128)
+#undef LA_RS_CASE
+    recurrent_steps_general_kernel<T><<<grid, 128, 0, st>>>(qq, kk, vv, S, Z, oo, p.N, (int)p.D, (int)p.M,
+                                                            p.eps, p.phi);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+int launch_recurrent_steps(const la_problem& p, const void* q, const void* k, const void* v,
+                           float* S, float* Z, void* out, cudaStream_t st) {
+    prof_begin(kProfRecurrent, st);
+    const int rc = p.dtype == LA_F32 ? recurrent_steps_dispatch<float>(p, q, k, v, S, Z, out, st)
+                                     : recurrent_steps_dispatch<__nv_bfloat16>(p, q, k, v, S, Z, out, st);
+    prof_end(kProfRecurrent, st);
+    return rc;
+}
+
 template <typename T>
 static int recurrent_dispatch(const la_problem& p, const void* q, const void* k, const void* v,
                               float* S, float* Z, void* out, cudaStream_t st) {

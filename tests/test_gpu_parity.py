@@ -160,6 +160,31 @@ def test_recurrent_steps_equal_causal_form(shape, dtype):
     assert_close(S2, So, dtype, "S_N of the parallel form")
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", [(2, 3, 1, 64, 64), (2, 3, 40, 64, 64), (1, 2, 24, 32, 32), (2, 2, 17, 16, 24), (1, 2, 9, 128, 64),
+                                   (3, 5, 130, 32, 64)])
+def test_recurrent_steps_in_one_launch(shape, dtype):
+    """N recurrent steps in one launch: bit-identical to N single-step launches, and equal to the oracle's
+    recurrence from the same non-zero state."""
+    B, H, N, D, M = shape
+    Q, K, V, _ = draw_qkvg(B, H, N, D, M, seed=sum(shape) + 3, dtype=dtype, with_grad=False)
+    g = torch.Generator().manual_seed(8)
+    S0 = torch.randn((B, H, D, M), generator=g) * 2.0
+    Z0 = torch.rand((B, H, D), generator=g) * 3.0 + 1.0
+    Qd, Kd, Vd = gpu(Q, K, V)
+    S, Z = S0.to(DEV), Z0.to(DEV)
+    out = la.la_recurrent_steps(Qd, Kd, Vd, S, Z)
+    S1, Z1 = S0.to(DEV), Z0.to(DEV)
+    one = [la.la_recurrent_step(Qd[:, :, t].contiguous(), Kd[:, :, t].contiguous(), Vd[:, :, t].contiguous(), S1, Z1)
+           for t in range(N)]
+    la.la_last_device_status()
+    assert torch.equal(out, torch.stack(one, dim=2)) and torch.equal(S, S1) and torch.equal(Z, Z1)
+    Or, _, Sr, Zr = oracle.causal_from_state(Q, K, V, S0.double().numpy(), Z0.double().numpy())
+    assert_close(out, Or, dtype, "out")
+    assert_close(S, Sr, dtype, "S_N")
+    assert_close(Z, Zr, dtype, "Z_N")
+
+
 def test_prefill_then_decode_handoff():
     B, H, N, D, M = 2, 2, 64, 32, 32
     Q, K, V, _ = draw_qkvg(B, H, N + 1, D, M, seed=9, dtype=torch.float32, with_grad=False)
