@@ -498,7 +498,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(w, 1),
+        "config": dict(workload_config(w, 1), timing="host wall clock around the oracle call on a bounded sample of the workload"),
         "cpu_baseline": {"value": value, "unit": "tokens/s", "kind": "oracle", "cores": cores, "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
