@@ -189,7 +189,6 @@ __device__ __forceinline__ uint64_t desc_mn(uint32_t addr, uint32_t lbo = kTileB
 // B operand whose every entry is 1: one 1 KB group of ones re-read for every K group (SBO = 0).
 __device__ __forceinline__ uint64_t desc_ones(uint32_t addr) { return sm100::umma_desc_sw128(addr, 16, 0); }
 
-__device__ __forceinline__ uint4 ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 __device__ __forceinline__ void stg128(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
 }
@@ -507,21 +506,6 @@ __device__ __forceinline__ void score_block_pack(const uint32_t (&v)[32], bool p
     }
 }
 
-// The same for a transposed score tile (rows = keys j, columns = queries i): the causal mask
-// keeps i >= j, so a block left of the diagonal (`present` false) is zeros and the diagonal
-// block keeps local columns >= lane.
-__device__ __forceinline__ void score_block_pack_t(const uint32_t (&v)[32], bool present, bool diagonal, int lane,
-                                                   uint32_t (&packed)[16]) {
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        float x0 = __uint_as_float(v[2 * j]), x1 = __uint_as_float(v[2 * j + 1]);
-        if (diagonal) {
-            if (2 * j < lane) x0 = 0.f;
-            if (2 * j + 1 < lane) x1 = 0.f;
-        }
-        packed[j] = present ? sm100::pack_bf16x2(x0, x1) : 0u;
-    }
-}
 
 // The same with one warp-uniform branch per block instead of per-element selects: a block off the
 // diagonal costs sixteen conversions, an absent block none.  (The score warps of the quadrant with
