@@ -633,75 +633,55 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             auto lo_mn = [&](uint32_t a, uint32_t lbo) { return (uint32_t)desc_mn(a, lbo); };
             auto stage_q = [&](int i) { return sbase + kKvOffStage + (uint32_t)(i % kKvStages) * kKvStageBytes; };
             bool ok = true;
-            if (warp == 17) {
-                auto issue_pt = [&](int i) {
-                    const uint32_t dQ = lo_k(stage_q(i)), dK = lo_k(stage_q(i) + kTileBytes);
-                    umma_group4(tmem + kKvColP, dK, 2, dQ, 2, idesc_pp, 0);
-                    umma_commit(&bars->p_full);
-                };
+            if (warp != 18) {
                 // The two score tiles are two independent pipelines, each with its own issuing thread, so that
                 // the score warps always have a tile to work on: Ph^T of chunk i+1 is issued as soon as the
                 // rounded Ph^T of chunk i has been consumed, and likewise dP^T.  The next tile overwrites the
-                // rounded copy only after the product that reads it (in-order execution within a thread).
-                ok = mbar_wait(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !*abort_flag;
-                if (ok) {
-                    tc_fence_after_sync();
-                    issue_pt(0);
-                }
-                #pragma unroll 1
-                for (int i = 0; i < L && ok; ++i) {
-                    const uint32_t dGmn = lo_mn(stage_q(i) + 3 * kTileBytes, kTileBytes);
-                    LA_TRACE(g_trace_dkv, i, 0);
-                    ok = mbar_wait(&bars->p_ready, i & 1, prm.status, kStatusPipeTimeout) &&
-                         mbar_wait(&bars->kr_full, i & 1, prm.status, kStatusMmaTimeout);
-                    if (!ok || *abort_flag) { ok = false; break; }
-                    tc_fence_after_sync();
-                    LA_TRACE(g_trace_dkv, i, 1);
-                    umma_group4_ta(tmem + kKvColDv, tmem + kKvColP, dGmn, 128, idesc_kmn, 1);            // gV += Ph^T G
-                    umma_group4_ta(tmem + kKvColDv, tmem + kKvColP + 64, dGmn + 512, 128, idesc_kmn, 1);
-                    umma_commit(&bars->dv_full);    // gV of this chunk is complete: its epilogue overlaps gk
-                    umma_commit(&bars->empty[i % kKvStages]);      // this thread's reads of the stage
-                    if (i + 1 < L) {
-                        ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
-                        if (!ok) break;
-                        tc_fence_after_sync();
-                        issue_pt(i + 1);
-                    }
-                    LA_TRACE(g_trace_dkv, i, 2);
-                }
-            } else if (warp == 19) {
-                auto issue_dpt = [&](int i) {
-                    const uint32_t dV = lo_k(stage_q(i) + 2 * kTileBytes), dG = lo_k(stage_q(i) + 3 * kTileBytes);
-                    umma_group4(tmem + kKvColDP, dV, 2, dG, 2, idesc_pp, 0);
-                    umma_bf16(tmem + kKvColDP, desc_ones(aOnes), desc_k(aAux), idesc_pp, 1);
-                    umma_commit(&bars->dp_full);
+                // rounded copy only after the product that reads it (in-order execution within a thread).  Both
+                // threads run this one loop on their own tile, accumulator, operands and barriers (one copy of
+                // the code in the instruction cache).
+                const bool dp = warp == 19;                                // the dP^T pipeline (else Ph^T)
+                const uint32_t col = dp ? kKvColDP : kKvColP;              // score tile
+                const uint32_t acc = dp ? kKvColDk : kKvColDv;             // what it is contracted into
+                const uint32_t offA = (dp ? 2u : 1u) * kTileBytes;         // tile = A B^T: [V | 1] [G | dl]^T  or  k qh^T
+                const uint32_t offB = (dp ? 3u : 0u) * kTileBytes;
+                const uint32_t offC = (dp ? 0u : 3u) * kTileBytes;         // acc += tile x C: qh  or  G
+                uint64_t* tile_full = dp ? &bars->dp_full : &bars->p_full;
+                uint64_t* tile_ready = dp ? &bars->dp_ready : &bars->p_ready;
+                uint64_t* acc_started = dp ? &bars->vr_full : &bars->kr_full;      // the state thread's first product
+                uint64_t* acc_full = dp ? &bars->dkv_full : &bars->dv_full;
+                auto issue_tile = [&](int i) {
+                    umma_group4(tmem + col, lo_k(stage_q(i) + offA), 2, lo_k(stage_q(i) + offB), 2, idesc_pp, 0);
+                    if (dp) umma_bf16(tmem + col, desc_ones(aOnes), desc_k(aAux), idesc_pp, 1);    // + dl_i (fifth K step)
+                    umma_commit(tile_full);
                 };
                 ok = mbar_wait(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !*abort_flag;
                 if (ok) {
                     tc_fence_after_sync();
-                    issue_dpt(0);
+                    issue_tile(0);
                 }
                 #pragma unroll 1
                 for (int i = 0; i < L && ok; ++i) {
-                    const uint32_t dQmn = lo_mn(stage_q(i), kTileBytes);
-                    ok = mbar_wait(&bars->dp_ready, i & 1, prm.status, kStatusPipeTimeout) &&
-                         mbar_wait(&bars->vr_full, i & 1, prm.status, kStatusMmaTimeout);
+                    const uint32_t dC = lo_mn(stage_q(i) + offC, kTileBytes);
+                    if (!dp) LA_TRACE(g_trace_dkv, i, 0);
+                    ok = mbar_wait(tile_ready, i & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait(acc_started, i & 1, prm.status, kStatusMmaTimeout);
                     if (!ok || *abort_flag) { ok = false; break; }
                     tc_fence_after_sync();
-                    LA_TRACE(g_trace_dkv, i, 3);
-                    umma_group4_ta(tmem + kKvColDk, tmem + kKvColDP, dQmn, 128, idesc_kmn, 1);           // gk += dP^T qh
-                    umma_group4_ta(tmem + kKvColDk, tmem + kKvColDP + 64, dQmn + 512, 128, idesc_kmn, 1);
-                    umma_commit(&bars->dkv_full);
-                    // vr_full(i) was awaited and covers the state thread's three products on this stage
+                    LA_TRACE(g_trace_dkv, i, dp ? 3 : 1);
+                    umma_group4_ta(tmem + acc, tmem + col, dC, 128, idesc_kmn, 1);                 // gV += Ph^T G / gk += dP^T qh
+                    umma_group4_ta(tmem + acc, tmem + col + 64, dC + 512, 128, idesc_kmn, 1);
+                    umma_commit(acc_full);      // gV is complete first: its epilogue overlaps gk
+                    // this thread's reads of the stage; the awaited vr_full(i) covers the state thread's products on it
                     umma_commit(&bars->empty[i % kKvStages]);
                     if (i + 1 < L) {
                         // mapped(i+1) also says that the dl column tile holds chunk i+1
                         ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
                         if (!ok) break;
                         tc_fence_after_sync();
-                        issue_dpt(i + 1);
+                        issue_tile(i + 1);
                     }
-                    LA_TRACE(g_trace_dkv, i, 4);
+                    LA_TRACE(g_trace_dkv, i, dp ? 4 : 2);
                 }
             } else {
                 #pragma unroll 1
