@@ -40,9 +40,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # ncu capture summarised under profiles/), keyed by workload; None until captured.
 NCU_TRAFFIC_BYTES = {
     # profiles/ncu_full_causal_kernels_N16384.md
-    ("causal_sweep_bf16_N16384", "causal_fwd_kernel"): 766_667_776,      # includes 268 MB of saved phi(Q), phi(K)
-    ("causal_sweep_bf16_N16384", "causal_bwd_dq_kernel"): 665_640_192,
-    ("causal_sweep_bf16_N16384", "causal_bwd_dkv_kernel"): 787_921_920,
+    ("causal_sweep_bf16_N16384", "causal_fwd_kernel"): 766_838_528,      # includes 268 MB of saved phi(Q), phi(K)
+    ("causal_sweep_bf16_N16384", "causal_bwd_dq_kernel"): 667_496_448,
+    ("causal_sweep_bf16_N16384", "causal_bwd_dkv_kernel"): 789_536_256,
 }
 
 
