@@ -307,6 +307,36 @@ def test_backward_chained_over_two_calls():
         assert_close(got, ref, torch.bfloat16, nm, grad=True)
 
 
+@pytest.mark.parametrize("dtype,D,N", [(torch.float32, 32, 200), (torch.bfloat16, 64, 1024)])
+def test_right_padded_causal_batches_need_no_mask(dtype, D, N):
+    """Sequences of different lengths, padded on the right to one N (here with large junk): causality keeps
+    the padding out of every real position's output, and an upstream gradient that is zero on the padding
+    keeps it out of every real position's gradient and makes the padding's own gradients zero.  Each sequence
+    is compared with the oracle run on its own length."""
+    B, H = 3, 2
+    lengths = [N, N - N // 3, 1 + N // 5]
+    Q, K, V, G = draw_qkvg(B, H, N, D, D, seed=29, dtype=dtype)
+    for b, n in enumerate(lengths):
+        Q[b, :, n:] = 7.0
+        K[b, :, n:] = 9.0
+        V[b, :, n:] = -50.0
+        G[b, :, n:] = 0.0
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    O = la.la_causal_forward(Qd, Kd, Vd)
+    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd)
+    la.la_last_device_status()
+    for b, n in enumerate(lengths):
+        sl = (slice(b, b + 1), slice(None), slice(0, n))
+        q, k, v, g = Q[sl], K[sl], V[sl], G[sl]
+        assert_close(O[sl], oracle.linear_attention(q, k, v, True)[0], dtype, f"O, length {n}")
+        rq, rk, rv = oracle.linear_attention_backward(q, k, v, g, True)
+        assert_close(dQ[sl], rq, dtype, f"dQ, length {n}", grad=True)
+        assert_close(dK[sl], rk, dtype, f"dK, length {n}", grad=True)
+        assert_close(dV[sl], rv, dtype, f"dV, length {n}", grad=True)
+        for t, nm in ((dQ, "dQ"), (dK, "dK"), (dV, "dV")):
+            assert float(t[b, :, n:].float().abs().max()) == 0.0 if n < N else True, f"{nm} on the padding"
+
+
 def test_gradient_invariants_hold_on_gpu_results():
     B, H, N, D, M = 2, 4, 512, 64, 64
     Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=11, dtype=torch.float32)
