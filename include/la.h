@@ -65,7 +65,9 @@ typedef enum {
     LA_OP_LINEAR_BACKWARD = 1,
     LA_OP_CAUSAL_FORWARD = 2,
     LA_OP_CAUSAL_BACKWARD = 3,
-    LA_OP_CAUSAL_SAVED = 4       /* size of the optional `saved` buffer, see la_causal_forward() */
+    LA_OP_CAUSAL_SAVED = 4,      /* size of the optional `saved` buffer, see la_causal_forward() */
+    LA_OP_LINEAR_VARLEN_FORWARD = 5,     /* la_linear_attention_varlen()          */
+    LA_OP_LINEAR_VARLEN_BACKWARD = 6     /* la_linear_attention_varlen_backward() */
 } la_op;
 
 typedef struct {
@@ -104,6 +106,28 @@ int la_linear_attention_backward(const la_problem* p, const void* Q, const void*
                                  const void* O, const float* den, const void* G,
                                  void* dQ, void* dK, void* dV,
                                  void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The non-causal form on a ragged batch: sequences of different lengths padded on the right to
+ * the common N of the tensors (a key-padding mask; the paper's speech data are such batches).
+ * lengths: [B] int32 on the device, 4-byte aligned; values are clipped to [0, N] on the device.
+ * For batch element b only positions i, j < lengths[b] exist:
+ *   O_i = phi(Q_i)^T sum_{j < len} phi(K_j) V_j^T / (phi(Q_i)^T sum_{j < len} phi(K_j) + eps),
+ * KV / Zs are the sums over the real positions, and O, den (and in the backward pass dQ, dK, dV)
+ * are written as zeros on the padding; what Q, K, V, G hold there is never used.  Workspace:
+ * la_workspace_bytes(p, LA_OP_LINEAR_VARLEN_FORWARD / _BACKWARD).  These calls run the general
+ * kernels for every problem (the tensor-core kernels take full-length batches only).  Everything
+ * else as for la_linear_attention() / la_linear_attention_backward().
+ */
+int la_linear_attention_varlen(const la_problem* p, const void* Q, const void* K, const void* V,
+                               const int32_t* lengths,
+                               void* O, float* den, float* KV, float* Zs,
+                               void* ws, size_t ws_bytes, void* stream);
+int la_linear_attention_varlen_backward(const la_problem* p, const void* Q, const void* K, const void* V,
+                                        const int32_t* lengths,
+                                        const void* O, const float* den, const void* G,
+                                        void* dQ, void* dK, void* dV,
+                                        void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Causal linear attention, Eq. 9-12 (Algorithm 1, forward, plus the normaliser):

@@ -18,10 +18,12 @@ LA_F32, LA_BF16 = 0, 1
 LA_PHI_ELU1, LA_PHI_IDENTITY = 0, 1
 LA_OP_LINEAR_FORWARD, LA_OP_LINEAR_BACKWARD, LA_OP_CAUSAL_FORWARD, LA_OP_CAUSAL_BACKWARD = 0, 1, 2, 3
 LA_OP_CAUSAL_SAVED = 4
+LA_OP_LINEAR_VARLEN_FORWARD, LA_OP_LINEAR_VARLEN_BACKWARD = 5, 6
 _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
     "la_feature_map", "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
+    "la_linear_attention_varlen", "la_linear_attention_varlen_backward",
     "la_causal_forward", "la_causal_forward_from", "la_causal_backward_from",
     "la_causal_backward", "la_recurrent_step", "la_recurrent_steps", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
@@ -58,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.la_linear_attention.argtypes = [pp] + [vp] * 7 + [vp, sz, vp]
         L.la_linear_attention_noalloc.argtypes = [pp] + [vp] * 7 + [vp]
         L.la_linear_attention_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
+        L.la_linear_attention_varlen.argtypes = [pp] + [vp] * 8 + [vp, sz, vp]
+        L.la_linear_attention_varlen_backward.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
         L.la_causal_forward.argtypes = [pp] + [vp] * 7 + [vp, sz] + [vp, sz, vp]
         L.la_causal_forward_from.argtypes = [pp] + [vp] * 9 + [vp, sz] + [vp, sz, vp]
         L.la_causal_backward_from.argtypes = [pp] + [vp] * 10 + [vp, sz] + [vp] * 5 + [vp, sz, vp]
@@ -334,3 +338,38 @@ def la_recurrent_steps(q, k, v, S, Z, phi="elu1", eps=0.0, out=None):
     _check(lib().la_recurrent_steps(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out),
                                     _stream(dev)))
     return out
+
+
+def _lengths_arg(lengths, B, dev):
+    if lengths.dtype != torch.int32 or tuple(lengths.shape) != (B,) or not lengths.is_cuda or not lengths.is_contiguous():
+        raise ValueError("lengths must be a contiguous int32 CUDA tensor of shape [B]")
+    return lengths
+
+
+def la_linear_attention_varlen(Q, K, V, lengths, phi="elu1", eps=0.0, O=None, den=None, KV=None, Zs=None, ws=None):
+    """Non-causal form on a right-padded ragged batch: lengths[b] real positions per batch element; O and den
+    are zero on the padding.  Returns O."""
+    dev = _dev(Q, K, V, O, den, KV, Zs)
+    p = _problem_of(Q, V, phi, eps)
+    _lengths_arg(lengths, p.B, dev)
+    O = torch.empty_like(V) if O is None else O
+    ws = workspace(p, LA_OP_LINEAR_VARLEN_FORWARD, dev) if ws is None else ws
+    _check(lib().la_linear_attention_varlen(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(O), _ptr(den),
+                                            _ptr(KV), _ptr(Zs), _ptr(ws), _nbytes(ws), _stream(dev)))
+    return O
+
+
+def la_linear_attention_varlen_backward(Q, K, V, G, lengths, phi="elu1", eps=0.0, O=None, den=None,
+                                        dQ=None, dK=None, dV=None, ws=None):
+    """Gradients of la_linear_attention_varlen; zero on the padding.  Returns (dQ, dK, dV)."""
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV)
+    p = _problem_of(Q, V, phi, eps)
+    _lengths_arg(lengths, p.B, dev)
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(K) if dK is None else dK
+    dV = torch.empty_like(V) if dV is None else dV
+    ws = workspace(p, LA_OP_LINEAR_VARLEN_BACKWARD, dev) if ws is None else ws
+    _check(lib().la_linear_attention_varlen_backward(
+        ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(O), _ptr(den), _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV),
+        _ptr(ws), _nbytes(ws), _stream(dev)))
+    return dQ, dK, dV

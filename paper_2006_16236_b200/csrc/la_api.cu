@@ -174,9 +174,10 @@ const char* la_profile_kernel_name(int kernel) {
 
 size_t la_workspace_bytes(const la_problem* p, int32_t op) {
     if (!p || p->B < 1 || p->H < 1 || p->N < 0 || p->D < 1 || p->M < 1 || p->D > 128 || p->M > 128) return 0;
-    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_CAUSAL_SAVED) return 0;
+    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_LINEAR_VARLEN_BACKWARD) return 0;
     if (p->N == 0) return 0;
     if (op == LA_OP_CAUSAL_SAVED) return tc_supported(*p, LA_OP_CAUSAL_BACKWARD) ? tc_causal_saved_bytes(*p) : 0;
+    if (op == LA_OP_LINEAR_VARLEN_FORWARD || op == LA_OP_LINEAR_VARLEN_BACKWARD) return general_workspace_bytes(*p, op);
     if (tc_supported(*p, op)) return tc_workspace_bytes(*p, op);
     return general_workspace_bytes(*p, op);
 }
@@ -209,7 +210,22 @@ int la_linear_attention(const la_problem* p, const void* Q, const void* K, const
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc_linear_forward(*p, Q, K, V, O, den, KV, Zs, ws, st);
-    return general_linear_forward(*p, Q, K, V, O, den, KV, Zs, ws, st);
+    return general_linear_forward(*p, Q, K, V, nullptr, O, den, KV, Zs, ws, st);
+}
+
+int la_linear_attention_varlen(const la_problem* p, const void* Q, const void* K, const void* V,
+                               const int32_t* lengths,
+                               void* O, float* den, float* KV, float* Zs,
+                               void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_problem(p, true)) return rc;
+    if (p->N == 0) return LA_OK;
+    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(O);
+    if (!lengths) return fail(LA_ERR_INVALID_ARG, "lengths is NULL");
+    if (reinterpret_cast<uintptr_t>(lengths) & 3u) return fail(LA_ERR_INVALID_ARG, "lengths is not 4-byte aligned");
+    LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(KV); LA_OPTIONAL_PTR(Zs);
+    if (int rc = check_ws(p, LA_OP_LINEAR_VARLEN_FORWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_arch()) return rc;
+    return general_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, ws, (cudaStream_t)stream);
 }
 
 int la_linear_attention_backward(const la_problem* p, const void* Q, const void* K, const void* V,
@@ -225,7 +241,24 @@ int la_linear_attention_backward(const la_problem* p, const void* Q, const void*
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc_linear_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
-    return general_linear_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
+    return general_linear_backward(*p, Q, K, V, nullptr, G, dQ, dK, dV, ws, st);
+}
+
+int la_linear_attention_varlen_backward(const la_problem* p, const void* Q, const void* K, const void* V,
+                                        const int32_t* lengths,
+                                        const void* O, const float* den, const void* G,
+                                        void* dQ, void* dK, void* dV,
+                                        void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_problem(p, true)) return rc;
+    if (p->N == 0) return LA_OK;
+    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(G);
+    LA_REQUIRE_PTR(dQ); LA_REQUIRE_PTR(dK); LA_REQUIRE_PTR(dV);
+    if (!lengths) return fail(LA_ERR_INVALID_ARG, "lengths is NULL");
+    if (reinterpret_cast<uintptr_t>(lengths) & 3u) return fail(LA_ERR_INVALID_ARG, "lengths is not 4-byte aligned");
+    LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den);
+    if (int rc = check_ws(p, LA_OP_LINEAR_VARLEN_BACKWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_arch()) return rc;
+    return general_linear_backward(*p, Q, K, V, lengths, G, dQ, dK, dV, ws, (cudaStream_t)stream);
 }
 
 static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {

@@ -95,9 +95,10 @@ int general_causal_forward(const la_problem& p, const void* Q, const void* K, co
 int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V,
                             const void* G, const StateArgs& sa, void* dQ, void* dK, void* dV, void* ws,
                             cudaStream_t st);
-int general_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V,
+// lengths ([B] int32, device, or null): real positions per batch element (the rest is padding)
+int general_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
                            void* O, float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
-int general_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V,
+int general_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
                             const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 
 }  // namespace la

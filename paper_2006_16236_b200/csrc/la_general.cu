@@ -326,18 +326,26 @@ Split choose_split(const la_problem& p) {
     return Split{(int)ns, len};
 }
 
+// Ragged batches (non-causal form): lengths[b] positions of batch element b are real, the rest is padding
+// that takes no part in any sum and receives zeros.  `real_end` clips a split's range to the sequence.
+__device__ __forceinline__ int64_t real_end(const int* lengths, int heads, int64_t bh, int64_t hi) {
+    if (!lengths) return hi;
+    const int64_t len = lengths[bh / heads];
+    return len < hi ? len : hi;
+}
+
 // part[bh][split] = sum over the split's positions of phi(X_i) [Y_i, 1]^T.
 template <typename IO>
 __global__ void __launch_bounds__(THREADS)
 general_kv_sum_kernel(const IO* __restrict__ X, const IO* __restrict__ Y, float* __restrict__ part,
-                      int64_t N, int64_t split_len, int D, int M, int phi) {
+                      int64_t N, int64_t split_len, int D, int M, int phi, const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
     const Dims dm = make_dims(D, M);
     float* sx = smem;
     float* sy = sx + T * dm.DS;
     float* sSt = sy + T * dm.MS;
     const int64_t bh = blockIdx.x, sp = blockIdx.y;
-    const int64_t lo = sp * split_len, hi = (lo + split_len) < N ? (lo + split_len) : N;
+    const int64_t lo = sp * split_len, hi = real_end(lengths, heads, bh, (lo + split_len) < N ? (lo + split_len) : N);
     X += bh * N * D; Y += bh * N * M;
     zero_fill(sSt, D * dm.MS);
     for (int64_t n0 = lo; n0 < hi; n0 += T) {
@@ -365,15 +373,20 @@ template <typename IO>
 __global__ void __launch_bounds__(THREADS)
 general_linear_apply_kernel(const IO* __restrict__ Q, const float* __restrict__ part, IO* __restrict__ O,
                             float* __restrict__ den, float* __restrict__ KV, float* __restrict__ Zs,
-                            int nsplit, int64_t N, int64_t split_len, int D, int M, float eps, int phi) {
+                            int nsplit, int64_t N, int64_t split_len, int D, int M, float eps, int phi,
+                            const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
     const Dims dm = make_dims(D, M);
     float* sq = smem;
     float* snd = sq + T * dm.DS;
     float* sSt = snd + T * dm.MS;
     const int64_t bh = blockIdx.x, sp = blockIdx.y;
-    const int64_t lo = sp * split_len, hi = (lo + split_len) < N ? (lo + split_len) : N;
+    const int64_t lo = sp * split_len, hi_all = (lo + split_len) < N ? (lo + split_len) : N;
+    const int64_t hi = real_end(lengths, heads, bh, hi_all);
     Q += bh * N * D; O += bh * N * M;
+    for (int64_t idx = (lo > hi ? lo : hi) * M + threadIdx.x; idx < hi_all * M; idx += THREADS) O[idx] = from_f32<IO>(0.f);
+    if (den)
+        for (int64_t i = (lo > hi ? lo : hi) + threadIdx.x; i < hi_all; i += THREADS) den[bh * N + i] = 0.f;
     load_reduced_state(sSt, part + bh * nsplit * (int64_t)(D * dm.MS), nsplit, D * dm.MS);
     __syncthreads();
     if (sp == 0) {
@@ -407,7 +420,7 @@ __global__ void __launch_bounds__(THREADS)
 general_linear_bwd_q_kernel(const IO* __restrict__ Q, const IO* __restrict__ G,
                             const float* __restrict__ part_s, IO* __restrict__ dQ,
                             float* __restrict__ part_r, int nsplit, int64_t N, int64_t split_len,
-                            int D, int M, float eps, int phi) {
+                            int D, int M, float eps, int phi, const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
     const Dims dm = make_dims(D, M);
     float* sq = smem;
@@ -416,8 +429,10 @@ general_linear_bwd_q_kernel(const IO* __restrict__ Q, const IO* __restrict__ G,
     float* sSt = snd + T * dm.MS;
     float* sRt = sSt + D * dm.MS;
     const int64_t bh = blockIdx.x, sp = blockIdx.y;
-    const int64_t lo = sp * split_len, hi = (lo + split_len) < N ? (lo + split_len) : N;
+    const int64_t lo = sp * split_len, hi_all = (lo + split_len) < N ? (lo + split_len) : N;
+    const int64_t hi = real_end(lengths, heads, bh, hi_all);
     Q += bh * N * D; G += bh * N * M; dQ += bh * N * D;
+    for (int64_t idx = (lo > hi ? lo : hi) * D + threadIdx.x; idx < hi_all * D; idx += THREADS) dQ[idx] = from_f32<IO>(0.f);
     load_reduced_state(sSt, part_s + bh * nsplit * (int64_t)(D * dm.MS), nsplit, D * dm.MS);
     zero_fill(sRt, D * dm.MS);
     for (int64_t n0 = lo; n0 < hi; n0 += T) {
@@ -448,15 +463,19 @@ template <typename IO>
 __global__ void __launch_bounds__(THREADS)
 general_linear_bwd_kv_kernel(const IO* __restrict__ K, const IO* __restrict__ V,
                              const float* __restrict__ part_r, IO* __restrict__ dK, IO* __restrict__ dV,
-                             int nsplit, int64_t N, int64_t split_len, int D, int M, int phi) {
+                             int nsplit, int64_t N, int64_t split_len, int D, int M, int phi,
+                             const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
     const Dims dm = make_dims(D, M);
     float* sk = smem;
     float* sv = sk + T * dm.DS;
     float* sRt = sv + T * dm.MS;
     const int64_t bh = blockIdx.x, sp = blockIdx.y;
-    const int64_t lo = sp * split_len, hi = (lo + split_len) < N ? (lo + split_len) : N;
+    const int64_t lo = sp * split_len, hi_all = (lo + split_len) < N ? (lo + split_len) : N;
+    const int64_t hi = real_end(lengths, heads, bh, hi_all);
     K += bh * N * D; V += bh * N * M; dK += bh * N * D; dV += bh * N * M;
+    for (int64_t idx = (lo > hi ? lo : hi) * D + threadIdx.x; idx < hi_all * D; idx += THREADS) dK[idx] = from_f32<IO>(0.f);
+    for (int64_t idx = (lo > hi ? lo : hi) * M + threadIdx.x; idx < hi_all * M; idx += THREADS) dV[idx] = from_f32<IO>(0.f);
     load_reduced_state(sRt, part_r + bh * nsplit * (int64_t)(D * dm.MS), nsplit, D * dm.MS);
     for (int64_t n0 = lo; n0 < hi; n0 += T) {
         const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
@@ -495,8 +514,10 @@ size_t general_workspace_bytes(const la_problem& p, int op) {
     switch (op) {
         case LA_OP_CAUSAL_FORWARD: return 0;
         case LA_OP_CAUSAL_BACKWARD: return bh * (size_t)p.N * 2 * sizeof(float);
-        case LA_OP_LINEAR_FORWARD: return bh * choose_split(p).nsplit * state_floats(p) * sizeof(float);
-        case LA_OP_LINEAR_BACKWARD: return 2 * bh * choose_split(p).nsplit * state_floats(p) * sizeof(float);
+        case LA_OP_LINEAR_FORWARD:
+        case LA_OP_LINEAR_VARLEN_FORWARD: return bh * choose_split(p).nsplit * state_floats(p) * sizeof(float);
+        case LA_OP_LINEAR_BACKWARD:
+        case LA_OP_LINEAR_VARLEN_BACKWARD: return 2 * bh * choose_split(p).nsplit * state_floats(p) * sizeof(float);
         default: return 0;
     }
 }
@@ -540,8 +561,8 @@ int general_causal_backward(const la_problem& p, const void* Q, const void* K, c
 }
 
 template <typename IO>
-static int linear_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
-                            float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
+static int linear_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
+                            void* O, float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
     const int D = (int)p.D, M = (int)p.M;
     const Split sp = choose_split(p);
     const dim3 grid((unsigned)(p.B * p.H), (unsigned)sp.nsplit);
@@ -550,7 +571,7 @@ static int linear_forward_t(const la_problem& p, const void* Q, const void* K, c
         const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
         auto kern = general_kv_sum_kernel<IO>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
-        kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part, p.N, sp.len, D, M, p.phi);
+        kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part, p.N, sp.len, D, M, p.phi, lengths, (int)p.H);
         LA_LAUNCHED();
     }
     {
@@ -558,20 +579,20 @@ static int linear_forward_t(const la_problem& p, const void* Q, const void* K, c
         auto kern = general_linear_apply_kernel<IO>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
         kern<<<grid, THREADS, smem, st>>>((const IO*)Q, part, (IO*)O, den, KV, Zs, sp.nsplit, p.N, sp.len, D, M,
-                                          p.eps, p.phi);
+                                          p.eps, p.phi, lengths, (int)p.H);
         LA_LAUNCHED();
     }
     return LA_OK;
 }
 
-int general_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O,
-                           float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
-    return p.dtype == LA_F32 ? linear_forward_t<float>(p, Q, K, V, O, den, KV, Zs, ws, st)
-                             : linear_forward_t<__nv_bfloat16>(p, Q, K, V, O, den, KV, Zs, ws, st);
+int general_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
+                           void* O, float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
+    return p.dtype == LA_F32 ? linear_forward_t<float>(p, Q, K, V, lengths, O, den, KV, Zs, ws, st)
+                             : linear_forward_t<__nv_bfloat16>(p, Q, K, V, lengths, O, den, KV, Zs, ws, st);
 }
 
 template <typename IO>
-static int linear_backward_t(const la_problem& p, const void* Q, const void* K, const void* V,
+static int linear_backward_t(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
                              const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
     const int D = (int)p.D, M = (int)p.M;
     const Split sp = choose_split(p);
@@ -582,7 +603,7 @@ static int linear_backward_t(const la_problem& p, const void* Q, const void* K, 
         const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
         auto kern = general_kv_sum_kernel<IO>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
-        kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part_s, p.N, sp.len, D, M, p.phi);
+        kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part_s, p.N, sp.len, D, M, p.phi, lengths, (int)p.H);
         LA_LAUNCHED();
     }
     {
@@ -590,7 +611,7 @@ static int linear_backward_t(const la_problem& p, const void* Q, const void* K, 
         auto kern = general_linear_bwd_q_kernel<IO>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
         kern<<<grid, THREADS, smem, st>>>((const IO*)Q, (const IO*)G, part_s, (IO*)dQ, part_r, sp.nsplit, p.N,
-                                          sp.len, D, M, p.eps, p.phi);
+                                          sp.len, D, M, p.eps, p.phi, lengths, (int)p.H);
         LA_LAUNCHED();
     }
     {
@@ -598,16 +619,16 @@ static int linear_backward_t(const la_problem& p, const void* Q, const void* K, 
         auto kern = general_linear_bwd_kv_kernel<IO>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
         kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part_r, (IO*)dK, (IO*)dV, sp.nsplit, p.N,
-                                          sp.len, D, M, p.phi);
+                                          sp.len, D, M, p.phi, lengths, (int)p.H);
         LA_LAUNCHED();
     }
     return LA_OK;
 }
 
-int general_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
-                            void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
-    return p.dtype == LA_F32 ? linear_backward_t<float>(p, Q, K, V, G, dQ, dK, dV, ws, st)
-                             : linear_backward_t<__nv_bfloat16>(p, Q, K, V, G, dQ, dK, dV, ws, st);
+int general_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
+                            const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    return p.dtype == LA_F32 ? linear_backward_t<float>(p, Q, K, V, lengths, G, dQ, dK, dV, ws, st)
+                             : linear_backward_t<__nv_bfloat16>(p, Q, K, V, lengths, G, dQ, dK, dV, ws, st);
 }
 
 }  // namespace la

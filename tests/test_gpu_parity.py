@@ -337,6 +337,47 @@ def test_right_padded_causal_batches_need_no_mask(dtype, D, N):
             assert float(t[b, :, n:].float().abs().max()) == 0.0 if n < N else True, f"{nm} on the padding"
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape,lengths", [((3, 2, 100, 16, 48), [100, 37, 1]), ((4, 2, 517, 64, 64), [517, 0, 300, 129]),
+                                           ((2, 4, 1024, 64, 64), [1024, 700])])
+def test_noncausal_ragged_batches(shape, lengths, dtype):
+    """Right-padded sequences of different lengths (key-padding mask): every sequence equals the oracle run on
+    its own length, sums included, and everything is zero on the padding whatever the tensors hold there."""
+    B, H, N, D, M = shape
+    Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=sum(shape) + 4, dtype=dtype)
+    for b, n in enumerate(lengths):
+        Q[b, :, n:] = 5.0
+        K[b, :, n:] = 6.0
+        V[b, :, n:] = -30.0
+        G[b, :, n:] = 2.0
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    ld = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    den = torch.empty((B, H, N), device=DEV)
+    KV = torch.empty((B, H, D, M), device=DEV)
+    Zs = torch.empty((B, H, D), device=DEV)
+    O = la.la_linear_attention_varlen(Qd, Kd, Vd, ld, den=den, KV=KV, Zs=Zs)
+    dQ, dK, dV = la.la_linear_attention_varlen_backward(Qd, Kd, Vd, Gd, ld)
+    la.la_last_device_status()
+    for b, n in enumerate(lengths):
+        pad = (slice(b, b + 1), slice(None), slice(n, N))
+        for t in (O, den, dQ, dK, dV):
+            assert n == N or float(t[pad].float().abs().max()) == 0.0
+        if n == 0:
+            assert float(KV[b].abs().max()) == 0.0 and float(Zs[b].abs().max()) == 0.0
+            continue
+        sl = (slice(b, b + 1), slice(None), slice(0, n))
+        q, k, v, g = Q[sl], K[sl], V[sl], G[sl]
+        Or, denr, Sr, Zr = oracle.linear_attention(q, k, v, False, return_state=True)
+        assert_close(O[sl], Or, dtype, f"O, length {n}")
+        assert_close(den[sl], denr, dtype, f"den, length {n}")
+        assert_close(KV[b:b + 1], Sr, dtype, f"KV, length {n}")
+        assert_close(Zs[b:b + 1], Zr, dtype, f"Zs, length {n}")
+        rq, rk, rv = oracle.linear_attention_backward(q, k, v, g, False)
+        assert_close(dQ[sl], rq, dtype, f"dQ, length {n}", grad=True)
+        assert_close(dK[sl], rk, dtype, f"dK, length {n}", grad=True)
+        assert_close(dV[sl], rv, dtype, f"dV, length {n}", grad=True)
+
+
 def test_gradient_invariants_hold_on_gpu_results():
     B, H, N, D, M = 2, 4, 512, 64, 64
     Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=11, dtype=torch.float32)

@@ -155,6 +155,17 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert back(_p(), dZ_in=odd) == -1
     assert back(_p()) == -3                                             # plain backward: needs its workspace
     assert back(_p(N=0)) == 0
+    # ragged batches: the lengths are required and 4-byte aligned
+    pv = _p()
+    need_v = la.la_workspace_bytes(pv, binding.LA_OP_LINEAR_VARLEN_FORWARD)
+    assert need_v > 0 and la.la_workspace_bytes(pv, binding.LA_OP_LINEAR_VARLEN_BACKWARD) >= need_v
+    assert L.la_linear_attention_varlen(ctypes.byref(pv), ok, ok, ok, null, ok, null, null, null, big, 1 << 40, null) == -1
+    assert b"lengths" in L.la_last_error()
+    assert L.la_linear_attention_varlen(ctypes.byref(pv), ok, ok, ok, ctypes.c_void_p(ok.value + 2), ok, null, null, null,
+                                        big, 1 << 40, null) == -1
+    assert L.la_linear_attention_varlen(ctypes.byref(pv), ok, ok, ok, ok, ok, null, null, null, null, 0, null) == -3
+    assert L.la_linear_attention_varlen_backward(ctypes.byref(pv), ok, ok, ok, null, null, null, ok, ok, ok, ok,
+                                                 big, 1 << 40, null) == -1
     assert L.la_feature_map(ok, ok, -5, 0, 0, null) == -1
     assert L.la_feature_map(ok, ok, 0, 0, 0, null) == 0
     assert L.la_feature_map(ok, ok, 4, 9, 0, null) == -1
