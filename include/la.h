@@ -115,8 +115,8 @@ int la_linear_attention_backward(const la_problem* p, const void* Q, const void*
  *   O_i = phi(Q_i)^T sum_{j < len} phi(K_j) V_j^T / (phi(Q_i)^T sum_{j < len} phi(K_j) + eps),
  * KV / Zs are the sums over the real positions, and O, den (and in the backward pass dQ, dK, dV)
  * are written as zeros on the padding; what Q, K, V, G hold there is never used.  Workspace:
- * la_workspace_bytes(p, LA_OP_LINEAR_VARLEN_FORWARD / _BACKWARD).  These calls run the general
- * kernels for every problem (the tensor-core kernels take full-length batches only).  Everything
+ * la_workspace_bytes(p, LA_OP_LINEAR_VARLEN_FORWARD / _BACKWARD).  The same kernels run as for the
+ * full-length calls (splits of a sequence skip the chunks that hold only padding).  Everything
  * else as for la_linear_attention() / la_linear_attention_backward().
  */
 int la_linear_attention_varlen(const la_problem* p, const void* Q, const void* K, const void* V,

@@ -177,7 +177,10 @@ size_t la_workspace_bytes(const la_problem* p, int32_t op) {
     if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_LINEAR_VARLEN_BACKWARD) return 0;
     if (p->N == 0) return 0;
     if (op == LA_OP_CAUSAL_SAVED) return tc_supported(*p, LA_OP_CAUSAL_BACKWARD) ? tc_causal_saved_bytes(*p) : 0;
-    if (op == LA_OP_LINEAR_VARLEN_FORWARD || op == LA_OP_LINEAR_VARLEN_BACKWARD) return general_workspace_bytes(*p, op);
+    if (op == LA_OP_LINEAR_VARLEN_FORWARD || op == LA_OP_LINEAR_VARLEN_BACKWARD) {
+        const int full = op == LA_OP_LINEAR_VARLEN_FORWARD ? LA_OP_LINEAR_FORWARD : LA_OP_LINEAR_BACKWARD;
+        return tc_supported(*p, full) ? tc_workspace_bytes(*p, full) : general_workspace_bytes(*p, op);
+    }
     if (tc_supported(*p, op)) return tc_workspace_bytes(*p, op);
     return general_workspace_bytes(*p, op);
 }
@@ -209,7 +212,7 @@ int la_linear_attention(const la_problem* p, const void* Q, const void* K, const
     if (int rc = check_ws(p, LA_OP_LINEAR_FORWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc_linear_forward(*p, Q, K, V, O, den, KV, Zs, ws, st);
+    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc_linear_forward(*p, Q, K, V, nullptr, O, den, KV, Zs, ws, st);
     return general_linear_forward(*p, Q, K, V, nullptr, O, den, KV, Zs, ws, st);
 }
 
@@ -225,7 +228,9 @@ int la_linear_attention_varlen(const la_problem* p, const void* Q, const void* K
     LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(KV); LA_OPTIONAL_PTR(Zs);
     if (int rc = check_ws(p, LA_OP_LINEAR_VARLEN_FORWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
-    return general_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, ws, (cudaStream_t)stream);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, ws, st);
+    return general_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, ws, st);
 }
 
 int la_linear_attention_backward(const la_problem* p, const void* Q, const void* K, const void* V,
@@ -240,7 +245,7 @@ int la_linear_attention_backward(const la_problem* p, const void* Q, const void*
     if (int rc = check_ws(p, LA_OP_LINEAR_BACKWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc_linear_backward(*p, Q, K, V, G, dQ, dK, dV, ws, st);
+    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc_linear_backward(*p, Q, K, V, nullptr, G, dQ, dK, dV, ws, st);
     return general_linear_backward(*p, Q, K, V, nullptr, G, dQ, dK, dV, ws, st);
 }
 
@@ -258,7 +263,9 @@ int la_linear_attention_varlen_backward(const la_problem* p, const void* Q, cons
     LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den);
     if (int rc = check_ws(p, LA_OP_LINEAR_VARLEN_BACKWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
-    return general_linear_backward(*p, Q, K, V, lengths, G, dQ, dK, dV, ws, (cudaStream_t)stream);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc_linear_backward(*p, Q, K, V, lengths, G, dQ, dK, dV, ws, st);
+    return general_linear_backward(*p, Q, K, V, lengths, G, dQ, dK, dV, ws, st);
 }
 
 static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {

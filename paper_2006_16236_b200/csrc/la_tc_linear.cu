@@ -83,6 +83,8 @@ struct LsParams {
     float* records;        // [BH][nseg][kRecFloats]
     const float* dn;       // null: forward sums (w_i = 1, aux = 1); else w_i = 1 / dn_i, aux = dl_i
     const float* dl;
+    const int* lengths;    // [B] real positions per batch element (right-padded ragged batch), or null
+    int heads;
     int* status;
     int64_t N;
     int chunks, chunks_per_seg, nseg;
@@ -101,9 +103,18 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const int seg = blockIdx.x % prm.nseg;
     const int64_t bh = blockIdx.x / prm.nseg;
     const int c_begin = seg * prm.chunks_per_seg;
-    const int L = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
+    const int L_all = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
     const bool reverse = prm.dn != nullptr;
+    // Ragged batch: only `real` rows of this split exist; chunks behind them are skipped and the rows behind
+    // them in the last chunk are zeroed after the load (at least one chunk runs, so that the record is written
+    // from an accumulator that holds zeros and not from one that was never started).
+    int64_t real = (int64_t)L_all * kChunk;
+    if (prm.lengths) {
+        const int64_t len = min((int64_t)max(prm.lengths[bh / prm.heads], 0), prm.N);
+        real = min(max(len - (int64_t)c_begin * kChunk, (int64_t)0), real);
+    }
+    const int L = max(1, (int)((real + kChunk - 1) / kChunk));
 
     if (tid == 0) {
         for (int s = 0; s < kLsStages; ++s) {
@@ -194,10 +205,25 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 w = 1.f / __ldg(prm.dn + row);
                 delta = __ldg(prm.dl + row);
             }
+            const bool padded = (int64_t)c * kChunk + t >= real;
+            if (padded) {           // whatever the tensors hold there must not be read as numbers
+                w = 0.f;
+                delta = 0.f;
+            }
             if (!mbar_wait(&bars->full[s], (c / kLsStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             uint8_t* rowX = smem + s * kLsStageBytes + t * 128;
-            if (elu) elu_row_inplace<true>(rowX, r7, w, prm.dim >> 3); else elu_row_inplace<false>(rowX, r7, w, prm.dim >> 3);
+            if (padded) {
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc) {
+                    sts128(rowX + (cc << 4), 0u, 0u, 0u, 0u);
+                    sts128(rowX + kTileBytes + (cc << 4), 0u, 0u, 0u, 0u);
+                }
+            } else if (elu) {
+                elu_row_inplace<true>(rowX, r7, w, prm.dim >> 3);
+            } else {
+                elu_row_inplace<false>(rowX, r7, w, prm.dim >> 3);
+            }
             if (reverse) {
                 uint8_t* rowW = rowX + 2 * kTileBytes;
                 uint8_t* rowA = rowX + 3 * kTileBytes;
@@ -279,6 +305,8 @@ struct ApParams {
     float* dl;                  // backward Q: dl_i (out)
     float* state_out;           // forward: KV [BH][64][64] (optional)
     float* vec_out;             // forward: Zs [BH][64] (optional)
+    const int* lengths;         // [B] real positions per batch element (right-padded ragged batch), or null
+    int heads;
     int* status;
     int64_t N;
     int chunks, chunks_per_seg, nseg;
@@ -306,8 +334,16 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     const int seg = blockIdx.x % prm.nseg;
     const int64_t bh = blockIdx.x / prm.nseg;
     const int c_begin = seg * prm.chunks_per_seg;
-    const int L = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
+    const int L_all = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
+    // Ragged batch: `len` positions of this sequence exist, `real` of them in this split.  Only the chunks that
+    // hold real rows go through the pipeline; the padding behind them is filled with zeros at the end.
+    int64_t len = prm.N, real = (int64_t)L_all * kChunk;
+    if (prm.lengths) {
+        len = min((int64_t)max(prm.lengths[bh / prm.heads], 0), prm.N);
+        real = min(max(len - (int64_t)c_begin * kChunk, (int64_t)0), real);
+    }
+    const int L = (int)((real + kChunk - 1) / kChunk);
 
     if (tid == 0) {
         for (int s = 0; s < kApStages; ++s) {
@@ -358,7 +394,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             sF[kDim * kDim + tid] = m;                                            // mu, just past the matrix
             if (kMode == kApplyForward && seg == 0 && tid < dim) {
                 // true sums for the caller: S = 1 ysum^T + A', Z = N 1 + a'
-                if (prm.vec_out) prm.vec_out[bh * dim + tid] = (float)prm.N + sA[tid];
+                if (prm.vec_out) prm.vec_out[bh * dim + tid] = (float)len + sA[tid];
                 if (prm.state_out)
                     for (int d = 0; d < dim; ++d)
                         prm.state_out[bh * (int64_t)(dim * dim) + d * dim + tid] = sF[d * kDim + tid] + ysum;
@@ -461,7 +497,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const bool elu = prm.phi == LA_PHI_ELU1;
-        const float fD = (float)prm.dim, fN = (float)prm.N;
+        const float fD = (float)prm.dim, fN = (float)len;
         // (columns beyond a 32-wide problem are zero padding: they add nothing to the sums, and the store clips them)
         float* sX = reinterpret_cast<float*>(smem + kApOffX);
         float* mine = sX + (hf * 128 + t) * 8;
@@ -472,6 +508,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         for (int c = 0; c < L; ++c) {
             const int s = c % kApStages, b = c & 1;
             const int64_t row = row0 + (int64_t)c * kChunk + t;
+            const bool padded = (int64_t)c * kChunk + t >= real;      // a row behind the sequence's end: zeros go out
             if (!mbar_wait(&bars->mapped[s], (c / kApStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             uint32_t xv[4][4];                       // this half of the x' = elu(X) row
@@ -540,7 +577,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 const float den = fN * x1sum + sScal[0] + xa;
                 const float inv = 1.f / (den + prm.eps);
                 const float w = x1sum * inv;
-                if (hf == 0 && prm.den) prm.den[row] = den;
+                if (hf == 0 && prm.den) prm.den[row] = padded ? 0.f : den;
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     const float* nu = nuH + cc * 8;
@@ -601,6 +638,13 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     }
                 }
             }
+            if (padded) {
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    sts128(out_row + (((hf * 4 + cc) ^ r7) << 4), 0u, 0u, 0u, 0u);
+                    if (kMode == kApplyBackwardKV) sts128(out_row + kTileBytes + (((hf * 4 + cc) ^ r7) << 4), 0u, 0u, 0u, 0u);
+                }
+            }
             tc_fence_before_sync();
             mbar_arrive(&bars->acc_free[b]);
             fence_proxy_async_smem();
@@ -613,6 +657,19 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             }
         }
         if (hf == 0 && lane == 0) tma_store_wait_all<0>();
+        if (L < L_all) {            // whole chunks of padding: zeros, written directly
+            const int e = hf * 128 + t;
+            const int64_t r_lo = row0 + (int64_t)L * kChunk, nrows = (int64_t)(L_all - L) * kChunk;
+            const int64_t n16 = nrows * prm.dim * 2 / 16;
+            uint4* o0 = reinterpret_cast<uint4*>(prm.out0 + r_lo * prm.dim);
+            for (int64_t i = e; i < n16; i += 256) o0[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (kMode == kApplyBackwardKV) {
+                uint4* o1 = reinterpret_cast<uint4*>(prm.out1 + r_lo * prm.dim);
+                for (int64_t i = e; i < n16; i += 256) o1[i] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            if (kMode == kApplyForward && prm.den)
+                for (int64_t i = e; i < nrows; i += 256) prm.den[r_lo + i] = 0.f;
+        }
     }
 
     tc_fence_before_sync();
@@ -639,7 +696,7 @@ Segmentation choose_splits(const la_problem& p) {
 }
 
 int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
-                const float* dn, const float* dl, float* records, cudaStream_t st) {
+                const float* dn, const float* dl, const int* lengths, float* records, cudaStream_t st) {
     static bool attr_done = false;
     if (!attr_done) {
         LA_CUDA_TRY(cudaFuncSetAttribute(linear_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLsSmemBytes));
@@ -649,6 +706,8 @@ int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& 
     prm.records = records;
     prm.dn = dn;
     prm.dl = dl;
+    prm.lengths = lengths;
+    prm.heads = (int)p.H;
     prm.status = device_status_ptr();
     if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
     prm.N = p.N;
@@ -674,6 +733,7 @@ int launch_apply(const la_problem& p, const Segmentation& sg, const CUtensorMap&
     }
     prm.status = device_status_ptr();
     if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
+    prm.heads = (int)p.H;
     prm.N = p.N;
     prm.chunks = (int)(p.N / kChunk);
     prm.chunks_per_seg = sg.chunks_per_seg;
@@ -702,8 +762,8 @@ size_t linear_backward_workspace(const la_problem& p) {
     return 2 * linear_forward_workspace(p) + 2 * (size_t)(p.B * p.H) * (size_t)p.N * sizeof(float);
 }
 
-int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, void* O, float* den,
-                   float* KV, float* Zs, void* ws, cudaStream_t st) {
+int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, void* O,
+                   float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
     const Segmentation sg = choose_splits(p);
     const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
     CUtensorMap mQ, mK, mV;
@@ -711,8 +771,9 @@ int linear_forward(const la_problem& p, const void* Q, const void* K, const void
     if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
     if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
     float* rec = (float*)ws;
-    if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, rec, st)) return rc;
+    if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, lengths, rec, st)) return rc;
     ApParams a = {};
+    a.lengths = lengths;
     a.records = rec;
     a.out0 = (__nv_bfloat16*)O;
     a.den = den;
@@ -721,8 +782,8 @@ int linear_forward(const la_problem& p, const void* Q, const void* K, const void
     return launch_apply<kApplyForward>(p, sg, mQ, mQ, a, st);
 }
 
-int linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
-                    void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+int linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
+                    const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
     const Segmentation sg = choose_splits(p);
     const size_t bh = (size_t)(p.B * p.H);
     const uint64_t rows = (uint64_t)(bh * p.N);
@@ -737,15 +798,17 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
     float* dn = (float*)w;      w += bh * (size_t)p.N * sizeof(float);
     float* dl = (float*)w;
 
-    if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, rec_s, st)) return rc;
+    if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, lengths, rec_s, st)) return rc;
     ApParams a = {};
+    a.lengths = lengths;
     a.records = rec_s;
     a.out0 = (__nv_bfloat16*)dQ;
     a.den = dn;
     a.dl = dl;
     if (int rc = launch_apply<kApplyBackwardQ>(p, sg, mQ, mG, a, st)) return rc;
-    if (int rc = launch_sums(p, sg, mQ, mG, dn, dl, rec_r, st)) return rc;
+    if (int rc = launch_sums(p, sg, mQ, mG, dn, dl, lengths, rec_r, st)) return rc;
     ApParams b = {};
+    b.lengths = lengths;
     b.records = rec_r;
     b.out0 = (__nv_bfloat16*)dK;
     b.out1 = (__nv_bfloat16*)dV;

@@ -339,17 +339,21 @@ def test_right_padded_causal_batches_need_no_mask(dtype, D, N):
 
 @pytest.mark.parametrize("dtype", DTYPES)
 @pytest.mark.parametrize("shape,lengths", [((3, 2, 100, 16, 48), [100, 37, 1]), ((4, 2, 517, 64, 64), [517, 0, 300, 129]),
-                                           ((2, 4, 1024, 64, 64), [1024, 700])])
+                                           ((2, 4, 1024, 64, 64), [1024, 700]),
+                                           ((5, 2, 2048, 64, 64), [2048, 0, 129, 1500, 1024]),
+                                           ((3, 2, 512, 32, 32), [512, 130, 1])])
 def test_noncausal_ragged_batches(shape, lengths, dtype):
     """Right-padded sequences of different lengths (key-padding mask): every sequence equals the oracle run on
-    its own length, sums included, and everything is zero on the padding whatever the tensors hold there."""
+    its own length, sums included, and everything is zero on the padding whatever the tensors hold there
+    (not even numbers).  The bf16 cases with D = M in {32, 64} and N a multiple of 128 run the tensor-core
+    kernels, whose splits end inside, at and before a sequence's end; the others the general kernels."""
     B, H, N, D, M = shape
     Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=sum(shape) + 4, dtype=dtype)
     for b, n in enumerate(lengths):
         Q[b, :, n:] = 5.0
-        K[b, :, n:] = 6.0
+        K[b, :, n:] = float("inf")
         V[b, :, n:] = -30.0
-        G[b, :, n:] = 2.0
+        G[b, :, n:] = float("nan")
     Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
     ld = torch.tensor(lengths, dtype=torch.int32, device=DEV)
     den = torch.empty((B, H, N), device=DEV)
