@@ -187,3 +187,49 @@ def recurrent_step(q, k, v, S, Z, phi: str = "elu1", eps: float = 0.0):
     _load().la_oracle_recurrent_step(B, H, D, M, PHI[phi], eps,
                                      _p(q), _p(k), _p(v), _p(S), _p(Z), _p(out))
     return out
+
+
+# ---------------------------------------------------------------------------
+# Degree-2 polynomial kernel (Section 3.2.1, "Feature Maps and Computational Cost"): the kernel
+# sim(a, b) = (a . b)^2 has the exact finite feature map phi(a) = vec(a a^T) of dimension C = D^2.
+# The paper names the kernel and its cost O(N D^2 M) without fixing its form; the homogeneous form is
+# the one whose feature map has exactly D^2 components.  Plain numpy, written from the definitions.
+# ---------------------------------------------------------------------------
+def poly2_feature_map(x, C_pad: int | None = None):
+    """phi(x)[..., i*D + j] = x_i x_j; columns D*D .. C_pad-1 (if asked for) are zero."""
+    x = _f64(x)
+    D = x.shape[-1]
+    C = D * D
+    C_pad = C if C_pad is None else int(C_pad)
+    if C_pad < C:
+        raise ValueError("C_pad is smaller than D*D")
+    y = np.zeros(x.shape[:-1] + (C_pad,))
+    for i in range(D):
+        for j in range(D):
+            y[..., i * D + j] = x[..., i] * x[..., j]
+    return y
+
+
+def poly2_feature_map_backward(x, dy):
+    """Gradient of poly2_feature_map: dx_i = sum_j (dy[i*D + j] + dy[j*D + i]) x_j."""
+    x, dy = _f64(x), _f64(dy)
+    D = x.shape[-1]
+    dx = np.zeros_like(x)
+    for i in range(D):
+        for j in range(D):
+            dx[..., i] += (dy[..., i * D + j] + dy[..., j * D + i]) * x[..., j]
+    return dx
+
+
+def poly2_attention(Q, K, V, causal: bool, eps: float = 0.0):
+    """Eq. 3 (Eq. 8 when causal) with sim(q, k) = (q . k)^2 on the explicit N x N matrix."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    B, H, N, _ = Q.shape
+    O = np.empty(V.shape)
+    for b in range(B):
+        for h in range(H):
+            A = (Q[b, h] @ K[b, h].T) ** 2
+            if causal:
+                A = np.tril(A)
+            O[b, h] = (A @ V[b, h]) / (A.sum(axis=1, keepdims=True) + eps)
+    return O

@@ -378,3 +378,54 @@ def test_linear_matches_quadratic_on_larger_case():
 
 def test_threads_reported():
     assert oracle.num_threads() >= 1
+
+
+# --------------------------------------------------------------------------
+# Degree-2 polynomial kernel (Section 3.2.1): exact finite feature map.
+# --------------------------------------------------------------------------
+def test_poly2_feature_map_hand_example_and_kernel_identity():
+    # a = (1, 2): a a^T = [[1, 2], [2, 4]], row-major; padding columns are zero
+    assert oracle.poly2_feature_map([1.0, 2.0], 8).tolist() == [1.0, 2.0, 2.0, 4.0, 0.0, 0.0, 0.0, 0.0]
+    # (3, -1).(1, 2) = 1, squared 1; by features: 9*1 + (-3)*2 + (-3)*2 + 1*4 = 1
+    assert float(oracle.poly2_feature_map([3.0, -1.0]) @ oracle.poly2_feature_map([1.0, 2.0])) == 1.0
+    rng = np.random.default_rng(3)
+    for D in (1, 3, 8, 11):
+        a, b = rng.standard_normal((50, D)), rng.standard_normal((50, D))
+        lhs = (oracle.poly2_feature_map(a, 128) * oracle.poly2_feature_map(b, 128)).sum(-1)
+        np.testing.assert_allclose(lhs, (a * b).sum(-1) ** 2, rtol=1e-12, atol=1e-12)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_poly2_attention_equals_linear_attention_on_the_features(causal):
+    """The similarity form on the N x N matrix of (q.k)^2 against the linear form (sums of phi(k) v^T)
+    on the explicit features: two codes that share nothing."""
+    rng = np.random.default_rng(5 + causal)
+    B, H, N, D, M = 2, 2, 37, 4, 6
+    Q, K, V = rng.standard_normal((B, H, N, D)), rng.standard_normal((B, H, N, D)), rng.standard_normal((B, H, N, M))
+    ref = oracle.poly2_attention(Q, K, V, causal)
+    fQ, fK = oracle.poly2_feature_map(Q, 24), oracle.poly2_feature_map(K, 24)
+    np.testing.assert_allclose(oracle.linear_attention(fQ, fK, V, causal, "identity")[0], ref, rtol=1e-9, atol=1e-11)
+    # hand case: one query, two keys: weights (q.k1)^2 : (q.k2)^2 = 4 : 1
+    o = oracle.poly2_attention([[[[1.0, 0.0]] * 2]], [[[[2.0, 5.0], [1.0, -3.0]]]], [[[[10.0], [20.0]]]], False)
+    np.testing.assert_allclose(o[0, 0, :, 0], [12.0, 12.0], rtol=1e-15)
+
+
+def test_poly2_backward_matches_finite_differences():
+    rng = np.random.default_rng(9)
+    B, H, N, D, M = 1, 2, 9, 3, 4
+    Q, K, V, G = (rng.standard_normal((B, H, N, d)) for d in (D, D, M, M))
+
+    def loss(q, k):
+        return float((oracle.poly2_attention(q, k, V, True) * G).sum())
+
+    fQ, fK = oracle.poly2_feature_map(Q, 16), oracle.poly2_feature_map(K, 16)
+    dfQ, dfK, _ = oracle.linear_attention_backward(fQ, fK, V, G, True, "identity")
+    dQ, dK = oracle.poly2_feature_map_backward(Q, dfQ), oracle.poly2_feature_map_backward(K, dfK)
+    h = 1e-6
+    for X, dX, which in ((Q, dQ, 0), (K, dK, 1)):
+        for idx in [(0, 0, 0, 0), (0, 1, 4, 2), (0, 0, 8, 1), (0, 1, 3, 0)]:
+            Xp, Xm = X.copy(), X.copy()
+            Xp[idx] += h
+            Xm[idx] -= h
+            fd = (loss(Xp, K) - loss(Xm, K)) / (2 * h) if which == 0 else (loss(Q, Xp) - loss(Q, Xm)) / (2 * h)
+            assert abs(fd - dX[idx]) <= 1e-6 * max(1.0, abs(fd)), (which, idx, fd, dX[idx])
