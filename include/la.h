@@ -85,6 +85,23 @@ typedef struct {
 int la_feature_map(const void* x, void* y, int64_t n, int32_t dtype, int32_t deriv, void* stream);
 
 /*
+ * Degree-2 polynomial kernel (Section 3.2.1, "Feature Maps and Computational Cost"): the kernel
+ * sim(a, b) = (a . b)^2 has the exact feature map phi(x) = vec(x x^T) of dimension D*D,
+ *   y[r][i*D + j] = x[r][i] * x[r][j]   (0 <= i, j < D),   y[r][c] = 0 for D*D <= c < C,
+ * so that phi(a) . phi(b) = (a . b)^2.  The attention calls take the mapped queries and keys with
+ * phi = LA_PHI_IDENTITY and D = C (the cost O(N D^2 M) the paper quotes); the zero padding lets C
+ * be the multiple of 8 they ask for.  The paper names the kernel without fixing its form: the
+ * homogeneous one is taken, the one whose feature map has exactly D^2 components.
+ * x: [rows, D], y: [rows, C] of `dtype` (device; y 16-byte aligned; x and y must not overlap).
+ * 1 <= D <= 11, D*D <= C <= 128, C a multiple of 8.  Products are formed in fp32 and rounded once.
+ * The backward call turns dy = dL/dy [rows, C] into dx[r][i] = sum_j (dy[r][i*D+j] + dy[r][j*D+i]) x[r][j]
+ * (fp32 sums; dx: [rows, D], must not alias x).
+ */
+int la_feature_map_poly2(const void* x, void* y, int64_t rows, int64_t D, int64_t C, int32_t dtype, void* stream);
+int la_feature_map_poly2_backward(const void* x, const void* dy, void* dx, int64_t rows, int64_t D, int64_t C,
+                                  int32_t dtype, void* stream);
+
+/*
  * Non-causal linear attention, Eq. 5-6:
  *   KV = sum_j phi(K_j) V_j^T,  Zs = sum_j phi(K_j)   (formed once per head),
  *   O_i = phi(Q_i)^T KV / (phi(Q_i)^T Zs + eps).

@@ -22,7 +22,8 @@ LA_OP_LINEAR_VARLEN_FORWARD, LA_OP_LINEAR_VARLEN_BACKWARD = 5, 6
 _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
-    "la_feature_map", "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
+    "la_feature_map", "la_feature_map_poly2", "la_feature_map_poly2_backward",
+    "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
     "la_linear_attention_varlen", "la_linear_attention_varlen_backward",
     "la_causal_forward", "la_causal_forward_from", "la_causal_backward_from",
     "la_causal_backward", "la_recurrent_step", "la_recurrent_steps", "la_workspace_bytes", "la_status_string",
@@ -57,6 +58,8 @@ def lib() -> ctypes.CDLL:
         vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
         pp = ctypes.POINTER(la_problem)
         L.la_feature_map.argtypes = [vp, vp, i64, i32, i32, vp]
+        L.la_feature_map_poly2.argtypes = [vp, vp, i64, i64, i64, i32, vp]
+        L.la_feature_map_poly2_backward.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp]
         L.la_linear_attention.argtypes = [pp] + [vp] * 7 + [vp, sz, vp]
         L.la_linear_attention_noalloc.argtypes = [pp] + [vp] * 7 + [vp]
         L.la_linear_attention_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
@@ -207,6 +210,32 @@ def la_feature_map(x: torch.Tensor, deriv: bool = False, out: torch.Tensor | Non
     y = torch.empty_like(x) if out is None else out
     _check(lib().la_feature_map(_ptr(x), _ptr(y), x.numel(), _dtype_code(x), int(deriv), _stream(dev)))
     return y
+
+
+def poly2_columns(D: int) -> int:
+    """Feature columns the degree-2 polynomial map of a D-vector is padded to: D*D rounded up to a multiple of 8."""
+    return (D * D + 7) // 8 * 8
+
+
+def la_feature_map_poly2(x: torch.Tensor, C: int | None = None, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Degree-2 polynomial feature map along the last axis: [..., D] -> [..., C] (C defaults to poly2_columns(D));
+    feed the result to the attention calls with phi="identity"."""
+    dev = _dev(x, out)
+    D = x.shape[-1]
+    C = poly2_columns(D) if C is None else C
+    y = torch.empty(x.shape[:-1] + (C,), dtype=x.dtype, device=x.device) if out is None else out
+    _check(lib().la_feature_map_poly2(_ptr(x), _ptr(y), x.numel() // max(D, 1), D, C, _dtype_code(x), _stream(dev)))
+    return y
+
+
+def la_feature_map_poly2_backward(x: torch.Tensor, dy: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Gradient of la_feature_map_poly2 with respect to x for an upstream gradient dy [..., C]."""
+    dev = _dev(x, dy, out)
+    D, C = x.shape[-1], dy.shape[-1]
+    dx = torch.empty_like(x) if out is None else out
+    _check(lib().la_feature_map_poly2_backward(_ptr(x), _ptr(dy), _ptr(dx), x.numel() // max(D, 1), D, C,
+                                               _dtype_code(x), _stream(dev)))
+    return dx
 
 
 def la_linear_attention(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, KV=None, Zs=None, ws=None):

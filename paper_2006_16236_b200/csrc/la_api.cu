@@ -202,6 +202,35 @@ int la_feature_map(const void* x, void* y, int64_t n, int32_t dtype, int32_t der
     return launch_feature_map(x, y, n, dtype, deriv != 0, (cudaStream_t)stream);
 }
 
+static int check_poly2(int64_t rows, int64_t D, int64_t C, int32_t dtype) {
+    if (rows < 0) return fail(LA_ERR_INVALID_ARG, "rows must be >= 0");
+    if (dtype != LA_F32 && dtype != LA_BF16) return fail(LA_ERR_INVALID_ARG, "dtype %d is not a la_dtype", dtype);
+    if (D < 1 || D > 11) return fail(LA_ERR_INVALID_ARG, "D=%lld: the feature dimension D*D must fit 128 columns", (long long)D);
+    if (C < D * D || C > 128 || C % 8) return fail(LA_ERR_INVALID_ARG, "C=%lld must be a multiple of 8 in [D*D, 128]", (long long)C);
+    return LA_OK;
+}
+
+int la_feature_map_poly2(const void* x, void* y, int64_t rows, int64_t D, int64_t C, int32_t dtype, void* stream) {
+    if (int rc = check_poly2(rows, D, C, dtype)) return rc;
+    if (rows == 0) return LA_OK;
+    if (!x) return fail(LA_ERR_INVALID_ARG, "x is NULL");
+    LA_REQUIRE_PTR(y);
+    if (int rc = check_arch()) return rc;
+    return launch_poly2_map(x, y, rows, (int)D, (int)C, dtype, (cudaStream_t)stream);
+}
+
+int la_feature_map_poly2_backward(const void* x, const void* dy, void* dx, int64_t rows, int64_t D, int64_t C,
+                                  int32_t dtype, void* stream) {
+    if (int rc = check_poly2(rows, D, C, dtype)) return rc;
+    if (rows == 0) return LA_OK;
+    if (!x) return fail(LA_ERR_INVALID_ARG, "x is NULL");
+    if (!dy) return fail(LA_ERR_INVALID_ARG, "dy is NULL");
+    if (!dx) return fail(LA_ERR_INVALID_ARG, "dx is NULL");
+    if (dx == x) return fail(LA_ERR_INVALID_ARG, "dx must not alias x");
+    if (int rc = check_arch()) return rc;
+    return launch_poly2_map_backward(x, dy, dx, rows, (int)D, (int)C, dtype, (cudaStream_t)stream);
+}
+
 int la_linear_attention(const la_problem* p, const void* Q, const void* K, const void* V,
                         void* O, float* den, float* KV, float* Zs,
                         void* ws, size_t ws_bytes, void* stream) {

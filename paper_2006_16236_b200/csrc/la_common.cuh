@@ -69,6 +69,9 @@ __device__ __forceinline__ float phi_slope_from_value(float y, int phi) {
 
 // ---- launchers implemented in the kernel files -------------------------------
 int launch_feature_map(const void* x, void* y, int64_t n, int dtype, int deriv, cudaStream_t st);
+int launch_poly2_map(const void* x, void* y, int64_t rows, int D, int C, int dtype, cudaStream_t st);
+int launch_poly2_map_backward(const void* x, const void* dy, void* dx, int64_t rows, int D, int C, int dtype,
+                              cudaStream_t st);
 
 int launch_recurrent_steps(const la_problem& p, const void* q, const void* k, const void* v,
                            float* S, float* Z, void* out, cudaStream_t st);

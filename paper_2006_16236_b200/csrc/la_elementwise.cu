@@ -46,6 +46,110 @@ int launch_feature_map(const void* x, void* y, int64_t n, int dtype, int deriv, 
 }
 
 // ---------------------------------------------------------------------------
+// Degree-2 polynomial kernel (Section 3.2.1): the exact feature map of sim(a, b) = (a . b)^2 is
+// phi(x) = vec(x x^T), y[r][i*D + j] = x[r][i] x[r][j]; columns D*D .. C-1 are zero padding, so that
+// the attention kernels (feature map = identity) can take C as their query/key dimension.
+// Bandwidth-bound on the C-wide side: a thread writes (forward) eight consecutive columns with
+// 16-byte stores; the D-wide row of x is re-read through L1.
+// ---------------------------------------------------------------------------
+// Thread layout of both kernels: threadIdx.x = position inside a row (group of eight columns / component i),
+// threadIdx.y = row inside the block; no division by a run-time number per element.
+template <typename T>
+__global__ void __launch_bounds__(256)
+poly2_map_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows, int D, int C) {
+    const int c0 = threadIdx.x << 3, DD = D * D;
+    const int i0 = c0 / D, j0 = c0 - i0 * D;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.y;
+    for (int64_t r = (int64_t)blockIdx.x * blockDim.y + threadIdx.y; r < rows; r += stride) {
+        const T* xr = x + r * D;
+        T out[8];
+        if (sizeof(T) == 2 && D == 8) {          // a group is row i0 of x x^T: x_i0 times the 16-byte row of x
+            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(xr));
+            const T* xe = reinterpret_cast<const T*>(&raw);
+            const float xi = to_f32<T>(__ldg(xr + (i0 & 7)));     // (a group of padding columns has no row)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) out[e] = from_f32<T>(c0 < DD ? xi * to_f32<T>(xe[e]) : 0.f);
+        } else {
+            int i = i0, j = j0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                out[e] = from_f32<T>(c0 + e < DD ? to_f32<T>(__ldg(xr + i)) * to_f32<T>(__ldg(xr + j)) : 0.f);
+                if (++j == D) { j = 0; ++i; }
+            }
+        }
+        T* dst = y + r * C + c0;
+        if (sizeof(T) == 2) {
+            *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(out);
+        } else {
+            reinterpret_cast<uint4*>(dst)[0] = reinterpret_cast<const uint4*>(out)[0];
+            reinterpret_cast<uint4*>(dst)[1] = reinterpret_cast<const uint4*>(out)[1];
+        }
+    }
+}
+
+// dx[r][i] = sum_j (dy[r][i*D + j] + dy[r][j*D + i]) x[r][j]; one thread per (r, i), fp32 sums.
+template <typename T>
+__global__ void __launch_bounds__(256)
+poly2_map_backward_kernel(const T* __restrict__ x, const T* __restrict__ dy, T* __restrict__ dx,
+                          int64_t rows, int D, int C) {
+    const int i = threadIdx.x;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.y;
+    for (int64_t r = (int64_t)blockIdx.x * blockDim.y + threadIdx.y; r < rows; r += stride) {
+        const T* xr = x + r * D;
+        const T* gr = dy + r * C;
+        float s = 0.f;
+        if (sizeof(T) == 2 && D == 8) {          // row i of dy and the row of x in one 16-byte load each
+            const uint4 rawg = __ldg(reinterpret_cast<const uint4*>(gr + i * 8));
+            const uint4 rawx = __ldg(reinterpret_cast<const uint4*>(xr));
+            const T* ge = reinterpret_cast<const T*>(&rawg);
+            const T* xe = reinterpret_cast<const T*>(&rawx);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                s = fmaf(to_f32<T>(ge[j]) + to_f32<T>(__ldg(gr + j * 8 + i)), to_f32<T>(xe[j]), s);
+        } else {
+            for (int j = 0; j < D; ++j)
+                s = fmaf(to_f32<T>(__ldg(gr + i * D + j)) + to_f32<T>(__ldg(gr + j * D + i)), to_f32<T>(__ldg(xr + j)), s);
+        }
+        dx[r * D + i] = from_f32<T>(s);
+    }
+}
+
+// blocks of (width, 256 / width) threads over the rows, at most 16 blocks per SM
+static void poly2_launch_shape(int64_t rows, int width, dim3* grid, dim3* block) {
+    const int rpb = 256 / width;
+    int64_t blocks = (rows + rpb - 1) / rpb;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    *grid = dim3((unsigned)blocks);
+    *block = dim3((unsigned)width, (unsigned)rpb);
+}
+
+int launch_poly2_map(const void* x, void* y, int64_t rows, int D, int C, int dtype, cudaStream_t st) {
+    if (rows == 0) return LA_OK;
+    dim3 grid, block;
+    poly2_launch_shape(rows, C >> 3, &grid, &block);
+    if (dtype == LA_F32)
+        poly2_map_kernel<float><<<grid, block, 0, st>>>((const float*)x, (float*)y, rows, D, C);
+    else
+        poly2_map_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, rows, D, C);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+int launch_poly2_map_backward(const void* x, const void* dy, void* dx, int64_t rows, int D, int C, int dtype,
+                              cudaStream_t st) {
+    if (rows == 0) return LA_OK;
+    dim3 grid, block;
+    poly2_launch_shape(rows, D, &grid, &block);
+    if (dtype == LA_F32)
+        poly2_map_backward_kernel<float><<<grid, block, 0, st>>>((const float*)x, (const float*)dy, (float*)dx, rows, D, C);
+    else
+        poly2_map_backward_kernel<__nv_bfloat16><<<grid, block, 0, st>>>(
+            (const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, (__nv_bfloat16*)dx, rows, D, C);
+    LA_LAUNCHED();
+    return LA_OK;
+}
+
+// ---------------------------------------------------------------------------
 // Recurrent step.  One CTA of 128 threads per (batch, head) state.  The D x M
 // fp32 state is streamed HBM -> registers -> HBM exactly once with 16-byte
 // accesses: a thread owns four consecutive columns of every RPP-th row, so a

@@ -382,6 +382,84 @@ def test_noncausal_ragged_batches(shape, lengths, dtype):
         assert_close(dV[sl], rv, dtype, f"dV, length {n}", grad=True)
 
 
+# --------------------------------------------------------------------------
+# Degree-2 polynomial kernel (Section 3.2.1): explicit feature map + identity-mode attention.
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("D,C", [(1, 8), (3, 16), (8, 64), (8, 72), (11, 128)])
+def test_poly2_feature_map_and_its_gradient(D, C, dtype):
+    rows = (3, 5, 67)                                   # 1005 rows: several blocks and a ragged tail
+    g = torch.Generator().manual_seed(100 * D + C)
+    x = torch.randn(rows + (D,), generator=g).to(dtype)
+    dy = torch.randn(rows + (C,), generator=g).to(dtype)
+    y = la.la_feature_map_poly2(x.to(DEV), C)
+    dx = la.la_feature_map_poly2_backward(x.to(DEV), dy.to(DEV))
+    ref = oracle.poly2_feature_map(x.double().numpy(), C)
+    tol = 2.0 ** -23 if dtype == torch.float32 else 2.0 ** -8       # one rounding of an exact product
+    got = y.double().cpu().numpy()
+    assert got.shape == ref.shape
+    assert np.all(np.abs(got - ref) <= tol * np.abs(ref)), np.abs(got - ref).max()
+    assert np.all(got[..., D * D:] == 0.0)
+    assert_close(dx, oracle.poly2_feature_map_backward(x.double().numpy(), dy.double().numpy()), dtype, "dx", grad=True)
+    assert la.la_feature_map_poly2(torch.empty((0, D), dtype=dtype, device=DEV), C).shape == (0, C)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("shape,signed", [((2, 2, 384, 8, 64), False), ((2, 2, 384, 8, 64), True),
+                                          ((1, 3, 200, 5, 24), True)])
+def test_poly2_attention_end_to_end(shape, signed, causal, dtype):
+    """Queries and keys -> features on the device -> attention with the identity map; gradients through both
+    steps.  D = 8 gives C = 64: in bf16 the tensor-core kernels; D = 5 (C = 25 padded to 32, M = 24) the
+    general ones.  The features are a stored tensor of the I/O type: the device's must equal the oracle's,
+    rounded once, bit for bit, and the attention step is judged on those, like every other input.  Against the
+    exact kernel (q.k)^2 on the N x N matrix the fp32 path meets the fp32 gate; in bf16 the 2^-9 rounding
+    of each stored feature is what remains (a weight (q.k)^2 is a sum of D^2 products that cancel), which
+    no kernel downstream can remove: only a loose bound is asserted there.
+    Signed queries and keys give signed features, and a weight that is small against the products it sums
+    (the first causal rows above all).  The general kernels (fp32 arithmetic) hold the usual gates there; the
+    tensor-core kernels round scores and state to bf16, an error relative to the products and not to their
+    sum: for signed features in bf16 they are held to 0.15, and to the usual gates for features of one sign."""
+    B, H, N, D, M = shape
+    Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=sum(shape) + causal, dtype=dtype)
+    if not signed:
+        Q, K = Q.abs(), K.abs()
+    loose = signed and dtype == torch.bfloat16 and D * D == 64 and N % 128 == 0        # tensor-core kernels
+
+    def check(x, ref, what, grad=False):
+        if loose:
+            from parity import max_rel_err
+            err = max_rel_err(x, ref)
+            assert err < 0.15, f"{what}: {err:.3e}"
+        else:
+            assert_close(x, ref, dtype, what, grad=grad)
+
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    fQ, fK = la.la_feature_map_poly2(Qd), la.la_feature_map_poly2(Kd)
+    fwd = la.la_causal_forward if causal else la.la_linear_attention
+    bwd = la.la_causal_backward if causal else la.la_linear_attention_backward
+    O = fwd(fQ, fK, Vd, phi="identity")
+    dfQ, dfK, dV = bwd(fQ, fK, Vd, Gd, phi="identity")
+    dQ, dK = la.la_feature_map_poly2_backward(Qd, dfQ), la.la_feature_map_poly2_backward(Kd, dfK)
+    la.la_last_device_status()
+    q, k, v, g = (t.double().numpy() for t in (Q, K, V, G))
+    C = fQ.shape[-1]
+    rounded = lambda a: torch.from_numpy(a).to(dtype).double().numpy()
+    rq, rk = rounded(oracle.poly2_feature_map(q, C)), rounded(oracle.poly2_feature_map(k, C))
+    assert np.array_equal(fQ.double().cpu().numpy(), rq) and np.array_equal(fK.double().cpu().numpy(), rk)
+    check(O, oracle.linear_attention(rq, rk, v, causal, "identity")[0], "O")
+    exact = oracle.poly2_attention(q, k, v, causal)
+    if dtype == torch.float32:
+        assert_close(O, exact, dtype, "O against the exact kernel")
+    else:
+        from parity import max_rel_err
+        assert max_rel_err(O, exact) < 0.2
+    rfq, rfk, rv = oracle.linear_attention_backward(rq, rk, v, g, causal, "identity")
+    check(dV, rv, "dV", grad=True)
+    check(dQ, oracle.poly2_feature_map_backward(q, rounded(rfq)), "dQ", grad=True)
+    check(dK, oracle.poly2_feature_map_backward(k, rounded(rfk)), "dK", grad=True)
+
+
 def test_gradient_invariants_hold_on_gpu_results():
     B, H, N, D, M = 2, 4, 512, 64, 64
     Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=11, dtype=torch.float32)

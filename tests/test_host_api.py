@@ -169,6 +169,17 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert L.la_feature_map(ok, ok, -5, 0, 0, null) == -1
     assert L.la_feature_map(ok, ok, 0, 0, 0, null) == 0
     assert L.la_feature_map(ok, ok, 4, 9, 0, null) == -1
+    # degree-2 polynomial map: D*D <= C <= 128, C a multiple of 8; nothing to do for zero rows
+    poly = lambda rows, D, C, dt=0, x=ok, y=ok: L.la_feature_map_poly2(x, y, rows, D, C, dt, null)
+    assert poly(0, 8, 64) == 0
+    assert poly(-1, 8, 64) == -1 and poly(4, 0, 8) == -1 and poly(4, 12, 144) == -1
+    assert poly(4, 8, 56) == -1 and poly(4, 3, 12) == -1 and poly(4, 3, 136) == -1 and poly(4, 8, 64, dt=7) == -1
+    assert poly(4, 8, 64, x=null) == -1 and poly(4, 8, 64, y=odd) == -1
+    assert L.la_feature_map_poly2_backward(ok, ok, ok, 4, 8, 64, 0, null) == -1          # dx aliases x
+    assert b"alias" in L.la_last_error()
+    assert L.la_feature_map_poly2_backward(ok, null, far, 4, 8, 64, 0, null) == -1
+    assert L.la_feature_map_poly2_backward(ok, ok, far, 0, 8, 64, 0, null) == 0
+    assert binding.poly2_columns(8) == 64 and binding.poly2_columns(5) == 32 and binding.poly2_columns(11) == 128
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
