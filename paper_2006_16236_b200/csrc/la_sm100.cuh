@@ -109,6 +109,12 @@ template <int N>
 __device__ __forceinline__ void tma_store_wait_all() {
     asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while
+// the kernel before it in the stream still runs; grid_dependency_wait() returns once that kernel has
+// completed and its writes are visible (nothing it wrote may be read, and nothing it reads overwritten,
+// before); allow_dependent_launch() lets the next such kernel be scheduled once every CTA has called it.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void allow_dependent_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }

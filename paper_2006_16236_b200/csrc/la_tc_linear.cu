@@ -33,6 +33,8 @@ namespace tc {
 
 using namespace sm100;
 
+LA_TRACE_DECL(g_trace_lin)
+
 namespace {
 
 // Record of one split: [A' (64x64) | a' (64) | ysum (64) | w0 (1) | pad]:
@@ -61,15 +63,35 @@ __device__ __forceinline__ void elu_row_inplace(uint8_t* row, uint32_t r7, float
     store_row(row, r7, v, nch);          // the zero padding of a 32-column row stays zero
 }
 
+// elu on logical chunks [4 hf, 4 hf + 4) of a row (those below nch).
+template <bool kElu>
+__device__ __forceinline__ void elu_half_row_inplace(uint8_t* row, uint32_t r7, float scale, int hf, int nch) {
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+        const int c = hf * 4 + cc;
+        if (c < nch) {
+            uint32_t v[4];
+            lds128(row + ((c ^ r7) << 4), v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float x0 = bf16_lo(v[j]), x1 = bf16_hi(v[j]);
+                v[j] = pack_bf16x2((kElu ? elu_fast(x0) : x0 - 1.f) * scale, (kElu ? elu_fast(x1) : x1 - 1.f) * scale);
+            }
+            sts128(row + ((c ^ r7) << 4), v[0], v[1], v[2], v[3]);
+        }
+    }
+}
+
 // ===========================================================================
-// Pre-pass: per-split sums.  Warps 0-3: elu on X (scaled by w_i), weight and aux tiles,
-// final read-out; warp 4: TMA; warp 5: MMA.
+// Pre-pass: per-split sums.  Warps 0-7: elu on X (scaled by w_i; two threads per row, half a row
+// each), aux tile, final read-out (warps 0-2); warp 8: TMA; warp 9: MMA.
 // ===========================================================================
-constexpr int kLsThreads = 192;
-constexpr int kLsStages = 3;
-constexpr uint32_t kLsStageBytes = 4 * kTileBytes;                  // X, Y, W (rows of w_i), aux (dl_i in 16 columns)
-constexpr uint32_t kLsOffOnes = kLsStages * kLsStageBytes;
-constexpr uint32_t kLsOffBar = kLsOffOnes + 1024;
+constexpr int kLsThreads = 320;
+// Four stages: a tile arrives about 2400 cycles after its load is issued, against about 1000 cycles of mapping
+// and 600 of MMA issue per chunk, so the ring has to hold the loads of three chunks ahead.
+constexpr int kLsStages = 4;
+constexpr uint32_t kLsStageBytes = 3 * kTileBytes;                  // X, Y, aux (columns 0..15: dl_i, 16..23: w_i)
+constexpr uint32_t kLsOffBar = kLsStages * kLsStageBytes;
 constexpr uint32_t kLsSmemBytes = kLsOffBar + 256 + 1024;
 
 struct LsBarriers {
@@ -106,6 +128,41 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const int L_all = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
     const bool reverse = prm.dn != nullptr;
+    LA_TRACE_CTA(g_trace_lin, 0);
+
+    if (tid == 0) {
+        for (int s = 0; s < kLsStages; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+            mbar_init(&bars->mapped[s], 256);
+        }
+        mbar_init(&bars->done, 1);
+        bars->abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 9) {
+        __syncwarp();
+        tmem_alloc(&bars->tmem_base, 256);
+        tmem_relinquish();
+    }
+    // The aux tile of a stage is the second 64-column block of both operands: of B = [Y | aux] (N = 80: its
+    // columns 0..15, dl_i, are read) and of A = [X | aux] (M = 128: accumulator row 64 + m is the sum weighted by
+    // column m; row 80, weighted by w_i in column 16, is the one read out; columns 24.. are never written and
+    // feed rows nobody reads).  Without per-position weights the tile is constant ones: written once here.
+    if (!reverse)
+        for (int s = 0; s < kLsStages; ++s)
+            for (int i = tid; i < kTileBytes / 4; i += kLsThreads)
+                reinterpret_cast<uint32_t*>(smem + s * kLsStageBytes + 2 * kTileBytes)[i] = 0x3F803F80u;
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = bars->tmem_base;
+    volatile int* abort_flag = &bars->abort_flag;
+    // everything above is private to the CTA; from here on memory of the kernel before this one is touched
+    allow_dependent_launch();
+    grid_dependency_wait();
+    LA_TRACE_CTA(g_trace_lin, 1);
     // Ragged batch: only `real` rows of this split exist; chunks behind them are skipped and the rows behind
     // them in the last chunk are zeroed after the load (at least one chunk runs, so that the record is written
     // from an accumulator that holds zeros and not from one that was never started).
@@ -116,37 +173,7 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     }
     const int L = max(1, (int)((real + kChunk - 1) / kChunk));
 
-    if (tid == 0) {
-        for (int s = 0; s < kLsStages; ++s) {
-            mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], 1);
-            mbar_init(&bars->mapped[s], 128);
-        }
-        mbar_init(&bars->done, 1);
-        bars->abort_flag = 0;
-        fence_mbar_init();
-    }
-    if (warp == 5) {
-        __syncwarp();
-        tmem_alloc(&bars->tmem_base, 256);
-        tmem_relinquish();
-    }
-    if (tid < 128)
-        for (int i = tid; i < 256; i += 128) reinterpret_cast<uint32_t*>(smem + kLsOffOnes)[i] = 0x3F803F80u;
-    // The aux tile of a stage is the second 64-column block of the B operand [Y | aux] (N = 80: its first 16
-    // columns are read).  Without per-position weights it is constant ones: written once here.
-    if (!reverse)
-        for (int s = 0; s < kLsStages; ++s)
-            for (int i = tid; i < kTileBytes / 4; i += kLsThreads)
-                reinterpret_cast<uint32_t*>(smem + s * kLsStageBytes + 3 * kTileBytes)[i] = 0x3F803F80u;
-    fence_proxy_async_smem();
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem = bars->tmem_base;
-    volatile int* abort_flag = &bars->abort_flag;
-
-    if (warp == 4) {
+    if (warp == 8) {
         if (lane == 0) {
             prefetch_tensormap(&mapX); prefetch_tensormap(&mapY);
             #pragma unroll 1
@@ -159,43 +186,43 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 if (*abort_flag) break;
                 uint8_t* st = smem + s * kLsStageBytes;
                 const int y = (int)(row0 + (int64_t)c * kChunk);
+                LA_TRACE(g_trace_lin, c, 2);
                 mbar_arrive_expect_tx(&bars->full[s], 2 * kTileBytes);
                 tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
                 tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         if (lane == 0) {
-            // one M = 64, N = 80 product per K group and accumulator: B = [Y | aux], the aux tile (two tiles
-            // further on in the stage) being the second 64-column block through the leading-offset field
-            const uint32_t idesc = umma_idesc_bf16(64, 80, 1, 1);
-            const uint32_t aOnes = sbase + kLsOffOnes;
+            // one M = 128, N = 80 product per K group: A = [X | aux], B = [Y | aux], the second 64-column block
+            // of either operand addressed through the leading-offset field.
+            // Accumulator rows 0..63: [A' | a'] = x'^T [Y | aux];  row 80: [ysum | w0] = w^T [Y | aux].
+            const uint32_t idesc = umma_idesc_bf16(128, 80, 1, 1);
             bool ok = true;
             #pragma unroll 1
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kLsStages;
-                const uint32_t aX = sbase + s * kLsStageBytes, aY = aX + kTileBytes, aW = aY + kTileBytes, aA = aW + kTileBytes;
+                const uint32_t aX = sbase + s * kLsStageBytes, aY = aX + kTileBytes, aA = aY + kTileBytes;
                 ok = mbar_wait(&bars->mapped[s], (c / kLsStages) & 1, prm.status, kStatusPipeTimeout);
                 if (!ok || *abort_flag) { ok = false; break; }
                 tc_fence_after_sync();
+                LA_TRACE(g_trace_lin, c, 0);
                 const uint32_t acc = (c != 0);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    const uint32_t a = acc | (k != 0);
-                    const uint64_t dX = desc_mn(aX + k * 2048), dYA = desc_mn(aY + k * 2048, aA - aY);
-                    const uint64_t dW = reverse ? desc_mn(aW + k * 2048) : desc_ones(aOnes);
-                    umma_bf16(tmem, dX, dYA, idesc, a);                  // [A' | a'] += x'^T [Y | aux]
-                    umma_bf16(tmem + 128, dW, dYA, idesc, a);            // [ysum | w0] += w^T [Y | aux] (all 64 rows alike)
+                    umma_bf16(tmem, desc_mn(aX + k * 2048, aA - aX), desc_mn(aY + k * 2048, aA - aY), idesc, acc | (k != 0));
                 }
                 umma_commit(&bars->empty[s]);
+                LA_TRACE(g_trace_lin, c, 1);
             }
             if (!ok) *abort_flag = 1;
             umma_commit(&bars->done);
         }
     } else {
-        const int t = tid;
+        const int t = tid & 127, hf = tid >> 7;
         const uint32_t r7 = t & 7;
         const bool elu = prm.phi == LA_PHI_ELU1;
+        const int nch = prm.dim >> 3;
         #pragma unroll 1
         for (int c = 0; c < L; ++c) {
             const int s = c % kLsStages;
@@ -212,64 +239,60 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             }
             if (!mbar_wait(&bars->full[s], (c / kLsStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
+            if (tid == 0) LA_TRACE(g_trace_lin, c, 5);
             uint8_t* rowX = smem + s * kLsStageBytes + t * 128;
             if (padded) {
 #pragma unroll
-                for (int cc = 0; cc < 8; ++cc) {
-                    sts128(rowX + (cc << 4), 0u, 0u, 0u, 0u);
-                    sts128(rowX + kTileBytes + (cc << 4), 0u, 0u, 0u, 0u);
+                for (int cc = 0; cc < 4; ++cc) {
+                    sts128(rowX + ((hf * 4 + cc) << 4), 0u, 0u, 0u, 0u);
+                    sts128(rowX + kTileBytes + ((hf * 4 + cc) << 4), 0u, 0u, 0u, 0u);
                 }
             } else if (elu) {
-                elu_row_inplace<true>(rowX, r7, w, prm.dim >> 3);
+                elu_half_row_inplace<true>(rowX, r7, w, hf, nch);
             } else {
-                elu_row_inplace<false>(rowX, r7, w, prm.dim >> 3);
+                elu_half_row_inplace<false>(rowX, r7, w, hf, nch);
             }
-            if (reverse) {
-                uint8_t* rowW = rowX + 2 * kTileBytes;
-                uint8_t* rowA = rowX + 3 * kTileBytes;
+            if (reverse && hf == 0) {
+                uint8_t* rowA = rowX + 2 * kTileBytes;
                 const uint32_t ww = pack_bf16x2(w, w), dd = pack_bf16x2(delta, delta);
-#pragma unroll
-                for (int cc = 0; cc < 8; ++cc) sts128(rowW + (cc << 4), ww, ww, ww, ww);
                 sts128(rowA + ((0 ^ r7) << 4), dd, dd, dd, dd);
                 sts128(rowA + ((1 ^ r7) << 4), dd, dd, dd, dd);
+                sts128(rowA + ((2 ^ r7) << 4), ww, ww, ww, ww);
             }
             fence_proxy_async_smem();
             mbar_arrive(&bars->mapped[s]);
+            if (tid == 0) LA_TRACE(g_trace_lin, c, 6);
         }
         // read-out of this split's record
         const bool ok = mbar_wait(&bars->done, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
+        LA_TRACE_CTA(g_trace_lin, 2);
         tc_fence_after_sync();
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         float* rec = prm.records + (bh * prm.nseg + seg) * (int64_t)kRecFloats;
-        const int d_row = warp * 16 + lane;
-        for (int h = 0; h < 2; ++h) {
-            uint32_t v[32];
-            tmem_ld32(tmem + lane_base + h * 32, v);
-            tmem_ld_wait();
-            if (ok && lane < 16)
-#pragma unroll
-                for (int j = 0; j < 32; ++j) rec[d_row * kDim + h * 32 + j] = __uint_as_float(v[j]);
-        }
-        const float z = __uint_as_float(tmem_ld1(tmem + lane_base + 64));
-        tmem_ld_wait();
-        if (ok && lane < 16) rec[kDim * kDim + d_row] = z;
-        if (warp == 0) {            // row 0 of the w-weighted sums
+        if (warp < 3) {             // warps 0, 1: accumulator rows 0..63; warp 2, lane 16: row 80, the w-weighted sums
+            const int d_row = warp * 32 + lane;
+            const bool mine = ok && (warp < 2 || lane == 16);
+            float* dst = warp < 2 ? rec + d_row * kDim : rec + kDim * kDim + kDim;
             for (int h = 0; h < 2; ++h) {
                 uint32_t v[32];
-                tmem_ld32(tmem + 128 + h * 32, v);
+                tmem_ld32(tmem + lane_base + h * 32, v);
                 tmem_ld_wait();
-                if (ok && lane == 0)
+                if (mine)
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) rec[kDim * kDim + kDim + h * 32 + j] = __uint_as_float(v[j]);
+                    for (int j = 0; j < 32; ++j) dst[h * 32 + j] = __uint_as_float(v[j]);
             }
-            const float w0 = __uint_as_float(tmem_ld1(tmem + 192));
+            const float z = __uint_as_float(tmem_ld1(tmem + lane_base + 64));
             tmem_ld_wait();
-            if (ok && lane == 0) rec[kDim * kDim + 2 * kDim] = reverse ? w0 : 0.f;
+            if (mine) {
+                if (warp < 2) rec[kDim * kDim + d_row] = z;
+                else rec[kDim * kDim + 2 * kDim] = reverse ? z : 0.f;
+            }
         }
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    LA_TRACE_CTA(g_trace_lin, 3);
+    if (warp == 9) {
         __syncwarp();
         tmem_dealloc(tmem, 256);
     }
@@ -336,14 +359,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     const int c_begin = seg * prm.chunks_per_seg;
     const int L_all = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
-    // Ragged batch: `len` positions of this sequence exist, `real` of them in this split.  Only the chunks that
-    // hold real rows go through the pipeline; the padding behind them is filled with zeros at the end.
-    int64_t len = prm.N, real = (int64_t)L_all * kChunk;
-    if (prm.lengths) {
-        len = min((int64_t)max(prm.lengths[bh / prm.heads], 0), prm.N);
-        real = min(max(len - (int64_t)c_begin * kChunk, (int64_t)0), real);
-    }
-    const int L = (int)((real + kChunk - 1) / kChunk);
+    LA_TRACE_CTA(g_trace_lin, 4);
 
     if (tid == 0) {
         for (int s = 0; s < kApStages; ++s) {
@@ -363,18 +379,59 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         tmem_alloc(&bars->tmem_base, 256);
         tmem_relinquish();
     }
+    __syncthreads();            // the barriers are initialised for the loads issued before the prologue below
+    // (set-up above is private to the CTA; the records below come from the kernel before this one)
+    allow_dependent_launch();
+    grid_dependency_wait();
+    // Ragged batch: `len` positions of this sequence exist, `real` of them in this split.  Only the chunks that
+    // hold real rows go through the pipeline; the padding behind them is filled with zeros at the end.
+    int64_t len = prm.N, real = (int64_t)L_all * kChunk;
+    if (prm.lengths) {
+        len = min((int64_t)max(prm.lengths[bh / prm.heads], 0), prm.N);
+        real = min(max(len - (int64_t)c_begin * kChunk, (int64_t)0), real);
+    }
+    const int L = (int)((real + kChunk - 1) / kChunk);
+    // the loads of the first chunks travel while the state is put together below
+    auto issue_load = [&](int c) {
+        const int s = c % kApStages;
+        uint8_t* st = smem + kApOffStage + s * 2 * kTileBytes;
+        const int y = (int)(row0 + (int64_t)c * kChunk);
+        mbar_arrive_expect_tx(&bars->full[s], kTiles * kTileBytes);
+        tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
+        if (kHasY) tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
+    };
+    if (warp == 8 && lane == 0) {
+        prefetch_tensormap(&mapX);
+        if (kHasY) prefetch_tensormap(&mapY);
+        for (int c = 0; c < min(L, kApStages); ++c) issue_load(c);
+    }
     // state of this head: add the split records (fp32), remove the column means, round the
-    // centred remainder to a bf16 operand tile.  The stage area is free until the pipeline starts.
+    // centred remainder to a bf16 operand tile.  Scratch: the output staging tiles, free until the first epilogue.
     {
         const float* rec = prm.records + bh * prm.nseg * (int64_t)kRecFloats;
-        float* sF = reinterpret_cast<float*>(smem + kApOffStage);                 // fp32 [64][64] scratch
-        for (int idx = tid; idx < kDim * kDim / 4; idx += kApThreads) {
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float* sF = reinterpret_cast<float*>(smem + kApOffOut);                   // fp32 [64][64] scratch (+ 64 means)
+        {
+            constexpr int kPer = (kDim * kDim / 4 + kApThreads - 1) / kApThreads;     // float4 slots per thread
+            float4 acc[kPer];
+#pragma unroll
+            for (int u = 0; u < kPer; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
             for (int n = 0; n < prm.nseg; ++n) {
-                const float4 a = __ldg(reinterpret_cast<const float4*>(rec + (int64_t)n * kRecFloats) + idx);
-                acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
+                const float4* src = reinterpret_cast<const float4*>(rec + (int64_t)n * kRecFloats);
+#pragma unroll
+                for (int u = 0; u < kPer; ++u) {        // independent loads: all in flight together
+                    const int idx = tid + u * kApThreads;
+                    if (idx < kDim * kDim / 4) {
+                        const float4 a = __ldg(src + idx);
+                        acc[u].x += a.x; acc[u].y += a.y; acc[u].z += a.z; acc[u].w += a.w;
+                    }
+                }
             }
-            reinterpret_cast<float4*>(sF)[idx] = acc;
+#pragma unroll
+            for (int u = 0; u < kPer; ++u) {
+                const int idx = tid + u * kApThreads;
+                if (idx < kDim * kDim / 4) reinterpret_cast<float4*>(sF)[idx] = acc[u];
+            }
         }
         if (tid < 2 * kDim + 1) {       // a' (64), ysum (64), w0 (1)
             float z = 0.f;
@@ -421,24 +478,18 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     tc_fence_after_sync();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
+    LA_TRACE_CTA(g_trace_lin, 5);
 
     if (warp == 8) {
         if (lane == 0) {
-            prefetch_tensormap(&mapX);
-            if (kHasY) prefetch_tensormap(&mapY);
             #pragma unroll 1
-            for (int c = 0; c < L; ++c) {
-                const int s = c % kApStages;
-                if (c >= kApStages && !mbar_wait(&bars->empty[s], ((c / kApStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
+            for (int c = kApStages; c < L; ++c) {
+                if (!mbar_wait(&bars->empty[c % kApStages], ((c / kApStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
                     *abort_flag = 1;
                     break;
                 }
                 if (*abort_flag) break;
-                uint8_t* st = smem + kApOffStage + s * 2 * kTileBytes;
-                const int y = (int)(row0 + (int64_t)c * kChunk);
-                mbar_arrive_expect_tx(&bars->full[s], kTiles * kTileBytes);
-                tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
-                if (kHasY) tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
+                issue_load(c);
             }
         }
     } else if (warp == 9) {
@@ -657,6 +708,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             }
         }
         if (hf == 0 && lane == 0) tma_store_wait_all<0>();
+        LA_TRACE_CTA(g_trace_lin, 6);
         if (L < L_all) {            // whole chunks of padding: zeros, written directly
             const int e = hf * 128 + t;
             const int64_t r_lo = row0 + (int64_t)L * kChunk, nrows = (int64_t)(L_all - L) * kChunk;
@@ -674,6 +726,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
 
     tc_fence_before_sync();
     __syncthreads();
+    LA_TRACE_CTA(g_trace_lin, 7);
     if (warp == 9) {
         __syncwarp();
         tmem_dealloc(tmem, 256);
@@ -693,6 +746,21 @@ Segmentation choose_splits(const la_problem& p) {
     const int cps = (chunks + nseg - 1) / nseg;
     nseg = (chunks + cps - 1) / cps;
     return Segmentation{nseg, cps};
+}
+
+// Launch configuration of a kernel that may start while the kernel before it in the stream drains (its set-up
+// overlaps that kernel's tail; it waits on the grid dependency before touching global memory).
+cudaLaunchConfig_t chained_launch(unsigned grid, unsigned block, size_t smem, cudaStream_t st, cudaLaunchAttribute* attr) {
+    attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr->val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cfg;
 }
 
 int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
@@ -717,8 +785,10 @@ int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& 
     prm.phi = p.phi;
     prm.dim = (int)p.D;
     prof_begin(kProfLinearSum, st);
-    linear_sum_kernel<<<(unsigned)(sg.nseg * p.B * p.H), kLsThreads, kLsSmemBytes, st>>>(mX, mY, prm);
-    LA_LAUNCHED();
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg = chained_launch((unsigned)(sg.nseg * p.B * p.H), kLsThreads, kLsSmemBytes, st, &attr);
+    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_sum_kernel, mX, mY, prm));
+    note_launch();
     prof_end(kProfLinearSum, st);
     return LA_OK;
 }
@@ -746,8 +816,10 @@ int launch_apply(const la_problem& p, const Segmentation& sg, const CUtensorMap&
     if (int rc = encode_tile_map(&mO0, prm.out0, rows, 32, (int)p.D)) return rc;
     if (int rc = encode_tile_map(&mO1, prm.out1 ? prm.out1 : prm.out0, rows, 32, (int)p.D)) return rc;
     prof_begin(kProfLinearApply, st);
-    linear_apply_kernel<kMode><<<(unsigned)(sg.nseg * p.B * p.H), kApThreads, kApSmemBytes, st>>>(mX, mY, mO0, mO1, prm);
-    LA_LAUNCHED();
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg = chained_launch((unsigned)(sg.nseg * p.B * p.H), kApThreads, kApSmemBytes, st, &attr);
+    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_apply_kernel<kMode>, mX, mY, mO0, mO1, prm));
+    note_launch();
     prof_end(kProfLinearApply, st);
     return LA_OK;
 }
@@ -817,3 +889,9 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
 
 }  // namespace tc
 }  // namespace la
+
+#ifdef LA_TC_TRACE
+extern "C" int la_debug_read_trace_lin(long long* out, int n) {
+    return (int)cudaMemcpyFromSymbol(out, la::tc::g_trace_lin, n * sizeof(long long));
+}
+#endif
