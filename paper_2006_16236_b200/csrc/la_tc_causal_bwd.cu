@@ -161,6 +161,9 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // everything above is private to the CTA; from here on memory of the kernel before this one is touched
+    allow_dependent_launch();
+    grid_dependency_wait();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
@@ -589,6 +592,9 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // everything above is private to the CTA; from here on memory of the kernel before this one is touched
+    allow_dependent_launch();
+    grid_dependency_wait();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
@@ -961,8 +967,10 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     prof_begin(kProfCausalBwdDq, st);
     CUtensorMap mDQ;
     if (int rc = encode_tile_map(&mDQ, dQ, rows, 32, (int)p.D)) return rc;      // one quadrant's rows per store
-    causal_bwd_dq_kernel<<<grid, kDqThreads, kDqSmemBytes, st>>>(mK, mV, mG, mQ, mDQ, a);
-    LA_LAUNCHED();
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg_q = chained_launch(grid, kDqThreads, kDqSmemBytes, st, &attr);
+    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_q, causal_bwd_dq_kernel, mK, mV, mG, mQ, mDQ, a));
+    note_launch();
     prof_end(kProfCausalBwdDq, st);
 
     // reverse sweep: dK, dV
@@ -986,8 +994,9 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     CUtensorMap mDK, mDV;
     if (int rc = encode_tile_map(&mDK, dK, rows, kChunk, (int)p.D)) return rc;
     if (int rc = encode_tile_map(&mDV, dV, rows, kChunk, (int)p.D)) return rc;
-    causal_bwd_dkv_kernel<<<grid, kKvThreads, kKvSmemBytes, st>>>(mQ, mK, mV, mG, mDK, mDV, b);
-    LA_LAUNCHED();
+    const cudaLaunchConfig_t cfg_kv = chained_launch(grid, kKvThreads, kKvSmemBytes, st, &attr);
+    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_kv, causal_bwd_dkv_kernel, mQ, mK, mV, mG, mDK, mDV, b));
+    note_launch();
     prof_end(kProfCausalBwdDkv, st);
     return LA_OK;
 }

@@ -136,6 +136,9 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // everything above is private to the CTA; from here on memory of the kernel before this one is touched
+    allow_dependent_launch();
+    grid_dependency_wait();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
@@ -541,8 +544,10 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     prm.dim = (int)p.D;
     prm.save = save ? 1 : 0;
     prof_begin(kProfCausalFwd, st);
-    causal_fwd_kernel<<<(unsigned)(pl.npieces() * pl.bh), kThreads, kSmemBytes, st>>>(mQ, mK, mV, mPQ, mPK, prm);
-    LA_LAUNCHED();
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg = chained_launch((unsigned)(pl.npieces() * pl.bh), kThreads, kSmemBytes, st, &attr);
+    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, causal_fwd_kernel, mQ, mK, mV, mPQ, mPK, prm));
+    note_launch();
     prof_end(kProfCausalFwd, st);
     return LA_OK;
 }

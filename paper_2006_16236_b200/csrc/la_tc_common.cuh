@@ -23,6 +23,22 @@ namespace tc {
 #define LA_TRACE_CTA(buf, slot) do { } while (0)
 #endif
 
+// Launch configuration of a kernel that may start while the kernel before it in the stream drains (its set-up
+// overlaps that kernel's tail; it waits on the grid dependency before touching global memory).
+inline cudaLaunchConfig_t chained_launch(unsigned grid, unsigned block, size_t smem, cudaStream_t st,
+                                         cudaLaunchAttribute* attr) {
+    attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr->val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cfg;
+}
+
 constexpr int kChunk = 128;                  // positions per chunk = MMA M
 constexpr int kDim = 64;                     // D = M = 64: one 128-byte swizzle row
 constexpr int kTileBytes = kChunk * kDim * 2;  // one [128][64] bf16 tile

@@ -748,21 +748,6 @@ Segmentation choose_splits(const la_problem& p) {
     return Segmentation{nseg, cps};
 }
 
-// Launch configuration of a kernel that may start while the kernel before it in the stream drains (its set-up
-// overlaps that kernel's tail; it waits on the grid dependency before touching global memory).
-cudaLaunchConfig_t chained_launch(unsigned grid, unsigned block, size_t smem, cudaStream_t st, cudaLaunchAttribute* attr) {
-    attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr->val.programmaticStreamSerializationAllowed = 1;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cfg;
-}
-
 int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
                 const float* dn, const float* dl, const int* lengths, float* records, cudaStream_t st) {
     static bool attr_done = false;

@@ -91,6 +91,9 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // everything above is private to the CTA; from here on memory of the kernel before this one is touched
+    allow_dependent_launch();
+    grid_dependency_wait();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
@@ -224,8 +227,10 @@ int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap&
     prm.map = map ? 1 : 0;
     prm.dim = (int)p.D;
     prof_begin(kProfSegmentSum, st);
-    segment_sum_kernel<<<(unsigned)(prm.parts_per_seq * p.B * p.H), kSumThreads, kSumSmemBytes, st>>>(mapX, mapY, prm);
-    LA_LAUNCHED();
+    cudaLaunchAttribute attr;
+    const cudaLaunchConfig_t cfg = chained_launch((unsigned)(prm.parts_per_seq * p.B * p.H), kSumThreads, kSumSmemBytes, st, &attr);
+    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, segment_sum_kernel, mapX, mapY, prm));
+    note_launch();
     prof_end(kProfSegmentSum, st);
     return LA_OK;
 }
