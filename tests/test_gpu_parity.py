@@ -575,6 +575,33 @@ def test_noncausal_workload_full_size():
             assert_close(got[sl], ref, dtype, f"d{nm}[{b},{h}]", grad=True)
 
 
+def test_noncausal_ragged_workload_full_size():
+    """The speech-shaped workload as a ragged batch (the paper's speech batches are: mean 800, max 2400
+    frames): lengths between a third of N and N, one full and one of a single chunk plus one position."""
+    w = WORKLOADS["noncausal_bf16_speech"]
+    dtype = w.torch_dtype
+    Q, K, V, G = draw_workload(w)
+    g = torch.Generator().manual_seed(w.seed + 5)
+    lengths = torch.randint(w.N // 3, w.N + 1, (w.B,), generator=g, dtype=torch.int32)
+    lengths[0], lengths[w.B - 1] = w.N, 129
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    ld = lengths.to(DEV)
+    O = la.la_linear_attention_varlen(Qd, Kd, Vd, ld)
+    dQ, dK, dV = la.la_linear_attention_varlen_backward(Qd, Kd, Vd, Gd, ld)
+    la.la_last_device_status()
+    for b, h in _sample_heads(w.B, w.H):
+        n = int(lengths[b])
+        sl = (slice(b, b + 1), slice(h, h + 1), slice(0, n))
+        q, k, v, gg = Q[sl], K[sl], V[sl], G[sl]
+        assert_close(O[sl], oracle.linear_attention(q, k, v, False)[0], dtype, f"O[{b},{h}], length {n}")
+        for got, ref, nm in zip((dQ, dK, dV), oracle.linear_attention_backward(q, k, v, gg, False), "QKV"):
+            assert_close(got[sl], ref, dtype, f"d{nm}[{b},{h}], length {n}", grad=True)
+    for b in range(w.B):
+        n = int(lengths[b])
+        for t in (O, dQ, dK, dV):
+            assert n == w.N or float(t[b, :, n:].float().abs().max()) == 0.0
+
+
 def test_decode_workload_full_size():
     w = WORKLOADS["decode_bf16_streams"]
     T = 3072
