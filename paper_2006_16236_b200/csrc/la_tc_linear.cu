@@ -533,10 +533,12 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             const int s = c % kApStages;
             if (!mbar_wait(&bars->full[s], (c / kApStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
+            if (t == 0) LA_TRACE(g_trace_lin, c, 14);
             uint8_t* rowX = smem + kApOffStage + s * 2 * kTileBytes + t * 128;
             if (elu) elu_row_inplace<true>(rowX, r7, 1.f, prm.dim >> 3); else elu_row_inplace<false>(rowX, r7, 1.f, prm.dim >> 3);
             fence_proxy_async_smem();
             mbar_arrive(&bars->mapped[s]);
+            if (t == 0) LA_TRACE(g_trace_lin, c, 15);
         }
     } else {
         // Epilogue: two warps per TMEM quadrant (warps 0-3: columns 0..31 of a row, warps 10-13: columns 32..63;
@@ -562,6 +564,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             const bool padded = (int64_t)c * kChunk + t >= real;      // a row behind the sequence's end: zeros go out
             if (!mbar_wait(&bars->mapped[s], (c / kApStages) & 1, prm.status, kStatusPipeTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
+            if (tid == 0) LA_TRACE(g_trace_lin, c, 8);
             uint32_t xv[4][4];                       // this half of the x' = elu(X) row
             const uint8_t* rowX = smem + kApOffStage + s * 2 * kTileBytes + t * 128;
 #pragma unroll
@@ -591,6 +594,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 }
             if (!mbar_wait(&bars->acc_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
+            if (tid == 0) LA_TRACE(g_trace_lin, c, 9);
             uint32_t acc[32];
             tmem_ld32(tmem + lane_base + b * 128 + hf * 32, acc);
             tmem_ld_wait();
@@ -610,6 +614,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             }
             // the pair's previous slab must have left the staging tile before either warp rewrites it below
             if (hf == 0 && lane == 0) tma_store_wait_read<0>();
+            if (tid == 0) LA_TRACE(g_trace_lin, c, 10);
             mine[0] = (sx4[0] + sx4[1]) + (sx4[2] + sx4[3]);
             mine[1] = (xa4[0] + xa4[1]) + (xa4[2] + xa4[3]);
             mine[2] = ynu_h;
@@ -621,6 +626,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             const float* hi = hf ? mine : other;
             const float sx = lo[0] + hi[0], xa = lo[1] + hi[1], ynu = lo[2] + hi[2], sh = lo[3] + hi[3], qh = lo[4] + hi[4];
             named_barrier(2 + quad, 64);            // the exchange slots may be rewritten after this
+            if (tid == 0) LA_TRACE(g_trace_lin, c, 11);
             const float x1sum = fD + sx;             // (1 + x') . 1
             uint8_t* out_row = smem + kApOffOut + t * 128;
             if (kMode == kApplyForward) {
@@ -696,6 +702,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     if (kMode == kApplyBackwardKV) sts128(out_row + kTileBytes + (((hf * 4 + cc) ^ r7) << 4), 0u, 0u, 0u, 0u);
                 }
             }
+            if (tid == 0) LA_TRACE(g_trace_lin, c, 12);
             tc_fence_before_sync();
             mbar_arrive(&bars->acc_free[b]);
             fence_proxy_async_smem();
@@ -706,6 +713,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 if (kMode == kApplyBackwardKV) tma_store_2d(&mapOut1, smem + kApOffOut + kTileBytes + quad * 32 * 128, 0, y);
                 tma_store_commit();
             }
+            if (tid == 0) LA_TRACE(g_trace_lin, c, 13);
         }
         if (hf == 0 && lane == 0) tma_store_wait_all<0>();
         LA_TRACE_CTA(g_trace_lin, 6);
