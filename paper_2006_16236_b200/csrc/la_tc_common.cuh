@@ -445,7 +445,14 @@ __device__ __noinline__ void state_add_given(uint32_t tmem_state, int quad, int 
     const bool owner = lane < 16;
     const bool in_row = owner && d_row < dim;
     sm100::tc_fence_after_sync();
-#pragma unroll 1
+    // the whole row of the given state is requested at once: one round trip to memory, not one per column group
+    float4 given[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+        given[j] = (in_row && s_in && j * 4 < dim) ? __ldg(reinterpret_cast<const float4*>(s_in + d_row * dim) + j)
+                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    const float z_given = (in_row && z_in) ? __ldg(z_in + d_row) : 0.f;
+#pragma unroll
     for (int g = 0; g < 4; ++g) {
         uint32_t v[16];
         sm100::tmem_ld16(tmem_state + lane_base + g * 16, v);
@@ -453,12 +460,10 @@ __device__ __noinline__ void state_add_given(uint32_t tmem_state, int quad, int 
         float acc[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) acc[j] = __uint_as_float(v[j]);
-        if (in_row && s_in && g * 16 < dim) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float4 b = __ldg(reinterpret_cast<const float4*>(s_in + d_row * dim + g * 16) + j);
-                acc[4 * j] += b.x; acc[4 * j + 1] += b.y; acc[4 * j + 2] += b.z; acc[4 * j + 3] += b.w;
-            }
+        for (int j = 0; j < 4; ++j) {
+            const float4 b = given[4 * g + j];
+            acc[4 * j] += b.x; acc[4 * j + 1] += b.y; acc[4 * j + 2] += b.z; acc[4 * j + 3] += b.w;
         }
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(acc[j]);
@@ -473,7 +478,7 @@ __device__ __noinline__ void state_add_given(uint32_t tmem_state, int quad, int 
     }
     float z = __uint_as_float(sm100::tmem_ld1(tmem_state + lane_base + 64));
     sm100::tmem_ld_wait();
-    if (in_row && z_in) z += __ldg(z_in + d_row);
+    z += z_given;
     uint32_t zz[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) zz[j] = (kForward || j == 0) ? __float_as_uint(z) : 0u;
