@@ -92,10 +92,10 @@ int la_feature_map(const void* x, void* y, int64_t n, int32_t dtype, int32_t der
  * phi = LA_PHI_IDENTITY and D = C (the cost O(N D^2 M) the paper quotes); the zero padding lets C
  * be the multiple of 8 they ask for.  The paper names the kernel without fixing its form: the
  * homogeneous one is taken, the one whose feature map has exactly D^2 components.
- * x: [rows, D], y: [rows, C] of `dtype` (device; y 16-byte aligned; x and y must not overlap).
+ * x: [rows, D], y: [rows, C] of `dtype` (device, 16-byte aligned; x and y must not overlap).
  * 1 <= D <= 11, D*D <= C <= 128, C a multiple of 8.  Products are formed in fp32 and rounded once.
  * The backward call turns dy = dL/dy [rows, C] into dx[r][i] = sum_j (dy[r][i*D+j] + dy[r][j*D+i]) x[r][j]
- * (fp32 sums; dx: [rows, D], must not alias x).
+ * (fp32 sums; dx: [rows, D], must not alias x; x, dy, dx 16-byte aligned).
  */
 int la_feature_map_poly2(const void* x, void* y, int64_t rows, int64_t D, int64_t C, int32_t dtype, void* stream);
 int la_feature_map_poly2_backward(const void* x, const void* dy, void* dx, int64_t rows, int64_t D, int64_t C,

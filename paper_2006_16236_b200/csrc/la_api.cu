@@ -213,7 +213,7 @@ static int check_poly2(int64_t rows, int64_t D, int64_t C, int32_t dtype) {
 int la_feature_map_poly2(const void* x, void* y, int64_t rows, int64_t D, int64_t C, int32_t dtype, void* stream) {
     if (int rc = check_poly2(rows, D, C, dtype)) return rc;
     if (rows == 0) return LA_OK;
-    if (!x) return fail(LA_ERR_INVALID_ARG, "x is NULL");
+    LA_REQUIRE_PTR(x);          // rows of eight bf16 are read with 16-byte loads
     LA_REQUIRE_PTR(y);
     if (int rc = check_arch()) return rc;
     return launch_poly2_map(x, y, rows, (int)D, (int)C, dtype, (cudaStream_t)stream);
@@ -223,9 +223,9 @@ int la_feature_map_poly2_backward(const void* x, const void* dy, void* dx, int64
                                   int32_t dtype, void* stream) {
     if (int rc = check_poly2(rows, D, C, dtype)) return rc;
     if (rows == 0) return LA_OK;
-    if (!x) return fail(LA_ERR_INVALID_ARG, "x is NULL");
-    if (!dy) return fail(LA_ERR_INVALID_ARG, "dy is NULL");
-    if (!dx) return fail(LA_ERR_INVALID_ARG, "dx is NULL");
+    LA_REQUIRE_PTR(x);
+    LA_REQUIRE_PTR(dy);
+    LA_REQUIRE_PTR(dx);
     if (dx == x) return fail(LA_ERR_INVALID_ARG, "dx must not alias x");
     if (int rc = check_arch()) return rc;
     return launch_poly2_map_backward(x, dy, dx, rows, (int)D, (int)C, dtype, (cudaStream_t)stream);

@@ -174,7 +174,7 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert poly(0, 8, 64) == 0
     assert poly(-1, 8, 64) == -1 and poly(4, 0, 8) == -1 and poly(4, 12, 144) == -1
     assert poly(4, 8, 56) == -1 and poly(4, 3, 12) == -1 and poly(4, 3, 136) == -1 and poly(4, 8, 64, dt=7) == -1
-    assert poly(4, 8, 64, x=null) == -1 and poly(4, 8, 64, y=odd) == -1
+    assert poly(4, 8, 64, x=null) == -1 and poly(4, 8, 64, y=odd) == -1 and poly(4, 8, 64, x=odd) == -1
     assert L.la_feature_map_poly2_backward(ok, ok, ok, 4, 8, 64, 0, null) == -1          # dx aliases x
     assert b"alias" in L.la_last_error()
     assert L.la_feature_map_poly2_backward(ok, null, far, 4, 8, 64, 0, null) == -1
