@@ -24,58 +24,139 @@ struct Dims {
 
 __device__ __forceinline__ Dims make_dims(int D, int M) { return Dims{D, M, D + 1, M + 1}; }
 
-// dst[i][d] = phi(src[i][d]) for i < cn, 0 for the padded rows (zero in feature
-// space: a padded key contributes nothing to any sum).
-template <typename IO>
-__device__ void load_mapped(float* dst, const IO* src, int cn, int D, int DS, int phi) {
-    for (int idx = threadIdx.x; idx < T * D; idx += THREADS) {
-        const int i = idx / D, d = idx - i * D;
-        dst[i * DS + d] = i < cn ? phi_apply(to_f32<IO>(src[(int64_t)i * D + d]), phi) : 0.f;
+// Register-blocked product of small shared-memory matrices:
+//   out(i, j) = sum_{k < K1} A1(i, k) B1(k, j) + sum_{k < K2} A2(i, k) B2(k, j),   i < I, j < J,
+// with X(i, k) = x[i * xi + k * xk] (any strides; I a multiple of RI, J of RJ; K2 = 0: one product).  A thread
+// owns RI x RJ outputs spread over the matrix (i = il + r I/RI, j = jl + s J/RJ), so that the lanes of a
+// warp read consecutive j of B (consecutive or padded-stride addresses) and broadcast A: RI + RJ loads feed
+// RI * RJ multiply-adds.  `store(i, j, value)` consumes the results.
+struct Mat { const float* p; int s0, s1; };      // element (a, b) at p[a * s0 + b * s1]
+
+template <int RI, int RJ, typename Store>
+__device__ __forceinline__ void block_product(int I, int J, Mat A1, Mat B1, int K1, Mat A2, Mat B2, int K2, Store store) {
+    const int ni = I / RI, nj = J / RJ;
+    for (int tile = threadIdx.x; tile < ni * nj; tile += THREADS) {
+        const int il = tile / nj, jl = tile - il * nj;
+        float acc[RI][RJ];
+#pragma unroll
+        for (int r = 0; r < RI; ++r)
+#pragma unroll
+            for (int c = 0; c < RJ; ++c) acc[r][c] = 0.f;
+        for (int pass = 0; pass < 2; ++pass) {
+            const Mat A = pass ? A2 : A1, B = pass ? B2 : B1;
+            const int K = pass ? K2 : K1;
+            const float* a0 = A.p + il * A.s0;
+            const float* b0 = B.p + jl * B.s1;
+#pragma unroll 4
+            for (int k = 0; k < K; ++k) {
+                float a[RI], b[RJ];
+#pragma unroll
+                for (int r = 0; r < RI; ++r) a[r] = a0[r * ni * A.s0 + k * A.s1];
+#pragma unroll
+                for (int c = 0; c < RJ; ++c) b[c] = b0[k * B.s0 + c * nj * B.s1];
+#pragma unroll
+                for (int r = 0; r < RI; ++r)
+#pragma unroll
+                    for (int c = 0; c < RJ; ++c) acc[r][c] = fmaf(a[r], b[c], acc[r][c]);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < RI; ++r)
+#pragma unroll
+            for (int c = 0; c < RJ; ++c) store(il + r * ni, jl + c * nj, acc[r][c]);
     }
 }
 
-// dst[i][0..M) = src[i][:], dst[i][M] = 1 (the ones column); padded rows are 0.
+// A chunk of rows ([cn][cols] of IO, contiguous in global memory, 16-byte aligned: chunks start at multiples
+// of T rows and cols is a multiple of 8) travels as up to FETCH 16-byte groups per thread, all requested
+// before any is used; rows cn..T-1 (beyond the sequence) read as zero bits.
+constexpr int FETCH = 4;       // T * 128 columns * 4 bytes / 16 bytes / THREADS
+
+template <typename IO>
+__device__ __forceinline__ void fetch_rows(uint4 (&r)[FETCH], const IO* src, int cn, int cols) {
+    constexpr int VEC = 16 / (int)sizeof(IO);
+    const int total = cn * (cols / VEC);
+#pragma unroll
+    for (int u = 0; u < FETCH; ++u) {
+        const int g = threadIdx.x + u * THREADS;
+        r[u] = g < total ? __ldg(reinterpret_cast<const uint4*>(src) + g) : make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
+// dst[i][c] = f(i, value) for the fetched rows (i < cn), 0 for the padded rows (zero in feature space: a
+// padded key contributes nothing to any sum).
+template <typename IO, typename F>
+__device__ __forceinline__ void store_rows(float* dst, const uint4 (&r)[FETCH], int cn, int cols, int stride, F f) {
+    constexpr int VEC = 16 / (int)sizeof(IO);
+    const int gpr = cols / VEC, all = T * gpr;
+#pragma unroll
+    for (int u = 0; u < FETCH; ++u) {
+        const int g = threadIdx.x + u * THREADS;
+        if (g < all) {
+            const int i = g / gpr, c0 = (g - i * gpr) * VEC;
+            const IO* e = reinterpret_cast<const IO*>(&r[u]);
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) dst[i * stride + c0 + j] = i < cn ? f(i, to_f32<IO>(e[j])) : 0.f;
+        }
+    }
+}
+
+// dst[i][d] = phi(x[i][d])
+template <typename IO>
+__device__ __forceinline__ void store_mapped(float* dst, const uint4 (&r)[FETCH], int cn, int D, int DS, int phi) {
+    store_rows<IO>(dst, r, cn, D, DS, [phi](int, float x) { return phi_apply(x, phi); });
+}
+
+// dst[i][0..M) = x[i][:], dst[i][M] = 1 (the ones column); padded rows are 0.
+template <typename IO>
+__device__ __forceinline__ void store_values_ext(float* dst, const uint4 (&r)[FETCH], int cn, int M, int MS) {
+    store_rows<IO>(dst, r, cn, M, MS, [](int, float x) { return x; });
+    for (int i = threadIdx.x; i < T; i += THREADS) dst[i * MS + M] = i < cn ? 1.f : 0.f;
+}
+
+template <typename IO>
+__device__ void load_mapped(float* dst, const IO* src, int cn, int D, int DS, int phi) {
+    uint4 r[FETCH];
+    fetch_rows<IO>(r, src, cn, D);
+    store_mapped<IO>(dst, r, cn, D, DS, phi);
+}
+
 template <typename IO>
 __device__ void load_values_ext(float* dst, const IO* src, int cn, int M, int MS) {
-    for (int idx = threadIdx.x; idx < T * MS; idx += THREADS) {
-        const int i = idx / MS, e = idx - i * MS;
-        float x = 0.f;
-        if (i < cn) x = e < M ? to_f32<IO>(src[(int64_t)i * M + e]) : 1.f;
-        dst[i * MS + e] = x;
-    }
+    uint4 r[FETCH];
+    fetch_rows<IO>(r, src, cn, M);
+    store_values_ext<IO>(dst, r, cn, M, MS);
 }
 
 // P[i][j] = q_i . k_j for j <= i (causal) else 0.
 __device__ void masked_scores(float* P, const float* q, const float* k, int D, int DS) {
-    for (int idx = threadIdx.x; idx < T * T; idx += THREADS) {
-        const int i = idx / T, j = idx - i * T;
-        float s = 0.f;
-        if (j <= i)
-            for (int d = 0; d < D; ++d) s = fmaf(q[i * DS + d], k[j * DS + d], s);
-        P[i * (T + 1) + j] = s;
-    }
+    block_product<2, 2>(T, T, Mat{q, DS, 1}, Mat{k, 1, DS}, D, Mat{q, 0, 0}, Mat{k, 0, 0}, 0,
+                        [&](int i, int j, float v) { P[i * (T + 1) + j] = j <= i ? v : 0.f; });
 }
 
 // nd[i][e] = sum_{j<=i} P[i][j] vt[j][e] + sum_d q[i][d] St[d][e]   (e in [0, M])
 __device__ void numerator_denominator(float* nd, const float* P, const float* vt, const float* q,
                                       const float* St, const Dims& dm, bool causal_part) {
-    for (int idx = threadIdx.x; idx < T * dm.MS; idx += THREADS) {
-        const int i = idx / dm.MS, e = idx - i * dm.MS;
+    // (P is zero right of the diagonal: the sum over all j of the chunk is the causal one)
+    block_product<2, 4>(T, dm.M, Mat{q, dm.DS, 1}, Mat{St, dm.MS, 1}, dm.D, Mat{P, T + 1, 1}, Mat{vt, dm.MS, 1},
+                        causal_part ? T : 0, [&](int i, int e, float v) { nd[i * dm.MS + e] = v; });
+    for (int i = threadIdx.x; i < T; i += THREADS) {            // the normaliser column e = M
         float s = 0.f;
         if (causal_part)
-            for (int j = 0; j <= i; ++j) s = fmaf(P[i * (T + 1) + j], vt[j * dm.MS + e], s);
-        for (int d = 0; d < dm.D; ++d) s = fmaf(q[i * dm.DS + d], St[d * dm.MS + e], s);
-        nd[i * dm.MS + e] = s;
+            for (int j = 0; j <= i; ++j) s = fmaf(P[i * (T + 1) + j], vt[j * dm.MS + dm.M], s);
+        for (int d = 0; d < dm.D; ++d) s = fmaf(q[i * dm.DS + d], St[d * dm.MS + dm.M], s);
+        nd[i * dm.MS + dm.M] = s;
     }
 }
 
 // St[d][e] += sum_i x[i][d] y[i][e]   (rank-T update of a D x (M+1) state)
 __device__ void state_update(float* St, const float* x, const float* y, const Dims& dm) {
-    for (int idx = threadIdx.x; idx < dm.D * dm.MS; idx += THREADS) {
-        const int d = idx / dm.MS, e = idx - d * dm.MS;
-        float s = St[idx];
-        for (int i = 0; i < T; ++i) s = fmaf(x[i * dm.DS + d], y[i * dm.MS + e], s);
-        St[idx] = s;
+    block_product<4, 4>(dm.D, dm.M, Mat{x, 1, dm.DS}, Mat{y, dm.MS, 1}, T, Mat{x, 0, 0}, Mat{y, 0, 0}, 0,
+                        [&](int d, int e, float v) { St[d * dm.MS + e] += v; });
+    for (int d = threadIdx.x; d < dm.D; d += THREADS) {         // column e = M
+        float s = St[d * dm.MS + dm.M];
+        for (int i = 0; i < T; ++i) s = fmaf(x[i * dm.DS + d], y[i * dm.MS + dm.M], s);
+        St[d * dm.MS + dm.M] = s;
     }
 }
 
@@ -110,13 +191,8 @@ __device__ void extend_upstream(float* g, const float* nd, const Dims& dm, float
 
 // dP[i][j] = Gt_i . Vt_j for j <= i (causal) else 0.
 __device__ void masked_dscores(float* dP, const float* gt, const float* vt, const Dims& dm) {
-    for (int idx = threadIdx.x; idx < T * T; idx += THREADS) {
-        const int i = idx / T, j = idx - i * T;
-        float s = 0.f;
-        if (j <= i)
-            for (int e = 0; e < dm.MS; ++e) s = fmaf(gt[i * dm.MS + e], vt[j * dm.MS + e], s);
-        dP[i * (T + 1) + j] = s;
-    }
+    block_product<2, 2>(T, T, Mat{gt, dm.MS, 1}, Mat{vt, 1, dm.MS}, dm.MS, Mat{gt, 0, 0}, Mat{vt, 0, 0}, 0,
+                        [&](int i, int j, float v) { dP[i * (T + 1) + j] = j <= i ? v : 0.f; });
 }
 
 size_t smem_floats_forward(int D, int M) {
@@ -154,12 +230,22 @@ general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K
         for (int d = threadIdx.x; d < D; d += THREADS) sSt[d * dm.MS + M] = Z_in[bh * D + d];
     }
 
+    // the rows of a chunk are requested one chunk ahead and wait in registers while the chunk before is worked on
+    uint4 rq[FETCH], rk[FETCH], rv[FETCH];
+    auto fetch = [&](int64_t n0) {
+        const int cn = (int)((N - n0) < T ? (N - n0) : T);
+        fetch_rows<IO>(rq, Q + n0 * D, cn, D);
+        fetch_rows<IO>(rk, K + n0 * D, cn, D);
+        fetch_rows<IO>(rv, V + n0 * M, cn, M);
+    };
+    if (N > 0) fetch(0);
     for (int64_t n0 = 0; n0 < N; n0 += T) {
         const int cn = (int)((N - n0) < T ? (N - n0) : T);
         __syncthreads();
-        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
-        load_mapped<IO>(sk, K + n0 * D, cn, D, dm.DS, phi);
-        load_values_ext<IO>(sv, V + n0 * M, cn, M, dm.MS);
+        store_mapped<IO>(sq, rq, cn, D, dm.DS, phi);
+        store_mapped<IO>(sk, rk, cn, D, dm.DS, phi);
+        store_values_ext<IO>(sv, rv, cn, M, dm.MS);
+        if (n0 + T < N) fetch(n0 + T);
         __syncthreads();
         masked_scores(sP, sq, sk, D, dm.DS);
         __syncthreads();
@@ -218,13 +304,24 @@ general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ 
             sSt[(idx / M) * dm.MS + idx % M] = sa.S_in[bh * D * M + idx];
         for (int d = threadIdx.x; d < D; d += THREADS) sSt[d * dm.MS + M] = sa.Z_in[bh * D + d];
     }
+    // the rows of a chunk are requested one chunk ahead and wait in registers while the chunk before is worked on
+    uint4 rq[FETCH], rk[FETCH], rv[FETCH], rg[FETCH];
+    auto fetch = [&](int64_t n0) {
+        const int cn = (int)((N - n0) < T ? (N - n0) : T);
+        fetch_rows<IO>(rq, Q + n0 * D, cn, D);
+        fetch_rows<IO>(rk, K + n0 * D, cn, D);
+        fetch_rows<IO>(rv, V + n0 * M, cn, M);
+        fetch_rows<IO>(rg, G + n0 * M, cn, M);
+    };
+    if (N > 0) fetch(0);
     for (int64_t n0 = 0; n0 < N; n0 += T) {
         const int cn = (int)((N - n0) < T ? (N - n0) : T);
         __syncthreads();
-        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
-        load_mapped<IO>(sk, K + n0 * D, cn, D, dm.DS, phi);
-        load_values_ext<IO>(sv, V + n0 * M, cn, M, dm.MS);
-        load_values_ext<IO>(sg, G + n0 * M, cn, M, dm.MS);
+        store_mapped<IO>(sq, rq, cn, D, dm.DS, phi);
+        store_mapped<IO>(sk, rk, cn, D, dm.DS, phi);
+        store_values_ext<IO>(sv, rv, cn, M, dm.MS);
+        store_values_ext<IO>(sg, rg, cn, M, dm.MS);
+        if (n0 + T < N) fetch(n0 + T);
         __syncthreads();
         masked_scores(sP, sq, sk, D, dm.DS);
         __syncthreads();
@@ -235,13 +332,11 @@ general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ 
         masked_dscores(sdP, sg, sv, dm);
         __syncthreads();
         // grad phi(Q_i) = sum_{j<=i} dP_ij k_j + St_{c-1} Gt_i
-        for (int idx = threadIdx.x; idx < cn * D; idx += THREADS) {
-            const int i = idx / D, d = idx - i * D;
-            float s = 0.f;
-            for (int j = 0; j <= i; ++j) s = fmaf(sdP[i * (T + 1) + j], sk[j * dm.DS + d], s);
-            for (int e = 0; e < dm.MS; ++e) s = fmaf(sSt[d * dm.MS + e], sg[i * dm.MS + e], s);
-            dQ[(n0 + i) * D + d] = from_f32<IO>(s * phi_slope_from_value(sq[i * dm.DS + d], phi));
-        }
+        // (dP is zero right of the diagonal)
+        block_product<2, 4>(T, D, Mat{sdP, T + 1, 1}, Mat{sk, dm.DS, 1}, T, Mat{sg, dm.MS, 1}, Mat{sSt, 1, dm.MS}, dm.MS,
+                            [&](int i, int d, float v) {
+                                if (i < cn) dQ[(n0 + i) * D + d] = from_f32<IO>(v * phi_slope_from_value(sq[i * dm.DS + d], phi));
+                            });
         __syncthreads();
         state_update(sSt, sk, sv, dm);
     }
@@ -259,40 +354,45 @@ general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ 
             for (int d = threadIdx.x; d < D; d += THREADS) sSt[d * dm.MS + M] = sa.dZ_out[bh * D + d];
     }
     const int64_t nchunks = (N + T - 1) / T;
+    float r_dn = 1.f, r_delta = 0.f;          // dn_i, delta_i of row threadIdx.x of the fetched chunk
+    auto fetch_back = [&](int64_t n0) {
+        const int cn = (int)((N - n0) < T ? (N - n0) : T);
+        fetch(n0);
+        if ((int)threadIdx.x < cn) {
+            r_dn = dn_all[n0 + threadIdx.x];
+            r_delta = delta_all[n0 + threadIdx.x];
+        }
+    };
+    if (nchunks > 0) fetch_back((nchunks - 1) * T);
+    float* s_dn = snd;                        // [T] dn_i of the chunk (snd is free in this sweep)
     for (int64_t c = nchunks - 1; c >= 0; --c) {
         const int64_t n0 = c * T;
         const int cn = (int)((N - n0) < T ? (N - n0) : T);
         __syncthreads();
-        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
-        load_mapped<IO>(sk, K + n0 * D, cn, D, dm.DS, phi);
-        load_values_ext<IO>(sv, V + n0 * M, cn, M, dm.MS);
-        for (int idx = threadIdx.x; idx < T * dm.MS; idx += THREADS) {
-            const int i = idx / dm.MS, e = idx - i * dm.MS;
-            float x = 0.f;
-            if (i < cn)
-                x = e < M ? to_f32<IO>(G[(n0 + i) * M + e]) / dn_all[n0 + i] : delta_all[n0 + i];
-            sg[idx] = x;
-        }
+        if ((int)threadIdx.x < T) s_dn[threadIdx.x] = (int)threadIdx.x < cn ? r_dn : 1.f;
+        store_mapped<IO>(sq, rq, cn, D, dm.DS, phi);
+        store_mapped<IO>(sk, rk, cn, D, dm.DS, phi);
+        store_values_ext<IO>(sv, rv, cn, M, dm.MS);
+        __syncthreads();
+        // Gt_i = [G_i / dn_i, delta_i]
+        store_rows<IO>(sg, rg, cn, M, dm.MS, [&](int i, float x) { return x / s_dn[i]; });
+        if ((int)threadIdx.x < T) sg[threadIdx.x * dm.MS + M] = (int)threadIdx.x < cn ? r_delta : 0.f;
+        if (c > 0) fetch_back(n0 - T);
         __syncthreads();
         masked_scores(sP, sq, sk, D, dm.DS);
         masked_dscores(sdP, sg, sv, dm);
         __syncthreads();
         // grad phi(K_j) = sum_{i>=j} dP_ij q_i + Rt_{c+1} Vt_j          (Eq. 14)
-        for (int idx = threadIdx.x; idx < cn * D; idx += THREADS) {
-            const int j = idx / D, d = idx - j * D;
-            float s = 0.f;
-            for (int i = j; i < T; ++i) s = fmaf(sdP[i * (T + 1) + j], sq[i * dm.DS + d], s);
-            for (int e = 0; e < dm.MS; ++e) s = fmaf(sSt[d * dm.MS + e], sv[j * dm.MS + e], s);
-            dK[(n0 + j) * D + d] = from_f32<IO>(s * phi_slope_from_value(sk[j * dm.DS + d], phi));
-        }
+        // (dP and P are zero right of the diagonal: summing over all i of the chunk keeps i >= j)
+        block_product<2, 4>(T, D, Mat{sdP, 1, T + 1}, Mat{sq, dm.DS, 1}, T, Mat{sv, dm.MS, 1}, Mat{sSt, 1, dm.MS}, dm.MS,
+                            [&](int j, int d, float v) {
+                                if (j < cn) dK[(n0 + j) * D + d] = from_f32<IO>(v * phi_slope_from_value(sk[j * dm.DS + d], phi));
+                            });
         // grad V_j = sum_{i>=j} P_ij Gt_i[0:M] + Rt_{c+1}^T k_j          (Eq. 15)
-        for (int idx = threadIdx.x; idx < cn * M; idx += THREADS) {
-            const int j = idx / M, e = idx - j * M;
-            float s = 0.f;
-            for (int i = j; i < T; ++i) s = fmaf(sP[i * (T + 1) + j], sg[i * dm.MS + e], s);
-            for (int d = 0; d < D; ++d) s = fmaf(sSt[d * dm.MS + e], sk[j * dm.DS + d], s);
-            dV[(n0 + j) * M + e] = from_f32<IO>(s);
-        }
+        block_product<2, 4>(T, M, Mat{sP, 1, T + 1}, Mat{sg, dm.MS, 1}, T, Mat{sk, dm.DS, 1}, Mat{sSt, dm.MS, 1}, D,
+                            [&](int j, int e, float v) {
+                                if (j < cn) dV[(n0 + j) * M + e] = from_f32<IO>(v);
+                            });
         __syncthreads();
         state_update(sSt, sq, sg, dm);
     }
@@ -445,12 +545,10 @@ general_linear_bwd_q_kernel(const IO* __restrict__ Q, const IO* __restrict__ G,
         __syncthreads();
         extend_upstream(sg, snd, dm, eps, cn, nullptr, nullptr);
         __syncthreads();
-        for (int idx = threadIdx.x; idx < cn * D; idx += THREADS) {
-            const int i = idx / D, d = idx - i * D;
-            float s = 0.f;
-            for (int e = 0; e < dm.MS; ++e) s = fmaf(sSt[d * dm.MS + e], sg[i * dm.MS + e], s);
-            dQ[(n0 + i) * D + d] = from_f32<IO>(s * phi_slope_from_value(sq[i * dm.DS + d], phi));
-        }
+        block_product<2, 4>(T, D, Mat{sg, dm.MS, 1}, Mat{sSt, 1, dm.MS}, dm.MS, Mat{sg, 0, 0}, Mat{sSt, 0, 0}, 0,
+                            [&](int i, int d, float v) {
+                                if (i < cn) dQ[(n0 + i) * D + d] = from_f32<IO>(v * phi_slope_from_value(sq[i * dm.DS + d], phi));
+                            });
         state_update(sRt, sq, sg, dm);
     }
     __syncthreads();
@@ -483,18 +581,14 @@ general_linear_bwd_kv_kernel(const IO* __restrict__ K, const IO* __restrict__ V,
         load_mapped<IO>(sk, K + n0 * D, cn, D, dm.DS, phi);
         load_values_ext<IO>(sv, V + n0 * M, cn, M, dm.MS);
         __syncthreads();
-        for (int idx = threadIdx.x; idx < cn * D; idx += THREADS) {
-            const int j = idx / D, d = idx - j * D;
-            float s = 0.f;
-            for (int e = 0; e < dm.MS; ++e) s = fmaf(sRt[d * dm.MS + e], sv[j * dm.MS + e], s);
-            dK[(n0 + j) * D + d] = from_f32<IO>(s * phi_slope_from_value(sk[j * dm.DS + d], phi));
-        }
-        for (int idx = threadIdx.x; idx < cn * M; idx += THREADS) {
-            const int j = idx / M, e = idx - j * M;
-            float s = 0.f;
-            for (int d = 0; d < D; ++d) s = fmaf(sRt[d * dm.MS + e], sk[j * dm.DS + d], s);
-            dV[(n0 + j) * M + e] = from_f32<IO>(s);
-        }
+        block_product<2, 4>(T, D, Mat{sv, dm.MS, 1}, Mat{sRt, 1, dm.MS}, dm.MS, Mat{sv, 0, 0}, Mat{sRt, 0, 0}, 0,
+                            [&](int j, int d, float v) {
+                                if (j < cn) dK[(n0 + j) * D + d] = from_f32<IO>(v * phi_slope_from_value(sk[j * dm.DS + d], phi));
+                            });
+        block_product<2, 4>(T, M, Mat{sk, dm.DS, 1}, Mat{sRt, dm.MS, 1}, D, Mat{sk, 0, 0}, Mat{sRt, 0, 0}, 0,
+                            [&](int j, int e, float v) {
+                                if (j < cn) dV[(n0 + j) * M + e] = from_f32<IO>(v);
+                            });
     }
 }
 
