@@ -114,20 +114,6 @@ __device__ __forceinline__ void store_values_ext(float* dst, const uint4 (&r)[FE
     for (int i = threadIdx.x; i < T; i += THREADS) dst[i * MS + M] = i < cn ? 1.f : 0.f;
 }
 
-template <typename IO>
-__device__ void load_mapped(float* dst, const IO* src, int cn, int D, int DS, int phi) {
-    uint4 r[FETCH];
-    fetch_rows<IO>(r, src, cn, D);
-    store_mapped<IO>(dst, r, cn, D, DS, phi);
-}
-
-template <typename IO>
-__device__ void load_values_ext(float* dst, const IO* src, int cn, int M, int MS) {
-    uint4 r[FETCH];
-    fetch_rows<IO>(r, src, cn, M);
-    store_values_ext<IO>(dst, r, cn, M, MS);
-}
-
 // P[i][j] = q_i . k_j for j <= i (causal) else 0.
 __device__ void masked_scores(float* P, const float* q, const float* k, int D, int DS) {
     block_product<2, 2>(T, T, Mat{q, DS, 1}, Mat{k, 1, DS}, D, Mat{q, 0, 0}, Mat{k, 0, 0}, 0,
@@ -448,11 +434,19 @@ general_kv_sum_kernel(const IO* __restrict__ X, const IO* __restrict__ Y, float*
     const int64_t lo = sp * split_len, hi = real_end(lengths, heads, bh, (lo + split_len) < N ? (lo + split_len) : N);
     X += bh * N * D; Y += bh * N * M;
     zero_fill(sSt, D * dm.MS);
+    uint4 rx[FETCH], ry[FETCH];               // the rows of the chunk after the one being worked on
+    auto fetch = [&](int64_t n0) {
+        const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
+        fetch_rows<IO>(rx, X + n0 * D, cn, D);
+        fetch_rows<IO>(ry, Y + n0 * M, cn, M);
+    };
+    if (lo < hi) fetch(lo);
     for (int64_t n0 = lo; n0 < hi; n0 += T) {
         const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
         __syncthreads();
-        load_mapped<IO>(sx, X + n0 * D, cn, D, dm.DS, phi);
-        load_values_ext<IO>(sy, Y + n0 * M, cn, M, dm.MS);
+        store_mapped<IO>(sx, rx, cn, D, dm.DS, phi);
+        store_values_ext<IO>(sy, ry, cn, M, dm.MS);
+        if (n0 + T < hi) fetch(n0 + T);
         __syncthreads();
         state_update(sSt, sx, sy, dm);
     }
@@ -496,10 +490,17 @@ general_linear_apply_kernel(const IO* __restrict__ Q, const float* __restrict__ 
         if (Zs)
             for (int d = threadIdx.x; d < D; d += THREADS) Zs[bh * D + d] = sSt[d * dm.MS + M];
     }
+    uint4 rx[FETCH];                          // the rows of the chunk after the one being worked on
+    auto fetch = [&](int64_t n0) {
+        const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
+        fetch_rows<IO>(rx, Q + n0 * D, cn, D);
+    };
+    if (lo < hi) fetch(lo);
     for (int64_t n0 = lo; n0 < hi; n0 += T) {
         const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
         __syncthreads();
-        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
+        store_mapped<IO>(sq, rx, cn, D, dm.DS, phi);
+        if (n0 + T < hi) fetch(n0 + T);
         __syncthreads();
         numerator_denominator(snd, nullptr, nullptr, sq, sSt, dm, false);
         __syncthreads();
@@ -535,11 +536,19 @@ general_linear_bwd_q_kernel(const IO* __restrict__ Q, const IO* __restrict__ G,
     for (int64_t idx = (lo > hi ? lo : hi) * D + threadIdx.x; idx < hi_all * D; idx += THREADS) dQ[idx] = from_f32<IO>(0.f);
     load_reduced_state(sSt, part_s + bh * nsplit * (int64_t)(D * dm.MS), nsplit, D * dm.MS);
     zero_fill(sRt, D * dm.MS);
+    uint4 rx[FETCH], ry[FETCH];               // the rows of the chunk after the one being worked on
+    auto fetch = [&](int64_t n0) {
+        const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
+        fetch_rows<IO>(rx, Q + n0 * D, cn, D);
+        fetch_rows<IO>(ry, G + n0 * M, cn, M);
+    };
+    if (lo < hi) fetch(lo);
     for (int64_t n0 = lo; n0 < hi; n0 += T) {
         const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
         __syncthreads();
-        load_mapped<IO>(sq, Q + n0 * D, cn, D, dm.DS, phi);
-        load_values_ext<IO>(sg, G + n0 * M, cn, M, dm.MS);
+        store_mapped<IO>(sq, rx, cn, D, dm.DS, phi);
+        store_values_ext<IO>(sg, ry, cn, M, dm.MS);
+        if (n0 + T < hi) fetch(n0 + T);
         __syncthreads();
         numerator_denominator(snd, nullptr, nullptr, sq, sSt, dm, false);
         __syncthreads();
@@ -575,11 +584,19 @@ general_linear_bwd_kv_kernel(const IO* __restrict__ K, const IO* __restrict__ V,
     for (int64_t idx = (lo > hi ? lo : hi) * D + threadIdx.x; idx < hi_all * D; idx += THREADS) dK[idx] = from_f32<IO>(0.f);
     for (int64_t idx = (lo > hi ? lo : hi) * M + threadIdx.x; idx < hi_all * M; idx += THREADS) dV[idx] = from_f32<IO>(0.f);
     load_reduced_state(sRt, part_r + bh * nsplit * (int64_t)(D * dm.MS), nsplit, D * dm.MS);
+    uint4 rx[FETCH], ry[FETCH];               // the rows of the chunk after the one being worked on
+    auto fetch = [&](int64_t n0) {
+        const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
+        fetch_rows<IO>(rx, K + n0 * D, cn, D);
+        fetch_rows<IO>(ry, V + n0 * M, cn, M);
+    };
+    if (lo < hi) fetch(lo);
     for (int64_t n0 = lo; n0 < hi; n0 += T) {
         const int cn = (int)((hi - n0) < T ? (hi - n0) : T);
         __syncthreads();
-        load_mapped<IO>(sk, K + n0 * D, cn, D, dm.DS, phi);
-        load_values_ext<IO>(sv, V + n0 * M, cn, M, dm.MS);
+        store_mapped<IO>(sk, rx, cn, D, dm.DS, phi);
+        store_values_ext<IO>(sv, ry, cn, M, dm.MS);
+        if (n0 + T < hi) fetch(n0 + T);
         __syncthreads();
         block_product<2, 4>(T, D, Mat{sv, dm.MS, 1}, Mat{sRt, 1, dm.MS}, dm.MS, Mat{sv, 0, 0}, Mat{sRt, 0, 0}, 0,
                             [&](int j, int d, float v) {
