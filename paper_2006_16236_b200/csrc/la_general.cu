@@ -191,13 +191,15 @@ size_t smem_floats_backward(int D, int M) {
 // ---------------------------------------------------------------------------
 // Causal forward: one CTA walks one (batch, head) sequence chunk by chunk.
 // ---------------------------------------------------------------------------
-template <typename IO>
+// KD: D = M = KD known at compile time (all tile strides become constants), or 0: any D, M.
+template <typename IO, int KD>
 __global__ void __launch_bounds__(THREADS)
 general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K, const IO* __restrict__ V,
                               const float* __restrict__ S_in, const float* __restrict__ Z_in,
                               IO* __restrict__ O, float* __restrict__ den, float* __restrict__ S_out,
-                              float* __restrict__ Z_out, int64_t N, int D, int M, float eps, int phi) {
+                              float* __restrict__ Z_out, int64_t N, int D_arg, int M_arg, float eps, int phi) {
     extern __shared__ float smem[];
+    const int D = KD ? KD : D_arg, M = KD ? KD : M_arg;
     const Dims dm = make_dims(D, M);
     float* sq = smem;
     float* sk = sq + T * dm.DS;
@@ -259,13 +261,14 @@ general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K
 // delta_i found in the forward sweep are parked in `aux` ([B,H,N,2] fp32) for
 // the reverse sweep; no per-position state is stored.
 // ---------------------------------------------------------------------------
-template <typename IO>
+template <typename IO, int KD>
 __global__ void __launch_bounds__(THREADS)
 general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K, const IO* __restrict__ V,
                                const IO* __restrict__ G, const StateArgs sa, IO* __restrict__ dQ,
                                IO* __restrict__ dK, IO* __restrict__ dV, float* __restrict__ aux,
-                               int64_t N, int D, int M, float eps, int phi) {
+                               int64_t N, int D_arg, int M_arg, float eps, int phi) {
     extern __shared__ float smem[];
+    const int D = KD ? KD : D_arg, M = KD ? KD : M_arg;
     const Dims dm = make_dims(D, M);
     float* sq = smem;
     float* sk = sq + T * dm.DS;
@@ -421,11 +424,12 @@ __device__ __forceinline__ int64_t real_end(const int* lengths, int heads, int64
 }
 
 // part[bh][split] = sum over the split's positions of phi(X_i) [Y_i, 1]^T.
-template <typename IO>
+template <typename IO, int KD>
 __global__ void __launch_bounds__(THREADS)
 general_kv_sum_kernel(const IO* __restrict__ X, const IO* __restrict__ Y, float* __restrict__ part,
-                      int64_t N, int64_t split_len, int D, int M, int phi, const int* __restrict__ lengths, int heads) {
+                      int64_t N, int64_t split_len, int D_arg, int M_arg, int phi, const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
+    const int D = KD ? KD : D_arg, M = KD ? KD : M_arg;
     const Dims dm = make_dims(D, M);
     float* sx = smem;
     float* sy = sx + T * dm.DS;
@@ -463,13 +467,14 @@ __device__ void load_reduced_state(float* sSt, const float* part, int nsplit, in
     }
 }
 
-template <typename IO>
+template <typename IO, int KD>
 __global__ void __launch_bounds__(THREADS)
 general_linear_apply_kernel(const IO* __restrict__ Q, const float* __restrict__ part, IO* __restrict__ O,
                             float* __restrict__ den, float* __restrict__ KV, float* __restrict__ Zs,
-                            int nsplit, int64_t N, int64_t split_len, int D, int M, float eps, int phi,
+                            int nsplit, int64_t N, int64_t split_len, int D_arg, int M_arg, float eps, int phi,
                             const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
+    const int D = KD ? KD : D_arg, M = KD ? KD : M_arg;
     const Dims dm = make_dims(D, M);
     float* sq = smem;
     float* snd = sq + T * dm.DS;
@@ -516,13 +521,14 @@ general_linear_apply_kernel(const IO* __restrict__ Q, const float* __restrict__ 
 // Backward, query side: with St = full sum, form Gt_i, write
 // grad phi(Q_i) = St Gt_i (Eq. 13 with the full sum) and accumulate this split's
 // part of Rt = sum_i phi(Q_i) Gt_i^T.
-template <typename IO>
+template <typename IO, int KD>
 __global__ void __launch_bounds__(THREADS)
 general_linear_bwd_q_kernel(const IO* __restrict__ Q, const IO* __restrict__ G,
                             const float* __restrict__ part_s, IO* __restrict__ dQ,
                             float* __restrict__ part_r, int nsplit, int64_t N, int64_t split_len,
-                            int D, int M, float eps, int phi, const int* __restrict__ lengths, int heads) {
+                            int D_arg, int M_arg, float eps, int phi, const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
+    const int D = KD ? KD : D_arg, M = KD ? KD : M_arg;
     const Dims dm = make_dims(D, M);
     float* sq = smem;
     float* sg = sq + T * dm.DS;
@@ -566,13 +572,14 @@ general_linear_bwd_q_kernel(const IO* __restrict__ Q, const IO* __restrict__ G,
 }
 
 // Backward, key/value side: grad phi(K_j) = Rt Vt_j (Eq. 14), grad V_j = (Rt^T phi(K_j))[0:M] (Eq. 15).
-template <typename IO>
+template <typename IO, int KD>
 __global__ void __launch_bounds__(THREADS)
 general_linear_bwd_kv_kernel(const IO* __restrict__ K, const IO* __restrict__ V,
                              const float* __restrict__ part_r, IO* __restrict__ dK, IO* __restrict__ dV,
-                             int nsplit, int64_t N, int64_t split_len, int D, int M, int phi,
+                             int nsplit, int64_t N, int64_t split_len, int D_arg, int M_arg, int phi,
                              const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
+    const int D = KD ? KD : D_arg, M = KD ? KD : M_arg;
     const Dims dm = make_dims(D, M);
     float* sk = smem;
     float* sv = sk + T * dm.DS;
@@ -637,7 +644,7 @@ template <typename IO>
 static int causal_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
                             const float* Z_in, void* O, float* den, float* S_out, float* Z_out, cudaStream_t st) {
     const size_t smem = smem_floats_forward((int)p.D, (int)p.M) * sizeof(float);
-    auto kern = general_causal_forward_kernel<IO>;
+    auto kern = p.D == 64 && p.M == 64 ? general_causal_forward_kernel<IO, 64> : general_causal_forward_kernel<IO, 0>;
     if (int rc = opt_in_smem(kern, smem)) return rc;
     kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, S_in, Z_in, (IO*)O, den,
                                                        S_out, Z_out, p.N, (int)p.D, (int)p.M, p.eps, p.phi);
@@ -656,7 +663,7 @@ static int causal_backward_t(const la_problem& p, const void* Q, const void* K, 
                              const void* G, const StateArgs& sa, void* dQ, void* dK, void* dV, void* ws,
                              cudaStream_t st) {
     const size_t smem = smem_floats_backward((int)p.D, (int)p.M) * sizeof(float);
-    auto kern = general_causal_backward_kernel<IO>;
+    auto kern = p.D == 64 && p.M == 64 ? general_causal_backward_kernel<IO, 64> : general_causal_backward_kernel<IO, 0>;
     if (int rc = opt_in_smem(kern, smem)) return rc;
     kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, (const IO*)G, sa,
                                                        (IO*)dQ, (IO*)dK, (IO*)dV, (float*)ws, p.N, (int)p.D,
@@ -680,14 +687,14 @@ static int linear_forward_t(const la_problem& p, const void* Q, const void* K, c
     float* part = (float*)ws;
     {
         const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
-        auto kern = general_kv_sum_kernel<IO>;
+        auto kern = D == 64 && M == 64 ? general_kv_sum_kernel<IO, 64> : general_kv_sum_kernel<IO, 0>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
         kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part, p.N, sp.len, D, M, p.phi, lengths, (int)p.H);
         LA_LAUNCHED();
     }
     {
         const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
-        auto kern = general_linear_apply_kernel<IO>;
+        auto kern = D == 64 && M == 64 ? general_linear_apply_kernel<IO, 64> : general_linear_apply_kernel<IO, 0>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
         kern<<<grid, THREADS, smem, st>>>((const IO*)Q, part, (IO*)O, den, KV, Zs, sp.nsplit, p.N, sp.len, D, M,
                                           p.eps, p.phi, lengths, (int)p.H);
@@ -712,14 +719,14 @@ static int linear_backward_t(const la_problem& p, const void* Q, const void* K, 
     float* part_r = part_s + (size_t)(p.B * p.H) * sp.nsplit * state_floats(p);
     {
         const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
-        auto kern = general_kv_sum_kernel<IO>;
+        auto kern = D == 64 && M == 64 ? general_kv_sum_kernel<IO, 64> : general_kv_sum_kernel<IO, 0>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
         kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part_s, p.N, sp.len, D, M, p.phi, lengths, (int)p.H);
         LA_LAUNCHED();
     }
     {
         const size_t smem = ((size_t)T * (D + 1) + (size_t)2 * T * (M + 1) + 2 * state_floats(p)) * sizeof(float);
-        auto kern = general_linear_bwd_q_kernel<IO>;
+        auto kern = D == 64 && M == 64 ? general_linear_bwd_q_kernel<IO, 64> : general_linear_bwd_q_kernel<IO, 0>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
         kern<<<grid, THREADS, smem, st>>>((const IO*)Q, (const IO*)G, part_s, (IO*)dQ, part_r, sp.nsplit, p.N,
                                           sp.len, D, M, p.eps, p.phi, lengths, (int)p.H);
@@ -727,7 +734,7 @@ static int linear_backward_t(const la_problem& p, const void* Q, const void* K, 
     }
     {
         const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
-        auto kern = general_linear_bwd_kv_kernel<IO>;
+        auto kern = D == 64 && M == 64 ? general_linear_bwd_kv_kernel<IO, 64> : general_linear_bwd_kv_kernel<IO, 0>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
         kern<<<grid, THREADS, smem, st>>>((const IO*)K, (const IO*)V, part_r, (IO*)dK, (IO*)dV, sp.nsplit, p.N,
                                           sp.len, D, M, p.phi, lengths, (int)p.H);
