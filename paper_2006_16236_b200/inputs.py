@@ -58,6 +58,8 @@ WORKLOADS = {
         _sweep(12), _sweep(13), _sweep(14), _sweep(15), _sweep(16),
         Workload("decode_bf16_streams", "decode", 256, 8, 3072, 64, 64, "bf16", 5, 1.0,
                  "many-stream autoregressive generation, one recurrent step per pixel"),
+        Workload("causal_fp32_N4096", "causal", 32, 8, 4096, 64, 64, "f32", 6, 1.0,
+                 "the N = 4096 point of the sequence-length benchmark in fp32 (general kernels)"),
     ]
 }
 

@@ -482,7 +482,7 @@ def _sample_heads(B, H, k=3):
 
 @pytest.mark.parametrize("name", ["causal_fp32_small", "causal_bf16_image", "causal_sweep_bf16_N4096",
                                   "causal_sweep_bf16_N8192", "causal_sweep_bf16_N16384",
-                                  "causal_sweep_bf16_N32768", "causal_sweep_bf16_N65536"])
+                                  "causal_sweep_bf16_N32768", "causal_sweep_bf16_N65536", "causal_fp32_N4096"])
 @pytest.mark.parametrize("keep", [False, True], ids=["recompute", "saved"])
 def test_causal_workloads_full_size(name, keep):
     w = WORKLOADS[name]
