@@ -124,7 +124,7 @@ __device__ void masked_scores(float* P, const float* q, const float* k, int D, i
 __device__ void numerator_denominator(float* nd, const float* P, const float* vt, const float* q,
                                       const float* St, const Dims& dm, bool causal_part) {
     // (P is zero right of the diagonal: the sum over all j of the chunk is the causal one)
-    block_product<2, 4>(T, dm.M, Mat{q, dm.DS, 1}, Mat{St, dm.MS, 1}, dm.D, Mat{P, T + 1, 1}, Mat{vt, dm.MS, 1},
+    block_product<4, 4>(T, dm.M, Mat{q, dm.DS, 1}, Mat{St, dm.MS, 1}, dm.D, Mat{P, T + 1, 1}, Mat{vt, dm.MS, 1},
                         causal_part ? T : 0, [&](int i, int e, float v) { nd[i * dm.MS + e] = v; });
     for (int i = threadIdx.x; i < T; i += THREADS) {            // the normaliser column e = M
         float s = 0.f;
@@ -322,7 +322,7 @@ general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ 
         __syncthreads();
         // grad phi(Q_i) = sum_{j<=i} dP_ij k_j + St_{c-1} Gt_i
         // (dP is zero right of the diagonal)
-        block_product<2, 4>(T, D, Mat{sdP, T + 1, 1}, Mat{sk, dm.DS, 1}, T, Mat{sg, dm.MS, 1}, Mat{sSt, 1, dm.MS}, dm.MS,
+        block_product<4, 4>(T, D, Mat{sdP, T + 1, 1}, Mat{sk, dm.DS, 1}, T, Mat{sg, dm.MS, 1}, Mat{sSt, 1, dm.MS}, dm.MS,
                             [&](int i, int d, float v) {
                                 if (i < cn) dQ[(n0 + i) * D + d] = from_f32<IO>(v * phi_slope_from_value(sq[i * dm.DS + d], phi));
                             });
@@ -373,12 +373,12 @@ general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ 
         __syncthreads();
         // grad phi(K_j) = sum_{i>=j} dP_ij q_i + Rt_{c+1} Vt_j          (Eq. 14)
         // (dP and P are zero right of the diagonal: summing over all i of the chunk keeps i >= j)
-        block_product<2, 4>(T, D, Mat{sdP, 1, T + 1}, Mat{sq, dm.DS, 1}, T, Mat{sv, dm.MS, 1}, Mat{sSt, 1, dm.MS}, dm.MS,
+        block_product<4, 4>(T, D, Mat{sdP, 1, T + 1}, Mat{sq, dm.DS, 1}, T, Mat{sv, dm.MS, 1}, Mat{sSt, 1, dm.MS}, dm.MS,
                             [&](int j, int d, float v) {
                                 if (j < cn) dK[(n0 + j) * D + d] = from_f32<IO>(v * phi_slope_from_value(sk[j * dm.DS + d], phi));
                             });
         // grad V_j = sum_{i>=j} P_ij Gt_i[0:M] + Rt_{c+1}^T k_j          (Eq. 15)
-        block_product<2, 4>(T, M, Mat{sP, 1, T + 1}, Mat{sg, dm.MS, 1}, T, Mat{sk, dm.DS, 1}, Mat{sSt, dm.MS, 1}, D,
+        block_product<4, 4>(T, M, Mat{sP, 1, T + 1}, Mat{sg, dm.MS, 1}, T, Mat{sk, dm.DS, 1}, Mat{sSt, dm.MS, 1}, D,
                             [&](int j, int e, float v) {
                                 if (j < cn) dV[(n0 + j) * M + e] = from_f32<IO>(v);
                             });
@@ -560,7 +560,7 @@ general_linear_bwd_q_kernel(const IO* __restrict__ Q, const IO* __restrict__ G,
         __syncthreads();
         extend_upstream(sg, snd, dm, eps, cn, nullptr, nullptr);
         __syncthreads();
-        block_product<2, 4>(T, D, Mat{sg, dm.MS, 1}, Mat{sSt, 1, dm.MS}, dm.MS, Mat{sg, 0, 0}, Mat{sSt, 0, 0}, 0,
+        block_product<4, 4>(T, D, Mat{sg, dm.MS, 1}, Mat{sSt, 1, dm.MS}, dm.MS, Mat{sg, 0, 0}, Mat{sSt, 0, 0}, 0,
                             [&](int i, int d, float v) {
                                 if (i < cn) dQ[(n0 + i) * D + d] = from_f32<IO>(v * phi_slope_from_value(sq[i * dm.DS + d], phi));
                             });
@@ -605,11 +605,11 @@ general_linear_bwd_kv_kernel(const IO* __restrict__ K, const IO* __restrict__ V,
         store_values_ext<IO>(sv, ry, cn, M, dm.MS);
         if (n0 + T < hi) fetch(n0 + T);
         __syncthreads();
-        block_product<2, 4>(T, D, Mat{sv, dm.MS, 1}, Mat{sRt, 1, dm.MS}, dm.MS, Mat{sv, 0, 0}, Mat{sRt, 0, 0}, 0,
+        block_product<4, 4>(T, D, Mat{sv, dm.MS, 1}, Mat{sRt, 1, dm.MS}, dm.MS, Mat{sv, 0, 0}, Mat{sRt, 0, 0}, 0,
                             [&](int j, int d, float v) {
                                 if (j < cn) dK[(n0 + j) * D + d] = from_f32<IO>(v * phi_slope_from_value(sk[j * dm.DS + d], phi));
                             });
-        block_product<2, 4>(T, M, Mat{sk, dm.DS, 1}, Mat{sRt, dm.MS, 1}, D, Mat{sk, 0, 0}, Mat{sRt, 0, 0}, 0,
+        block_product<4, 4>(T, M, Mat{sk, dm.DS, 1}, Mat{sRt, dm.MS, 1}, D, Mat{sk, 0, 0}, Mat{sRt, 0, 0}, 0,
                             [&](int j, int e, float v) {
                                 if (j < cn) dV[(n0 + j) * M + e] = from_f32<IO>(v);
                             });
