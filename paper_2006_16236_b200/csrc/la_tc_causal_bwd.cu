@@ -182,6 +182,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 if (*abort_flag) break;
                 uint8_t* st = smem + kDqOffStage + s * 4 * kTileBytes;
                 const int y = (int)(row0 + (int64_t)c * kChunk);
+                LA_TRACE(g_trace_dq, c, 13);
                 mbar_arrive_expect_tx(&bars->full[s], 4 * kTileBytes);
                 tma_load_2d(st + kTileBytes, &mapV, 0, y, &bars->full[s]);
                 tma_load_2d(st + 2 * kTileBytes, &mapG, 0, y, &bars->full[s]);
