@@ -159,7 +159,7 @@ class CausalStep:
         self.host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in [self.O] + self.grads]
         self.causal = w.kind == "causal"
         # a training step keeps phi(Q), phi(K) from the forward for the backward (None: nothing to keep)
-        self.saved = la.saved_buffer(self.d[0], self.d[2]) if self.causal else None
+        self.saved = la.saved_buffer(self.d[0], self.d[2]) if self.causal else la.linear_saved_buffer(self.d[0], self.d[2])
         # a step in the middle of a longer sequence: the forward continues from a given state and returns the
         # final one, the backward takes the final state's upstream gradient and returns the initial state's
         self.state = None
@@ -180,7 +180,7 @@ class CausalStep:
         elif self.causal:
             self.la.la_causal_forward(Q, K, V, O=self.O, den=self.den, saved=self.saved)
         else:
-            self.la.la_linear_attention(Q, K, V, O=self.O, den=self.den)
+            self.la.la_linear_attention(Q, K, V, O=self.O, den=self.den, saved=self.saved)
 
     def bwd(self):
         Q, K, V, G = self.d
@@ -193,7 +193,7 @@ class CausalStep:
         elif self.causal:
             self.la.la_causal_backward(Q, K, V, G, O=self.O, den=self.den, saved=self.saved, dQ=dQ, dK=dK, dV=dV)
         else:
-            self.la.la_linear_attention_backward(Q, K, V, G, O=self.O, den=self.den, dQ=dQ, dK=dK, dV=dV)
+            self.la.la_linear_attention_backward(Q, K, V, G, O=self.O, den=self.den, dQ=dQ, dK=dK, dV=dV, saved=self.saved)
 
     def step(self):
         self.fwd()

@@ -67,7 +67,8 @@ typedef enum {
     LA_OP_CAUSAL_BACKWARD = 3,
     LA_OP_CAUSAL_SAVED = 4,      /* size of the optional `saved` buffer, see la_causal_forward() */
     LA_OP_LINEAR_VARLEN_FORWARD = 5,     /* la_linear_attention_varlen()          */
-    LA_OP_LINEAR_VARLEN_BACKWARD = 6     /* la_linear_attention_varlen_backward() */
+    LA_OP_LINEAR_VARLEN_BACKWARD = 6,    /* la_linear_attention_varlen_backward() */
+    LA_OP_LINEAR_SAVED = 7               /* size of the optional `saved` buffer, see la_linear_attention_keep() */
 } la_op;
 
 typedef struct {
@@ -145,6 +146,29 @@ int la_linear_attention_varlen_backward(const la_problem* p, const void* Q, cons
                                         const void* O, const float* den, const void* G,
                                         void* dQ, void* dK, void* dV,
                                         void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The non-causal form for a training step: the forward keeps what it computed once per head, as the
+ * paper's "compute KV once and reuse it" does for the queries, so that the backward pass does not form
+ * the sums over the keys again.  lengths: NULL (full-length batch) or as for the _varlen calls.
+ * saved (device, 16-byte aligned, la_workspace_bytes(p, LA_OP_LINEAR_SAVED) bytes, owned by the caller):
+ * written by la_linear_attention_keep() (per-split sums of phi(K_j) [V_j | 1]^T; layout private to the
+ * library), valid for la_linear_attention_backward_kept() with the same problem, lengths, K and V until
+ * overwritten.  With saved == NULL the calls behave exactly like the plain / _varlen ones; with a saved
+ * buffer the forward does not touch its workspace (ws may be NULL) and the results of both calls are the
+ * same bit for bit as without.
+ */
+int la_linear_attention_keep(const la_problem* p, const void* Q, const void* K, const void* V,
+                             const int32_t* lengths,
+                             void* O, float* den, float* KV, float* Zs,
+                             void* saved, size_t saved_bytes,
+                             void* ws, size_t ws_bytes, void* stream);
+int la_linear_attention_backward_kept(const la_problem* p, const void* Q, const void* K, const void* V,
+                                      const int32_t* lengths,
+                                      const void* saved, size_t saved_bytes,
+                                      const void* O, const float* den, const void* G,
+                                      void* dQ, void* dK, void* dV,
+                                      void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Causal linear attention, Eq. 9-12 (Algorithm 1, forward, plus the normaliser):

@@ -19,12 +19,14 @@ LA_PHI_ELU1, LA_PHI_IDENTITY = 0, 1
 LA_OP_LINEAR_FORWARD, LA_OP_LINEAR_BACKWARD, LA_OP_CAUSAL_FORWARD, LA_OP_CAUSAL_BACKWARD = 0, 1, 2, 3
 LA_OP_CAUSAL_SAVED = 4
 LA_OP_LINEAR_VARLEN_FORWARD, LA_OP_LINEAR_VARLEN_BACKWARD = 5, 6
+LA_OP_LINEAR_SAVED = 7
 _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
     "la_feature_map", "la_feature_map_poly2", "la_feature_map_poly2_backward",
     "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
     "la_linear_attention_varlen", "la_linear_attention_varlen_backward",
+    "la_linear_attention_keep", "la_linear_attention_backward_kept",
     "la_causal_forward", "la_causal_forward_from", "la_causal_backward_from",
     "la_causal_backward", "la_recurrent_step", "la_recurrent_steps", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
@@ -65,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.la_linear_attention_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
         L.la_linear_attention_varlen.argtypes = [pp] + [vp] * 8 + [vp, sz, vp]
         L.la_linear_attention_varlen_backward.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
+        L.la_linear_attention_keep.argtypes = [pp] + [vp] * 8 + [vp, sz, vp, sz, vp]
+        L.la_linear_attention_backward_kept.argtypes = [pp] + [vp] * 4 + [vp, sz] + [vp] * 6 + [vp, sz, vp]
         L.la_causal_forward.argtypes = [pp] + [vp] * 7 + [vp, sz] + [vp, sz, vp]
         L.la_causal_forward_from.argtypes = [pp] + [vp] * 9 + [vp, sz] + [vp, sz, vp]
         L.la_causal_backward_from.argtypes = [pp] + [vp] * 10 + [vp, sz] + [vp] * 5 + [vp, sz, vp]
@@ -238,11 +242,28 @@ def la_feature_map_poly2_backward(x: torch.Tensor, dy: torch.Tensor, out: torch.
     return dx
 
 
-def la_linear_attention(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, KV=None, Zs=None, ws=None):
-    """Non-causal form.  Returns O; pass preallocated den / KV / Zs tensors to receive them."""
-    dev = _dev(Q, K, V, O, den, KV, Zs)
+def linear_saved_buffer(Q, V, phi="elu1", eps=0.0):
+    """A buffer for what la_linear_attention() keeps for la_linear_attention_backward() (per-split sums over the keys)."""
+    p = _problem_of(Q, V, phi, eps)
+    need = lib().la_workspace_bytes(ctypes.byref(p), LA_OP_LINEAR_SAVED)
+    return None if need == 0 else torch.empty(need, dtype=torch.uint8, device=Q.device)
+
+
+def la_linear_attention(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, KV=None, Zs=None, ws=None, saved=None,
+                        lengths=None):
+    """Non-causal form.  Returns O; pass preallocated den / KV / Zs tensors to receive them, and a
+    linear_saved_buffer() to keep the sums over the keys for the backward pass (la_linear_attention_keep;
+    lengths: optional [B] int32 device tensor of a right-padded ragged batch)."""
+    dev = _dev(Q, K, V, O, den, KV, Zs, saved, lengths)
     p = _problem_of(Q, V, phi, eps)
     O = torch.empty_like(V) if O is None else O
+    if saved is not None:
+        _check(lib().la_linear_attention_keep(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(O), _ptr(den),
+                                              _ptr(KV), _ptr(Zs), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws),
+                                              _stream(dev)))
+        return O
+    if lengths is not None:
+        return la_linear_attention_varlen(Q, K, V, lengths, phi, eps, O, den, KV, Zs, ws)
     ws = workspace(p, LA_OP_LINEAR_FORWARD, dev) if ws is None else ws
     _check(lib().la_linear_attention(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(KV),
                                      _ptr(Zs), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
@@ -265,13 +286,22 @@ def la_linear_attention_noalloc(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, 
 
 
 def la_linear_attention_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None,
-                                 dQ=None, dK=None, dV=None, ws=None):
-    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV)
+                                 dQ=None, dK=None, dV=None, ws=None, saved=None, lengths=None):
+    """Gradients of the non-causal form.  saved: what la_linear_attention(..., saved=...) kept for the same
+    problem (la_linear_attention_backward_kept); lengths as there.  Returns (dQ, dK, dV)."""
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved, lengths)
     p = _problem_of(Q, V, phi, eps)
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(V) if dV is None else dV
+    if saved is None and lengths is not None:
+        return la_linear_attention_varlen_backward(Q, K, V, G, lengths, phi, eps, O, den, dQ, dK, dV, ws)
     ws = workspace(p, LA_OP_LINEAR_BACKWARD, dev) if ws is None else ws
+    if saved is not None:
+        _check(lib().la_linear_attention_backward_kept(
+            ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(saved), _nbytes(saved), _ptr(O), _ptr(den),
+            _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), _nbytes(ws), _stream(dev)))
+        return dQ, dK, dV
     _check(lib().la_linear_attention_backward(
         ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV),
         _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(dev)))

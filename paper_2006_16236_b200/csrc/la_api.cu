@@ -174,8 +174,9 @@ const char* la_profile_kernel_name(int kernel) {
 
 size_t la_workspace_bytes(const la_problem* p, int32_t op) {
     if (!p || p->B < 1 || p->H < 1 || p->N < 0 || p->D < 1 || p->M < 1 || p->D > 128 || p->M > 128) return 0;
-    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_LINEAR_VARLEN_BACKWARD) return 0;
+    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_LINEAR_SAVED) return 0;
     if (p->N == 0) return 0;
+    if (op == LA_OP_LINEAR_SAVED) op = LA_OP_LINEAR_FORWARD;          // the saved buffer holds what the forward's workspace holds
     if (op == LA_OP_CAUSAL_SAVED) return tc_supported(*p, LA_OP_CAUSAL_BACKWARD) ? tc_causal_saved_bytes(*p) : 0;
     if (op == LA_OP_LINEAR_VARLEN_FORWARD || op == LA_OP_LINEAR_VARLEN_BACKWARD) {
         const int full = op == LA_OP_LINEAR_VARLEN_FORWARD ? LA_OP_LINEAR_FORWARD : LA_OP_LINEAR_BACKWARD;
@@ -231,51 +232,79 @@ int la_feature_map_poly2_backward(const void* x, const void* dy, void* dx, int64
     return launch_poly2_map_backward(x, dy, dx, rows, (int)D, (int)C, dtype, (cudaStream_t)stream);
 }
 
-int la_linear_attention(const la_problem* p, const void* Q, const void* K, const void* V,
-                        void* O, float* den, float* KV, float* Zs,
-                        void* ws, size_t ws_bytes, void* stream) {
+// The optional buffer in which the non-causal forward keeps its per-split sums for the backward pass.
+static int check_linear_saved(const la_problem* p, const void* saved, size_t saved_bytes) {
+    if (!saved) return LA_OK;
+    if (!aligned16(saved)) return fail(LA_ERR_INVALID_ARG, "saved is not 16-byte aligned");
+    const size_t need = la_workspace_bytes(p, LA_OP_LINEAR_SAVED);
+    if (saved_bytes < need)
+        return fail(LA_ERR_WORKSPACE, "saved buffer too small: %zu bytes given, %zu needed", saved_bytes, need);
+    return LA_OK;
+}
+
+// All non-causal forward entry points: `lengths` given (ragged batch) or not, `saved` given or not.
+static int linear_forward_common(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
+                                 bool ragged, void* O, float* den, float* KV, float* Zs, void* saved, size_t saved_bytes,
+                                 void* ws, size_t ws_bytes, void* stream) {
     if (int rc = check_problem(p, true)) return rc;
     if (p->N == 0) return LA_OK;
     LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(O);
+    if (ragged && !lengths) return fail(LA_ERR_INVALID_ARG, "lengths is NULL");
+    if (reinterpret_cast<uintptr_t>(lengths) & 3u) return fail(LA_ERR_INVALID_ARG, "lengths is not 4-byte aligned");
     LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(KV); LA_OPTIONAL_PTR(Zs);
-    if (int rc = check_ws(p, LA_OP_LINEAR_FORWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_linear_saved(p, saved, saved_bytes)) return rc;
+    if (!saved)         // with a saved buffer the sums go there and the workspace is not touched
+        if (int rc = check_ws(p, lengths ? LA_OP_LINEAR_VARLEN_FORWARD : LA_OP_LINEAR_FORWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc_linear_forward(*p, Q, K, V, nullptr, O, den, KV, Zs, ws, st);
-    return general_linear_forward(*p, Q, K, V, nullptr, O, den, KV, Zs, ws, st);
+    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
+    return general_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
+}
+
+static int linear_backward_common(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
+                                  bool ragged, const void* saved, size_t saved_bytes, const void* O, const float* den,
+                                  const void* G, void* dQ, void* dK, void* dV, void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_problem(p, true)) return rc;
+    if (p->N == 0) return LA_OK;
+    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(G);
+    LA_REQUIRE_PTR(dQ); LA_REQUIRE_PTR(dK); LA_REQUIRE_PTR(dV);
+    if (ragged && !lengths) return fail(LA_ERR_INVALID_ARG, "lengths is NULL");
+    if (reinterpret_cast<uintptr_t>(lengths) & 3u) return fail(LA_ERR_INVALID_ARG, "lengths is not 4-byte aligned");
+    LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den);
+    if (int rc = check_linear_saved(p, saved, saved_bytes)) return rc;
+    if (int rc = check_ws(p, lengths ? LA_OP_LINEAR_VARLEN_BACKWARD : LA_OP_LINEAR_BACKWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_arch()) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc_linear_backward(*p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
+    return general_linear_backward(*p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
+}
+
+int la_linear_attention(const la_problem* p, const void* Q, const void* K, const void* V,
+                        void* O, float* den, float* KV, float* Zs,
+                        void* ws, size_t ws_bytes, void* stream) {
+    return linear_forward_common(p, Q, K, V, nullptr, false, O, den, KV, Zs, nullptr, 0, ws, ws_bytes, stream);
 }
 
 int la_linear_attention_varlen(const la_problem* p, const void* Q, const void* K, const void* V,
                                const int32_t* lengths,
                                void* O, float* den, float* KV, float* Zs,
                                void* ws, size_t ws_bytes, void* stream) {
-    if (int rc = check_problem(p, true)) return rc;
-    if (p->N == 0) return LA_OK;
-    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(O);
-    if (!lengths) return fail(LA_ERR_INVALID_ARG, "lengths is NULL");
-    if (reinterpret_cast<uintptr_t>(lengths) & 3u) return fail(LA_ERR_INVALID_ARG, "lengths is not 4-byte aligned");
-    LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(KV); LA_OPTIONAL_PTR(Zs);
-    if (int rc = check_ws(p, LA_OP_LINEAR_VARLEN_FORWARD, ws, ws_bytes)) return rc;
-    if (int rc = check_arch()) return rc;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, ws, st);
-    return general_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, ws, st);
+    return linear_forward_common(p, Q, K, V, lengths, true, O, den, KV, Zs, nullptr, 0, ws, ws_bytes, stream);
+}
+
+int la_linear_attention_keep(const la_problem* p, const void* Q, const void* K, const void* V,
+                             const int32_t* lengths,
+                             void* O, float* den, float* KV, float* Zs,
+                             void* saved, size_t saved_bytes,
+                             void* ws, size_t ws_bytes, void* stream) {
+    return linear_forward_common(p, Q, K, V, lengths, false, O, den, KV, Zs, saved, saved_bytes, ws, ws_bytes, stream);
 }
 
 int la_linear_attention_backward(const la_problem* p, const void* Q, const void* K, const void* V,
                                  const void* O, const float* den, const void* G,
                                  void* dQ, void* dK, void* dV,
                                  void* ws, size_t ws_bytes, void* stream) {
-    if (int rc = check_problem(p, true)) return rc;
-    if (p->N == 0) return LA_OK;
-    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(G);
-    LA_REQUIRE_PTR(dQ); LA_REQUIRE_PTR(dK); LA_REQUIRE_PTR(dV);
-    LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den);
-    if (int rc = check_ws(p, LA_OP_LINEAR_BACKWARD, ws, ws_bytes)) return rc;
-    if (int rc = check_arch()) return rc;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc_linear_backward(*p, Q, K, V, nullptr, G, dQ, dK, dV, ws, st);
-    return general_linear_backward(*p, Q, K, V, nullptr, G, dQ, dK, dV, ws, st);
+    return linear_backward_common(p, Q, K, V, nullptr, false, nullptr, 0, O, den, G, dQ, dK, dV, ws, ws_bytes, stream);
 }
 
 int la_linear_attention_varlen_backward(const la_problem* p, const void* Q, const void* K, const void* V,
@@ -283,18 +312,16 @@ int la_linear_attention_varlen_backward(const la_problem* p, const void* Q, cons
                                         const void* O, const float* den, const void* G,
                                         void* dQ, void* dK, void* dV,
                                         void* ws, size_t ws_bytes, void* stream) {
-    if (int rc = check_problem(p, true)) return rc;
-    if (p->N == 0) return LA_OK;
-    LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(G);
-    LA_REQUIRE_PTR(dQ); LA_REQUIRE_PTR(dK); LA_REQUIRE_PTR(dV);
-    if (!lengths) return fail(LA_ERR_INVALID_ARG, "lengths is NULL");
-    if (reinterpret_cast<uintptr_t>(lengths) & 3u) return fail(LA_ERR_INVALID_ARG, "lengths is not 4-byte aligned");
-    LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den);
-    if (int rc = check_ws(p, LA_OP_LINEAR_VARLEN_BACKWARD, ws, ws_bytes)) return rc;
-    if (int rc = check_arch()) return rc;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc_linear_backward(*p, Q, K, V, lengths, G, dQ, dK, dV, ws, st);
-    return general_linear_backward(*p, Q, K, V, lengths, G, dQ, dK, dV, ws, st);
+    return linear_backward_common(p, Q, K, V, lengths, true, nullptr, 0, O, den, G, dQ, dK, dV, ws, ws_bytes, stream);
+}
+
+int la_linear_attention_backward_kept(const la_problem* p, const void* Q, const void* K, const void* V,
+                                      const int32_t* lengths,
+                                      const void* saved, size_t saved_bytes,
+                                      const void* O, const float* den, const void* G,
+                                      void* dQ, void* dK, void* dV,
+                                      void* ws, size_t ws_bytes, void* stream) {
+    return linear_backward_common(p, Q, K, V, lengths, false, saved, saved_bytes, O, den, G, dQ, dK, dV, ws, ws_bytes, stream);
 }
 
 static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {

@@ -98,10 +98,11 @@ int general_causal_forward(const la_problem& p, const void* Q, const void* K, co
 int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V,
                             const void* G, const StateArgs& sa, void* dQ, void* dK, void* dV, void* ws,
                             cudaStream_t st);
-// lengths ([B] int32, device, or null): real positions per batch element (the rest is padding)
+// lengths ([B] int32, device, or null): real positions per batch element (the rest is padding);
+// saved (or null): where the forward leaves its per-split sums and the backward finds them
 int general_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                           void* O, float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
+                           void* O, float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st);
 int general_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                            const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+                            const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 
 }  // namespace la

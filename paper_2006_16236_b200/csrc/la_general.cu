@@ -680,11 +680,11 @@ int general_causal_backward(const la_problem& p, const void* Q, const void* K, c
 
 template <typename IO>
 static int linear_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                            void* O, float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
+                            void* O, float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st) {
     const int D = (int)p.D, M = (int)p.M;
     const Split sp = choose_split(p);
     const dim3 grid((unsigned)(p.B * p.H), (unsigned)sp.nsplit);
-    float* part = (float*)ws;
+    float* part = saved ? (float*)saved : (float*)ws;        // the per-split sums, kept for the backward pass if asked
     {
         const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
         auto kern = D == 64 && M == 64 ? general_kv_sum_kernel<IO, 64> : general_kv_sum_kernel<IO, 0>;
@@ -704,20 +704,22 @@ static int linear_forward_t(const la_problem& p, const void* Q, const void* K, c
 }
 
 int general_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                           void* O, float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
-    return p.dtype == LA_F32 ? linear_forward_t<float>(p, Q, K, V, lengths, O, den, KV, Zs, ws, st)
-                             : linear_forward_t<__nv_bfloat16>(p, Q, K, V, lengths, O, den, KV, Zs, ws, st);
+                           void* O, float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st) {
+    return p.dtype == LA_F32 ? linear_forward_t<float>(p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st)
+                             : linear_forward_t<__nv_bfloat16>(p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
 }
 
 template <typename IO>
 static int linear_backward_t(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                             const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+                             const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
     const int D = (int)p.D, M = (int)p.M;
     const Split sp = choose_split(p);
     const dim3 grid((unsigned)(p.B * p.H), (unsigned)sp.nsplit);
     float* part_s = (float*)ws;
     float* part_r = part_s + (size_t)(p.B * p.H) * sp.nsplit * state_floats(p);
-    {
+    if (saved) {
+        part_s = (float*)saved;           // the forward's own sums: nothing to recompute
+    } else {
         const size_t smem = ((size_t)T * (D + 1) + (size_t)T * (M + 1) + state_floats(p)) * sizeof(float);
         auto kern = D == 64 && M == 64 ? general_kv_sum_kernel<IO, 64> : general_kv_sum_kernel<IO, 0>;
         if (int rc = opt_in_smem(kern, smem)) return rc;
@@ -744,9 +746,9 @@ static int linear_backward_t(const la_problem& p, const void* Q, const void* K, 
 }
 
 int general_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                            const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
-    return p.dtype == LA_F32 ? linear_backward_t<float>(p, Q, K, V, lengths, G, dQ, dK, dV, ws, st)
-                             : linear_backward_t<__nv_bfloat16>(p, Q, K, V, lengths, G, dQ, dK, dV, ws, st);
+                            const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    return p.dtype == LA_F32 ? linear_backward_t<float>(p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st)
+                             : linear_backward_t<__nv_bfloat16>(p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
 }
 
 }  // namespace la

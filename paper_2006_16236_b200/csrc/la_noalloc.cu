@@ -83,5 +83,5 @@ extern "C" int la_linear_attention_noalloc(const la_problem* p, const void* Q, c
     if (int rc = scratch_for_current_device(&scratch)) return rc;
     // Every partial sum the second kernel reads is written by the first one in the same call,
     // so nothing in the array has to start at zero.
-    return general_linear_forward(*p, Q, K, V, nullptr, O, den, KV, Zs, scratch, (cudaStream_t)stream);
+    return general_linear_forward(*p, Q, K, V, nullptr, O, den, KV, Zs, nullptr, scratch, (cudaStream_t)stream);
 }

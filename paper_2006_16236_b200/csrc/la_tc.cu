@@ -79,12 +79,12 @@ int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const 
     return tc::causal_backward(p, Q, K, V, G, sa, saved, dQ, dK, dV, ws, st);
 }
 int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, void* O,
-                      float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
-    return tc::linear_forward(p, Q, K, V, lengths, O, den, KV, Zs, ws, st);
+                      float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st) {
+    return tc::linear_forward(p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
 }
 int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                       const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
-    return tc::linear_backward(p, Q, K, V, lengths, G, dQ, dK, dV, ws, st);
+                       const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    return tc::linear_backward(p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
 }
 
 }  // namespace la

@@ -18,10 +18,11 @@ int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const 
                        const float* den, const void* G, const StateArgs& sa, const void* saved, void* dQ, void* dK,
                        void* dV, void* ws, cudaStream_t st);
 // lengths ([B] int32, device, or null): real positions per batch element of a right-padded ragged batch
+// saved (or null): where the forward leaves its per-split sums and the backward finds them
 int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, void* O,
-                      float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
+                      float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st);
 int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                       const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+                       const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 
 namespace tc {
 size_t causal_forward_workspace(const la_problem& p);
@@ -35,9 +36,9 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
 size_t linear_forward_workspace(const la_problem& p);
 size_t linear_backward_workspace(const la_problem& p);
 int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, void* O,
-                   float* den, float* KV, float* Zs, void* ws, cudaStream_t st);
+                   float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st);
 int linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                    const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+                    const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 }  // namespace tc
 
 }  // namespace la

@@ -828,14 +828,14 @@ size_t linear_backward_workspace(const la_problem& p) {
 }
 
 int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, void* O,
-                   float* den, float* KV, float* Zs, void* ws, cudaStream_t st) {
+                   float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st) {
     const Segmentation sg = choose_splits(p);
     const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
     CUtensorMap mQ, mK, mV;
     if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
     if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
     if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
-    float* rec = (float*)ws;
+    float* rec = saved ? (float*)saved : (float*)ws;      // the split records, kept for the backward pass if asked
     if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, lengths, rec, st)) return rc;
     ApParams a = {};
     a.lengths = lengths;
@@ -848,7 +848,7 @@ int linear_forward(const la_problem& p, const void* Q, const void* K, const void
 }
 
 int linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                    const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+                    const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
     const Segmentation sg = choose_splits(p);
     const size_t bh = (size_t)(p.B * p.H);
     const uint64_t rows = (uint64_t)(bh * p.N);
@@ -863,7 +863,8 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
     float* dn = (float*)w;      w += bh * (size_t)p.N * sizeof(float);
     float* dl = (float*)w;
 
-    if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, lengths, rec_s, st)) return rc;
+    if (saved) rec_s = (float*)saved;         // the forward's own records: nothing to recompute
+    else if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, lengths, rec_s, st)) return rc;
     ApParams a = {};
     a.lengths = lengths;
     a.records = rec_s;

@@ -575,6 +575,30 @@ def test_noncausal_workload_full_size():
             assert_close(got[sl], ref, dtype, f"d{nm}[{b},{h}]", grad=True)
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape,lengths", [((2, 3, 512, 64, 64), None), ((3, 2, 1024, 64, 64), [1024, 130, 700]),
+                                           ((2, 2, 200, 16, 24), None), ((2, 2, 200, 16, 24), [200, 77])])
+def test_noncausal_saved_sums_give_identical_results(shape, lengths, dtype):
+    """What the non-causal forward keeps for the backward pass (the per-split sums over the keys) changes no bit
+    of either call's results, on the tensor-core and on the general kernels, full-length and ragged; and the
+    forward leaves its workspace alone when it is given a saved buffer."""
+    B, H, N, D, M = shape
+    Q, K, V, G = gpu(*draw_qkvg(B, H, N, D, M, seed=sum(shape) + 9, dtype=dtype))
+    ld = None if lengths is None else torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    saved = la.linear_saved_buffer(Q, V)
+    assert saved is not None and saved.numel() > 0
+    O0 = la.la_linear_attention(Q, K, V, lengths=ld)
+    g0 = la.la_linear_attention_backward(Q, K, V, G, lengths=ld)
+    saved.fill_(0xFF)
+    O1 = la.la_linear_attention(Q, K, V, lengths=ld, saved=saved)
+    assert int((saved != 0xFF).sum()) > 0
+    g1 = la.la_linear_attention_backward(Q, K, V, G, lengths=ld, saved=saved)
+    la.la_last_device_status()
+    assert torch.equal(O0, O1)
+    for a, b, nm in zip(g0, g1, "QKV"):
+        assert torch.equal(a, b), f"d{nm} differs with the saved sums"
+
+
 def test_noncausal_ragged_workload_full_size():
     """The speech-shaped workload as a ragged batch (the paper's speech batches are: mean 800, max 2400
     frames): lengths between a third of N and N, one full and one of a single chunk plus one position."""

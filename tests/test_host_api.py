@@ -166,6 +166,18 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert L.la_linear_attention_varlen(ctypes.byref(pv), ok, ok, ok, ok, ok, null, null, null, null, 0, null) == -3
     assert L.la_linear_attention_varlen_backward(ctypes.byref(pv), ok, ok, ok, null, null, null, ok, ok, ok, ok,
                                                  big, 1 << 40, null) == -1
+    # the non-causal saved buffer: optional, 16-byte aligned, large enough; with it the forward needs no workspace
+    need_s = la.la_workspace_bytes(pv, binding.LA_OP_LINEAR_SAVED)
+    assert need_s == la.la_workspace_bytes(pv, binding.LA_OP_LINEAR_FORWARD) > 0
+    keep = lambda saved, nbytes, ws=null, wsb=0: L.la_linear_attention_keep(ctypes.byref(pv), ok, ok, ok, null, ok, null, null,
+                                                                          null, saved, nbytes, ws, wsb, null)
+    assert keep(odd, 1 << 40) == -1 and b"saved" in L.la_last_error()
+    assert keep(ok, need_s - 1) == -3
+    assert keep(null, 0) == -3                                          # no saved buffer: the workspace is required
+    assert L.la_linear_attention_backward_kept(ctypes.byref(pv), ok, ok, ok, null, ok, need_s - 1, null, null, ok, ok, ok, ok,
+                                               big, 1 << 40, null) == -3
+    assert L.la_linear_attention_backward_kept(ctypes.byref(pv), ok, ok, ok, null, ok, need_s, null, null, ok, ok, ok, ok,
+                                               null, 0, null) == -3     # the backward still needs its workspace
     assert L.la_feature_map(ok, ok, -5, 0, 0, null) == -1
     assert L.la_feature_map(ok, ok, 0, 0, 0, null) == 0
     assert L.la_feature_map(ok, ok, 4, 9, 0, null) == -1
