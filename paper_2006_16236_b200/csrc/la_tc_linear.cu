@@ -311,11 +311,17 @@ constexpr uint32_t kApOffVec = kApOffState + kDim * 128;              // fp32 [3
 constexpr uint32_t kApOffBar = kApOffVec + 1024;
 constexpr uint32_t kApOffOut = (kApOffBar + 256 + 1023) & ~1023u;      // two result tiles on their way out
 constexpr uint32_t kApOffX = kApOffOut + 2 * kTileBytes;               // fp32 [2 halves][128 rows][8]: partial sums exchanged
-constexpr uint32_t kApSmemBytes = kApOffX + 2 * 128 * 8 * 4 + 1024;    // + slack for the 1 KB alignment of the base
+// backward Q only: the chunk's weighted queries x' / dn and its aux tile (columns 0..15: dl_i, 16..23: 1 / dn_i),
+// operands of the reverse sums that this pass forms on the side (see the sum kernel for the product)
+constexpr uint32_t kApOffXS = kApOffX + 2 * 128 * 8 * 4;
+constexpr uint32_t kApOffAux = kApOffXS + kTileBytes;
+constexpr uint32_t kApSmemBytes = kApOffAux + kTileBytes + 1024;       // + slack for the 1 KB alignment of the base
+constexpr uint32_t kApColSums = 256;                                   // TMEM columns of the reverse sums (80)
 
 struct ApBarriers {
     uint64_t full[kApStages], empty[kApStages], mapped[kApStages];
     uint64_t acc_full[2], acc_free[2];
+    uint64_t xs_ready, xs_free, sums_done;      // backward Q: hand-offs of the weighted tile and the end of the reverse sums
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -324,8 +330,8 @@ struct ApParams {
     const float* records;       // [BH][nseg][kRecFloats]: summed by every CTA
     __nv_bfloat16* out0;        // forward: O;  backward Q: dQ;  backward K/V: dK
     __nv_bfloat16* out1;        // backward K/V: dV
-    float* den;                 // forward: q.Z (optional);  backward Q: dn_i (out)
-    float* dl;                  // backward Q: dl_i (out)
+    float* den;                 // forward: q.Z (optional)
+    float* rec_out;             // backward Q: [BH][nseg][kRecFloats] reverse sums of this pass's rows (out)
     float* state_out;           // forward: KV [BH][64][64] (optional)
     float* vec_out;             // forward: Zs [BH][64] (optional)
     const int* lengths;         // [B] real positions per batch element (right-padded ragged batch), or null
@@ -364,19 +370,23 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     if (tid == 0) {
         for (int s = 0; s < kApStages; ++s) {
             mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], 1 + 256);      // MMA commit + epilogue threads (they read the X and Y rows)
+            // MMA commit + epilogue threads (they read the X and Y rows) (+ the commit of the reverse sums, which read Y)
+            mbar_init(&bars->empty[s], 1 + 256 + (kMode == kApplyBackwardQ ? 1 : 0));
             mbar_init(&bars->mapped[s], 128);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&bars->acc_full[b], 1);
             mbar_init(&bars->acc_free[b], 256);
         }
+        mbar_init(&bars->xs_ready, 256);
+        mbar_init(&bars->xs_free, 1);
+        mbar_init(&bars->sums_done, 1);
         bars->abort_flag = 0;
         fence_mbar_init();
     }
     if (warp == 9) {
         __syncwarp();
-        tmem_alloc(&bars->tmem_base, 256);
+        tmem_alloc(&bars->tmem_base, 512);
         tmem_relinquish();
     }
     __syncthreads();            // the barriers are initialised for the loads issued before the prologue below
@@ -498,6 +508,23 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
             const uint32_t aSt = sbase + kApOffState;
             bool ok = true;
+            // backward Q: the reverse sums of chunk c, [A' | a'] += (x' / dn)^T [G | dl] and (row 80) the sums weighted by
+            // 1 / dn, once the epilogue threads have written the weighted tile: one M = 128, N = 80 product per K
+            // group, A = [XS | aux], B = [G | aux] (second blocks through the leading-offset field)
+            auto issue_sums = [&](int c) -> bool {
+                if (!mbar_wait(&bars->xs_ready, c & 1, prm.status, kStatusPipeTimeout) || *abort_flag) return false;
+                tc_fence_after_sync();
+                const uint32_t idesc = umma_idesc_bf16(128, 80, 1, 1);
+                const uint32_t aXS = sbase + kApOffXS, aAux = sbase + kApOffAux;
+                const uint32_t aG = sbase + kApOffStage + (c % kApStages) * 2 * kTileBytes + kTileBytes;
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16(tmem + kApColSums, desc_mn(aXS + k * 2048, aAux - aXS), desc_mn(aG + k * 2048, aAux - aG), idesc,
+                              (c | k) != 0);
+                umma_commit(&bars->empty[c % kApStages]);
+                umma_commit(&bars->xs_free);
+                return true;
+            };
             #pragma unroll 1
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kApStages, b = c & 1;
@@ -521,7 +548,10 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 }
                 umma_commit(&bars->acc_full[b]);
                 umma_commit(&bars->empty[s]);
+                if (kMode == kApplyBackwardQ && c >= 1) ok = issue_sums(c - 1);
             }
+            if (kMode == kApplyBackwardQ && ok && L >= 1) ok = issue_sums(L - 1);
+            if (kMode == kApplyBackwardQ) umma_commit(&bars->sums_done);
             if (!ok) *abort_flag = 1;
         }
     } else if (warp >= 4 && warp < 8) {
@@ -656,10 +686,30 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     const float dl = -q_h * scale;                                // dl_i = -(G_i . O_i)
                     c1 = fmaf(dl, fN, ynu);                                       // (G.nu) + dl N
                     cz = dl;
+                    // operands of the reverse sums: the weighted queries x' / dn, and [dl_i | 1 / dn_i] in the aux tile
+                    // (rows behind the sequence's end: zeros, also in the G tile, whatever it holds there)
+                    if (c > 0 && !mbar_wait(&bars->xs_free, (c - 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
+                    const float wq = padded ? 0.f : scale, dq = padded ? 0.f : dl;
+                    uint8_t* xs_row = smem + kApOffXS + t * 128;
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc)
+                        sts128(xs_row + (((hf * 4 + cc) ^ r7) << 4),
+                               pack_bf16x2(bf16_lo(xv[cc][0]) * wq, bf16_hi(xv[cc][0]) * wq), pack_bf16x2(bf16_lo(xv[cc][1]) * wq, bf16_hi(xv[cc][1]) * wq),
+                               pack_bf16x2(bf16_lo(xv[cc][2]) * wq, bf16_hi(xv[cc][2]) * wq), pack_bf16x2(bf16_lo(xv[cc][3]) * wq, bf16_hi(xv[cc][3]) * wq));
                     if (hf == 0) {
-                        prm.den[row] = dn;
-                        prm.dl[row] = dl;
+                        uint8_t* aux_row = smem + kApOffAux + t * 128;
+                        const uint32_t dd = pack_bf16x2(dq, dq), ww = pack_bf16x2(wq, wq);
+                        sts128(aux_row + ((0 ^ r7) << 4), dd, dd, dd, dd);
+                        sts128(aux_row + ((1 ^ r7) << 4), dd, dd, dd, dd);
+                        sts128(aux_row + ((2 ^ r7) << 4), ww, ww, ww, ww);
                     }
+                    if (padded) {
+                        uint8_t* g_row = smem + kApOffStage + s * 2 * kTileBytes + kTileBytes + t * 128;
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) sts128(g_row + ((hf * 4 + cc) << 4), 0u, 0u, 0u, 0u);
+                    }
+                    fence_proxy_async_smem();
+                    mbar_arrive(&bars->xs_ready);
                 } else {
                     c1 = ynu + sScal[1];
                     cz = 1.f;
@@ -717,6 +767,30 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         }
         if (hf == 0 && lane == 0) tma_store_wait_all<0>();
         LA_TRACE_CTA(g_trace_lin, 6);
+        if (kMode == kApplyBackwardQ && warp < 3) {
+            // this split's record of the reverse sums: accumulator rows 0..63 (warps 0, 1) and row 80 (warp 2, lane 16),
+            // zeros if the split holds no real row
+            const bool ok = mbar_wait(&bars->sums_done, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
+            tc_fence_after_sync();
+            float* rec = prm.rec_out + (bh * prm.nseg + seg) * (int64_t)kRecFloats;
+            const int d_row = warp * 32 + lane;
+            const bool mine = ok && (warp < 2 || lane == 16);
+            float* dst = warp < 2 ? rec + d_row * kDim : rec + kDim * kDim + kDim;
+            for (int h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_base + kApColSums + h * 32, v);
+                tmem_ld_wait();
+                if (mine)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) dst[h * 32 + j] = L > 0 ? __uint_as_float(v[j]) : 0.f;
+            }
+            const float z = __uint_as_float(tmem_ld1(tmem + lane_base + kApColSums + 64));
+            tmem_ld_wait();
+            if (mine) {
+                if (warp < 2) rec[kDim * kDim + d_row] = L > 0 ? z : 0.f;
+                else rec[kDim * kDim + 2 * kDim] = L > 0 ? z : 0.f;
+            }
+        }
         if (L < L_all) {            // whole chunks of padding: zeros, written directly
             const int e = hf * 128 + t;
             const int64_t r_lo = row0 + (int64_t)L * kChunk, nrows = (int64_t)(L_all - L) * kChunk;
@@ -737,7 +811,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     LA_TRACE_CTA(g_trace_lin, 7);
     if (warp == 9) {
         __syncwarp();
-        tmem_dealloc(tmem, 256);
+        tmem_dealloc(tmem, 512);
     }
 }
 
@@ -824,7 +898,7 @@ size_t linear_forward_workspace(const la_problem& p) {
 }
 
 size_t linear_backward_workspace(const la_problem& p) {
-    return 2 * linear_forward_workspace(p) + 2 * (size_t)(p.B * p.H) * (size_t)p.N * sizeof(float);
+    return 2 * linear_forward_workspace(p);
 }
 
 int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, void* O,
@@ -860,8 +934,6 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
     uint8_t* w = (uint8_t*)ws;
     float* rec_s = (float*)w;   w += bh * sg.nseg * kRecFloats * sizeof(float);
     float* rec_r = (float*)w;   w += bh * sg.nseg * kRecFloats * sizeof(float);
-    float* dn = (float*)w;      w += bh * (size_t)p.N * sizeof(float);
-    float* dl = (float*)w;
 
     if (saved) rec_s = (float*)saved;         // the forward's own records: nothing to recompute
     else if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, lengths, rec_s, st)) return rc;
@@ -869,10 +941,8 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.lengths = lengths;
     a.records = rec_s;
     a.out0 = (__nv_bfloat16*)dQ;
-    a.den = dn;
-    a.dl = dl;
+    a.rec_out = rec_r;          // the reverse sums of Q / dn and G are formed by the same pass
     if (int rc = launch_apply<kApplyBackwardQ>(p, sg, mQ, mG, a, st)) return rc;
-    if (int rc = launch_sums(p, sg, mQ, mG, dn, dl, lengths, rec_r, st)) return rc;
     ApParams b = {};
     b.lengths = lengths;
     b.records = rec_r;
