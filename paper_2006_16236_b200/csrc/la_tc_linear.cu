@@ -38,8 +38,8 @@ LA_TRACE_DECL(g_trace_lin)
 namespace {
 
 // Record of one split: [A' (64x64) | a' (64) | ysum (64) | w0 (1) | pad]:
-//   forward sums : A' = sum k'_j V_j^T, a' = sum k'_j, ysum = sum V_j,        w0 unused
-//   reverse sums : A' = sum qh'_i G_i^T, a' = sum qh'_i dl_i, ysum = sum G_i / dn_i, w0 = sum dl_i / dn_i
+//   forward sums (sum kernel)            : A' = sum k'_j V_j^T, a' = sum k'_j, ysum = sum V_j,        w0 unused
+//   reverse sums (backward-Q apply pass) : A' = sum qh'_i G_i^T, a' = sum qh'_i dl_i, ysum = sum G_i / dn_i, w0 = sum dl_i / dn_i
 constexpr int kRecFloats = kDim * kDim + kDim + kDim + 8;
 
 __device__ __forceinline__ float elu_fast(float x) {      // elu(x) = phi(x) - 1
@@ -87,11 +87,13 @@ __device__ __forceinline__ void elu_half_row_inplace(uint8_t* row, uint32_t r7, 
 // each), aux tile, final read-out (warps 0-2); warp 8: TMA; warp 9: MMA.
 // ===========================================================================
 constexpr int kLsThreads = 320;
-// Four stages: a tile arrives about 2400 cycles after its load is issued, against about 1000 cycles of mapping
-// and 600 of MMA issue per chunk, so the ring has to hold the loads of three chunks ahead.
-constexpr int kLsStages = 4;
-constexpr uint32_t kLsStageBytes = 3 * kTileBytes;                  // X, Y, aux (columns 0..15: dl_i, 16..23: w_i)
-constexpr uint32_t kLsOffBar = kLsStages * kLsStageBytes;
+// Six stages of {X, Y}: a tile arrives 2400-4000 cycles after its load is issued, against about 1000 cycles of
+// mapping and 600 of MMA issue per chunk, so the ring has to hold the loads of several chunks ahead.  One aux
+// tile (constant ones) serves every stage.
+constexpr int kLsStages = 6;
+constexpr uint32_t kLsStageBytes = 2 * kTileBytes;                  // X, Y
+constexpr uint32_t kLsOffAux = kLsStages * kLsStageBytes;           // [128][64] ones: second block of both operands
+constexpr uint32_t kLsOffBar = kLsOffAux + kTileBytes;
 constexpr uint32_t kLsSmemBytes = kLsOffBar + 256 + 1024;
 
 struct LsBarriers {
@@ -103,8 +105,6 @@ struct LsBarriers {
 
 struct LsParams {
     float* records;        // [BH][nseg][kRecFloats]
-    const float* dn;       // null: forward sums (w_i = 1, aux = 1); else w_i = 1 / dn_i, aux = dl_i
-    const float* dl;
     const int* lengths;    // [B] real positions per batch element (right-padded ragged batch), or null
     int heads;
     int* status;
@@ -127,7 +127,6 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const int c_begin = seg * prm.chunks_per_seg;
     const int L_all = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
-    const bool reverse = prm.dn != nullptr;
     LA_TRACE_CTA(g_trace_lin, 0);
 
     if (tid == 0) {
@@ -145,14 +144,10 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         tmem_alloc(&bars->tmem_base, 256);
         tmem_relinquish();
     }
-    // The aux tile of a stage is the second 64-column block of both operands: of B = [Y | aux] (N = 80: its
-    // columns 0..15, dl_i, are read) and of A = [X | aux] (M = 128: accumulator row 64 + m is the sum weighted by
-    // column m; row 80, weighted by w_i in column 16, is the one read out; columns 24.. are never written and
-    // feed rows nobody reads).  Without per-position weights the tile is constant ones: written once here.
-    if (!reverse)
-        for (int s = 0; s < kLsStages; ++s)
-            for (int i = tid; i < kTileBytes / 4; i += kLsThreads)
-                reinterpret_cast<uint32_t*>(smem + s * kLsStageBytes + 2 * kTileBytes)[i] = 0x3F803F80u;
+    // The aux tile is the second 64-column block of both operands: of B = [Y | aux] (N = 80: its columns 0..15
+    // are read) and of A = [X | aux] (M = 128: accumulator row 64 + m is the sum weighted by column m; row 80 is
+    // the one read out).  It is constant ones: [A' | a'] = x'^T [Y | 1] and [ysum | count] = 1^T [Y | 1].
+    for (int i = tid; i < kTileBytes / 4; i += kLsThreads) reinterpret_cast<uint32_t*>(smem + kLsOffAux)[i] = 0x3F803F80u;
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
@@ -196,13 +191,13 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         if (lane == 0) {
             // one M = 128, N = 80 product per K group: A = [X | aux], B = [Y | aux], the second 64-column block
             // of either operand addressed through the leading-offset field.
-            // Accumulator rows 0..63: [A' | a'] = x'^T [Y | aux];  row 80: [ysum | w0] = w^T [Y | aux].
+            // Accumulator rows 0..63: [A' | a'] = x'^T [Y | 1];  row 80: [ysum | count] = 1^T [Y | 1].
             const uint32_t idesc = umma_idesc_bf16(128, 80, 1, 1);
             bool ok = true;
             #pragma unroll 1
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kLsStages;
-                const uint32_t aX = sbase + s * kLsStageBytes, aY = aX + kTileBytes, aA = aY + kTileBytes;
+                const uint32_t aX = sbase + s * kLsStageBytes, aY = aX + kTileBytes, aA = sbase + kLsOffAux;
                 ok = mbar_wait(&bars->mapped[s], (c / kLsStages) & 1, prm.status, kStatusPipeTimeout);
                 if (!ok || *abort_flag) { ok = false; break; }
                 tc_fence_after_sync();
@@ -226,17 +221,7 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         #pragma unroll 1
         for (int c = 0; c < L; ++c) {
             const int s = c % kLsStages;
-            const int64_t row = row0 + (int64_t)c * kChunk + t;
-            float w = 1.f, delta = 0.f;
-            if (reverse) {
-                w = 1.f / __ldg(prm.dn + row);
-                delta = __ldg(prm.dl + row);
-            }
-            const bool padded = (int64_t)c * kChunk + t >= real;
-            if (padded) {           // whatever the tensors hold there must not be read as numbers
-                w = 0.f;
-                delta = 0.f;
-            }
+            const bool padded = (int64_t)c * kChunk + t >= real;      // whatever the tensors hold there is not read as numbers
             if (!mbar_wait(&bars->full[s], (c / kLsStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             if (tid == 0) LA_TRACE(g_trace_lin, c, 5);
@@ -248,16 +233,9 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     sts128(rowX + kTileBytes + ((hf * 4 + cc) << 4), 0u, 0u, 0u, 0u);
                 }
             } else if (elu) {
-                elu_half_row_inplace<true>(rowX, r7, w, hf, nch);
+                elu_half_row_inplace<true>(rowX, r7, 1.f, hf, nch);
             } else {
-                elu_half_row_inplace<false>(rowX, r7, w, hf, nch);
-            }
-            if (reverse && hf == 0) {
-                uint8_t* rowA = rowX + 2 * kTileBytes;
-                const uint32_t ww = pack_bf16x2(w, w), dd = pack_bf16x2(delta, delta);
-                sts128(rowA + ((0 ^ r7) << 4), dd, dd, dd, dd);
-                sts128(rowA + ((1 ^ r7) << 4), dd, dd, dd, dd);
-                sts128(rowA + ((2 ^ r7) << 4), ww, ww, ww, ww);
+                elu_half_row_inplace<false>(rowX, r7, 1.f, hf, nch);
             }
             fence_proxy_async_smem();
             mbar_arrive(&bars->mapped[s]);
@@ -285,7 +263,7 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             tmem_ld_wait();
             if (mine) {
                 if (warp < 2) rec[kDim * kDim + d_row] = z;
-                else rec[kDim * kDim + 2 * kDim] = reverse ? z : 0.f;
+                else rec[kDim * kDim + 2 * kDim] = 0.f;        // (the count: unused)
             }
         }
     }
@@ -831,7 +809,7 @@ Segmentation choose_splits(const la_problem& p) {
 }
 
 int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
-                const float* dn, const float* dl, const int* lengths, float* records, cudaStream_t st) {
+                const int* lengths, float* records, cudaStream_t st) {
     static bool attr_done = false;
     if (!attr_done) {
         LA_CUDA_TRY(cudaFuncSetAttribute(linear_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLsSmemBytes));
@@ -839,8 +817,6 @@ int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& 
     }
     LsParams prm;
     prm.records = records;
-    prm.dn = dn;
-    prm.dl = dl;
     prm.lengths = lengths;
     prm.heads = (int)p.H;
     prm.status = device_status_ptr();
@@ -910,7 +886,7 @@ int linear_forward(const la_problem& p, const void* Q, const void* K, const void
     if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
     if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
     float* rec = saved ? (float*)saved : (float*)ws;      // the split records, kept for the backward pass if asked
-    if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, lengths, rec, st)) return rc;
+    if (int rc = launch_sums(p, sg, mK, mV, lengths, rec, st)) return rc;
     ApParams a = {};
     a.lengths = lengths;
     a.records = rec;
@@ -936,7 +912,7 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
     float* rec_r = (float*)w;   w += bh * sg.nseg * kRecFloats * sizeof(float);
 
     if (saved) rec_s = (float*)saved;         // the forward's own records: nothing to recompute
-    else if (int rc = launch_sums(p, sg, mK, mV, nullptr, nullptr, lengths, rec_s, st)) return rc;
+    else if (int rc = launch_sums(p, sg, mK, mV, lengths, rec_s, st)) return rc;
     ApParams a = {};
     a.lengths = lengths;
     a.records = rec_s;
