@@ -196,7 +196,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                         if (!ok || *abort_flag) { ok = false; break; }
                         tc_fence_after_sync();
                         const uint32_t nQ = lo_k(stage_addr(c + 1)), nK = lo_k(stage_addr(c + 1) + kTileBytes);
-#pragma unroll
+#pragma unroll 1
                         for (int k = 0; k < 4; ++k)
                             umma_bf16(tmem + kColP + (b ^ 1) * 128, mk(nQ + 2 * k), mk(nK + 2 * k), idesc_p, k > 0);
                         umma_commit(&bars->p_full[b ^ 1]);
@@ -211,7 +211,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     LA_TRACE(g_trace_fwd, c, 3);
                     const uint32_t aV = stage_addr(c) + 2 * kTileBytes;
                     const uint32_t dV1 = lo_mn(aV, aOnes - aV);
-#pragma unroll
+#pragma unroll 1
                     for (int k = 0; k < 8; ++k)
                         umma_bf16_ta(tmem + kColNum + b * kNumStride, tmem + kColP + b * 128 + (k >> 2) * 64 + (k & 3) * 8,
                                      mk(dV1 + kStepV1 * k), idesc_num, 1);
@@ -233,7 +233,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                                  : mbar_wait(&bars->s_drained, (c - 1) & 1, prm.status, kStatusPipeTimeout));
                     if (!ok || *abort_flag) { ok = false; break; }
                     tc_fence_after_sync();
-#pragma unroll
+#pragma unroll 1
                     for (int k = 0; k < 8; ++k)
                         umma_bf16(tmem + kColS, mk(dKmn + 128 * k), mk(dV1 + kStepV1 * k), idesc_s, 1);
                     umma_commit(&bars->s_full);
@@ -244,7 +244,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint32_t dS = lo_mn(sbase + kOffS + (b ^ 1) * kStateTileBytes, kDim * 128);
-#pragma unroll
+#pragma unroll 1
                     for (int k = 0; k < 4; ++k)
                         umma_bf16(tmem + kColNum + b * kNumStride, mk(dQ + 2 * k), mk(dS + 128 * k), idesc_num, k > 0);
                     umma_commit(&bars->qs_full[b]);
