@@ -261,13 +261,20 @@ int la_recurrent_steps(const la_problem* p, const void* q, const void* k, const 
  * device) is not tolerable.  The price: every GPU on which the library is loaded holds
  * those LA_NOALLOC_SCRATCH_BYTES until the process exits, used or not.
  *
- *  - The call allocates and frees nothing, on the host or the device, and calls no
+ *  - The call itself allocates and frees nothing, on the host or the device, and calls no
  *    allocating library routine.  It always runs the general fp32-arithmetic kernels.
+ *    One caveat about the FIRST call on a device: the CUDA runtime loads a library's
+ *    device code lazily, and the address look-up of that first call is where the driver
+ *    may load this module and place the array in device memory.  That placement is the
+ *    driver's, not a cudaMalloc, but it does take device memory at that moment; a caller
+ *    under a strict budget should make one warm-up call (any small problem) while it is
+ *    still allowed to grow.
  *  - Problems whose scratch need (B*H*splits*D*(M+1)*4 bytes, at most a few splits per
  *    head) exceeds the array are rejected with LA_ERR_WORKSPACE and a message naming
  *    both sizes; nothing is enqueued.
  *  - The first call on each device looks up the array's device address (with that device
- *    current) and caches it; make that first call before starting any stream capture.
+ *    current) and caches it; make that first call before starting any stream capture
+ *    (it is also the call the caveat above is about).
  *  - All calls on a device share the one array, which keeps the previous call's contents.
  *    Nothing in it needs clearing between calls (each call overwrites what it reads), but
  *    two calls whose kernels overlap on the GPU (different streams) race on it: run them
@@ -288,8 +295,9 @@ const char* la_status_string(int status);
 const char* la_last_error(void);
 
 /* Synchronises `stream`, then reports whether any kernel of this library gave up
- * on a bounded wait since the last call (LA_ERR_DEVICE_TIMEOUT) and clears the
- * flag; LA_OK otherwise.  The context stays usable either way. */
+ * on a bounded wait since the last call (LA_ERR_DEVICE_TIMEOUT), or refused a saved
+ * buffer written under another piece plan (LA_ERR_INVALID_ARG, see la_plan_override()),
+ * and clears the flag; LA_OK otherwise.  The context stays usable either way. */
 int la_last_device_status(void* stream);
 
 /*
@@ -307,6 +315,18 @@ int la_last_device_status(void* stream);
  *                                              sequence b % (B*H)) }.
  */
 int la_causal_plan(const la_problem* p, int32_t* out, int capacity);
+
+/*
+ * Overrides of the automatic plans, for A/B checks and tests (no counterpart in the paper; host only).
+ * causal_pieces: equal pieces per sequence in the causal kernels; causal_short: length in chunks of the
+ * short middle piece (0: none); linear_splits: splits per sequence in the non-causal kernels.  -1 leaves a
+ * choice automatic; la_plan_override(-1, -1, -1) restores the defaults.  The setting is process-wide and
+ * read by every later call, la_workspace_bytes() and la_causal_plan() included: change it only between
+ * steps, size workspaces and saved buffers after the change, and never between a forward pass that
+ * fills a saved buffer and the backward pass that reads it (the backward pass notices: it computes
+ * nothing and la_last_device_status() returns LA_ERR_INVALID_ARG).
+ */
+int la_plan_override(int32_t causal_pieces, int32_t causal_short, int32_t linear_splits);
 
 /*
  * Gradient of the causal form continued from a state, for
@@ -343,7 +363,7 @@ long long la_kernel_launches(void);
  * la_profile_enable(0) stops recording.  la_profile_read() waits for the recorded events and
  * returns the mean duration in milliseconds and the number of launches of one kernel:
  * 0 causal_fwd_kernel, 1 causal_bwd_dq_kernel, 2 causal_bwd_dkv_kernel, 3 segment_sum_kernel,
- * 4 segment_scan_kernel, 5 linear_sum_kernel, 6 linear_apply_kernel, 7 recurrent_step_kernel.
+ * 4 (unused, empty name), 5 linear_sum_kernel, 6 linear_apply_kernel, 7 recurrent_step_kernel.
  * Not thread-safe; meant for a benchmark's single launching thread.
  */
 int la_profile_enable(int on);

@@ -9,7 +9,7 @@ from .binding import (  # noqa: F401
     la_linear_attention_varlen, la_linear_attention_varlen_backward,
     la_causal_forward, la_causal_backward, la_recurrent_step, la_recurrent_steps,
     la_workspace_bytes, la_last_device_status, la_kernel_launches, la_profile_enable, la_profile_read, la_version,
-    la_causal_plan,
+    la_causal_plan, la_plan_override,
     LA_F32, LA_BF16, LA_PHI_ELU1, LA_PHI_IDENTITY,
     LA_OP_LINEAR_FORWARD, LA_OP_LINEAR_BACKWARD, LA_OP_CAUSAL_FORWARD, LA_OP_CAUSAL_BACKWARD, LA_OP_CAUSAL_SAVED,
 )

@@ -30,7 +30,7 @@ EXPORTS = [
     "la_causal_forward", "la_causal_forward_from", "la_causal_backward_from",
     "la_causal_backward", "la_recurrent_step", "la_recurrent_steps", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
-    "la_profile_kernel_name", "la_version", "la_causal_plan",
+    "la_profile_kernel_name", "la_version", "la_causal_plan", "la_plan_override",
 ]
 
 
@@ -100,6 +100,13 @@ def _check(rc: int) -> None:
         raise LaError(rc, L.la_status_string(rc).decode(), L.la_last_error().decode())
 
 
+def _call(dev, fn, *args) -> None:
+    """One library call with `dev` current: the library launches on, and keeps its per-device state for,
+    the current device, which need not be the one the tensors live on."""
+    with torch.cuda.device(dev):
+        _check(fn(*args))
+
+
 def _dtype_code(t: torch.Tensor) -> int:
     if t.dtype == torch.float32:
         return LA_F32
@@ -117,6 +124,8 @@ def _stream(device) -> ctypes.c_void_p:
 
 
 def _dev(*ts):
+    """All tensors given (None: not given) must be contiguous and live on one CUDA device; returns it."""
+    dev = None
     for t in ts:
         if t is None:
             continue
@@ -124,7 +133,42 @@ def _dev(*ts):
             raise ValueError("tensors must live on a CUDA device")
         if not t.is_contiguous():
             raise ValueError("tensors must be contiguous")
-    return ts[0].device
+        if dev is None:
+            dev = t.device
+        elif t.device != dev:
+            raise ValueError(f"all tensors of a call must live on one device (got {dev} and {t.device})")
+    return dev
+
+
+_KINDS = {
+    # kind -> (shape as a function of the problem, dtype: None = the I/O type of Q)
+    "qk": (lambda p: (p.B, p.H, p.N, p.D), None),
+    "v": (lambda p: (p.B, p.H, p.N, p.M), None),
+    "row": (lambda p: (p.B, p.H, p.N), torch.float32),
+    "S": (lambda p: (p.B, p.H, p.D, p.M), torch.float32),
+    "Z": (lambda p: (p.B, p.H, p.D), torch.float32),
+    "q1": (lambda p: (p.B, p.H, p.D), None),
+    "v1": (lambda p: (p.B, p.H, p.M), None),
+}
+
+
+def _expect(p: la_problem, io_dtype, **named):
+    """Shape and dtype of every tensor handed to the library, checked before any pointer is taken: the kernels
+    trust the problem descriptor, so a short or mistyped tensor would be read or written past its end.
+    named: name=(tensor or None, kind); see _KINDS."""
+    for name, (t, kind) in named.items():
+        if t is None:
+            continue
+        shape_of, dtype = _KINDS[kind]
+        want_shape, want_dtype = tuple(shape_of(p)), (io_dtype if dtype is None else dtype)
+        if tuple(t.shape) != want_shape or t.dtype != want_dtype:
+            raise ValueError(f"{name} must have shape {list(want_shape)} and dtype {want_dtype} "
+                             f"(got {list(t.shape)}, {t.dtype})")
+
+
+def _buffer(name, t):
+    if t is not None and (t.dtype != torch.uint8 or t.dim() != 1):
+        raise ValueError(f"{name} must be a 1-D uint8 tensor (got {list(t.shape)}, {t.dtype})")
 
 
 def make_problem(B, H, N, D, M, dtype_code, phi="elu1", eps=0.0) -> la_problem:
@@ -185,6 +229,11 @@ def la_causal_plan(p: la_problem):
     return out
 
 
+def la_plan_override(causal_pieces: int = -1, causal_short: int = -1, linear_splits: int = -1) -> None:
+    """Process-wide overrides of the automatic piece / split plans (A/B checks and tests); no arguments: automatic."""
+    _check(lib().la_plan_override(int(causal_pieces), int(causal_short), int(linear_splits)))
+
+
 def la_profile_enable(on: bool) -> None:
     _check(lib().la_profile_enable(int(on)))
 
@@ -206,13 +255,16 @@ def la_version() -> str:
 
 def la_last_device_status(device=None) -> None:
     """Synchronise the current stream; raise LaError if a kernel gave up on a bounded wait."""
-    _check(lib().la_last_device_status(_stream(device)))
+    with torch.cuda.device(torch.cuda.current_device() if device is None else device):
+        _check(lib().la_last_device_status(_stream(device)))
 
 
 def la_feature_map(x: torch.Tensor, deriv: bool = False, out: torch.Tensor | None = None) -> torch.Tensor:
+    if out is not None and (out.shape != x.shape or out.dtype != x.dtype):
+        raise ValueError(f"out must have shape {list(x.shape)} and dtype {x.dtype}")
     dev = _dev(x, out)
     y = torch.empty_like(x) if out is None else out
-    _check(lib().la_feature_map(_ptr(x), _ptr(y), x.numel(), _dtype_code(x), int(deriv), _stream(dev)))
+    _call(dev, lib().la_feature_map, _ptr(x), _ptr(y), x.numel(), _dtype_code(x), int(deriv), _stream(dev))
     return y
 
 
@@ -224,21 +276,27 @@ def poly2_columns(D: int) -> int:
 def la_feature_map_poly2(x: torch.Tensor, C: int | None = None, out: torch.Tensor | None = None) -> torch.Tensor:
     """Degree-2 polynomial feature map along the last axis: [..., D] -> [..., C] (C defaults to poly2_columns(D));
     feed the result to the attention calls with phi="identity"."""
-    dev = _dev(x, out)
     D = x.shape[-1]
     C = poly2_columns(D) if C is None else C
+    if out is not None and (tuple(out.shape) != tuple(x.shape[:-1]) + (C,) or out.dtype != x.dtype):
+        raise ValueError(f"out must have shape {list(x.shape[:-1]) + [C]} and dtype {x.dtype}")
+    dev = _dev(x, out)
     y = torch.empty(x.shape[:-1] + (C,), dtype=x.dtype, device=x.device) if out is None else out
-    _check(lib().la_feature_map_poly2(_ptr(x), _ptr(y), x.numel() // max(D, 1), D, C, _dtype_code(x), _stream(dev)))
+    _call(dev, lib().la_feature_map_poly2, _ptr(x), _ptr(y), x.numel() // max(D, 1), D, C, _dtype_code(x), _stream(dev))
     return y
 
 
 def la_feature_map_poly2_backward(x: torch.Tensor, dy: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
     """Gradient of la_feature_map_poly2 with respect to x for an upstream gradient dy [..., C]."""
-    dev = _dev(x, dy, out)
     D, C = x.shape[-1], dy.shape[-1]
+    if dy.shape[:-1] != x.shape[:-1] or dy.dtype != x.dtype:
+        raise ValueError(f"dy must have shape {list(x.shape[:-1])} + [C] and dtype {x.dtype}")
+    if out is not None and (out.shape != x.shape or out.dtype != x.dtype):
+        raise ValueError(f"out must have shape {list(x.shape)} and dtype {x.dtype}")
+    dev = _dev(x, dy, out)
     dx = torch.empty_like(x) if out is None else out
-    _check(lib().la_feature_map_poly2_backward(_ptr(x), _ptr(dy), _ptr(dx), x.numel() // max(D, 1), D, C,
-                                               _dtype_code(x), _stream(dev)))
+    _call(dev, lib().la_feature_map_poly2_backward, _ptr(x), _ptr(dy), _ptr(dx), x.numel() // max(D, 1), D, C,
+                                               _dtype_code(x), _stream(dev))
     return dx
 
 
@@ -254,20 +312,24 @@ def la_linear_attention(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, KV=None,
     """Non-causal form.  Returns O; pass preallocated den / KV / Zs tensors to receive them, and a
     linear_saved_buffer() to keep the sums over the keys for the backward pass (la_linear_attention_keep;
     lengths: optional [B] int32 device tensor of a right-padded ragged batch)."""
-    dev = _dev(Q, K, V, O, den, KV, Zs, saved, lengths)
     p = _problem_of(Q, V, phi, eps)
+    _expect(p, Q.dtype, Q=(Q, "qk"), K=(K, "qk"), V=(V, "v"), O=(O, "v"), den=(den, "row"), KV=(KV, "S"), Zs=(Zs, "Z"))
+    _buffer("saved", saved), _buffer("ws", ws)
+    if lengths is not None:
+        _lengths_arg(lengths, p.B, None)
+    dev = _dev(Q, K, V, O, den, KV, Zs, saved, lengths, ws)
     O = torch.empty_like(V) if O is None else O
     if saved is not None:
-        _check(lib().la_linear_attention_keep(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(O), _ptr(den),
+        _call(dev, lib().la_linear_attention_keep, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(O), _ptr(den),
                                               _ptr(KV), _ptr(Zs), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws),
-                                              _stream(dev)))
+                                              _stream(dev))
         return O
     if lengths is not None:
         return la_linear_attention_varlen(Q, K, V, lengths, phi, eps, O, den, KV, Zs, ws)
     ws = workspace(p, LA_OP_LINEAR_FORWARD, dev) if ws is None else ws
-    _check(lib().la_linear_attention(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(KV),
+    _call(dev, lib().la_linear_attention, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(KV),
                                      _ptr(Zs), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
-                                     _stream(dev)))
+                                     _stream(dev))
     return O
 
 
@@ -277,11 +339,12 @@ def la_linear_attention_noalloc(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, 
     For callers that may not allocate device memory around the call; here only the output
     tensor is created when `O` is not passed in.  Raises LaError (LA_ERR_WORKSPACE) when the
     problem needs more scratch than the array holds."""
-    dev = _dev(Q, K, V, O, den, KV, Zs)
     p = _problem_of(Q, V, phi, eps)
+    _expect(p, Q.dtype, Q=(Q, "qk"), K=(K, "qk"), V=(V, "v"), O=(O, "v"), den=(den, "row"), KV=(KV, "S"), Zs=(Zs, "Z"))
+    dev = _dev(Q, K, V, O, den, KV, Zs)
     O = torch.empty_like(V) if O is None else O
-    _check(lib().la_linear_attention_noalloc(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den),
-                                             _ptr(KV), _ptr(Zs), _stream(dev)))
+    _call(dev, lib().la_linear_attention_noalloc, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den),
+                                             _ptr(KV), _ptr(Zs), _stream(dev))
     return O
 
 
@@ -289,8 +352,13 @@ def la_linear_attention_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=No
                                  dQ=None, dK=None, dV=None, ws=None, saved=None, lengths=None):
     """Gradients of the non-causal form.  saved: what la_linear_attention(..., saved=...) kept for the same
     problem (la_linear_attention_backward_kept); lengths as there.  Returns (dQ, dK, dV)."""
-    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved, lengths)
     p = _problem_of(Q, V, phi, eps)
+    _expect(p, Q.dtype, Q=(Q, "qk"), K=(K, "qk"), V=(V, "v"), G=(G, "v"), O=(O, "v"), den=(den, "row"),
+            dQ=(dQ, "qk"), dK=(dK, "qk"), dV=(dV, "v"))
+    _buffer("saved", saved), _buffer("ws", ws)
+    if lengths is not None:
+        _lengths_arg(lengths, p.B, None)
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved, lengths, ws)
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(V) if dV is None else dV
@@ -298,13 +366,11 @@ def la_linear_attention_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=No
         return la_linear_attention_varlen_backward(Q, K, V, G, lengths, phi, eps, O, den, dQ, dK, dV, ws)
     ws = workspace(p, LA_OP_LINEAR_BACKWARD, dev) if ws is None else ws
     if saved is not None:
-        _check(lib().la_linear_attention_backward_kept(
-            ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(saved), _nbytes(saved), _ptr(O), _ptr(den),
-            _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), _nbytes(ws), _stream(dev)))
+        _call(dev, lib().la_linear_attention_backward_kept, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(saved), _nbytes(saved), _ptr(O), _ptr(den),
+            _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), _nbytes(ws), _stream(dev))
         return dQ, dK, dV
-    _check(lib().la_linear_attention_backward(
-        ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV),
-        _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(dev)))
+    _call(dev, lib().la_linear_attention_backward, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV),
+        _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream(dev))
     return dQ, dK, dV
 
 
@@ -324,20 +390,20 @@ def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None
     """Causal form.  Returns O; pass preallocated den / S_out / Z_out tensors to receive them, and a
     saved_buffer() to keep phi(Q), phi(K) for the backward pass.  S_in / Z_in (fp32 [B,H,D,M] / [B,H,D]):
     the state the sequence continues from (la_causal_forward_from)."""
-    dev = _dev(Q, K, V, O, den, S_out, Z_out, saved, S_in, Z_in)
     p = _problem_of(Q, V, phi, eps)
+    _expect(p, Q.dtype, Q=(Q, "qk"), K=(K, "qk"), V=(V, "v"), O=(O, "v"), den=(den, "row"), S_out=(S_out, "S"),
+            Z_out=(Z_out, "Z"), S_in=(S_in, "S"), Z_in=(Z_in, "Z"))
+    _buffer("saved", saved), _buffer("ws", ws)
+    dev = _dev(Q, K, V, O, den, S_out, Z_out, saved, S_in, Z_in, ws)
     O = torch.empty_like(V) if O is None else O
     ws = workspace(p, LA_OP_CAUSAL_FORWARD, dev) if ws is None else ws
     if S_in is None and Z_in is None:
-        _check(lib().la_causal_forward(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(S_out),
-                                       _ptr(Z_out), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(dev)))
+        _call(dev, lib().la_causal_forward, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(S_out),
+                                       _ptr(Z_out), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(dev))
     else:
-        for t, shape in ((S_in, (p.B, p.H, p.D, p.M)), (Z_in, (p.B, p.H, p.D))):
-            if t is not None and (t.dtype != torch.float32 or tuple(t.shape) != shape or not t.is_contiguous()):
-                raise ValueError("S_in / Z_in must be contiguous fp32 tensors of shape [B,H,D,M] / [B,H,D]")
-        _check(lib().la_causal_forward_from(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(S_in), _ptr(Z_in), _ptr(O),
+        _call(dev, lib().la_causal_forward_from, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(S_in), _ptr(Z_in), _ptr(O),
                                             _ptr(den), _ptr(S_out), _ptr(Z_out), _ptr(saved), _nbytes(saved), _ptr(ws),
-                                            _nbytes(ws), _stream(dev)))
+                                            _nbytes(ws), _stream(dev))
     return O
 
 
@@ -346,61 +412,56 @@ def la_causal_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None, saved=
     """Gradients of the causal form; returns (dQ, dK, dV).  With any of the state arguments (fp32 [B,H,D,M] /
     [B,H,D]: the state the forward started from, the upstream gradient of its final state, and tensors that
     receive the gradient of the initial state) the call is la_causal_backward_from."""
-    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved, S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in)
     p = _problem_of(Q, V, phi, eps)
+    _expect(p, Q.dtype, Q=(Q, "qk"), K=(K, "qk"), V=(V, "v"), G=(G, "v"), O=(O, "v"), den=(den, "row"),
+            dQ=(dQ, "qk"), dK=(dK, "qk"), dV=(dV, "v"), S_in=(S_in, "S"), Z_in=(Z_in, "Z"), dS_out=(dS_out, "S"),
+            dZ_out=(dZ_out, "Z"), dS_in=(dS_in, "S"), dZ_in=(dZ_in, "Z"))
+    _buffer("saved", saved), _buffer("ws", ws)
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved, S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in, ws)
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(V) if dV is None else dV
     ws = workspace(p, LA_OP_CAUSAL_BACKWARD, dev) if ws is None else ws
     state = (S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in)
     if all(t is None for t in state):
-        _check(lib().la_causal_backward(
-            ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(saved), _nbytes(saved),
-            _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), _nbytes(ws), _stream(dev)))
+        _call(dev, lib().la_causal_backward, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(G), _ptr(saved), _nbytes(saved),
+            _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), _nbytes(ws), _stream(dev))
     else:
-        for t, shape in zip(state, ((p.B, p.H, p.D, p.M), (p.B, p.H, p.D)) * 3):
-            if t is not None and (t.dtype != torch.float32 or tuple(t.shape) != shape or not t.is_contiguous()):
-                raise ValueError("state arguments must be contiguous fp32 tensors of shape [B,H,D,M] / [B,H,D]")
-        _check(lib().la_causal_backward_from(
-            ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(S_in), _ptr(Z_in), _ptr(O), _ptr(den), _ptr(G),
+        _call(dev, lib().la_causal_backward_from, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(S_in), _ptr(Z_in), _ptr(O), _ptr(den), _ptr(G),
             _ptr(dS_out), _ptr(dZ_out), _ptr(saved), _nbytes(saved), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dS_in), _ptr(dZ_in),
-            _ptr(ws), _nbytes(ws), _stream(dev)))
+            _ptr(ws), _nbytes(ws), _stream(dev))
     return dQ, dK, dV
 
 
 def la_recurrent_step(q, k, v, S, Z, phi="elu1", eps=0.0, out=None):
     """One decode step: S, Z (fp32) are updated in place; returns out [B,H,M]."""
-    dev = _dev(q, k, v, S, Z, out)
-    if q.dim() != 3 or v.dim() != 3 or S.dtype != torch.float32 or Z.dtype != torch.float32:
+    if q.dim() != 3 or v.dim() != 3:
         raise ValueError("expected q,k [B,H,D], v [B,H,M], fp32 S [B,H,D,M] and Z [B,H,D]")
     B, H, D = q.shape
     M = v.shape[2]
-    if tuple(S.shape) != (B, H, D, M) or tuple(Z.shape) != (B, H, D):
-        raise ValueError("state shape mismatch")
     p = make_problem(B, H, 1, D, M, _dtype_code(q), phi, eps)
+    _expect(p, q.dtype, q=(q, "q1"), k=(k, "q1"), v=(v, "v1"), S=(S, "S"), Z=(Z, "Z"), out=(out, "v1"))
+    dev = _dev(q, k, v, S, Z, out)
     out = torch.empty_like(v) if out is None else out
-    _check(lib().la_recurrent_step(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out),
-                                   _stream(dev)))
+    _call(dev, lib().la_recurrent_step, ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out),
+                                   _stream(dev))
     return out
 
 
 def la_recurrent_steps(q, k, v, S, Z, phi="elu1", eps=0.0, out=None):
     """N decode steps in one launch (all inputs known beforehand): q, k [B,H,N,D], v [B,H,N,M]; S, Z (fp32)
     are updated in place; returns out [B,H,N,M]."""
-    dev = _dev(q, k, v, S, Z, out)
-    if q.dim() != 4 or v.dim() != 4 or S.dtype != torch.float32 or Z.dtype != torch.float32:
-        raise ValueError("expected q,k [B,H,N,D], v [B,H,N,M], fp32 S [B,H,D,M] and Z [B,H,D]")
     p = _problem_of(q, v, phi, eps)
-    if tuple(S.shape) != (p.B, p.H, p.D, p.M) or tuple(Z.shape) != (p.B, p.H, p.D):
-        raise ValueError("state shape mismatch")
+    _expect(p, q.dtype, q=(q, "qk"), k=(k, "qk"), v=(v, "v"), S=(S, "S"), Z=(Z, "Z"), out=(out, "v"))
+    dev = _dev(q, k, v, S, Z, out)
     out = torch.empty_like(v) if out is None else out
-    _check(lib().la_recurrent_steps(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out),
-                                    _stream(dev)))
+    _call(dev, lib().la_recurrent_steps, ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out),
+                                    _stream(dev))
     return out
 
 
 def _lengths_arg(lengths, B, dev):
-    if lengths.dtype != torch.int32 or tuple(lengths.shape) != (B,) or not lengths.is_cuda or not lengths.is_contiguous():
+    if lengths.dtype != torch.int32 or tuple(lengths.shape) != (B,) or not lengths.is_contiguous():
         raise ValueError("lengths must be a contiguous int32 CUDA tensor of shape [B]")
     return lengths
 
@@ -408,27 +469,31 @@ def _lengths_arg(lengths, B, dev):
 def la_linear_attention_varlen(Q, K, V, lengths, phi="elu1", eps=0.0, O=None, den=None, KV=None, Zs=None, ws=None):
     """Non-causal form on a right-padded ragged batch: lengths[b] real positions per batch element; O and den
     are zero on the padding.  Returns O."""
-    dev = _dev(Q, K, V, O, den, KV, Zs)
     p = _problem_of(Q, V, phi, eps)
-    _lengths_arg(lengths, p.B, dev)
+    _expect(p, Q.dtype, Q=(Q, "qk"), K=(K, "qk"), V=(V, "v"), O=(O, "v"), den=(den, "row"), KV=(KV, "S"), Zs=(Zs, "Z"))
+    _buffer("ws", ws)
+    _lengths_arg(lengths, p.B, None)
+    dev = _dev(Q, K, V, O, den, KV, Zs, lengths, ws)
     O = torch.empty_like(V) if O is None else O
     ws = workspace(p, LA_OP_LINEAR_VARLEN_FORWARD, dev) if ws is None else ws
-    _check(lib().la_linear_attention_varlen(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(O), _ptr(den),
-                                            _ptr(KV), _ptr(Zs), _ptr(ws), _nbytes(ws), _stream(dev)))
+    _call(dev, lib().la_linear_attention_varlen, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(O), _ptr(den),
+                                            _ptr(KV), _ptr(Zs), _ptr(ws), _nbytes(ws), _stream(dev))
     return O
 
 
 def la_linear_attention_varlen_backward(Q, K, V, G, lengths, phi="elu1", eps=0.0, O=None, den=None,
                                         dQ=None, dK=None, dV=None, ws=None):
     """Gradients of la_linear_attention_varlen; zero on the padding.  Returns (dQ, dK, dV)."""
-    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV)
     p = _problem_of(Q, V, phi, eps)
-    _lengths_arg(lengths, p.B, dev)
+    _expect(p, Q.dtype, Q=(Q, "qk"), K=(K, "qk"), V=(V, "v"), G=(G, "v"), O=(O, "v"), den=(den, "row"),
+            dQ=(dQ, "qk"), dK=(dK, "qk"), dV=(dV, "v"))
+    _buffer("ws", ws)
+    _lengths_arg(lengths, p.B, None)
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, lengths, ws)
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(V) if dV is None else dV
     ws = workspace(p, LA_OP_LINEAR_VARLEN_BACKWARD, dev) if ws is None else ws
-    _check(lib().la_linear_attention_varlen_backward(
-        ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(O), _ptr(den), _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV),
-        _ptr(ws), _nbytes(ws), _stream(dev)))
+    _call(dev, lib().la_linear_attention_varlen_backward, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(O), _ptr(den), _ptr(G), _ptr(dQ), _ptr(dK), _ptr(dV),
+        _ptr(ws), _nbytes(ws), _stream(dev))
     return dQ, dK, dV

@@ -53,7 +53,7 @@ int* device_status_ptr() {
     return (int*)p;
 }
 
-static int check_arch() {
+int check_arch() {
     static thread_local int cached_dev = -1, cached_rc = 0;
     int dev = 0;
     LA_CUDA_TRY(cudaGetDevice(&dev));
@@ -66,9 +66,9 @@ static int check_arch() {
     return LA_OK;
 }
 
-static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-static int check_problem(const la_problem* p, bool need_n) {
+int check_problem(const la_problem* p, bool need_n) {
     if (!p) return fail(LA_ERR_INVALID_ARG, "problem descriptor is NULL");
     if (p->B < 1 || p->H < 1 || p->D < 1 || p->M < 1 || (need_n && p->N < 0))
         return fail(LA_ERR_INVALID_ARG, "sizes must be B,H,D,M >= 1 and N >= 0 (got B=%lld H=%lld N=%lld D=%lld M=%lld)",
@@ -167,7 +167,7 @@ int la_profile_read(int kernel, double* mean_ms, int* launches) {
 
 const char* la_profile_kernel_name(int kernel) {
     static const char* names[kProfCount] = {"causal_fwd_kernel", "causal_bwd_dq_kernel", "causal_bwd_dkv_kernel",
-                                            "segment_sum_kernel", "segment_scan_kernel", "linear_sum_kernel",
+                                            "segment_sum_kernel", "", "linear_sum_kernel",
                                             "linear_apply_kernel", "recurrent_step_kernel"};
     return kernel >= 0 && kernel < kProfCount ? names[kernel] : "";
 }
@@ -191,6 +191,13 @@ int la_causal_plan(const la_problem* p, int32_t* out, int capacity) {
     if (capacity < 0 || (capacity > 0 && !out)) return fail(LA_ERR_INVALID_ARG, "out is NULL or capacity is negative");
     if (p->N == 0 || !tc_supported(*p, LA_OP_CAUSAL_FORWARD)) return 0;
     return tc_causal_plan(*p, out, capacity);
+}
+
+int la_plan_override(int32_t causal_pieces, int32_t causal_short, int32_t linear_splits) {
+    if (causal_pieces < -1 || causal_pieces == 0 || causal_short < -1 || linear_splits < -1 || linear_splits == 0)
+        return fail(LA_ERR_INVALID_ARG, "overrides are -1 (automatic) or positive counts (causal_short may be 0: no short piece)");
+    tc_set_plan_override(causal_pieces, causal_short, linear_splits);
+    return LA_OK;
 }
 
 int la_feature_map(const void* x, void* y, int64_t n, int32_t dtype, int32_t deriv, void* stream) {
@@ -440,6 +447,9 @@ int la_last_device_status(void* stream) {
     if (word == 0) return LA_OK;
     int zero = 0;
     LA_CUDA_TRY(cudaMemcpyToSymbol(g_device_status_word, &zero, sizeof(int)));
+    if (word & 8)
+        return fail(LA_ERR_INVALID_ARG, "a saved buffer was written by a forward pass with another piece plan (another "
+                                        "la_plan_override() setting or device): the backward pass computed nothing (device status 0x%x)", word);
     return fail(LA_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (device status 0x%x)", word);
 }
 

@@ -26,6 +26,13 @@ int cuda_fail(cudaError_t e, const char* what);
         if (e__ != cudaSuccess) return ::la::cuda_fail(e__, #expr); \
     } while (0)
 
+// Argument checks shared by every entry point (defined in la_api.cu): sizes, enums and limits of a
+// problem descriptor (need_n: N is used and must be >= 0 and not too long); 16-byte alignment;
+// compute capability 10.x of the current device (cached per device and thread).
+int check_problem(const la_problem* p, bool need_n);
+bool aligned16(const void* p);
+int check_arch();
+
 // Device status word: kernels that give up on a bounded wait OR a code into it.
 // Returns its device address for the current device (NULL on failure).
 int* device_status_ptr();
@@ -36,7 +43,7 @@ void note_launch();
 // Optional per-kernel timing with CUDA events on the launch stream (see la_profile_enable()).
 // Indices are part of the C ABI (la_profile_read); no-ops unless profiling is switched on.
 enum ProfKernel {
-    kProfCausalFwd = 0, kProfCausalBwdDq = 1, kProfCausalBwdDkv = 2, kProfSegmentSum = 3, kProfSegmentScan = 4,
+    kProfCausalFwd = 0, kProfCausalBwdDq = 1, kProfCausalBwdDkv = 2, kProfSegmentSum = 3, kProfUnused = 4,
     kProfLinearSum = 5, kProfLinearApply = 6, kProfRecurrent = 7, kProfCount = 8
 };
 void prof_begin(int kernel, cudaStream_t st);

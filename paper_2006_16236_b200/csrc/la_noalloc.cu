@@ -41,8 +41,6 @@ int scratch_for_current_device(void** out) {
     return LA_OK;
 }
 
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
 }  // namespace
 }  // namespace la
 
@@ -50,15 +48,7 @@ using namespace la;
 
 extern "C" int la_linear_attention_noalloc(const la_problem* p, const void* Q, const void* K, const void* V,
                                            void* O, float* den, float* KV, float* Zs, void* stream) {
-    if (!p) return fail(LA_ERR_INVALID_ARG, "problem descriptor is NULL");
-    if (p->B < 1 || p->H < 1 || p->N < 0 || p->D < 1 || p->M < 1)
-        return fail(LA_ERR_INVALID_ARG, "sizes must be B,H,D,M >= 1 and N >= 0");
-    if (p->dtype != LA_F32 && p->dtype != LA_BF16) return fail(LA_ERR_INVALID_ARG, "dtype %d is not a la_dtype", p->dtype);
-    if (p->phi != LA_PHI_ELU1 && p->phi != LA_PHI_IDENTITY) return fail(LA_ERR_INVALID_ARG, "phi %d is not a la_phi", p->phi);
-    if (!(p->eps >= 0.f)) return fail(LA_ERR_INVALID_ARG, "eps must be >= 0");
-    if (p->D % 8 || p->M % 8 || p->D > 128 || p->M > 128)
-        return fail(LA_ERR_UNSUPPORTED, "D and M must be multiples of 8 in [8,128]");
-    if (p->B * p->H > 0x7fffffffLL) return fail(LA_ERR_UNSUPPORTED, "B*H exceeds 2^31-1");
+    if (int rc = check_problem(p, true)) return rc;        // the same checks as la_linear_attention()
     if (p->N == 0) return LA_OK;
     const void* required[4] = {Q, K, V, O};
     for (const void* ptr : required) {
@@ -74,10 +64,7 @@ extern "C" int la_linear_attention_noalloc(const la_problem* p, const void* Q, c
                     "this problem needs %zu bytes of scratch but the built-in array holds %zu: use "
                     "la_linear_attention with a caller-provided workspace",
                     need, (size_t)LA_NOALLOC_SCRATCH_BYTES);
-    int major = 0, dev = 0;
-    LA_CUDA_TRY(cudaGetDevice(&dev));
-    LA_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
-    if (major != 10) return fail(LA_ERR_ARCH, "device %d has compute capability %d.x; this library is built for sm_100a only", dev, major);
+    if (int rc = check_arch()) return rc;
 
     void* scratch = nullptr;
     if (int rc = scratch_for_current_device(&scratch)) return rc;

@@ -32,6 +32,7 @@ constexpr uint32_t kWaitLimit = 4u << 20;
 constexpr int kStatusTmaTimeout = 1;
 constexpr int kStatusMmaTimeout = 2;
 constexpr int kStatusPipeTimeout = 4;
+constexpr int kStatusPlanMismatch = 8;      // a saved buffer was written under another piece plan
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));

@@ -8,7 +8,81 @@ namespace la {
 
 namespace tc {
 
+static std::atomic<int> g_override_pieces{-1}, g_override_short{-1}, g_override_splits{-1};
+
+PlanOverride plan_override() {
+    return PlanOverride{g_override_pieces.load(std::memory_order_relaxed), g_override_short.load(std::memory_order_relaxed),
+                        g_override_splits.load(std::memory_order_relaxed)};
+}
+void set_plan_override(int pieces, int short_len, int splits);
+void set_plan_override(int pieces, int short_len, int splits) {
+    g_override_pieces.store(pieces, std::memory_order_relaxed);
+    g_override_short.store(short_len, std::memory_order_relaxed);
+    g_override_splits.store(splits, std::memory_order_relaxed);
+}
+
+int sm_count() {
+    static thread_local int cached_dev = -1, cached_sms = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();         // no device: not an error of the caller's
+        return 148;
+    }
+    if (dev != cached_dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+            cudaGetLastError();
+            return 148;
+        }
+        cached_dev = dev;
+        cached_sms = n;
+    }
+    return cached_sms;
+}
+
+// Encoding a tensor map is a driver call of a microsecond or two and a training loop passes the same few
+// tensors again and again: the last maps of the calling thread are kept, keyed by everything that goes in.
+namespace {
+struct MapKey {
+    const void* base;
+    uint64_t rows;
+    uint32_t box_rows;
+    int cols, dev;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && rows == o.rows && box_rows == o.box_rows && cols == o.cols && dev == o.dev;
+    }
+};
+constexpr int kMapCache = 32;
+struct MapCache {
+    MapKey key[kMapCache];
+    CUtensorMap map[kMapCache];
+    bool used[kMapCache];
+    int next;
+};
+thread_local MapCache g_maps = {};
+}  // namespace
+
+static int encode_tile_map_uncached(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols);
+
 int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols) {
+    int dev = 0;
+    LA_CUDA_TRY(cudaGetDevice(&dev));
+    const MapKey key{base, rows, box_rows, cols, dev};
+    for (int i = 0; i < kMapCache; ++i)
+        if (g_maps.used[i] && g_maps.key[i] == key) {
+            *map = g_maps.map[i];
+            return LA_OK;
+        }
+    if (int rc = encode_tile_map_uncached(map, base, rows, box_rows, cols)) return rc;
+    const int slot = g_maps.next;
+    g_maps.next = (slot + 1) % kMapCache;
+    g_maps.key[slot] = key;
+    g_maps.map[slot] = *map;
+    g_maps.used[slot] = true;
+    return LA_OK;
+}
+
+static int encode_tile_map_uncached(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols) {
     static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     if (!encode) {
         void* fn = nullptr;
@@ -51,6 +125,9 @@ size_t tc_workspace_bytes(const la_problem& p, int op) {
 }
 
 size_t tc_causal_saved_bytes(const la_problem& p) { return tc::causal_saved_bytes(p); }
+void tc_set_plan_override(int causal_pieces, int causal_short, int linear_splits) {
+    tc::set_plan_override(causal_pieces, causal_short, linear_splits);
+}
 int tc_causal_plan(const la_problem& p, int32_t* out, int capacity) {
     const tc::CausalPlan pl = tc::choose_plan(p);
     const int np = pl.npieces(), nq = pl.nparts();

@@ -9,6 +9,8 @@ bool tc_supported(const la_problem& p, int op);
 size_t tc_workspace_bytes(const la_problem& p, int op);
 
 size_t tc_causal_saved_bytes(const la_problem& p);
+// process-wide overrides of the automatic plans (see la_plan_override)
+void tc_set_plan_override(int causal_pieces, int causal_short, int linear_splits);
 // pieces, parts, piece_begin[], piece_first_part[], part_begin[], launch_order[] (see la_causal_plan)
 int tc_causal_plan(const la_problem& p, int32_t* out, int capacity);
 int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,

@@ -20,8 +20,8 @@
 // Every product runs on tcgen05 with fp32 accumulators in TMEM; the running states
 // stay in TMEM in fp32 and are re-rounded to a bf16 operand tile once per chunk.  No
 // per-position state is ever stored.  Sequences are cut into segments that run on
-// different SMs; a segment starts from the exclusive prefix (forward sweep) or suffix
-// (reverse sweep) of per-segment sums produced by a pre-pass and a scan.
+// different SMs; a segment starts from the sum of the pre-pass records of the parts before it
+// (forward sweep) or after it (reverse sweep), which it adds up itself.
 #include "la_tc.cuh"
 #include "la_tc_common.cuh"
 
@@ -56,7 +56,7 @@ namespace {
 // Warps 0-7 ("score/epilogue" warps, two per TMEM quadrant: the pair shares the 128 rows
 // of the quadrant, one warp per 32-column half): mask + round dP of chunk c+1, then the dQ
 // epilogue of chunk c.  Warps 8-11: phi(K), phi(Q) in place and the state conversion.
-// Warp 12: TMA.  Warp 13: MMA issue.
+// Warp 12: TMA.  Warps 13, 14: MMA issue (13 also allocates TMEM).
 // ===========================================================================
 constexpr int kDqStages = 2;
 constexpr int kDqThreads = 480;
@@ -98,6 +98,7 @@ struct DqParams {
     int phi;
     int dim;                    // D = M: 64, or 32 (tiles zero-padded to 64 columns)
     int map;                    // apply the feature map on load (0: the inputs are already phi(Q), phi(K))
+    const int* stamp;           // the plan the forward recorded in the saved buffer, or null (no saved buffer)
 };
 
 __global__ void __launch_bounds__(kDqThreads, 1)
@@ -166,8 +167,17 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     grid_dependency_wait();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
+    bool mismatch = false;      // the saved buffer must come from a forward pass with this very plan
+    if (prm.stamp) {
+        int want[kPlanStampInts];
+        plan_stamp(plan, prm.dim, want);
+#pragma unroll
+        for (int i = 0; i < kPlanStampInts; ++i) mismatch = mismatch || __ldg(prm.stamp + i) != want[i];
+    }
 
-    if (warp == 12) {
+    if (mismatch) {             // the same for every thread: nothing is started, the CTA leaves through the common exit
+        if (tid == 0) atomicOr(prm.status, kStatusPlanMismatch);
+    } else if (warp == 12) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG); prefetch_tensormap(&mapQ);
@@ -941,12 +951,9 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     int* status = device_status_ptr();
     if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
 
-    static bool attr_done = false;
-    if (!attr_done) {
-        LA_CUDA_TRY(cudaFuncSetAttribute(causal_bwd_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDqSmemBytes));
-        LA_CUDA_TRY(cudaFuncSetAttribute(causal_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kKvSmemBytes));
-        attr_done = true;
-    }
+    static std::atomic<uint64_t> attr_dq{0}, attr_dkv{0};
+    if (int rc = opt_in_smem_once(causal_bwd_dq_kernel, kDqSmemBytes, attr_dq)) return rc;
+    if (int rc = opt_in_smem_once(causal_bwd_dkv_kernel, kKvSmemBytes, attr_dkv)) return rc;
     const unsigned grid = (unsigned)(pl.npieces() * bh);
 
     // forward sweep: dQ, and dn_i, dl_i for the reverse sweep
@@ -965,6 +972,7 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.phi = p.phi;
     a.dim = (int)p.D;
     a.map = map ? 1 : 0;
+    a.stamp = sv ? (const int*)(sv + sl.stamp) : nullptr;
     prof_begin(kProfCausalBwdDq, st);
     CUtensorMap mDQ;
     if (int rc = encode_tile_map(&mDQ, dQ, rows, 32, (int)p.D)) return rc;      // one quadrant's rows per store

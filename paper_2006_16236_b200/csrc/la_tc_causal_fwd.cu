@@ -77,6 +77,7 @@ struct FwdParams {
     int phi;
     int dim;               // D = M: 64, or 32 (tiles zero-padded to 64 columns)
     int save;              // store the mapped phi(Q), phi(K) tiles for the backward pass
+    int* stamp;            // where the plan is recorded for the backward pass (in the saved buffer), or null
 };
 
 // ---------------------------------------------------------------------------
@@ -145,6 +146,12 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     if (warp == 16) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            if (prm.stamp && blockIdx.x == 0) {
+                int st[kPlanStampInts];
+                plan_stamp(plan, prm.dim, st);
+#pragma unroll
+                for (int i = 0; i < kPlanStampInts; ++i) prm.stamp[i] = st[i];
+            }
             prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV);
             #pragma unroll 1
             for (int c = 0; c < L; ++c) {
@@ -452,7 +459,8 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 }  // namespace
 
 CausalPlan choose_plan(const la_problem& p) {
-    constexpr int kSms = 148;
+    const int kSms = sm_count();
+    const PlanOverride ov = plan_override();        // A/B checks: a fixed number of equal pieces, a fixed short length
     CausalPlan pl;
     pl.chunks = (int)(p.N / kChunk);
     pl.bh = (int)(p.B * p.H);
@@ -460,8 +468,8 @@ CausalPlan choose_plan(const la_problem& p) {
     pl.m = 0;
     pl.spos = 0;
     pl.sub = 1;
-    const char* forced = getenv("LA_TC_NSEG");         // equal pieces, for A/B checks
-    int nlong = forced ? atoi(forced) : (pl.bh < 120 ? kSms / pl.bh : 1);
+    const bool forced = ov.causal_pieces > 0;
+    int nlong = forced ? ov.causal_pieces : (pl.bh < 120 ? kSms / pl.bh : 1);
     if (nlong > pl.chunks / 2) nlong = pl.chunks / 2;   // a piece is at least two chunks
     if (nlong < 1) nlong = 1;
     pl.nlong = nlong;
@@ -475,7 +483,7 @@ CausalPlan choose_plan(const la_problem& p) {
         const int rounds = (pl.bh + rest - 1) / rest;
         const double startup = 3.0;
         int m = (int)(((double)pl.chunks / nlong - (rounds - 1) * startup) / (rounds + 1.0 / nlong));
-        if (const char* e = getenv("LA_TC_SHORT")) m = atoi(e);        // A/B checks
+        if (ov.causal_short >= 0) m = ov.causal_short;
         if (m >= 4 && (pl.chunks - m) / nlong >= 2) {
             pl.m = m;
             pl.spos = nlong / 2;
@@ -518,11 +526,8 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     int* status = device_status_ptr();
     if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
 
-    static bool attr_done = false;
-    if (!attr_done) {
-        LA_CUDA_TRY(cudaFuncSetAttribute(causal_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-        attr_done = true;
-    }
+    static std::atomic<uint64_t> attr_done{0};
+    if (int rc = opt_in_smem_once(causal_fwd_kernel, kSmemBytes, attr_done)) return rc;
     // the pre-pass records go straight into the saved buffer when there is one
     float* records = sv ? (float*)(sv + sl.records) : (float*)ws;
     if (pl.npieces() > 1) {
@@ -543,6 +548,7 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     prm.phi = p.phi;
     prm.dim = (int)p.D;
     prm.save = save ? 1 : 0;
+    prm.stamp = sv ? (int*)(sv + sl.stamp) : nullptr;
     prof_begin(kProfCausalFwd, st);
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = chained_launch((unsigned)(pl.npieces() * pl.bh), kThreads, kSmemBytes, st, &attr);

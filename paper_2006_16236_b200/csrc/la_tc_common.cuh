@@ -3,6 +3,8 @@
 // for the feature map on a swizzled tile row.
 #pragma once
 
+#include <atomic>
+
 #include <cudaTypedefs.h>
 
 #include "la_common.cuh"
@@ -38,6 +40,29 @@ inline cudaLaunchConfig_t chained_launch(unsigned grid, unsigned block, size_t s
     cfg.numAttrs = 1;
     return cfg;
 }
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize belongs to a (function, device) pair: it is set the first
+// time a kernel is launched on each device (`done`: one bit per device ordinal, one word per kernel).
+template <typename Kernel>
+inline int opt_in_smem_once(Kernel kernel, size_t bytes, std::atomic<uint64_t>& done) {
+    int dev = 0;
+    LA_CUDA_TRY(cudaGetDevice(&dev));
+    const uint64_t bit = dev >= 0 && dev < 64 ? 1ull << dev : 0;
+    if (bit && (done.load(std::memory_order_acquire) & bit)) return LA_OK;
+    LA_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    done.fetch_or(bit, std::memory_order_release);
+    return LA_OK;
+}
+
+// SMs of the current device (148 on a B200; also the answer when no device can be asked, so that the
+// host-only plan and workspace queries work without one).
+int sm_count();
+
+// Overrides of the automatic piece / split plans, set through la_plan_override() (-1: automatic).
+struct PlanOverride {
+    int causal_pieces, causal_short, linear_splits;
+};
+PlanOverride plan_override();
 
 constexpr int kChunk = 128;                  // positions per chunk = MMA M
 constexpr int kDim = 64;                     // D = M = 64: one 128-byte swizzle row
@@ -117,15 +142,24 @@ int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap&
 // then reads the mapped tensors in place of Q and K, evaluates no exponential and skips its
 // own forward pre-pass; its results are the same bit for bit.
 struct SavedLayout {
-    size_t phiq, phik, records, bytes;      // byte offsets of the three parts; total size
+    size_t phiq, phik, records, stamp, bytes;      // byte offsets of the four parts; total size
 };
+// The forward also stamps the buffer with the plan it used (kPlanStampInts integers); a backward pass whose
+// own plan differs (an override changed in between, another device) reports kStatusPlanMismatch and
+// computes nothing, instead of reading records at offsets they were not written at.
+constexpr int kPlanStampInts = 8;
+__host__ __device__ inline void plan_stamp(const CausalPlan& pl, int dim, int (&out)[kPlanStampInts]) {
+    out[0] = 0x4c41504c;    // "LAPL"
+    out[1] = pl.chunks; out[2] = pl.bh; out[3] = pl.nlong; out[4] = pl.m; out[5] = pl.spos; out[6] = pl.sub; out[7] = dim;
+}
 inline SavedLayout saved_layout(const la_problem& p, const CausalPlan& pl) {
     const size_t rows = (size_t)(p.B * p.H * p.N);
     const size_t tensor = (rows * (size_t)p.D * 2 + 1023) & ~(size_t)1023;
     SavedLayout l;
     l.phiq = 0;
     l.phik = tensor;
-    l.records = 2 * tensor;
+    l.stamp = 2 * tensor;            // at an offset that does not depend on the plan
+    l.records = l.stamp + 1024;
     l.bytes = l.records + (pl.npieces() > 1 ? (size_t)(p.B * p.H) * pl.nparts() * kStateFloats * sizeof(float) : 0);
     return l;
 }

@@ -799,8 +799,8 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
 Segmentation choose_splits(const la_problem& p) {
     const int chunks = (int)(p.N / kChunk);
     const int64_t bh = p.B * p.H;
-    int nseg = (int)(148 / bh);
-    if (const char* e = getenv("LA_TC_SPLITS")) nseg = atoi(e);        // A/B checks
+    int nseg = (int)(sm_count() / bh);
+    if (plan_override().linear_splits > 0) nseg = plan_override().linear_splits;        // A/B checks
     if (nseg > chunks / 2) nseg = chunks / 2;
     if (nseg < 1) nseg = 1;
     const int cps = (chunks + nseg - 1) / nseg;
@@ -810,11 +810,8 @@ Segmentation choose_splits(const la_problem& p) {
 
 int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
                 const int* lengths, float* records, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        LA_CUDA_TRY(cudaFuncSetAttribute(linear_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLsSmemBytes));
-        attr_done = true;
-    }
+    static std::atomic<uint64_t> attr_done{0};
+    if (int rc = opt_in_smem_once(linear_sum_kernel, kLsSmemBytes, attr_done)) return rc;
     LsParams prm;
     prm.records = records;
     prm.lengths = lengths;
@@ -839,11 +836,8 @@ int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& 
 template <int kMode>
 int launch_apply(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
                  ApParams prm, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        LA_CUDA_TRY(cudaFuncSetAttribute(linear_apply_kernel<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kApSmemBytes));
-        attr_done = true;
-    }
+    static std::atomic<uint64_t> attr_done{0};          // one per instantiation (kMode)
+    if (int rc = opt_in_smem_once(linear_apply_kernel<kMode>, kApSmemBytes, attr_done)) return rc;
     prm.status = device_status_ptr();
     if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
     prm.heads = (int)p.H;

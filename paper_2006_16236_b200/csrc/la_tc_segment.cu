@@ -207,11 +207,8 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
 int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap& mapX, const CUtensorMap& mapY,
                    const float* dn, const float* dl, float* records, bool reverse, bool map, cudaStream_t st) {
     if (pl.npieces() <= 1) return LA_OK;
-    static bool attr_done = false;
-    if (!attr_done) {
-        LA_CUDA_TRY(cudaFuncSetAttribute(segment_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSumSmemBytes));
-        attr_done = true;
-    }
+    static std::atomic<uint64_t> attr_done{0};
+    if (int rc = opt_in_smem_once(segment_sum_kernel, kSumSmemBytes, attr_done)) return rc;
     SumParams prm;
     prm.records = records;
     prm.dn = dn;

@@ -81,22 +81,28 @@ def test_noncausal_forward_backward(shape, dtype):
     la.la_last_device_status()
 
 
-@pytest.mark.parametrize("plan", [{"LA_TC_NSEG": "1"}, {"LA_TC_NSEG": "3"}, {"LA_TC_NSEG": "5"}, {"LA_TC_SHORT": "0"},
-                                  {"LA_TC_SHORT": "4"}, {"LA_TC_SHORT": "7"}],
-                         ids=lambda d: ",".join(f"{k[6:].lower()}={v}" for k, v in d.items()))
+@pytest.fixture
+def plan_override():
+    """la_plan_override() for one test; the automatic plans are restored afterwards."""
+    yield la.la_plan_override
+    la.la_plan_override()
+
+
+@pytest.mark.parametrize("plan", [{"causal_pieces": 1}, {"causal_pieces": 3}, {"causal_pieces": 5}, {"causal_short": 0},
+                                  {"causal_short": 4}, {"causal_short": 7}],
+                         ids=lambda d: ",".join(f"{k[7:]}={v}" for k, v in d.items()))
 @pytest.mark.parametrize("keep", [False, True], ids=["recompute", "saved"])
-def test_causal_results_do_not_depend_on_the_piece_plan(monkeypatch, plan, keep):
+def test_causal_results_do_not_depend_on_the_piece_plan(plan_override, plan, keep):
     """The cut of a sequence into pieces and pre-pass parts (ragged lengths, a short middle piece, one piece)
     is an implementation choice: every plan has to give the oracle's result.  B*H = 64, 18 chunks."""
-    for k, v in plan.items():
-        monkeypatch.setenv(k, v)
+    plan_override(**plan)
     B, H, N, D = 4, 16, 18 * 128, 64
     p = la.make_problem(B, H, N, D, D, la.LA_BF16)
     pl = la.la_causal_plan(p)
-    if "LA_TC_NSEG" in plan:
-        assert pl["pieces"] == int(plan["LA_TC_NSEG"])
+    if "causal_pieces" in plan:
+        assert pl["pieces"] == plan["causal_pieces"]
     else:
-        short = int(plan["LA_TC_SHORT"])
+        short = plan["causal_short"]
         assert pl["pieces"] == (3 if short >= 4 else 2)
         if short >= 4:
             assert pl["piece_begin"][2] - pl["piece_begin"][1] == short
@@ -114,6 +120,37 @@ def test_causal_results_do_not_depend_on_the_piece_plan(monkeypatch, plan, keep)
         assert_close(dQ[sl], rq, torch.bfloat16, f"dQ[{b},{h}]", grad=True)
         assert_close(dK[sl], rk, torch.bfloat16, f"dK[{b},{h}]", grad=True)
         assert_close(dV[sl], rv, torch.bfloat16, f"dV[{b},{h}]", grad=True)
+
+
+def test_backward_refuses_a_saved_buffer_of_another_plan(plan_override):
+    """The saved buffer carries the plan of the forward pass that filled it.  A backward pass under another
+    plan would look for the pre-pass records at other offsets: it reports the mismatch and computes nothing."""
+    B, H, N, D = 4, 16, 18 * 128, 64
+    Q, K, V, G = draw_qkvg(B, H, N, D, D, seed=78, dtype=torch.bfloat16)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    p = la.make_problem(B, H, N, D, D, la.LA_BF16)
+    need = []
+    for pieces in (2, 3):
+        plan_override(causal_pieces=pieces)
+        need.append(la.la_workspace_bytes(p, la.LA_OP_CAUSAL_SAVED))
+    saved = torch.empty(max(need), dtype=torch.uint8, device=DEV)       # large enough under either plan
+    la.la_causal_forward(Qd, Kd, Vd, saved=saved)                       # ... filled under the plan of three pieces
+    plan_override(causal_pieces=2)
+    dQ = torch.full_like(Qd, 7.0)
+    la.la_causal_backward(Qd, Kd, Vd, Gd, saved=saved, dQ=dQ)
+    with pytest.raises(la.LaError) as e:
+        la.la_last_device_status()
+    assert e.value.status == -1 and "plan" in str(e.value)
+    assert torch.all(dQ == 7.0)                 # the forward sweep wrote nothing
+    la.la_last_device_status()                  # the flag is cleared, the context usable
+    plan_override(causal_pieces=3)
+    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd, saved=saved)
+    la.la_last_device_status()
+    sl = (slice(1, 2), slice(5, 6))
+    rq, rk, rv = oracle.linear_attention_backward(Q[sl], K[sl], V[sl], G[sl], True)
+    assert_close(dQ[sl], rq, torch.bfloat16, "dQ", grad=True)
+    assert_close(dK[sl], rk, torch.bfloat16, "dK", grad=True)
+    assert_close(dV[sl], rv, torch.bfloat16, "dV", grad=True)
 
 
 @pytest.mark.parametrize("causal", [True, False])

@@ -5,6 +5,7 @@ import os
 import re
 
 import pytest
+import torch
 
 import paper_2006_16236_b200 as la
 from paper_2006_16236_b200 import binding, build
@@ -79,7 +80,7 @@ def test_causal_plan_tiles_every_sequence(L, bh, chunks):
     assert all(lens[i] + 1 >= lens[i + 1] for i in range(n - 1))
     # work per SM: no more CTAs of the long kind than SMs
     nlong = sum(1 for x in lens if x + 1 >= lens[0])
-    assert bh * nlong <= 148 or n == 1 or nlong == 1 or os.environ.get("LA_TC_NSEG")
+    assert bh * nlong <= 148 or n == 1 or nlong == 1
 
 
 def test_causal_plan_of_the_bench_workload(L):
@@ -199,3 +200,61 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         binding.lib()
+
+
+def test_plan_override_is_an_explicit_call(L):
+    p = la.make_problem(4, 16, 18 * 128, 64, 64, la.LA_BF16)
+    auto = la.la_causal_plan(p)
+    try:
+        la.la_plan_override(causal_pieces=5)
+        assert la.la_causal_plan(p)["pieces"] == 5
+        la.la_plan_override(causal_short=0)
+        assert la.la_causal_plan(p)["pieces"] == 2
+        assert L.la_plan_override(0, -1, -1) == -1 and L.la_plan_override(-1, -2, -1) == -1
+    finally:
+        la.la_plan_override()
+    assert la.la_causal_plan(p) == auto
+
+
+def _cpu(shape, dtype=torch.float32):
+    return torch.zeros(shape, dtype=dtype)
+
+
+def test_binding_rejects_mismatched_tensors_before_any_pointer_is_taken():
+    """The kernels trust the problem descriptor, which the binding derives from Q and V: every other tensor
+    must agree with it.  CPU tensors throughout: a check that let one of these through would then stop at
+    "must live on a CUDA device", never at a launch."""
+    B, H, N, D, M = 2, 3, 16, 32, 16
+    Q, K, V, G = _cpu((B, H, N, D)), _cpu((B, H, N, D)), _cpu((B, H, N, M)), _cpu((B, H, N, M))
+    bad = [
+        (la.la_causal_forward, (Q, _cpu((B, H, N - 1, D)), V), {}, "K"),
+        (la.la_causal_forward, (Q, K.bfloat16(), V), {}, "K"),
+        (la.la_causal_forward, (Q, K, _cpu((B, H, N + 1, M))), {}, "V"),
+        (la.la_causal_forward, (Q, K, V), {"den": _cpu((B, H, N), torch.bfloat16)}, "den"),
+        (la.la_causal_forward, (Q, K, V), {"den": _cpu((B, H, N - 1))}, "den"),
+        (la.la_causal_forward, (Q, K, V), {"O": _cpu((B, H, N, D))}, "O"),
+        (la.la_causal_forward, (Q, K, V), {"S_out": _cpu((B, H, M, D))}, "S_out"),
+        (la.la_causal_forward, (Q, K, V), {"Z_in": _cpu((B, H, D), torch.float64), "S_in": _cpu((B, H, D, M))}, "Z_in"),
+        (la.la_causal_forward, (Q, K, V), {"saved": _cpu((64,))}, "saved"),
+        (la.la_causal_backward, (Q, K, V, _cpu((B, H, N, D))), {}, "G"),
+        (la.la_causal_backward, (Q, K, V, G), {"dK": _cpu((B, H, N, D), torch.bfloat16)}, "dK"),
+        (la.la_causal_backward, (Q, K, V, G), {"dS_in": _cpu((B, H, D))}, "dS_in"),
+        (la.la_linear_attention, (Q, K, V), {"KV": _cpu((B, H, D, M), torch.bfloat16)}, "KV"),
+        (la.la_linear_attention, (Q, K, V), {"Zs": _cpu((B, H, M))}, "Zs"),
+        (la.la_linear_attention_backward, (Q, K, V, G), {"dV": _cpu((B, H, N, D))}, "dV"),
+        (la.la_linear_attention_varlen, (Q, K, V, torch.zeros(B, dtype=torch.int64)), {}, "lengths"),
+        (la.la_linear_attention_noalloc, (Q, K, V), {"den": _cpu((B, H, N + 3))}, "den"),
+        (la.la_recurrent_step, (Q[:, :, 0], K[:, :, 0], V[:, :, 0], _cpu((B, H, D, M), torch.bfloat16), _cpu((B, H, D))), {}, "S"),
+        (la.la_recurrent_step, (Q[:, :, 0], K[:, :, 1:3, 0], V[:, :, 0], _cpu((B, H, D, M)), _cpu((B, H, D))), {}, "k"),
+        (la.la_recurrent_steps, (Q, K, V, _cpu((B, H, D, M)), _cpu((B, H, M))), {}, "Z"),
+        (la.la_feature_map, (Q,), {"out": _cpu((B, H, N, D), torch.bfloat16)}, "out"),
+        (la.la_feature_map_poly2, (_cpu((B, N, 4)),), {"out": _cpu((B, N, 8))}, "out"),
+    ]
+    for fn, args, kw, name in bad:
+        with pytest.raises(ValueError, match=name):
+            fn(*args, **kw)
+    # well-formed arguments get as far as the device check and no further
+    for fn, args in ((la.la_causal_forward, (Q, K, V)), (la.la_causal_backward, (Q, K, V, G)),
+                     (la.la_linear_attention, (Q, K, V)), (la.la_feature_map, (Q,))):
+        with pytest.raises(ValueError, match="CUDA device"):
+            fn(*args)
