@@ -12,6 +12,28 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (sm_100a)")
 
 
+def pytest_sessionfinish(session, exitstatus):
+    """After a GPU session: the three error figures of every comparison with the oracle, worst case per tensor
+    name and dtype, as a text table under gpurun_out/ (the scratch folder of a GPU run)."""
+    try:
+        from parity import parity_report
+    except ImportError:
+        return
+    out_dir = os.path.join(ROOT, "gpurun_out")
+    if not parity_report or not os.path.isdir(out_dir):
+        return
+    worst = {}
+    for what, dtype, shape, row, gated, rms in parity_report:
+        import re
+        key = (re.sub(r"(, length|step) \d+", r"\1 *", what.split("[")[0]), dtype)
+        w = worst.setdefault(key, [0.0, 0.0, 0.0, 0])
+        w[0], w[1], w[2], w[3] = max(w[0], row), max(w[1], gated), max(w[2], rms), w[3] + 1
+    with open(os.path.join(out_dir, "parity_report.txt"), "w") as f:
+        f.write("tensor dtype comparisons row gated rms   (maxima over all comparisons of the session)\n")
+        for (what, dtype), (row, gated, rms, n) in sorted(worst.items()):
+            f.write(f"{what or '-'} {dtype} {n} {row:.3e} {gated:.3e} {rms:.3e}\n")
+
+
 def load_rational_fixture(name):
     """Parse tests/golden/<name>: 'label rows cols' headers followed by rationals."""
     from fractions import Fraction

@@ -1,31 +1,43 @@
-"""Error measure and tolerances shared by the GPU parity tests.
+"""Error measures and tolerances of the GPU parity tests: the one place they are defined.
 
-Every output is a set of vectors, one per position (a row of O, dQ, dK, dV, a row of
-the state, ...; a [B,H,N] tensor such as den is a set of 1-vectors).  "Relative error" is
-taken per position in the max norm,
+Every output is a set of vectors, one per position (a row of O, dQ, dK, dV, a row of the
+state; a [B,H,N] tensor such as den is a set of 1-vectors).  Three figures are computed
+for every comparison, all of them maxima over the whole tensor:
 
-    err = max over positions i of  ||x_i - r_i||_inf / scale_i ,
-    scale_i = max(||r_i||_inf, median of ||r_j||_inf over the 33 positions around i),
+  row      ||x_i - r_i||_inf / ||r_i||_inf per position i: the largest deviation of any
+           element relative to the largest element of the vector it belongs to.  Rows of
+           the reference that are exactly zero (the gradient of the first causal query:
+           O_1 = V_1 whatever Q_1 is; a whole tensor when N = 1) have no scale of their
+           own and are compared against the largest row of the tensor.
+  gated    the same with scale_i = max(||r_i||_inf, median of ||r_j||_inf over the 33
+           positions around i).  The neighbourhood median only matters for a row much
+           smaller than its neighbours.  Such rows exist by chance, not only analytically:
+           with nearly uniform attention (the speech-shaped workload scales its inputs by
+           1/8) a gradient row is close to c_i (1,...,1) with c_i of either sign, and among
+           10^5 rows some c_i fall within 10^-4 of zero.  The error of such a row is set
+           by the terms that cancel in it, which have the size of the rows next to it, so
+           that is the scale it is judged against.  For O and den the floor is inert in
+           every test (|O_i| is an average of values, den_i > 0 grows with i: no row is
+           small against its neighbours); it is applied uniformly so that there is one
+           measure, not one per tensor.
+  rms      element-wise |x - r| / max(|r|, rms of r over the row), rows floored as in
+           `gated`: every element against its own size, small elements against the row.
 
-the largest deviation of any element, relative to the largest element of the vector
-it belongs to.  The median over the neighbouring positions only matters for a vector
-that is much smaller than its neighbours: a row that vanishes analytically (the
-gradient of the first causal query: O_1 = V_1 whatever Q_1 is) or by chance (with
-nearly uniform attention a gradient row is close to c_i (1,...,1) with c_i of either
-sign, and among thousands of rows some c_i fall arbitrarily close to 0); such a row
-has no scale of its own and is judged against the rows next to it.  A tensor that is
-zero altogether (N = 1) is compared absolutely.  Gates: 1e-4 for fp32 I/O, 2e-2 for
-bf16 I/O (fp32 accumulation); inputs are rounded to the I/O type once and both sides
-consume those rounded values.
-
-A stricter element-wise variant, |x - r| / max(|r|, rms of r over the row), is also
-computed (`max_rel_err_rms`).  fp32 results and the bf16 forward outputs meet the same
-gates under it; bf16 gradients are allowed 5e-2 there: every gradient element is a
-difference of terms about 2.4 times its own size (the gradient of a normalised
-average is orthogonal to phi(Q_i)), each term carries the 2^-9 rounding of the bf16
-tensor-core operands, and the maximum over 10^7..10^8 elements sits 5-6 standard
-deviations out, which lands at 2-3e-2 of the row rms for any implementation that
-feeds bf16 phi(Q), phi(K) tiles to the tensor cores.
+Gates (TOL): `gated` <= 1e-4 for fp32 I/O and <= 2e-2 for bf16 I/O (fp32 accumulation),
+for every tensor; inputs are rounded to the I/O type once and both sides consume the
+rounded values.  `rms` is held to the same gates for fp32 and for the bf16 forward
+outputs, and to 5e-2 for bf16 gradients (TOL_RMS_GRAD).  That last figure is a measured
+floor plus head-room, not a convenience: tests/test_parity_floor.py takes the fp64 oracle
+and rounds nothing but the two tensor-core operands phi(Q), phi(K) to bf16 (no rounded
+scores, states or outputs), and already reads 2.0e-2 to 2.5e-2 under `rms` for dQ and
+1.5e-2 to 2.4e-2 for dK on a few heads of the benchmark shapes (every gradient element is
+a difference of terms about 2.4 times its own size, each carrying the 2^-9 operand
+rounding: sigma = 0.34 % of the row rms, and the maximum over 10^6..10^8 elements sits 6-7
+sigma out).  Any kernel that feeds bf16 feature tiles to the tensor cores inherits that
+floor; the kernels here measure 3.2e-2 (dQ) and 2.9e-2 (dK) at full size with all of
+their roundings.  `row` is reported for every comparison (parity_report); it is gated at
+TOL where the inputs have unit scale (the causal benchmark workloads at full size: 1.6e-2
+at most for bf16 gradients) and left ungated where rows vanish by chance.
 """
 import numpy as np
 import torch
@@ -33,18 +45,30 @@ import torch
 TOL = {torch.float32: 1e-4, torch.bfloat16: 2e-2}
 TOL_RMS_GRAD = {torch.float32: 1e-4, torch.bfloat16: 5e-2}
 
+# (what, dtype, row, gated, rms) of every assert_close() of this process, for the report
+# that tests/conftest.py writes at the end of a GPU session
+parity_report = []
+
 
 def _as_f64(x):
     return x.detach().double().cpu().numpy() if hasattr(x, "detach") else np.asarray(x, np.float64)
 
 
-def _row_floor(ref, row_scale):
+def _shaped(x, ref):
+    x, ref = _as_f64(x), np.asarray(ref, np.float64)
+    assert x.shape == ref.shape, (x.shape, ref.shape)
+    if ref.ndim == 3:                                         # [B,H,N]: one scalar per position
+        x, ref = x[..., None], ref[..., None]
+    return x, ref
+
+
+def _row_floor(ref, row_scale, neighbours=True):
     """row_scale: [..., N, 1] norm of each position's vector -> the scale it is judged against."""
-    from scipy.ndimage import median_filter
     biggest = np.abs(ref).max()
     if biggest < 1e-12:                                       # whole tensor analytically zero (N = 1)
         return np.ones_like(row_scale)
-    if row_scale.shape[-2] > 1:
+    if neighbours and row_scale.shape[-2] > 1:
+        from scipy.ndimage import median_filter
         size = [1] * row_scale.ndim
         size[-2] = 33
         row_scale = np.maximum(row_scale, median_filter(row_scale, size=size, mode="mirror"))
@@ -52,37 +76,50 @@ def _row_floor(ref, row_scale):
 
 
 def max_rel_err(x, ref) -> float:
-    """Per-position relative error in the max norm (the gated measure)."""
-    x, ref = _as_f64(x), np.asarray(ref, np.float64)
-    assert x.shape == ref.shape, (x.shape, ref.shape)
+    """`gated`: per-position relative error in the max norm, small rows judged against their neighbours."""
+    if np.asarray(ref).ndim == 1:                             # element-wise map: plain relative error
+        x, ref = _as_f64(x), np.asarray(ref, np.float64)
+        assert x.shape == ref.shape, (x.shape, ref.shape)
+        return float((np.abs(x - ref) / np.maximum(np.abs(ref), 1e-30)).max()) if x.size else 0.0
+    x, ref = _shaped(x, ref)
     if x.size == 0:
         return 0.0
     assert np.isfinite(x).all(), "non-finite values in the result"
-    if ref.ndim == 1:                                         # element-wise map: plain relative error
-        return float((np.abs(x - ref) / np.maximum(np.abs(ref), 1e-30)).max())
-    if ref.ndim == 3:                                         # [B,H,N]: one scalar per position
-        x, ref = x[..., None], ref[..., None]
     floor = _row_floor(ref, np.abs(ref).max(axis=-1, keepdims=True))
     return float((np.abs(x - ref) / floor).max())
 
 
-def max_rel_err_rms(x, ref) -> float:
-    """Element-wise |x - r| / max(|r|, rms of r over the row)."""
-    x, ref = _as_f64(x), np.asarray(ref, np.float64)
+def max_rel_err_row(x, ref) -> float:
+    """`row`: the same with every non-zero row judged against itself alone."""
+    if np.asarray(ref).ndim == 1:
+        return max_rel_err(x, ref)
+    x, ref = _shaped(x, ref)
     if x.size == 0:
         return 0.0
-    if ref.ndim == 1:
+    floor = _row_floor(ref, np.abs(ref).max(axis=-1, keepdims=True), neighbours=False)
+    return float((np.abs(x - ref) / floor).max())
+
+
+def max_rel_err_rms(x, ref) -> float:
+    """`rms`: element-wise |x - r| / max(|r|, rms of r over the row)."""
+    if np.asarray(ref).ndim == 1:
         return max_rel_err(x, ref)
-    if ref.ndim == 3:
-        x, ref = x[..., None], ref[..., None]
+    x, ref = _shaped(x, ref)
+    if x.size == 0:
+        return 0.0
     rms = _row_floor(ref, np.sqrt((ref ** 2).mean(axis=-1, keepdims=True)))
     return float((np.abs(x - ref) / np.maximum(np.abs(ref), rms)).max())
 
 
-def assert_close(x, ref, dtype, what="", grad=False):
+def assert_close(x, ref, dtype, what="", grad=False, gate_row=False):
+    """gate_row: also hold the plain per-row figure (no neighbourhood floor) to TOL; used where no row of the
+    reference is small by chance (the benchmark workloads with inputs of unit scale)."""
     err = max_rel_err(x, ref)
-    assert err <= TOL[dtype], f"{what}: max relative error {err:.3e} > {TOL[dtype]:.0e}"
     strict = max_rel_err_rms(x, ref)
+    row = max_rel_err_row(x, ref)
+    parity_report.append((what, str(dtype).replace("torch.", ""), tuple(np.asarray(ref).shape), row, err, strict))
+    assert err <= TOL[dtype], f"{what}: max relative error {err:.3e} > {TOL[dtype]:.0e}"
+    assert not gate_row or row <= TOL[dtype], f"{what}: max relative error of a row against itself {row:.3e} > {TOL[dtype]:.0e}"
     gate = TOL_RMS_GRAD[dtype] if grad else TOL[dtype]
     assert strict <= gate, f"{what}: element-wise error over the row rms {strict:.3e} > {gate:.0e}"
     return err

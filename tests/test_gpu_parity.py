@@ -537,10 +537,12 @@ def test_causal_workloads_full_size(name, keep):
         sl = (slice(b, b + 1), slice(h, h + 1))
         q, k, v, g = Q[sl], K[sl], V[sl], G[sl]
         Or, denr = oracle.linear_attention(q, k, v, True)
-        assert_close(O[sl], Or, dtype, f"{name} O[{b},{h}]")
-        assert_close(den[sl], denr, dtype, f"{name} den[{b},{h}]")
+        # unit-scale inputs: no row of any reference tensor is small by chance, so every row is also held to
+        # the tolerance against itself alone (no neighbourhood floor)
+        assert_close(O[sl], Or, dtype, f"{name} O[{b},{h}]", gate_row=True)
+        assert_close(den[sl], denr, dtype, f"{name} den[{b},{h}]", gate_row=True)
         for got, ref, nm in zip((dQ, dK, dV), oracle.linear_attention_backward(q, k, v, g, True), "QKV"):
-            assert_close(got[sl], ref, dtype, f"{name} d{nm}[{b},{h}]", grad=True)
+            assert_close(got[sl], ref, dtype, f"{name} d{nm}[{b},{h}]", grad=True, gate_row=True)
     # size-independent properties on the whole result
     assert torch.isfinite(O.float()).all() and torch.isfinite(dQ.float()).all()
     assert torch.allclose(O[:, :, 0].float(), Vd[:, :, 0].float(), rtol=1e-2, atol=1e-2)     # O_1 = V_1
