@@ -27,7 +27,10 @@ namespace sm100 {
 // Give-up limit of every spin wait.  With the back-off below one try costs on the
 // order of 100 ns or more, so the limit is a few hundred milliseconds: far beyond any
 // legitimate wait, short enough to return control to the host.
-constexpr uint32_t kWaitLimit = 4u << 20;
+#ifndef LA_WAIT_LIMIT
+#define LA_WAIT_LIMIT (4u << 20)        // a test of the give-up path builds with a small limit
+#endif
+constexpr uint32_t kWaitLimit = LA_WAIT_LIMIT;
 
 constexpr int kStatusTmaTimeout = 1;
 constexpr int kStatusMmaTimeout = 2;
