@@ -36,14 +36,16 @@ METRIC = "causal LA fwd+bwd tokens/s"
 DEFAULT_WORKLOAD = "causal_sweep_bf16_N16384"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from an
-# ncu capture summarised under profiles/), keyed by workload; None until captured.
-NCU_TRAFFIC_BYTES = {
-    # profiles/ncu_full_causal_kernels_N16384.md
-    ("causal_sweep_bf16_N16384", "causal_fwd_kernel"): 766_838_528,      # includes 268 MB of saved phi(Q), phi(K)
-    ("causal_sweep_bf16_N16384", "causal_bwd_dq_kernel"): 667_496_448,
-    ("causal_sweep_bf16_N16384", "causal_bwd_dkv_kernel"): 789_536_256,
-}
+def ncu_traffic():
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the library's kernels, by
+    workload and kernel, as the last ncu capture of this source tree recorded them in a tracked JSON file
+    (written by `python -m paper_2006_16236_b200.ncu_summary`); {} when there is none."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f)
+    except (OSError, ValueError):
+        return {}
 
 
 def peaks():
@@ -343,11 +345,18 @@ def bench_attention(la, w, dev, steps, warmup, world, rank, pk, do_e2e=True, fro
         dom_ms = max(bwd_ms, fwd_ms)
         dom_bytes = algorithmic_bytes(w, "bwd" if bwd_ms >= fwd_ms else "fwd")
     ach = dom_bytes / dom_ms * 1e-6
+    traffic = ncu_traffic()
     res["roofline"] = {
         "kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
         "peak_source": pk["source"] + " copy bandwidth (burst figure: the kernel is timed alone by its own event pair)",
         "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms,
-        "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
+        "traffic": traffic.get("bytes_per_launch", {}).get(w.name, {}).get(dom),
+        "traffic_source": traffic.get("source"),
+        # the whole step against the same peak: every input of forward + backward read once, every output written
+        # once (4De+4 and 7De+4 bytes per token-head), over the time of the step.  `frac` above is the dominant
+        # kernel on the bytes that kernel has to move; the second sweep's re-reads, the saved tiles and the
+        # pre-passes only show here.
+        "step_frac": res["hbm_frac"], "step_algorithmic_bytes": algorithmic_bytes(w, "both"), "step_ms": ms,
     }
     if do_e2e:
         e_steps = max(4, min(steps, 10))
@@ -395,6 +404,21 @@ def bench_decode(la, w, dev, pk, n_steps=None, batch=None):
     for t in range(16):
         la.la_recurrent_step(q_t[t], k_t[t], v_t[t], S, Z, out=out[t])
     us_eager = timed(run_all)
+    # the same loop as a C caller would issue it: the exported function with ready-made arguments, none of the
+    # binding's per-call checks and allocations
+    import ctypes
+    from paper_2006_16236_b200 import binding
+    fn = binding.lib().la_recurrent_step
+    pr = ctypes.byref(binding.make_problem(w.B, w.H, 1, w.D, w.M, binding.LA_BF16 if w.dtype == "bf16" else binding.LA_F32))
+    vp = ctypes.c_void_p
+    argv = [(vp(q_t[t].data_ptr()), vp(k_t[t].data_ptr()), vp(v_t[t].data_ptr()), vp(out[t].data_ptr())) for t in range(T)]
+    Sp, Zp, st = vp(S.data_ptr()), vp(Z.data_ptr()), vp(torch.cuda.current_stream().cuda_stream)
+
+    def run_raw():
+        for q, k, v, o in argv:
+            fn(pr, q, k, v, Sp, Zp, o, st)
+
+    us_raw = timed(run_raw)
     us_graph = None
     try:
         side = torch.cuda.Stream()
@@ -410,10 +434,10 @@ def bench_decode(la, w, dev, pk, n_steps=None, batch=None):
         us_graph = None
         graph_error = repr(exc)
     la.la_last_device_status()
-    us = min(us_eager, us_graph) if us_graph else us_eager
+    us = min(us_eager, us_raw, us_graph) if us_graph else min(us_eager, us_raw)
     gbs = algorithmic_bytes(w, "both") / us * 1e-3
     res = {"workload": w.name, "steps_per_s": 1e6 / us, "us_per_step": us, "launches": T,
-           "us_per_step_host_issued": us_eager, "us_per_step_cuda_graph": us_graph,
+           "us_per_step_host_issued": us_eager, "us_per_step_host_issued_raw_c_abi": us_raw, "us_per_step_cuda_graph": us_graph,
            "alg_gbs": gbs, "hbm_frac": gbs / pk["hbm_gbs"], "state_bytes": S.numel() * 4,
            "note": ("state fits the 126 MB L2, so the fraction may exceed the DRAM roofline"
                     if S.numel() * 4 < 100e6 else "state exceeds L2: every step streams it from and to HBM")}
@@ -500,9 +524,20 @@ def cpu_baseline(w, budget_s=15.0):
         oracle_step(oracle, w, data)
     dt = (time.perf_counter() - t0) / reps
     frac = cores / (w.B * w.H)
+    # the same on one thread, on one (batch, head) pair
+    one = [t[:, :1] for t in data]
+    oracle.set_threads(1)
+    try:
+        t0 = time.perf_counter()
+        oracle_step(oracle, w, one)
+        dt1 = time.perf_counter() - t0
+    finally:
+        oracle.set_threads(cores)
     return {"value": w.tokens * frac / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle",
             "sample": f"{cores} of {w.B * w.H} (batch, head) pairs of {w.name}, fwd+bwd, {reps} repetitions; "
-                      "rate scaled to whole-workload tokens"}
+                      "rate scaled to whole-workload tokens",
+            "one_thread": {"value": w.tokens / (w.B * w.H) / dt1, "unit": "tokens/s", "cores": 1,
+                           "sample": f"1 of {w.B * w.H} (batch, head) pairs, fwd+bwd, once; rate scaled to whole-workload tokens"}}
 
 
 def run_reference(args):
@@ -550,6 +585,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[k for k, v in WORKLOADS.items() if v.kind != "decode"])
     ap.add_argument("--main-only", action="store_true", help="skip the other hot-path rows and the CPU baseline")
+    ap.add_argument("--decode-only", type=int, default=0, metavar="T",
+                    help="only the recurrent-decode rows, T steps each (a short run for a profiler capture)")
+    ap.add_argument("--decode-batch", type=int, default=0, metavar="B",
+                    help="with --decode-only: only the row with B streams per head (default: 256 and 2048)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -566,6 +605,12 @@ def main():
     pk = peaks()
     w = WORKLOADS[args.workload]
 
+    if args.decode_only:
+        dw = next(v for v in WORKLOADS.values() if v.kind == "decode")
+        batches = [args.decode_batch] if args.decode_batch else [dw.B, 2048]
+        print(json.dumps({"rows": {f"{dw.name}_B{b}": bench_decode(la, dw, dev, pk, n_steps=args.decode_only, batch=b)
+                                   for b in batches}}))
+        return
     main_res = bench_attention(la, w, dev, args.steps, args.warmup, world, rank, pk)
 
     rows = {}
