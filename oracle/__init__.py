@@ -233,3 +233,25 @@ def poly2_attention(Q, K, V, causal: bool, eps: float = 0.0):
                 A = np.tril(A)
             O[b, h] = (A @ V[b, h]) / (A.sum(axis=1, keepdims=True) + eps)
     return O
+
+
+# ---------------------------------------------------------------------------
+# One decode step of a whole attention sublayer, Eq. 16-20 with the projections written out:
+#   q = x W_Q, k = x W_K, v = x W_V (split into H heads), s_i = s_{i-1} + phi(k) v^T, z_i = z_{i-1} + phi(k),
+#   a = phi(q)^T s_i / (phi(q)^T z_i + eps) per head,  y = a W_O + x.
+# The feed-forward part f_l of Eq. 20 stays with the caller (it acts on each position alone).  The
+# projections are numpy matrix products; the state update and read-out are recurrent_step above.
+# ---------------------------------------------------------------------------
+def decode_layer_step(x, Wq, Wk, Wv, Wo, S, Z, phi: str = "elu1", eps: float = 0.0):
+    """x [B,F]; Wq, Wk [F,H*D], Wv [F,H*M], Wo [H*M,F] (float64, applied as x @ W); S [B,H,D,M] and Z [B,H,D]
+    (contiguous float64) are updated IN PLACE.  Returns y [B,F]."""
+    x, Wq, Wk, Wv, Wo = (_f64(t) for t in (x, Wq, Wk, Wv, Wo))
+    B, H, D, M = S.shape
+    if x.ndim != 2 or x.shape[0] != B or Wq.shape != (x.shape[1], H * D) or Wk.shape != Wq.shape \
+            or Wv.shape != (x.shape[1], H * M) or Wo.shape != (H * M, x.shape[1]):
+        raise ValueError("shape mismatch between x, the projections and the state")
+    q = (x @ Wq).reshape(B, H, D)
+    k = (x @ Wk).reshape(B, H, D)
+    v = (x @ Wv).reshape(B, H, M)
+    a = recurrent_step(q, k, v, S, Z, phi, eps)
+    return a.reshape(B, H * M) @ Wo + x

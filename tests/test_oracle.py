@@ -429,3 +429,55 @@ def test_poly2_backward_matches_finite_differences():
             Xm[idx] -= h
             fd = (loss(Xp, K) - loss(Xm, K)) / (2 * h) if which == 0 else (loss(Q, Xp) - loss(Q, Xm)) / (2 * h)
             assert abs(fd - dX[idx]) <= 1e-6 * max(1.0, abs(fd)), (which, idx, fd, dX[idx])
+
+
+# ---------------------------------------------------------------------------
+# Decode step of a whole attention sublayer (Eq. 16-20 with the projections)
+# ---------------------------------------------------------------------------
+def _layer_weights(F, H, D, M, seed):
+    rng = np.random.default_rng(seed)
+    s = 1.0 / np.sqrt(F)
+    return (rng.standard_normal((F, H * D)) * s, rng.standard_normal((F, H * D)) * s,
+            rng.standard_normal((F, H * M)) * s, rng.standard_normal((H * M, F)) * s)
+
+
+def test_decode_layer_unrolled_equals_the_parallel_form_on_projected_inputs():
+    """T steps of the layer, one position at a time, against Eq. 2's projections followed by the causal
+    N x N definition (Eq. 8 with the feature-map kernel) and the output projection with its residual."""
+    B, H, D, M, T = 3, 2, 4, 5, 9
+    F = 6
+    Wq, Wk, Wv, Wo = _layer_weights(F, H, D, M, 1)
+    X = np.random.default_rng(2).standard_normal((B, T, F))
+    S, Z = np.zeros((B, H, D, M)), np.zeros((B, H, D))
+    ys = np.stack([oracle.decode_layer_step(X[:, t], Wq, Wk, Wv, Wo, S, Z) for t in range(T)], 1)
+    heads = lambda A, W, E: (A @ W).reshape(B, T, H, E).transpose(0, 2, 1, 3)
+    O = oracle.attention_quadratic(heads(X, Wq, D), heads(X, Wk, D), heads(X, Wv, M), True)
+    want = O.transpose(0, 2, 1, 3).reshape(B, T, H * M) @ Wo + X
+    np.testing.assert_allclose(ys, want, rtol=1e-11, atol=1e-12)
+
+
+def test_decode_layer_special_cases():
+    B, H, D, M, F = 2, 2, 3, 3, 6
+    Wq, Wk, Wv, Wo = _layer_weights(F, H, D, M, 3)
+    x = np.random.default_rng(4).standard_normal((B, F))
+    # a zero output projection leaves the residual alone, and the state still advances by phi(k) v^T
+    S, Z = np.zeros((B, H, D, M)), np.zeros((B, H, D))
+    y = oracle.decode_layer_step(x, Wq, Wk, Wv, np.zeros_like(Wo), S, Z)
+    np.testing.assert_array_equal(y, x)
+    k, v = (x @ Wk).reshape(B, H, D), (x @ Wv).reshape(B, H, M)
+    np.testing.assert_allclose(S, oracle.feature_map(k)[..., None] * v[:, :, None, :], rtol=1e-13)
+    np.testing.assert_allclose(Z, oracle.feature_map(k), rtol=1e-13)
+    # identity projections (F = H D = H M): the layer is the bare recurrent step plus the residual, and the
+    # first step of a fresh sequence returns its own value (O_1 = V_1), so y = 2 x
+    I = np.eye(F)
+    S, Z = np.zeros((B, H, D, M)), np.zeros((B, H, D))
+    np.testing.assert_allclose(oracle.decode_layer_step(x, I, I, I, I, S, Z), 2 * x, rtol=1e-13)
+    # by hand: one stream, one head, D = M = 1, all weights 1/2, x = (2): q = k = v = 1, phi = 2,
+    # s = 2 * 1 = 2, z = 2, a = (2 * 2) / (2 * 2) = 1, y = 1 * 1/2 + 2 = 5/2; second step x = (-2): q = k = v = -1,
+    # phi = e^-1, s = 2 - e^-1, z = 2 + e^-1, a = s / z, y = a / 2 - 2
+    S, Z = np.zeros((1, 1, 1, 1)), np.zeros((1, 1, 1))
+    h = np.full((1, 1), 0.5)
+    assert oracle.decode_layer_step(np.array([[2.0]]), h, h, h, h, S, Z)[0, 0] == 2.5
+    e = np.exp(-1.0)
+    y2 = oracle.decode_layer_step(np.array([[-2.0]]), h, h, h, h, S, Z)[0, 0]
+    np.testing.assert_allclose(y2, 0.5 * (2 - e) / (2 + e) - 2, rtol=1e-14)
