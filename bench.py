@@ -469,6 +469,88 @@ def bench_decode(la, w, dev, pk, n_steps=None, batch=None):
     return res
 
 
+def bench_decode_layer(la, w, dev, pk, T=512):
+    """T tokens through la_decode_layer_step (projections + recurrent step + output projection + residual per
+    token), each token's input being the previous token's output (two buffers alternate), as in generation:
+    issued call by call through the binding, through the raw C ABI, and replayed from a CUDA graph."""
+    import ctypes
+    from paper_2006_16236_b200 import binding
+    B, H, D = w.B, w.H, w.D
+    F = H * D
+    g = torch.Generator().manual_seed(w.seed + 3)
+    s = 1.0 / F ** 0.5
+    Wqkv = (torch.randn((3 * F, F), generator=g) * s).to(torch.bfloat16).to(dev)
+    Wo = (torch.randn((F, F), generator=g) * s * 0.1).to(torch.bfloat16).to(dev)
+    x0 = torch.randn((B, F), generator=g).to(torch.bfloat16).to(dev)
+    buf = [x0.clone(), torch.empty_like(x0)]
+    S = torch.zeros((B, H, D, D), device=dev)
+    Z = torch.zeros((B, H, D), device=dev)
+    p = la.make_problem(B, H, 1, D, D, la.LA_BF16)
+    ws = la.workspace(p, la.LA_OP_DECODE_LAYER, dev)
+
+    def reset():
+        buf[0].copy_(x0)
+        S.zero_()
+        Z.zero_()
+
+    def run_binding():
+        for t in range(T):
+            la.la_decode_layer_step(buf[t & 1], Wqkv, Wo, S, Z, out=buf[(t + 1) & 1], ws=ws)
+
+    fn = binding.lib().la_decode_layer_step
+    vp = ctypes.c_void_p
+    pr, st = ctypes.byref(p), vp(torch.cuda.current_stream().cuda_stream)
+    args = [(vp(buf[t & 1].data_ptr()), vp(buf[(t + 1) & 1].data_ptr())) for t in range(2)]
+    fixed = (vp(Wqkv.data_ptr()), vp(Wo.data_ptr()), vp(S.data_ptr()), vp(Z.data_ptr()))
+    wsp, wsn = vp(ws.data_ptr()), ws.numel()
+
+    def run_raw(stream=st):
+        for t in range(T):
+            x, y = args[t & 1]
+            fn(pr, x, fixed[0], fixed[1], fixed[2], fixed[3], y, wsp, wsn, stream)
+
+    def timed(fnc):
+        reset()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fnc()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / T
+
+    run_raw()
+    res = {"workload": f"decode_layer_B{B}_H{H}_D{D}", "tokens": T, "launches_per_token": 3,
+           "us_per_token_host_issued": timed(run_binding), "us_per_token_host_issued_raw_c_abi": timed(run_raw)}
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                run_raw(vp(side.cuda_stream))
+        torch.cuda.current_stream().wait_stream(side)
+        timed(graph.replay)
+        res["us_per_token_cuda_graph"] = timed(graph.replay)
+    except Exception as exc:  # noqa: BLE001 - report, keep the eager numbers
+        res["graph_error"] = repr(exc)
+    la.la_profile_enable(True)
+    reset()
+    run_raw()
+    torch.cuda.synchronize()
+    res["kernels_us"] = {k: round(v[0] * 1e3, 2) for k, v in la.la_profile_read().items() if v[1]}
+    la.la_profile_enable(False)
+    la.la_last_device_status()
+    best = min(v for k, v in res.items() if k.startswith("us_per_token"))
+    res["tokens_per_s_per_stream"] = 1e6 / best
+    # the bytes a token has to move: the fp32 state read and written once, the weights read once, x in, y out
+    nbytes = B * H * (8 * D * D + 8 * D) + 4 * F * F * 2 + 2 * B * F * 2
+    res["alg_gbs"] = nbytes / best * 1e-3
+    res["hbm_frac"] = res["alg_gbs"] / pk["hbm_gbs"]
+    res["note"] = "state (32 MiB) and weights (2 MiB) fit the L2: the fraction is against the HBM copy bandwidth for scale only"
+    return res
+
+
 # --------------------------------------------------------------------------- CPU oracle arm
 def bench_poly2(la, w, dev, pk, iters=10):
     """Degree-2 polynomial feature map (Section 3.2.1) and its gradient on the headline workload's rows with
@@ -608,8 +690,10 @@ def main():
     if args.decode_only:
         dw = next(v for v in WORKLOADS.values() if v.kind == "decode")
         batches = [args.decode_batch] if args.decode_batch else [dw.B, 2048]
-        print(json.dumps({"rows": {f"{dw.name}_B{b}": bench_decode(la, dw, dev, pk, n_steps=args.decode_only, batch=b)
-                                   for b in batches}}))
+        rows = {f"{dw.name}_B{b}": bench_decode(la, dw, dev, pk, n_steps=args.decode_only, batch=b) for b in batches}
+        if not args.decode_batch:
+            rows["decode_layer"] = bench_decode_layer(la, dw, dev, pk, T=args.decode_only)
+        print(json.dumps({"rows": rows}))
         return
     main_res = bench_attention(la, w, dev, args.steps, args.warmup, world, rank, pk)
 
@@ -622,6 +706,7 @@ def main():
             if ww.kind == "decode":
                 rows[name] = bench_decode(la, ww, dev, pk)
                 rows[name + "_B2048"] = bench_decode(la, ww, dev, pk, n_steps=256, batch=2048)
+                rows["decode_layer"] = bench_decode_layer(la, ww, dev, pk)
             else:
                 r = bench_attention(la, ww, dev, k, wu, 1, 0, pk, do_e2e=False)
                 rows[name] = {kk: r[kk] for kk in ("value", "ms_per_step", "fwd_ms", "bwd_ms", "alg_gbs", "hbm_frac",

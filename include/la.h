@@ -68,7 +68,8 @@ typedef enum {
     LA_OP_CAUSAL_SAVED = 4,      /* size of the optional `saved` buffer, see la_causal_forward() */
     LA_OP_LINEAR_VARLEN_FORWARD = 5,     /* la_linear_attention_varlen()          */
     LA_OP_LINEAR_VARLEN_BACKWARD = 6,    /* la_linear_attention_varlen_backward() */
-    LA_OP_LINEAR_SAVED = 7               /* size of the optional `saved` buffer, see la_linear_attention_keep() */
+    LA_OP_LINEAR_SAVED = 7,              /* size of the optional `saved` buffer, see la_linear_attention_keep() */
+    LA_OP_DECODE_LAYER = 8               /* la_decode_layer_step()                */
 } la_op;
 
 typedef struct {
@@ -249,6 +250,26 @@ int la_recurrent_steps(const la_problem* p, const void* q, const void* k, const 
                        float* S, float* Z, void* out, void* stream);
 
 /*
+ * One decode step of a whole attention sublayer: Eq. 16-20 with the projections of Eq. 2 written
+ * out, for B independent streams of model width F = H * D,
+ *   q = x W_Q,  k = x W_K,  v = x W_V                     (split into H heads of D = M columns)
+ *   S += phi(k) v^T,  Z += phi(k),  a = phi(q)^T S / (phi(q)^T Z + eps)      (per head, update first)
+ *   y = a W_O + x                                          (output projection and residual)
+ * so that the token produced from y can be fed back as the next x without the caller touching q, k, v.
+ * The position-wise feed-forward part f_l of Eq. 20 stays with the caller.  p: B, H, D = M = 64, dtype
+ * LA_BF16, phi, eps (N ignored).  x, y: [B, F] bf16.  Wqkv: [3F, F] bf16, row-major "outputs x inputs"
+ * (row r < F is column r of W_Q, rows F..2F-1 of W_K, 2F..3F-1 of W_V: the layout of a fused linear
+ * layer's weight); Wo: [F, F] likewise.  S [B,H,D,M], Z [B,H,D] fp32, updated in place (zero them for a
+ * new sequence).  ws: la_workspace_bytes(p, LA_OP_DECODE_LAYER) bytes (q, k, v, a as bf16: they are
+ * rounded to bf16 between the three kernels).  y must not alias x.  Three launches: projection
+ * (tensor cores), recurrent step, projection with the residual in its epilogue; asynchronous on
+ * `stream`.  Other dtypes or head sizes: LA_ERR_UNSUPPORTED (use la_recurrent_step with your own
+ * projections).
+ */
+int la_decode_layer_step(const la_problem* p, const void* x, const void* Wqkv, const void* Wo,
+                         float* S, float* Z, void* y, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Non-causal forward for callers that cannot allocate device memory (the paper has no
  * counterpart: this is a deployment convenience, not part of the method).
  *
@@ -363,7 +384,7 @@ long long la_kernel_launches(void);
  * la_profile_enable(0) stops recording.  la_profile_read() waits for the recorded events and
  * returns the mean duration in milliseconds and the number of launches of one kernel:
  * 0 causal_fwd_kernel, 1 causal_bwd_dq_kernel, 2 causal_bwd_dkv_kernel, 3 segment_sum_kernel,
- * 4 (unused, empty name), 5 linear_sum_kernel, 6 linear_apply_kernel, 7 recurrent_step_kernel.
+ * 4 projection_gemm_kernel, 5 linear_sum_kernel, 6 linear_apply_kernel, 7 recurrent_step_kernel.
  * Not thread-safe; meant for a benchmark's single launching thread.
  */
 int la_profile_enable(int on);

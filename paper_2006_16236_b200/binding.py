@@ -20,6 +20,7 @@ LA_OP_LINEAR_FORWARD, LA_OP_LINEAR_BACKWARD, LA_OP_CAUSAL_FORWARD, LA_OP_CAUSAL_
 LA_OP_CAUSAL_SAVED = 4
 LA_OP_LINEAR_VARLEN_FORWARD, LA_OP_LINEAR_VARLEN_BACKWARD = 5, 6
 LA_OP_LINEAR_SAVED = 7
+LA_OP_DECODE_LAYER = 8
 _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
@@ -31,6 +32,7 @@ EXPORTS = [
     "la_causal_backward", "la_recurrent_step", "la_recurrent_steps", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
     "la_profile_kernel_name", "la_version", "la_causal_plan", "la_plan_override",
+    "la_decode_layer_step",
 ]
 
 
@@ -75,6 +77,7 @@ def lib() -> ctypes.CDLL:
         L.la_causal_backward.argtypes = [pp] + [vp] * 6 + [vp, sz] + [vp] * 3 + [vp, sz, vp]
         L.la_recurrent_step.argtypes = [pp] + [vp] * 6 + [vp]
         L.la_recurrent_steps.argtypes = [pp] + [vp] * 6 + [vp]
+        L.la_decode_layer_step.argtypes = [pp] + [vp] * 6 + [vp, sz, vp]
         L.la_workspace_bytes.argtypes = [pp, i32]
         L.la_workspace_bytes.restype = sz
         L.la_status_string.argtypes = [ctypes.c_int]
@@ -103,6 +106,9 @@ def _check(rc: int) -> None:
 def _call(dev, fn, *args) -> None:
     """One library call with `dev` current: the library launches on, and keeps its per-device state for,
     the current device, which need not be the one the tensors live on."""
+    if dev.index == torch.cuda.current_device():
+        _check(fn(*args))
+        return
     with torch.cuda.device(dev):
         _check(fn(*args))
 
@@ -445,6 +451,28 @@ def la_recurrent_step(q, k, v, S, Z, phi="elu1", eps=0.0, out=None):
     out = torch.empty_like(v) if out is None else out
     _call(dev, lib().la_recurrent_step, ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out),
                                    _stream(dev))
+    return out
+
+
+def la_decode_layer_step(x, Wqkv, Wo, S, Z, phi="elu1", eps=0.0, out=None, ws=None):
+    """One decode step of a whole attention sublayer: x [B,F] -> y [B,F] with F = H*D (bf16, D = M = 64);
+    Wqkv [3F,F] and Wo [F,F] are "outputs x inputs" like a linear layer's weight; S [B,H,D,M], Z [B,H,D] (fp32)
+    are updated in place.  Returns y = attention(x) W_O + x."""
+    if S.dim() != 4 or x.dim() != 2:
+        raise ValueError("expected x [B,F], fp32 S [B,H,D,M] and Z [B,H,D]")
+    B, H, D, M = S.shape
+    F = H * D
+    p = make_problem(B, H, 1, D, M, _dtype_code(x), phi, eps)
+    _expect(p, x.dtype, S=(S, "S"), Z=(Z, "Z"))
+    for name, t, shape in (("x", x, (B, F)), ("Wqkv", Wqkv, (3 * F, F)), ("Wo", Wo, (F, F)), ("out", out, (B, F))):
+        if t is not None and (tuple(t.shape) != shape or t.dtype != x.dtype):
+            raise ValueError(f"{name} must have shape {list(shape)} and dtype {x.dtype} (got {list(t.shape)}, {t.dtype})")
+    _buffer("ws", ws)
+    dev = _dev(x, Wqkv, Wo, S, Z, out, ws)
+    out = torch.empty_like(x) if out is None else out
+    ws = workspace(p, LA_OP_DECODE_LAYER, dev) if ws is None else ws
+    _call(dev, lib().la_decode_layer_step, ctypes.byref(p), _ptr(x), _ptr(Wqkv), _ptr(Wo), _ptr(S), _ptr(Z), _ptr(out),
+          _ptr(ws), _nbytes(ws), _stream(dev))
     return out
 
 

@@ -167,14 +167,15 @@ int la_profile_read(int kernel, double* mean_ms, int* launches) {
 
 const char* la_profile_kernel_name(int kernel) {
     static const char* names[kProfCount] = {"causal_fwd_kernel", "causal_bwd_dq_kernel", "causal_bwd_dkv_kernel",
-                                            "segment_sum_kernel", "", "linear_sum_kernel",
+                                            "segment_sum_kernel", "projection_gemm_kernel", "linear_sum_kernel",
                                             "linear_apply_kernel", "recurrent_step_kernel"};
     return kernel >= 0 && kernel < kProfCount ? names[kernel] : "";
 }
 
 size_t la_workspace_bytes(const la_problem* p, int32_t op) {
     if (!p || p->B < 1 || p->H < 1 || p->N < 0 || p->D < 1 || p->M < 1 || p->D > 128 || p->M > 128) return 0;
-    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_LINEAR_SAVED) return 0;
+    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_DECODE_LAYER) return 0;
+    if (op == LA_OP_DECODE_LAYER) return decode_layer_supported(*p) ? decode_layer_workspace(*p) : 0;
     if (p->N == 0) return 0;
     if (op == LA_OP_LINEAR_SAVED) op = LA_OP_LINEAR_FORWARD;          // the saved buffer holds what the forward's workspace holds
     if (op == LA_OP_CAUSAL_SAVED) return tc_supported(*p, LA_OP_CAUSAL_BACKWARD) ? tc_causal_saved_bytes(*p) : 0;
@@ -428,6 +429,22 @@ int la_recurrent_step(const la_problem* p, const void* q, const void* k, const v
     LA_REQUIRE_PTR(S); LA_REQUIRE_PTR(Z); LA_REQUIRE_PTR(out);
     if (int rc = check_arch()) return rc;
     return launch_recurrent_step(*p, q, k, v, S, Z, out, (cudaStream_t)stream);
+}
+
+int la_decode_layer_step(const la_problem* p, const void* x, const void* Wqkv, const void* Wo,
+                         float* S, float* Z, void* y, void* ws, size_t ws_bytes, void* stream) {
+    if (int rc = check_problem(p, false)) return rc;
+    if (!decode_layer_supported(*p))
+        return fail(LA_ERR_UNSUPPORTED, "the fused decode layer takes bf16 with D = M = 64 (got dtype %d, D=%lld, M=%lld)",
+                    p->dtype, (long long)p->D, (long long)p->M);
+    if (p->B * p->H * p->D >= (1LL << 31) || p->H * p->D > 65536)
+        return fail(LA_ERR_UNSUPPORTED, "B * H * D must be below 2^31 and the model width H * D at most 65536");
+    LA_REQUIRE_PTR(x); LA_REQUIRE_PTR(Wqkv); LA_REQUIRE_PTR(Wo);
+    LA_REQUIRE_PTR(S); LA_REQUIRE_PTR(Z); LA_REQUIRE_PTR(y);
+    if (y == x) return fail(LA_ERR_INVALID_ARG, "y must not alias x (x is read again for the residual while y is written)");
+    if (int rc = check_ws(p, LA_OP_DECODE_LAYER, ws, ws_bytes)) return rc;
+    if (int rc = check_arch()) return rc;
+    return decode_layer_step(*p, x, Wqkv, Wo, S, Z, y, ws, (cudaStream_t)stream);
 }
 
 int la_recurrent_steps(const la_problem* p, const void* q, const void* k, const void* v,

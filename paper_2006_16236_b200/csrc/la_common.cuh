@@ -43,7 +43,7 @@ void note_launch();
 // Optional per-kernel timing with CUDA events on the launch stream (see la_profile_enable()).
 // Indices are part of the C ABI (la_profile_read); no-ops unless profiling is switched on.
 enum ProfKernel {
-    kProfCausalFwd = 0, kProfCausalBwdDq = 1, kProfCausalBwdDkv = 2, kProfSegmentSum = 3, kProfUnused = 4,
+    kProfCausalFwd = 0, kProfCausalBwdDq = 1, kProfCausalBwdDkv = 2, kProfSegmentSum = 3, kProfProjection = 4,
     kProfLinearSum = 5, kProfLinearApply = 6, kProfRecurrent = 7, kProfCount = 8
 };
 void prof_begin(int kernel, cudaStream_t st);
@@ -82,8 +82,16 @@ int launch_poly2_map_backward(const void* x, const void* dy, void* dx, int64_t r
 
 int launch_recurrent_steps(const la_problem& p, const void* q, const void* k, const void* v,
                            float* S, float* Z, void* out, cudaStream_t st);
+// chained: launch as a programmatic dependent of the kernel before it in the stream (its launch overlaps that
+// kernel's tail; it waits for that kernel before it reads anything)
 int launch_recurrent_step(const la_problem& p, const void* q, const void* k, const void* v,
-                          float* S, float* Z, void* out, cudaStream_t st);
+                          float* S, float* Z, void* out, cudaStream_t st, bool chained = false);
+
+// Decode step of a whole attention sublayer (projections + recurrent step + output projection), bf16, D = M = 64
+bool decode_layer_supported(const la_problem& p);
+size_t decode_layer_workspace(const la_problem& p);
+int decode_layer_step(const la_problem& p, const void* x, const void* Wqkv, const void* Wo, float* S, float* Z,
+                      void* y, void* ws, cudaStream_t st);
 
 // State arguments of the causal backward pass (device, fp32, any of them may be null): the state the
 // forward started from, the upstream gradient of the final state, and where the gradient of the

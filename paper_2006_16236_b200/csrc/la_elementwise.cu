@@ -176,6 +176,11 @@ recurrent_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T*
     const int64_t bh = blockIdx.x;
     const int c4 = tid % TPR, r0 = tid / TPR;
 
+    // When launched as a programmatic dependent of the kernel before it in the stream (the decode layer does
+    // that), this is where that kernel's results become visible; in an ordinary launch both are no-ops.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     float4* Sp = reinterpret_cast<float4*>(S + bh * (int64_t)(D * M));
     float4 s[PASSES];
 #pragma unroll
@@ -430,10 +435,24 @@ int launch_recurrent_steps(const la_problem& p, const void* q, const void* k, co
 
 template <typename T>
 static int recurrent_dispatch(const la_problem& p, const void* q, const void* k, const void* v,
-                              float* S, float* Z, void* out, cudaStream_t st) {
+                              float* S, float* Z, void* out, cudaStream_t st, bool chained) {
     const unsigned grid = (unsigned)(p.B * p.H);
     const T *qq = (const T*)q, *kk = (const T*)k, *vv = (const T*)v;
     T* oo = (T*)out;
+    if (chained && p.D == 64 && p.M == 64) {        // between the two projections of a decode layer: see the kernel
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(128);
+        cfg.stream = st;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, recurrent_step_kernel<T, 64, 64>, qq, kk, vv, S, Z, oo, p.eps, p.phi));
+        note_launch();
+        return LA_OK;
+    }
 #define LA_RS_CASE(DD, MM)                                                                     \
     if (p.D == DD && p.M == MM) {                                                              \
         recurrent_step_kernel<T, DD, MM><<<grid, 128, 0, st>>>(qq, kk, vv, S, Z, oo, p.eps, p.phi); \
@@ -450,10 +469,10 @@ static int recurrent_dispatch(const la_problem& p, const void* q, const void* k,
 }
 
 int launch_recurrent_step(const la_problem& p, const void* q, const void* k, const void* v,
-                          float* S, float* Z, void* out, cudaStream_t st) {
+                          float* S, float* Z, void* out, cudaStream_t st, bool chained) {
     prof_begin(kProfRecurrent, st);
-    const int rc = p.dtype == LA_F32 ? recurrent_dispatch<float>(p, q, k, v, S, Z, out, st)
-                                     : recurrent_dispatch<__nv_bfloat16>(p, q, k, v, S, Z, out, st);
+    const int rc = p.dtype == LA_F32 ? recurrent_dispatch<float>(p, q, k, v, S, Z, out, st, chained)
+                                     : recurrent_dispatch<__nv_bfloat16>(p, q, k, v, S, Z, out, st, chained);
     prof_end(kProfRecurrent, st);
     return rc;
 }

@@ -689,3 +689,43 @@ def test_decode_workload_full_size():
     O = la.la_causal_forward(*(t[bsub].contiguous().to(DEV) for t in (Q, K, V)))
     err = (O.float() - outs[bsub].float()).abs().max().item()
     assert err < 0.05, err
+
+
+@pytest.mark.parametrize("B,H", [(256, 8), (3, 2), (130, 4)])
+def test_decode_layer_steps_against_the_oracle(B, H):
+    """A whole attention sublayer per token (projections, state update and read-out, output projection,
+    residual), 12 tokens fed one at a time; the next token's input is made from the previous output, so the
+    steps depend on each other as in generation.  The oracle walks the same steps in fp64 on the values the
+    GPU actually saw as inputs (x is rounded to bf16 once per step on both sides)."""
+    D = 64
+    F = H * D
+    g = torch.Generator().manual_seed(100 + B)
+    s = 1.0 / F ** 0.5
+    Wqkv = (torch.randn((3 * F, F), generator=g) * s).to(torch.bfloat16)
+    Wo = (torch.randn((F, F), generator=g) * s).to(torch.bfloat16)
+    x = torch.randn((B, F), generator=g).to(torch.bfloat16)
+    S = torch.zeros((B, H, D, D), device=DEV)
+    Z = torch.zeros((B, H, D), device=DEV)
+    So, Zo = np.zeros((B, H, D, D)), np.zeros((B, H, D))
+    Wd, Wod = Wqkv.to(DEV), Wo.to(DEV)
+    W = Wqkv.double().numpy()
+    Wq, Wk, Wv, Wout = W[:F].T, W[F:2 * F].T, W[2 * F:].T, Wo.double().numpy().T
+    for t in range(12):
+        y = la.la_decode_layer_step(x.to(DEV), Wd, Wod, S, Z)
+        ref = oracle.decode_layer_step(x.double().numpy(), Wq, Wk, Wv, Wout, So, Zo)
+        assert_close(y, ref, torch.bfloat16, f"layer step {t}")
+        # the next input: a bounded function of this output (what the rest of a model would do), taken from the GPU
+        x = torch.tanh(y.float().cpu()).to(torch.bfloat16) + (0.1 * torch.randn((B, F), generator=g)).to(torch.bfloat16)
+    la.la_last_device_status()
+    assert_close(S, So, torch.bfloat16, "layer S")
+    assert_close(Z, Zo, torch.bfloat16, "layer Z")
+
+
+def test_decode_layer_rejects_what_it_does_not_take():
+    B, H, D = 4, 2, 32
+    x = torch.zeros((B, H * D), dtype=torch.bfloat16, device=DEV)
+    W3, W1 = torch.zeros((3 * H * D, H * D), dtype=torch.bfloat16, device=DEV), torch.zeros((H * D, H * D), dtype=torch.bfloat16, device=DEV)
+    S, Z = torch.zeros((B, H, D, D), device=DEV), torch.zeros((B, H, D), device=DEV)
+    with pytest.raises(la.LaError) as e:
+        la.la_decode_layer_step(x, W3, W1, S, Z)
+    assert e.value.status == -2
