@@ -69,7 +69,9 @@ typedef enum {
     LA_OP_LINEAR_VARLEN_FORWARD = 5,     /* la_linear_attention_varlen()          */
     LA_OP_LINEAR_VARLEN_BACKWARD = 6,    /* la_linear_attention_varlen_backward() */
     LA_OP_LINEAR_SAVED = 7,              /* size of the optional `saved` buffer, see la_linear_attention_keep() */
-    LA_OP_DECODE_LAYER = 8               /* la_decode_layer_step()                */
+    LA_OP_DECODE_LAYER = 8,              /* la_decode_layer_step()                */
+    LA_OP_CAUSAL_VARLEN_FORWARD = 9,     /* la_causal_forward_varlen()            */
+    LA_OP_CAUSAL_VARLEN_BACKWARD = 10    /* la_causal_backward_varlen()           */
 } la_op;
 
 typedef struct {
@@ -371,6 +373,36 @@ int la_causal_backward_from(const la_problem* p, const void* Q, const void* K, c
                             const void* saved, size_t saved_bytes,
                             void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
                             void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The causal form on a right-padded ragged batch (speech-style batches: sequences of different lengths
+ * padded to a common N; Eq. 9-12 and 16-20 per sequence on its own length).  lengths: [B] int32 (device),
+ * lengths[b] in [0, N] = real positions of batch element b (all its heads); the N - lengths[b] rows behind
+ * them are padding whose contents are never used, whatever they hold (Inf and NaN included).  O and den are
+ * zero on the padding.  S_out / Z_out (optional) receive the state after each sequence's OWN last position,
+ * so that a ragged prefill hands every stream over to la_recurrent_step() at the right place; S_in / Z_in
+ * (both or neither) as for la_causal_forward_from().  ws: la_workspace_bytes(p, LA_OP_CAUSAL_VARLEN_FORWARD).
+ * Causality alone already keeps right padding out of every real position's output; what this call adds is
+ * the state at the true end, zeros instead of garbage on the padding, indifference to non-finite padding,
+ * and no time spent on it.
+ */
+int la_causal_forward_varlen(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
+                             const float* S_in, const float* Z_in,
+                             void* O, float* den, float* S_out, float* Z_out,
+                             void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Gradients of la_causal_forward_varlen() (Eq. 13-15 per sequence on its own length): dQ, dK, dV are zero on
+ * the padding, and G is not read there.  The state arguments are those of la_causal_backward_from(): dS_out /
+ * dZ_out is the upstream gradient of the state at each sequence's own end, dS_in / dZ_in receive the gradient
+ * of the state it started from.  ws: la_workspace_bytes(p, LA_OP_CAUSAL_VARLEN_BACKWARD).
+ */
+int la_causal_backward_varlen(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
+                              const float* S_in, const float* Z_in,
+                              const void* O, const float* den, const void* G,
+                              const float* dS_out, const float* dZ_out,
+                              void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
+                              void* ws, size_t ws_bytes, void* stream);
 
 /* Number of GPU kernels this library has enqueued in this process so far (all
  * threads, all entry points); a diagnostic for benchmarks. */

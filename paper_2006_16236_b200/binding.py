@@ -21,6 +21,7 @@ LA_OP_CAUSAL_SAVED = 4
 LA_OP_LINEAR_VARLEN_FORWARD, LA_OP_LINEAR_VARLEN_BACKWARD = 5, 6
 LA_OP_LINEAR_SAVED = 7
 LA_OP_DECODE_LAYER = 8
+LA_OP_CAUSAL_VARLEN_FORWARD, LA_OP_CAUSAL_VARLEN_BACKWARD = 9, 10
 _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
@@ -32,7 +33,7 @@ EXPORTS = [
     "la_causal_backward", "la_recurrent_step", "la_recurrent_steps", "la_workspace_bytes", "la_status_string",
     "la_last_error", "la_last_device_status", "la_kernel_launches", "la_profile_enable", "la_profile_read",
     "la_profile_kernel_name", "la_version", "la_causal_plan", "la_plan_override",
-    "la_decode_layer_step",
+    "la_decode_layer_step", "la_causal_forward_varlen", "la_causal_backward_varlen",
 ]
 
 
@@ -75,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.la_causal_forward_from.argtypes = [pp] + [vp] * 9 + [vp, sz] + [vp, sz, vp]
         L.la_causal_backward_from.argtypes = [pp] + [vp] * 10 + [vp, sz] + [vp] * 5 + [vp, sz, vp]
         L.la_causal_backward.argtypes = [pp] + [vp] * 6 + [vp, sz] + [vp] * 3 + [vp, sz, vp]
+        L.la_causal_forward_varlen.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
+        L.la_causal_backward_varlen.argtypes = [pp] + [vp] * 16 + [vp, sz, vp]
         L.la_recurrent_step.argtypes = [pp] + [vp] * 6 + [vp]
         L.la_recurrent_steps.argtypes = [pp] + [vp] * 6 + [vp]
         L.la_decode_layer_step.argtypes = [pp] + [vp] * 6 + [vp, sz, vp]
@@ -392,7 +395,7 @@ def saved_buffer(Q, V, phi="elu1", eps=0.0):
 
 
 def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None, Z_out=None, saved=None, ws=None,
-                      S_in=None, Z_in=None):
+                      S_in=None, Z_in=None, lengths=None):
     """Causal form.  Returns O; pass preallocated den / S_out / Z_out tensors to receive them, and a
     saved_buffer() to keep phi(Q), phi(K) for the backward pass.  S_in / Z_in (fp32 [B,H,D,M] / [B,H,D]):
     the state the sequence continues from (la_causal_forward_from)."""
@@ -400,8 +403,17 @@ def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None
     _expect(p, Q.dtype, Q=(Q, "qk"), K=(K, "qk"), V=(V, "v"), O=(O, "v"), den=(den, "row"), S_out=(S_out, "S"),
             Z_out=(Z_out, "Z"), S_in=(S_in, "S"), Z_in=(Z_in, "Z"))
     _buffer("saved", saved), _buffer("ws", ws)
-    dev = _dev(Q, K, V, O, den, S_out, Z_out, saved, S_in, Z_in, ws)
+    if lengths is not None:
+        _lengths_arg(lengths, p.B, None)
+        if saved is not None:
+            raise ValueError("a ragged batch (lengths) keeps nothing for the backward pass: do not pass `saved`")
+    dev = _dev(Q, K, V, O, den, S_out, Z_out, saved, S_in, Z_in, ws, lengths)
     O = torch.empty_like(V) if O is None else O
+    if lengths is not None:             # la_causal_forward_varlen: right-padded ragged batch
+        ws = workspace(p, LA_OP_CAUSAL_VARLEN_FORWARD, dev) if ws is None else ws
+        _call(dev, lib().la_causal_forward_varlen, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(S_in),
+              _ptr(Z_in), _ptr(O), _ptr(den), _ptr(S_out), _ptr(Z_out), _ptr(ws), _nbytes(ws), _stream(dev))
+        return O
     ws = workspace(p, LA_OP_CAUSAL_FORWARD, dev) if ws is None else ws
     if S_in is None and Z_in is None:
         _call(dev, lib().la_causal_forward, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(den), _ptr(S_out),
@@ -414,7 +426,7 @@ def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None
 
 
 def la_causal_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None, saved=None, dQ=None, dK=None, dV=None,
-                       ws=None, S_in=None, Z_in=None, dS_out=None, dZ_out=None, dS_in=None, dZ_in=None):
+                       ws=None, S_in=None, Z_in=None, dS_out=None, dZ_out=None, dS_in=None, dZ_in=None, lengths=None):
     """Gradients of the causal form; returns (dQ, dK, dV).  With any of the state arguments (fp32 [B,H,D,M] /
     [B,H,D]: the state the forward started from, the upstream gradient of its final state, and tensors that
     receive the gradient of the initial state) the call is la_causal_backward_from."""
@@ -423,10 +435,20 @@ def la_causal_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None, saved=
             dQ=(dQ, "qk"), dK=(dK, "qk"), dV=(dV, "v"), S_in=(S_in, "S"), Z_in=(Z_in, "Z"), dS_out=(dS_out, "S"),
             dZ_out=(dZ_out, "Z"), dS_in=(dS_in, "S"), dZ_in=(dZ_in, "Z"))
     _buffer("saved", saved), _buffer("ws", ws)
-    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved, S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in, ws)
+    if lengths is not None:
+        _lengths_arg(lengths, p.B, None)
+        if saved is not None:
+            raise ValueError("a ragged batch (lengths) keeps nothing for the backward pass: do not pass `saved`")
+    dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved, S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in, ws, lengths)
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(V) if dV is None else dV
+    if lengths is not None:             # la_causal_backward_varlen
+        ws = workspace(p, LA_OP_CAUSAL_VARLEN_BACKWARD, dev) if ws is None else ws
+        _call(dev, lib().la_causal_backward_varlen, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(S_in),
+              _ptr(Z_in), _ptr(O), _ptr(den), _ptr(G), _ptr(dS_out), _ptr(dZ_out), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dS_in),
+              _ptr(dZ_in), _ptr(ws), _nbytes(ws), _stream(dev))
+        return dQ, dK, dV
     ws = workspace(p, LA_OP_CAUSAL_BACKWARD, dev) if ws is None else ws
     state = (S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in)
     if all(t is None for t in state):

@@ -174,7 +174,9 @@ const char* la_profile_kernel_name(int kernel) {
 
 size_t la_workspace_bytes(const la_problem* p, int32_t op) {
     if (!p || p->B < 1 || p->H < 1 || p->N < 0 || p->D < 1 || p->M < 1 || p->D > 128 || p->M > 128) return 0;
-    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_DECODE_LAYER) return 0;
+    if (op < LA_OP_LINEAR_FORWARD || op > LA_OP_CAUSAL_VARLEN_BACKWARD) return 0;
+    if (op == LA_OP_CAUSAL_VARLEN_FORWARD) op = LA_OP_CAUSAL_FORWARD;         // the ragged calls run the same kernels
+    if (op == LA_OP_CAUSAL_VARLEN_BACKWARD) op = LA_OP_CAUSAL_BACKWARD;
     if (op == LA_OP_DECODE_LAYER) return decode_layer_supported(*p) ? decode_layer_workspace(*p) : 0;
     if (p->N == 0) return 0;
     if (op == LA_OP_LINEAR_SAVED) op = LA_OP_LINEAR_FORWARD;          // the saved buffer holds what the forward's workspace holds
@@ -337,12 +339,17 @@ static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
     return a && b && x < y + nb && y < x + na;
 }
 
-int la_causal_forward_from(const la_problem* p, const void* Q, const void* K, const void* V,
-                           const float* S_in, const float* Z_in,
-                           void* O, float* den, float* S_out, float* Z_out,
-                           void* saved, size_t saved_bytes,
-                           void* ws, size_t ws_bytes, void* stream) {
+}  // extern "C"
+
+// All causal forward entry points: from a state or from zero, `lengths` given (ragged batch) or not.
+static int causal_forward_common(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
+                                 bool ragged, const float* S_in, const float* Z_in,
+                                 void* O, float* den, float* S_out, float* Z_out,
+                                 void* saved, size_t saved_bytes,
+                                 void* ws, size_t ws_bytes, void* stream) {
     if (int rc = check_problem(p, true)) return rc;
+    if (ragged && !lengths) return fail(LA_ERR_INVALID_ARG, "lengths is NULL");
+    if (reinterpret_cast<uintptr_t>(lengths) & 3u) return fail(LA_ERR_INVALID_ARG, "lengths is not 4-byte aligned");
     if ((S_in == nullptr) != (Z_in == nullptr)) return fail(LA_ERR_INVALID_ARG, "S_in and Z_in must both be given or both be NULL");
     LA_OPTIONAL_PTR(S_in); LA_OPTIONAL_PTR(Z_in);
     LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(S_out); LA_OPTIONAL_PTR(Z_out);
@@ -358,12 +365,29 @@ int la_causal_forward_from(const la_problem* p, const void* Q, const void* K, co
     }
     LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(O);
     LA_OPTIONAL_PTR(saved);
-    if (int rc = check_ws(p, LA_OP_CAUSAL_FORWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_ws(p, lengths ? LA_OP_CAUSAL_VARLEN_FORWARD : LA_OP_CAUSAL_FORWARD, ws, ws_bytes)) return rc;
     if (int rc = check_saved(p, saved, saved_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     if (tc_supported(*p, LA_OP_CAUSAL_FORWARD))
-        return tc_causal_forward(*p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
-    return general_causal_forward(*p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, st);
+        return tc_causal_forward(*p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
+    return general_causal_forward(*p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, st);
+}
+
+extern "C" {
+
+int la_causal_forward_from(const la_problem* p, const void* Q, const void* K, const void* V,
+                           const float* S_in, const float* Z_in,
+                           void* O, float* den, float* S_out, float* Z_out,
+                           void* saved, size_t saved_bytes,
+                           void* ws, size_t ws_bytes, void* stream) {
+    return causal_forward_common(p, Q, K, V, nullptr, false, S_in, Z_in, O, den, S_out, Z_out, saved, saved_bytes, ws, ws_bytes, stream);
+}
+
+int la_causal_forward_varlen(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
+                             const float* S_in, const float* Z_in,
+                             void* O, float* den, float* S_out, float* Z_out,
+                             void* ws, size_t ws_bytes, void* stream) {
+    return causal_forward_common(p, Q, K, V, lengths, true, S_in, Z_in, O, den, S_out, Z_out, nullptr, 0, ws, ws_bytes, stream);
 }
 
 int la_causal_forward(const la_problem* p, const void* Q, const void* K, const void* V,
@@ -373,14 +397,18 @@ int la_causal_forward(const la_problem* p, const void* Q, const void* K, const v
     return la_causal_forward_from(p, Q, K, V, nullptr, nullptr, O, den, S_out, Z_out, saved, saved_bytes, ws, ws_bytes, stream);
 }
 
-int la_causal_backward_from(const la_problem* p, const void* Q, const void* K, const void* V,
-                            const float* S_in, const float* Z_in,
-                            const void* O, const float* den, const void* G,
-                            const float* dS_out, const float* dZ_out,
-                            const void* saved, size_t saved_bytes,
-                            void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
-                            void* ws, size_t ws_bytes, void* stream) {
+}  // extern "C"
+
+static int causal_backward_common(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
+                                  bool ragged, const float* S_in, const float* Z_in,
+                                  const void* O, const float* den, const void* G,
+                                  const float* dS_out, const float* dZ_out,
+                                  const void* saved, size_t saved_bytes,
+                                  void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
+                                  void* ws, size_t ws_bytes, void* stream) {
     if (int rc = check_problem(p, true)) return rc;
+    if (ragged && !lengths) return fail(LA_ERR_INVALID_ARG, "lengths is NULL");
+    if (reinterpret_cast<uintptr_t>(lengths) & 3u) return fail(LA_ERR_INVALID_ARG, "lengths is not 4-byte aligned");
     if ((S_in == nullptr) != (Z_in == nullptr)) return fail(LA_ERR_INVALID_ARG, "S_in and Z_in must both be given or both be NULL");
     LA_OPTIONAL_PTR(S_in); LA_OPTIONAL_PTR(Z_in); LA_OPTIONAL_PTR(dS_out); LA_OPTIONAL_PTR(dZ_out);
     LA_OPTIONAL_PTR(dS_in); LA_OPTIONAL_PTR(dZ_in);
@@ -403,14 +431,37 @@ int la_causal_backward_from(const la_problem* p, const void* Q, const void* K, c
     LA_REQUIRE_PTR(Q); LA_REQUIRE_PTR(K); LA_REQUIRE_PTR(V); LA_REQUIRE_PTR(G);
     LA_REQUIRE_PTR(dQ); LA_REQUIRE_PTR(dK); LA_REQUIRE_PTR(dV);
     LA_OPTIONAL_PTR(O); LA_OPTIONAL_PTR(den); LA_OPTIONAL_PTR(saved);
-    if (int rc = check_ws(p, LA_OP_CAUSAL_BACKWARD, ws, ws_bytes)) return rc;
+    if (int rc = check_ws(p, lengths ? LA_OP_CAUSAL_VARLEN_BACKWARD : LA_OP_CAUSAL_BACKWARD, ws, ws_bytes)) return rc;
     if (int rc = check_saved(p, saved, saved_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     StateArgs sa;
     sa.S_in = S_in; sa.Z_in = Z_in; sa.dS_out = dS_out; sa.dZ_out = dZ_out; sa.dS_in = dS_in; sa.dZ_in = dZ_in;
     if (tc_supported(*p, LA_OP_CAUSAL_BACKWARD))
-        return tc_causal_backward(*p, Q, K, V, O, den, G, sa, saved, dQ, dK, dV, ws, st);
-    return general_causal_backward(*p, Q, K, V, G, sa, dQ, dK, dV, ws, st);
+        return tc_causal_backward(*p, Q, K, V, lengths, O, den, G, sa, saved, dQ, dK, dV, ws, st);
+    return general_causal_backward(*p, Q, K, V, lengths, G, sa, dQ, dK, dV, ws, st);
+}
+
+extern "C" {
+
+int la_causal_backward_from(const la_problem* p, const void* Q, const void* K, const void* V,
+                            const float* S_in, const float* Z_in,
+                            const void* O, const float* den, const void* G,
+                            const float* dS_out, const float* dZ_out,
+                            const void* saved, size_t saved_bytes,
+                            void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
+                            void* ws, size_t ws_bytes, void* stream) {
+    return causal_backward_common(p, Q, K, V, nullptr, false, S_in, Z_in, O, den, G, dS_out, dZ_out, saved, saved_bytes,
+                                  dQ, dK, dV, dS_in, dZ_in, ws, ws_bytes, stream);
+}
+
+int la_causal_backward_varlen(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
+                              const float* S_in, const float* Z_in,
+                              const void* O, const float* den, const void* G,
+                              const float* dS_out, const float* dZ_out,
+                              void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
+                              void* ws, size_t ws_bytes, void* stream) {
+    return causal_backward_common(p, Q, K, V, lengths, true, S_in, Z_in, O, den, G, dS_out, dZ_out, nullptr, 0,
+                                  dQ, dK, dV, dS_in, dZ_in, ws, ws_bytes, stream);
 }
 
 int la_causal_backward(const la_problem* p, const void* Q, const void* K, const void* V,

@@ -107,10 +107,11 @@ struct StateArgs {
 
 // General (any D, M multiple of 8 up to 128, any N) fp32-arithmetic kernels.
 size_t general_workspace_bytes(const la_problem& p, int op);
-int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V,
+// lengths ([B] int32, device, or null): real positions per batch element of a right-padded ragged batch
+int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
                            const float* S_in, const float* Z_in,
                            void* O, float* den, float* S_out, float* Z_out, cudaStream_t st);
-int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V,
+int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
                             const void* G, const StateArgs& sa, void* dQ, void* dK, void* dV, void* ws,
                             cudaStream_t st);
 // lengths ([B] int32, device, or null): real positions per batch element (the rest is padding);

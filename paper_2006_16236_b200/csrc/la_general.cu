@@ -197,7 +197,8 @@ __global__ void __launch_bounds__(THREADS)
 general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K, const IO* __restrict__ V,
                               const float* __restrict__ S_in, const float* __restrict__ Z_in,
                               IO* __restrict__ O, float* __restrict__ den, float* __restrict__ S_out,
-                              float* __restrict__ Z_out, int64_t N, int D_arg, int M_arg, float eps, int phi) {
+                              float* __restrict__ Z_out, int64_t Nfull, int D_arg, int M_arg, float eps, int phi,
+                              const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
     const int D = KD ? KD : D_arg, M = KD ? KD : M_arg;
     const Dims dm = make_dims(D, M);
@@ -209,7 +210,14 @@ general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K
     float* sP = sSt + D * dm.MS;
 
     const int64_t bh = blockIdx.x;
-    Q += bh * N * D; K += bh * N * D; V += bh * N * M; O += bh * N * M;
+    // a right-padded ragged batch: only the first N positions of this sequence are real, the rest of its
+    // Nfull rows is padding that is neither read nor summed and receives zeros
+    int64_t N = Nfull;
+    if (lengths) {
+        const int64_t len = lengths[bh / heads];
+        N = len < 0 ? 0 : (len < Nfull ? len : Nfull);
+    }
+    Q += bh * Nfull * D; K += bh * Nfull * D; V += bh * Nfull * M; O += bh * Nfull * M;
     zero_fill(sSt, D * dm.MS);
     if (S_in) {                 // continue from a given state (Eq. 16-20 started from S_in, Z_in)
         __syncthreads();
@@ -244,10 +252,13 @@ general_causal_forward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K
             O[(n0 + i) * M + e] = from_f32<IO>(snd[i * dm.MS + e] / (snd[i * dm.MS + M] + eps));
         }
         if (den)
-            for (int i = threadIdx.x; i < cn; i += THREADS) den[bh * N + n0 + i] = snd[i * dm.MS + M];
+            for (int i = threadIdx.x; i < cn; i += THREADS) den[bh * Nfull + n0 + i] = snd[i * dm.MS + M];
         state_update(sSt, sk, sv, dm);
     }
     __syncthreads();
+    for (int64_t idx = N * M + threadIdx.x; idx < Nfull * M; idx += THREADS) O[idx] = from_f32<IO>(0.f);
+    if (den)
+        for (int64_t i = N + threadIdx.x; i < Nfull; i += THREADS) den[bh * Nfull + i] = 0.f;
     if (S_out)
         for (int idx = threadIdx.x; idx < D * M; idx += THREADS)
             S_out[bh * D * M + idx] = sSt[(idx / M) * dm.MS + idx % M];
@@ -266,7 +277,8 @@ __global__ void __launch_bounds__(THREADS)
 general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ K, const IO* __restrict__ V,
                                const IO* __restrict__ G, const StateArgs sa, IO* __restrict__ dQ,
                                IO* __restrict__ dK, IO* __restrict__ dV, float* __restrict__ aux,
-                               int64_t N, int D_arg, int M_arg, float eps, int phi) {
+                               int64_t Nfull, int D_arg, int M_arg, float eps, int phi,
+                               const int* __restrict__ lengths, int heads) {
     extern __shared__ float smem[];
     const int D = KD ? KD : D_arg, M = KD ? KD : M_arg;
     const Dims dm = make_dims(D, M);
@@ -280,10 +292,20 @@ general_causal_backward_kernel(const IO* __restrict__ Q, const IO* __restrict__ 
     float* sdP = sP + T * (T + 1);
 
     const int64_t bh = blockIdx.x;
-    Q += bh * N * D; K += bh * N * D; V += bh * N * M; G += bh * N * M;
-    dQ += bh * N * D; dK += bh * N * D; dV += bh * N * M;
-    float* dn_all = aux + bh * N * 2;
-    float* delta_all = dn_all + N;
+    int64_t N = Nfull;          // real positions of this sequence (see the forward kernel)
+    if (lengths) {
+        const int64_t len = lengths[bh / heads];
+        N = len < 0 ? 0 : (len < Nfull ? len : Nfull);
+    }
+    Q += bh * Nfull * D; K += bh * Nfull * D; V += bh * Nfull * M; G += bh * Nfull * M;
+    dQ += bh * Nfull * D; dK += bh * Nfull * D; dV += bh * Nfull * M;
+    float* dn_all = aux + bh * Nfull * 2;
+    float* delta_all = dn_all + Nfull;
+    for (int64_t idx = N * D + threadIdx.x; idx < Nfull * D; idx += THREADS) {
+        dQ[idx] = from_f32<IO>(0.f);
+        dK[idx] = from_f32<IO>(0.f);
+    }
+    for (int64_t idx = N * M + threadIdx.x; idx < Nfull * M; idx += THREADS) dV[idx] = from_f32<IO>(0.f);
 
     // ---- forward sweep: St = running sum of phi(K_j) Vt_j^T (from the given state, if any) ----
     zero_fill(sSt, D * dm.MS);
@@ -641,25 +663,25 @@ size_t general_workspace_bytes(const la_problem& p, int op) {
 }
 
 template <typename IO>
-static int causal_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+static int causal_forward_t(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const float* S_in,
                             const float* Z_in, void* O, float* den, float* S_out, float* Z_out, cudaStream_t st) {
     const size_t smem = smem_floats_forward((int)p.D, (int)p.M) * sizeof(float);
     auto kern = p.D == 64 && p.M == 64 ? general_causal_forward_kernel<IO, 64> : general_causal_forward_kernel<IO, 0>;
     if (int rc = opt_in_smem(kern, smem)) return rc;
     kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, S_in, Z_in, (IO*)O, den,
-                                                       S_out, Z_out, p.N, (int)p.D, (int)p.M, p.eps, p.phi);
+                                                       S_out, Z_out, p.N, (int)p.D, (int)p.M, p.eps, p.phi, lengths, (int)p.H);
     LA_LAUNCHED();
     return LA_OK;
 }
 
-int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+int general_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const float* S_in,
                            const float* Z_in, void* O, float* den, float* S_out, float* Z_out, cudaStream_t st) {
-    return p.dtype == LA_F32 ? causal_forward_t<float>(p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, st)
-                             : causal_forward_t<__nv_bfloat16>(p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, st);
+    return p.dtype == LA_F32 ? causal_forward_t<float>(p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, st)
+                             : causal_forward_t<__nv_bfloat16>(p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, st);
 }
 
 template <typename IO>
-static int causal_backward_t(const la_problem& p, const void* Q, const void* K, const void* V,
+static int causal_backward_t(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
                              const void* G, const StateArgs& sa, void* dQ, void* dK, void* dV, void* ws,
                              cudaStream_t st) {
     const size_t smem = smem_floats_backward((int)p.D, (int)p.M) * sizeof(float);
@@ -667,15 +689,15 @@ static int causal_backward_t(const la_problem& p, const void* Q, const void* K, 
     if (int rc = opt_in_smem(kern, smem)) return rc;
     kern<<<(unsigned)(p.B * p.H), THREADS, smem, st>>>((const IO*)Q, (const IO*)K, (const IO*)V, (const IO*)G, sa,
                                                        (IO*)dQ, (IO*)dK, (IO*)dV, (float*)ws, p.N, (int)p.D,
-                                                       (int)p.M, p.eps, p.phi);
+                                                       (int)p.M, p.eps, p.phi, lengths, (int)p.H);
     LA_LAUNCHED();
     return LA_OK;
 }
 
-int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+int general_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const void* G,
                             const StateArgs& sa, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
-    return p.dtype == LA_F32 ? causal_backward_t<float>(p, Q, K, V, G, sa, dQ, dK, dV, ws, st)
-                             : causal_backward_t<__nv_bfloat16>(p, Q, K, V, G, sa, dQ, dK, dV, ws, st);
+    return p.dtype == LA_F32 ? causal_backward_t<float>(p, Q, K, V, lengths, G, sa, dQ, dK, dV, ws, st)
+                             : causal_backward_t<__nv_bfloat16>(p, Q, K, V, lengths, G, sa, dQ, dK, dV, ws, st);
 }
 
 template <typename IO>

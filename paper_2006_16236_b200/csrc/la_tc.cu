@@ -144,16 +144,16 @@ int tc_causal_plan(const la_problem& p, int32_t* out, int capacity) {
     for (int s = 0; s < np; ++s) put(pl.piece_of_slot(s));
     return n;
 }
-int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const float* S_in,
                       const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
                       cudaStream_t st) {
-    return tc::causal_forward(p, Q, K, V, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
+    return tc::causal_forward(p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
 }
-int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* O,
+int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const void* O,
                        const float* den, const void* G, const StateArgs& sa, const void* saved, void* dQ, void* dK,
                        void* dV, void* ws, cudaStream_t st) {
     (void)O; (void)den;      // everything needed is recomputed consistently
-    return tc::causal_backward(p, Q, K, V, G, sa, saved, dQ, dK, dV, ws, st);
+    return tc::causal_backward(p, Q, K, V, lengths, G, sa, saved, dQ, dK, dV, ws, st);
 }
 int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, void* O,
                       float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st) {

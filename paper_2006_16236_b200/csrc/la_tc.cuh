@@ -13,10 +13,11 @@ size_t tc_causal_saved_bytes(const la_problem& p);
 void tc_set_plan_override(int causal_pieces, int causal_short, int linear_splits);
 // pieces, parts, piece_begin[], piece_first_part[], part_begin[], launch_order[] (see la_causal_plan)
 int tc_causal_plan(const la_problem& p, int32_t* out, int capacity);
-int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+// lengths ([B] int32, device, or null): real positions per batch element of a right-padded ragged batch
+int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const float* S_in,
                       const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
                       cudaStream_t st);
-int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* O,
+int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const void* O,
                        const float* den, const void* G, const StateArgs& sa, const void* saved, void* dQ, void* dK,
                        void* dV, void* ws, cudaStream_t st);
 // lengths ([B] int32, device, or null): real positions per batch element of a right-padded ragged batch
@@ -29,11 +30,11 @@ int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const 
 namespace tc {
 size_t causal_forward_workspace(const la_problem& p);
 size_t causal_saved_bytes(const la_problem& p);
-int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const float* S_in,
                    const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
                    cudaStream_t st);
 size_t causal_backward_workspace(const la_problem& p);
-int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const void* G,
                     const StateArgs& sa, const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 size_t linear_forward_workspace(const la_problem& p);
 size_t linear_backward_workspace(const la_problem& p);

@@ -920,8 +920,9 @@ size_t causal_backward_workspace(const la_problem& p) {
     return bytes;
 }
 
-int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const void* G,
+int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const void* G,
                     const StateArgs& sa, const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+    if (lengths) return general_causal_backward(p, Q, K, V, lengths, G, sa, dQ, dK, dV, ws, st);
     const CausalPlan pl = choose_plan(p);
     // With what the forward saved, phi(Q) and phi(K) are read as tensors (no feature map on load)
     // and the forward pre-pass records are the forward's own.

@@ -509,9 +509,10 @@ size_t causal_forward_workspace(const la_problem& p) {
 
 size_t causal_saved_bytes(const la_problem& p) { return saved_layout(p, choose_plan(p)).bytes; }
 
-int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const float* S_in,
+int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const float* S_in,
                    const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
                    cudaStream_t st) {
+    if (lengths) return general_causal_forward(p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, st);
     const CausalPlan pl = choose_plan(p);
     const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
     const SavedLayout sl = saved_layout(p, pl);

@@ -729,3 +729,88 @@ def test_decode_layer_rejects_what_it_does_not_take():
     with pytest.raises(la.LaError) as e:
         la.la_decode_layer_step(x, W3, W1, S, Z)
     assert e.value.status == -2
+
+
+def _poison_padding(tensors, lengths):
+    """Inf and NaN on everything behind each sequence's end: none of it may reach a result."""
+    for i, t in enumerate(tensors):
+        for b, n in enumerate(lengths):
+            t[b, :, n:] = float("nan") if (i + b) % 2 else float("inf")
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape,lengths", [
+    ((4, 2, 100, 16, 48), [100, 37, 1, 0]),                       # general kernels, ragged chunk tails
+    ((3, 2, 384, 64, 64), [384, 129, 300]),                       # bf16: the tensor-core shapes
+    ((6, 4, 1024, 64, 64), [1024, 0, 1, 128, 641, 900]),          # whole chunks, a chunk boundary, nothing at all
+    ((2, 32, 2304, 64, 64), [2304, 1000]),                        # B*H = 64: sequences cut into pieces with a pre-pass
+])
+def test_causal_ragged_batches(shape, lengths, dtype):
+    """la_causal_forward_varlen / _backward_varlen on a right-padded batch: every sequence against the oracle run
+    on its own length; zeros on the padding, which holds Inf and NaN on the way in; the state handed back is the
+    one at each sequence's own end, and a decode step continues from it (a ragged prefill followed by
+    generation, checked against the N x N definition of the sequence one token longer)."""
+    B, H, N, D, M = shape
+    Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=300 + N + D, dtype=dtype)
+    nxt = draw_qkvg(B, H, 1, D, M, seed=301 + N, dtype=dtype, with_grad=False)[:3]
+    clean = [t.clone() for t in (Q, K, V, G)]
+    _poison_padding((Q, K, V, G), lengths)
+    Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
+    ln = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    den = torch.full((B, H, N), 7.0, device=DEV)
+    S = torch.full((B, H, D, M), 7.0, device=DEV)
+    Z = torch.full((B, H, D), 7.0, device=DEV)
+    O = la.la_causal_forward(Qd, Kd, Vd, lengths=ln, den=den, S_out=S, Z_out=Z)
+    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd, lengths=ln)
+    la.la_last_device_status()
+    # one decode step per stream from the state the ragged prefill handed back
+    q1, k1, v1 = (t[:, :, 0].contiguous() for t in gpu(*nxt))
+    out1 = la.la_recurrent_step(q1, k1, v1, S.clone(), Z.clone())
+    for b, n in enumerate(lengths):
+        sl = slice(b, b + 1)
+        q, k, v, g = (t[sl, :, :n] for t in clean)
+        for t, nm in ((O, "O"), (den, "den"), (dQ, "dQ"), (dK, "dK"), (dV, "dV")):
+            assert torch.all(t[sl, :, n:] == 0), f"{nm}: padding of sequence {b} is not zero"
+        Or, denr, Sr, Zr = oracle.linear_attention(q, k, v, True, return_state=True)
+        assert_close(S[sl], Sr, dtype, f"S at the end, length {n}")
+        assert_close(Z[sl], Zr, dtype, f"Z at the end, length {n}")
+        if n:
+            assert_close(O[sl, :, :n], Or, dtype, f"O, length {n}")
+            assert_close(den[sl, :, :n], denr, dtype, f"den, length {n}")
+            for got, ref, nm in zip((dQ, dK, dV), oracle.linear_attention_backward(q, k, v, g, True), "QKV"):
+                assert_close(got[sl, :, :n], ref, dtype, f"d{nm}, length {n}", grad=True)
+        longer = [torch.cat([a, c[sl]], 2) for a, c in zip((q, k, v), nxt)]
+        assert_close(out1[sl], oracle.attention_quadratic(*longer, True)[:, :, n], dtype, f"decode after prefill, length {n}")
+
+
+def test_causal_ragged_batch_from_a_state_with_state_gradients():
+    """The ragged calls with every state argument: the sequences continue from S_0, Z_0, the upstream gradient
+    of the state at each sequence's own end comes in, the gradient of the initial state goes out."""
+    B, H, N, D = 3, 2, 512, 64
+    lengths = [512, 200, 77]
+    dtype = torch.bfloat16
+    Q, K, V, G = draw_qkvg(B, H, N, D, D, seed=410, dtype=dtype)
+    g = torch.Generator().manual_seed(411)
+    S0, Z0 = torch.rand((B, H, D, D), generator=g) * 2 - 1, torch.rand((B, H, D), generator=g) * 4 + 1
+    dS, dZ = (torch.rand((B, H, D, D), generator=g) - 0.5) * 0.02, (torch.rand((B, H, D), generator=g) - 0.5) * 0.02
+    Qd, Kd, Vd, Gd, S0d, Z0d, dSd, dZd = gpu(Q, K, V, G, S0, Z0, dS, dZ)
+    ln = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    S1, Z1 = torch.empty_like(S0d), torch.empty_like(Z0d)
+    O = la.la_causal_forward(Qd, Kd, Vd, lengths=ln, S_in=S0d, Z_in=Z0d, S_out=S1, Z_out=Z1)
+    dS0, dZ0 = torch.empty_like(S0d), torch.empty_like(Z0d)
+    dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd, lengths=ln, S_in=S0d, Z_in=Z0d, dS_out=dSd, dZ_out=dZd,
+                                       dS_in=dS0, dZ_in=dZ0)
+    la.la_last_device_status()
+    for b, n in enumerate(lengths):
+        sl = slice(b, b + 1)
+        q, k, v, gg = (t[sl, :, :n] for t in (Q, K, V, G))
+        Or, _, Sr, Zr = oracle.causal_from_state(q, k, v, S0[sl], Z0[sl])
+        assert_close(O[sl, :, :n], Or, dtype, f"O from a state, length {n}")
+        assert_close(S1[sl], Sr, dtype, f"S_N from a state, length {n}")
+        assert_close(Z1[sl], Zr, dtype, f"Z_N from a state, length {n}")
+        rq, rk, rv, rS, rZ = oracle.causal_backward_from_state(q, k, v, S0[sl], Z0[sl], gg, dS[sl], dZ[sl])
+        assert_close(dQ[sl, :, :n], rq, dtype, f"dQ from a state, length {n}", grad=True)
+        assert_close(dK[sl, :, :n], rk, dtype, f"dK from a state, length {n}", grad=True)
+        assert_close(dV[sl, :, :n], rv, dtype, f"dV from a state, length {n}", grad=True)
+        assert_close(dS0[sl], rS, dtype, f"dS_0, length {n}")
+        assert_close(dZ0[sl], rZ, dtype, f"dZ_0, length {n}")
