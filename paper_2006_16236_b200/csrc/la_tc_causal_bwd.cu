@@ -99,8 +99,14 @@ struct DqParams {
     int dim;                    // D = M: 64, or 32 (tiles zero-padded to 64 columns)
     int map;                    // apply the feature map on load (0: the inputs are already phi(Q), phi(K))
     const int* stamp;           // the plan the forward recorded in the saved buffer, or null (no saved buffer)
+    const int* lengths;         // [B] real positions per batch element of a right-padded ragged batch (kVarlen only)
+    int heads;
+    __nv_bfloat16* dQ;          // for the rows of padding, which are zeroed with plain stores (kVarlen only)
 };
 
+// kVarlen: a right-padded ragged batch (see the forward kernel): chunks behind a sequence's end are skipped and
+// their dQ rows zeroed, the padded rows of the chunk that holds the end are zeroed in shared memory.
+template <bool kVarlen>
 __global__ void __launch_bounds__(kDqThreads, 1)
 causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                      const __grid_constant__ CUtensorMap mapG, const __grid_constant__ CUtensorMap mapQ,
@@ -117,7 +123,11 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     const int64_t bh = blockIdx.x % plan.bh;                        // long pieces first: see CausalPlan
     const int piece = plan.piece_of_slot(blockIdx.x / plan.bh);
     const int c_begin = plan.piece_begin(piece);
-    const int L = plan.piece_begin(piece + 1) - c_begin;
+    const int L_full = plan.piece_begin(piece + 1) - c_begin;
+    RaggedSpan span{L_full, kChunk, false};
+    if (kVarlen) span = ragged_span(prm.lengths, prm.heads, bh, prm.N, c_begin, L_full);
+    const int L = span.chunks;                  // chunks this CTA processes
+    const int tail_rows = span.tail_rows;       // real rows of the last of them
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
 
     if (tid == 0) {
@@ -177,6 +187,8 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
 
     if (mismatch) {             // the same for every thread: nothing is started, the CTA leaves through the common exit
         if (tid == 0) atomicOr(prm.status, kStatusPlanMismatch);
+    } else if (kVarlen && L == 0) {
+        // this piece is all padding: nothing to sweep (its dQ rows are zeroed below)
     } else if (warp == 12) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -309,6 +321,13 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 uint8_t* rowK = smem + kDqOffStage + s * 4 * kTileBytes + t * 128;
                 phi_row_inplace(rowK, r7, prm.dim >> 3);
                 phi_row_inplace(rowK + 3 * kTileBytes, r7, prm.dim >> 3);
+                fence_proxy_async_smem();
+            }
+            if (kVarlen && c == L - 1 && t >= tail_rows) {      // padding: no key feature, no value, no upstream gradient
+                uint8_t* rowK = smem + kDqOffStage + s * 4 * kTileBytes + t * 128;
+                zero_row(rowK);
+                zero_row(rowK + kTileBytes);
+                zero_row(rowK + 2 * kTileBytes);
                 fence_proxy_async_smem();
             }
             mbar_arrive(&bars->mapped[s]);
@@ -446,9 +465,10 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             const float inv = 1.f / dn;
             const float delta = -qg * inv;                  // = -(G_i . O_i)
             const int64_t row = row0 + (int64_t)c * kChunk + t;
+            const bool pad = kVarlen && c == L - 1 && t >= tail_rows;     // a padded row of the chunk that holds the sequence's end
             if (half == 0) {
-                prm.dn[row] = dn;
-                prm.dl[row] = delta;
+                prm.dn[row] = pad ? 1.f : dn;
+                prm.dl[row] = pad ? 0.f : delta;
             }
             // dQ leaves through a staging tile: each quadrant (two warps, 32 rows) fills its 4 KB slab and one
             // of its threads stores it with TMA: full 128-byte rows per request instead of 32 rows per store
@@ -467,7 +487,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                         g0 *= q0 > 1.f ? 1.f : q0;
                         g1 *= q1 > 1.f ? 1.f : q1;
                     }
-                    outp[j] = pack_bf16x2(g0, g1);
+                    outp[j] = pad ? 0u : pack_bf16x2(g0, g1);
                 }
                 sts128(out_row + (((half * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
             }
@@ -483,6 +503,17 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         }
         if (half == 0 && lane == 0) tma_store_wait_all<0>();
         if (!ok) *abort_flag = 1;
+    }
+    if (kVarlen && warp < 8 && !mismatch) {      // chunks of this piece behind the sequence's end: zero gradient
+        const int t = (warp & 3) * 32 + lane, half = warp >> 2;
+        #pragma unroll 1
+        for (int c = L; c < L_full; ++c) {
+            if (half * 32 < prm.dim) {
+                __nv_bfloat16* dst = prm.dQ + (row0 + (int64_t)c * kChunk + t) * prm.dim + half * 32;
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) stg128(dst + cc * 8, 0u, 0u, 0u, 0u);
+            }
+        }
     }
 
     tc_fence_before_sync();
@@ -538,8 +569,15 @@ struct KvParams {
     int phi;
     int dim;
     int map;                    // apply the feature map on load (0: the inputs are already phi(Q), phi(K))
+    const int* lengths;         // [B] real positions per batch element of a right-padded ragged batch (kVarlen only)
+    int heads;
+    __nv_bfloat16* dK;          // for the rows of padding, which are zeroed with plain stores (kVarlen only)
+    __nv_bfloat16* dV;
 };
 
+// kVarlen: a right-padded ragged batch (see the forward kernel): the sweep starts at the sequence's last real
+// chunk, whose padded rows are zeroed in shared memory; the dK, dV rows of the skipped chunks are zeroed.
+template <bool kVarlen>
 __global__ void __launch_bounds__(kKvThreads, 1)
 causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                       const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapG,
@@ -555,8 +593,13 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
     const int64_t bh = blockIdx.x % plan.bh;                        // long pieces first: see CausalPlan
     const int piece = plan.piece_of_slot(blockIdx.x / plan.bh);
     const int c_begin = plan.piece_begin(piece);
-    const int c_end = plan.piece_begin(piece + 1);
-    const int L = c_end - c_begin;
+    const int L_full = plan.piece_begin(piece + 1) - c_begin;
+    RaggedSpan span{L_full, kChunk, false};
+    if (kVarlen) span = ragged_span(prm.lengths, prm.heads, bh, prm.N, c_begin, L_full);
+    const int L = span.chunks;                  // chunks this CTA processes
+    const int tail_rows = span.tail_rows;       // real rows of the first one it visits (the sequence's last)
+    const int c_end = c_begin + L;
+    const bool idle = kVarlen && L == 0;        // all padding: only the state gradient passes through (warps 8-11)
     // iteration i visits chunk c_end - 1 - i
     auto chunk_row = [&](int i) { return bh * prm.N + (int64_t)(c_end - 1 - i) * kChunk; };
 
@@ -609,7 +652,9 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
-    if (warp == 16) {
+    if (idle && (warp < 8 || warp >= 12)) {
+        // nothing to sweep
+    } else if (warp == 16) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG);
@@ -758,6 +803,12 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             if (i >= 1 && !mbar_wait(&bars->r_full, (i - 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             if (t == 0) LA_TRACE(g_trace_dkv, i, 15);
             // dl_i as a bf16 high and low part in columns 0 and 1 (the rest of the row stays zero)
+            if (kVarlen && i == 0 && t >= tail_rows) {          // padding: the row takes no part in any product
+                zero_row(rowQ);
+                zero_row(rowQ + kTileBytes);
+                zero_row(rowQ + 2 * kTileBytes);
+                zero_row(rowQ + 3 * kTileBytes);
+            }
             const float dl_hi = bf16_lo(pack_bf16x2(delta, 0.f));
             sts128(smem + kKvOffAux + t * 128 + ((0 ^ r7) << 4), pack_bf16x2(dl_hi, delta - dl_hi), 0u, 0u, 0u);
             fence_proxy_async_smem();
@@ -862,7 +913,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                             const float g1 = __uint_as_float(v[cc * 8 + 2 * j + 1]) + rr[2 * j + 1];
                             const float s0 = fmaxf(fminf(bf16_lo(kf[j]), 1.f), slope_floor);
                             const float s1 = fmaxf(fminf(bf16_hi(kf[j]), 1.f), slope_floor);
-                            outp[j] = pack_bf16x2(g0 * s0, g1 * s1);
+                            outp[j] = (kVarlen && i == 0 && t >= tail_rows) ? 0u : pack_bf16x2(g0 * s0, g1 * s1);
                         }
                         sts128(const_cast<uint8_t*>(rowK) + (((h * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
                     }
@@ -884,6 +935,16 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             rstate_write(tmem + kKvColR, quad, lane, prm.dS_in ? prm.dS_in + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
                          prm.dZ_in ? prm.dZ_in + bh * prm.dim : nullptr, prm.dim);
         if (t == 0) tma_store_wait_all<0>();
+        if (kVarlen) {          // chunks of this piece behind the sequence's end: zero gradient
+            #pragma unroll 1
+            for (int c = c_end; c < c_begin + L_full; ++c) {
+                const int64_t row = bh * prm.N + (int64_t)c * kChunk + t;
+                for (int cc = 0; cc < prm.dim / 8; ++cc) {
+                    stg128(prm.dK + row * prm.dim + cc * 8, 0u, 0u, 0u, 0u);
+                    stg128(prm.dV + row * prm.dim + cc * 8, 0u, 0u, 0u, 0u);
+                }
+            }
+        }
     } else {
         // ------------------------------------------- score warps: Ph^T and dP^T, masked and rounded in place
         const int quad = warp & 3, half = warp >> 2;
@@ -922,7 +983,7 @@ size_t causal_backward_workspace(const la_problem& p) {
 
 int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const void* G,
                     const StateArgs& sa, const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
-    if (lengths) return general_causal_backward(p, Q, K, V, lengths, G, sa, dQ, dK, dV, ws, st);
+    if (lengths) saved = nullptr;       // a ragged batch keeps nothing from the forward pass
     const CausalPlan pl = choose_plan(p);
     // With what the forward saved, phi(Q) and phi(K) are read as tensors (no feature map on load)
     // and the forward pre-pass records are the forward's own.
@@ -952,14 +1013,19 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     int* status = device_status_ptr();
     if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
 
-    static std::atomic<uint64_t> attr_dq{0}, attr_dkv{0};
-    if (int rc = opt_in_smem_once(causal_bwd_dq_kernel, kDqSmemBytes, attr_dq)) return rc;
-    if (int rc = opt_in_smem_once(causal_bwd_dkv_kernel, kKvSmemBytes, attr_dkv)) return rc;
+    static std::atomic<uint64_t> attr_dq{0}, attr_dkv{0}, attr_dq_ragged{0}, attr_dkv_ragged{0};
+    if (lengths) {
+        if (int rc = opt_in_smem_once(causal_bwd_dq_kernel<true>, kDqSmemBytes, attr_dq_ragged)) return rc;
+        if (int rc = opt_in_smem_once(causal_bwd_dkv_kernel<true>, kKvSmemBytes, attr_dkv_ragged)) return rc;
+    } else {
+        if (int rc = opt_in_smem_once(causal_bwd_dq_kernel<false>, kDqSmemBytes, attr_dq)) return rc;
+        if (int rc = opt_in_smem_once(causal_bwd_dkv_kernel<false>, kKvSmemBytes, attr_dkv)) return rc;
+    }
     const unsigned grid = (unsigned)(pl.npieces() * bh);
 
     // forward sweep: dQ, and dn_i, dl_i for the reverse sweep
     if (sv) rec_s = (float*)(sv + sl.records);
-    else if (int rc = segment_states(p, pl, mK, mV, nullptr, nullptr, rec_s, /*reverse=*/false, map, st)) return rc;
+    else if (int rc = segment_states(p, pl, mK, mV, nullptr, nullptr, rec_s, /*reverse=*/false, map, st, lengths)) return rc;
     DqParams a;
     a.dn = dn;
     a.dl = dl;
@@ -974,17 +1040,21 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.dim = (int)p.D;
     a.map = map ? 1 : 0;
     a.stamp = sv ? (const int*)(sv + sl.stamp) : nullptr;
+    a.lengths = lengths;
+    a.heads = (int)p.H;
+    a.dQ = (__nv_bfloat16*)dQ;
     prof_begin(kProfCausalBwdDq, st);
     CUtensorMap mDQ;
     if (int rc = encode_tile_map(&mDQ, dQ, rows, 32, (int)p.D)) return rc;      // one quadrant's rows per store
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg_q = chained_launch(grid, kDqThreads, kDqSmemBytes, st, &attr);
-    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_q, causal_bwd_dq_kernel, mK, mV, mG, mQ, mDQ, a));
+    if (lengths) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_q, causal_bwd_dq_kernel<true>, mK, mV, mG, mQ, mDQ, a));
+    else LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_q, causal_bwd_dq_kernel<false>, mK, mV, mG, mQ, mDQ, a));
     note_launch();
     prof_end(kProfCausalBwdDq, st);
 
     // reverse sweep: dK, dV
-    if (int rc = segment_states(p, pl, mQ, mG, dn, dl, rec_r, /*reverse=*/true, map, st)) return rc;
+    if (int rc = segment_states(p, pl, mQ, mG, dn, dl, rec_r, /*reverse=*/true, map, st, lengths)) return rc;
     KvParams b;
     b.dn = dn;
     b.dl = dl;
@@ -1000,12 +1070,17 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     b.phi = p.phi;
     b.dim = (int)p.D;
     b.map = map ? 1 : 0;
+    b.lengths = lengths;
+    b.heads = (int)p.H;
+    b.dK = (__nv_bfloat16*)dK;
+    b.dV = (__nv_bfloat16*)dV;
     prof_begin(kProfCausalBwdDkv, st);
     CUtensorMap mDK, mDV;
     if (int rc = encode_tile_map(&mDK, dK, rows, kChunk, (int)p.D)) return rc;
     if (int rc = encode_tile_map(&mDV, dV, rows, kChunk, (int)p.D)) return rc;
     const cudaLaunchConfig_t cfg_kv = chained_launch(grid, kKvThreads, kKvSmemBytes, st, &attr);
-    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_kv, causal_bwd_dkv_kernel, mQ, mK, mV, mG, mDK, mDV, b));
+    if (lengths) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_kv, causal_bwd_dkv_kernel<true>, mQ, mK, mV, mG, mDK, mDV, b));
+    else LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_kv, causal_bwd_dkv_kernel<false>, mQ, mK, mV, mG, mDK, mDV, b));
     note_launch();
     prof_end(kProfCausalBwdDkv, st);
     return LA_OK;

@@ -78,11 +78,17 @@ struct FwdParams {
     int dim;               // D = M: 64, or 32 (tiles zero-padded to 64 columns)
     int save;              // store the mapped phi(Q), phi(K) tiles for the backward pass
     int* stamp;            // where the plan is recorded for the backward pass (in the saved buffer), or null
+    const int* lengths;    // [B] real positions per batch element of a right-padded ragged batch (kVarlen only)
+    int heads;
 };
 
 // ---------------------------------------------------------------------------
 // Main kernel.
 // ---------------------------------------------------------------------------
+// kVarlen: a right-padded ragged batch (prm.lengths): chunks behind a sequence's end are skipped and their
+// outputs zeroed, the padded rows of the chunk that holds the end are zeroed in shared memory.  The other
+// instantiation carries none of that code.
+template <bool kVarlen>
 __global__ void __launch_bounds__(kThreads, 1)
 causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapPQ,
@@ -97,7 +103,12 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     const int piece = plan.piece_of_slot(blockIdx.x / plan.bh);
     const bool last_piece = piece == plan.npieces() - 1;
     const int c_begin = plan.piece_begin(piece);
-    const int L = plan.piece_begin(piece + 1) - c_begin;
+    const int L_full = plan.piece_begin(piece + 1) - c_begin;
+    RaggedSpan span{L_full, kChunk, last_piece};
+    if (kVarlen) span = ragged_span(prm.lengths, prm.heads, bh, prm.N, c_begin, L_full);
+    const int L = span.chunks;                                        // chunks this CTA processes
+    const int tail_rows = span.tail_rows;                             // real rows of the last of them
+    const bool ends_here = span.has_end;                              // the final state is this CTA's to write
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;      // first global row of this segment
 
     LA_TRACE_CTA(g_trace_fwd, 0);
@@ -273,6 +284,10 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 phi_row_inplace(tile + t * 128, r7, prm.dim >> 3);
                 fence_proxy_async_smem();
             }
+            if (kVarlen && c == L - 1 && t >= tail_rows) {      // padding: its values take no part in any product
+                zero_row(tile + 2 * kTileBytes + t * 128);
+                fence_proxy_async_smem();
+            }
             if (prm.save) {         // the whole mapped tile goes out with one bulk store
                 named_barrier(3, 128);
                 if (t == 0) {
@@ -295,7 +310,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 if (*abort_flag) { ok = false; break; }
                 if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
                 tc_fence_after_sync();
-                const bool fin = (c == L - 1) && last_piece;
+                const bool fin = (c == L - 1) && ends_here;
                 uint8_t* tile = smem + kOffS + (c & 1) * kStateTileBytes;
                 state_half_to_tiles(tmem + kColS, quad, lane, 1, tile, nullptr, &bars->s_drained,
                                     fin && prm.S_out ? prm.S_out + bh * (int64_t)(prm.dim * prm.dim) : nullptr, nullptr, prm.dim);
@@ -333,6 +348,10 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 phi_row_inplace(tile + t * 128, r7, prm.dim >> 3);
                 fence_proxy_async_smem();
             }
+            if (kVarlen && c == L - 1 && t >= tail_rows) {      // padding: no feature, so no score and no state update
+                zero_row(tile + t * 128);
+                fence_proxy_async_smem();
+            }
             if (prm.save) {
                 named_barrier(4, 128);
                 if (t == 0) {
@@ -357,7 +376,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 if (!mbar_wait(&bars->s_full, c & 1, prm.status, kStatusMmaTimeout)) { ok = false; break; }
                 tc_fence_after_sync();
                 if (t == 0) LA_TRACE(g_trace_fwd, c, 7);
-                const bool fin = (c == L - 1) && last_piece;
+                const bool fin = (c == L - 1) && ends_here;
                 uint8_t* tile = smem + kOffS + (c & 1) * kStateTileBytes;
                 state_half_to_tiles(tmem + kColS, quad, lane, 0, tile, tile + kDim * 128, &bars->s_drained,
                                     fin && prm.S_out ? prm.S_out + bh * (int64_t)(prm.dim * prm.dim) : nullptr,
@@ -417,6 +436,15 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             mbar_arrive(&bars->o_drained[b]);
             const float inv = 1.f / (den + prm.eps);
             const int64_t row = row0 + (int64_t)c * kChunk + t;
+            if (kVarlen && c == L - 1 && t >= tail_rows) {  // a padded row of the chunk that holds the sequence's end
+                if (half == 0 && prm.den) prm.den[row] = 0.f;
+                if (half * 32 < prm.dim) {
+                    __nv_bfloat16* dst = prm.O + row * prm.dim + half * 32;
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) stg128(dst + cc * 8, 0u, 0u, 0u, 0u);
+                }
+                return true;
+            }
             if (half == 0 && prm.den) prm.den[row] = den;
             if (half * 32 < prm.dim) {                      // columns beyond a 32-wide problem are padding
                 __nv_bfloat16* dst = prm.O + row * prm.dim + half * 32;
@@ -445,6 +473,18 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             if (c >= 1) ok = epilogue(c - 1);
         }
         if (!ok) *abort_flag = 1;
+        if (kVarlen) {          // chunks of this piece behind the sequence's end: zeros
+            #pragma unroll 1
+            for (int c = L; c < L_full; ++c) {
+                const int64_t row = row0 + (int64_t)c * kChunk + t;
+                if (half == 0 && prm.den) prm.den[row] = 0.f;
+                if (half * 32 < prm.dim) {
+                    __nv_bfloat16* dst = prm.O + row * prm.dim + half * 32;
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) stg128(dst + cc * 8, 0u, 0u, 0u, 0u);
+                }
+            }
+        }
     }
 
     tc_fence_before_sync();
@@ -512,7 +552,7 @@ size_t causal_saved_bytes(const la_problem& p) { return saved_layout(p, choose_p
 int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const float* S_in,
                    const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
                    cudaStream_t st) {
-    if (lengths) return general_causal_forward(p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, st);
+    if (lengths) saved = nullptr;       // a ragged batch keeps nothing for the backward pass
     const CausalPlan pl = choose_plan(p);
     const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
     const SavedLayout sl = saved_layout(p, pl);
@@ -527,12 +567,26 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     int* status = device_status_ptr();
     if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
 
-    static std::atomic<uint64_t> attr_done{0};
-    if (int rc = opt_in_smem_once(causal_fwd_kernel, kSmemBytes, attr_done)) return rc;
+    static std::atomic<uint64_t> attr_done{0}, attr_done_ragged{0};
+    if (int rc = lengths ? opt_in_smem_once(causal_fwd_kernel<true>, kSmemBytes, attr_done_ragged)
+                         : opt_in_smem_once(causal_fwd_kernel<false>, kSmemBytes, attr_done)) return rc;
     // the pre-pass records go straight into the saved buffer when there is one
     float* records = sv ? (float*)(sv + sl.records) : (float*)ws;
     if (pl.npieces() > 1) {
-        if (int rc = segment_states(p, pl, mK, mV, nullptr, nullptr, records, /*reverse=*/false, p.phi == LA_PHI_ELU1, st)) return rc;
+        if (int rc = segment_states(p, pl, mK, mV, nullptr, nullptr, records, /*reverse=*/false, p.phi == LA_PHI_ELU1, st, lengths)) return rc;
+    }
+    if (lengths) {
+        // the final state is written by the CTA that holds a sequence's last real chunk; a sequence without any
+        // keeps the state it started from
+        const size_t s_bytes = (size_t)(p.B * p.H * p.D * p.M) * sizeof(float), z_bytes = (size_t)(p.B * p.H * p.D) * sizeof(float);
+        if (S_out) {
+            if (S_in) LA_CUDA_TRY(cudaMemcpyAsync(S_out, S_in, s_bytes, cudaMemcpyDeviceToDevice, st));
+            else LA_CUDA_TRY(cudaMemsetAsync(S_out, 0, s_bytes, st));
+        }
+        if (Z_out) {
+            if (Z_in) LA_CUDA_TRY(cudaMemcpyAsync(Z_out, Z_in, z_bytes, cudaMemcpyDeviceToDevice, st));
+            else LA_CUDA_TRY(cudaMemsetAsync(Z_out, 0, z_bytes, st));
+        }
     }
     FwdParams prm;
     prm.O = (__nv_bfloat16*)O;
@@ -550,10 +604,13 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     prm.dim = (int)p.D;
     prm.save = save ? 1 : 0;
     prm.stamp = sv ? (int*)(sv + sl.stamp) : nullptr;
+    prm.lengths = lengths;
+    prm.heads = (int)p.H;
     prof_begin(kProfCausalFwd, st);
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = chained_launch((unsigned)(pl.npieces() * pl.bh), kThreads, kSmemBytes, st, &attr);
-    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, causal_fwd_kernel, mQ, mK, mV, mPQ, mPK, prm));
+    if (lengths) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, causal_fwd_kernel<true>, mQ, mK, mV, mPQ, mPK, prm));
+    else LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, causal_fwd_kernel<false>, mQ, mK, mV, mPQ, mPK, prm));
     note_launch();
     prof_end(kProfCausalFwd, st);
     return LA_OK;

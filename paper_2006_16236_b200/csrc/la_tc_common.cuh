@@ -133,8 +133,10 @@ CausalPlan choose_plan(const la_problem& p);
 
 // Per-part sums of phi(X)^T [Y | a] into `records` (forward: the parts before the last piece; reverse:
 // the parts after the first piece)
+// lengths ([B] int32, device, or null): real positions per batch element of a right-padded ragged batch
 int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap& mapX, const CUtensorMap& mapY,
-                   const float* dn, const float* dl, float* records, bool reverse, bool map, cudaStream_t st);
+                   const float* dn, const float* dl, float* records, bool reverse, bool map, cudaStream_t st,
+                   const int* lengths = nullptr);
 
 // What the causal forward leaves for the causal backward when the caller passes a `saved`
 // buffer: the mapped phi(Q) and phi(K) ([B*H*N, D] bf16 each, exactly the operands the
@@ -256,6 +258,29 @@ __device__ __forceinline__ void map_row_inplace(uint8_t* row, uint32_t r7, float
 }
 __device__ __forceinline__ void phi_row_inplace(uint8_t* row, uint32_t r7, int nch = 8) {
     map_row_inplace<true, false>(row, r7, 1.f, nch);
+}
+
+// Right-padded ragged batches.  Of the chunks [c_begin, c_begin + n_full) a CTA is responsible for, only those
+// that hold real positions of the sequence are processed; the last of them may be partly padding.
+struct RaggedSpan {
+    int chunks;         // chunks of the span to process (0: the span is all padding)
+    int tail_rows;      // real rows of the last processed chunk (kChunk unless the sequence ends inside it)
+    bool has_end;       // the sequence's last real chunk lies in this span
+};
+__device__ __forceinline__ RaggedSpan ragged_span(const int* lengths, int heads, int64_t bh, int64_t N, int c_begin, int n_full) {
+    int64_t len = lengths[bh / heads];
+    len = len < 0 ? 0 : (len < N ? len : N);
+    const int nc = (int)((len + kChunk - 1) / kChunk);              // chunks of the sequence with real rows
+    RaggedSpan r;
+    r.chunks = nc - c_begin < 0 ? 0 : (nc - c_begin < n_full ? nc - c_begin : n_full);
+    r.has_end = r.chunks > 0 && c_begin + r.chunks == nc;
+    r.tail_rows = r.has_end ? (int)(len - (int64_t)(nc - 1) * kChunk) : kChunk;
+    return r;
+}
+// A whole 128-byte tile row of zeros (padding rows of a ragged batch: whatever they held, they contribute nothing).
+__device__ __forceinline__ void zero_row(uint8_t* row) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) sts128(row + (c << 4), 0u, 0u, 0u, 0u);
 }
 
 __device__ __forceinline__ uint64_t desc_k(uint32_t addr) { return sm100::umma_desc_sw128(addr, 16, 1024); }

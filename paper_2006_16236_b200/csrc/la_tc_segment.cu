@@ -48,8 +48,13 @@ struct SumParams {
     float eps;
     int map;               // apply the feature map to X on load
     int dim;
+    const int* lengths;    // [B] real positions per batch element of a right-padded ragged batch (kVarlen only)
+    int heads;
 };
 
+// kVarlen: a right-padded ragged batch: only the chunks of the part that hold real positions are summed, the
+// padded rows of the chunk that holds a sequence's end are zeroed, a part that is all padding gives a zero record.
+template <bool kVarlen>
 __global__ void __launch_bounds__(kSumThreads, 2)
 segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                    const SumParams prm) {
@@ -61,7 +66,10 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     const int seg = prm.first_part + blockIdx.x % prm.parts_per_seq;       // index of this part
     const int64_t bh = blockIdx.x / prm.parts_per_seq;
     const int c_begin = prm.plan.part_begin(seg);
-    const int L = prm.plan.part_begin(seg + 1) - c_begin;
+    const int L_full = prm.plan.part_begin(seg + 1) - c_begin;
+    RaggedSpan span{L_full, kChunk, false};
+    if (kVarlen) span = ragged_span(prm.lengths, prm.heads, bh, prm.N, c_begin, L_full);
+    const int L = span.chunks;
     const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
     const bool scaled = prm.dn != nullptr;
 
@@ -161,6 +169,11 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
                 else phi_row_inplace(rowX, r7, prm.dim >> 3);
             }
             else if (scaled) map_row_inplace<false>(rowX, r7, inv, prm.dim >> 3);
+            if (kVarlen && c == L - 1 && t >= span.tail_rows) {     // padding: no feature, no value, no dl
+                zero_row(rowX);
+                zero_row(rowX + kTileBytes);
+                delta = 0.f;
+            }
             if (scaled) {
                 // the single column tile is still an operand of the previous chunk's products
                 if (c >= 1 && !mbar_wait(&bars->empty[(c - 1) % kSumStages], ((c - 1) / kSumStages) & 1, prm.status,
@@ -176,6 +189,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
         }
         if (t == 0) LA_TRACE(g_trace_seg, 100, 7);
         // read-out: the [S | Z]-shaped record of this (bh, seg)
+        const bool empty = kVarlen && L == 0;           // nothing was summed: the accumulator holds no result
         const bool ok = mbar_wait(&bars->done, 0, prm.status, kStatusMmaTimeout) && !*abort_flag;
         tc_fence_after_sync();
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
@@ -187,11 +201,11 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             tmem_ld_wait();
             if (ok && lane < 16)
 #pragma unroll
-                for (int j = 0; j < 32; ++j) rec[d_row * kDim + h * 32 + j] = __uint_as_float(v[j]);
+                for (int j = 0; j < 32; ++j) rec[d_row * kDim + h * 32 + j] = empty ? 0.f : __uint_as_float(v[j]);
         }
         const float z = __uint_as_float(tmem_ld1(tmem + lane_base + 64));
         tmem_ld_wait();
-        if (ok && lane < 16) rec[kDim * kDim + d_row] = z;
+        if (ok && lane < 16) rec[kDim * kDim + d_row] = empty ? 0.f : z;
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -205,10 +219,12 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
 }  // namespace
 
 int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap& mapX, const CUtensorMap& mapY,
-                   const float* dn, const float* dl, float* records, bool reverse, bool map, cudaStream_t st) {
+                   const float* dn, const float* dl, float* records, bool reverse, bool map, cudaStream_t st,
+                   const int* lengths) {
     if (pl.npieces() <= 1) return LA_OK;
-    static std::atomic<uint64_t> attr_done{0};
-    if (int rc = opt_in_smem_once(segment_sum_kernel, kSumSmemBytes, attr_done)) return rc;
+    static std::atomic<uint64_t> attr_done{0}, attr_done_ragged{0};
+    if (int rc = lengths ? opt_in_smem_once(segment_sum_kernel<true>, kSumSmemBytes, attr_done_ragged)
+                         : opt_in_smem_once(segment_sum_kernel<false>, kSumSmemBytes, attr_done)) return rc;
     SumParams prm;
     prm.records = records;
     prm.dn = dn;
@@ -223,10 +239,13 @@ int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap&
     prm.eps = p.eps;
     prm.map = map ? 1 : 0;
     prm.dim = (int)p.D;
+    prm.lengths = lengths;
+    prm.heads = (int)p.H;
     prof_begin(kProfSegmentSum, st);
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = chained_launch((unsigned)(prm.parts_per_seq * p.B * p.H), kSumThreads, kSumSmemBytes, st, &attr);
-    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, segment_sum_kernel, mapX, mapY, prm));
+    if (lengths) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, segment_sum_kernel<true>, mapX, mapY, prm));
+    else LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, segment_sum_kernel<false>, mapX, mapY, prm));
     note_launch();
     prof_end(kProfSegmentSum, st);
     return LA_OK;

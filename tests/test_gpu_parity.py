@@ -791,8 +791,8 @@ def test_causal_ragged_batch_from_a_state_with_state_gradients():
     dtype = torch.bfloat16
     Q, K, V, G = draw_qkvg(B, H, N, D, D, seed=410, dtype=dtype)
     g = torch.Generator().manual_seed(411)
-    S0, Z0 = torch.rand((B, H, D, D), generator=g) * 2 - 1, torch.rand((B, H, D), generator=g) * 4 + 1
-    dS, dZ = (torch.rand((B, H, D, D), generator=g) - 0.5) * 0.02, (torch.rand((B, H, D), generator=g) - 0.5) * 0.02
+    S0, Z0 = torch.randn((B, H, D, D), generator=g) * 3.0, torch.rand((B, H, D), generator=g) * 4.0 + 1.0
+    dS, dZ = torch.randn((B, H, D, D), generator=g) * 0.05, torch.randn((B, H, D), generator=g) * 0.05
     Qd, Kd, Vd, Gd, S0d, Z0d, dSd, dZd = gpu(Q, K, V, G, S0, Z0, dS, dZ)
     ln = torch.tensor(lengths, dtype=torch.int32, device=DEV)
     S1, Z1 = torch.empty_like(S0d), torch.empty_like(Z0d)
@@ -812,5 +812,5 @@ def test_causal_ragged_batch_from_a_state_with_state_gradients():
         assert_close(dQ[sl, :, :n], rq, dtype, f"dQ from a state, length {n}", grad=True)
         assert_close(dK[sl, :, :n], rk, dtype, f"dK from a state, length {n}", grad=True)
         assert_close(dV[sl, :, :n], rv, dtype, f"dV from a state, length {n}", grad=True)
-        assert_close(dS0[sl], rS, dtype, f"dS_0, length {n}")
-        assert_close(dZ0[sl], rZ, dtype, f"dZ_0, length {n}")
+        assert_close(dS0[sl], rS, dtype, f"dS_0, length {n}", grad=True)
+        assert_close(dZ0[sl], rZ, dtype, f"dZ_0, length {n}", grad=True)
