@@ -180,7 +180,7 @@ size_t la_workspace_bytes(const la_problem* p, int32_t op) {
     if (op == LA_OP_DECODE_LAYER) return decode_layer_supported(*p) ? decode_layer_workspace(*p) : 0;
     if (p->N == 0) return 0;
     if (op == LA_OP_LINEAR_SAVED) op = LA_OP_LINEAR_FORWARD;          // the saved buffer holds what the forward's workspace holds
-    if (op == LA_OP_CAUSAL_SAVED) return tc_supported(*p, LA_OP_CAUSAL_BACKWARD) ? tc_causal_saved_bytes(*p) : 0;
+    if (op == LA_OP_CAUSAL_SAVED) return tc_supported(*p, LA_OP_CAUSAL_BACKWARD) ? tc::causal_saved_bytes(*p) : 0;
     if (op == LA_OP_LINEAR_VARLEN_FORWARD || op == LA_OP_LINEAR_VARLEN_BACKWARD) {
         const int full = op == LA_OP_LINEAR_VARLEN_FORWARD ? LA_OP_LINEAR_FORWARD : LA_OP_LINEAR_BACKWARD;
         return tc_supported(*p, full) ? tc_workspace_bytes(*p, full) : general_workspace_bytes(*p, op);
@@ -199,7 +199,7 @@ int la_causal_plan(const la_problem* p, int32_t* out, int capacity) {
 int la_plan_override(int32_t causal_pieces, int32_t causal_short, int32_t linear_splits) {
     if (causal_pieces < -1 || causal_pieces == 0 || causal_short < -1 || linear_splits < -1 || linear_splits == 0)
         return fail(LA_ERR_INVALID_ARG, "overrides are -1 (automatic) or positive counts (causal_short may be 0: no short piece)");
-    tc_set_plan_override(causal_pieces, causal_short, linear_splits);
+    tc::set_plan_override(causal_pieces, causal_short, linear_splits);
     return LA_OK;
 }
 
@@ -267,7 +267,7 @@ static int linear_forward_common(const la_problem* p, const void* Q, const void*
         if (int rc = check_ws(p, lengths ? LA_OP_LINEAR_VARLEN_FORWARD : LA_OP_LINEAR_FORWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
+    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc::linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
     return general_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
 }
 
@@ -285,7 +285,7 @@ static int linear_backward_common(const la_problem* p, const void* Q, const void
     if (int rc = check_ws(p, lengths ? LA_OP_LINEAR_VARLEN_BACKWARD : LA_OP_LINEAR_BACKWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc_linear_backward(*p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
+    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc::linear_backward(*p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
     return general_linear_backward(*p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
 }
 
@@ -369,7 +369,7 @@ static int causal_forward_common(const la_problem* p, const void* Q, const void*
     if (int rc = check_saved(p, saved, saved_bytes)) return rc;
     if (int rc = check_arch()) return rc;
     if (tc_supported(*p, LA_OP_CAUSAL_FORWARD))
-        return tc_causal_forward(*p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
+        return tc::causal_forward(*p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
     return general_causal_forward(*p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, st);
 }
 
@@ -437,7 +437,7 @@ static int causal_backward_common(const la_problem* p, const void* Q, const void
     StateArgs sa;
     sa.S_in = S_in; sa.Z_in = Z_in; sa.dS_out = dS_out; sa.dZ_out = dZ_out; sa.dS_in = dS_in; sa.dZ_in = dZ_in;
     if (tc_supported(*p, LA_OP_CAUSAL_BACKWARD))
-        return tc_causal_backward(*p, Q, K, V, lengths, O, den, G, sa, saved, dQ, dK, dV, ws, st);
+        return tc::causal_backward(*p, Q, K, V, lengths, G, sa, saved, dQ, dK, dV, ws, st);
     return general_causal_backward(*p, Q, K, V, lengths, G, sa, dQ, dK, dV, ws, st);
 }
 

@@ -14,7 +14,6 @@ PlanOverride plan_override() {
     return PlanOverride{g_override_pieces.load(std::memory_order_relaxed), g_override_short.load(std::memory_order_relaxed),
                         g_override_splits.load(std::memory_order_relaxed)};
 }
-void set_plan_override(int pieces, int short_len, int splits);
 void set_plan_override(int pieces, int short_len, int splits) {
     g_override_pieces.store(pieces, std::memory_order_relaxed);
     g_override_short.store(short_len, std::memory_order_relaxed);
@@ -124,10 +123,6 @@ size_t tc_workspace_bytes(const la_problem& p, int op) {
     }
 }
 
-size_t tc_causal_saved_bytes(const la_problem& p) { return tc::causal_saved_bytes(p); }
-void tc_set_plan_override(int causal_pieces, int causal_short, int linear_splits) {
-    tc::set_plan_override(causal_pieces, causal_short, linear_splits);
-}
 int tc_causal_plan(const la_problem& p, int32_t* out, int capacity) {
     const tc::CausalPlan pl = tc::choose_plan(p);
     const int np = pl.npieces(), nq = pl.nparts();
@@ -144,24 +139,4 @@ int tc_causal_plan(const la_problem& p, int32_t* out, int capacity) {
     for (int s = 0; s < np; ++s) put(pl.piece_of_slot(s));
     return n;
 }
-int tc_causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const float* S_in,
-                      const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
-                      cudaStream_t st) {
-    return tc::causal_forward(p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
-}
-int tc_causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const void* O,
-                       const float* den, const void* G, const StateArgs& sa, const void* saved, void* dQ, void* dK,
-                       void* dV, void* ws, cudaStream_t st) {
-    (void)O; (void)den;      // everything needed is recomputed consistently
-    return tc::causal_backward(p, Q, K, V, lengths, G, sa, saved, dQ, dK, dV, ws, st);
-}
-int tc_linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, void* O,
-                      float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st) {
-    return tc::linear_forward(p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
-}
-int tc_linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
-                       const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
-    return tc::linear_backward(p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
-}
-
 }  // namespace la

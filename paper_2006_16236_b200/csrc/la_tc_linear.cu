@@ -23,8 +23,9 @@
 // with ysum = sum_j V_j, gsum = sum_i G_i / dn_i, rho0 = sum_i dl_i / dn_i, qh' = q' / dn.
 // The column sums of S'' and R'' vanish, so (1 + x')^T S'' = x'^T S''.
 //
-// CTA = 10 warps: warps 0-3 epilogue (thread t owns chunk row t = TMEM lane t), warps 4-7
-// apply elu to the X tile in place, warp 8 TMA, warp 9 MMA issue.
+// Sum kernel: 10 warps (0-7 apply elu to the X tile in place, half a row per thread; 8 TMA; 9 MMA issue).
+// Apply kernel: 14 warps (0-7 epilogue, two per TMEM quadrant, half a chunk row each; 8-11 apply elu to the
+// X tile in place; 12 TMA; 13 MMA issue).
 #include "la_tc.cuh"
 #include "la_tc_common.cuh"
 
