@@ -230,6 +230,38 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
                  : "memory");
 }
 
+// The same two for a warp that runs its issue loop with all 32 lanes (addresses and descriptors then stay
+// in uniform registers instead of being moved there for every instruction, which a loop under
+// `if (lane == 0)` has to do): `leader` is true in exactly one lane (elect_one()), every operand is the same
+// in all lanes.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t is_leader;
+    asm volatile("{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\tselp.u32 %0, 1, 0, e;\n\t}" : "=r"(is_leader));
+    return is_leader != 0;
+}
+__device__ __forceinline__ void umma_bf16(bool leader, uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, e;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 e, %5, 0;\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"((uint32_t)leader)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(bool leader, uint64_t* bar) {
+    asm volatile(
+        "{\n\t.reg .pred e;\n\t"
+        "setp.ne.b32 e, %1, 0;\n\t"
+        "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)), "r"((uint32_t)leader)
+        : "memory");
+}
+// Bounded wait by a whole warp: the same answer in every lane, and known to the compiler as such.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, int* status, int code) {
+    return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, status, code));
+}
+
 // Named barrier among `count` threads (count a multiple of 32); id 0 is __syncthreads.
 __device__ __forceinline__ void named_barrier(int id, int count) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");

@@ -56,10 +56,10 @@ namespace {
 // Warps 0-7 ("score/epilogue" warps, two per TMEM quadrant: the pair shares the 128 rows
 // of the quadrant, one warp per 32-column half): mask + round dP of chunk c+1, then the dQ
 // epilogue of chunk c.  Warps 8-11: phi(K), phi(Q) in place and the state conversion.
-// Warp 12: TMA.  Warps 13, 14: MMA issue (13 also allocates TMEM).
+// Warp 12: TMA.  Warps 13, 14, 15: MMA issue (13 also allocates TMEM).
 // ===========================================================================
 constexpr int kDqStages = 2;
-constexpr int kDqThreads = 480;
+constexpr int kDqThreads = 512;
 constexpr uint32_t kDqColDP = 0;       // 128
 constexpr uint32_t kDqColGt = 128;     // 2 x 64: h of even / odd chunks
 constexpr uint32_t kDqColT = 256;      // 2 x 64: T = L k of even / odd chunks
@@ -214,12 +214,17 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         }
     } else if (warp >= 13) {
         // ------------------------------------------------------------- MMA issuers
-        // Two threads share the issue work (an issuing thread needs about 100 cycles per tcgen05.mma here,
-        // more than the tensor pipe does).  Warp 13: the score tile dP = G V^T and the product that consumes
-        // its rounded copy, h += dP k.  Warp 14: everything that involves the running state (h = G S^T,
-        // St += k^T [V | 1]) and T = L k.  MMAs of one thread execute in order; gst_full orders the two
-        // threads' writes to the h accumulator and tells warp 13 that warp 14 is done with a stage.
-        if (lane == 0) {
+        // Three warps share the issue work, each running its loop with all lanes and issuing through an
+        // elected one: addresses and descriptors then live in uniform registers (about 40 cycles per
+        // tcgen05.mma; a loop under `if (lane == 0)` moves them there for every instruction and needs 100).
+        // Warp 15: the score tile dP = G V^T of the next chunk, as soon as the score warps have taken the
+        // previous one out of TMEM.  Warp 13: the product that consumes the rounded copy, h += dP k.  Warp 14:
+        // everything that involves the running state (h = G S^T, St += k^T [V | 1]) and T = L k.  MMAs of one
+        // thread execute in order; gst_full orders the two threads' writes to the h accumulator and tells
+        // warp 13 that warp 14 is done with a stage; the score warps wait for dq_full(c) before they overwrite
+        // the shared-memory score tile that h += dP k of chunk c reads.
+        {
+            const bool leader = elect_one();
             const uint32_t idesc_dp = umma_idesc_bf16(128, 128, 0, 0);
             const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
             const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
@@ -232,44 +237,37 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             auto lo_mn = [&](uint32_t a, uint32_t lbo) { return (uint32_t)desc_mn(a, lbo); };
             auto stage_k = [&](int c) { return sbase + kDqOffStage + (uint32_t)(c % kDqStages) * 4 * kTileBytes; };
             bool ok = true;
-            if (warp == 13) {
-                auto issue_dp = [&](int c) {    // dP = G V^T needs only the raw tiles
+            if (warp == 15) {
+                #pragma unroll 1
+                for (int c = 0; c < L && ok; ++c) {     // dP = G V^T needs only the raw tiles
+                    ok = mbar_wait_warp(&bars->full[c % kDqStages], (c / kDqStages) & 1, prm.status, kStatusTmaTimeout);
+                    if (ok && c >= 1) ok = mbar_wait_warp(&bars->dp_ready, (c - 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
                     const uint32_t dV = lo_k(stage_k(c) + kTileBytes), dG = lo_k(stage_k(c) + 2 * kTileBytes);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kDqColDP, mk(dG + 2 * k), mk(dV + 2 * k), idesc_dp, k > 0);
-                    umma_commit(&bars->dp_full);
-                };
-                ok = mbar_wait(&bars->full[0], 0, prm.status, kStatusTmaTimeout) && !*abort_flag;
-                if (ok) {
-                    tc_fence_after_sync();
-                    issue_dp(0);
+                    for (int k = 0; k < 4; ++k) umma_bf16(leader, tmem + kDqColDP, mk(dG + 2 * k), mk(dV + 2 * k), idesc_dp, k > 0);
+                    umma_commit(leader, &bars->dp_full);
                 }
+            } else if (warp == 13) {
                 #pragma unroll 1
                 for (int c = 0; c < L && ok; ++c) {
                     const int b = c & 1;
-                    LA_TRACE(g_trace_dq, c, 0);
-                    ok = mbar_wait(&bars->dp_ready, c & 1, prm.status, kStatusPipeTimeout) &&
-                         mbar_wait(&bars->gst_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout);
-                    if (!ok || *abort_flag) { ok = false; break; }
+                    if (leader) LA_TRACE(g_trace_dq, c, 0);
+                    ok = mbar_wait_warp(&bars->dp_ready, c & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait_warp(&bars->gst_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout);
+                    if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
-                    LA_TRACE(g_trace_dq, c, 3);
+                    if (leader) LA_TRACE(g_trace_dq, c, 3);
                     const uint32_t dDP = lo_k(aDP), dKmn = lo_mn(stage_k(c), kTileBytes);
 #pragma unroll
                     for (int k = 0; k < 8; ++k)      // h += dP k
-                        umma_bf16(tmem + kDqColGt + b * 64, mk(dDP + (k >> 2) * (kTileBytes >> 4) + (k & 3) * 2), mk(dKmn + 128 * k),
+                        umma_bf16(leader, tmem + kDqColGt + b * 64, mk(dDP + (k >> 2) * (kTileBytes >> 4) + (k & 3) * 2), mk(dKmn + 128 * k),
                                   idesc_kmn, 1);
-                    umma_commit(&bars->dq_full[b]);
-                    // gst_full(c) was awaited: it covers the other thread's products on this stage
-                    umma_commit(&bars->empty[c % kDqStages]);
-                    LA_TRACE(g_trace_dq, c, 4);
-                    // the score tile in TMEM is free (dp_ready(c)); the shared-memory copy is rewritten only after
-                    // dp_full(c+1), which this commit orders behind h += dP k
-                    if (c + 1 < L) {
-                        ok = mbar_wait(&bars->full[(c + 1) % kDqStages], ((c + 1) / kDqStages) & 1, prm.status, kStatusTmaTimeout);
-                        if (!ok) break;
-                        tc_fence_after_sync();
-                        issue_dp(c + 1);
-                    }
+                    umma_commit(leader, &bars->dq_full[b]);
+                    // gst_full(c) and dp_ready(c) were awaited: they cover the other threads' products on this stage
+                    umma_commit(leader, &bars->empty[c % kDqStages]);
+                    if (leader) LA_TRACE(g_trace_dq, c, 4);
                 }
             } else {
                 #pragma unroll 1
@@ -278,25 +276,25 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                     const uint32_t aK = stage_k(c), aV = aK + kTileBytes, aG = aV + kTileBytes;
                     const uint32_t dKmn = lo_mn(aK, kTileBytes), dV1 = lo_mn(aV, aOnes - aV), dG = lo_k(aG), dS = lo_k(aS), dL = lo_k(aL);
                     constexpr uint32_t kStepV1 = 128u - (128u << 16);
-                    ok = mbar_wait(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout) &&
-                         mbar_wait(&bars->state_ready, c & 1, prm.status, kStatusPipeTimeout);
-                    if (ok && c >= 2) ok = mbar_wait(&bars->dq_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
-                    if (!ok || *abort_flag) { ok = false; break; }
+                    ok = mbar_wait_warp(&bars->mapped[s], (c / kDqStages) & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait_warp(&bars->state_ready, c & 1, prm.status, kStatusPipeTimeout);
+                    if (ok && c >= 2) ok = mbar_wait_warp(&bars->dq_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
-                    LA_TRACE(g_trace_dq, c, 1);
+                    if (leader) LA_TRACE(g_trace_dq, c, 1);
 #pragma unroll
                     for (int k = 0; k < 4; ++k)      // h = G S_{c-1}^T (before the state tile is rewritten)
-                        umma_bf16(tmem + kDqColGt + b * 64, mk(dG + 2 * k), mk(dS + 2 * k), idesc_kk, k > 0);
+                        umma_bf16(leader, tmem + kDqColGt + b * 64, mk(dG + 2 * k), mk(dS + 2 * k), idesc_kk, k > 0);
 #pragma unroll
                     for (int k = 0; k < 8; ++k)      // [S | Z] += k^T [V | 1]: the ones region is the second 64-column block
-                        umma_bf16(tmem + kDqColS, mk(dKmn + 128 * k), mk(dV1 + kStepV1 * k), idesc_s, 1);
-                    umma_commit(&bars->s_full);
+                        umma_bf16(leader, tmem + kDqColS, mk(dKmn + 128 * k), mk(dV1 + kStepV1 * k), idesc_s, 1);
+                    umma_commit(leader, &bars->s_full);
 #pragma unroll
                     for (int k = 0; k < 8; ++k)      // T = L k  (row-wise prefix sums of k inside the chunk)
-                        umma_bf16(tmem + kDqColT + b * 64, mk(dL + (k >> 2) * (kTileBytes >> 4) + (k & 3) * 2), mk(dKmn + 128 * k),
+                        umma_bf16(leader, tmem + kDqColT + b * 64, mk(dL + (k >> 2) * (kTileBytes >> 4) + (k & 3) * 2), mk(dKmn + 128 * k),
                                   idesc_kmn, k > 0);
-                    umma_commit(&bars->gst_full[b]);
-                    LA_TRACE(g_trace_dq, c, 2);
+                    umma_commit(leader, &bars->gst_full[b]);
+                    if (leader) LA_TRACE(g_trace_dq, c, 2);
                 }
             }
             if (!ok) *abort_flag = 1;
@@ -367,12 +365,17 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         const bool elu = prm.phi == LA_PHI_ELU1;
         float m_prev = 0.f;                                 // centring offset of the chunk whose epilogue is pending
 
+        bool scores_ok = true;
         auto process_scores = [&](int c) -> float {         // chunk c: TMEM dP -> masked bf16 tile
             float m = 0.f;
             if (c_begin + c == 0) {                          // first chunk of the sequence: centre on dP_i0
                 m = __uint_as_float(tmem_ld1(src));
                 tmem_ld_wait();
             }
+            // the shared-memory tile is still the A operand of h += dP k of the chunk before, which another
+            // thread issues: it must have completed before the tile is overwritten
+            if (c >= 1 && !mbar_wait(&bars->dq_full[(c - 1) & 1], ((c - 1) >> 1) & 1, prm.status, kStatusMmaTimeout))
+                scores_ok = false;
             if (has0) {
                 uint32_t v[32];
                 tmem_ld32(src + blk0 * 32, v);
@@ -419,6 +422,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 tc_fence_after_sync();
                 if (warp == 3 && lane == 0) LA_TRACE(g_trace_dq, c + 1, 11);
                 m_next = process_scores(c + 1);
+                if (!scores_ok) { ok = false; break; }
                 if (warp == 3 && lane == 0) LA_TRACE(g_trace_dq, c + 1, 12);
             }
             // ---- epilogue of chunk c: this thread owns columns [32 half, 32 half + 32) of row t
