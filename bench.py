@@ -519,8 +519,9 @@ def bench_decode_layer(la, w, dev, pk, T=512):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) * 1e3 / T
 
+    n0 = la.la_kernel_launches()
     run_raw()
-    res = {"workload": f"decode_layer_B{B}_H{H}_D{D}", "tokens": T, "launches_per_token": 3,
+    res = {"workload": f"decode_layer_B{B}_H{H}_D{D}", "tokens": T, "launches_per_token": (la.la_kernel_launches() - n0) // T,
            "us_per_token_host_issued": timed(run_binding), "us_per_token_host_issued_raw_c_abi": timed(run_raw)}
     try:
         side = torch.cuda.Stream()

@@ -691,7 +691,8 @@ def test_decode_workload_full_size():
     assert err < 0.05, err
 
 
-@pytest.mark.parametrize("B,H", [(256, 8), (3, 2), (130, 4)])
+@pytest.mark.parametrize("B,H", [(256, 8), (3, 2), (130, 4), (37, 5), (20, 12)],
+                         ids=["B256_H8", "B3_H2", "B130_H4", "B37_H5_odd_heads", "B20_H12"])
 def test_decode_layer_steps_against_the_oracle(B, H):
     """A whole attention sublayer per token (projections, state update and read-out, output projection,
     residual), 12 tokens fed one at a time; the next token's input is made from the previous output, so the
