@@ -307,6 +307,19 @@ int la_decode_layer_step(const la_problem* p, const void* x, const void* Wqkv, c
 int la_linear_attention_noalloc(const la_problem* p, const void* Q, const void* K, const void* V,
                                 void* O, float* den, float* KV, float* Zs, void* stream);
 
+/*
+ * Checked mode (no counterpart in the paper): with the environment variable LA_DEBUG=1 set when the
+ * library is first used, the attention, recurrent-step and decode-layer entry points look every
+ * tensor argument up with the driver before anything is enqueued (device memory of the current
+ * device? does the allocation that holds it reach as far as the call reads or writes, given the
+ * sizes in la_problem?) and return LA_ERR_INVALID_ARG otherwise; after enqueueing they synchronise
+ * `stream` and report a bounded wait that ran out (LA_ERR_DEVICE_TIMEOUT), a refused saved buffer or
+ * a CUDA error from the call itself instead of leaving it to la_last_device_status().  Under a
+ * caching allocator the allocation is the allocator's block, so the span check is a lower bound on
+ * strictness.  Meant for bring-up on shared GPUs, where an out-of-bounds access must not reach the
+ * device; it costs a synchronisation per call and must not be used during stream capture.
+ */
+
 /* Bytes of workspace `op` needs for problem p (pure host function; 0 if none).
  * Returns 0 for invalid problems as well: the entry point reports the error. */
 size_t la_workspace_bytes(const la_problem* p, int32_t op);

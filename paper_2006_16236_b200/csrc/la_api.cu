@@ -1,6 +1,7 @@
 // C ABI of the linear-attention library: argument validation, dispatch between
 // the tensor-core and the general kernels, status reporting.  Nothing here
 // allocates device memory or synchronises (except la_last_device_status).
+#include <cuda.h>
 #include <atomic>
 #include <stdarg.h>
 #include <stdio.h>
@@ -84,6 +85,80 @@ int check_problem(const la_problem* p, bool need_n) {
         return fail(LA_ERR_UNSUPPORTED, "sequence too long");
     return LA_OK;
 }
+
+// ---------------------------------------------------------------------------------------------------------
+// Checked mode (environment variable LA_DEBUG=1, read once): before anything is enqueued every tensor argument
+// is looked up with the driver (device memory of the current device? does the allocation that holds it reach
+// as far as the call will read or write?), and after the call the stream is synchronised and the device
+// status word and the CUDA error state are read, so that a failure is reported by the call that caused it.
+// It turns an out-of-bounds access on a shared GPU into an error code on the host.  Off by default: the
+// look-ups and the synchronisation cost tens of microseconds per call.
+static bool debug_mode() {
+    static const bool on = [] {
+        const char* v = getenv("LA_DEBUG");
+        return v && atoi(v) != 0;
+    }();
+    return on;
+}
+
+static int debug_span(const void* ptr, size_t bytes, const char* name) {
+    if (!debug_mode() || !ptr || !bytes) return LA_OK;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, ptr) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(LA_ERR_INVALID_ARG, "checked mode: %s (%p) is not a pointer CUDA knows", name, ptr);
+    }
+    if (at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged)
+        return fail(LA_ERR_INVALID_ARG, "checked mode: %s (%p) is not device memory", name, ptr);
+    int dev = 0;
+    LA_CUDA_TRY(cudaGetDevice(&dev));
+    if (at.type == cudaMemoryTypeDevice && at.device != dev)
+        return fail(LA_ERR_INVALID_ARG, "checked mode: %s lives on device %d, the current device is %d", name, at.device, dev);
+    typedef CUresult (*range_fn)(CUdeviceptr*, size_t*, CUdeviceptr);
+    static range_fn range = [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuMemGetAddressRange", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            fn = nullptr;
+        return reinterpret_cast<range_fn>(fn);
+    }();
+    if (!range) return LA_OK;
+    CUdeviceptr base = 0;
+    size_t size = 0;
+    if (range(&base, &size, (CUdeviceptr)(uintptr_t)ptr) != CUDA_SUCCESS) return LA_OK;      // not a plain allocation: no range to check
+    const uintptr_t end = (uintptr_t)ptr + bytes, alloc_end = (uintptr_t)base + size;
+    if (end > alloc_end)
+        return fail(LA_ERR_INVALID_ARG, "checked mode: %s needs %zu bytes at %p, its allocation ends %zu bytes earlier", name,
+                    bytes, ptr, (size_t)(end - alloc_end));
+    return LA_OK;
+}
+#define LA_DEBUG_SPAN(ptr, bytes)                                   \
+    do {                                                            \
+        if (int rc_ = debug_span(ptr, bytes, #ptr)) return rc_;     \
+    } while (0)
+
+extern "C" int la_last_device_status(void* stream);
+// the tail of every compute entry point: in checked mode the call's own failures surface here
+static int debug_finish(int rc, void* stream) {
+    if (rc != LA_OK || !debug_mode()) return rc;
+    if (int st = la_last_device_status(stream)) return st;
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(LA_ERR_CUDA, "checked mode: %s after the call", cudaGetErrorString(e));
+    return LA_OK;
+}
+
+struct TensorBytes {        // sizes of the tensors of a problem, for the span checks
+    size_t qk, vo, den, s, z;
+    explicit TensorBytes(const la_problem& p) {
+        const size_t e = p.dtype == LA_BF16 ? 2 : 4, bh = (size_t)(p.B * p.H);
+        qk = bh * (size_t)p.N * (size_t)p.D * e;
+        vo = bh * (size_t)p.N * (size_t)p.M * e;
+        den = bh * (size_t)p.N * sizeof(float);
+        s = bh * (size_t)(p.D * p.M) * sizeof(float);
+        z = bh * (size_t)p.D * sizeof(float);
+    }
+};
 
 #define LA_REQUIRE_PTR(ptr)                                                                \
     do {                                                                                   \
@@ -266,9 +341,14 @@ static int linear_forward_common(const la_problem* p, const void* Q, const void*
     if (!saved)         // with a saved buffer the sums go there and the workspace is not touched
         if (int rc = check_ws(p, lengths ? LA_OP_LINEAR_VARLEN_FORWARD : LA_OP_LINEAR_FORWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
+    const TensorBytes tb(*p);
+    LA_DEBUG_SPAN(Q, tb.qk); LA_DEBUG_SPAN(K, tb.qk); LA_DEBUG_SPAN(V, tb.vo); LA_DEBUG_SPAN(O, tb.vo);
+    LA_DEBUG_SPAN(den, tb.den); LA_DEBUG_SPAN(KV, tb.s); LA_DEBUG_SPAN(Zs, tb.z);
+    LA_DEBUG_SPAN(lengths, (size_t)p->B * 4); LA_DEBUG_SPAN(ws, ws_bytes); LA_DEBUG_SPAN(saved, saved_bytes);
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_FORWARD)) return tc::linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
-    return general_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st);
+    if (tc_supported(*p, LA_OP_LINEAR_FORWARD))
+        return debug_finish(tc::linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st), stream);
+    return debug_finish(general_linear_forward(*p, Q, K, V, lengths, O, den, KV, Zs, saved, ws, st), stream);
 }
 
 static int linear_backward_common(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
@@ -284,9 +364,14 @@ static int linear_backward_common(const la_problem* p, const void* Q, const void
     if (int rc = check_linear_saved(p, saved, saved_bytes)) return rc;
     if (int rc = check_ws(p, lengths ? LA_OP_LINEAR_VARLEN_BACKWARD : LA_OP_LINEAR_BACKWARD, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
+    const TensorBytes tb(*p);
+    LA_DEBUG_SPAN(Q, tb.qk); LA_DEBUG_SPAN(K, tb.qk); LA_DEBUG_SPAN(V, tb.vo); LA_DEBUG_SPAN(G, tb.vo);
+    LA_DEBUG_SPAN(dQ, tb.qk); LA_DEBUG_SPAN(dK, tb.qk); LA_DEBUG_SPAN(dV, tb.vo);
+    LA_DEBUG_SPAN(lengths, (size_t)p->B * 4); LA_DEBUG_SPAN(ws, ws_bytes); LA_DEBUG_SPAN(saved, saved_bytes);
     cudaStream_t st = (cudaStream_t)stream;
-    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD)) return tc::linear_backward(*p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
-    return general_linear_backward(*p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st);
+    if (tc_supported(*p, LA_OP_LINEAR_BACKWARD))
+        return debug_finish(tc::linear_backward(*p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st), stream);
+    return debug_finish(general_linear_backward(*p, Q, K, V, lengths, saved, G, dQ, dK, dV, ws, st), stream);
 }
 
 int la_linear_attention(const la_problem* p, const void* Q, const void* K, const void* V,
@@ -368,9 +453,14 @@ static int causal_forward_common(const la_problem* p, const void* Q, const void*
     if (int rc = check_ws(p, lengths ? LA_OP_CAUSAL_VARLEN_FORWARD : LA_OP_CAUSAL_FORWARD, ws, ws_bytes)) return rc;
     if (int rc = check_saved(p, saved, saved_bytes)) return rc;
     if (int rc = check_arch()) return rc;
+    const TensorBytes tb(*p);
+    LA_DEBUG_SPAN(Q, tb.qk); LA_DEBUG_SPAN(K, tb.qk); LA_DEBUG_SPAN(V, tb.vo); LA_DEBUG_SPAN(O, tb.vo);
+    LA_DEBUG_SPAN(den, tb.den); LA_DEBUG_SPAN(S_in, tb.s); LA_DEBUG_SPAN(Z_in, tb.z); LA_DEBUG_SPAN(S_out, tb.s);
+    LA_DEBUG_SPAN(Z_out, tb.z); LA_DEBUG_SPAN(lengths, (size_t)p->B * 4); LA_DEBUG_SPAN(ws, ws_bytes);
+    LA_DEBUG_SPAN(saved, saved_bytes);
     if (tc_supported(*p, LA_OP_CAUSAL_FORWARD))
-        return tc::causal_forward(*p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st);
-    return general_causal_forward(*p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, st);
+        return debug_finish(tc::causal_forward(*p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, saved, ws, st), stream);
+    return debug_finish(general_causal_forward(*p, Q, K, V, lengths, S_in, Z_in, O, den, S_out, Z_out, st), stream);
 }
 
 extern "C" {
@@ -436,9 +526,15 @@ static int causal_backward_common(const la_problem* p, const void* Q, const void
     if (int rc = check_arch()) return rc;
     StateArgs sa;
     sa.S_in = S_in; sa.Z_in = Z_in; sa.dS_out = dS_out; sa.dZ_out = dZ_out; sa.dS_in = dS_in; sa.dZ_in = dZ_in;
+    const TensorBytes tb(*p);
+    LA_DEBUG_SPAN(Q, tb.qk); LA_DEBUG_SPAN(K, tb.qk); LA_DEBUG_SPAN(V, tb.vo); LA_DEBUG_SPAN(G, tb.vo);
+    LA_DEBUG_SPAN(dQ, tb.qk); LA_DEBUG_SPAN(dK, tb.qk); LA_DEBUG_SPAN(dV, tb.vo);
+    LA_DEBUG_SPAN(S_in, tb.s); LA_DEBUG_SPAN(Z_in, tb.z); LA_DEBUG_SPAN(dS_out, tb.s); LA_DEBUG_SPAN(dZ_out, tb.z);
+    LA_DEBUG_SPAN(dS_in, tb.s); LA_DEBUG_SPAN(dZ_in, tb.z); LA_DEBUG_SPAN(lengths, (size_t)p->B * 4);
+    LA_DEBUG_SPAN(ws, ws_bytes); LA_DEBUG_SPAN(saved, saved_bytes);
     if (tc_supported(*p, LA_OP_CAUSAL_BACKWARD))
-        return tc::causal_backward(*p, Q, K, V, lengths, G, sa, saved, dQ, dK, dV, ws, st);
-    return general_causal_backward(*p, Q, K, V, lengths, G, sa, dQ, dK, dV, ws, st);
+        return debug_finish(tc::causal_backward(*p, Q, K, V, lengths, G, sa, saved, dQ, dK, dV, ws, st), stream);
+    return debug_finish(general_causal_backward(*p, Q, K, V, lengths, G, sa, dQ, dK, dV, ws, st), stream);
 }
 
 extern "C" {
@@ -479,7 +575,14 @@ int la_recurrent_step(const la_problem* p, const void* q, const void* k, const v
     LA_REQUIRE_PTR(q); LA_REQUIRE_PTR(k); LA_REQUIRE_PTR(v);
     LA_REQUIRE_PTR(S); LA_REQUIRE_PTR(Z); LA_REQUIRE_PTR(out);
     if (int rc = check_arch()) return rc;
-    return launch_recurrent_step(*p, q, k, v, S, Z, out, (cudaStream_t)stream);
+    {
+        la_problem one = *p;
+        one.N = 1;
+        const TensorBytes tb(one);
+        LA_DEBUG_SPAN(q, tb.qk); LA_DEBUG_SPAN(k, tb.qk); LA_DEBUG_SPAN(v, tb.vo); LA_DEBUG_SPAN(out, tb.vo);
+        LA_DEBUG_SPAN(S, tb.s); LA_DEBUG_SPAN(Z, tb.z);
+    }
+    return debug_finish(launch_recurrent_step(*p, q, k, v, S, Z, out, (cudaStream_t)stream), stream);
 }
 
 int la_decode_layer_step(const la_problem* p, const void* x, const void* Wqkv, const void* Wo,
@@ -495,7 +598,13 @@ int la_decode_layer_step(const la_problem* p, const void* x, const void* Wqkv, c
     if (y == x) return fail(LA_ERR_INVALID_ARG, "y must not alias x (x is read again for the residual while y is written)");
     if (int rc = check_ws(p, LA_OP_DECODE_LAYER, ws, ws_bytes)) return rc;
     if (int rc = check_arch()) return rc;
-    return decode_layer_step(*p, x, Wqkv, Wo, S, Z, y, ws, (cudaStream_t)stream);
+    {
+        const size_t F = (size_t)(p->H * p->D), xb = (size_t)p->B * F * 2;
+        const TensorBytes tb(*p);
+        LA_DEBUG_SPAN(x, xb); LA_DEBUG_SPAN(y, xb); LA_DEBUG_SPAN(Wqkv, 3 * F * F * 2); LA_DEBUG_SPAN(Wo, F * F * 2);
+        LA_DEBUG_SPAN(S, tb.s); LA_DEBUG_SPAN(Z, tb.z); LA_DEBUG_SPAN(ws, ws_bytes);
+    }
+    return debug_finish(decode_layer_step(*p, x, Wqkv, Wo, S, Z, y, ws, (cudaStream_t)stream), stream);
 }
 
 int la_recurrent_steps(const la_problem* p, const void* q, const void* k, const void* v,
@@ -505,7 +614,12 @@ int la_recurrent_steps(const la_problem* p, const void* q, const void* k, const 
     LA_REQUIRE_PTR(q); LA_REQUIRE_PTR(k); LA_REQUIRE_PTR(v);
     LA_REQUIRE_PTR(S); LA_REQUIRE_PTR(Z); LA_REQUIRE_PTR(out);
     if (int rc = check_arch()) return rc;
-    return launch_recurrent_steps(*p, q, k, v, S, Z, out, (cudaStream_t)stream);
+    {
+        const TensorBytes tb(*p);
+        LA_DEBUG_SPAN(q, tb.qk); LA_DEBUG_SPAN(k, tb.qk); LA_DEBUG_SPAN(v, tb.vo); LA_DEBUG_SPAN(out, tb.vo);
+        LA_DEBUG_SPAN(S, tb.s); LA_DEBUG_SPAN(Z, tb.z);
+    }
+    return debug_finish(launch_recurrent_steps(*p, q, k, v, S, Z, out, (cudaStream_t)stream), stream);
 }
 
 int la_last_device_status(void* stream) {
