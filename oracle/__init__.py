@@ -236,6 +236,30 @@ def poly2_attention(Q, K, V, causal: bool, eps: float = 0.0):
 
 
 # ---------------------------------------------------------------------------
+# Random Fourier features for the Gaussian (RBF) kernel, which the paper's conclusion names as a feature map
+# to explore and does not write down.  Reading: the classical construction with the frequencies given by the
+# caller, W [C/2, D], in its paired form
+#     phi(x) = sqrt(2 / C) [cos(W x), sin(W x)]   in R^C,
+# for which phi(x) . phi(y) = (2 / C) sum_c cos(w_c . (x - y)) exactly (a function of x - y alone, |phi(x)| = 1),
+# and whose expectation over w_c ~ N(0, I) is exp(-|x - y|^2 / 2).  Plain numpy, written from the definition.
+# ---------------------------------------------------------------------------
+def rff_feature_map(x, W):
+    """x [..., D], W [C/2, D] -> [..., C]: sqrt(2/C) cos(x W^T) in the first C/2 columns, sqrt(2/C) sin(x W^T) in the rest."""
+    x, W = _f64(x), _f64(W)
+    z = x @ W.T
+    return np.concatenate([np.cos(z), np.sin(z)], axis=-1) * np.sqrt(1.0 / W.shape[0])
+
+
+def rff_feature_map_backward(x, W, dy):
+    """Gradient of rff_feature_map with respect to x: dx = sqrt(2/C) (-sin(z) * dy_cos + cos(z) * dy_sin) W, z = x W^T."""
+    x, W, dy = _f64(x), _f64(W), _f64(dy)
+    h = W.shape[0]
+    z = x @ W.T
+    t = (-np.sin(z) * dy[..., :h] + np.cos(z) * dy[..., h:]) * np.sqrt(1.0 / h)
+    return t @ W
+
+
+# ---------------------------------------------------------------------------
 # One decode step of a whole attention sublayer, Eq. 16-20 with the projections written out:
 #   q = x W_Q, k = x W_K, v = x W_V (split into H heads), s_i = s_{i-1} + phi(k) v^T, z_i = z_{i-1} + phi(k),
 #   a = phi(q)^T s_i / (phi(q)^T z_i + eps) per head,  y = a W_O + x.

@@ -481,3 +481,57 @@ def test_decode_layer_special_cases():
     e = np.exp(-1.0)
     y2 = oracle.decode_layer_step(np.array([[-2.0]]), h, h, h, h, S, Z)[0, 0]
     np.testing.assert_allclose(y2, 0.5 * (2 - e) / (2 + e) - 2, rtol=1e-14)
+
+
+# ---------------------------------------------------------------------------
+# Random Fourier features (the conclusion's "approximating the RBF kernel with random Fourier features")
+# ---------------------------------------------------------------------------
+def test_rff_hand_example_norm_and_shift_invariance():
+    # D = 1, one frequency pi/2, x = 1: z = pi/2, phi = sqrt(2/2) [cos z, sin z] = [0, 1]
+    y = oracle.rff_feature_map([1.0], [[np.pi / 2]])
+    assert abs(y[0]) < 1e-15 and y[1] == 1.0
+    # two frequencies 0 and pi at x = 1: sqrt(1/2) [cos 0, cos pi, sin 0, sin pi] = [s, -s, 0, 0]
+    y = oracle.rff_feature_map([1.0], [[0.0], [np.pi]])
+    s = 0.5 ** 0.5
+    assert np.allclose(y, [s, -s, 0.0, 0.0], atol=1e-15)
+    rng = np.random.default_rng(5)
+    W = rng.standard_normal((24, 6))
+    x, yv, shift = rng.standard_normal((3, 7, 6))
+    fx, fy = oracle.rff_feature_map(x, W), oracle.rff_feature_map(yv, W)
+    # |phi(x)| = 1 whatever x and W are (cos^2 + sin^2 per frequency)
+    assert np.allclose((fx ** 2).sum(-1), 1.0, atol=1e-14)
+    # phi(x) . phi(y) = (2/C) sum_c cos(w_c . (x - y)): a function of the difference alone
+    direct = np.cos((x - yv) @ W.T).mean(-1)
+    assert np.allclose((fx * fy).sum(-1), direct, atol=1e-14)
+    moved = (oracle.rff_feature_map(x + shift, W) * oracle.rff_feature_map(yv + shift, W)).sum(-1)
+    assert np.allclose(moved, direct, atol=1e-13)
+
+
+def test_rff_approximates_the_gaussian_kernel_within_its_sampling_error():
+    """With w_c ~ N(0, I) the mean of cos(w . d) is exp(-|d|^2 / 2) and its variance is below 1/2 per frequency:
+    20000 frequencies give a standard error below 0.005; five of them is the bound held here."""
+    rng = np.random.default_rng(6)
+    D, half = 4, 20000
+    W = rng.standard_normal((half, D))
+    x, y = rng.standard_normal((2, 16, D)) * 0.7
+    approx = (oracle.rff_feature_map(x, W) * oracle.rff_feature_map(y, W)).sum(-1)
+    exact = np.exp(-((x - y) ** 2).sum(-1) / 2)
+    assert np.abs(approx - exact).max() < 5 * (0.5 / half) ** 0.5
+
+
+def test_rff_backward_matches_finite_differences():
+    rng = np.random.default_rng(7)
+    W = rng.standard_normal((5, 3))
+    x = rng.standard_normal((4, 3))
+    dy = rng.standard_normal((4, 10))
+    dx = oracle.rff_feature_map_backward(x, W, dy)
+    h = 1e-6
+    for i in range(4):
+        for j in range(3):
+            xp, xm = x.copy(), x.copy()
+            xp[i, j] += h
+            xm[i, j] -= h
+            fd = ((oracle.rff_feature_map(xp, W) - oracle.rff_feature_map(xm, W)) * dy).sum() / (2 * h)
+            assert abs(fd - dx[i, j]) < 1e-7 * max(1.0, abs(fd))
+    # a frequency of zero contributes a constant feature: no gradient through it
+    assert np.allclose(oracle.rff_feature_map_backward(x, np.zeros((5, 3)), dy), 0.0)
