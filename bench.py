@@ -581,6 +581,36 @@ def bench_poly2(la, w, dev, pk, iters=10):
     return out
 
 
+def bench_rff(la, w, dev, pk, iters=10):
+    """Random Fourier features (the map the paper's conclusion proposes) and their gradient on the headline
+    workload's rows with D = 64 inputs and C = 64 features (what the tensor-core attention kernels take): two
+    tensors alternate, so that a launch's 270 MB are not in L2 from the launch before."""
+    rows, D, C = w.B * w.H * w.N, 64, 64
+    g = torch.Generator(device="cpu").manual_seed(w.seed + 19)
+    W = torch.randn((C // 2, D), generator=g).to(torch.bfloat16).to(dev)
+    xs = [(torch.randn((rows, D), generator=g) * 0.5).to(torch.bfloat16).to(dev) for _ in range(2)]
+    ys = [torch.empty((rows, C), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    dxs = [torch.empty_like(x) for x in xs]
+    out = {"rows": rows, "D": D, "C": C, "dtype": "bf16"}
+    for name, fn, nbytes in (
+            ("forward", lambda i: la.la_feature_map_rff(xs[i], W, out=ys[i]), rows * (D + C) * 2),
+            ("backward", lambda i: la.la_feature_map_rff_backward(xs[i], W, ys[i], out=dxs[i]), rows * (2 * D + C) * 2)):
+        for i in range(4):
+            fn(i & 1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(dev)
+        e0.record()
+        for i in range(iters):
+            fn(i & 1)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1) / iters
+        out[name] = {"ms": round(ms, 4), "alg_gbs": round(nbytes / ms / 1e6, 1),
+                     "hbm_frac": round(nbytes / ms / 1e6 / pk["hbm_gbs"], 3)}
+    la.la_last_device_status()
+    return out
+
+
 def oracle_sample(w, pairs):
     """Inputs of the first `pairs` (batch, head) pairs of workload w, as [1, pairs, N, .]."""
     Q, K, V, G = draw_qkvg(1, pairs, w.N, w.D, w.M, w.seed, w.torch_dtype, w.scale)
@@ -719,6 +749,7 @@ def main():
                                                               "gpu_launches", "kernels_ms")}
         rows[w.name + "_from_state"]["unit"] = "tokens/s"
         rows["feature_map_poly2"] = bench_poly2(la, w, dev, pk)
+        rows["feature_map_rff"] = bench_rff(la, w, dev, pk)
 
     cpu = None
     if rank == 0 and world == 1 and not args.main_only:

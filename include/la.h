@@ -106,6 +106,27 @@ int la_feature_map_poly2_backward(const void* x, const void* dy, void* dx, int64
                                   int32_t dtype, void* stream);
 
 /*
+ * Random Fourier features for the Gaussian kernel (the feature map the paper's conclusion proposes to
+ * explore; Section 3.2.1: a feature map of dimension C costs O(N C M)).  The paper gives no formula; the
+ * classical paired construction is taken, with the frequencies supplied by the caller:
+ *   y[r] = sqrt(2 / C) [cos(W x[r]), sin(W x[r])],   W: [C/2, D] row-major,
+ * cosines in columns [0, C/2), sines in [C/2, C), so that y[r] . y[s] = (2 / C) sum_c cos(w_c . (x[r] - x[s])),
+ * whose mean over w_c ~ N(0, I) is exp(-|x[r] - x[s]|^2 / 2), and |y[r]| = 1.  Apply it to Q and K and call
+ * the attention entry points with phi = LA_PHI_IDENTITY and D = C.  The features have either sign: the
+ * weights of Eq. 4 are then not guaranteed positive, which is the caller's concern.
+ * x: [rows, D], y: [rows, C], W: [C/2, D], all bf16 (dtype LA_BF16), device, 16-byte aligned, no overlap.
+ * D a multiple of 8 in [8, 64]; C = 64 or 128; 1 <= rows < 2^31.  Other shapes or LA_F32: LA_ERR_UNSUPPORTED.
+ * The projection runs on the tensor cores (fp32 accumulation), sine and cosine on the special-function unit
+ * after a range reduction; one rounding to bf16 on output.
+ * The backward call turns dy = dL/dy [rows, C] into
+ *   dx[r] = sqrt(2 / C) (-sin(W x[r]) * dy_cos[r] + cos(W x[r]) * dy_sin[r]) W        (dx: [rows, D]),
+ * the inner factor being rounded to bf16 before the second product.  W is treated as a constant.
+ */
+int la_feature_map_rff(const void* x, const void* W, void* y, int64_t rows, int64_t D, int64_t C, int32_t dtype, void* stream);
+int la_feature_map_rff_backward(const void* x, const void* W, const void* dy, void* dx, int64_t rows, int64_t D, int64_t C,
+                                int32_t dtype, void* stream);
+
+/*
  * Non-causal linear attention, Eq. 5-6:
  *   KV = sum_j phi(K_j) V_j^T,  Zs = sum_j phi(K_j)   (formed once per head),
  *   O_i = phi(Q_i)^T KV / (phi(Q_i)^T Zs + eps).

@@ -25,7 +25,8 @@ LA_OP_CAUSAL_VARLEN_FORWARD, LA_OP_CAUSAL_VARLEN_BACKWARD = 9, 10
 _PHI = {"elu1": LA_PHI_ELU1, "identity": LA_PHI_IDENTITY}
 
 EXPORTS = [
-    "la_feature_map", "la_feature_map_poly2", "la_feature_map_poly2_backward",
+    "la_feature_map", "la_feature_map_poly2", "la_feature_map_poly2_backward", "la_feature_map_rff",
+    "la_feature_map_rff_backward",
     "la_linear_attention", "la_linear_attention_noalloc", "la_linear_attention_backward",
     "la_linear_attention_varlen", "la_linear_attention_varlen_backward",
     "la_linear_attention_keep", "la_linear_attention_backward_kept",
@@ -65,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.la_feature_map.argtypes = [vp, vp, i64, i32, i32, vp]
         L.la_feature_map_poly2.argtypes = [vp, vp, i64, i64, i64, i32, vp]
         L.la_feature_map_poly2_backward.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp]
+        L.la_feature_map_rff.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp]
+        L.la_feature_map_rff_backward.argtypes = [vp, vp, vp, vp, i64, i64, i64, i32, vp]
         L.la_linear_attention.argtypes = [pp] + [vp] * 7 + [vp, sz, vp]
         L.la_linear_attention_noalloc.argtypes = [pp] + [vp] * 7 + [vp]
         L.la_linear_attention_backward.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
@@ -306,6 +309,38 @@ def la_feature_map_poly2_backward(x: torch.Tensor, dy: torch.Tensor, out: torch.
     dx = torch.empty_like(x) if out is None else out
     _call(dev, lib().la_feature_map_poly2_backward, _ptr(x), _ptr(dy), _ptr(dx), x.numel() // max(D, 1), D, C,
                                                _dtype_code(x), _stream(dev))
+    return dx
+
+
+def la_feature_map_rff(x: torch.Tensor, W: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Random Fourier features along the last axis: x [..., D], frequencies W [C/2, D] -> [..., C] =
+    sqrt(2/C) [cos(x W^T), sin(x W^T)] (bf16); feed the result to the attention calls with phi="identity"."""
+    D = x.shape[-1]
+    if W.dim() != 2 or W.shape[1] != D or W.dtype != x.dtype:
+        raise ValueError(f"W must have shape [C/2, {D}] and dtype {x.dtype} (got {list(W.shape)}, {W.dtype})")
+    C = 2 * W.shape[0]
+    if out is not None and (tuple(out.shape) != tuple(x.shape[:-1]) + (C,) or out.dtype != x.dtype):
+        raise ValueError(f"out must have shape {list(x.shape[:-1]) + [C]} and dtype {x.dtype}")
+    dev = _dev(x, W, out)
+    y = torch.empty(x.shape[:-1] + (C,), dtype=x.dtype, device=x.device) if out is None else out
+    _call(dev, lib().la_feature_map_rff, _ptr(x), _ptr(W), _ptr(y), x.numel() // max(D, 1), D, C, _dtype_code(x), _stream(dev))
+    return y
+
+
+def la_feature_map_rff_backward(x: torch.Tensor, W: torch.Tensor, dy: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Gradient of la_feature_map_rff with respect to x for an upstream gradient dy [..., C] (W is a constant)."""
+    D = x.shape[-1]
+    if W.dim() != 2 or W.shape[1] != D or W.dtype != x.dtype:
+        raise ValueError(f"W must have shape [C/2, {D}] and dtype {x.dtype} (got {list(W.shape)}, {W.dtype})")
+    C = 2 * W.shape[0]
+    if tuple(dy.shape) != tuple(x.shape[:-1]) + (C,) or dy.dtype != x.dtype:
+        raise ValueError(f"dy must have shape {list(x.shape[:-1]) + [C]} and dtype {x.dtype}")
+    if out is not None and (out.shape != x.shape or out.dtype != x.dtype):
+        raise ValueError(f"out must have shape {list(x.shape)} and dtype {x.dtype}")
+    dev = _dev(x, W, dy, out)
+    dx = torch.empty_like(x) if out is None else out
+    _call(dev, lib().la_feature_map_rff_backward, _ptr(x), _ptr(W), _ptr(dy), _ptr(dx), x.numel() // max(D, 1), D, C,
+          _dtype_code(x), _stream(dev))
     return dx
 
 

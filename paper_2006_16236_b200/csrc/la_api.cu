@@ -318,6 +318,36 @@ int la_feature_map_poly2_backward(const void* x, const void* dy, void* dx, int64
 }
 
 // The optional buffer in which the non-causal forward keeps its per-split sums for the backward pass.
+static int check_rff(int64_t rows, int64_t D, int64_t C, int32_t dtype) {
+    if (rows < 0 || D < 1 || C < 2) return fail(LA_ERR_INVALID_ARG, "rows >= 0, D >= 1 and C >= 2 are required");
+    if (dtype != LA_F32 && dtype != LA_BF16) return fail(LA_ERR_INVALID_ARG, "dtype %d is not a la_dtype", dtype);
+    if (rows > 0 && !tc::rff_supported(rows, D, C, dtype))
+        return fail(LA_ERR_UNSUPPORTED, "random Fourier features take bf16, D a multiple of 8 in [8, 64], C = 64 or 128, rows < 2^31 "
+                                        "(got dtype %d, D=%lld, C=%lld, rows=%lld)", dtype, (long long)D, (long long)C, (long long)rows);
+    return LA_OK;
+}
+
+int la_feature_map_rff(const void* x, const void* W, void* y, int64_t rows, int64_t D, int64_t C, int32_t dtype, void* stream) {
+    if (int rc = check_rff(rows, D, C, dtype)) return rc;
+    if (rows == 0) return LA_OK;
+    LA_REQUIRE_PTR(x); LA_REQUIRE_PTR(W); LA_REQUIRE_PTR(y);
+    if (int rc = check_arch()) return rc;
+    LA_DEBUG_SPAN(x, (size_t)(rows * D) * 2); LA_DEBUG_SPAN(W, (size_t)(C / 2 * D) * 2); LA_DEBUG_SPAN(y, (size_t)(rows * C) * 2);
+    return debug_finish(tc::rff_forward(x, W, y, rows, (int)D, (int)C, (cudaStream_t)stream), stream);
+}
+
+int la_feature_map_rff_backward(const void* x, const void* W, const void* dy, void* dx, int64_t rows, int64_t D, int64_t C,
+                                int32_t dtype, void* stream) {
+    if (int rc = check_rff(rows, D, C, dtype)) return rc;
+    if (rows == 0) return LA_OK;
+    LA_REQUIRE_PTR(x); LA_REQUIRE_PTR(W); LA_REQUIRE_PTR(dy); LA_REQUIRE_PTR(dx);
+    if (dx == x) return fail(LA_ERR_INVALID_ARG, "dx must not alias x");
+    if (int rc = check_arch()) return rc;
+    LA_DEBUG_SPAN(x, (size_t)(rows * D) * 2); LA_DEBUG_SPAN(W, (size_t)(C / 2 * D) * 2); LA_DEBUG_SPAN(dy, (size_t)(rows * C) * 2);
+    LA_DEBUG_SPAN(dx, (size_t)(rows * D) * 2);
+    return debug_finish(tc::rff_backward(x, W, dy, dx, rows, (int)D, (int)C, (cudaStream_t)stream), stream);
+}
+
 static int check_linear_saved(const la_problem* p, const void* saved, size_t saved_bytes) {
     if (!saved) return LA_OK;
     if (!aligned16(saved)) return fail(LA_ERR_INVALID_ARG, "saved is not 16-byte aligned");

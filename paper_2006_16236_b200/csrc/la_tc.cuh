@@ -30,6 +30,10 @@ int linear_forward(const la_problem& p, const void* Q, const void* K, const void
                    float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st);
 int linear_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths,
                     const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+// random Fourier features (la_rff.cu)
+bool rff_supported(int64_t rows, int64_t D, int64_t C, int dtype);
+int rff_forward(const void* x, const void* W, void* y, int64_t rows, int D, int C, cudaStream_t st);
+int rff_backward(const void* x, const void* W, const void* dy, void* dx, int64_t rows, int D, int C, cudaStream_t st);
 }  // namespace tc
 
 }  // namespace la

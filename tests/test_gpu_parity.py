@@ -441,6 +441,62 @@ def test_poly2_feature_map_and_its_gradient(D, C, dtype):
     assert la.la_feature_map_poly2(torch.empty((0, D), dtype=dtype, device=DEV), C).shape == (0, C)
 
 
+@pytest.mark.parametrize("D,C,rows", [(64, 64, (3, 5, 67)), (64, 128, (2, 700)), (32, 64, (1000,)), (8, 128, (130,)), (64, 64, (40000,))],
+                         ids=["D64_C64", "D64_C128", "D32_C64", "D8_C128", "D64_C64_many_tiles"])
+def test_rff_feature_map_and_its_gradient(D, C, rows):
+    """Random Fourier features on the tensor cores against the oracle: several row tiles per CTA, a ragged last
+    tile, input widths below one K block (zero-filled by TMA) and both output widths."""
+    g = torch.Generator().manual_seed(10 * D + C)
+    x = torch.randn(rows + (D,), generator=g).to(torch.bfloat16)
+    W = torch.randn((C // 2, D), generator=g).to(torch.bfloat16)
+    dy = torch.randn(rows + (C,), generator=g).to(torch.bfloat16)
+    y = la.la_feature_map_rff(x.to(DEV), W.to(DEV))
+    dx = la.la_feature_map_rff_backward(x.to(DEV), W.to(DEV), dy.to(DEV))
+    la.la_last_device_status()
+    xr, Wr = x.double().numpy(), W.double().numpy()
+    ref = oracle.rff_feature_map(xr, Wr)
+    got = y.double().cpu().numpy()
+    assert got.shape == ref.shape
+    # every feature is below sqrt(2/C) in size: one bf16 rounding of that plus the fast sine's error
+    assert np.abs(got - ref).max() <= (2.0 / C) ** 0.5 * 2.0 ** -8 * 1.5, np.abs(got - ref).max()
+    assert_close(y, ref, torch.bfloat16, "rff y")
+    assert_close(dx, oracle.rff_feature_map_backward(xr, Wr, dy.double().numpy()), torch.bfloat16, "rff dx", grad=True)
+    # the same call again gives the same bits
+    assert torch.equal(y, la.la_feature_map_rff(x.to(DEV), W.to(DEV)))
+    assert la.la_feature_map_rff(torch.empty((0, D), dtype=torch.bfloat16, device=DEV), W.to(DEV)).shape == (0, C)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_rff_attention_end_to_end(causal):
+    """Queries and keys -> random Fourier features on the device -> attention with the identity map (the general
+    kernels: C = 128) and gradients back through both steps, against the oracle on the device's own features (a
+    stored bf16 tensor, like every other input).  Small inputs and few positions per head keep the weights of
+    Eq. 4, which are not guaranteed positive for signed features, away from zero."""
+    B, H, N, D, C = 2, 2, 96, 64, 128
+    Q, K, V, G = draw_qkvg(B, H, N, D, C, seed=77 + causal, dtype=torch.bfloat16)
+    Q, K = (Q * 0.05).to(torch.bfloat16), (K * 0.05).to(torch.bfloat16)
+    W = torch.randn((C // 2, D), generator=torch.Generator().manual_seed(3)).to(torch.bfloat16)
+    Qd, Kd, Vd, Gd, Wd = gpu(Q, K, V, G, W)
+    fQ, fK = la.la_feature_map_rff(Qd, Wd), la.la_feature_map_rff(Kd, Wd)
+    fwd = la.la_causal_forward if causal else la.la_linear_attention
+    bwd = la.la_causal_backward if causal else la.la_linear_attention_backward
+    O = fwd(fQ, fK, Vd, phi="identity")
+    dfQ, dfK, dV = bwd(fQ, fK, Vd, Gd, phi="identity")
+    dQ, dK = la.la_feature_map_rff_backward(Qd, Wd, dfQ), la.la_feature_map_rff_backward(Kd, Wd, dfK)
+    la.la_last_device_status()
+    fq, fk = fQ.double().cpu().numpy(), fK.double().cpu().numpy()
+    Vr, Gr, Wr = V.double().numpy(), G.double().numpy(), W.double().numpy()
+    Oref = oracle.linear_attention(fq, fk, Vr, causal, phi="identity")[0]
+    gq, gk, gv = oracle.linear_attention_backward(fq, fk, Vr, Gr, causal, phi="identity")
+    assert_close(O, Oref, torch.bfloat16, "rff attention O")
+    assert_close(dV, gv, torch.bfloat16, "rff attention dV", grad=True)
+    # the map's gradient is judged on the upstream gradient the device handed it
+    assert_close(dQ, oracle.rff_feature_map_backward(Q.double().numpy(), Wr, dfQ.double().cpu().numpy()), torch.bfloat16, "rff dQ", grad=True)
+    assert_close(dK, oracle.rff_feature_map_backward(K.double().numpy(), Wr, dfK.double().cpu().numpy()), torch.bfloat16, "rff dK", grad=True)
+    assert_close(dfQ, gq, torch.bfloat16, "rff attention dphi(Q)", grad=True)
+    assert_close(dfK, gk, torch.bfloat16, "rff attention dphi(K)", grad=True)
+
+
 @pytest.mark.parametrize("dtype", DTYPES)
 @pytest.mark.parametrize("causal", [False, True])
 @pytest.mark.parametrize("shape,signed", [((2, 2, 384, 8, 64), False), ((2, 2, 384, 8, 64), True),

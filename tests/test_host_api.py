@@ -193,6 +193,15 @@ def test_bad_arguments_are_rejected_on_the_host(L):
     assert L.la_feature_map_poly2_backward(ok, null, far, 4, 8, 64, 0, null) == -1
     assert L.la_feature_map_poly2_backward(ok, ok, far, 0, 8, 64, 0, null) == 0
     assert binding.poly2_columns(8) == 64 and binding.poly2_columns(5) == 32 and binding.poly2_columns(11) == 128
+    # random Fourier features: bf16 (dtype 1), D a multiple of 8 in [8, 64], C = 64 or 128; all refusals come before any CUDA call
+    rff = lambda rows, D, C, dt=1, x=ok, W=ok, y=ok: L.la_feature_map_rff(x, W, y, rows, D, C, dt, null)
+    assert rff(0, 64, 64) == 0
+    assert rff(-1, 64, 64) == -1 and rff(4, 0, 64) == -1 and rff(4, 64, 64, dt=5) == -1
+    assert rff(4, 64, 64, dt=0) == -2 and rff(4, 72, 64) == -2 and rff(4, 12, 64) == -2 and rff(4, 64, 96) == -2
+    assert rff(4, 64, 64, x=null) == -1 and rff(4, 64, 64, W=odd) == -1 and rff(4, 64, 64, y=null) == -1
+    assert L.la_feature_map_rff_backward(ok, ok, ok, ok, 4, 64, 64, 1, null) == -1          # dx aliases x
+    assert L.la_feature_map_rff_backward(ok, ok, null, far, 4, 64, 64, 1, null) == -1
+    assert L.la_feature_map_rff_backward(ok, ok, ok, far, 0, 64, 64, 1, null) == 0
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
