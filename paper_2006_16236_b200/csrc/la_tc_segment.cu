@@ -102,6 +102,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     // everything above is private to the CTA; from here on memory of the kernel before this one is touched
     allow_dependent_launch();
     grid_dependency_wait();
+    LA_TRACE_CTA(g_trace_seg, 2);
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
