@@ -182,12 +182,13 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         }
     } else if (warp >= 17) {
         // ------------------------------------------------------------- MMA issuers
-        // Two threads share the issue work (a tcgen05.mma occupies its issuing thread for about
-        // as long as it occupies the tensor pipe, and the waits of one stream would otherwise hold
-        // up the other): warp 17 issues the score products P and P [V | 1], warp 18 the state
-        // update and q [S | Z].  MMAs of one thread execute in order; the two accumulations into
-        // the same numerator are ordered through qs_full.
-        if (lane == 0) {
+        // Two warps share the issue work (the waits of one stream of products would otherwise hold up the
+        // other): warp 17 issues the score products P and P [V | 1], warp 18 the state update and
+        // q [S | Z].  Each runs its loop with all 32 lanes and issues through an elected lane, which keeps
+        // addresses and descriptors in uniform registers.  MMAs of one thread execute in order; the two
+        // accumulations into the same numerator are ordered through qs_full.
+        {
+            const bool leader = elect_one();
             const uint32_t idesc_p = umma_idesc_bf16(128, 128, 0, 0);
             const uint32_t idesc_num = umma_idesc_bf16(128, 80, 0, 1);
             const uint32_t idesc_s = umma_idesc_bf16(64, 80, 1, 1);
@@ -210,33 +211,33 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     if (c + 1 < L) {
                         // the buffer's previous readers are done: p_ready(c-1) was awaited before
                         // P [V | 1] of chunk c-1 was issued, and this thread's MMAs run in order
-                        ok = mbar_wait(&bars->mapped[(c + 1) % kStages], ((c + 1) / kStages) & 1, prm.status, kStatusPipeTimeout);
-                        if (!ok || *abort_flag) { ok = false; break; }
+                        ok = mbar_wait_warp(&bars->mapped[(c + 1) % kStages], ((c + 1) / kStages) & 1, prm.status, kStatusPipeTimeout);
+                        if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
                         tc_fence_after_sync();
                         const uint32_t nQ = lo_k(stage_addr(c + 1)), nK = lo_k(stage_addr(c + 1) + kTileBytes);
 #pragma unroll 1
                         for (int k = 0; k < 4; ++k)
-                            umma_bf16(tmem + kColP + (b ^ 1) * 128, mk(nQ + 2 * k), mk(nK + 2 * k), idesc_p, k > 0);
-                        umma_commit(&bars->p_full[b ^ 1]);
+                            umma_bf16(leader, tmem + kColP + (b ^ 1) * 128, mk(nQ + 2 * k), mk(nK + 2 * k), idesc_p, k > 0);
+                        umma_commit(leader, &bars->p_full[b ^ 1]);
                     }
                     if (c < 0) continue;
-                    LA_TRACE(g_trace_fwd, c, 2);
+                    if (leader) LA_TRACE(g_trace_fwd, c, 2);
                     // += P [V | 1] with the rounded, masked P read from TMEM, on top of q [S | Z]
-                    ok = mbar_wait(&bars->p_ready[b], (c >> 1) & 1, prm.status, kStatusPipeTimeout) &&
-                         mbar_wait(&bars->qs_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout);
+                    ok = mbar_wait_warp(&bars->p_ready[b], (c >> 1) & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait_warp(&bars->qs_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    LA_TRACE(g_trace_fwd, c, 3);
+                    if (leader) LA_TRACE(g_trace_fwd, c, 3);
                     const uint32_t aV = stage_addr(c) + 2 * kTileBytes;
                     const uint32_t dV1 = lo_mn(aV, aOnes - aV);
 #pragma unroll 1
                     for (int k = 0; k < 8; ++k)
-                        umma_bf16_ta(tmem + kColNum + b * kNumStride, tmem + kColP + b * 128 + (k >> 2) * 64 + (k & 3) * 8,
+                        umma_bf16_ta(leader, tmem + kColNum + b * kNumStride, tmem + kColP + b * 128 + (k >> 2) * 64 + (k & 3) * 8,
                                      mk(dV1 + kStepV1 * k), idesc_num, 1);
-                    umma_commit(&bars->o_full[b]);
+                    umma_commit(leader, &bars->o_full[b]);
                     // qs_full(c) was awaited: every MMA of either thread that reads this stage is covered
-                    umma_commit(&bars->empty[c % kStages]);
-                    LA_TRACE(g_trace_fwd, c, 4);
+                    umma_commit(leader, &bars->empty[c % kStages]);
+                    if (leader) LA_TRACE(g_trace_fwd, c, 4);
                 }
             } else {
                 #pragma unroll 1
@@ -244,28 +245,28 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     const int s = c % kStages, b = c & 1;
                     const uint32_t aQ = stage_addr(c), aK = aQ + kTileBytes, aV = aK + kTileBytes;
                     const uint32_t dQ = lo_k(aQ), dKmn = lo_mn(aK, kTileBytes), dV1 = lo_mn(aV, aOnes - aV);
-                    LA_TRACE(g_trace_fwd, c, 0);
+                    if (leader) LA_TRACE(g_trace_fwd, c, 0);
                     // St_c = St_{c-1} + k^T [V | 1]: the accumulator must have been read out (or initialised)
-                    ok = mbar_wait(&bars->mapped[s], (c / kStages) & 1, prm.status, kStatusPipeTimeout) &&
-                         (c == 0 ? mbar_wait(&bars->state_ready[1], 0, prm.status, kStatusPipeTimeout)
-                                 : mbar_wait(&bars->s_drained, (c - 1) & 1, prm.status, kStatusPipeTimeout));
-                    if (!ok || *abort_flag) { ok = false; break; }
+                    ok = mbar_wait_warp(&bars->mapped[s], (c / kStages) & 1, prm.status, kStatusPipeTimeout) &&
+                         (c == 0 ? mbar_wait_warp(&bars->state_ready[1], 0, prm.status, kStatusPipeTimeout)
+                                 : mbar_wait_warp(&bars->s_drained, (c - 1) & 1, prm.status, kStatusPipeTimeout));
+                    if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
 #pragma unroll 1
                     for (int k = 0; k < 8; ++k)
-                        umma_bf16(tmem + kColS, mk(dKmn + 128 * k), mk(dV1 + kStepV1 * k), idesc_s, 1);
-                    umma_commit(&bars->s_full);
-                    LA_TRACE(g_trace_fwd, c, 1);
+                        umma_bf16(leader, tmem + kColS, mk(dKmn + 128 * k), mk(dV1 + kStepV1 * k), idesc_s, 1);
+                    umma_commit(leader, &bars->s_full);
+                    if (leader) LA_TRACE(g_trace_fwd, c, 1);
                     // [num | den] = q [S | Z]_{c-1}: tile (c-1) & 1 holds the state before this chunk
-                    ok = mbar_wait(&bars->state_ready[b ^ 1], (c >> 1) & 1, prm.status, kStatusPipeTimeout);
-                    if (ok && c >= 2) ok = mbar_wait(&bars->o_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
+                    ok = mbar_wait_warp(&bars->state_ready[b ^ 1], (c >> 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (ok && c >= 2) ok = mbar_wait_warp(&bars->o_drained[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint32_t dS = lo_mn(sbase + kOffS + (b ^ 1) * kStateTileBytes, kDim * 128);
 #pragma unroll 1
                     for (int k = 0; k < 4; ++k)
-                        umma_bf16(tmem + kColNum + b * kNumStride, mk(dQ + 2 * k), mk(dS + 128 * k), idesc_num, k > 0);
-                    umma_commit(&bars->qs_full[b]);
+                        umma_bf16(leader, tmem + kColNum + b * kNumStride, mk(dQ + 2 * k), mk(dS + 128 * k), idesc_num, k > 0);
+                    umma_commit(leader, &bars->qs_full[b]);
                 }
             }
             if (!ok) *abort_flag = 1;

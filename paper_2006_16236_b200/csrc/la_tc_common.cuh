@@ -732,6 +732,18 @@ __device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, u
         : "memory");
 }
 
+// the same issued from a warp-wide loop by its elected lane (see umma_bf16(leader, ...))
+__device__ __forceinline__ void umma_bf16_ta(bool leader, uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, e;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 e, %5, 0;\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"((uint32_t)leader)
+        : "memory");
+}
+
 // Four tcgen05.mma over consecutive K groups of one product, out of line: the low descriptor words
 // advance by a_step / b_step per K group (2 for a K-major operand inside a 128-byte swizzle row, 128
 // for an MN-major operand whose K groups are 2 KB apart); the first one accumulates only if
