@@ -189,7 +189,8 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             }
         }
     } else if (warp == 9) {
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             // one M = 128, N = 80 product per K group: A = [X | aux], B = [Y | aux], the second 64-column block
             // of either operand addressed through the leading-offset field.
             // Accumulator rows 0..63: [A' | a'] = x'^T [Y | 1];  row 80: [ysum | count] = 1^T [Y | 1].
@@ -199,20 +200,20 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kLsStages;
                 const uint32_t aX = sbase + s * kLsStageBytes, aY = aX + kTileBytes, aA = sbase + kLsOffAux;
-                ok = mbar_wait(&bars->mapped[s], (c / kLsStages) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok || *abort_flag) { ok = false; break; }
+                ok = mbar_wait_warp(&bars->mapped[s], (c / kLsStages) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
-                LA_TRACE(g_trace_lin, c, 0);
+                if (leader) LA_TRACE(g_trace_lin, c, 0);
                 const uint32_t acc = (c != 0);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    umma_bf16(tmem, desc_mn(aX + k * 2048, aA - aX), desc_mn(aY + k * 2048, aA - aY), idesc, acc | (k != 0));
+                    umma_bf16(leader, tmem, desc_mn(aX + k * 2048, aA - aX), desc_mn(aY + k * 2048, aA - aY), idesc, acc | (k != 0));
                 }
-                umma_commit(&bars->empty[s]);
-                LA_TRACE(g_trace_lin, c, 1);
+                umma_commit(leader, &bars->empty[s]);
+                if (leader) LA_TRACE(g_trace_lin, c, 1);
             }
             if (!ok) *abort_flag = 1;
-            umma_commit(&bars->done);
+            umma_commit(leader, &bars->done);
         }
     } else {
         const int t = tid & 127, hf = tid >> 7;
@@ -482,7 +483,8 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             }
         }
     } else if (warp == 9) {
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
             const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);
             const uint32_t aSt = sbase + kApOffState;
@@ -491,46 +493,46 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             // 1 / dn, once the epilogue threads have written the weighted tile: one M = 128, N = 80 product per K
             // group, A = [XS | aux], B = [G | aux] (second blocks through the leading-offset field)
             auto issue_sums = [&](int c) -> bool {
-                if (!mbar_wait(&bars->xs_ready, c & 1, prm.status, kStatusPipeTimeout) || *abort_flag) return false;
+                if (!mbar_wait_warp(&bars->xs_ready, c & 1, prm.status, kStatusPipeTimeout) || __any_sync(0xFFFFFFFFu, *abort_flag)) return false;
                 tc_fence_after_sync();
                 const uint32_t idesc = umma_idesc_bf16(128, 80, 1, 1);
                 const uint32_t aXS = sbase + kApOffXS, aAux = sbase + kApOffAux;
                 const uint32_t aG = sbase + kApOffStage + (c % kApStages) * 2 * kTileBytes + kTileBytes;
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    umma_bf16(tmem + kApColSums, desc_mn(aXS + k * 2048, aAux - aXS), desc_mn(aG + k * 2048, aAux - aG), idesc,
+                    umma_bf16(leader, tmem + kApColSums, desc_mn(aXS + k * 2048, aAux - aXS), desc_mn(aG + k * 2048, aAux - aG), idesc,
                               (c | k) != 0);
-                umma_commit(&bars->empty[c % kApStages]);
-                umma_commit(&bars->xs_free);
+                umma_commit(leader, &bars->empty[c % kApStages]);
+                umma_commit(leader, &bars->xs_free);
                 return true;
             };
             #pragma unroll 1
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kApStages, b = c & 1;
                 const uint32_t aX = sbase + kApOffStage + s * 2 * kTileBytes, aY = aX + kTileBytes;
-                ok = mbar_wait(&bars->mapped[s], (c / kApStages) & 1, prm.status, kStatusPipeTimeout);
-                if (ok && c >= 2) ok = mbar_wait(&bars->acc_free[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok || *abort_flag) { ok = false; break; }
+                ok = mbar_wait_warp(&bars->mapped[s], (c / kApStages) & 1, prm.status, kStatusPipeTimeout);
+                if (ok && c >= 2) ok = mbar_wait_warp(&bars->acc_free[b], ((c >> 1) - 1) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d0 = tmem + b * 128, d1 = d0 + 64;
                 if (kMode == kApplyForward) {
                     for (int k = 0; k < 4; ++k)      // q' S''
-                        umma_bf16(d0, desc_k(aX + k * 32), desc_mn(aSt + k * 2048), idesc_kmn, k > 0);
+                        umma_bf16(leader, d0, desc_k(aX + k * 32), desc_mn(aSt + k * 2048), idesc_kmn, k > 0);
                 } else if (kMode == kApplyBackwardQ) {
                     for (int k = 0; k < 4; ++k)      // h'' = G S''^T
-                        umma_bf16(d0, desc_k(aY + k * 32), desc_k(aSt + k * 32), idesc_kk, k > 0);
+                        umma_bf16(leader, d0, desc_k(aY + k * 32), desc_k(aSt + k * 32), idesc_kk, k > 0);
                 } else {
                     for (int k = 0; k < 4; ++k)      // V R''^T
-                        umma_bf16(d0, desc_k(aY + k * 32), desc_k(aSt + k * 32), idesc_kk, k > 0);
+                        umma_bf16(leader, d0, desc_k(aY + k * 32), desc_k(aSt + k * 32), idesc_kk, k > 0);
                     for (int k = 0; k < 4; ++k)      // k' R''
-                        umma_bf16(d1, desc_k(aX + k * 32), desc_mn(aSt + k * 2048), idesc_kmn, k > 0);
+                        umma_bf16(leader, d1, desc_k(aX + k * 32), desc_mn(aSt + k * 2048), idesc_kmn, k > 0);
                 }
-                umma_commit(&bars->acc_full[b]);
-                umma_commit(&bars->empty[s]);
+                umma_commit(leader, &bars->acc_full[b]);
+                umma_commit(leader, &bars->empty[s]);
                 if (kMode == kApplyBackwardQ && c >= 1) ok = issue_sums(c - 1);
             }
             if (kMode == kApplyBackwardQ && ok && L >= 1) ok = issue_sums(L - 1);
-            if (kMode == kApplyBackwardQ) umma_commit(&bars->sums_done);
+            if (kMode == kApplyBackwardQ) umma_commit(leader, &bars->sums_done);
             if (!ok) *abort_flag = 1;
         }
     } else if (warp >= 4 && warp < 8) {

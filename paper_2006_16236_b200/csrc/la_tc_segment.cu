@@ -126,7 +126,8 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             }
         }
     } else if (warp == 5) {
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             // one M = 64, N = 80 product per K group: B = [Y | a], the second 64-column block being the
             // column tile (same K group)
             const uint32_t idesc = umma_idesc_bf16(64, 80, 1, 1);
@@ -136,18 +137,18 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
             for (int c = 0; c < L && ok; ++c) {
                 const int s = c % kSumStages;
                 const uint32_t aX = sbase + s * kSumStageBytes, aY = aX + kTileBytes;
-                ok = mbar_wait(&bars->mapped[s], (c / kSumStages) & 1, prm.status, kStatusPipeTimeout);
-                if (!ok || *abort_flag) { ok = false; break; }
+                ok = mbar_wait_warp(&bars->mapped[s], (c / kSumStages) & 1, prm.status, kStatusPipeTimeout);
+                if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
-                LA_TRACE(g_trace_seg, c, 0);
+                if (leader) LA_TRACE(g_trace_seg, c, 0);
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    umma_bf16(tmem, desc_mn(aX + k * 2048), desc_mn(aY + k * 2048, aAux - aY), idesc, (c | k) != 0);
-                umma_commit(&bars->empty[s]);
-                LA_TRACE(g_trace_seg, c, 1);
+                    umma_bf16(leader, tmem, desc_mn(aX + k * 2048), desc_mn(aY + k * 2048, aAux - aY), idesc, (c | k) != 0);
+                umma_commit(leader, &bars->empty[s]);
+                if (leader) LA_TRACE(g_trace_seg, c, 1);
             }
             if (!ok) *abort_flag = 1;
-            umma_commit(&bars->done);
+            umma_commit(leader, &bars->done);
         }
     } else {
         const int t = tid;
