@@ -419,6 +419,14 @@ def bench_decode(la, w, dev, pk, n_steps=None, batch=None):
             fn(pr, q, k, v, Sp, Zp, o, st)
 
     us_raw = timed(run_raw)
+    # the binding's prepared form: arguments checked and marshalled once per buffer set, then one foreign call per step
+    steps = [la.prepare_recurrent_step(q_t[t], k_t[t], v_t[t], S, Z, out=out[t]) for t in range(T)]
+
+    def run_prepared():
+        for step in steps:
+            step()
+
+    us_prepared = timed(run_prepared)
     us_graph = None
     try:
         side = torch.cuda.Stream()
@@ -437,7 +445,8 @@ def bench_decode(la, w, dev, pk, n_steps=None, batch=None):
     us = min(us_eager, us_raw, us_graph) if us_graph else min(us_eager, us_raw)
     gbs = algorithmic_bytes(w, "both") / us * 1e-3
     res = {"workload": w.name, "steps_per_s": 1e6 / us, "us_per_step": us, "launches": T,
-           "us_per_step_host_issued": us_eager, "us_per_step_host_issued_raw_c_abi": us_raw, "us_per_step_cuda_graph": us_graph,
+           "us_per_step_host_issued": us_eager, "us_per_step_host_issued_raw_c_abi": us_raw, "us_per_step_host_issued_prepared": us_prepared,
+           "us_per_step_cuda_graph": us_graph,
            "alg_gbs": gbs, "hbm_frac": gbs / pk["hbm_gbs"], "state_bytes": S.numel() * 4,
            "note": ("state fits the 126 MB L2, so the fraction may exceed the DRAM roofline"
                     if S.numel() * 4 < 100e6 else "state exceeds L2: every step streams it from and to HBM")}

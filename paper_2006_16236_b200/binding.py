@@ -511,6 +511,39 @@ def la_recurrent_step(q, k, v, S, Z, phi="elu1", eps=0.0, out=None):
     return out
 
 
+class PreparedStep:
+    """A decode call whose arguments were checked and marshalled once: calling it enqueues the same library call
+    again on the stream it was prepared on (the tensors are updated in place, as in a generation loop whose
+    buffers do not move).  Per call it costs one foreign-function call instead of the argument checks."""
+
+    __slots__ = ("_fn", "_args", "_keep", "_dev", "out")
+
+    def __init__(self, fn, args, keep, dev, out):
+        self._fn, self._args, self._keep, self._dev, self.out = fn, args, keep, dev, out
+
+    def __call__(self):
+        rc = self._fn(*self._args)
+        if rc != 0:
+            _check(rc)
+        return self.out
+
+
+def prepare_recurrent_step(q, k, v, S, Z, phi="elu1", eps=0.0, out=None) -> PreparedStep:
+    """la_recurrent_step with its checks done once: returns a callable that repeats the step on the same tensors
+    (refill q, k, v in place between calls) on the stream that is current now, with the tensors' device current."""
+    if q.dim() != 3 or v.dim() != 3:
+        raise ValueError("expected q,k [B,H,D], v [B,H,M], fp32 S [B,H,D,M] and Z [B,H,D]")
+    B, H, D = q.shape
+    p = make_problem(B, H, 1, D, v.shape[2], _dtype_code(q), phi, eps)
+    _expect(p, q.dtype, q=(q, "q1"), k=(k, "q1"), v=(v, "v1"), S=(S, "S"), Z=(Z, "Z"), out=(out, "v1"))
+    dev = _dev(q, k, v, S, Z, out)
+    if dev.index != torch.cuda.current_device():
+        raise ValueError("make the tensors' device current before preparing a step")
+    out = torch.empty_like(v) if out is None else out
+    args = (ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(S), _ptr(Z), _ptr(out), _stream(dev))
+    return PreparedStep(lib().la_recurrent_step, args, (p, q, k, v, S, Z, out), dev, out)
+
+
 def la_decode_layer_step(x, Wqkv, Wo, S, Z, phi="elu1", eps=0.0, out=None, ws=None):
     """One decode step of a whole attention sublayer: x [B,F] -> y [B,F] with F = H*D (bf16, D = M = 64);
     Wqkv [3F,F] and Wo [F,F] are "outputs x inputs" like a linear layer's weight; S [B,H,D,M], Z [B,H,D] (fp32)

@@ -612,7 +612,9 @@ int la_recurrent_step(const la_problem* p, const void* q, const void* k, const v
         LA_DEBUG_SPAN(q, tb.qk); LA_DEBUG_SPAN(k, tb.qk); LA_DEBUG_SPAN(v, tb.vo); LA_DEBUG_SPAN(out, tb.vo);
         LA_DEBUG_SPAN(S, tb.s); LA_DEBUG_SPAN(Z, tb.z);
     }
-    return debug_finish(launch_recurrent_step(*p, q, k, v, S, Z, out, (cudaStream_t)stream), stream);
+    // launched as a programmatic dependent: a decode loop's next step is scheduled while this one runs (the kernel
+    // waits for its predecessor in the stream before it touches memory)
+    return debug_finish(launch_recurrent_step(*p, q, k, v, S, Z, out, (cudaStream_t)stream, /*chained=*/true), stream);
 }
 
 int la_decode_layer_step(const la_problem* p, const void* x, const void* Wqkv, const void* Wo,

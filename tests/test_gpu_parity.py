@@ -778,6 +778,26 @@ def test_decode_layer_steps_against_the_oracle(B, H):
     assert_close(Z, Zo, torch.bfloat16, "layer Z")
 
 
+def test_prepared_recurrent_step_repeats_the_regular_call():
+    """The prepared form (checks and marshalling done once) enqueues exactly the regular call: same bits, state
+    updated in place, inputs refilled in place between the steps."""
+    B, H, D, M, T = 5, 3, 64, 64, 6
+    Q, K, V, _ = draw_qkvg(B, H, T, D, M, seed=9, dtype=torch.bfloat16, with_grad=False)
+    qs, ks, vs = (t.transpose(1, 2).transpose(0, 1).contiguous().to(DEV) for t in (Q, K, V))     # [T,B,H,.]
+    S1, Z1 = torch.zeros((B, H, D, M), device=DEV), torch.zeros((B, H, D), device=DEV)
+    S2, Z2 = torch.zeros_like(S1), torch.zeros_like(Z1)
+    q, k, v = torch.empty_like(qs[0]), torch.empty_like(ks[0]), torch.empty_like(vs[0])
+    step = la.prepare_recurrent_step(q, k, v, S2, Z2)
+    for t in range(T):
+        ref = la.la_recurrent_step(qs[t], ks[t], vs[t], S1, Z1)
+        q.copy_(qs[t]); k.copy_(ks[t]); v.copy_(vs[t])
+        out = step()
+        assert torch.equal(out, ref), t
+    assert torch.equal(S1, S2) and torch.equal(Z1, Z2)
+    with pytest.raises(ValueError):
+        la.prepare_recurrent_step(q, k, v, S2[:, :2], Z2)
+
+
 def test_decode_layer_rejects_what_it_does_not_take():
     B, H, D = 4, 2, 32
     x = torch.zeros((B, H * D), dtype=torch.bfloat16, device=DEV)
