@@ -87,24 +87,24 @@ projection_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
             }
         }
     } else if (warp == 5) {
-        if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16(128, kGemmTileN, 0, 0);
-            bool ok = true;
-            #pragma unroll 1
-            for (int kb = 0; kb < prm.kblocks && ok; ++kb) {
-                const int s = kb % kGemmStages;
-                ok = mbar_wait(&bars->full[s], (kb / kGemmStages) & 1, prm.status, kStatusTmaTimeout);
-                if (!ok || *abort_flag) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t aA = sbase + s * kGemmStageBytes, aW = aA + kTileBytes;
+        // all 32 lanes run the loop and an elected one issues: addresses and descriptors stay in uniform registers
+        const bool leader = elect_one();
+        const uint32_t idesc = umma_idesc_bf16(128, kGemmTileN, 0, 0);
+        bool ok = true;
+        #pragma unroll 1
+        for (int kb = 0; kb < prm.kblocks && ok; ++kb) {
+            const int s = kb % kGemmStages;
+            ok = mbar_wait_warp(&bars->full[s], (kb / kGemmStages) & 1, prm.status, kStatusTmaTimeout);
+            if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t aA = sbase + s * kGemmStageBytes, aW = aA + kTileBytes;
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    umma_bf16(tmem, desc_k(aA + 32 * k), desc_k(aW + 32 * k), idesc, (kb | k) != 0);
-                umma_commit(&bars->empty[s]);
-            }
-            if (!ok) *abort_flag = 1;
-            umma_commit(&bars->done);
+            for (int k = 0; k < 4; ++k)
+                umma_bf16(leader, tmem, desc_k(aA + 32 * k), desc_k(aW + 32 * k), idesc, (kb | k) != 0);
+            umma_commit(leader, &bars->empty[s]);
         }
+        if (!ok) *abort_flag = 1;
+        umma_commit(leader, &bars->done);
     } else {
         // epilogue: row t of the tile, 64 columns
         const int t = tid;
