@@ -682,14 +682,15 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         }
     } else if (warp >= 17) {
         // ------------------------------------------------------------- MMA issuers
-        // Three threads share the issue work (an issuing thread needs 100 to 140 cycles per tcgen05.mma here,
-        // about twice what the tensor pipe does).  Warps 17 and 19: one score tile each and the product that
+        // Three warps share the issue work; each runs its loop with all 32 lanes and issues through an elected
+        // lane (operands stay in uniform registers: about 40 cycles per tcgen05.mma instead of 100 to 140).  Warps 17 and 19: one score tile each and the product that
         // consumes it (transposed tiles, rows = keys: Ph^T = k qh^T, then gV += Ph^T G; dP^T = [V | 1] [G | dl]^T,
         // whose fifth K step is (ones in two columns) x (dl_i split into a bf16 high and low part), then
         // gk += dP^T qh; the rounded tiles are read from TMEM).  Warp 18: everything that involves the running
         // state ([R | r] += qh^T [G | dl]; gV = k R, gk = V R^T, which start the two accumulators).  MMAs of
         // one thread execute in order; kr_full / vr_full order two threads' writes to one accumulator.
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             const uint32_t idesc_pp = umma_idesc_bf16(128, 128, 0, 0);
             const uint32_t idesc_kk = umma_idesc_bf16(128, 64, 0, 0);
             const uint32_t idesc_kmn = umma_idesc_bf16(128, 64, 0, 1);     // also: A from TMEM, B MN-major
@@ -717,11 +718,11 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 uint64_t* acc_started = dp ? &bars->vr_full : &bars->kr_full;      // the state thread's first product
                 uint64_t* acc_full = dp ? &bars->dkv_full : &bars->dv_full;
                 auto issue_tile = [&](int i) {
-                    umma_group4(tmem + col, lo_k(stage_q(i) + offA), 2, lo_k(stage_q(i) + offB), 2, idesc_pp, 0);
-                    if (dp) umma_bf16(tmem + col, desc_ones(aOnes), desc_k(aAux), idesc_pp, 1);    // + dl_i (fifth K step)
-                    umma_commit(tile_full);
+                    umma_group4(leader, tmem + col, lo_k(stage_q(i) + offA), 2, lo_k(stage_q(i) + offB), 2, idesc_pp, 0);
+                    if (dp) umma_bf16(leader, tmem + col, desc_ones(aOnes), desc_k(aAux), idesc_pp, 1);    // + dl_i (fifth K step)
+                    umma_commit(leader, tile_full);
                 };
-                ok = mbar_wait(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !*abort_flag;
+                ok = mbar_wait_warp(&bars->mapped[0], 0, prm.status, kStatusPipeTimeout) && !__any_sync(0xFFFFFFFFu, *abort_flag);
                 if (ok) {
                     tc_fence_after_sync();
                     issue_tile(0);
@@ -729,25 +730,25 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 #pragma unroll 1
                 for (int i = 0; i < L && ok; ++i) {
                     const uint32_t dC = lo_mn(stage_q(i) + offC, kTileBytes);
-                    if (!dp) LA_TRACE(g_trace_dkv, i, 0);
-                    ok = mbar_wait(tile_ready, i & 1, prm.status, kStatusPipeTimeout) &&
-                         mbar_wait(acc_started, i & 1, prm.status, kStatusMmaTimeout);
-                    if (!ok || *abort_flag) { ok = false; break; }
+                    if (leader && !dp) LA_TRACE(g_trace_dkv, i, 0);
+                    ok = mbar_wait_warp(tile_ready, i & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait_warp(acc_started, i & 1, prm.status, kStatusMmaTimeout);
+                    if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
-                    LA_TRACE(g_trace_dkv, i, dp ? 3 : 1);
-                    umma_group4_ta(tmem + acc, tmem + col, dC, 128, idesc_kmn, 1);                 // gV += Ph^T G / gk += dP^T qh
-                    umma_group4_ta(tmem + acc, tmem + col + 64, dC + 512, 128, idesc_kmn, 1);
-                    umma_commit(acc_full);      // gV is complete first: its epilogue overlaps gk
+                    if (leader) LA_TRACE(g_trace_dkv, i, dp ? 3 : 1);
+                    umma_group4_ta(leader, tmem + acc, tmem + col, dC, 128, idesc_kmn, 1);                 // gV += Ph^T G / gk += dP^T qh
+                    umma_group4_ta(leader, tmem + acc, tmem + col + 64, dC + 512, 128, idesc_kmn, 1);
+                    umma_commit(leader, acc_full);      // gV is complete first: its epilogue overlaps gk
                     // this thread's reads of the stage; the awaited vr_full(i) covers the state thread's products on it
-                    umma_commit(&bars->empty[i % kKvStages]);
+                    umma_commit(leader, &bars->empty[i % kKvStages]);
                     if (i + 1 < L) {
                         // mapped(i+1) also says that the dl column tile holds chunk i+1
-                        ok = mbar_wait(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
+                        ok = mbar_wait_warp(&bars->mapped[(i + 1) % kKvStages], ((i + 1) / kKvStages) & 1, prm.status, kStatusPipeTimeout);
                         if (!ok) break;
                         tc_fence_after_sync();
                         issue_tile(i + 1);
                     }
-                    LA_TRACE(g_trace_dkv, i, dp ? 4 : 2);
+                    if (leader) LA_TRACE(g_trace_dkv, i, dp ? 4 : 2);
                 }
             } else {
                 #pragma unroll 1
@@ -757,29 +758,29 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     const uint32_t dQmn = lo_mn(aQ, kTileBytes), dG1 = lo_mn(aG, aAux - aG);
                     // gV = k R_{c+1} starts its accumulator as soon as the epilogue of the previous chunk has taken the
                     // old values out of TMEM (the score thread waits for it before gV += Ph^T G)
-                    ok = mbar_wait(&bars->mapped[i % kKvStages], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout) &&
-                         mbar_wait(&bars->state_ready, i & 1, prm.status, kStatusPipeTimeout);
-                    if (ok && i >= 1) ok = mbar_wait(&bars->dv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
-                    if (!ok || *abort_flag) { ok = false; break; }
+                    ok = mbar_wait_warp(&bars->mapped[i % kKvStages], (i / kKvStages) & 1, prm.status, kStatusPipeTimeout) &&
+                         mbar_wait_warp(&bars->state_ready, i & 1, prm.status, kStatusPipeTimeout);
+                    if (ok && i >= 1) ok = mbar_wait_warp(&bars->dv_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (!ok || __any_sync(0xFFFFFFFFu, *abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
-                    umma_group4(tmem + kKvColDv, lo_k(aK), 2, lo_mn(aR, kTileBytes), 128, idesc_kmn, 0);
-                    umma_commit(&bars->kr_full);
+                    umma_group4(leader, tmem + kKvColDv, lo_k(aK), 2, lo_mn(aR, kTileBytes), 128, idesc_kmn, 0);
+                    umma_commit(leader, &bars->kr_full);
                     // [R | r] += qh^T [G | dl], the dl column tile being the second 64-column block of B.  The
                     // previous state has been converted (state_ready), and dP^T of this chunk, which reads the same
                     // column tile, must be done (dp_full): the operand warps take r_full as the signal that the tile
                     // may be rewritten.
-                    ok = mbar_wait(&bars->dp_full, i & 1, prm.status, kStatusMmaTimeout);
+                    ok = mbar_wait_warp(&bars->dp_full, i & 1, prm.status, kStatusMmaTimeout);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    umma_group4(tmem + kKvColR, dQmn, 128, dG1, 128, idesc_r, 1);
-                    umma_group4(tmem + kKvColR, dQmn + 512, 128, dG1 + 512, 128, idesc_r, 1);
-                    umma_commit(&bars->r_full);
+                    umma_group4(leader, tmem + kKvColR, dQmn, 128, dG1, 128, idesc_r, 1);
+                    umma_group4(leader, tmem + kKvColR, dQmn + 512, 128, dG1 + 512, 128, idesc_r, 1);
+                    umma_commit(leader, &bars->r_full);
                     // gk = V R_{c+1}^T likewise, once the previous gk has been taken out
-                    if (i >= 1) ok = mbar_wait(&bars->dk_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
+                    if (i >= 1) ok = mbar_wait_warp(&bars->dk_drained, (i - 1) & 1, prm.status, kStatusPipeTimeout);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    umma_group4(tmem + kKvColDk, lo_k(aV), 2, lo_k(aR), 2, idesc_kk, 0);
-                    umma_commit(&bars->vr_full);
+                    umma_group4(leader, tmem + kKvColDk, lo_k(aV), 2, lo_k(aR), 2, idesc_kk, 0);
+                    umma_commit(leader, &bars->vr_full);
                 }
             }
             if (!ok) *abort_flag = 1;

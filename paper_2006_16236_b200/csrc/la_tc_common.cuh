@@ -744,26 +744,25 @@ __device__ __forceinline__ void umma_bf16_ta(bool leader, uint32_t d_tmem, uint3
         : "memory");
 }
 
-// Four tcgen05.mma over consecutive K groups of one product, out of line: the low descriptor words
-// advance by a_step / b_step per K group (2 for a K-major operand inside a 128-byte swizzle row, 128
-// for an MN-major operand whose K groups are 2 KB apart); the first one accumulates only if
-// `acc_first`.  An issuing thread spends about a dozen instructions per MMA on moving operands to
-// uniform registers; sharing one copy between all products of a kernel keeps the issuing loops, which
-// run next to every other role's loop, small enough for the instruction cache.
-static __device__ __noinline__ void umma_group4(uint32_t d_tmem, uint32_t a_lo, uint32_t a_step, uint32_t b_lo, uint32_t b_step,
-                                         uint32_t idesc, uint32_t acc_first) {
+// Four tcgen05.mma over consecutive K groups of one product, issued from a warp-wide loop through its elected
+// lane (see umma_bf16(leader, ...)): the low descriptor words advance by a_step / b_step per K group (2 for a
+// K-major operand inside a 128-byte swizzle row, 128 for an MN-major operand whose K groups are 2 KB apart);
+// the first one accumulates only if `acc_first`.  Inline: with the operands in uniform registers a product is a
+// handful of instructions, and a call would move them back into vector registers (issued from a one-lane
+// loop these groups were out of line, a dozen instructions per product).
+__device__ __forceinline__ void umma_group4(bool leader, uint32_t d_tmem, uint32_t a_lo, uint32_t a_step, uint32_t b_lo,
+                                            uint32_t b_step, uint32_t idesc, uint32_t acc_first) {
     const uint64_t hi = desc_k(0) & 0xFFFFFFFF00000000ull;
 #pragma unroll
     for (uint32_t k = 0; k < 4; ++k)
-        sm100::umma_bf16(d_tmem, hi | (a_lo + k * a_step), hi | (b_lo + k * b_step), idesc, k > 0 ? 1u : acc_first);
+        sm100::umma_bf16(leader, d_tmem, hi | (a_lo + k * a_step), hi | (b_lo + k * b_step), idesc, k > 0 ? 1u : acc_first);
 }
-// The same with the A operand in TMEM (eight columns of bf16 pairs per K group).
-static __device__ __noinline__ void umma_group4_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_step, uint32_t idesc,
-                                            uint32_t acc_first) {
+__device__ __forceinline__ void umma_group4_ta(bool leader, uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_step,
+                                               uint32_t idesc, uint32_t acc_first) {
     const uint64_t hi = desc_k(0) & 0xFFFFFFFF00000000ull;
 #pragma unroll
     for (uint32_t k = 0; k < 4; ++k)
-        umma_bf16_ta(d_tmem, a_tmem + k * 8, hi | (b_lo + k * b_step), idesc, k > 0 ? 1u : acc_first);
+        umma_bf16_ta(leader, d_tmem, a_tmem + k * 8, hi | (b_lo + k * b_step), idesc, k > 0 ? 1u : acc_first);
 }
 
 }  // namespace tc
