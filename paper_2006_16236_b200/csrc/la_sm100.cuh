@@ -257,6 +257,23 @@ __device__ __forceinline__ void umma_commit(bool leader, uint64_t* bar) {
         ::"r"(smem_u32(bar)), "r"((uint32_t)leader)
         : "memory");
 }
+// The producer's two instructions for a warp-wide loop: executed by the elected lane only.
+__device__ __forceinline__ void mbar_arrive_expect_tx(bool leader, uint64_t* bar, uint32_t bytes) {
+    asm volatile(
+        "{\n\t.reg .pred e;\n\t"
+        "setp.ne.b32 e, %2, 0;\n\t"
+        "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}"
+        ::"r"(smem_u32(bar)), "r"(bytes), "r"((uint32_t)leader)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(bool leader, void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "{\n\t.reg .pred e;\n\t"
+        "setp.ne.b32 e, %5, 0;\n\t"
+        "@e cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n\t}"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)), "r"((uint32_t)leader)
+        : "memory");
+}
 // Bounded wait by a whole warp: the same answer in every lane, and known to the compiler as such.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, int* status, int code) {
     return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, status, code));

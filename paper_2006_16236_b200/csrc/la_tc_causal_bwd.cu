@@ -191,26 +191,30 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         // this piece is all padding: nothing to sweep (its dQ rows are zeroed below)
     } else if (warp == 12) {
         // ------------------------------------------------------------ TMA producer
+        // warp-wide loop, the elected lane issues (as in the MMA warps: the time from a stage's release to the
+        // requests for its next tiles is part of the longest chain of this two-stage kernel)
+        const bool leader = elect_one();
         if (lane == 0) {
             prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG); prefetch_tensormap(&mapQ);
             prefetch_tensormap(&mapDQ);
-            #pragma unroll 1
-            for (int c = 0; c < L; ++c) {
-                const int s = c % kDqStages;
-                if (c >= kDqStages && !mbar_wait(&bars->empty[s], ((c / kDqStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
-                    *abort_flag = 1;
-                    break;
-                }
-                if (*abort_flag) break;
-                uint8_t* st = smem + kDqOffStage + s * 4 * kTileBytes;
-                const int y = (int)(row0 + (int64_t)c * kChunk);
-                LA_TRACE(g_trace_dq, c, 13);
-                mbar_arrive_expect_tx(&bars->full[s], 4 * kTileBytes);
-                tma_load_2d(st + kTileBytes, &mapV, 0, y, &bars->full[s]);
-                tma_load_2d(st + 2 * kTileBytes, &mapG, 0, y, &bars->full[s]);
-                tma_load_2d(st, &mapK, 0, y, &bars->full[s]);
-                tma_load_2d(st + 3 * kTileBytes, &mapQ, 0, y, &bars->full[s]);
+        }
+        __syncwarp();
+        #pragma unroll 1
+        for (int c = 0; c < L; ++c) {
+            const int s = c % kDqStages;
+            if (c >= kDqStages && !mbar_wait_warp(&bars->empty[s], ((c / kDqStages) - 1) & 1, prm.status, kStatusPipeTimeout)) {
+                *abort_flag = 1;
+                break;
             }
+            if (__any_sync(0xFFFFFFFFu, *abort_flag)) break;
+            uint8_t* st = smem + kDqOffStage + s * 4 * kTileBytes;
+            const int y = (int)(row0 + (int64_t)c * kChunk);
+            if (leader) LA_TRACE(g_trace_dq, c, 13);
+            mbar_arrive_expect_tx(leader, &bars->full[s], 4 * kTileBytes);
+            tma_load_2d(leader, st + kTileBytes, &mapV, 0, y, &bars->full[s]);
+            tma_load_2d(leader, st + 2 * kTileBytes, &mapG, 0, y, &bars->full[s]);
+            tma_load_2d(leader, st, &mapK, 0, y, &bars->full[s]);
+            tma_load_2d(leader, st + 3 * kTileBytes, &mapQ, 0, y, &bars->full[s]);
         }
     } else if (warp >= 13) {
         // ------------------------------------------------------------- MMA issuers
