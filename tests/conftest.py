@@ -14,7 +14,7 @@ def pytest_configure(config):
 
 def pytest_sessionfinish(session, exitstatus):
     """After a GPU session: the three error figures of every comparison with the oracle, worst case per tensor
-    name and dtype, as a text table under gpurun_out/ (the scratch folder of a GPU run)."""
+    name and dtype, as a text table in the run's output folder (written only where that folder exists)."""
     try:
         from parity import parity_report
     except ImportError:
