@@ -194,6 +194,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         // warp-wide loop, the elected lane issues (as in the MMA warps: the time from a stage's release to the
         // requests for its next tiles is part of the longest chain of this two-stage kernel)
         const bool leader = elect_one();
+        const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
         if (lane == 0) {
             prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG); prefetch_tensormap(&mapQ);
             prefetch_tensormap(&mapDQ);
@@ -210,11 +211,14 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             uint8_t* st = smem + kDqOffStage + s * 4 * kTileBytes;
             const int y = (int)(row0 + (int64_t)c * kChunk);
             if (leader) LA_TRACE(g_trace_dq, c, 13);
+            // the reverse sweep starts where this piece ends: its last chunks are asked to stay in L2, the rest,
+            // which will be long gone by then, to leave first
+            const uint64_t pol = c >= L_full - kKeepTailChunks ? pol_keep : pol_stream;
             mbar_arrive_expect_tx(leader, &bars->full[s], 4 * kTileBytes);
-            tma_load_2d(leader, st + kTileBytes, &mapV, 0, y, &bars->full[s]);
-            tma_load_2d(leader, st + 2 * kTileBytes, &mapG, 0, y, &bars->full[s]);
-            tma_load_2d(leader, st, &mapK, 0, y, &bars->full[s]);
-            tma_load_2d(leader, st + 3 * kTileBytes, &mapQ, 0, y, &bars->full[s]);
+            tma_load_2d(leader, st + kTileBytes, &mapV, 0, y, &bars->full[s], pol);
+            tma_load_2d(leader, st + 2 * kTileBytes, &mapG, 0, y, &bars->full[s], pol);
+            tma_load_2d(leader, st, &mapK, 0, y, &bars->full[s], pol);
+            tma_load_2d(leader, st + 3 * kTileBytes, &mapQ, 0, y, &bars->full[s], pol);
         }
     } else if (warp >= 13) {
         // ------------------------------------------------------------- MMA issuers
@@ -667,6 +671,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         if (lane == 0) {
             prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV); prefetch_tensormap(&mapG);
             prefetch_tensormap(&mapDK); prefetch_tensormap(&mapDV);
+            const uint64_t pol_stream = l2_policy_evict_first();
             #pragma unroll 1
             for (int i = 0; i < L; ++i) {
                 const int s = i % kKvStages;
@@ -678,10 +683,12 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 uint8_t* st = smem + kKvOffStage + s * kKvStageBytes;
                 const int y = (int)chunk_row(i);
                 mbar_arrive_expect_tx(&bars->full[s], kKvStageBytes);
-                tma_load_2d(st, &mapQ, 0, y, &bars->full[s]);
-                tma_load_2d(st + kTileBytes, &mapK, 0, y, &bars->full[s]);
-                tma_load_2d(st + 2 * kTileBytes, &mapV, 0, y, &bars->full[s]);
-                tma_load_2d(st + 3 * kTileBytes, &mapG, 0, y, &bars->full[s]);
+                // read once, and nothing of it is wanted again: asked to leave L2 first, so that the tiles kept for the
+                // pieces that start later are not pushed out by this stream
+                tma_load_2d(true, st, &mapQ, 0, y, &bars->full[s], pol_stream);
+                tma_load_2d(true, st + kTileBytes, &mapK, 0, y, &bars->full[s], pol_stream);
+                tma_load_2d(true, st + 2 * kTileBytes, &mapV, 0, y, &bars->full[s], pol_stream);
+                tma_load_2d(true, st + 3 * kTileBytes, &mapG, 0, y, &bars->full[s], pol_stream);
             }
         }
     } else if (warp >= 17) {

@@ -127,7 +127,29 @@ struct CausalPlan {
         const int b = piece_begin(k), len = piece_begin(k + 1) - b;
         return b + i * (len / sub) + (i < len % sub ? i : len % sub);
     }
+    // is chunk g of the sequence among the last `keep` chunks of its piece?  (the reverse sweep starts there: those
+    // tiles are asked to stay in L2 by the kernels that read them shortly before it)
+    __host__ __device__ bool in_piece_tail(int g, int keep) const {
+        for (int k = 1; k <= npieces(); ++k) {
+            const int e = piece_begin(k);
+            if (g < e) return g >= e - keep;
+        }
+        return false;
+    }
+    // ... or among its first `keep` chunks (where the forward sweeps start)?
+    __host__ __device__ bool in_piece_head(int g, int keep) const {
+        for (int k = 0; k < npieces(); ++k) {
+            const int b = piece_begin(k);
+            if (g >= b && g < b + keep) return true;
+        }
+        return false;
+    }
 };
+
+// Chunks at the end of every piece whose tiles the forward sweep of the backward pass and the reverse pre-pass ask
+// L2 to keep for the reverse sweep (192 pieces x 7 chunks x 64 KB = 86 MB of the 126 MB L2 at the benchmark
+// shape); every other tile of those kernels is read once and asked to leave first.
+constexpr int kKeepTailChunks = 7;
 
 CausalPlan choose_plan(const la_problem& p);
 

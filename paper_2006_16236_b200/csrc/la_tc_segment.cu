@@ -109,6 +109,10 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     if (warp == 4) {
         if (lane == 0) {
             prefetch_tensormap(&mapX); prefetch_tensormap(&mapY);
+            // a pre-pass reads what a sweep reads next: the tiles that sweep starts with (the end of every piece for the
+            // reverse sweep, the beginning for a forward sweep) are asked to stay in L2, everything else, read once
+            // here, to leave first
+            const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
             #pragma unroll 1
             for (int c = 0; c < L; ++c) {
                 const int s = c % kSumStages;
@@ -121,8 +125,11 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
                 const int y = (int)(row0 + (int64_t)c * kChunk);
                 LA_TRACE(g_trace_seg, c, 2);
                 mbar_arrive_expect_tx(&bars->full[s], 2 * kTileBytes);
-                tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
-                tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
+                const bool wanted_soon = scaled ? prm.plan.in_piece_tail(c_begin + c, kKeepTailChunks)
+                                                : prm.plan.in_piece_head(c_begin + c, kKeepTailChunks);
+                const uint64_t pol = wanted_soon ? pol_keep : pol_stream;
+                tma_load_2d(true, st, &mapX, 0, y, &bars->full[s], pol);
+                tma_load_2d(true, st + kTileBytes, &mapY, 0, y, &bars->full[s], pol);
             }
         }
     } else if (warp == 5) {
