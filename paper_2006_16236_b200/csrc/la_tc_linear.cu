@@ -585,23 +585,23 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 uint32_t yv[4][4];
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) lds128(rowX + kTileBytes + (((hf * 4 + cc) ^ r7) << 4), yv[cc]);
-                float p4[4] = {0.f, 0.f, 0.f, 0.f};
+                // (two columns per instruction from here on: the epilogue is bound by instruction issue)
+                f32x2 p4[4] = {0, 0, 0, 0};
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        p4[j] = fmaf(bf16_lo(yv[cc][j]), nuH[cc * 8 + 2 * j], fmaf(bf16_hi(yv[cc][j]), nuH[cc * 8 + 2 * j + 1], p4[j]));
-                ynu_h = (p4[0] + p4[1]) + (p4[2] + p4[3]);
+                    for (int j = 0; j < 4; ++j) p4[j] = fma2(pair_bf16(yv[cc][j]), pair_ld(nuH + cc * 8 + 2 * j), p4[j]);
+                ynu_h = pair_sum(add2(add2(p4[0], p4[1]), add2(p4[2], p4[3])));
             }
             mbar_arrive(&bars->empty[s]);
-            float sx4[4] = {0.f, 0.f, 0.f, 0.f}, xa4[4] = {0.f, 0.f, 0.f, 0.f};
+            f32x2 sx4[4] = {0, 0, 0, 0}, xa4[4] = {0, 0, 0, 0};
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const float x0 = bf16_lo(xv[cc][j]), x1 = bf16_hi(xv[cc][j]);
-                    sx4[j] += x0 + x1;
-                    xa4[j] = fmaf(x0, aH[cc * 8 + 2 * j], fmaf(x1, aH[cc * 8 + 2 * j + 1], xa4[j]));
+                    const f32x2 x2 = pair_bf16(xv[cc][j]);
+                    sx4[j] = add2(sx4[j], x2);
+                    xa4[j] = fma2(x2, pair_ld(aH + cc * 8 + 2 * j), xa4[j]);
                 }
             if (!mbar_wait(&bars->acc_full[b], (c >> 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             tc_fence_after_sync();
@@ -611,23 +611,23 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             tmem_ld_wait();
             float sh_h = 0.f, qh_h = 0.f;
             if (kMode == kApplyBackwardQ) {
-                float sh4[4] = {0.f, 0.f, 0.f, 0.f}, qh4[4] = {0.f, 0.f, 0.f, 0.f};
+                f32x2 sh4[4] = {0, 0, 0, 0}, qh4[4] = {0, 0, 0, 0};
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const float h0 = __uint_as_float(acc[cc * 8 + 2 * j]), h1 = __uint_as_float(acc[cc * 8 + 2 * j + 1]);
-                        sh4[j] += h0 + h1;
-                        qh4[j] = fmaf(bf16_lo(xv[cc][j]), h0, fmaf(bf16_hi(xv[cc][j]), h1, qh4[j]));
+                        const f32x2 h2 = pair(acc[cc * 8 + 2 * j], acc[cc * 8 + 2 * j + 1]);
+                        sh4[j] = add2(sh4[j], h2);
+                        qh4[j] = fma2(pair_bf16(xv[cc][j]), h2, qh4[j]);
                     }
-                sh_h = (sh4[0] + sh4[1]) + (sh4[2] + sh4[3]);
-                qh_h = (qh4[0] + qh4[1]) + (qh4[2] + qh4[3]);
+                sh_h = pair_sum(add2(add2(sh4[0], sh4[1]), add2(sh4[2], sh4[3])));
+                qh_h = pair_sum(add2(add2(qh4[0], qh4[1]), add2(qh4[2], qh4[3])));
             }
             // the pair's previous slab must have left the staging tile before either warp rewrites it below
             if (hf == 0 && lane == 0) tma_store_wait_read<0>();
             if (tid == 0) LA_TRACE(g_trace_lin, c, 10);
-            mine[0] = (sx4[0] + sx4[1]) + (sx4[2] + sx4[3]);
-            mine[1] = (xa4[0] + xa4[1]) + (xa4[2] + xa4[3]);
+            mine[0] = pair_sum(add2(add2(sx4[0], sx4[1]), add2(sx4[2], sx4[3])));
+            mine[1] = pair_sum(add2(add2(xa4[0], xa4[1]), add2(xa4[2], xa4[3])));
             mine[2] = ynu_h;
             mine[3] = sh_h;
             mine[4] = qh_h;
@@ -646,14 +646,15 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 const float inv = 1.f / (den + prm.eps);
                 const float w = x1sum * inv;
                 if (hf == 0 && prm.den) prm.den[row] = padded ? 0.f : den;
+                const f32x2 inv2 = pair(inv, inv), w2 = pair(w, w);
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
-                    const float* nu = nuH + cc * 8;
-                    sts128(out_row + (((hf * 4 + cc) ^ r7) << 4),
-                           pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 0]), inv, w * nu[0]), fmaf(__uint_as_float(acc[cc * 8 + 1]), inv, w * nu[1])),
-                           pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 2]), inv, w * nu[2]), fmaf(__uint_as_float(acc[cc * 8 + 3]), inv, w * nu[3])),
-                           pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 4]), inv, w * nu[4]), fmaf(__uint_as_float(acc[cc * 8 + 5]), inv, w * nu[5])),
-                           pack_bf16x2(fmaf(__uint_as_float(acc[cc * 8 + 6]), inv, w * nu[6]), fmaf(__uint_as_float(acc[cc * 8 + 7]), inv, w * nu[7])));
+                    uint32_t outp[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)     // acc * inv + w * nu
+                        outp[j] = pack_bf16x2(fma2(pair(acc[cc * 8 + 2 * j], acc[cc * 8 + 2 * j + 1]), inv2,
+                                                   mul2(w2, pair_ld(nuH + cc * 8 + 2 * j))));
+                    sts128(out_row + (((hf * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
                 }
             } else {
                 // backward Q:  h = (G.nu) 1 + h'',  Z = N 1 + Z',  gq = (h - (q.h / dn) Z) / dn
@@ -672,11 +673,12 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     if (c > 0 && !mbar_wait(&bars->xs_free, (c - 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
                     const float wq = padded ? 0.f : scale, dq = padded ? 0.f : dl;
                     uint8_t* xs_row = smem + kApOffXS + t * 128;
+                    const f32x2 wq2 = pair(wq, wq);
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc)
                         sts128(xs_row + (((hf * 4 + cc) ^ r7) << 4),
-                               pack_bf16x2(bf16_lo(xv[cc][0]) * wq, bf16_hi(xv[cc][0]) * wq), pack_bf16x2(bf16_lo(xv[cc][1]) * wq, bf16_hi(xv[cc][1]) * wq),
-                               pack_bf16x2(bf16_lo(xv[cc][2]) * wq, bf16_hi(xv[cc][2]) * wq), pack_bf16x2(bf16_lo(xv[cc][3]) * wq, bf16_hi(xv[cc][3]) * wq));
+                               pack_bf16x2(mul2(pair_bf16(xv[cc][0]), wq2)), pack_bf16x2(mul2(pair_bf16(xv[cc][1]), wq2)),
+                               pack_bf16x2(mul2(pair_bf16(xv[cc][2]), wq2)), pack_bf16x2(mul2(pair_bf16(xv[cc][3]), wq2)));
                     if (hf == 0) {
                         uint8_t* aux_row = smem + kApOffAux + t * 128;
                         const uint32_t dd = pack_bf16x2(dq, dq), ww = pack_bf16x2(wq, wq);
@@ -695,34 +697,31 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                     c1 = ynu + sScal[1];
                     cz = 1.f;
                 }
+                const f32x2 scale2 = pair(scale, scale), cz2 = pair(cz, cz), c12 = pair(c1, c1), one2 = pair(1.f, 1.f);
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     uint32_t outp[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const int e = cc * 8 + 2 * j;
-                        float g0 = scale * (fmaf(cz, aH[e], __uint_as_float(acc[e])) + c1);
-                        float g1 = scale * (fmaf(cz, aH[e + 1], __uint_as_float(acc[e + 1])) + c1);
-                        if (elu) {          // phi'(x) from x' = elu(x): 1 where x' > 0, else 1 + x'
-                            const float x0 = bf16_lo(xv[cc][j]), x1 = bf16_hi(xv[cc][j]);
-                            g0 *= x0 > 0.f ? 1.f : 1.f + x0;
-                            g1 *= x1 > 0.f ? 1.f : 1.f + x1;
-                        }
-                        outp[j] = pack_bf16x2(g0, g1);
+                        f32x2 g2 = mul2(scale2, add2(fma2(cz2, pair_ld(aH + e), pair(acc[e], acc[e + 1])), c12));
+                        // phi'(x) from x' = elu(x): 1 where x' > 0, else 1 + x', i.e. 1 + min(x', 0)
+                        if (elu) g2 = mul2(g2, add2(pair_bf16(min_bf16x2(xv[cc][j], 0u)), one2));
+                        outp[j] = pack_bf16x2(g2);
                     }
                     sts128(out_row + (((hf * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
                 }
                 if (kMode == kApplyBackwardKV) {
                     tmem_ld32(tmem + lane_base + b * 128 + 64 + hf * 32, acc);
                     tmem_ld_wait();
+                    const f32x2 xs2 = pair(x1sum, x1sum);
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {       // gV = (1 + k').1 nu_R + k' R''
-                        const float* nu = nuH + cc * 8;
-                        sts128(out_row + kTileBytes + (((hf * 4 + cc) ^ r7) << 4),
-                               pack_bf16x2(fmaf(x1sum, nu[0], __uint_as_float(acc[cc * 8 + 0])), fmaf(x1sum, nu[1], __uint_as_float(acc[cc * 8 + 1]))),
-                               pack_bf16x2(fmaf(x1sum, nu[2], __uint_as_float(acc[cc * 8 + 2])), fmaf(x1sum, nu[3], __uint_as_float(acc[cc * 8 + 3]))),
-                               pack_bf16x2(fmaf(x1sum, nu[4], __uint_as_float(acc[cc * 8 + 4])), fmaf(x1sum, nu[5], __uint_as_float(acc[cc * 8 + 5]))),
-                               pack_bf16x2(fmaf(x1sum, nu[6], __uint_as_float(acc[cc * 8 + 6])), fmaf(x1sum, nu[7], __uint_as_float(acc[cc * 8 + 7]))));
+                        uint32_t outp[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            outp[j] = pack_bf16x2(fma2(xs2, pair_ld(nuH + cc * 8 + 2 * j), pair(acc[cc * 8 + 2 * j], acc[cc * 8 + 2 * j + 1])));
+                        sts128(out_row + kTileBytes + (((hf * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
                     }
                 }
             }
