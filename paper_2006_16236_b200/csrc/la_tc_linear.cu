@@ -432,9 +432,18 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         }
         __syncthreads();
         const int dim = prm.dim;
-        if (tid < kDim) {               // column tid: mean over the dim real rows; nu = ysum + mu
+        // column sums in two steps (a thread alone would walk its column for a microsecond): four threads per column
+        // take every fourth row, in a fixed order, and leave their partial sums behind the matrix
+        float* sPartial = sF + kDim * kDim + kDim;                                // fp32 [4][64]
+        if (tid < 4 * kDim) {
+            const int col = tid & (kDim - 1), part = tid >> 6;
             float m = 0.f;
-            for (int d = 0; d < dim; ++d) m += sF[d * kDim + tid];
+            for (int d = part; d < dim; d += 4) m += sF[d * kDim + col];
+            sPartial[part * kDim + col] = m;
+        }
+        __syncthreads();
+        if (tid < kDim) {               // column tid: mean over the dim real rows; nu = ysum + mu
+            float m = (sPartial[tid] + sPartial[kDim + tid]) + (sPartial[2 * kDim + tid] + sPartial[3 * kDim + tid]);
             m *= 1.f / dim;
             const float ysum = sNu[tid];
             sNu[tid] = ysum + m;
@@ -447,10 +456,11 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                         prm.state_out[bh * (int64_t)(dim * dim) + d * dim + tid] = sF[d * kDim + tid] + ysum;
             }
         }
-        if (tid == 64) {
-            float z = 0.f;
-            for (int d = 0; d < kDim; ++d) z += sA[d];
-            sScal[0] = z;
+        if (warp == 2) {                // sum of a' (64 values, two per lane, then a butterfly: the same order in every CTA)
+            float z = sA[lane] + sA[lane + 32];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
+            if (lane == 0) sScal[0] = z;
         }
         __syncthreads();
         for (int idx = tid; idx < kDim * kDim / 8; idx += kApThreads) {       // 8 consecutive columns of one row
