@@ -590,6 +590,42 @@ def bench_poly2(la, w, dev, pk, iters=10):
     return out
 
 
+def bench_ragged(la, w, dev, pk, iters=10):
+    """The headline shape as a right-padded ragged batch (lengths uniform in [N/2, N], the mix of a speech batch):
+    forward + backward through the calls that take `lengths`, against the same tensors processed at full length.
+    No saved buffer on either side (the ragged calls do not take one)."""
+    Q, K, V, G = (t.to(dev) for t in draw_qkvg(w.B, w.H, w.N, w.D, w.M, w.seed, w.torch_dtype, w.scale))
+    g = torch.Generator(device="cpu").manual_seed(w.seed + 23)
+    lengths = torch.randint(w.N // 2, w.N + 1, (w.B,), generator=g, dtype=torch.int32)
+    ln = lengths.to(dev)
+    O, den = torch.empty_like(V), torch.empty((w.B, w.H, w.N), device=dev)
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+
+    def ragged():
+        la.la_causal_forward(Q, K, V, lengths=ln, O=O, den=den)
+        la.la_causal_backward(Q, K, V, G, lengths=ln, dQ=dQ, dK=dK, dV=dV)
+
+    def full():
+        la.la_causal_forward(Q, K, V, O=O, den=den)
+        la.la_causal_backward(Q, K, V, G, dQ=dQ, dK=dK, dV=dV)
+
+    out = {"lengths": lengths.tolist(), "real_fraction": round(float(lengths.sum()) / (w.B * w.N), 3)}
+    for name, fn in (("ragged_ms", ragged), ("full_length_ms", full)):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(dev)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        out[name] = round(e0.elapsed_time(e1) / iters, 4)
+    out["real_tokens_per_s"] = round(float(lengths.sum()) / (out["ragged_ms"] * 1e-3), 1)
+    la.la_last_device_status()
+    return out
+
+
 def bench_rff(la, w, dev, pk, iters=10):
     """Random Fourier features (the map the paper's conclusion proposes) and their gradient on the headline
     workload's rows with D = 64 inputs and C = 64 features (what the tensor-core attention kernels take): two
@@ -759,6 +795,7 @@ def main():
         rows[w.name + "_from_state"]["unit"] = "tokens/s"
         rows["feature_map_poly2"] = bench_poly2(la, w, dev, pk)
         rows["feature_map_rff"] = bench_rff(la, w, dev, pk)
+        rows[w.name + "_ragged"] = bench_ragged(la, w, dev, pk)
 
     cpu = None
     if rank == 0 and world == 1 and not args.main_only:
