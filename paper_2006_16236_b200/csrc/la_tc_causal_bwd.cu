@@ -173,8 +173,10 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     __syncthreads();
     tc_fence_after_sync();
     // everything above is private to the CTA; from here on memory of the kernel before this one is touched
-    allow_dependent_launch();
+    // (wait first, then let the next kernel be scheduled: the reverse pre-pass fetches its first tiles before it
+    // waits in turn, which is safe only if everything before this kernel is complete by then)
     grid_dependency_wait();
+    allow_dependent_launch();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
     bool mismatch = false;      // the saved buffer must come from a forward pass with this very plan
@@ -658,9 +660,13 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    // everything above is private to the CTA; from here on memory of the kernel before this one is touched
+    // everything above is private to the CTA; from here on memory of the kernel before this one is touched.  The
+    // kernel before this one (the reverse pre-pass) writes records only, and everything before IT is complete
+    // when this kernel is scheduled (it waits before it lets its successor go): the TMA producer may request
+    // the first tiles, which are inputs of the call, before it waits, so that they arrive while the pre-pass
+    // is still draining.
     allow_dependent_launch();
-    grid_dependency_wait();
+    if (warp != 16) grid_dependency_wait();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
@@ -680,6 +686,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                     break;
                 }
                 if (*abort_flag) break;
+                if (i == kKvStages) grid_dependency_wait();     // (nothing this thread does depends on it: for symmetry)
                 uint8_t* st = smem + kKvOffStage + s * kKvStageBytes;
                 const int y = (int)chunk_row(i);
                 mbar_arrive_expect_tx(&bars->full[s], kKvStageBytes);

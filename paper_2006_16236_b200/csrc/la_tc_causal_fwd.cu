@@ -149,8 +149,13 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     __syncthreads();
     tc_fence_after_sync();
     // everything above is private to the CTA; from here on memory of the kernel before this one is touched
+    // With a pre-pass of the same call before this kernel (it waits for everything before it, then lets this kernel
+    // be scheduled, and writes records only) the TMA producer requests its first tiles, which are inputs of the
+    // call, before it waits: they arrive while the pre-pass drains.  Without one this may be the first kernel of
+    // the call, and everybody waits first.
     allow_dependent_launch();
-    grid_dependency_wait();
+    const bool early_loads = prm.init != nullptr && warp == 16;
+    if (!early_loads) grid_dependency_wait();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
@@ -158,6 +163,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             if (prm.stamp && blockIdx.x == 0) {
+                grid_dependency_wait();         // a write to global memory: after the wait
                 int st[kPlanStampInts];
                 plan_stamp(plan, prm.dim, st);
 #pragma unroll
@@ -172,6 +178,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     break;
                 }
                 if (*abort_flag) break;
+                if (early_loads && c == kStages) grid_dependency_wait();    // (nothing this thread does depends on it)
                 uint8_t* st = smem + kOffStage + s * kStageBytes;
                 const int y = (int)(row0 + (int64_t)c * kChunk);
                 mbar_arrive_expect_tx(&bars->full[s], kStageBytes);

@@ -100,8 +100,17 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
     __syncthreads();
     tc_fence_after_sync();
     // everything above is private to the CTA; from here on memory of the kernel before this one is touched
-    allow_dependent_launch();
-    grid_dependency_wait();
+    // wait first, then let the next kernel be scheduled: a kernel that follows this one may then fetch its own
+    // inputs before it waits in turn, knowing that everything before this kernel is complete
+    // The reverse pre-pass follows the dQ sweep of the same call and reads, as tiles, only inputs of that call and
+    // the saved tiles of an earlier one: its TMA producer requests the first tiles before it waits (they arrive
+    // while the sweep before it drains); the per-row scalars of that sweep are read by the other warps, after
+    // their wait.  (The forward pre-pass may be the first kernel of a call: everybody waits first.)
+    const bool early_loads = scaled && warp == 4;
+    if (!early_loads) {
+        grid_dependency_wait();
+        allow_dependent_launch();
+    }
     LA_TRACE_CTA(g_trace_seg, 2);
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
@@ -121,6 +130,10 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
                     break;
                 }
                 if (*abort_flag) break;
+                if (early_loads && c == kSumStages) {
+                    grid_dependency_wait();
+                    allow_dependent_launch();
+                }
                 uint8_t* st = smem + s * kSumStageBytes;
                 const int y = (int)(row0 + (int64_t)c * kChunk);
                 LA_TRACE(g_trace_seg, c, 2);
@@ -131,6 +144,10 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
                 tma_load_2d(true, st, &mapX, 0, y, &bars->full[s], pol);
                 tma_load_2d(true, st + kTileBytes, &mapY, 0, y, &bars->full[s], pol);
             }
+        }
+        if (early_loads && L <= kSumStages) {        // a part of at most three chunks: the loop never got there
+            grid_dependency_wait();
+            allow_dependent_launch();
         }
     } else if (warp == 5) {
         {
