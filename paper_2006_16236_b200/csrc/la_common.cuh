@@ -83,9 +83,11 @@ int launch_poly2_map_backward(const void* x, const void* dy, void* dx, int64_t r
 int launch_recurrent_steps(const la_problem& p, const void* q, const void* k, const void* v,
                            float* S, float* Z, void* out, cudaStream_t st);
 // chained: launch as a programmatic dependent of the kernel before it in the stream (its launch overlaps that
-// kernel's tail; it waits for that kernel before it reads anything)
+// kernel's tail; it waits for that kernel before it reads anything).  early_state (with chained, D = M = 64):
+// the state is read before that wait; only for a caller whose kernel in front belongs to the same call, leaves
+// the state alone, and itself waits before it lets this one be scheduled.
 int launch_recurrent_step(const la_problem& p, const void* q, const void* k, const void* v,
-                          float* S, float* Z, void* out, cudaStream_t st, bool chained = false);
+                          float* S, float* Z, void* out, cudaStream_t st, bool chained = false, bool early_state = false);
 
 // Decode step of a whole attention sublayer (projections + recurrent step + output projection), bf16, D = M = 64
 bool decode_layer_supported(const la_problem& p);

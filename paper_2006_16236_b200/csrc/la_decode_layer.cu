@@ -36,6 +36,7 @@ struct GemmParams {
     const __nv_bfloat16* res;   // residual [rows][out_cols] added in the epilogue, or null
     int* status;
     int rows, kblocks, out_cols;
+    int early_w;                // the weight tiles of the first ring are requested before the dependency wait
 };
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
@@ -64,15 +65,29 @@ projection_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    // everything above is private to the CTA; from here on memory of the kernel before this one is touched
-    allow_dependent_launch();
+    // Everything above is private to the CTA; from here on memory of the kernel before this one is touched.
+    // Every thread waits for that kernel and only then lets the next one be scheduled (a kernel behind this one
+    // may read, before its own wait, what no kernel of the call writes: by then everything older is complete).
+    // With early_w (the output projection: its weights are written by no kernel of the call and the kernels in
+    // front of it kept that order) the producer requests the weight tiles of the first ring before it waits.
+    const bool early_w = prm.early_w != 0 && warp == 4 && lane == 0;
+    const int ring = min(prm.kblocks, kGemmStages);
+    if (early_w) {
+        prefetch_tensormap(&mapW);
+        for (int kb = 0; kb < ring; ++kb) {
+            mbar_arrive_expect_tx(&bars->full[kb], kGemmStageBytes);
+            tma_load_2d(smem + kb * kGemmStageBytes + kTileBytes, &mapW, kb * kDim, n0, &bars->full[kb]);
+        }
+    }
     grid_dependency_wait();
+    allow_dependent_launch();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
 
     if (warp == 4) {
         if (lane == 0) {
-            prefetch_tensormap(&mapA); prefetch_tensormap(&mapW);
+            prefetch_tensormap(&mapA);
+            if (!early_w) prefetch_tensormap(&mapW);
             #pragma unroll 1
             for (int kb = 0; kb < prm.kblocks; ++kb) {
                 const int s = kb % kGemmStages;
@@ -81,9 +96,10 @@ projection_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
                     break;
                 }
                 uint8_t* st = smem + s * kGemmStageBytes;
-                mbar_arrive_expect_tx(&bars->full[s], kGemmStageBytes);
+                const bool w_requested = early_w && kb < ring;
+                if (!w_requested) mbar_arrive_expect_tx(&bars->full[s], kGemmStageBytes);
                 tma_load_2d(st, &mapA, kb * kDim, row0, &bars->full[s]);               // rows past the end read as zeros
-                tma_load_2d(st + kTileBytes, &mapW, kb * kDim, n0, &bars->full[s]);
+                if (!w_requested) tma_load_2d(st + kTileBytes, &mapW, kb * kDim, n0, &bars->full[s]);
             }
         }
     } else if (warp == 5) {
@@ -148,7 +164,7 @@ projection_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
 
 // C[rows][n] = A[rows][K] W[n][K]^T (+ res): n = n_out * out_cols columns in all, written to out[0..n_out-1]
 int projection_gemm(const void* A, const void* W, int rows, int K, int n_out, int out_cols, __nv_bfloat16* const* out,
-                    const void* res, cudaStream_t st) {
+                    const void* res, bool early_w, cudaStream_t st) {
     CUtensorMap mA, mW;
     if (int rc = encode_tile_map(&mA, A, (uint64_t)rows, kChunk, K)) return rc;
     if (int rc = encode_tile_map(&mW, W, (uint64_t)n_out * out_cols, kGemmTileN, K)) return rc;
@@ -162,6 +178,7 @@ int projection_gemm(const void* A, const void* W, int rows, int K, int n_out, in
     prm.rows = rows;
     prm.kblocks = K / kDim;
     prm.out_cols = out_cols;
+    prm.early_w = early_w ? 1 : 0;
     prof_begin(kProfProjection, st);
     cudaLaunchAttribute attr;
     cudaLaunchConfig_t cfg = chained_launch((unsigned)(n_out * out_cols / kGemmTileN), kGemmThreads, kGemmSmemBytes, st, &attr);
@@ -188,10 +205,12 @@ int decode_layer_step(const la_problem& p, const void* x, const void* Wqkv, cons
     __nv_bfloat16* q = (__nv_bfloat16*)ws;
     __nv_bfloat16* qkv[3] = {q, q + (size_t)B * F, q + 2 * (size_t)B * F};
     __nv_bfloat16* a = q + 3 * (size_t)B * F;
-    if (int rc = tc::projection_gemm(x, Wqkv, B, F, 3, F, qkv, nullptr, st)) return rc;
-    if (int rc = launch_recurrent_step(p, qkv[0], qkv[1], qkv[2], S, Z, a, st, /*chained=*/true)) return rc;
+    // The first kernel of the call waits for everything before it; the two behind it start on what no kernel of
+    // the call writes (the state, the output weights) while the kernel in front of them still runs.
+    if (int rc = tc::projection_gemm(x, Wqkv, B, F, 3, F, qkv, nullptr, /*early_w=*/false, st)) return rc;
+    if (int rc = launch_recurrent_step(p, qkv[0], qkv[1], qkv[2], S, Z, a, st, /*chained=*/true, /*early_state=*/true)) return rc;
     __nv_bfloat16* yy[1] = {(__nv_bfloat16*)y};
-    return tc::projection_gemm(a, Wo, B, F, 1, F, yy, x, st);
+    return tc::projection_gemm(a, Wo, B, F, 1, F, yy, x, /*early_w=*/true, st);
 }
 
 }  // namespace la

@@ -157,7 +157,11 @@ int launch_poly2_map_backward(const void* x, const void* dy, void* dx, int64_t r
 // else is waited on.  phi(q)^T S is reduced with warp shuffles and one shared
 // memory hop across the four warps; phi(q)^T Z likewise.
 // ---------------------------------------------------------------------------
-template <typename T, int D, int M>
+// kEarlyState (the decode layer's use only): the state is read BEFORE the dependency wait.  The kernel in
+// front is then the projection of the same call, which never touches the state, waited for everything before it
+// and only then let this kernel be scheduled, so the last writer of the state has completed: the state, which
+// is all the traffic of this kernel, streams in while that projection runs.
+template <typename T, int D, int M, bool kEarlyState = false>
 __global__ void __launch_bounds__(128)
 recurrent_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                       float* __restrict__ S, float* __restrict__ Z, T* __restrict__ out,
@@ -178,13 +182,18 @@ recurrent_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T*
 
     // When launched as a programmatic dependent of the kernel before it in the stream (the decode layer does
     // that), this is where that kernel's results become visible; in an ordinary launch both are no-ops.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
     float4* Sp = reinterpret_cast<float4*>(S + bh * (int64_t)(D * M));
     float4 s[PASSES];
+    if (kEarlyState) {
 #pragma unroll
-    for (int p = 0; p < PASSES; ++p) s[p] = Sp[(r0 + p * RPP) * TPR + c4];
+        for (int p = 0; p < PASSES; ++p) s[p] = Sp[(r0 + p * RPP) * TPR + c4];
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!kEarlyState) {
+#pragma unroll
+        for (int p = 0; p < PASSES; ++p) s[p] = Sp[(r0 + p * RPP) * TPR + c4];
+    }
 
     float zq = 0.f;
     if (tid < D) {
@@ -435,11 +444,11 @@ int launch_recurrent_steps(const la_problem& p, const void* q, const void* k, co
 
 template <typename T>
 static int recurrent_dispatch(const la_problem& p, const void* q, const void* k, const void* v,
-                              float* S, float* Z, void* out, cudaStream_t st, bool chained) {
+                              float* S, float* Z, void* out, cudaStream_t st, bool chained, bool early_state) {
     const unsigned grid = (unsigned)(p.B * p.H);
     const T *qq = (const T*)q, *kk = (const T*)k, *vv = (const T*)v;
     T* oo = (T*)out;
-    if (chained && p.D == 64 && p.M == 64) {        // between the two projections of a decode layer: see the kernel
+    if (chained && p.D == 64 && p.M == 64) {        // a programmatic dependent of the kernel before it: see the kernel
         cudaLaunchAttribute attr;
         attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr.val.programmaticStreamSerializationAllowed = 1;
@@ -449,7 +458,8 @@ static int recurrent_dispatch(const la_problem& p, const void* q, const void* k,
         cfg.stream = st;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
-        LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, recurrent_step_kernel<T, 64, 64>, qq, kk, vv, S, Z, oo, p.eps, p.phi));
+        if (early_state) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, recurrent_step_kernel<T, 64, 64, true>, qq, kk, vv, S, Z, oo, p.eps, p.phi));
+        else LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, recurrent_step_kernel<T, 64, 64>, qq, kk, vv, S, Z, oo, p.eps, p.phi));
         note_launch();
         return LA_OK;
     }
@@ -469,10 +479,10 @@ static int recurrent_dispatch(const la_problem& p, const void* q, const void* k,
 }
 
 int launch_recurrent_step(const la_problem& p, const void* q, const void* k, const void* v,
-                          float* S, float* Z, void* out, cudaStream_t st, bool chained) {
+                          float* S, float* Z, void* out, cudaStream_t st, bool chained, bool early_state) {
     prof_begin(kProfRecurrent, st);
-    const int rc = p.dtype == LA_F32 ? recurrent_dispatch<float>(p, q, k, v, S, Z, out, st, chained)
-                                     : recurrent_dispatch<__nv_bfloat16>(p, q, k, v, S, Z, out, st, chained);
+    const int rc = p.dtype == LA_F32 ? recurrent_dispatch<float>(p, q, k, v, S, Z, out, st, chained, early_state)
+                                     : recurrent_dispatch<__nv_bfloat16>(p, q, k, v, S, Z, out, st, chained, early_state);
     prof_end(kProfRecurrent, st);
     return rc;
 }

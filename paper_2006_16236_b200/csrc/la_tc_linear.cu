@@ -155,9 +155,11 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     tc_fence_after_sync();
     const uint32_t tmem = bars->tmem_base;
     volatile int* abort_flag = &bars->abort_flag;
-    // everything above is private to the CTA; from here on memory of the kernel before this one is touched
-    allow_dependent_launch();
+    // everything above is private to the CTA; from here on memory of the kernel before this one is touched.
+    // (Wait first, then let the next kernel be scheduled: an apply kernel behind this one requests its first
+    // tiles before it waits in turn, which is safe only if everything before this kernel is complete by then.)
     grid_dependency_wait();
+    allow_dependent_launch();
     LA_TRACE_CTA(g_trace_lin, 1);
     // Ragged batch: only `real` rows of this split exist; chunks behind them are skipped and the rows behind
     // them in the last chunk are zeroed after the load (at least one chunk runs, so that the record is written
@@ -322,6 +324,7 @@ struct ApParams {
     float eps;
     int phi;
     int dim;                    // D = M: 64, or 32 (tiles zero-padded to 64 columns)
+    int early;                  // a kernel of the same call runs in front: the first tiles are requested before the wait
 };
 
 template <int kMode>
@@ -371,8 +374,14 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     }
     __syncthreads();            // the barriers are initialised for the loads issued before the prologue below
     // (set-up above is private to the CTA; the records below come from the kernel before this one)
-    allow_dependent_launch();
-    grid_dependency_wait();
+    // The tiles of this pass are inputs of the call.  Behind another kernel of the same call (which waited for
+    // everything before it and only then let this one be scheduled) the first of them are requested before the
+    // wait and arrive while that kernel drains; as the first kernel of a call everything waits first.
+    const bool early = prm.early != 0;
+    if (!early) {
+        grid_dependency_wait();
+        allow_dependent_launch();
+    }
     // Ragged batch: `len` positions of this sequence exist, `real` of them in this split.  Only the chunks that
     // hold real rows go through the pipeline; the padding behind them is filled with zeros at the end.
     int64_t len = prm.N, real = (int64_t)L_all * kChunk;
@@ -394,6 +403,10 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         prefetch_tensormap(&mapX);
         if (kHasY) prefetch_tensormap(&mapY);
         for (int c = 0; c < min(L, kApStages); ++c) issue_load(c);
+    }
+    if (early) {
+        grid_dependency_wait();
+        allow_dependent_launch();
     }
     // state of this head: add the split records (fp32), remove the column means, round the
     // centred remainder to a bf16 operand tile.  Scratch: the output staging tiles, free until the first epilogue.
@@ -900,6 +913,7 @@ int linear_forward(const la_problem& p, const void* Q, const void* K, const void
     a.den = den;
     a.state_out = KV;
     a.vec_out = Zs;
+    a.early = 1;                // behind the sum kernel
     return launch_apply<kApplyForward>(p, sg, mQ, mQ, a, st);
 }
 
@@ -920,6 +934,7 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
     if (saved) rec_s = (float*)saved;         // the forward's own records: nothing to recompute
     else if (int rc = launch_sums(p, sg, mK, mV, lengths, rec_s, st)) return rc;
     ApParams a = {};
+    a.early = saved ? 0 : 1;    // the first kernel of the call with saved records, else behind the sum kernel
     a.lengths = lengths;
     a.records = rec_s;
     a.out0 = (__nv_bfloat16*)dQ;
@@ -930,6 +945,7 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
     b.records = rec_r;
     b.out0 = (__nv_bfloat16*)dK;
     b.out1 = (__nv_bfloat16*)dV;
+    b.early = 1;                // behind the dQ pass
     return launch_apply<kApplyBackwardKV>(p, sg, mK, mV, b, st);
 }
 
