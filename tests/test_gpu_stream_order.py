@@ -1,0 +1,94 @@
+"""Stream order around the calls: what a kernel enqueued just before a call wrote is what the call reads.
+
+The kernels of one call follow each other as programmatic dependents, and several of them request
+their first tiles (or read the decode state) before they wait for the kernel in front of them.
+That is only right if everything enqueued BEFORE the call is complete by then.  Here the inputs
+of every call are rewritten in the stream immediately before it (long copies, no host
+synchronisation anywhere, two alternating sets of values, so that stale data would be the other
+set's), and every result has to be bit-identical to the one of a fully synchronised run.
+"""
+import pytest
+import torch
+
+import paper_2006_16236_b200 as la
+from paper_2006_16236_b200.inputs import WORKLOADS, draw_workload
+
+pytestmark = pytest.mark.gpu
+DEV = torch.device("cuda")
+
+
+def _calls(kind):
+    if kind == "causal":
+        return la.la_causal_forward, la.la_causal_backward, la.saved_buffer
+    return la.la_linear_attention, la.la_linear_attention_backward, la.linear_saved_buffer
+
+
+@pytest.mark.parametrize("keep", [False, True], ids=["recompute", "saved"])
+@pytest.mark.parametrize("name", ["causal_sweep_bf16_N16384", "causal_sweep_bf16_N65536", "noncausal_bf16_speech"])
+def test_inputs_written_in_stream_just_before_a_call_are_seen(name, keep):
+    w = WORKLOADS[name]
+    fwd, bwd, make_saved = _calls(w.kind)
+    set_a = [t.to(DEV) for t in draw_workload(w)]
+    set_b = [(t.flip(2) * 0.75).contiguous() for t in set_a]            # other values at every position
+    Q, K, V, G = (torch.empty_like(t) for t in set_a)
+    O, dQ, dK, dV = torch.empty_like(V), torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    saved = make_saved(Q, V) if keep else None
+    kw = {"saved": saved} if keep else {}
+
+    def run(src, synced):
+        def gap():
+            if synced:
+                torch.cuda.synchronize()
+        Q.copy_(src[0]); K.copy_(src[1]); V.copy_(src[2]); gap()
+        fwd(Q, K, V, O=O, **kw); gap()
+        G.copy_(src[3]); gap()
+        bwd(Q, K, V, G, dQ=dQ, dK=dK, dV=dV, **kw); gap()
+        return [t.clone() for t in (O, dQ, dK, dV)]
+
+    want = {0: run(set_a, True), 1: run(set_b, True)}
+    assert not torch.equal(want[0][0], want[1][0])
+    torch.cuda.synchronize()
+    got = [(i & 1, run(set_b if i & 1 else set_a, False)) for i in range(6)]
+    torch.cuda.synchronize()
+    la.la_last_device_status()
+    for i, (which, res) in enumerate(got):
+        for a, b, nm in zip(want[which], res, ("O", "dQ", "dK", "dV")):
+            assert torch.equal(a, b), f"{name}: {nm} of unsynchronised repeat {i} differs from the synchronised run"
+
+
+def test_decode_layer_fed_back_on_the_device_without_synchronisation():
+    """Generation loop on the device: the next input is made from the previous output by ordinary stream-ordered
+    kernels; the step kernel reads the state, and the output projection its weights, before waiting for the
+    kernel in front of them.  Same bits as with a host synchronisation after every operation."""
+    B, H, D, T = 256, 8, 64, 24
+    F = H * D
+    g = torch.Generator().manual_seed(5)
+    s = 1.0 / F ** 0.5
+    Wqkv = (torch.randn((3 * F, F), generator=g) * s).to(torch.bfloat16).to(DEV)
+    Wo = (torch.randn((F, F), generator=g) * s).to(torch.bfloat16).to(DEV)
+    x0 = torch.randn((B, F), generator=g).to(torch.bfloat16).to(DEV)
+
+    def run(synced):
+        S = torch.zeros((B, H, D, D), device=DEV)
+        Z = torch.zeros((B, H, D), device=DEV)
+        x, ys = x0.clone(), []
+        for t in range(T):
+            y = la.la_decode_layer_step(x, Wqkv, Wo, S, Z)
+            if synced:
+                torch.cuda.synchronize()
+            ys.append(y)
+            x = torch.tanh(y.float()).to(torch.bfloat16)
+            if t == T // 2:
+                S.mul_(0.5)         # the state rewritten in the stream between two calls
+                Z.mul_(0.5)
+            if synced:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        return ys, S, Z
+
+    ys1, S1, Z1 = run(True)
+    ys2, S2, Z2 = run(False)
+    la.la_last_device_status()
+    for t, (a, b) in enumerate(zip(ys1, ys2)):
+        assert torch.equal(a, b), f"token {t}"
+    assert torch.equal(S1, S2) and torch.equal(Z1, Z2)
