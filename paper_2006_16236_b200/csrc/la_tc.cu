@@ -44,11 +44,12 @@ int sm_count() {
 namespace {
 struct MapKey {
     const void* base;
-    uint64_t rows;
+    uint64_t rows;          // 2-D map: rows in all; 3-D map: positions per sequence
+    uint64_t seqs;          // 3-D map: sequences; 0 for a 2-D map
     uint32_t box_rows;
     int cols, dev;
     bool operator==(const MapKey& o) const {
-        return base == o.base && rows == o.rows && box_rows == o.box_rows && cols == o.cols && dev == o.dev;
+        return base == o.base && rows == o.rows && seqs == o.seqs && box_rows == o.box_rows && cols == o.cols && dev == o.dev;
     }
 };
 constexpr int kMapCache = 32;
@@ -61,18 +62,18 @@ struct MapCache {
 thread_local MapCache g_maps = {};
 }  // namespace
 
-static int encode_tile_map_uncached(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols);
+static int encode_tile_map_uncached(CUtensorMap* map, const void* base, uint64_t seqs, uint64_t rows, uint32_t box_rows, int cols);
 
-int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols) {
+static int encode_cached(CUtensorMap* map, const void* base, uint64_t seqs, uint64_t rows, uint32_t box_rows, int cols) {
     int dev = 0;
     LA_CUDA_TRY(cudaGetDevice(&dev));
-    const MapKey key{base, rows, box_rows, cols, dev};
+    const MapKey key{base, rows, seqs, box_rows, cols, dev};
     for (int i = 0; i < kMapCache; ++i)
         if (g_maps.used[i] && g_maps.key[i] == key) {
             *map = g_maps.map[i];
             return LA_OK;
         }
-    if (int rc = encode_tile_map_uncached(map, base, rows, box_rows, cols)) return rc;
+    if (int rc = encode_tile_map_uncached(map, base, seqs, rows, box_rows, cols)) return rc;
     const int slot = g_maps.next;
     g_maps.next = (slot + 1) % kMapCache;
     g_maps.key[slot] = key;
@@ -81,7 +82,16 @@ int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t 
     return LA_OK;
 }
 
-static int encode_tile_map_uncached(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols) {
+int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols) {
+    return encode_cached(map, base, 0, rows, box_rows, cols);
+}
+int encode_seq_tile_map(CUtensorMap* map, const void* base, uint64_t seqs, uint64_t n, uint32_t box_rows, int cols) {
+    return encode_cached(map, base, seqs, n, box_rows, cols);
+}
+
+// seqs == 0: a 2-D map over [rows][cols]; otherwise a 3-D map over [seqs][rows][cols] whose boxes hold rows of one
+// sequence only (a box that reaches past a sequence's end is filled with zeros on a load and clipped on a store)
+static int encode_tile_map_uncached(CUtensorMap* map, const void* base, uint64_t seqs, uint64_t rows, uint32_t box_rows, int cols) {
     static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     if (!encode) {
         void* fn = nullptr;
@@ -91,11 +101,11 @@ static int encode_tile_map_uncached(CUtensorMap* map, const void* base, uint64_t
             return fail(LA_ERR_CUDA, "the driver does not export cuTensorMapEncodeTiled");
         encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
     }
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kDim, box_rows};
-    const cuuint32_t elem_strides[2] = {1, 1};
-    const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+    const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)seqs};
+    const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * rows};
+    const cuuint32_t box[3] = {(cuuint32_t)kDim, box_rows, 1};
+    const cuuint32_t elem_strides[3] = {1, 1, 1};
+    const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, seqs ? 3 : 2, const_cast<void*>(base), dims, strides, box,
                               elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(LA_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -108,7 +118,7 @@ bool tc_supported(const la_problem& p, int op) {
     static const bool disabled = getenv("LA_DISABLE_TC") != nullptr;
     if (disabled) return false;
     if (p.dtype != LA_BF16 || p.D != p.M || (p.D != 32 && p.D != 64)) return false;
-    if (p.N < tc::kChunk || p.N % tc::kChunk) return false;
+    if (p.N < 1) return false;      // any length: a last chunk that is not full is handled as padding
     if (p.B * p.H * p.N >= (1LL << 31)) return false;          // TMA coordinates are 32-bit
     return op >= LA_OP_LINEAR_FORWARD && op <= LA_OP_CAUSAL_BACKWARD;
 }

@@ -211,16 +211,16 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             }
             if (__any_sync(0xFFFFFFFFu, *abort_flag)) break;
             uint8_t* st = smem + kDqOffStage + s * 4 * kTileBytes;
-            const int y = (int)(row0 + (int64_t)c * kChunk);
+            const int y = (c_begin + c) * kChunk, z = (int)bh;      // position in the sequence; sequence
             if (leader) LA_TRACE(g_trace_dq, c, 13);
             // the reverse sweep starts where this piece ends: its last chunks are asked to stay in L2, the rest,
             // which will be long gone by then, to leave first
             const uint64_t pol = c >= L_full - kKeepTailChunks ? pol_keep : pol_stream;
             mbar_arrive_expect_tx(leader, &bars->full[s], 4 * kTileBytes);
-            tma_load_2d(leader, st + kTileBytes, &mapV, 0, y, &bars->full[s], pol);
-            tma_load_2d(leader, st + 2 * kTileBytes, &mapG, 0, y, &bars->full[s], pol);
-            tma_load_2d(leader, st, &mapK, 0, y, &bars->full[s], pol);
-            tma_load_2d(leader, st + 3 * kTileBytes, &mapQ, 0, y, &bars->full[s], pol);
+            tile_load<kVarlen>(leader, st + kTileBytes, &mapV, y, z, prm.N, &bars->full[s], pol);
+            tile_load<kVarlen>(leader, st + 2 * kTileBytes, &mapG, y, z, prm.N, &bars->full[s], pol);
+            tile_load<kVarlen>(leader, st, &mapK, y, z, prm.N, &bars->full[s], pol);
+            tile_load<kVarlen>(leader, st + 3 * kTileBytes, &mapQ, y, z, prm.N, &bars->full[s], pol);
         }
     } else if (warp >= 13) {
         // ------------------------------------------------------------- MMA issuers
@@ -480,7 +480,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             const float delta = -qg * inv;                  // = -(G_i . O_i)
             const int64_t row = row0 + (int64_t)c * kChunk + t;
             const bool pad = kVarlen && c == L - 1 && t >= tail_rows;     // a padded row of the chunk that holds the sequence's end
-            if (half == 0) {
+            if (half == 0 && !(pad && (int64_t)(c_begin + c) * kChunk + t >= prm.N)) {     // (a padded row may lie past the sequence's N)
                 prm.dn[row] = pad ? 1.f : dn;
                 prm.dl[row] = pad ? 0.f : delta;
             }
@@ -508,7 +508,8 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             fence_proxy_async_smem();
             named_barrier(2 + quad, 64);
             if (half == 0 && lane == 0) {
-                tma_store_2d(&mapDQ, smem + kDqOffOut + quad * 32 * 128, 0, (int)(row0 + (int64_t)c * kChunk + quad * 32));
+                const int y = (c_begin + c) * kChunk + quad * 32;       // rows past the sequence's N are clipped by the store
+                if (!kVarlen || y < prm.N) tile_store<kVarlen>(&mapDQ, smem + kDqOffOut + quad * 32 * 128, y, (int)bh, prm.N);
                 tma_store_commit();
             }
             if (tid == 0) LA_TRACE(g_trace_dq, c, 10);
@@ -522,7 +523,7 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         const int t = (warp & 3) * 32 + lane, half = warp >> 2;
         #pragma unroll 1
         for (int c = L; c < L_full; ++c) {
-            if (half * 32 < prm.dim) {
+            if (half * 32 < prm.dim && (int64_t)(c_begin + c) * kChunk + t < prm.N) {
                 __nv_bfloat16* dst = prm.dQ + (row0 + (int64_t)c * kChunk + t) * prm.dim + half * 32;
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) stg128(dst + cc * 8, 0u, 0u, 0u, 0u);
@@ -615,7 +616,8 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
     const int c_end = c_begin + L;
     const bool idle = kVarlen && L == 0;        // all padding: only the state gradient passes through (warps 8-11)
     // iteration i visits chunk c_end - 1 - i
-    auto chunk_row = [&](int i) { return bh * prm.N + (int64_t)(c_end - 1 - i) * kChunk; };
+    auto chunk_pos = [&](int i) { return (c_end - 1 - i) * kChunk; };               // position of its first row in the sequence
+    auto chunk_row = [&](int i) { return bh * prm.N + (int64_t)chunk_pos(i); };     // the same as a row of the whole tensor
 
     LA_TRACE_CTA(g_trace_dkv, 0);
     if (sbase & 1023u) {            // the swizzled tiles need a 1 KB aligned base: report, touch nothing
@@ -688,14 +690,14 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                 if (*abort_flag) break;
                 if (i == kKvStages) grid_dependency_wait();     // (nothing this thread does depends on it: for symmetry)
                 uint8_t* st = smem + kKvOffStage + s * kKvStageBytes;
-                const int y = (int)chunk_row(i);
+                const int y = chunk_pos(i), z = (int)bh;
                 mbar_arrive_expect_tx(&bars->full[s], kKvStageBytes);
                 // read once, and nothing of it is wanted again: asked to leave L2 first, so that the tiles kept for the
                 // pieces that start later are not pushed out by this stream
-                tma_load_2d(true, st, &mapQ, 0, y, &bars->full[s], pol_stream);
-                tma_load_2d(true, st + kTileBytes, &mapK, 0, y, &bars->full[s], pol_stream);
-                tma_load_2d(true, st + 2 * kTileBytes, &mapV, 0, y, &bars->full[s], pol_stream);
-                tma_load_2d(true, st + 3 * kTileBytes, &mapG, 0, y, &bars->full[s], pol_stream);
+                tile_load<kVarlen>(true, st, &mapQ, y, z, prm.N, &bars->full[s], pol_stream);
+                tile_load<kVarlen>(true, st + kTileBytes, &mapK, y, z, prm.N, &bars->full[s], pol_stream);
+                tile_load<kVarlen>(true, st + 2 * kTileBytes, &mapV, y, z, prm.N, &bars->full[s], pol_stream);
+                tile_load<kVarlen>(true, st + 3 * kTileBytes, &mapG, y, z, prm.N, &bars->full[s], pol_stream);
             }
         }
     } else if (warp >= 17) {
@@ -812,8 +814,9 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         for (int i = 0; i < L; ++i) {
             const int s = i % kKvStages;
             const int64_t row = chunk_row(i) + t;
-            const float inv = 1.f / __ldg(prm.dn + row);
-            const float delta = __ldg(prm.dl + row);
+            const bool pad = kVarlen && i == 0 && t >= tail_rows;       // (a padded row may lie past the sequence's N)
+            const float inv = pad ? 1.f : 1.f / __ldg(prm.dn + row);
+            const float delta = pad ? 0.f : __ldg(prm.dl + row);
             if (!mbar_wait(&bars->full[s], (i / kKvStages) & 1, prm.status, kStatusTmaTimeout)) { *abort_flag = 1; break; }
             if (*abort_flag) break;
             if (t == 0) LA_TRACE(g_trace_dkv, i, 5);
@@ -826,7 +829,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             if (i >= 1 && !mbar_wait(&bars->r_full, (i - 1) & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
             if (t == 0) LA_TRACE(g_trace_dkv, i, 15);
             // dl_i as a bf16 high and low part in columns 0 and 1 (the rest of the row stays zero)
-            if (kVarlen && i == 0 && t >= tail_rows) {          // padding: the row takes no part in any product
+            if (pad) {                                          // padding: the row takes no part in any product
                 zero_row(rowQ);
                 zero_row(rowQ + kTileBytes);
                 zero_row(rowQ + 2 * kTileBytes);
@@ -905,7 +908,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             fence_proxy_async_smem();
             named_barrier(1, 128);
             if (t == 0) {
-                tma_store_2d(&mapDV, smem + kKvOffStage + s * kKvStageBytes + 3 * kTileBytes, 0, (int)chunk_row(i));
+                tile_store<kVarlen>(&mapDV, smem + kKvOffStage + s * kKvStageBytes + 3 * kTileBytes, chunk_pos(i), (int)bh, prm.N);
                 tma_store_commit();
             }
             if (!mbar_wait(&bars->dkv_full, i & 1, prm.status, kStatusMmaTimeout)) { *abort_flag = 1; break; }
@@ -945,7 +948,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             fence_proxy_async_smem();
             named_barrier(1, 128);          // all dK rows are in the tile; also orders the r double buffer
             if (t == 0) {
-                tma_store_2d(&mapDK, smem + kKvOffStage + s * kKvStageBytes + kTileBytes, 0, (int)chunk_row(i));
+                tile_store<kVarlen>(&mapDK, smem + kKvOffStage + s * kKvStageBytes + kTileBytes, chunk_pos(i), (int)bh, prm.N);
                 tma_store_commit();
                 tma_store_wait_read<0>();           // both tiles have been read: the stage may be refilled
                 mbar_arrive(&bars->empty[s]);
@@ -962,6 +965,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
             #pragma unroll 1
             for (int c = c_end; c < c_begin + L_full; ++c) {
                 const int64_t row = bh * prm.N + (int64_t)c * kChunk + t;
+                if ((int64_t)c * kChunk + t >= prm.N) continue;             // past the sequence: not in memory
                 for (int cc = 0; cc < prm.dim / 8; ++cc) {
                     stg128(prm.dK + row * prm.dim + cc * 8, 0u, 0u, 0u, 0u);
                     stg128(prm.dV + row * prm.dim + cc * 8, 0u, 0u, 0u, 0u);
@@ -1019,7 +1023,8 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
         K = sv + sl.phik;
     }
     const size_t bh = (size_t)(p.B * p.H);
-    const uint64_t rows = (uint64_t)(bh * p.N);
+    const uint64_t n = (uint64_t)p.N;
+    const bool ragged = ragged_problem(p, lengths);
 
     // workspace carve-up (see causal_backward_workspace)
     uint8_t* w = (uint8_t*)ws;
@@ -1029,15 +1034,15 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     float* dl = (float*)w;
 
     CUtensorMap mQ, mK, mV, mG;
-    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mG, G, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mQ, Q, ragged, bh, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mK, K, ragged, bh, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mV, V, ragged, bh, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mG, G, ragged, bh, n, kChunk, (int)p.D)) return rc;
     int* status = device_status_ptr();
     if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
 
     static std::atomic<uint64_t> attr_dq{0}, attr_dkv{0}, attr_dq_ragged{0}, attr_dkv_ragged{0};
-    if (lengths) {
+    if (ragged) {
         if (int rc = opt_in_smem_once(causal_bwd_dq_kernel<true>, kDqSmemBytes, attr_dq_ragged)) return rc;
         if (int rc = opt_in_smem_once(causal_bwd_dkv_kernel<true>, kKvSmemBytes, attr_dkv_ragged)) return rc;
     } else {
@@ -1068,10 +1073,10 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     a.dQ = (__nv_bfloat16*)dQ;
     prof_begin(kProfCausalBwdDq, st);
     CUtensorMap mDQ;
-    if (int rc = encode_tile_map(&mDQ, dQ, rows, 32, (int)p.D)) return rc;      // one quadrant's rows per store
+    if (int rc = encode_attention_map(&mDQ, dQ, ragged, bh, n, 32, (int)p.D)) return rc;      // one quadrant's rows per store
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg_q = chained_launch(grid, kDqThreads, kDqSmemBytes, st, &attr);
-    if (lengths) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_q, causal_bwd_dq_kernel<true>, mK, mV, mG, mQ, mDQ, a));
+    if (ragged) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_q, causal_bwd_dq_kernel<true>, mK, mV, mG, mQ, mDQ, a));
     else LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_q, causal_bwd_dq_kernel<false>, mK, mV, mG, mQ, mDQ, a));
     note_launch();
     prof_end(kProfCausalBwdDq, st);
@@ -1099,10 +1104,10 @@ int causal_backward(const la_problem& p, const void* Q, const void* K, const voi
     b.dV = (__nv_bfloat16*)dV;
     prof_begin(kProfCausalBwdDkv, st);
     CUtensorMap mDK, mDV;
-    if (int rc = encode_tile_map(&mDK, dK, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mDV, dV, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mDK, dK, ragged, bh, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mDV, dV, ragged, bh, n, kChunk, (int)p.D)) return rc;
     const cudaLaunchConfig_t cfg_kv = chained_launch(grid, kKvThreads, kKvSmemBytes, st, &attr);
-    if (lengths) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_kv, causal_bwd_dkv_kernel<true>, mQ, mK, mV, mG, mDK, mDV, b));
+    if (ragged) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_kv, causal_bwd_dkv_kernel<true>, mQ, mK, mV, mG, mDK, mDV, b));
     else LA_CUDA_TRY(cudaLaunchKernelEx(&cfg_kv, causal_bwd_dkv_kernel<false>, mQ, mK, mV, mG, mDK, mDV, b));
     note_launch();
     prof_end(kProfCausalBwdDkv, st);

@@ -180,11 +180,11 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 if (*abort_flag) break;
                 if (early_loads && c == kStages) grid_dependency_wait();    // (nothing this thread does depends on it)
                 uint8_t* st = smem + kOffStage + s * kStageBytes;
-                const int y = (int)(row0 + (int64_t)c * kChunk);
+                const int y = (c_begin + c) * kChunk, z = (int)bh;      // position in the sequence; sequence
                 mbar_arrive_expect_tx(&bars->full[s], kStageBytes);
-                tma_load_2d(st, &mapQ, 0, y, &bars->full[s]);
-                tma_load_2d(st + kTileBytes, &mapK, 0, y, &bars->full[s]);
-                tma_load_2d(st + 2 * kTileBytes, &mapV, 0, y, &bars->full[s]);
+                tile_load<kVarlen>(st, &mapQ, y, z, prm.N, &bars->full[s]);
+                tile_load<kVarlen>(st + kTileBytes, &mapK, y, z, prm.N, &bars->full[s]);
+                tile_load<kVarlen>(st + 2 * kTileBytes, &mapV, y, z, prm.N, &bars->full[s]);
             }
         }
     } else if (warp >= 17) {
@@ -303,7 +303,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                         tma_store_wait_read<0>();
                         mbar_arrive(&bars->empty[(c - 1) % kStages]);
                     }
-                    tma_store_2d(&mapPQ, tile, 0, (int)(row0 + (int64_t)c * kChunk));
+                    tile_store<kVarlen>(&mapPQ, tile, (c_begin + c) * kChunk, (int)bh, prm.N);
                     tma_store_commit();
                 }
             }
@@ -367,7 +367,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                         tma_store_wait_read<0>();
                         mbar_arrive(&bars->empty[(c - 1) % kStages]);
                     }
-                    tma_store_2d(&mapPK, tile, 0, (int)(row0 + (int64_t)c * kChunk));
+                    tile_store<kVarlen>(&mapPK, tile, (c_begin + c) * kChunk, (int)bh, prm.N);
                     tma_store_commit();
                 }
             }
@@ -445,6 +445,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             const float inv = 1.f / (den + prm.eps);
             const int64_t row = row0 + (int64_t)c * kChunk + t;
             if (kVarlen && c == L - 1 && t >= tail_rows) {  // a padded row of the chunk that holds the sequence's end
+                if ((int64_t)(c_begin + c) * kChunk + t >= prm.N) return true;      // past the sequence: not in memory
                 if (half == 0 && prm.den) prm.den[row] = 0.f;
                 if (half * 32 < prm.dim) {
                     __nv_bfloat16* dst = prm.O + row * prm.dim + half * 32;
@@ -485,6 +486,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             #pragma unroll 1
             for (int c = L; c < L_full; ++c) {
                 const int64_t row = row0 + (int64_t)c * kChunk + t;
+                if ((int64_t)(c_begin + c) * kChunk + t >= prm.N) continue;         // past the sequence: not in memory
                 if (half == 0 && prm.den) prm.den[row] = 0.f;
                 if (half * 32 < prm.dim) {
                     __nv_bfloat16* dst = prm.O + row * prm.dim + half * 32;
@@ -510,7 +512,7 @@ CausalPlan choose_plan(const la_problem& p) {
     const int kSms = sm_count();
     const PlanOverride ov = plan_override();        // A/B checks: a fixed number of equal pieces, a fixed short length
     CausalPlan pl;
-    pl.chunks = (int)(p.N / kChunk);
+    pl.chunks = chunks_of(p.N);
     pl.bh = (int)(p.B * p.H);
     pl.nlong = 1;
     pl.m = 0;
@@ -562,21 +564,22 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
                    cudaStream_t st) {
     if (lengths) saved = nullptr;       // a ragged batch keeps nothing for the backward pass
     const CausalPlan pl = choose_plan(p);
-    const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
+    const uint64_t seqs = (uint64_t)(p.B * p.H), n = (uint64_t)p.N;
+    const bool ragged = ragged_problem(p, lengths);
     const SavedLayout sl = saved_layout(p, pl);
     uint8_t* sv = (uint8_t*)saved;
     const bool save = sv != nullptr && p.phi == LA_PHI_ELU1;     // with identity features Q, K are the mapped tensors
     CUtensorMap mQ, mK, mV, mPQ, mPK;
-    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mPQ, save ? sv + sl.phiq : Q, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mPK, save ? sv + sl.phik : K, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mQ, Q, ragged, seqs, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mK, K, ragged, seqs, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mV, V, ragged, seqs, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mPQ, save ? sv + sl.phiq : Q, ragged, seqs, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mPK, save ? sv + sl.phik : K, ragged, seqs, n, kChunk, (int)p.D)) return rc;
     int* status = device_status_ptr();
     if (!status) return fail(LA_ERR_CUDA, "device status word unavailable");
 
     static std::atomic<uint64_t> attr_done{0}, attr_done_ragged{0};
-    if (int rc = lengths ? opt_in_smem_once(causal_fwd_kernel<true>, kSmemBytes, attr_done_ragged)
+    if (int rc = ragged ? opt_in_smem_once(causal_fwd_kernel<true>, kSmemBytes, attr_done_ragged)
                          : opt_in_smem_once(causal_fwd_kernel<false>, kSmemBytes, attr_done)) return rc;
     // the pre-pass records go straight into the saved buffer when there is one
     float* records = sv ? (float*)(sv + sl.records) : (float*)ws;
@@ -617,7 +620,7 @@ int causal_forward(const la_problem& p, const void* Q, const void* K, const void
     prof_begin(kProfCausalFwd, st);
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = chained_launch((unsigned)(pl.npieces() * pl.bh), kThreads, kSmemBytes, st, &attr);
-    if (lengths) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, causal_fwd_kernel<true>, mQ, mK, mV, mPQ, mPK, prm));
+    if (ragged) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, causal_fwd_kernel<true>, mQ, mK, mV, mPQ, mPK, prm));
     else LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, causal_fwd_kernel<false>, mQ, mK, mV, mPQ, mPK, prm));
     note_launch();
     prof_end(kProfCausalFwd, st);

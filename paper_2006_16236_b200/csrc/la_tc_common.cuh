@@ -152,6 +152,10 @@ struct CausalPlan {
 constexpr int kKeepTailChunks = 7;
 
 CausalPlan choose_plan(const la_problem& p);
+// chunks of a sequence of N positions (the last one may be partial); the ragged variants of the kernels run when
+// a batch carries lengths or N is not a multiple of the chunk
+inline int chunks_of(int64_t N) { return (int)((N + kChunk - 1) / kChunk); }
+inline bool ragged_problem(const la_problem& p, const int* lengths) { return lengths != nullptr || p.N % kChunk != 0; }
 
 // Per-part sums of phi(X)^T [Y | a] into `records` (forward: the parts before the last piece; reverse:
 // the parts after the first piece)
@@ -193,6 +197,8 @@ inline SavedLayout saved_layout(const la_problem& p, const CausalPlan& pl) {
 // loads fill it with zeros (zero features and zero values contribute nothing to any product),
 // stores clip it.  The kernels then run as for 64 and only touch `cols` columns in global memory.
 int encode_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int cols = kDim);
+// The same over [seqs][n][cols] with boxes of one sequence's rows: coordinates (column, position, sequence)
+int encode_seq_tile_map(CUtensorMap* map, const void* base, uint64_t seqs, uint64_t n, uint32_t box_rows, int cols = kDim);
 
 // ---------------------------------------------------------------------------
 // Feature map on one 128-byte row of a swizzled tile, in place: thread-per-row.
@@ -282,15 +288,18 @@ __device__ __forceinline__ void phi_row_inplace(uint8_t* row, uint32_t r7, int n
     map_row_inplace<true, false>(row, r7, 1.f, nch);
 }
 
-// Right-padded ragged batches.  Of the chunks [c_begin, c_begin + n_full) a CTA is responsible for, only those
-// that hold real positions of the sequence are processed; the last of them may be partly padding.
+// Right-padded ragged batches, and sequences whose length N is not a multiple of the chunk (lengths == nullptr:
+// every sequence has N positions).  Of the chunks [c_begin, c_begin + n_full) a CTA is responsible for, only those
+// that hold real positions of the sequence are processed; the last of them may be partly padding.  Rows of a
+// chunk at positions >= N do not exist in memory (they would be the next sequence's): the 3-D tile loads read
+// zeros there and the tile stores clip them; plain loads and stores skip them.
 struct RaggedSpan {
     int chunks;         // chunks of the span to process (0: the span is all padding)
     int tail_rows;      // real rows of the last processed chunk (kChunk unless the sequence ends inside it)
     bool has_end;       // the sequence's last real chunk lies in this span
 };
 __device__ __forceinline__ RaggedSpan ragged_span(const int* lengths, int heads, int64_t bh, int64_t N, int c_begin, int n_full) {
-    int64_t len = lengths[bh / heads];
+    int64_t len = lengths ? lengths[bh / heads] : N;
     len = len < 0 ? 0 : (len < N ? len : N);
     const int nc = (int)((len + kChunk - 1) / kChunk);              // chunks of the sequence with real rows
     RaggedSpan r;
@@ -299,6 +308,30 @@ __device__ __forceinline__ RaggedSpan ragged_span(const int* lengths, int heads,
     r.tail_rows = r.has_end ? (int)(len - (int64_t)(nc - 1) * kChunk) : kChunk;
     return r;
 }
+// Tile transfers of the attention kernels: position `pos` of sequence `seq` (N positions each).  Whole chunks only
+// (k3d false): the tensor is one [seqs * N][cols] matrix and the tile a 2-D box, which the TMA unit handles a little
+// faster (0.3 % of the benchmark step); otherwise a 3-D box over [seqs][N][cols] that ends with its sequence.
+template <bool k3d>
+__device__ __forceinline__ void tile_load(void* dst, const CUtensorMap* map, int pos, int seq, int64_t N, uint64_t* bar) {
+    if (k3d) sm100::tma_load_3d(dst, map, 0, pos, seq, bar);
+    else sm100::tma_load_2d(dst, map, 0, (int)(seq * N + pos), bar);
+}
+template <bool k3d>
+__device__ __forceinline__ void tile_load(bool leader, void* dst, const CUtensorMap* map, int pos, int seq, int64_t N, uint64_t* bar,
+                                          uint64_t policy) {
+    if (k3d) sm100::tma_load_3d(leader, dst, map, 0, pos, seq, bar, policy);
+    else sm100::tma_load_2d(leader, dst, map, 0, (int)(seq * N + pos), bar, policy);
+}
+template <bool k3d>
+__device__ __forceinline__ void tile_store(const CUtensorMap* map, const void* src, int pos, int seq, int64_t N) {
+    if (k3d) sm100::tma_store_3d(map, src, 0, pos, seq);
+    else sm100::tma_store_2d(map, src, 0, (int)(seq * N + pos));
+}
+// the map that goes with them
+inline int encode_attention_map(CUtensorMap* map, const void* base, bool three_d, uint64_t seqs, uint64_t n, uint32_t box_rows, int cols) {
+    return three_d ? encode_seq_tile_map(map, base, seqs, n, box_rows, cols) : encode_tile_map(map, base, seqs * n, box_rows, cols);
+}
+
 // A whole 128-byte tile row of zeros (padding rows of a ragged batch: whatever they held, they contribute nothing).
 __device__ __forceinline__ void zero_row(uint8_t* row) {
 #pragma unroll

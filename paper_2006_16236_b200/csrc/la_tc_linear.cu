@@ -115,6 +115,7 @@ struct LsParams {
     int dim;
 };
 
+template <bool k3d>         // N is not a multiple of the chunk: the tiles are 3-D boxes that end with their sequence
 __global__ void __launch_bounds__(kLsThreads, 1)
 linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                   const LsParams prm) {
@@ -127,7 +128,6 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const int64_t bh = blockIdx.x / prm.nseg;
     const int c_begin = seg * prm.chunks_per_seg;
     const int L_all = min(prm.chunks, c_begin + prm.chunks_per_seg) - c_begin;
-    const int64_t row0 = bh * prm.N + (int64_t)c_begin * kChunk;
     LA_TRACE_CTA(g_trace_lin, 0);
 
     if (tid == 0) {
@@ -164,9 +164,11 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     // Ragged batch: only `real` rows of this split exist; chunks behind them are skipped and the rows behind
     // them in the last chunk are zeroed after the load (at least one chunk runs, so that the record is written
     // from an accumulator that holds zeros and not from one that was never started).
+    // (Without lengths every sequence has N positions, and N need not be a multiple of the chunk: rows of the last
+    // chunk at positions >= N are not in memory; the 3-D tile loads read zeros there.)
     int64_t real = (int64_t)L_all * kChunk;
-    if (prm.lengths) {
-        const int64_t len = min((int64_t)max(prm.lengths[bh / prm.heads], 0), prm.N);
+    {
+        const int64_t len = prm.lengths ? min((int64_t)max(prm.lengths[bh / prm.heads], 0), prm.N) : prm.N;
         real = min(max(len - (int64_t)c_begin * kChunk, (int64_t)0), real);
     }
     const int L = max(1, (int)((real + kChunk - 1) / kChunk));
@@ -183,11 +185,11 @@ linear_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 }
                 if (*abort_flag) break;
                 uint8_t* st = smem + s * kLsStageBytes;
-                const int y = (int)(row0 + (int64_t)c * kChunk);
+                const int y = (c_begin + c) * kChunk, z = (int)bh;      // position in the sequence; sequence
                 LA_TRACE(g_trace_lin, c, 2);
                 mbar_arrive_expect_tx(&bars->full[s], 2 * kTileBytes);
-                tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
-                tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
+                tile_load<k3d>(st, &mapX, y, z, prm.N, &bars->full[s]);
+                tile_load<k3d>(st + kTileBytes, &mapY, y, z, prm.N, &bars->full[s]);
             }
         }
     } else if (warp == 9) {
@@ -327,7 +329,7 @@ struct ApParams {
     int early;                  // a kernel of the same call runs in front: the first tiles are requested before the wait
 };
 
-template <int kMode>
+template <int kMode, bool k3d>
 __global__ void __launch_bounds__(kApThreads, 1)
 linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                     const __grid_constant__ CUtensorMap mapOut0, const __grid_constant__ CUtensorMap mapOut1,
@@ -384,20 +386,20 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     }
     // Ragged batch: `len` positions of this sequence exist, `real` of them in this split.  Only the chunks that
     // hold real rows go through the pipeline; the padding behind them is filled with zeros at the end.
+    // (Without lengths len = N, which need not be a multiple of the chunk: rows at positions >= N are not in memory;
+    // the tile loads read zeros there, the tile stores clip them and the plain stores below skip them.)
     int64_t len = prm.N, real = (int64_t)L_all * kChunk;
-    if (prm.lengths) {
-        len = min((int64_t)max(prm.lengths[bh / prm.heads], 0), prm.N);
-        real = min(max(len - (int64_t)c_begin * kChunk, (int64_t)0), real);
-    }
+    if (prm.lengths) len = min((int64_t)max(prm.lengths[bh / prm.heads], 0), prm.N);
+    real = min(max(len - (int64_t)c_begin * kChunk, (int64_t)0), real);
     const int L = (int)((real + kChunk - 1) / kChunk);
     // the loads of the first chunks travel while the state is put together below
     auto issue_load = [&](int c) {
         const int s = c % kApStages;
         uint8_t* st = smem + kApOffStage + s * 2 * kTileBytes;
-        const int y = (int)(row0 + (int64_t)c * kChunk);
+        const int y = (c_begin + c) * kChunk, z = (int)bh;          // position in the sequence; sequence
         mbar_arrive_expect_tx(&bars->full[s], kTiles * kTileBytes);
-        tma_load_2d(st, &mapX, 0, y, &bars->full[s]);
-        if (kHasY) tma_load_2d(st + kTileBytes, &mapY, 0, y, &bars->full[s]);
+        tile_load<k3d>(st, &mapX, y, z, prm.N, &bars->full[s]);
+        if (kHasY) tile_load<k3d>(st + kTileBytes, &mapY, y, z, prm.N, &bars->full[s]);
     };
     if (warp == 8 && lane == 0) {
         prefetch_tensormap(&mapX);
@@ -668,7 +670,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
                 const float den = fN * x1sum + sScal[0] + xa;
                 const float inv = 1.f / (den + prm.eps);
                 const float w = x1sum * inv;
-                if (hf == 0 && prm.den) prm.den[row] = padded ? 0.f : den;
+                if (hf == 0 && prm.den && (!k3d || (int64_t)(c_begin + c) * kChunk + t < prm.N)) prm.den[row] = padded ? 0.f : den;
                 const f32x2 inv2 = pair(inv, inv), w2 = pair(w, w);
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
@@ -761,9 +763,11 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
             fence_proxy_async_smem();
             named_barrier(2 + quad, 64);            // both halves of the 32 rows are in the slab
             if (hf == 0 && lane == 0) {
-                const int y = (int)(row0 + (int64_t)c * kChunk + quad * 32);
-                tma_store_2d(&mapOut0, smem + kApOffOut + quad * 32 * 128, 0, y);
-                if (kMode == kApplyBackwardKV) tma_store_2d(&mapOut1, smem + kApOffOut + kTileBytes + quad * 32 * 128, 0, y);
+                const int y = (c_begin + c) * kChunk + quad * 32;       // rows at positions >= N are clipped by the store
+                if (!k3d || y < prm.N) {
+                    tile_store<k3d>(&mapOut0, smem + kApOffOut + quad * 32 * 128, y, (int)bh, prm.N);
+                    if (kMode == kApplyBackwardKV) tile_store<k3d>(&mapOut1, smem + kApOffOut + kTileBytes + quad * 32 * 128, y, (int)bh, prm.N);
+                }
                 tma_store_commit();
             }
             if (tid == 0) LA_TRACE(g_trace_lin, c, 13);
@@ -796,7 +800,8 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         }
         if (L < L_all) {            // whole chunks of padding: zeros, written directly
             const int e = hf * 128 + t;
-            const int64_t r_lo = row0 + (int64_t)L * kChunk, nrows = (int64_t)(L_all - L) * kChunk;
+            const int64_t r_lo = row0 + (int64_t)L * kChunk;
+            const int64_t nrows = max((int64_t)0, min((int64_t)(L_all - L) * kChunk, prm.N - (int64_t)(c_begin + L) * kChunk));
             const int64_t n16 = nrows * prm.dim * 2 / 16;
             uint4* o0 = reinterpret_cast<uint4*>(prm.out0 + r_lo * prm.dim);
             for (int64_t i = e; i < n16; i += 256) o0[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -822,7 +827,7 @@ linear_apply_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
 // 16 chunks take 0.24 ms per forward + backward, five splits of 6-7 chunks 0.33 ms: a CTA's start-up costs
 // several chunk times, and more CTAs than resident slots run in waves), at least two chunks each.
 Segmentation choose_splits(const la_problem& p) {
-    const int chunks = (int)(p.N / kChunk);
+    const int chunks = chunks_of(p.N);
     const int64_t bh = p.B * p.H;
     int nseg = (int)(sm_count() / bh);
     if (plan_override().linear_splits > 0) nseg = plan_override().linear_splits;        // A/B checks
@@ -833,10 +838,11 @@ Segmentation choose_splits(const la_problem& p) {
     return Segmentation{nseg, cps};
 }
 
-int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
-                const int* lengths, float* records, cudaStream_t st) {
-    static std::atomic<uint64_t> attr_done{0};
-    if (int rc = opt_in_smem_once(linear_sum_kernel, kLsSmemBytes, attr_done)) return rc;
+template <bool k3d>
+int launch_sums_as(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
+                   const int* lengths, float* records, cudaStream_t st) {
+    static std::atomic<uint64_t> attr_done{0};          // one per instantiation
+    if (int rc = opt_in_smem_once(linear_sum_kernel<k3d>, kLsSmemBytes, attr_done)) return rc;
     LsParams prm;
     prm.records = records;
     prm.lengths = lengths;
@@ -844,7 +850,7 @@ int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& 
     prm.status = device_status_ptr();
     if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
     prm.N = p.N;
-    prm.chunks = (int)(p.N / kChunk);
+    prm.chunks = chunks_of(p.N);
     prm.chunks_per_seg = sg.chunks_per_seg;
     prm.nseg = sg.nseg;
     prm.phi = p.phi;
@@ -852,38 +858,51 @@ int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& 
     prof_begin(kProfLinearSum, st);
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = chained_launch((unsigned)(sg.nseg * p.B * p.H), kLsThreads, kLsSmemBytes, st, &attr);
-    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_sum_kernel, mX, mY, prm));
+    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_sum_kernel<k3d>, mX, mY, prm));
     note_launch();
     prof_end(kProfLinearSum, st);
     return LA_OK;
 }
 
-template <int kMode>
-int launch_apply(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
-                 ApParams prm, cudaStream_t st) {
-    static std::atomic<uint64_t> attr_done{0};          // one per instantiation (kMode)
-    if (int rc = opt_in_smem_once(linear_apply_kernel<kMode>, kApSmemBytes, attr_done)) return rc;
+int launch_sums(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
+                const int* lengths, float* records, cudaStream_t st) {
+    return p.N % kChunk ? launch_sums_as<true>(p, sg, mX, mY, lengths, records, st)
+                        : launch_sums_as<false>(p, sg, mX, mY, lengths, records, st);
+}
+
+template <int kMode, bool k3d>
+int launch_apply_as(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
+                    ApParams prm, cudaStream_t st) {
+    static std::atomic<uint64_t> attr_done{0};          // one per instantiation
+    if (int rc = opt_in_smem_once(linear_apply_kernel<kMode, k3d>, kApSmemBytes, attr_done)) return rc;
     prm.status = device_status_ptr();
     if (!prm.status) return fail(LA_ERR_CUDA, "device status word unavailable");
     prm.heads = (int)p.H;
     prm.N = p.N;
-    prm.chunks = (int)(p.N / kChunk);
+    prm.chunks = chunks_of(p.N);
     prm.chunks_per_seg = sg.chunks_per_seg;
     prm.nseg = sg.nseg;
     prm.eps = p.eps;
     prm.phi = p.phi;
     prm.dim = (int)p.D;
-    const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
+    const uint64_t seqs = (uint64_t)(p.B * p.H), n = (uint64_t)p.N;
     CUtensorMap mO0, mO1;                   // one warp's 32 rows per store
-    if (int rc = encode_tile_map(&mO0, prm.out0, rows, 32, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mO1, prm.out1 ? prm.out1 : prm.out0, rows, 32, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mO0, prm.out0, p.N % kChunk != 0, seqs, n, 32, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mO1, prm.out1 ? prm.out1 : prm.out0, p.N % kChunk != 0, seqs, n, 32, (int)p.D)) return rc;
     prof_begin(kProfLinearApply, st);
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = chained_launch((unsigned)(sg.nseg * p.B * p.H), kApThreads, kApSmemBytes, st, &attr);
-    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_apply_kernel<kMode>, mX, mY, mO0, mO1, prm));
+    LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_apply_kernel<kMode, k3d>, mX, mY, mO0, mO1, prm));
     note_launch();
     prof_end(kProfLinearApply, st);
     return LA_OK;
+}
+
+template <int kMode>
+int launch_apply(const la_problem& p, const Segmentation& sg, const CUtensorMap& mX, const CUtensorMap& mY,
+                 const ApParams& prm, cudaStream_t st) {
+    return p.N % kChunk ? launch_apply_as<kMode, true>(p, sg, mX, mY, prm, st)
+                        : launch_apply_as<kMode, false>(p, sg, mX, mY, prm, st);
 }
 
 }  // namespace
@@ -899,11 +918,11 @@ size_t linear_backward_workspace(const la_problem& p) {
 int linear_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, void* O,
                    float* den, float* KV, float* Zs, void* saved, void* ws, cudaStream_t st) {
     const Segmentation sg = choose_splits(p);
-    const uint64_t rows = (uint64_t)(p.B * p.H * p.N);
+    const uint64_t seqs = (uint64_t)(p.B * p.H), n = (uint64_t)p.N;
     CUtensorMap mQ, mK, mV;
-    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mQ, Q, p.N % kChunk != 0, seqs, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mK, K, p.N % kChunk != 0, seqs, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mV, V, p.N % kChunk != 0, seqs, n, kChunk, (int)p.D)) return rc;
     float* rec = saved ? (float*)saved : (float*)ws;      // the split records, kept for the backward pass if asked
     if (int rc = launch_sums(p, sg, mK, mV, lengths, rec, st)) return rc;
     ApParams a = {};
@@ -921,12 +940,12 @@ int linear_backward(const la_problem& p, const void* Q, const void* K, const voi
                     const void* saved, const void* G, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
     const Segmentation sg = choose_splits(p);
     const size_t bh = (size_t)(p.B * p.H);
-    const uint64_t rows = (uint64_t)(bh * p.N);
+    const uint64_t n = (uint64_t)p.N;
     CUtensorMap mQ, mK, mV, mG;
-    if (int rc = encode_tile_map(&mQ, Q, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mK, K, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mV, V, rows, kChunk, (int)p.D)) return rc;
-    if (int rc = encode_tile_map(&mG, G, rows, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mQ, Q, p.N % kChunk != 0, bh, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mK, K, p.N % kChunk != 0, bh, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mV, V, p.N % kChunk != 0, bh, n, kChunk, (int)p.D)) return rc;
+    if (int rc = encode_attention_map(&mG, G, p.N % kChunk != 0, bh, n, kChunk, (int)p.D)) return rc;
     uint8_t* w = (uint8_t*)ws;
     float* rec_s = (float*)w;   w += bh * sg.nseg * kRecFloats * sizeof(float);
     float* rec_r = (float*)w;   w += bh * sg.nseg * kRecFloats * sizeof(float);

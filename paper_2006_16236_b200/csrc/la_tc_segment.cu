@@ -135,14 +135,14 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
                     allow_dependent_launch();
                 }
                 uint8_t* st = smem + s * kSumStageBytes;
-                const int y = (int)(row0 + (int64_t)c * kChunk);
+                const int y = (c_begin + c) * kChunk, z = (int)bh;      // position in the sequence; sequence
                 LA_TRACE(g_trace_seg, c, 2);
                 mbar_arrive_expect_tx(&bars->full[s], 2 * kTileBytes);
                 const bool wanted_soon = scaled ? prm.plan.in_piece_tail(c_begin + c, kKeepTailChunks)
                                                 : prm.plan.in_piece_head(c_begin + c, kKeepTailChunks);
                 const uint64_t pol = wanted_soon ? pol_keep : pol_stream;
-                tma_load_2d(true, st, &mapX, 0, y, &bars->full[s], pol);
-                tma_load_2d(true, st + kTileBytes, &mapY, 0, y, &bars->full[s], pol);
+                tile_load<kVarlen>(true, st, &mapX, y, z, prm.N, &bars->full[s], pol);
+                tile_load<kVarlen>(true, st + kTileBytes, &mapY, y, z, prm.N, &bars->full[s], pol);
             }
         }
         if (early_loads && L <= kSumStages) {        // a part of at most three chunks: the loop never got there
@@ -181,8 +181,9 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
         for (int c = 0; c < L; ++c) {
             const int s = c % kSumStages;
             const int64_t row = row0 + (int64_t)c * kChunk + t;
+            const bool pad = kVarlen && c == L - 1 && t >= span.tail_rows;      // (a padded row may lie past the sequence's N)
             float inv = 1.f, delta = 0.f;
-            if (scaled) {
+            if (scaled && !pad) {
                 inv = 1.f / __ldg(prm.dn + row);
                 delta = __ldg(prm.dl + row);
             }
@@ -195,7 +196,7 @@ segment_sum_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_consta
                 else phi_row_inplace(rowX, r7, prm.dim >> 3);
             }
             else if (scaled) map_row_inplace<false>(rowX, r7, inv, prm.dim >> 3);
-            if (kVarlen && c == L - 1 && t >= span.tail_rows) {     // padding: no feature, no value, no dl
+            if (pad) {                                              // padding: no feature, no value, no dl
                 zero_row(rowX);
                 zero_row(rowX + kTileBytes);
                 delta = 0.f;
@@ -249,7 +250,8 @@ int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap&
                    const int* lengths) {
     if (pl.npieces() <= 1) return LA_OK;
     static std::atomic<uint64_t> attr_done{0}, attr_done_ragged{0};
-    if (int rc = lengths ? opt_in_smem_once(segment_sum_kernel<true>, kSumSmemBytes, attr_done_ragged)
+    const bool ragged = ragged_problem(p, lengths);
+    if (int rc = ragged ? opt_in_smem_once(segment_sum_kernel<true>, kSumSmemBytes, attr_done_ragged)
                          : opt_in_smem_once(segment_sum_kernel<false>, kSumSmemBytes, attr_done)) return rc;
     SumParams prm;
     prm.records = records;
@@ -270,7 +272,7 @@ int segment_states(const la_problem& p, const CausalPlan& pl, const CUtensorMap&
     prof_begin(kProfSegmentSum, st);
     cudaLaunchAttribute attr;
     const cudaLaunchConfig_t cfg = chained_launch((unsigned)(prm.parts_per_seq * p.B * p.H), kSumThreads, kSumSmemBytes, st, &attr);
-    if (lengths) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, segment_sum_kernel<true>, mapX, mapY, prm));
+    if (ragged) LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, segment_sum_kernel<true>, mapX, mapY, prm));
     else LA_CUDA_TRY(cudaLaunchKernelEx(&cfg, segment_sum_kernel<false>, mapX, mapY, prm));
     note_launch();
     prof_end(kProfSegmentSum, st);

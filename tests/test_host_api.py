@@ -92,7 +92,10 @@ def test_causal_plan_of_the_bench_workload(L):
     assert 8 <= short <= 16 and abs((pb[1] - pb[0]) - (pb[3] - pb[2])) <= 1
     # problems that run the general kernels have no plan
     assert la.la_causal_plan(la.make_problem(1, 2, 256, 32, 32, la.LA_F32)) is None
-    assert la.la_causal_plan(la.make_problem(1, 2, 200, 64, 64, la.LA_BF16)) is None
+    assert la.la_causal_plan(la.make_problem(1, 2, 256, 64, 48, la.LA_BF16)) is None
+    # a length that is not a multiple of the chunk: the last chunk is partial
+    ragged = la.la_causal_plan(la.make_problem(1, 2, 200, 64, 64, la.LA_BF16))
+    assert ragged is not None and ragged["piece_begin"][-1] == 2
 
 
 def test_bad_arguments_are_rejected_on_the_host(L):
