@@ -240,7 +240,7 @@ def test_prefill_then_decode_handoff():
                                    (4, 16, 18 * 128, 64, 64)])
 def test_causal_forward_from_a_state(shape, dtype):
     """The recurrence of Eq. 16-20 started from a given S_0, Z_0 (general kernels and, for bf16 D = M in
-    {32, 64} with N a multiple of 128, the tensor-core kernel with several pieces per sequence)."""
+    {32, 64}, the tensor-core kernel, with several pieces per sequence at the larger shapes)."""
     B, H, N, D, M = shape
     Q, K, V, _ = draw_qkvg(B, H, N, D, M, seed=sum(shape) + 1, dtype=dtype, with_grad=False)
     g = torch.Generator().manual_seed(5)
@@ -382,7 +382,7 @@ def test_right_padded_causal_batches_need_no_mask(dtype, D, N):
 def test_noncausal_ragged_batches(shape, lengths, dtype):
     """Right-padded sequences of different lengths (key-padding mask): every sequence equals the oracle run on
     its own length, sums included, and everything is zero on the padding whatever the tensors hold there
-    (not even numbers).  The bf16 cases with D = M in {32, 64} and N a multiple of 128 run the tensor-core
+    (not even numbers).  The bf16 cases with D = M in {32, 64} run the tensor-core
     kernels, whose splits end inside, at and before a sequence's end; the others the general kernels."""
     B, H, N, D, M = shape
     Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=sum(shape) + 4, dtype=dtype)
@@ -517,7 +517,7 @@ def test_poly2_attention_end_to_end(shape, signed, causal, dtype):
     Q, K, V, G = draw_qkvg(B, H, N, D, M, seed=sum(shape) + causal, dtype=dtype)
     if not signed:
         Q, K = Q.abs(), K.abs()
-    loose = signed and dtype == torch.bfloat16 and D * D == 64 and N % 128 == 0        # tensor-core kernels
+    loose = signed and dtype == torch.bfloat16 and D * D == 64 and M == 64           # tensor-core kernels
 
     def check(x, ref, what, grad=False):
         if loose:
