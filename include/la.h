@@ -22,10 +22,10 @@
  *    accumulation are fp32.  Data pointers must be 16-byte aligned.
  *  - Outputs must not alias inputs (S and Z of la_recurrent_step are in-out).
  *  - Supported sizes: D and M multiples of 8 in [8, 128]; B, H >= 1; N >= 0
- *    (N == 0 is a successful no-op).  bf16 problems with D = M in {32, 64} and N
- *    a multiple of the chunk length run on the tensor-core kernels, everything
- *    else on the general fp32-arithmetic kernels; results agree within the
- *    rounding of the I/O type.
+ *    (N == 0 is a successful no-op).  bf16 problems with D = M in {32, 64} run
+ *    on the tensor-core kernels (any N: a last chunk of fewer than 128
+ *    positions is handled as padding), everything else on the general
+ *    fp32-arithmetic kernels; results agree within the rounding of the I/O type.
  *  - Return value: LA_OK (0) or a negative la_status.  All argument checks run
  *    on the host before anything is enqueued; a failed check enqueues nothing.
  *    The library never aborts, throws or traps.  la_last_error() returns a
