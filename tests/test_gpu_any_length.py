@@ -38,7 +38,8 @@ def _untouched(tails):
         assert bool((tail == MARK).all()), f"{nm}: something was stored behind the tensor's end"
 
 
-SHAPES = [(2, 3, 100, 64), (2, 3, 129, 64), (1, 5, 200, 32), (2, 8, 784, 32), (3, 2, 1000, 64), (1, 70, 700, 64)]
+SHAPES = [(2, 3, 100, 64), (2, 3, 129, 64), (1, 5, 200, 32), (2, 8, 784, 32), (3, 2, 1000, 64), (1, 70, 700, 64),
+          (2, 2, 1, 64), (1, 3, 127, 32), (1, 2, 2, 32)]
 
 
 @pytest.mark.parametrize("keep", [False, True], ids=["recompute", "saved"])
@@ -76,7 +77,7 @@ def test_causal_any_length(shape, keep):
     assert_close(Z, fk.sum(2), torch.bfloat16, "Z_out")
 
 
-@pytest.mark.parametrize("shape", SHAPES[:5], ids=lambda s: "B%d_H%d_N%d_D%d" % s)
+@pytest.mark.parametrize("shape", SHAPES[:5] + SHAPES[6:], ids=lambda s: "B%d_H%d_N%d_D%d" % s)
 def test_noncausal_any_length(shape):
     B, H, N, D = shape
     Q, K, V, G = draw_qkvg(B, H, N, D, D, 11 + N, torch.bfloat16, 0.5)
@@ -132,3 +133,26 @@ def test_lengths_inside_a_batch_whose_own_length_is_odd(causal):
         assert_close(outs["O"][b:b + 1, :, :n], O_ref, torch.bfloat16, f"O of sequence {b}")
         for nm, ref in zip(("dQ", "dK", "dV"), oracle.linear_attention_backward(q, k, v, g, causal=causal)):
             assert_close(outs[nm][b:b + 1, :, :n], ref, torch.bfloat16, f"{nm} of sequence {b}", grad=True)
+
+
+def test_prefill_in_odd_pieces_then_decode():
+    """A prompt of 300 positions fed in calls of 77, 200 and 23 positions (none a multiple of the chunk), each
+    continuing from the state the call before left, then two decode steps: the same outputs as the whole sequence."""
+    B, H, D = 2, 3, 64
+    cuts = [77, 200, 23]
+    N = sum(cuts) + 2
+    Q, K, V, _ = draw_qkvg(B, H, N, D, D, 3, torch.bfloat16, 1.0, with_grad=False)
+    O_ref = oracle.linear_attention(*(t.double().numpy() for t in (Q, K, V)), causal=True)[0]
+    S = torch.zeros((B, H, D, D), device=DEV)
+    Z = torch.zeros((B, H, D), device=DEV)
+    lo = 0
+    for n in cuts:
+        q, k, v = (t[:, :, lo:lo + n].contiguous().to(DEV) for t in (Q, K, V))
+        S2, Z2 = torch.empty_like(S), torch.empty_like(Z)
+        O = la.la_causal_forward(q, k, v, S_in=S, Z_in=Z, S_out=S2, Z_out=Z2)
+        assert_close(O, O_ref[:, :, lo:lo + n], torch.bfloat16, f"positions {lo}..{lo + n}")
+        S, Z, lo = S2, Z2, lo + n
+    for i in range(lo, N):
+        out = la.la_recurrent_step(Q[:, :, i].contiguous().to(DEV), K[:, :, i].contiguous().to(DEV), V[:, :, i].contiguous().to(DEV), S, Z)
+        assert_close(out, O_ref[:, :, i], torch.bfloat16, f"decode step {i}")
+    la.la_last_device_status()
