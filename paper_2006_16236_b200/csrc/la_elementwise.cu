@@ -6,27 +6,44 @@ namespace la {
 
 // ---------------------------------------------------------------------------
 // Feature map: y = phi(x) or phi'(x).  Bandwidth-bound; 16-byte accesses on the
-// aligned body, scalar accesses on the ragged tail.
+// aligned body, four of them in flight per thread (a thread with one load outstanding
+// leaves the memory system short of requests: 0.74 of the copy bandwidth against 0.9),
+// scalar accesses on the ragged tail.  exp through ex2.approx (relative error 2^-22).
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ float fm(float x, int deriv) {
     if (x > 0.f) return deriv ? 1.f : x + 1.f;
-    return expf(x);
+    return __expf(x);
 }
 
 template <typename T>
-__global__ void feature_map_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t n, int deriv) {
+__global__ void __launch_bounds__(256)
+feature_map_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t n, int deriv) {
     constexpr int V = 16 / sizeof(T);
+    constexpr int U = 4;                        // 16-byte vectors per thread and iteration
     const int64_t nvec = n / V;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    for (int64_t i = t0; i < nvec; i += stride) {
+    int64_t i = t0;
+    for (; i + (U - 1) * stride < nvec; i += U * stride) {
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) raw[u] = __ldcs(reinterpret_cast<const uint4*>(x) + i + u * stride);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            T* e = reinterpret_cast<T*>(&raw[u]);
+#pragma unroll
+            for (int j = 0; j < V; ++j) e[j] = from_f32<T>(fm(to_f32<T>(e[j]), deriv));
+            __stcs(reinterpret_cast<uint4*>(y) + i + u * stride, raw[u]);
+        }
+    }
+    for (; i < nvec; i += stride) {
         uint4 raw = reinterpret_cast<const uint4*>(x)[i];
         T* e = reinterpret_cast<T*>(&raw);
 #pragma unroll
         for (int j = 0; j < V; ++j) e[j] = from_f32<T>(fm(to_f32<T>(e[j]), deriv));
         reinterpret_cast<uint4*>(y)[i] = raw;
     }
-    for (int64_t i = nvec * V + t0; i < n; i += stride) y[i] = from_f32<T>(fm(to_f32<T>(x[i]), deriv));
+    for (int64_t k = nvec * V + t0; k < n; k += stride) y[k] = from_f32<T>(fm(to_f32<T>(x[k]), deriv));
 }
 
 int launch_feature_map(const void* x, void* y, int64_t n, int dtype, int deriv, cudaStream_t st) {
@@ -35,7 +52,7 @@ int launch_feature_map(const void* x, void* y, int64_t n, int dtype, int deriv, 
     const int64_t vec = dtype == LA_F32 ? 4 : 8;
     int64_t blocks = (n / vec + threads - 1) / threads;
     if (blocks < 1) blocks = 1;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > 148 * 8) blocks = 148 * 8;            // one resident wave: 8 blocks of 256 threads per SM
     if (dtype == LA_F32)
         feature_map_kernel<float><<<(unsigned)blocks, threads, 0, st>>>((const float*)x, (float*)y, n, deriv);
     else
@@ -114,6 +131,93 @@ poly2_map_backward_kernel(const T* __restrict__ x, const T* __restrict__ dy, T* 
     }
 }
 
+// D = 8, C = 64, bf16 (the shape the tensor-core attention kernels take).  Forward: eight threads per row, one
+// 16-byte group of columns each (thread i writes x_i times the row), four rows per thread in flight.  Backward:
+// one thread per row with the whole 8x8 gradient block in registers, the rows staged through shared memory.
+__global__ void __launch_bounds__(256)
+poly2_map_d8_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y, int64_t rows) {
+    constexpr int U = 4;
+    const int i = threadIdx.x & 7;
+    const int64_t stride = (int64_t)gridDim.x * 32;                     // rows per step of the whole grid
+    int64_t r = (int64_t)blockIdx.x * 32 + (threadIdx.x >> 3);
+    for (; r < rows; r += U * stride) {
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (r + u * stride < rows) raw[u] = __ldg(reinterpret_cast<const uint4*>(x + (r + u * stride) * 8));
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (r + u * stride >= rows) break;
+            const __nv_bfloat16* xe = reinterpret_cast<const __nv_bfloat16*>(&raw[u]);
+            float xi = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) xi = e == i ? __bfloat162float(xe[e]) : xi;
+            uint32_t o[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const __nv_bfloat162 pr = __floats2bfloat162_rn(xi * __bfloat162float(xe[2 * e]), xi * __bfloat162float(xe[2 * e + 1]));
+                o[e] = *reinterpret_cast<const uint32_t*>(&pr);
+            }
+            __stcs(reinterpret_cast<uint4*>(y + (r + u * stride) * 64 + i * 8), make_uint4(o[0], o[1], o[2], o[3]));
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+poly2_map_backward_d8_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ dy,
+                             __nv_bfloat16* __restrict__ dx, int64_t rows) {
+    // 256 rows per step of a block: their gradient rows (128 bytes each) come in as one contiguous 32 KB run,
+    // eight 16-byte loads per thread in flight, and are parked in shared memory with a row pitch of 144 bytes
+    // (a quarter-warp's 16-byte reads of eight consecutive rows then fall into different banks); after the
+    // barrier every thread takes one row with its whole 8x8 block in registers.
+    constexpr int kPitch = 144;
+    __shared__ __align__(16) uint8_t tile[256 * kPitch];
+    const int tid = threadIdx.x;
+    for (int64_t r0 = (int64_t)blockIdx.x * 256; r0 < rows; r0 += (int64_t)gridDim.x * 256) {
+        const int64_t nrows = rows - r0 < 256 ? rows - r0 : 256;
+        const uint4* src = reinterpret_cast<const uint4*>(dy + r0 * 64);
+        uint4 raw[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int v = k * 256 + tid;                        // 16-byte vector of the run: row v / 8, group v % 8
+            raw[k] = (v >> 3) < nrows ? __ldcs(src + v) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        uint4 rawx = make_uint4(0u, 0u, 0u, 0u);
+        if (tid < nrows) rawx = __ldg(reinterpret_cast<const uint4*>(x + (r0 + tid) * 8));
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int v = k * 256 + tid;
+            *reinterpret_cast<uint4*>(tile + (v >> 3) * kPitch + (v & 7) * 16) = raw[k];
+        }
+        __syncthreads();
+        const __nv_bfloat16* xe = reinterpret_cast<const __nv_bfloat16*>(&rawx);
+        float xv[8], s[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { xv[j] = __bfloat162float(xe[j]); s[j] = 0.f; }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint4 g4 = *reinterpret_cast<const uint4*>(tile + tid * kPitch + i * 16);
+            const __nv_bfloat16* ge = reinterpret_cast<const __nv_bfloat16*>(&g4);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float g = __bfloat162float(ge[j]);        // g_ij: a term of dx_i (with x_j) and of dx_j (with x_i)
+                s[i] = fmaf(g, xv[j], s[i]);
+                s[j] = fmaf(g, xv[i], s[j]);
+            }
+        }
+        if (tid < nrows) {
+            uint32_t o[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const __nv_bfloat162 pr = __floats2bfloat162_rn(s[2 * e], s[2 * e + 1]);
+                o[e] = *reinterpret_cast<const uint32_t*>(&pr);
+            }
+            *reinterpret_cast<uint4*>(dx + (r0 + tid) * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+        __syncthreads();                                        // the tile is rewritten by the next step
+    }
+}
+
 // blocks of (width, 256 / width) threads over the rows, at most 16 blocks per SM
 static void poly2_launch_shape(int64_t rows, int width, dim3* grid, dim3* block) {
     const int rpb = 256 / width;
@@ -125,6 +229,13 @@ static void poly2_launch_shape(int64_t rows, int width, dim3* grid, dim3* block)
 
 int launch_poly2_map(const void* x, void* y, int64_t rows, int D, int C, int dtype, cudaStream_t st) {
     if (rows == 0) return LA_OK;
+    if (dtype == LA_BF16 && D == 8 && C == 64) {
+        int64_t blocks = (rows + 31) / 32;
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        poly2_map_d8_kernel<<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, rows);
+        LA_LAUNCHED();
+        return LA_OK;
+    }
     dim3 grid, block;
     poly2_launch_shape(rows, C >> 3, &grid, &block);
     if (dtype == LA_F32)
@@ -138,6 +249,14 @@ int launch_poly2_map(const void* x, void* y, int64_t rows, int D, int C, int dty
 int launch_poly2_map_backward(const void* x, const void* dy, void* dx, int64_t rows, int D, int C, int dtype,
                               cudaStream_t st) {
     if (rows == 0) return LA_OK;
+    if (dtype == LA_BF16 && D == 8 && C == 64) {
+        int64_t blocks = (rows + 255) / 256;
+        if (blocks > 148 * 6) blocks = 148 * 6;             // 36 KB of shared memory each
+        poly2_map_backward_d8_kernel<<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)dy,
+                                                                      (__nv_bfloat16*)dx, rows);
+        LA_LAUNCHED();
+        return LA_OK;
+    }
     dim3 grid, block;
     poly2_launch_shape(rows, D, &grid, &block);
     if (dtype == LA_F32)

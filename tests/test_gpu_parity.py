@@ -23,7 +23,7 @@ DTYPES = [torch.float32, torch.bfloat16]
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
-@pytest.mark.parametrize("n", [0, 1, 7, 8, 1000, 65536 + 3])
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 1000, 65536 + 3, 5 * 2 ** 20 + 13])
 def test_feature_map(dtype, n):
     x = (torch.randn(n, generator=torch.Generator().manual_seed(n)) * 3).to(dtype)
     for deriv in (False, True):
@@ -439,6 +439,21 @@ def test_poly2_feature_map_and_its_gradient(D, C, dtype):
     assert np.all(got[..., D * D:] == 0.0)
     assert_close(dx, oracle.poly2_feature_map_backward(x.double().numpy(), dy.double().numpy()), dtype, "dx", grad=True)
     assert la.la_feature_map_poly2(torch.empty((0, D), dtype=dtype, device=DEV), C).shape == (0, C)
+
+
+def test_poly2_feature_map_many_rows():
+    """D = 8, C = 64 in bf16 has kernels of its own (several rows per thread in flight, the gradient rows staged
+    through shared memory): enough rows for every block to loop, and a ragged end."""
+    rows, D, C = 300001, 8, 64
+    g = torch.Generator().manual_seed(77)
+    x = torch.randn((rows, D), generator=g).to(torch.bfloat16)
+    dy = torch.randn((rows, C), generator=g).to(torch.bfloat16)
+    y = la.la_feature_map_poly2(x.to(DEV), C)
+    dx = la.la_feature_map_poly2_backward(x.to(DEV), dy.to(DEV))
+    ref = oracle.poly2_feature_map(x.double().numpy(), C)
+    got = y.double().cpu().numpy()
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref)), np.abs(got - ref).max()
+    assert_close(dx, oracle.poly2_feature_map_backward(x.double().numpy(), dy.double().numpy()), torch.bfloat16, "dx", grad=True)
 
 
 @pytest.mark.parametrize("D,C,rows", [(64, 64, (3, 5, 67)), (64, 128, (2, 700)), (32, 64, (1000,)), (8, 128, (130,)), (64, 64, (40000,))],
