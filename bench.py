@@ -626,6 +626,31 @@ def bench_ragged(la, w, dev, pk, iters=10):
     return out
 
 
+def bench_feature_map(la, w, dev, pk, iters=10):
+    """The stand-alone feature map of Eq. 7 on the headline workload's Q (value and slope): two tensors alternate,
+    so that a launch's 268 MB are not in L2 from the launch before."""
+    rows, D = w.B * w.H * w.N, w.D
+    g = torch.Generator(device="cpu").manual_seed(w.seed + 29)
+    xs = [torch.randn((rows, D), generator=g).to(w.torch_dtype).to(dev) for _ in range(2)]
+    ys = [torch.empty_like(x) for x in xs]
+    nbytes = 2 * rows * D * xs[0].element_size()
+    out = {"rows": rows, "D": D, "dtype": w.dtype}
+    for name, deriv in (("value", False), ("slope", True)):
+        for i in range(4):
+            la.la_feature_map(xs[i & 1], deriv=deriv, out=ys[i & 1])
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(dev)
+        e0.record()
+        for i in range(iters):
+            la.la_feature_map(xs[i & 1], deriv=deriv, out=ys[i & 1])
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1) / iters
+        out[name] = {"ms": round(ms, 4), "alg_gbs": round(nbytes / ms / 1e6, 1),
+                     "hbm_frac": round(nbytes / ms / 1e6 / pk["hbm_gbs"], 3)}
+    return out
+
+
 def bench_rff(la, w, dev, pk, iters=10):
     """Random Fourier features (the map the paper's conclusion proposes) and their gradient on the headline
     workload's rows with D = 64 inputs and C = 64 features (what the tensor-core attention kernels take): two
@@ -793,6 +818,7 @@ def main():
         rows[w.name + "_from_state"] = {kk: r[kk] for kk in ("value", "ms_per_step", "fwd_ms", "bwd_ms", "alg_gbs", "hbm_frac",
                                                               "gpu_launches", "kernels_ms")}
         rows[w.name + "_from_state"]["unit"] = "tokens/s"
+        rows["feature_map_elu1"] = bench_feature_map(la, w, dev, pk)
         rows["feature_map_poly2"] = bench_poly2(la, w, dev, pk)
         rows["feature_map_rff"] = bench_rff(la, w, dev, pk)
         rows[w.name + "_ragged"] = bench_ragged(la, w, dev, pk)
