@@ -391,6 +391,12 @@ __device__ __forceinline__ uint32_t min_bf16x2(uint32_t a, uint32_t b) {
     return r;
 }
 
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
 // Byte offset of element (row, col) of a [rows][64] bf16 tile in the swizzled layout.
 __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t col) {
     return row * 128u + ((((col >> 3) ^ (row & 7u)) << 4) | ((col & 7u) << 1));

@@ -446,21 +446,22 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             tmem_ld32(tmem + lane_base + kDqColT + b * 64 + half * 32, tt);
             tmem_ld_wait();
             tc_fence_before_sync();
-            const float m = m_prev;
-            float qg4[4] = {0.f, 0.f, 0.f, 0.f}, qz4[4] = {0.f, 0.f, 0.f, 0.f};
+            // (two columns per instruction from here on: the kernel is bound by instruction issue, and this
+            // epilogue is a fifth of a chunk's instructions)
+            const f32x2 m2 = pair(m_prev, m_prev);
+            f32x2 h2[16], z2[16];
+            f32x2 qg2[4] = {0, 0, 0, 0}, qz2[4] = {0, 0, 0, 0};
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const int e = cc * 8 + 2 * j;
-                    const float q0 = bf16_lo(qv[cc][j]), q1 = bf16_hi(qv[cc][j]);
-                    const float t0 = __uint_as_float(tt[e]), t1 = __uint_as_float(tt[e + 1]);
-                    const float h0 = fmaf(m, t0, __uint_as_float(g[e])), h1 = fmaf(m, t1, __uint_as_float(g[e + 1]));
-                    const float z0 = zprev[e] + t0, z1 = zprev[e + 1] + t1;
-                    g[e] = __float_as_uint(h0); g[e + 1] = __float_as_uint(h1);
-                    tt[e] = __float_as_uint(z0); tt[e + 1] = __float_as_uint(z1);
-                    qg4[j] = fmaf(q0, h0, fmaf(q1, h1, qg4[j]));
-                    qz4[j] = fmaf(q0, z0, fmaf(q1, z1, qz4[j]));
+                    const int e = cc * 8 + 2 * j, p2 = cc * 4 + j;
+                    const f32x2 q2 = pair_bf16(qv[cc][j]);
+                    const f32x2 t2 = pair(tt[e], tt[e + 1]);
+                    h2[p2] = fma2(m2, t2, pair(g[e], g[e + 1]));
+                    z2[p2] = add2(pair_ld(zprev + e), t2);
+                    qg2[j] = fma2(q2, h2[p2], qg2[j]);
+                    qz2[j] = fma2(q2, z2[p2], qz2[j]);
                 }
             // both accumulators are in registers and Z_{c-1} has been consumed: the MMA warp may reuse
             // this accumulator pair, and the state warps the Z buffer (only after this arrival)
@@ -469,8 +470,8 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             // the quadrant's previous dQ slab must have left the staging tile before it is rewritten below
             if (half == 0 && lane == 0) tma_store_wait_read<0>();
             float* xch = sX + (half * 128 + t) * 2;
-            xch[0] = (qg4[0] + qg4[1]) + (qg4[2] + qg4[3]);
-            xch[1] = (qz4[0] + qz4[1]) + (qz4[2] + qz4[3]);
+            xch[0] = pair_sum(add2(add2(qg2[0], qg2[1]), add2(qg2[2], qg2[3])));
+            xch[1] = pair_sum(add2(add2(qz2[0], qz2[1]), add2(qz2[2], qz2[3])));
             named_barrier(2 + quad, 64);
             const float* other = sX + ((half ^ 1) * 128 + t) * 2;
             const float qg = xch[0] + other[0], qz = xch[1] + other[1];
@@ -488,20 +489,17 @@ causal_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             // of its threads stores it with TMA: full 128-byte rows per request instead of 32 rows per store
             // instruction.  Columns beyond a 32-wide problem are padding: the store clips them.
             uint8_t* out_row = smem + kDqOffOut + t * 128;
+            const f32x2 inv2 = pair(inv, inv), delta2 = pair(delta, delta);
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
                 uint32_t outp[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const int e = cc * 8 + 2 * j;
-                    float g0 = inv * fmaf(delta, __uint_as_float(tt[e]), __uint_as_float(g[e]));
-                    float g1 = inv * fmaf(delta, __uint_as_float(tt[e + 1]), __uint_as_float(g[e + 1]));
-                    if (elu) {          // phi'(x) from phi(x): 1 where x > 0 (phi > 1), else phi(x)
-                        const float q0 = bf16_lo(qv[cc][j]), q1 = bf16_hi(qv[cc][j]);
-                        g0 *= q0 > 1.f ? 1.f : q0;
-                        g1 *= q1 > 1.f ? 1.f : q1;
-                    }
-                    outp[j] = pad ? 0u : pack_bf16x2(g0, g1);
+                    const int p2 = cc * 4 + j;
+                    f32x2 gq = mul2(inv2, fma2(delta2, z2[p2], h2[p2]));
+                    // phi'(x) from phi(x): 1 where x > 0 (phi > 1), else phi(x), i.e. min(phi, 1)
+                    if (elu) gq = mul2(gq, pair_bf16(min_bf16x2(qv[cc][j], 0x3F803F80u)));
+                    outp[j] = pad ? 0u : pack_bf16x2(gq);
                 }
                 sts128(out_row + (((half * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
             }
@@ -848,7 +846,7 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
         const uint32_t r7 = t & 7;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const float* rec = prm.init ? prm.init + bh * (int64_t)plan.nparts() * kStateFloats : nullptr;
-        const float slope_floor = prm.phi == LA_PHI_ELU1 ? 0.f : 1.f;
+        const uint32_t floor2 = prm.phi == LA_PHI_ELU1 ? 0u : 0x3F803F80u;     // slope >= 0 (elu + 1) or = 1 (identity), as a bf16 pair
         rstate_init(tmem + kKvColR, quad, lane, smem + kKvOffR, sRv + 64, rec, rec ? plan.piece_first_part(piece + 1) : 0,
                    rec ? plan.nparts() : 0);
         if (prm.dS_out || prm.dZ_out)       // upstream gradient of the final state: every piece's reverse sum starts from it
@@ -934,12 +932,10 @@ causal_bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
                         const float4 rb = *reinterpret_cast<const float4*>(rprev + h * 32 + cc * 8 + 4);
                         const float rr[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float g0 = __uint_as_float(v[cc * 8 + 2 * j]) + rr[2 * j];
-                            const float g1 = __uint_as_float(v[cc * 8 + 2 * j + 1]) + rr[2 * j + 1];
-                            const float s0 = fmaxf(fminf(bf16_lo(kf[j]), 1.f), slope_floor);
-                            const float s1 = fmaxf(fminf(bf16_hi(kf[j]), 1.f), slope_floor);
-                            outp[j] = (kVarlen && i == 0 && t >= tail_rows) ? 0u : pack_bf16x2(g0 * s0, g1 * s1);
+                        for (int j = 0; j < 4; ++j) {       // two columns per instruction: issue-bound
+                            const f32x2 g2 = add2(pair(v[cc * 8 + 2 * j], v[cc * 8 + 2 * j + 1]), pair(rr[2 * j], rr[2 * j + 1]));
+                            const uint32_t slope = max_bf16x2(min_bf16x2(kf[j], 0x3F803F80u), floor2);
+                            outp[j] = (kVarlen && i == 0 && t >= tail_rows) ? 0u : pack_bf16x2(mul2(g2, pair_bf16(slope)));
                         }
                         sts128(const_cast<uint8_t*>(rowK) + (((h * 4 + cc) ^ r7) << 4), outp[0], outp[1], outp[2], outp[3]);
                     }

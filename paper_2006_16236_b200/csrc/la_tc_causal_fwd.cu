@@ -443,6 +443,7 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             tc_fence_before_sync();
             mbar_arrive(&bars->o_drained[b]);
             const float inv = 1.f / (den + prm.eps);
+            const f32x2 inv2 = pair(inv, inv);
             const int64_t row = row0 + (int64_t)c * kChunk + t;
             if (kVarlen && c == L - 1 && t >= tail_rows) {  // a padded row of the chunk that holds the sequence's end
                 if ((int64_t)(c_begin + c) * kChunk + t >= prm.N) return true;      // past the sequence: not in memory
@@ -458,12 +459,12 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             if (half * 32 < prm.dim) {                      // columns beyond a 32-wide problem are padding
                 __nv_bfloat16* dst = prm.O + row * prm.dim + half * 32;
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
+                for (int cc = 0; cc < 4; ++cc)              // two columns per multiply
                     stg128(dst + cc * 8,
-                           pack_bf16x2(__uint_as_float(v[cc * 8 + 0]) * inv, __uint_as_float(v[cc * 8 + 1]) * inv),
-                           pack_bf16x2(__uint_as_float(v[cc * 8 + 2]) * inv, __uint_as_float(v[cc * 8 + 3]) * inv),
-                           pack_bf16x2(__uint_as_float(v[cc * 8 + 4]) * inv, __uint_as_float(v[cc * 8 + 5]) * inv),
-                           pack_bf16x2(__uint_as_float(v[cc * 8 + 6]) * inv, __uint_as_float(v[cc * 8 + 7]) * inv));
+                           pack_bf16x2(mul2(pair(v[cc * 8 + 0], v[cc * 8 + 1]), inv2)),
+                           pack_bf16x2(mul2(pair(v[cc * 8 + 2], v[cc * 8 + 3]), inv2)),
+                           pack_bf16x2(mul2(pair(v[cc * 8 + 4], v[cc * 8 + 5]), inv2)),
+                           pack_bf16x2(mul2(pair(v[cc * 8 + 6], v[cc * 8 + 7]), inv2)));
             }
             if (tid == 0) LA_TRACE(g_trace_fwd, c, 10);
             return true;

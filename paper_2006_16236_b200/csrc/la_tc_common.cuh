@@ -274,6 +274,8 @@ __device__ __forceinline__ void map_row_inplace(uint8_t* row, uint32_t r7, float
             for (int j = 0; j < 4; ++j) {
                 if (kElu && !kScale) {
                     v[i][j] = phi_pair(v[i][j]);
+                } else if (!kElu && kScale) {           // one multiply for the pair
+                    v[i][j] = sm100::pack_bf16x2(sm100::mul2(sm100::pair_bf16(v[i][j]), sm100::pair(scale, scale)));
                 } else {
                     const float x0 = sm100::bf16_lo(v[i][j]), x1 = sm100::bf16_hi(v[i][j]);
                     const float y0 = kElu ? phi_fast(x0) : x0, y1 = kElu ? phi_fast(x1) : x1;
@@ -355,9 +357,11 @@ __device__ __forceinline__ void stg128(void* p, uint32_t a, uint32_t b, uint32_t
 __device__ __forceinline__ void score_block_store(const uint32_t (&v)[32], uint8_t* tile_row, uint32_t r7, int blk,
                                                   bool diagonal, int lane, float add) {
     uint32_t packed[16];
+    const sm100::f32x2 add2 = sm100::pair(add, add);
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        float x0 = __uint_as_float(v[2 * j]) + add, x1 = __uint_as_float(v[2 * j + 1]) + add;
+        float x0, x1;
+        sm100::unpair(sm100::add2(sm100::pair(v[2 * j], v[2 * j + 1]), add2), x0, x1);      // one add for two columns
         if (diagonal) {
             if (2 * j > lane) x0 = 0.f;
             if (2 * j + 1 > lane) x1 = 0.f;
