@@ -419,11 +419,11 @@ causal_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             uint32_t v[32], pk[16];
             if (hasA) tmem_ld32(pb + blkA * 32, v);
             tmem_ld_wait();
-            score_block_pack(v, hasA, blkA == quad, lane, pk);
+            score_block_round<false>(v, hasA, blkA == quad, lane, pk);
             if (hasB) tmem_ld32(pb + blkB * 32, v);
             tmem_st16(pb + half * 64, pk);
             tmem_ld_wait();
-            score_block_pack(v, hasB, blkB == quad, lane, pk);
+            score_block_round<false>(v, hasB, blkB == quad, lane, pk);
             tmem_st16(pb + half * 64 + 16, pk);
             tmem_st_wait();
             tc_fence_before_sync();

@@ -658,21 +658,7 @@ static __device__ __noinline__ void rstate_write(uint32_t tmem_state, int quad, 
 
 // One 32-column block of fp32 scores -> 16 packed bf16 pairs (pair j = columns 2j, 2j+1), with
 // the causal mask on the diagonal block; a block above the diagonal (`present` false) is zeros.
-__device__ __forceinline__ void score_block_pack(const uint32_t (&v)[32], bool present, bool diagonal, int lane,
-                                                 uint32_t (&packed)[16]) {
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        float x0 = __uint_as_float(v[2 * j]), x1 = __uint_as_float(v[2 * j + 1]);
-        if (diagonal) {
-            if (2 * j > lane) x0 = 0.f;
-            if (2 * j + 1 > lane) x1 = 0.f;
-        }
-        packed[j] = present ? sm100::pack_bf16x2(x0, x1) : 0u;
-    }
-}
-
-
-// The same with one warp-uniform branch per block instead of per-element selects: a block off the
+// One warp-uniform branch per block instead of per-element selects: a block off the
 // diagonal costs sixteen conversions, an absent block none.  (The score warps of the quadrant with
 // four present blocks set the pace of a chunk, and most of their blocks are off the diagonal.)
 template <bool kTransposed>
