@@ -358,15 +358,18 @@ __device__ __forceinline__ void score_block_store(const uint32_t (&v)[32], uint8
                                                   bool diagonal, int lane, float add) {
     uint32_t packed[16];
     const sm100::f32x2 add2 = sm100::pair(add, add);
+    if (!diagonal) {            // (one warp-uniform branch per block instead of a select per element)
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        float x0, x1;
-        sm100::unpair(sm100::add2(sm100::pair(v[2 * j], v[2 * j + 1]), add2), x0, x1);      // one add for two columns
-        if (diagonal) {
+        for (int j = 0; j < 16; ++j) packed[j] = sm100::pack_bf16x2(sm100::add2(sm100::pair(v[2 * j], v[2 * j + 1]), add2));
+    } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            float x0, x1;
+            sm100::unpair(sm100::add2(sm100::pair(v[2 * j], v[2 * j + 1]), add2), x0, x1);      // one add for two columns
             if (2 * j > lane) x0 = 0.f;
             if (2 * j + 1 > lane) x1 = 0.f;
+            packed[j] = sm100::pack_bf16x2(x0, x1);
         }
-        packed[j] = sm100::pack_bf16x2(x0, x1);
     }
     uint8_t* base = tile_row + (blk >> 1) * kTileBytes;
 #pragma unroll
