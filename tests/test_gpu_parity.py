@@ -237,7 +237,7 @@ def test_prefill_then_decode_handoff():
 
 @pytest.mark.parametrize("dtype", DTYPES)
 @pytest.mark.parametrize("shape", [(2, 3, 100, 16, 48), (1, 2, 31, 64, 64), (2, 2, 640, 32, 32), (1, 4, 384, 64, 64),
-                                   (4, 16, 18 * 128, 64, 64)])
+                                   (4, 16, 18 * 128, 64, 64), (2, 8, 1000, 64, 64)])
 def test_causal_forward_from_a_state(shape, dtype):
     """The recurrence of Eq. 16-20 started from a given S_0, Z_0 (general kernels and, for bf16 D = M in
     {32, 64}, the tensor-core kernel, with several pieces per sequence at the larger shapes)."""
@@ -289,7 +289,8 @@ def test_chunked_prefill_then_decode(dtype, D, chunks):
 
 @pytest.mark.parametrize("dtype", DTYPES)
 @pytest.mark.parametrize("keep", [False, True], ids=["recompute", "saved"])
-@pytest.mark.parametrize("shape", [(2, 3, 100, 16, 48), (1, 2, 31, 64, 64), (2, 2, 640, 32, 32), (4, 16, 18 * 128, 64, 64)])
+@pytest.mark.parametrize("shape", [(2, 3, 100, 16, 48), (1, 2, 31, 64, 64), (2, 2, 640, 32, 32), (4, 16, 18 * 128, 64, 64),
+                                   (2, 8, 1000, 64, 64)])
 def test_causal_backward_from_a_state(shape, keep, dtype):
     """Algorithm 1 (backward) with the forward sum started from [S_0 | Z_0] and the reverse sum from an upstream
     gradient of the final state; the gradient of the initial state is what the reverse sum ends with."""
