@@ -592,8 +592,8 @@ def bench_poly2(la, w, dev, pk, iters=10):
 
 def bench_ragged(la, w, dev, pk, iters=10):
     """The headline shape as a right-padded ragged batch (lengths uniform in [N/2, N], the mix of a speech batch):
-    forward + backward through the calls that take `lengths`, against the same tensors processed at full length.
-    No saved buffer on either side (the ragged calls do not take one)."""
+    forward + backward through the calls that take `lengths`, against the same tensors processed at full length,
+    both with the saved buffer."""
     Q, K, V, G = (t.to(dev) for t in draw_qkvg(w.B, w.H, w.N, w.D, w.M, w.seed, w.torch_dtype, w.scale))
     g = torch.Generator(device="cpu").manual_seed(w.seed + 23)
     lengths = torch.randint(w.N // 2, w.N + 1, (w.B,), generator=g, dtype=torch.int32)
@@ -601,13 +601,15 @@ def bench_ragged(la, w, dev, pk, iters=10):
     O, den = torch.empty_like(V), torch.empty((w.B, w.H, w.N), device=dev)
     dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
 
+    saved = la.saved_buffer(Q, V)
+
     def ragged():
-        la.la_causal_forward(Q, K, V, lengths=ln, O=O, den=den)
-        la.la_causal_backward(Q, K, V, G, lengths=ln, dQ=dQ, dK=dK, dV=dV)
+        la.la_causal_forward(Q, K, V, lengths=ln, O=O, den=den, saved=saved)
+        la.la_causal_backward(Q, K, V, G, lengths=ln, dQ=dQ, dK=dK, dV=dV, saved=saved)
 
     def full():
-        la.la_causal_forward(Q, K, V, O=O, den=den)
-        la.la_causal_backward(Q, K, V, G, dQ=dQ, dK=dK, dV=dV)
+        la.la_causal_forward(Q, K, V, O=O, den=den, saved=saved)
+        la.la_causal_backward(Q, K, V, G, dQ=dQ, dK=dK, dV=dV, saved=saved)
 
     out = {"lengths": lengths.tolist(), "real_fraction": round(float(lengths.sum()) / (w.B * w.N), 3)}
     for name, fn in (("ragged_ms", ragged), ("full_length_ms", full)):

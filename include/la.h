@@ -418,23 +418,27 @@ int la_causal_backward_from(const la_problem* p, const void* Q, const void* K, c
  * (both or neither) as for la_causal_forward_from().  ws: la_workspace_bytes(p, LA_OP_CAUSAL_VARLEN_FORWARD).
  * Causality alone already keeps right padding out of every real position's output; what this call adds is
  * the state at the true end, zeros instead of garbage on the padding, indifference to non-finite padding,
- * and no time spent on it.
+ * and no time spent on it.  saved / saved_bytes: as for la_causal_forward() (optional; what is kept covers the
+ * real positions only, and the backward call must be given the same lengths).
  */
 int la_causal_forward_varlen(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
                              const float* S_in, const float* Z_in,
                              void* O, float* den, float* S_out, float* Z_out,
+                             void* saved, size_t saved_bytes,
                              void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Gradients of la_causal_forward_varlen() (Eq. 13-15 per sequence on its own length): dQ, dK, dV are zero on
  * the padding, and G is not read there.  The state arguments are those of la_causal_backward_from(): dS_out /
  * dZ_out is the upstream gradient of the state at each sequence's own end, dS_in / dZ_in receive the gradient
- * of the state it started from.  ws: la_workspace_bytes(p, LA_OP_CAUSAL_VARLEN_BACKWARD).
+ * of the state it started from.  saved / saved_bytes: the buffer la_causal_forward_varlen() filled for the same
+ * problem and lengths, or NULL / 0.  ws: la_workspace_bytes(p, LA_OP_CAUSAL_VARLEN_BACKWARD).
  */
 int la_causal_backward_varlen(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
                               const float* S_in, const float* Z_in,
                               const void* O, const float* den, const void* G,
                               const float* dS_out, const float* dZ_out,
+                              const void* saved, size_t saved_bytes,
                               void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
                               void* ws, size_t ws_bytes, void* stream);
 

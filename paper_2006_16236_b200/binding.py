@@ -79,8 +79,8 @@ def lib() -> ctypes.CDLL:
         L.la_causal_forward_from.argtypes = [pp] + [vp] * 9 + [vp, sz] + [vp, sz, vp]
         L.la_causal_backward_from.argtypes = [pp] + [vp] * 10 + [vp, sz] + [vp] * 5 + [vp, sz, vp]
         L.la_causal_backward.argtypes = [pp] + [vp] * 6 + [vp, sz] + [vp] * 3 + [vp, sz, vp]
-        L.la_causal_forward_varlen.argtypes = [pp] + [vp] * 10 + [vp, sz, vp]
-        L.la_causal_backward_varlen.argtypes = [pp] + [vp] * 16 + [vp, sz, vp]
+        L.la_causal_forward_varlen.argtypes = [pp] + [vp] * 10 + [vp, sz, vp, sz, vp]
+        L.la_causal_backward_varlen.argtypes = [pp] + [vp] * 11 + [vp, sz] + [vp] * 5 + [vp, sz, vp]
         L.la_recurrent_step.argtypes = [pp] + [vp] * 6 + [vp]
         L.la_recurrent_steps.argtypes = [pp] + [vp] * 6 + [vp]
         L.la_decode_layer_step.argtypes = [pp] + [vp] * 6 + [vp, sz, vp]
@@ -440,14 +440,13 @@ def la_causal_forward(Q, K, V, phi="elu1", eps=0.0, O=None, den=None, S_out=None
     _buffer("saved", saved), _buffer("ws", ws)
     if lengths is not None:
         _lengths_arg(lengths, p.B, None)
-        if saved is not None:
-            raise ValueError("a ragged batch (lengths) keeps nothing for the backward pass: do not pass `saved`")
     dev = _dev(Q, K, V, O, den, S_out, Z_out, saved, S_in, Z_in, ws, lengths)
     O = torch.empty_like(V) if O is None else O
     if lengths is not None:             # la_causal_forward_varlen: right-padded ragged batch
         ws = workspace(p, LA_OP_CAUSAL_VARLEN_FORWARD, dev) if ws is None else ws
         _call(dev, lib().la_causal_forward_varlen, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(S_in),
-              _ptr(Z_in), _ptr(O), _ptr(den), _ptr(S_out), _ptr(Z_out), _ptr(ws), _nbytes(ws), _stream(dev))
+              _ptr(Z_in), _ptr(O), _ptr(den), _ptr(S_out), _ptr(Z_out), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws),
+              _stream(dev))
         return O
     ws = workspace(p, LA_OP_CAUSAL_FORWARD, dev) if ws is None else ws
     if S_in is None and Z_in is None:
@@ -472,8 +471,6 @@ def la_causal_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None, saved=
     _buffer("saved", saved), _buffer("ws", ws)
     if lengths is not None:
         _lengths_arg(lengths, p.B, None)
-        if saved is not None:
-            raise ValueError("a ragged batch (lengths) keeps nothing for the backward pass: do not pass `saved`")
     dev = _dev(Q, K, V, G, O, den, dQ, dK, dV, saved, S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in, ws, lengths)
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
@@ -481,8 +478,8 @@ def la_causal_backward(Q, K, V, G, phi="elu1", eps=0.0, O=None, den=None, saved=
     if lengths is not None:             # la_causal_backward_varlen
         ws = workspace(p, LA_OP_CAUSAL_VARLEN_BACKWARD, dev) if ws is None else ws
         _call(dev, lib().la_causal_backward_varlen, ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(lengths), _ptr(S_in),
-              _ptr(Z_in), _ptr(O), _ptr(den), _ptr(G), _ptr(dS_out), _ptr(dZ_out), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dS_in),
-              _ptr(dZ_in), _ptr(ws), _nbytes(ws), _stream(dev))
+              _ptr(Z_in), _ptr(O), _ptr(den), _ptr(G), _ptr(dS_out), _ptr(dZ_out), _ptr(saved), _nbytes(saved), _ptr(dQ), _ptr(dK),
+              _ptr(dV), _ptr(dS_in), _ptr(dZ_in), _ptr(ws), _nbytes(ws), _stream(dev))
         return dQ, dK, dV
     ws = workspace(p, LA_OP_CAUSAL_BACKWARD, dev) if ws is None else ws
     state = (S_in, Z_in, dS_out, dZ_out, dS_in, dZ_in)

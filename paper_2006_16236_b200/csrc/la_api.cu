@@ -506,8 +506,9 @@ int la_causal_forward_from(const la_problem* p, const void* Q, const void* K, co
 int la_causal_forward_varlen(const la_problem* p, const void* Q, const void* K, const void* V, const int32_t* lengths,
                              const float* S_in, const float* Z_in,
                              void* O, float* den, float* S_out, float* Z_out,
+                             void* saved, size_t saved_bytes,
                              void* ws, size_t ws_bytes, void* stream) {
-    return causal_forward_common(p, Q, K, V, lengths, true, S_in, Z_in, O, den, S_out, Z_out, nullptr, 0, ws, ws_bytes, stream);
+    return causal_forward_common(p, Q, K, V, lengths, true, S_in, Z_in, O, den, S_out, Z_out, saved, saved_bytes, ws, ws_bytes, stream);
 }
 
 int la_causal_forward(const la_problem* p, const void* Q, const void* K, const void* V,
@@ -584,9 +585,10 @@ int la_causal_backward_varlen(const la_problem* p, const void* Q, const void* K,
                               const float* S_in, const float* Z_in,
                               const void* O, const float* den, const void* G,
                               const float* dS_out, const float* dZ_out,
+                              const void* saved, size_t saved_bytes,
                               void* dQ, void* dK, void* dV, float* dS_in, float* dZ_in,
                               void* ws, size_t ws_bytes, void* stream) {
-    return causal_backward_common(p, Q, K, V, lengths, true, S_in, Z_in, O, den, G, dS_out, dZ_out, nullptr, 0,
+    return causal_backward_common(p, Q, K, V, lengths, true, S_in, Z_in, O, den, G, dS_out, dZ_out, saved, saved_bytes,
                                   dQ, dK, dV, dS_in, dZ_in, ws, ws_bytes, stream);
 }
 

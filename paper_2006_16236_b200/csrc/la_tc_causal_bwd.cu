@@ -1006,7 +1006,6 @@ size_t causal_backward_workspace(const la_problem& p) {
 
 int causal_backward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const void* G,
                     const StateArgs& sa, const void* saved, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
-    if (lengths) saved = nullptr;       // a ragged batch keeps nothing from the forward pass
     const CausalPlan pl = choose_plan(p);
     // With what the forward saved, phi(Q) and phi(K) are read as tensors (no feature map on load)
     // and the forward pre-pass records are the forward's own.

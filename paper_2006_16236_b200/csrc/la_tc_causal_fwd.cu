@@ -563,7 +563,6 @@ size_t causal_saved_bytes(const la_problem& p) { return saved_layout(p, choose_p
 int causal_forward(const la_problem& p, const void* Q, const void* K, const void* V, const int* lengths, const float* S_in,
                    const float* Z_in, void* O, float* den, float* S_out, float* Z_out, void* saved, void* ws,
                    cudaStream_t st) {
-    if (lengths) saved = nullptr;       // a ragged batch keeps nothing for the backward pass
     const CausalPlan pl = choose_plan(p);
     const uint64_t seqs = (uint64_t)(p.B * p.H), n = (uint64_t)p.N;
     const bool ragged = ragged_problem(p, lengths);

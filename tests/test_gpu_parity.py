@@ -856,6 +856,18 @@ def test_causal_ragged_batches(shape, lengths, dtype):
     O = la.la_causal_forward(Qd, Kd, Vd, lengths=ln, den=den, S_out=S, Z_out=Z)
     dQ, dK, dV = la.la_causal_backward(Qd, Kd, Vd, Gd, lengths=ln)
     la.la_last_device_status()
+    # the same with a saved buffer (poisoned beforehand: what lies behind a sequence's end in it is never read):
+    # the forward's result does not depend on it, dQ is bit-identical, dK and dV agree to rounding
+    saved = la.saved_buffer(Qd, Vd)
+    if saved is not None:
+        saved.fill_(0xFF)
+        O2 = la.la_causal_forward(Qd, Kd, Vd, lengths=ln, saved=saved)
+        g2 = la.la_causal_backward(Qd, Kd, Vd, Gd, lengths=ln, saved=saved)
+        la.la_last_device_status()
+        assert torch.equal(O2, O) and torch.equal(g2[0], dQ)
+        for a, b2, nm in zip((dK, dV), g2[1:], "KV"):
+            assert torch.all(b2.isfinite()), f"d{nm} with the saved buffer"
+            assert_close(b2, a.double().cpu().numpy(), dtype, f"d{nm} saved vs recomputed", grad=True)
     # one decode step per stream from the state the ragged prefill handed back
     q1, k1, v1 = (t[:, :, 0].contiguous() for t in gpu(*nxt))
     out1 = la.la_recurrent_step(q1, k1, v1, S.clone(), Z.clone())
