@@ -1,4 +1,6 @@
 """GPU parity: the CUDA library (through its C ABI) against the fp64 oracle, element by element."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -125,6 +127,8 @@ def test_causal_results_do_not_depend_on_the_piece_plan(plan_override, plan, kee
 def test_backward_refuses_a_saved_buffer_of_another_plan(plan_override):
     """The saved buffer carries the plan of the forward pass that filled it.  A backward pass under another
     plan would look for the pre-pass records at other offsets: it reports the mismatch and computes nothing."""
+    if os.environ.get("LA_DEBUG"):
+        pytest.skip("in checked mode the call itself reads the status and raises; this test reads it afterwards")
     B, H, N, D = 4, 16, 18 * 128, 64
     Q, K, V, G = draw_qkvg(B, H, N, D, D, seed=78, dtype=torch.bfloat16)
     Qd, Kd, Vd, Gd = gpu(Q, K, V, G)
